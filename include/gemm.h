@@ -1,0 +1,177 @@
+/*
+ * b200 GEMM -- C ABI of the dense matrix-multiply hot path for NVIDIA B200 (sm_100a).
+ *
+ *     D = act( alpha * op(A) * op(B) + beta * C + bias )
+ *
+ * This is the GEMM kernel family of the paper's case study (Section 5.4; the
+ * strategy census of Table 1: tensor cores, tiling, vectorised and asynchronous
+ * copies, swizzled layouts, multi-stage pipelines, thread-block swizzle),
+ * re-designed for Blackwell: TMA-fed mbarrier pipelines, tcgen05.mma with the
+ * accumulator in tensor memory, optional 2-CTA tiles, a persistent swizzled tile
+ * scheduler, a TMEM -> shared -> TMA-store epilogue and a stream-K path for
+ * skinny memory-bound shapes.  Plan-time selection of the path follows the
+ * roofline classification of Section 4.3 (memory-bound / compute-bound by
+ * arithmetic intensity against the machine ridge).
+ *
+ * Conventions
+ *   Storage is ROW-MAJOR.  transa = GEMM_OP_N: A is stored M x K (lda >= K);
+ *   GEMM_OP_T: A is stored K x M (lda >= M).  transb = GEMM_OP_N: B is stored
+ *   K x N (ldb >= N); GEMM_OP_T: B is stored N x K (ldb >= K), i.e. "B
+ *   column-major" / an nn.Linear weight.  C and D share one buffer: M x N,
+ *   ldc >= N, read only when beta != 0 and then overwritten.  A and B have one
+ *   16-bit dtype (bf16 or fp16); products are accumulated in fp32; C/D is fp32,
+ *   bf16 or fp16 (round to nearest even, no saturation).  bias is fp32[N], added
+ *   per output column and not scaled by alpha.  With batch_count > 1, matrix b
+ *   starts b * stride_{a,b,c} elements into its buffer.
+ *
+ * Pointers named "device" must be device memory of the current CUDA device;
+ * the caller owns every buffer (A, B, C, bias, workspace) and keeps it alive
+ * until the stream work has completed.  The library owns the plan object and a
+ * small device status word per plan.  No call synchronises the device except
+ * gemm_plan_status().  Nothing throws; every failure is a gemm_status_t, and an
+ * argument error launches nothing.
+ */
+#ifndef B200_GEMM_H_
+#define B200_GEMM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct gemm_plan_s* gemm_plan_t; /* opaque, host memory */
+typedef void* gemm_stream_t;             /* a cudaStream_t (NULL = default stream) */
+
+typedef enum {
+  GEMM_OK = 0,
+  GEMM_ERR_NULL = 1,        /* a required pointer is NULL */
+  GEMM_ERR_INVALID_ARG = 2, /* bad extent, leading dimension, enum value or struct_size */
+  GEMM_ERR_UNSUPPORTED = 3, /* valid request the library does not implement */
+  GEMM_ERR_ALIGNMENT = 4,   /* pointer, leading dimension or stride not 16-byte aligned */
+  GEMM_ERR_WORKSPACE = 5,   /* workspace NULL or smaller than gemm_workspace_bytes() */
+  GEMM_ERR_ARCH = 6,        /* no CUDA device, or the device is not sm_100 */
+  GEMM_ERR_CUDA = 7,        /* a CUDA runtime / driver call failed */
+  GEMM_ERR_TIMEOUT = 8      /* a bounded device-side wait expired (see gemm_plan_status) */
+} gemm_status_t;
+
+typedef enum { GEMM_BF16 = 0, GEMM_F16 = 1, GEMM_F32 = 2 } gemm_dtype_t;
+typedef enum { GEMM_OP_N = 0, GEMM_OP_T = 1 } gemm_op_t;
+typedef enum {
+  GEMM_EPI_NONE = 0,
+  GEMM_EPI_BIAS = 1,
+  GEMM_EPI_RELU = 2,
+  GEMM_EPI_BIAS_RELU = 3,
+  GEMM_EPI_GELU_ERF = 4,     /* x * Phi(x) with the exact error function */
+  GEMM_EPI_BIAS_GELU_ERF = 5
+} gemm_epilogue_t;
+
+/* Roofline class of a problem (Section 4.3 of the paper, applied at plan time). */
+typedef enum { GEMM_REGIME_MEMORY = 0, GEMM_REGIME_MIDDLE = 1, GEMM_REGIME_COMPUTE = 2 } gemm_regime_t;
+/* Kernel family a plan selected. */
+typedef enum { GEMM_VARIANT_DENSE_1CTA = 1, GEMM_VARIANT_DENSE_2CTA = 2, GEMM_VARIANT_SKINNY_STREAMK = 3 } gemm_variant_t;
+
+/* gemm_desc_t.flags: 0 = let the plan decide everything. */
+#define GEMM_FLAG_VARIANT_SHIFT 4          /* bits 4-7: force a gemm_variant_t (0 = automatic) */
+#define GEMM_FLAG_VARIANT_MASK 0xF0u
+#define GEMM_FLAG_TILE_N_SHIFT 8           /* bits 8-15: force tile N / 16 (0 = automatic) */
+#define GEMM_FLAG_TILE_N_MASK 0xFF00u
+#define GEMM_FLAG_RASTER_SHIFT 16          /* bits 16-23: force the raster group height in tiles (0 = automatic) */
+#define GEMM_FLAG_RASTER_MASK 0xFF0000u
+#define GEMM_FLAG_STAGES_SHIFT 24          /* bits 24-27: force the pipeline depth (0 = automatic) */
+#define GEMM_FLAG_STAGES_MASK 0xF000000u
+#define GEMM_FLAG_DEBUG_STALL 0x80000000u  /* test hook: one producer arrival is withheld so that a bounded
+                                              wait expires and GEMM_ERR_TIMEOUT is reported */
+
+typedef struct {
+  uint32_t struct_size;  /* = sizeof(gemm_desc_t) */
+  uint32_t flags;        /* GEMM_FLAG_* */
+  int64_t M, N, K;       /* op(A) is M x K, op(B) is K x N, C/D is M x N; all >= 1 */
+  int32_t transa, transb;     /* gemm_op_t */
+  int32_t ab_dtype;           /* gemm_dtype_t: GEMM_BF16 or GEMM_F16, for both A and B */
+  int32_t c_dtype;            /* gemm_dtype_t of C/D */
+  int64_t lda, ldb, ldc;      /* leading dimensions in elements */
+  int32_t batch_count;        /* >= 1 */
+  int32_t epilogue;           /* gemm_epilogue_t */
+  int64_t stride_a, stride_b, stride_c; /* elements between consecutive matrices; ignored when batch_count == 1 */
+} gemm_desc_t;
+
+typedef struct {
+  uint32_t struct_size;  /* = sizeof(gemm_info_t), set by the caller */
+  int32_t variant;       /* gemm_variant_t */
+  int32_t regime;        /* gemm_regime_t */
+  int32_t tile_m, tile_n, tile_k; /* output tile of one CTA (1-CTA) or CTA pair (2-CTA); skinny: tile over N, M-pad, K */
+  int32_t stages;        /* depth of the shared-memory ring */
+  int32_t cluster_size;  /* 1 or 2 */
+  int32_t grid;          /* CTAs launched */
+  int32_t raster_group;  /* tile rows swept together by the scheduler */
+  int32_t split;         /* skinny: maximum number of CTAs contributing to one output tile; dense: 1 */
+  int32_t smem_bytes;    /* dynamic shared memory per CTA */
+  int64_t num_tiles;     /* output tiles (dense) or k-block work units (skinny) */
+  double flops;          /* 2 * M * N * K * batch */
+  double min_bytes;      /* compulsory HBM traffic */
+  double intensity;      /* flops / min_bytes */
+  size_t workspace_bytes;
+} gemm_info_t;
+
+/*
+ * gemm_plan -- validate `desc` (host pointer), classify the problem on the
+ * roofline (Section 4.3), choose the kernel variant, tile shape, pipeline depth,
+ * cluster size, raster order and stream-K split, and return a plan (host
+ * memory).  If a CUDA device is current, also allocates the plan's 16-byte
+ * device status word and reads the SM count; without a device the plan is still
+ * created (148 SMs assumed) so that planning can be inspected, and gemm_run
+ * reports GEMM_ERR_ARCH.  Errors: NULL -> GEMM_ERR_NULL; extents < 1, leading
+ * dimension smaller than the row length, unknown enum, wrong struct_size ->
+ * GEMM_ERR_INVALID_ARG; lda/ldb/ldc or batch strides whose byte size is not a
+ * multiple of 16 -> GEMM_ERR_ALIGNMENT; fp32 A/B or an impossible forced
+ * variant -> GEMM_ERR_UNSUPPORTED.
+ */
+gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan);
+
+/* Bytes of device workspace gemm_run needs for this plan (0 for the dense variants;
+ * stream-K partial tiles and arrival counters for the skinny variant).  0 on a NULL plan. */
+size_t gemm_workspace_bytes(gemm_plan_t plan);
+
+/*
+ * gemm_run -- enqueue D = act(alpha*op(A)*op(B) + beta*C + bias) on `stream`
+ * (asynchronous; the hot path of Section 5.4).  A, B, C: device pointers, 16-byte
+ * aligned, laid out as `desc` said.  bias: device fp32[N], required iff the
+ * epilogue has a bias.  C is read only when beta != 0.  workspace: device
+ * memory of at least gemm_workspace_bytes(plan) bytes, 16-byte aligned (may be NULL when
+ * that is 0); concurrent runs of one plan need distinct workspaces.  alpha and
+ * beta are host scalars.  Errors are returned before anything is launched:
+ * GEMM_ERR_NULL, GEMM_ERR_ALIGNMENT, GEMM_ERR_WORKSPACE, GEMM_ERR_ARCH,
+ * GEMM_ERR_CUDA (tensor-map encoding or launch failure).
+ */
+gemm_status_t gemm_run(gemm_plan_t plan, const void* A, const void* B, void* C, const float* bias, float alpha,
+                       float beta, void* workspace, size_t workspace_bytes, gemm_stream_t stream);
+
+/*
+ * gemm_plan_status -- synchronise the device and read the plan's status word:
+ * GEMM_OK, or GEMM_ERR_TIMEOUT if a bounded device-side wait of an earlier run
+ * expired (the kernel then returned early and its output is undefined).  The
+ * word is cleared by the read.
+ */
+gemm_status_t gemm_plan_status(gemm_plan_t plan);
+
+/* Override the device-side wait limit of this plan (default 2000 ms; minimum 1 ms). */
+gemm_status_t gemm_plan_set_timeout_ms(gemm_plan_t plan, uint32_t ms);
+
+/* Copy the plan's decisions into *out (out->struct_size must be sizeof(gemm_info_t)). */
+gemm_status_t gemm_plan_info(gemm_plan_t plan, gemm_info_t* out);
+
+/* Free the plan and its status word.  NULL is accepted. */
+gemm_status_t gemm_destroy(gemm_plan_t plan);
+
+/* Static string for a status code. */
+const char* gemm_status_string(gemm_status_t s);
+
+/* Detail of the last GEMM_ERR_CUDA on this thread (CUDA error name), or "". */
+const char* gemm_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* B200_GEMM_H_ */

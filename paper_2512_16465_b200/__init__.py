@@ -1,0 +1,209 @@
+"""Python binding of the b200 GEMM C-ABI library (``include/gemm.h``).
+
+Argument marshalling only: every step of ``D = act(alpha * op(A) @ op(B) + beta * C + bias)``
+runs in the CUDA kernels of ``libb200gemm.so``.  PyTorch is used for device memory and
+streams.  There is no CPU or library fallback: if the shared library cannot be loaded
+the import raises.
+
+Low-level calls mirror the C names: :func:`gemm_plan`, :func:`gemm_workspace_bytes`,
+:func:`gemm_run`, :func:`gemm_plan_status`, :func:`gemm_plan_info`, :func:`gemm_destroy`.
+:class:`Plan` wraps them for torch tensors.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+from . import build as _build
+
+BF16, F16, F32 = 0, 1, 2
+OP_N, OP_T = 0, 1
+EPI_NONE, EPI_BIAS, EPI_RELU, EPI_BIAS_RELU, EPI_GELU_ERF, EPI_BIAS_GELU_ERF = range(6)
+VARIANT_AUTO, VARIANT_DENSE_1CTA, VARIANT_DENSE_2CTA, VARIANT_SKINNY_STREAMK = 0, 1, 2, 3
+REGIME_NAMES = {0: "memory-bound", 1: "middle-zone", 2: "compute-bound"}
+FLAG_DEBUG_STALL = 0x80000000
+
+OK, ERR_NULL, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = range(9)
+
+
+class GemmError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        detail = _lib.gemm_last_cuda_error().decode() if status in (ERR_CUDA, ERR_TIMEOUT) else ""
+        super().__init__(f"{where}: {_lib.gemm_status_string(status).decode()}" + (f" ({detail})" if detail else ""))
+
+
+class Desc(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_uint32), ("flags", ctypes.c_uint32),
+                ("M", ctypes.c_int64), ("N", ctypes.c_int64), ("K", ctypes.c_int64),
+                ("transa", ctypes.c_int32), ("transb", ctypes.c_int32),
+                ("ab_dtype", ctypes.c_int32), ("c_dtype", ctypes.c_int32),
+                ("lda", ctypes.c_int64), ("ldb", ctypes.c_int64), ("ldc", ctypes.c_int64),
+                ("batch_count", ctypes.c_int32), ("epilogue", ctypes.c_int32),
+                ("stride_a", ctypes.c_int64), ("stride_b", ctypes.c_int64), ("stride_c", ctypes.c_int64)]
+
+
+class Info(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_uint32), ("variant", ctypes.c_int32), ("regime", ctypes.c_int32),
+                ("tile_m", ctypes.c_int32), ("tile_n", ctypes.c_int32), ("tile_k", ctypes.c_int32),
+                ("stages", ctypes.c_int32), ("cluster_size", ctypes.c_int32), ("grid", ctypes.c_int32),
+                ("raster_group", ctypes.c_int32), ("split", ctypes.c_int32), ("smem_bytes", ctypes.c_int32),
+                ("num_tiles", ctypes.c_int64), ("flops", ctypes.c_double), ("min_bytes", ctypes.c_double),
+                ("intensity", ctypes.c_double), ("workspace_bytes", ctypes.c_size_t)]
+
+    def as_dict(self) -> dict:
+        return {k: getattr(self, k) for k, _ in self._fields_ if k != "struct_size"}
+
+
+EXPORTS = ("gemm_plan", "gemm_workspace_bytes", "gemm_run", "gemm_plan_status", "gemm_plan_set_timeout_ms",
+           "gemm_plan_info", "gemm_destroy", "gemm_status_string", "gemm_last_cuda_error")
+
+
+def _load() -> ctypes.CDLL:
+    path = _build.LIB
+    if not os.path.exists(path):
+        path = _build.build()          # raises if nvcc is missing or compilation fails
+    L = ctypes.CDLL(path)
+    vp = ctypes.c_void_p
+    L.gemm_plan.restype = ctypes.c_int
+    L.gemm_plan.argtypes = [ctypes.POINTER(Desc), ctypes.POINTER(vp)]
+    L.gemm_workspace_bytes.restype = ctypes.c_size_t
+    L.gemm_workspace_bytes.argtypes = [vp]
+    L.gemm_run.restype = ctypes.c_int
+    L.gemm_run.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, ctypes.c_float, vp, ctypes.c_size_t, vp]
+    L.gemm_plan_status.restype = ctypes.c_int
+    L.gemm_plan_status.argtypes = [vp]
+    L.gemm_plan_set_timeout_ms.restype = ctypes.c_int
+    L.gemm_plan_set_timeout_ms.argtypes = [vp, ctypes.c_uint32]
+    L.gemm_plan_info.restype = ctypes.c_int
+    L.gemm_plan_info.argtypes = [vp, ctypes.POINTER(Info)]
+    L.gemm_destroy.restype = ctypes.c_int
+    L.gemm_destroy.argtypes = [vp]
+    L.gemm_status_string.restype = ctypes.c_char_p
+    L.gemm_status_string.argtypes = [ctypes.c_int]
+    L.gemm_last_cuda_error.restype = ctypes.c_char_p
+    L.gemm_last_cuda_error.argtypes = []
+    return L
+
+
+_lib = _load()
+LIB_PATH = _build.LIB
+
+
+def make_flags(variant: int = 0, tile_n: int = 0, raster: int = 0, stages: int = 0, debug_stall: bool = False) -> int:
+    """Pack the GEMM_FLAG_* fields of ``gemm_desc_t.flags`` (0 everywhere = automatic)."""
+    assert tile_n % 16 == 0
+    return ((variant & 0xF) << 4) | (((tile_n // 16) & 0xFF) << 8) | ((raster & 0xFF) << 16) | ((stages & 0xF) << 24) | \
+        (FLAG_DEBUG_STALL if debug_stall else 0)
+
+
+def make_desc(M, N, K, transa=OP_N, transb=OP_T, ab_dtype=BF16, c_dtype=F32, lda=0, ldb=0, ldc=0, batch=1,
+              stride_a=0, stride_b=0, stride_c=0, epilogue=EPI_NONE, flags=0) -> Desc:
+    """Build a ``gemm_desc_t``; zero leading dimensions / strides mean "tight"."""
+    lda = lda or (M if transa else K)
+    ldb = ldb or (K if transb else N)
+    ldc = ldc or N
+    stride_a = stride_a or (K if transa else M) * lda
+    stride_b = stride_b or (N if transb else K) * ldb
+    stride_c = stride_c or M * ldc
+    return Desc(ctypes.sizeof(Desc), flags, M, N, K, transa, transb, ab_dtype, c_dtype, lda, ldb, ldc, batch, epilogue,
+                stride_a, stride_b, stride_c)
+
+
+# ----------------------------------------------------------------------- C-named calls
+
+def gemm_plan(desc: Desc) -> int:
+    """``gemm_plan``: returns the opaque plan handle or raises :class:`GemmError`."""
+    h = ctypes.c_void_p()
+    st = _lib.gemm_plan(ctypes.byref(desc), ctypes.byref(h))
+    if st != OK:
+        raise GemmError(st, "gemm_plan")
+    return h.value
+
+
+def gemm_workspace_bytes(plan: int) -> int:
+    return int(_lib.gemm_workspace_bytes(plan))
+
+
+def gemm_run(plan: int, A: int, B: int, C: int, bias: int, alpha: float, beta: float, workspace: int,
+             workspace_bytes: int, stream: int) -> None:
+    """``gemm_run`` on raw device addresses (ints) and a raw ``cudaStream_t`` value."""
+    st = _lib.gemm_run(plan, A, B, C, bias or None, alpha, beta, workspace or None, workspace_bytes, stream or None)
+    if st != OK:
+        raise GemmError(st, "gemm_run")
+
+
+def gemm_plan_status(plan: int) -> int:
+    return int(_lib.gemm_plan_status(plan))
+
+
+def gemm_plan_info(plan: int) -> dict:
+    info = Info()
+    info.struct_size = ctypes.sizeof(Info)
+    st = _lib.gemm_plan_info(plan, ctypes.byref(info))
+    if st != OK:
+        raise GemmError(st, "gemm_plan_info")
+    return info.as_dict()
+
+
+def gemm_destroy(plan: int) -> None:
+    _lib.gemm_destroy(plan)
+
+
+def status_string(st: int) -> str:
+    return _lib.gemm_status_string(st).decode()
+
+
+# ----------------------------------------------------------------------- torch convenience
+
+def _torch_dtype_code(t) -> int:
+    import torch
+    return {torch.bfloat16: BF16, torch.float16: F16, torch.float32: F32}[t]
+
+
+class Plan:
+    """A planned GEMM bound to torch tensors.  ``run`` enqueues on the current torch stream."""
+
+    def __init__(self, desc: Desc):
+        self.desc = desc
+        self.handle = gemm_plan(desc)
+        self.info = gemm_plan_info(self.handle)
+        self.workspace_bytes = gemm_workspace_bytes(self.handle)
+        self._ws = None
+
+    def workspace(self, device=None):
+        import torch
+        if self._ws is None and self.workspace_bytes:
+            self._ws = torch.empty(self.workspace_bytes, dtype=torch.uint8, device=device or "cuda")
+        return self._ws
+
+    def run(self, A, B, C, bias=None, alpha: float = 1.0, beta: float = 0.0, workspace=None, stream: Optional[int] = None):
+        import torch
+        if not (A.is_cuda and B.is_cuda and C.is_cuda):
+            raise ValueError("A, B and C must be CUDA tensors")
+        if _torch_dtype_code(A.dtype) != self.desc.ab_dtype or _torch_dtype_code(B.dtype) != self.desc.ab_dtype or \
+                _torch_dtype_code(C.dtype) != self.desc.c_dtype:
+            raise ValueError("tensor dtypes do not match the plan")
+        ws = workspace if workspace is not None else self.workspace(A.device)
+        s = torch.cuda.current_stream(A.device).cuda_stream if stream is None else stream
+        gemm_run(self.handle, A.data_ptr(), B.data_ptr(), C.data_ptr(), 0 if bias is None else bias.data_ptr(),
+                 float(alpha), float(beta), 0 if ws is None else ws.data_ptr(), 0 if ws is None else ws.numel(), s)
+        return C
+
+    def status(self) -> int:
+        return gemm_plan_status(self.handle)
+
+    def set_timeout_ms(self, ms: int) -> None:
+        _lib.gemm_plan_set_timeout_ms(self.handle, ms)
+
+    def close(self):
+        if self.handle:
+            gemm_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,430 @@
+// Dense GEMM kernel for sm_100a: persistent, warp-specialised, TMA -> shared ring -> tcgen05.mma
+// (accumulator in tensor memory, double buffered) -> epilogue warps -> swizzled staging -> TMA store.
+//
+// Roles inside one CTA (64 + 128 * EPI_WG threads):
+//   warp 0, lane 0   TMA producer: fills the STAGES-deep ring of (A tile, B tile) k-blocks
+//   warp 1, lane 0   MMA issuer: 4 x tcgen05.mma (K = 16 each) per k-block, commits free the ring slot;
+//                    warp 1 also owns the tensor-memory allocation
+//   warps 2..        epilogue: tcgen05.ld 32 lanes x 32 columns, alpha/beta/bias/activation in fp32,
+//                    convert, write a 32-row x 128-byte swizzled slab, one TMA store per slab per warp
+//
+// CG = 2 runs the same code on a cluster of two CTAs that share one 256 x BN tile: each CTA loads
+// its own 128 rows of A and its half of the B tile, the leader CTA (cluster rank 0) issues
+// tcgen05.mma.cta_group::2 for both, and each CTA drains its own 128 accumulator rows.
+//
+// Everything about the problem (tile N, stage count, operand major-ness, dtypes, epilogue) is a
+// run-time field of DenseParams; the only compile-time choices are CG and EPI_WG.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include "ptx.cuh"
+
+namespace b200 {
+
+constexpr int kBlockK = 64;         // K elements per ring stage = one 128-byte swizzle row of 16-bit data
+constexpr int kUmmaK = 16;          // K of one tcgen05.mma for 16-bit inputs
+constexpr int kCtaM = 128;          // accumulator rows per CTA = TMEM lanes
+constexpr int kMaxStages = 12;
+constexpr int kSlabBytes = 32 * 128;  // epilogue staging slab of one warp: 32 rows x 128 bytes
+
+// device status word values (also used by the skinny kernel)
+constexpr uint32_t kStatusTimeout = 0x80000000u;  // | role << 8 | detail
+
+struct DenseParams {
+  int M, N, K, batch;
+  int tiles_m, tiles_n;  // tiles per matrix; a tile is (128*CG) x bn
+  int num_tiles;         // batch * tiles_m * tiles_n
+  int raster_group;      // tile rows swept together (column-wise inside the group)
+  int bn;                // tile N (multiple of 64, <= 256)
+  int stages;            // ring depth
+  int num_kb;            // ceil(K / 64)
+  uint32_t tmem_cols;    // power of two >= 2 * bn
+  uint32_t idesc;        // tcgen05 instruction descriptor
+  uint32_t a_stage_bytes, b_stage_bytes;  // per CTA, per stage
+  int a_kmajor, b_kmajor;                 // 1: K contiguous in memory; 0: M (resp. N) contiguous
+  int b_rows;                             // rows of B (N extent) this CTA loads per stage
+  uint64_t a_desc_hi, b_desc_hi;          // descriptor bits above the start address
+  uint32_t a_kstep, b_kstep;              // start-address advance per K = 16 slice, bytes
+  int out_dtype;                          // 0 bf16, 1 f16, 2 f32
+  int epilogue;                           // gemm_epilogue_t
+  float alpha, beta;
+  const float* bias;
+  const void* c_in;                       // = D buffer; read when beta != 0
+  long long ldc, stride_c;                // elements
+  uint32_t* status;                       // device status word
+  unsigned long long timeout_ns;
+  uint32_t debug_flags;                   // bit 0: withhold one producer arrival (timeout test hook)
+};
+
+struct WaitCtx {
+  volatile uint32_t* s_abort;  // shared: set once any thread of the CTA gave up
+  uint32_t* g_status;          // global status word (also polled, so that an abort spreads between CTAs)
+  unsigned long long timeout_ns;
+};
+
+// Bounded mbarrier wait.  Returns false when the wait was abandoned: either this thread ran out of
+// time (it then records `code` in the status word) or another thread already aborted.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, const WaitCtx& w, uint32_t code) {
+  const uint64_t t0 = globaltimer_ns();
+  uint32_t it = 0;
+  while (true) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((++it & 31u) == 0u) {
+      if (*w.s_abort) return false;
+      if (*reinterpret_cast<volatile uint32_t*>(w.g_status) != 0u) {
+        *w.s_abort = 1u;
+        return false;
+      }
+      if (globaltimer_ns() - t0 > w.timeout_ns) {
+        *w.s_abort = 1u;
+        atomicCAS(w.g_status, 0u, kStatusTimeout | code);
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& w, uint32_t code) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, w, code);
+}
+
+struct TileCoord {
+  int batch, tm, tn;
+};
+// Linear tile id -> (batch, tile row, tile column).  Inside one matrix, tiles are visited in groups
+// of `raster_group` tile rows; inside a group the row index runs fastest, so the CTAs that are
+// resident together work on a compact block of the output and share A and B panels in L2.
+__device__ __forceinline__ TileCoord decode_tile(int t, int tiles_m, int tiles_n, int raster_group) {
+  TileCoord c;
+  const int per_matrix = tiles_m * tiles_n;
+  c.batch = t / per_matrix;
+  const int r = t - c.batch * per_matrix;
+  const int group_sz = raster_group * tiles_n;
+  const int g = r / group_sz;
+  const int first_m = g * raster_group;
+  const int gm = min(raster_group, tiles_m - first_m);
+  const int within = r - g * group_sz;
+  c.tn = within / gm;
+  c.tm = first_m + (within - c.tn * gm);
+  return c;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t d;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
+  uint32_t d;
+  asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+__device__ __forceinline__ float gelu_erf(float x) { return 0.5f * x * (1.0f + erff(x * 0.70710678118654752f)); }
+
+// alpha/beta/bias/activation on 32 consecutive columns of one output row, in fp32.
+__device__ __forceinline__ void epilogue_math(float (&v)[32], const uint32_t (&acc)[32], const DenseParams& p, long long row,
+                                              int col0, int batch) {
+#pragma unroll
+  for (int j = 0; j < 32; ++j) v[j] = p.alpha * __uint_as_float(acc[j]);
+  if (p.beta != 0.0f && row < p.M) {
+    const long long off = static_cast<long long>(batch) * p.stride_c + row * p.ldc + col0;
+    if (col0 + 32 <= p.N) {
+      if (p.out_dtype == 2) {
+        const float4* src = reinterpret_cast<const float4*>(static_cast<const float*>(p.c_in) + off);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const float4 c = src[j];
+          v[4 * j + 0] += p.beta * c.x;
+          v[4 * j + 1] += p.beta * c.y;
+          v[4 * j + 2] += p.beta * c.z;
+          v[4 * j + 3] += p.beta * c.w;
+        }
+      } else {
+        const uint4* src = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(p.c_in) + off);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const uint4 c = src[j];
+          const uint32_t w[4] = {c.x, c.y, c.z, c.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            float lo, hi;
+            if (p.out_dtype == 0) {
+              lo = __uint_as_float(w[e] << 16);
+              hi = __uint_as_float(w[e] & 0xFFFF0000u);
+            } else {
+              const __half2 h = *reinterpret_cast<const __half2*>(&w[e]);
+              lo = __low2float(h);
+              hi = __high2float(h);
+            }
+            v[8 * j + 2 * e + 0] += p.beta * lo;
+            v[8 * j + 2 * e + 1] += p.beta * hi;
+          }
+        }
+      }
+    } else {
+      for (int j = 0; j < 32; ++j) {
+        if (col0 + j < p.N) {
+          float c;
+          if (p.out_dtype == 2) c = static_cast<const float*>(p.c_in)[off + j];
+          else if (p.out_dtype == 0) c = __bfloat162float(static_cast<const __nv_bfloat16*>(p.c_in)[off + j]);
+          else c = __half2float(static_cast<const __half*>(p.c_in)[off + j]);
+          v[j] += p.beta * c;
+        }
+      }
+    }
+  }
+  if (p.epilogue & 1) {  // bias variants are the odd enum values
+    if (col0 + 32 <= p.N) {
+      const float4* b4 = reinterpret_cast<const float4*>(p.bias + col0);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const float4 b = __ldg(b4 + j);
+        v[4 * j + 0] += b.x;
+        v[4 * j + 1] += b.y;
+        v[4 * j + 2] += b.z;
+        v[4 * j + 3] += b.w;
+      }
+    } else {
+      for (int j = 0; j < 32; ++j)
+        if (col0 + j < p.N) v[j] += __ldg(p.bias + col0 + j);
+    }
+  }
+  if (p.epilogue == 2 || p.epilogue == 3) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.0f);
+  } else if (p.epilogue >= 4) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = gelu_erf(v[j]);
+  }
+}
+
+template <int CG>
+__device__ __forceinline__ void producer_role(const DenseParams& p, const CUtensorMap* tmA, const CUtensorMap* tmB,
+                                              uint32_t tiles_base, uint32_t full0, uint32_t empty0, uint32_t cta_rank,
+                                              int cluster_id, int num_clusters, const WaitCtx& w) {
+  const uint32_t stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
+  uint32_t kc = 0;
+  bool stall_pending = (p.debug_flags & 1u) != 0u;
+  for (int tile = cluster_id; tile < p.num_tiles; tile += num_clusters) {
+    const TileCoord tc = decode_tile(tile, p.tiles_m, p.tiles_n, p.raster_group);
+    const int m0 = tc.tm * (kCtaM * CG) + static_cast<int>(cta_rank) * kCtaM;
+    const int n0 = tc.tn * p.bn + (CG == 2 ? static_cast<int>(cta_rank) * p.b_rows : 0);
+    for (int kb = 0; kb < p.num_kb; ++kb, ++kc) {
+      const uint32_t s = kc % static_cast<uint32_t>(p.stages);
+      const uint32_t ph = (kc / static_cast<uint32_t>(p.stages)) & 1u;
+      if (!mbar_wait(empty0 + 8u * s, ph ^ 1u, w, (1u << 8) | s)) return;
+      if (stall_pending) {  // test hook: this stage is never filled nor signalled
+        stall_pending = false;
+        continue;
+      }
+      const uint32_t full_local = full0 + 8u * s;
+      if (CG == 1 || cta_rank == 0) mbar_arrive_expect_tx(full_local, stage_bytes * CG);
+      const uint32_t bar = (CG == 1) ? full_local : mapa(full_local, 0);
+      const uint32_t sa = tiles_base + s * stage_bytes;
+      const uint32_t sb = sa + p.a_stage_bytes;
+      const int k0 = kb * kBlockK;
+      auto load = [&](uint32_t dst, const CUtensorMap* map, int x, int y) {
+        if constexpr (CG == 1) tma_load_3d(dst, map, bar, x, y, tc.batch);
+        else tma_load_3d_pair(dst, map, bar, x, y, tc.batch);
+      };
+      if (p.a_kmajor) {
+        load(sa, tmA, k0, m0);
+      } else {
+        load(sa, tmA, m0, k0);
+        load(sa + 8192u, tmA, m0 + 64, k0);
+      }
+      if (p.b_kmajor) {
+        load(sb, tmB, k0, n0);
+      } else {
+        for (int g = 0; g < p.b_rows / 64; ++g) load(sb + 8192u * g, tmB, n0 + 64 * g, k0);
+      }
+    }
+  }
+}
+
+template <int CG>
+__device__ __forceinline__ void mma_role(const DenseParams& p, uint32_t tiles_base, uint32_t full0, uint32_t empty0,
+                                         uint32_t tfull0, uint32_t tempty0, uint32_t tmem_base, int cluster_id,
+                                         int num_clusters, const WaitCtx& w) {
+  const uint32_t stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
+  uint32_t kc = 0, it = 0;
+  for (int tile = cluster_id; tile < p.num_tiles; tile += num_clusters, ++it) {
+    const uint32_t buf = it & 1u;
+    const uint32_t aph = (it >> 1) & 1u;
+    if (!mbar_wait(tempty0 + 8u * buf, aph ^ 1u, w, (2u << 8) | 0x80u | buf)) return;
+    tc_fence_after();
+    const uint32_t d_tmem = tmem_base + buf * static_cast<uint32_t>(p.bn);
+    for (int kb = 0; kb < p.num_kb; ++kb, ++kc) {
+      const uint32_t s = kc % static_cast<uint32_t>(p.stages);
+      const uint32_t ph = (kc / static_cast<uint32_t>(p.stages)) & 1u;
+      if (!mbar_wait(full0 + 8u * s, ph, w, (2u << 8) | s)) return;
+      tc_fence_after();
+      const uint32_t sa = tiles_base + s * stage_bytes;
+      const uint32_t sb = sa + p.a_stage_bytes;
+#pragma unroll
+      for (int k = 0; k < kBlockK / kUmmaK; ++k) {
+        umma_f16<CG>(d_tmem, smem_desc(p.a_desc_hi, sa + k * p.a_kstep), smem_desc(p.b_desc_hi, sb + k * p.b_kstep),
+                     p.idesc, static_cast<uint32_t>((kb | k) != 0));
+      }
+      umma_commit<CG>(empty0 + 8u * s);  // ring slot reusable once these MMAs have read it
+      if constexpr (CG == 2) umma_commit<CG>(mapa(empty0 + 8u * s, 1));
+    }
+    umma_commit<CG>(tfull0 + 8u * buf);  // accumulator complete
+    if constexpr (CG == 2) umma_commit<CG>(mapa(tfull0 + 8u * buf, 1));
+  }
+}
+
+template <int CG, int EPI_WG>
+__device__ __forceinline__ void epilogue_role(const DenseParams& p, const CUtensorMap* tmD, uint32_t staging, uint32_t tfull0,
+                                              uint32_t tempty0, uint32_t tmem_base, uint32_t cta_rank, int cluster_id,
+                                              int num_clusters, const WaitCtx& w) {
+  const uint32_t warp = threadIdx.x >> 5;
+  const uint32_t lane = lane_id();
+  const uint32_t q = warp & 3u;            // TMEM lane quarter this warp may read
+  const uint32_t ew = warp - 2u;           // epilogue warp index
+  const uint32_t wg = ew >> 2;             // epilogue warpgroup: takes every EPI_WG-th slab
+  const uint32_t stg = staging + ew * (2u * kSlabBytes);
+  const int slab_cols = (p.out_dtype == 2) ? 32 : 64;
+  const int nslabs = p.bn / slab_cols;
+  uint32_t it = 0, nstore = 0;
+  for (int tile = cluster_id; tile < p.num_tiles; tile += num_clusters, ++it) {
+    const TileCoord tc = decode_tile(tile, p.tiles_m, p.tiles_n, p.raster_group);
+    const uint32_t buf = it & 1u;
+    const uint32_t ph = (it >> 1) & 1u;
+    if (!mbar_wait(tfull0 + 8u * buf, ph, w, (3u << 8) | buf)) return;
+    tc_fence_after();
+    const int row0 = tc.tm * (kCtaM * CG) + static_cast<int>(cta_rank) * kCtaM + static_cast<int>(q) * 32;
+    const long long row = row0 + static_cast<int>(lane);
+    const uint32_t t_row = tmem_base + ((q * 32u) << 16) + buf * static_cast<uint32_t>(p.bn);
+    for (int sl = static_cast<int>(wg); sl < nslabs; sl += EPI_WG, ++nstore) {
+      const int col0 = tc.tn * p.bn + sl * slab_cols;
+      const uint32_t sbuf = stg + (nstore & 1u) * kSlabBytes;
+      if (lane == 0) bulk_wait_group_read<1>();  // the store that last read this slab buffer is done
+      __syncwarp();
+      const uint32_t srow = sbuf + lane * 128u;
+      const uint32_t sw = lane & 7u;
+      uint32_t acc[32];
+      float v[32];
+      if (p.out_dtype == 2) {
+        tmem_ld_32x32(t_row + static_cast<uint32_t>(sl * 32), acc);
+        tmem_ld_wait();
+        epilogue_math(v, acc, p, row, col0, tc.batch);
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          st_shared_v4(srow + ((static_cast<uint32_t>(j) ^ sw) << 4), __float_as_uint(v[4 * j]), __float_as_uint(v[4 * j + 1]),
+                       __float_as_uint(v[4 * j + 2]), __float_as_uint(v[4 * j + 3]));
+      } else {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          tmem_ld_32x32(t_row + static_cast<uint32_t>(sl * 64 + h * 32), acc);
+          tmem_ld_wait();
+          epilogue_math(v, acc, p, row, col0 + h * 32, tc.batch);
+          uint32_t pk[16];
+          if (p.out_dtype == 0) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) pk[j] = pack_bf16x2(v[2 * j], v[2 * j + 1]);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) pk[j] = pack_f16x2(v[2 * j], v[2 * j + 1]);
+          }
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            st_shared_v4(srow + ((static_cast<uint32_t>(4 * h + j) ^ sw) << 4), pk[4 * j], pk[4 * j + 1], pk[4 * j + 2],
+                         pk[4 * j + 3]);
+        }
+      }
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) {
+        if (row0 < p.M && col0 < p.N) tma_store_3d(tmD, sbuf, col0, row0, tc.batch);
+        bulk_commit_group();
+      }
+    }
+    // every tcgen05.ld of this accumulator buffer has completed: hand it back to the MMA issuer
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) {
+      if constexpr (CG == 1) mbar_arrive(tempty0 + 8u * buf);
+      else mbar_arrive_cluster(mapa(tempty0 + 8u * buf, 0));
+    }
+  }
+  if (lane == 0) bulk_wait_group<0>();
+}
+
+template <int CG, int EPI_WG>
+__global__ void __launch_bounds__(64 + 128 * EPI_WG, 1)
+dense_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                  const __grid_constant__ CUtensorMap tmD, const DenseParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_addr(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;  // 128-byte swizzle atoms need 1024-byte alignment
+  uint8_t* gen = smem_raw + (base - raw);
+  const uint32_t warp = threadIdx.x >> 5;
+  const uint32_t cta_rank = (CG == 2) ? cluster_ctarank() : 0u;
+  const int cluster_id = static_cast<int>(blockIdx.x) / CG;
+  const int num_clusters = static_cast<int>(gridDim.x) / CG;
+
+  const uint32_t stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
+  const uint32_t staging_off = static_cast<uint32_t>(p.stages) * stage_bytes;
+  const uint32_t bars_off = staging_off + 4u * EPI_WG * 2u * kSlabBytes;
+  const uint32_t full0 = base + bars_off;
+  const uint32_t empty0 = full0 + 8u * kMaxStages;
+  const uint32_t tfull0 = empty0 + 8u * kMaxStages;
+  const uint32_t tempty0 = tfull0 + 16u;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + bars_off + 16u * kMaxStages + 32u);
+  volatile uint32_t* s_abort = tmem_slot + 1;
+  const WaitCtx w{s_abort, p.status, p.timeout_ns};
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(full0 + 8u * s, 1);
+      mbar_init(empty0 + 8u * s, 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(tfull0 + 8u * b, 1);
+      mbar_init(tempty0 + 8u * b, 4u * EPI_WG * CG);
+    }
+    *s_abort = 0u;
+    fence_mbar_init();
+    prefetch_tensormap(&tmA);
+    prefetch_tensormap(&tmB);
+    prefetch_tensormap(&tmD);
+  }
+  if (warp == 1) {
+    tmem_alloc<CG>(smem_addr(const_cast<uint32_t*>(tmem_slot)), p.tmem_cols);
+    tmem_relinquish<CG>();
+  }
+  tc_fence_before();
+  __syncthreads();
+  if constexpr (CG == 2) {  // the peer's barriers must exist before anything signals them
+    cluster_arrive();
+    cluster_wait();
+  }
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane_id() == 0) producer_role<CG>(p, &tmA, &tmB, base, full0, empty0, cta_rank, cluster_id, num_clusters, w);
+    __syncwarp();
+  } else if (warp == 1) {
+    if (lane_id() == 0 && cta_rank == 0)
+      mma_role<CG>(p, base, full0, empty0, tfull0, tempty0, tmem_base, cluster_id, num_clusters, w);
+    __syncwarp();
+  } else {
+    epilogue_role<CG, EPI_WG>(p, &tmD, base + staging_off, tfull0, tempty0, tmem_base, cta_rank, cluster_id, num_clusters, w);
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if constexpr (CG == 2) {  // neither CTA may free tensor memory or exit while its peer still uses the pair
+    cluster_arrive();
+    cluster_wait();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc<CG>(tmem_base, p.tmem_cols);
+  }
+}
+
+}  // namespace b200

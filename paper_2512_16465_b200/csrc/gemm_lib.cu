@@ -1,0 +1,537 @@
+// Host side of the b200 GEMM library: the C ABI of include/gemm.h.
+//   gemm_plan  : validation, roofline classification, variant / tile / stage / raster choice (host only)
+//   gemm_run   : tensor-map encoding and the kernel launch (asynchronous)
+// No cuBLAS / CUTLASS, no fallback path: an unsupported request is an error code.
+#include "../../include/gemm.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+#include <new>
+
+#include "dense_kernel.cuh"
+#include "skinny_kernel.cuh"
+
+using namespace b200;
+
+namespace {
+
+constexpr int kDefaultSmCount = 148;        // B200
+constexpr int kMaxSmemOptin = 232448;       // 227 KB dynamic shared memory per CTA on sm_100
+// Machine ridges for the plan-time roofline class (FLOP per byte): tensor-core ridge and CUDA-core ridge
+// from the public B200 figures (2250 TFLOP/s dense 16-bit, about 75 TFLOP/s fp32 FMA, 8 TB/s HBM3e).
+constexpr double kRidgeTensor = 2250.0e12 / 8.0e12;
+constexpr double kRidgeCudaCore = 75.0e12 / 8.0e12;
+
+thread_local char g_last_cuda_error[160] = "";
+
+void note_cuda_error(const char* what, const char* name) {
+  snprintf(g_last_cuda_error, sizeof g_last_cuda_error, "%s: %s", what, name ? name : "?");
+}
+
+using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn get_encode_fn() {
+  static EncodeFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeFn>(p);
+  });
+  return fn;
+}
+
+int elem_bytes(int dtype) { return dtype == GEMM_F32 ? 4 : 2; }
+
+CUtensorMapDataType tm_dtype(int dtype) {
+  return dtype == GEMM_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16
+                            : (dtype == GEMM_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32);
+}
+
+// 3-D tiled map over a row-major matrix batch: dim0 = contiguous extent, dim1 = rows, dim2 = batch.
+// 128-byte swizzle, out-of-bounds elements read as zero / are not written.
+bool encode_map(CUtensorMap* m, int dtype, const void* base, uint64_t inner, uint64_t rows, uint64_t batch, uint64_t ld,
+                uint64_t batch_stride, uint32_t box_inner, uint32_t box_rows) {
+  EncodeFn fn = get_encode_fn();
+  if (!fn) {
+    note_cuda_error("cuTensorMapEncodeTiled", "driver entry point not found");
+    return false;
+  }
+  const uint64_t eb = static_cast<uint64_t>(elem_bytes(dtype));
+  cuuint64_t dims[3] = {inner, rows, batch};
+  cuuint64_t strides[2] = {ld * eb, (batch > 1 ? batch_stride : rows * ld) * eb};
+  cuuint32_t box[3] = {box_inner, box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(m, tm_dtype(dtype), 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    char buf[64];
+    snprintf(buf, sizeof buf, "CUresult %d", static_cast<int>(r));
+    note_cuda_error("cuTensorMapEncodeTiled", buf);
+    return false;
+  }
+  return true;
+}
+
+int ceil_div(long long a, long long b) { return static_cast<int>((a + b - 1) / b); }
+
+}  // namespace
+
+struct gemm_plan_s {
+  gemm_desc_t d;
+  gemm_info_t info;
+  int variant;     // gemm_variant_t
+  int cg;          // CTAs per tile (dense)
+  int epi_wg;      // epilogue warpgroups (dense)
+  int bn;          // tile N (dense)
+  int stages;
+  int raster_group;
+  int grid;
+  int smem_bytes;
+  int sm_count;
+  bool has_device;
+  bool arch_ok;
+  uint32_t* d_status;
+  uint32_t timeout_ms;
+  DenseParams dense;     // filled at plan time except pointers / scalars
+  SkinnyPlan skinny;     // stream-K decomposition of the skinny variant
+};
+
+namespace {
+
+bool has_bias(int epi) { return epi == GEMM_EPI_BIAS || epi == GEMM_EPI_BIAS_RELU || epi == GEMM_EPI_BIAS_GELU_ERF; }
+
+gemm_status_t validate(const gemm_desc_t* d) {
+  if (d->struct_size != sizeof(gemm_desc_t)) return GEMM_ERR_INVALID_ARG;
+  if (d->M < 1 || d->N < 1 || d->K < 1 || d->batch_count < 1) return GEMM_ERR_INVALID_ARG;
+  if (d->M > 0x7FFFFFFFll || d->N > 0x7FFFFFFFll || d->K > 0x7FFFFFFFll) return GEMM_ERR_INVALID_ARG;
+  if ((d->transa != GEMM_OP_N && d->transa != GEMM_OP_T) || (d->transb != GEMM_OP_N && d->transb != GEMM_OP_T))
+    return GEMM_ERR_INVALID_ARG;
+  if (d->ab_dtype < GEMM_BF16 || d->ab_dtype > GEMM_F32 || d->c_dtype < GEMM_BF16 || d->c_dtype > GEMM_F32)
+    return GEMM_ERR_INVALID_ARG;
+  if (d->epilogue < GEMM_EPI_NONE || d->epilogue > GEMM_EPI_BIAS_GELU_ERF) return GEMM_ERR_INVALID_ARG;
+  if (d->ab_dtype == GEMM_F32) return GEMM_ERR_UNSUPPORTED;
+  const int64_t a_row = d->transa == GEMM_OP_N ? d->K : d->M;
+  const int64_t b_row = d->transb == GEMM_OP_N ? d->N : d->K;
+  if (d->lda < a_row || d->ldb < b_row || d->ldc < d->N) return GEMM_ERR_INVALID_ARG;
+  const int64_t a_rows = d->transa == GEMM_OP_N ? d->M : d->K;
+  const int64_t b_rows = d->transb == GEMM_OP_N ? d->K : d->N;
+  if (d->batch_count > 1) {
+    if (d->stride_a < 0 || d->stride_b < 0 || d->stride_c < 0) return GEMM_ERR_INVALID_ARG;
+    if (d->stride_c < (d->M - 1) * d->ldc + d->N) return GEMM_ERR_INVALID_ARG;  // outputs would overlap
+    if (d->stride_a == 0 || d->stride_b == 0) return GEMM_ERR_UNSUPPORTED;      // operand broadcast
+    (void)a_rows;
+    (void)b_rows;
+  }
+  const int eab = 2, ec = elem_bytes(d->c_dtype);
+  if ((d->lda * eab) % 16 || (d->ldb * eab) % 16 || (d->ldc * ec) % 16) return GEMM_ERR_ALIGNMENT;
+  if (d->batch_count > 1 && ((d->stride_a * eab) % 16 || (d->stride_b * eab) % 16 || (d->stride_c * ec) % 16))
+    return GEMM_ERR_ALIGNMENT;
+  return GEMM_OK;
+}
+
+int dense_smem_bytes(int stages, int a_stage, int b_stage, int epi_wg) {
+  return 1024 /*alignment slack*/ + stages * (a_stage + b_stage) + 4 * epi_wg * 2 * kSlabBytes + 16 * kMaxStages + 64;
+}
+
+// Fill plan->dense and the launch geometry for a dense variant.
+gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_raster, int forced_stages) {
+  const gemm_desc_t& d = pl->d;
+  const int a_kmajor = d.transa == GEMM_OP_N;
+  const int b_kmajor = d.transb == GEMM_OP_T;
+  const int tile_m = kCtaM * cg;
+  const int tiles_m = ceil_div(d.M, tile_m);
+  // tile N: the widest tile that still gives every SM (pair) work; B tiles with N contiguous are loaded in
+  // 64-column boxes per CTA, so a pair needs bn % 128 == 0 there
+  const int bn_step = (!b_kmajor && cg == 2) ? 128 : 64;
+  int bn = forced_bn;
+  if (bn == 0) {
+    const int units = pl->sm_count / cg;
+    bn = 256;
+    while (bn > bn_step) {
+      const long long tiles = static_cast<long long>(tiles_m) * ceil_div(d.N, bn) * d.batch_count;
+      if (tiles >= units && d.N > bn / 2) break;
+      bn -= bn_step;  // 256 -> 192 -> 128 -> 64
+      if (bn == 192) bn = 128;
+    }
+  }
+  if (bn < bn_step || bn > 256 || bn % bn_step) return GEMM_ERR_UNSUPPORTED;
+  const int tiles_n = ceil_div(d.N, bn);
+  const int b_rows = bn / cg;
+  const int a_stage = kCtaM * kBlockK * 2;
+  const int b_stage = b_rows * kBlockK * 2;
+  const int epi_wg = 1;
+  int stages = forced_stages;
+  if (stages == 0) {
+    stages = (kMaxSmemOptin - dense_smem_bytes(0, a_stage, b_stage, epi_wg)) / (a_stage + b_stage);
+    stages = std::min(stages, 8);
+  }
+  if (stages < 2 || stages > kMaxStages) return GEMM_ERR_UNSUPPORTED;
+  const int smem = dense_smem_bytes(stages, a_stage, b_stage, epi_wg);
+  if (smem > kMaxSmemOptin) return GEMM_ERR_UNSUPPORTED;
+  const long long num_tiles = static_cast<long long>(tiles_m) * tiles_n * d.batch_count;
+  if (num_tiles > 0x7FFFFFFFll) return GEMM_ERR_UNSUPPORTED;
+  // raster group height G: the resident tiles cover G tile rows x (units / G) tile columns; operand traffic from L2
+  // is smallest when that block is square in elements, G * tile_m ~ (units / G) * bn
+  int raster = forced_raster;
+  if (raster == 0) {
+    const double units = static_cast<double>(pl->sm_count / cg);
+    raster = static_cast<int>(std::lround(std::sqrt(units * bn / tile_m)));
+    raster = std::max(1, raster);
+  }
+  raster = std::max(1, std::min(raster, tiles_m));
+
+  DenseParams& p = pl->dense;
+  memset(&p, 0, sizeof p);
+  p.M = static_cast<int>(d.M);
+  p.N = static_cast<int>(d.N);
+  p.K = static_cast<int>(d.K);
+  p.batch = d.batch_count;
+  p.tiles_m = tiles_m;
+  p.tiles_n = tiles_n;
+  p.num_tiles = static_cast<int>(num_tiles);
+  p.raster_group = raster;
+  p.bn = bn;
+  p.stages = stages;
+  p.num_kb = ceil_div(d.K, kBlockK);
+  uint32_t cols = 32;
+  while (cols < 2u * bn) cols <<= 1;
+  p.tmem_cols = cols;
+  p.idesc = make_idesc(d.ab_dtype == GEMM_BF16, !a_kmajor, !b_kmajor, tile_m, bn);
+  p.a_stage_bytes = a_stage;
+  p.b_stage_bytes = b_stage;
+  p.a_kmajor = a_kmajor;
+  p.b_kmajor = b_kmajor;
+  p.b_rows = b_rows;
+  // K-major tile: rows of 128 bytes, 8-row swizzle atoms 1024 bytes apart (stride offset); the leading offset is unused.
+  // MN-major tile: 64-element (128-byte) runs along M/N, k rows 128 bytes apart, 8-k-row atoms 1024 bytes apart
+  // (stride offset) and the next 64-element run group one whole 64 x 64 box = 8192 bytes further (leading offset).
+  p.a_desc_hi = a_kmajor ? make_smem_desc_hi(16, 1024) : make_smem_desc_hi(8192, 1024);
+  p.b_desc_hi = b_kmajor ? make_smem_desc_hi(16, 1024) : make_smem_desc_hi(8192, 1024);
+  p.a_kstep = a_kmajor ? kUmmaK * 2 : kUmmaK * 128;
+  p.b_kstep = b_kmajor ? kUmmaK * 2 : kUmmaK * 128;
+  p.out_dtype = d.c_dtype;
+  p.epilogue = d.epilogue;
+  p.ldc = d.ldc;
+  p.stride_c = d.batch_count > 1 ? d.stride_c : 0;
+  p.debug_flags = (d.flags & GEMM_FLAG_DEBUG_STALL) ? 1u : 0u;
+
+  pl->cg = cg;
+  pl->epi_wg = epi_wg;
+  pl->bn = bn;
+  pl->stages = stages;
+  pl->raster_group = raster;
+  pl->smem_bytes = smem;
+  const int units = pl->sm_count / cg;
+  pl->grid = static_cast<int>(std::min<long long>(num_tiles, units)) * cg;
+  pl->variant = cg == 2 ? GEMM_VARIANT_DENSE_2CTA : GEMM_VARIANT_DENSE_1CTA;
+
+  gemm_info_t& info = pl->info;
+  info.variant = pl->variant;
+  info.tile_m = tile_m;
+  info.tile_n = bn;
+  info.tile_k = kBlockK;
+  info.stages = stages;
+  info.cluster_size = cg;
+  info.grid = pl->grid;
+  info.raster_group = raster;
+  info.split = 1;
+  info.smem_bytes = smem;
+  info.num_tiles = num_tiles;
+  info.workspace_bytes = 0;
+  return GEMM_OK;
+}
+
+gemm_status_t plan_skinny(gemm_plan_s* pl, int forced_stages) {
+  const gemm_desc_t& d = pl->d;
+  if (d.transa != GEMM_OP_N || d.transb != GEMM_OP_T) return GEMM_ERR_UNSUPPORTED;  // both operands K-contiguous
+  if (d.M > kSkinnyMaxM || d.batch_count != 1) return GEMM_ERR_UNSUPPORTED;
+  SkinnyPlan& s = pl->skinny;
+  if (!skinny_make_plan(&s, static_cast<int>(d.M), static_cast<int>(d.N), static_cast<int>(d.K), pl->sm_count, forced_stages,
+                        kMaxSmemOptin))
+    return GEMM_ERR_UNSUPPORTED;
+  pl->variant = GEMM_VARIANT_SKINNY_STREAMK;
+  pl->cg = 1;
+  pl->stages = s.stages;
+  pl->grid = s.grid;
+  pl->smem_bytes = s.smem_bytes;
+  gemm_info_t& info = pl->info;
+  info.variant = pl->variant;
+  info.tile_m = kSkinnyTileN;  // rows of the weight matrix (output columns) per tile
+  info.tile_n = s.m_pad;
+  info.tile_k = kBlockK;
+  info.stages = s.stages;
+  info.cluster_size = 1;
+  info.grid = s.grid;
+  info.raster_group = 1;
+  info.split = s.max_contributors;
+  info.smem_bytes = s.smem_bytes;
+  info.num_tiles = s.total_units;
+  info.workspace_bytes = s.workspace_bytes;
+  return GEMM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
+  if (!desc || !out_plan) return GEMM_ERR_NULL;
+  *out_plan = nullptr;
+  gemm_status_t st = validate(desc);
+  if (st != GEMM_OK) return st;
+  gemm_plan_s* pl = new (std::nothrow) gemm_plan_s();
+  if (!pl) return GEMM_ERR_CUDA;
+  memset(pl, 0, sizeof *pl);
+  pl->d = *desc;
+  if (pl->d.batch_count == 1) pl->d.stride_a = pl->d.stride_b = pl->d.stride_c = 0;
+  pl->timeout_ms = 2000;
+  pl->sm_count = kDefaultSmCount;
+  int dev = -1;
+  if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0) {
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, dev) == cudaSuccess) {
+      pl->has_device = true;
+      pl->arch_ok = prop.major == 10;
+      if (pl->arch_ok) pl->sm_count = prop.multiProcessorCount;
+    }
+  }
+  (void)cudaGetLastError();
+
+  // roofline class (Section 4.3): compulsory traffic vs. work
+  const gemm_desc_t& d = pl->d;
+  const double eb = 2.0, ec = elem_bytes(d.c_dtype);
+  const double flops = 2.0 * d.M * d.N * d.K * d.batch_count;
+  double bytes = d.batch_count * (static_cast<double>(d.M) * d.K + static_cast<double>(d.K) * d.N) * eb +
+                 d.batch_count * static_cast<double>(d.M) * d.N * ec;
+  if (has_bias(d.epilogue)) bytes += 4.0 * d.N;
+  gemm_info_t& info = pl->info;
+  info.struct_size = sizeof(gemm_info_t);
+  info.flops = flops;
+  info.min_bytes = bytes;  // beta is a run-time scalar: the C read is not counted here
+  info.intensity = flops / bytes;
+  info.regime = info.intensity < kRidgeCudaCore ? GEMM_REGIME_MEMORY
+                                                : (info.intensity < kRidgeTensor ? GEMM_REGIME_MIDDLE : GEMM_REGIME_COMPUTE);
+
+  const int forced_variant = (d.flags & GEMM_FLAG_VARIANT_MASK) >> GEMM_FLAG_VARIANT_SHIFT;
+  const int forced_bn = static_cast<int>((d.flags & GEMM_FLAG_TILE_N_MASK) >> GEMM_FLAG_TILE_N_SHIFT) * 16;
+  const int forced_raster = (d.flags & GEMM_FLAG_RASTER_MASK) >> GEMM_FLAG_RASTER_SHIFT;
+  const int forced_stages = (d.flags & GEMM_FLAG_STAGES_MASK) >> GEMM_FLAG_STAGES_SHIFT;
+  int variant = forced_variant;
+  if (variant == 0) {
+    // memory-bound problems with a handful of rows stream the weight matrix once: stream-K path;
+    // everything else is a dense tiled GEMM, paired CTAs when there are at least two tile rows
+    const bool skinny_ok = d.M <= kSkinnyMaxM && d.batch_count == 1 && d.transa == GEMM_OP_N && d.transb == GEMM_OP_T;
+    if (skinny_ok && info.intensity < 4.0 * kRidgeCudaCore) variant = GEMM_VARIANT_SKINNY_STREAMK;
+    else variant = GEMM_VARIANT_DENSE_1CTA;
+  }
+  if (variant == GEMM_VARIANT_DENSE_1CTA) st = plan_dense(pl, 1, forced_bn, forced_raster, forced_stages);
+  else if (variant == GEMM_VARIANT_DENSE_2CTA) st = plan_dense(pl, 2, forced_bn, forced_raster, forced_stages);
+  else if (variant == GEMM_VARIANT_SKINNY_STREAMK) st = plan_skinny(pl, forced_stages);
+  else st = GEMM_ERR_INVALID_ARG;
+  if (st != GEMM_OK) {
+    delete pl;
+    return st;
+  }
+  if (pl->has_device && pl->arch_ok) {
+    if (cudaMalloc(&pl->d_status, 16) != cudaSuccess || cudaMemset(pl->d_status, 0, 16) != cudaSuccess) {
+      note_cuda_error("cudaMalloc(status word)", cudaGetErrorName(cudaGetLastError()));
+      delete pl;
+      return GEMM_ERR_CUDA;
+    }
+  }
+  if (getenv("B200GEMM_LOG")) {
+    fprintf(stderr,
+            "[b200gemm] M=%lld N=%lld K=%lld batch=%d AI=%.1f regime=%d variant=%d tile=%dx%dx%d stages=%d cluster=%d "
+            "grid=%d raster=%d split=%d smem=%d ws=%zu\n",
+            (long long)d.M, (long long)d.N, (long long)d.K, d.batch_count, info.intensity, info.regime, info.variant,
+            info.tile_m, info.tile_n, info.tile_k, info.stages, info.cluster_size, info.grid, info.raster_group, info.split,
+            info.smem_bytes, info.workspace_bytes);
+  }
+  *out_plan = pl;
+  return GEMM_OK;
+}
+
+size_t gemm_workspace_bytes(gemm_plan_t plan) { return plan ? plan->info.workspace_bytes : 0; }
+
+gemm_status_t gemm_plan_info(gemm_plan_t plan, gemm_info_t* out) {
+  if (!plan || !out) return GEMM_ERR_NULL;
+  if (out->struct_size != sizeof(gemm_info_t)) return GEMM_ERR_INVALID_ARG;
+  *out = plan->info;
+  return GEMM_OK;
+}
+
+gemm_status_t gemm_plan_set_timeout_ms(gemm_plan_t plan, uint32_t ms) {
+  if (!plan) return GEMM_ERR_NULL;
+  plan->timeout_ms = std::max(1u, ms);
+  return GEMM_OK;
+}
+
+gemm_status_t gemm_plan_status(gemm_plan_t plan) {
+  if (!plan) return GEMM_ERR_NULL;
+  if (!plan->d_status) return GEMM_ERR_ARCH;
+  uint32_t h[4] = {0, 0, 0, 0};
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e == cudaSuccess) e = cudaMemcpy(h, plan->d_status, 16, cudaMemcpyDeviceToHost);
+  if (e == cudaSuccess) e = cudaMemset(plan->d_status, 0, 16);
+  if (e != cudaSuccess) {
+    note_cuda_error("gemm_plan_status", cudaGetErrorName(e));
+    return GEMM_ERR_CUDA;
+  }
+  if (h[0] & kStatusTimeout) {
+    snprintf(g_last_cuda_error, sizeof g_last_cuda_error, "device wait expired: role %u detail 0x%02x", (h[0] >> 8) & 0xFF,
+             h[0] & 0xFF);
+    return GEMM_ERR_TIMEOUT;
+  }
+  return GEMM_OK;
+}
+
+gemm_status_t gemm_destroy(gemm_plan_t plan) {
+  if (!plan) return GEMM_OK;
+  gemm_status_t st = GEMM_OK;
+  if (plan->d_status && cudaFree(plan->d_status) != cudaSuccess) {
+    note_cuda_error("cudaFree", cudaGetErrorName(cudaGetLastError()));
+    st = GEMM_ERR_CUDA;
+  }
+  delete plan;
+  return st;
+}
+
+const char* gemm_status_string(gemm_status_t s) {
+  switch (s) {
+    case GEMM_OK: return "GEMM_OK";
+    case GEMM_ERR_NULL: return "GEMM_ERR_NULL";
+    case GEMM_ERR_INVALID_ARG: return "GEMM_ERR_INVALID_ARG";
+    case GEMM_ERR_UNSUPPORTED: return "GEMM_ERR_UNSUPPORTED";
+    case GEMM_ERR_ALIGNMENT: return "GEMM_ERR_ALIGNMENT";
+    case GEMM_ERR_WORKSPACE: return "GEMM_ERR_WORKSPACE";
+    case GEMM_ERR_ARCH: return "GEMM_ERR_ARCH";
+    case GEMM_ERR_CUDA: return "GEMM_ERR_CUDA";
+    case GEMM_ERR_TIMEOUT: return "GEMM_ERR_TIMEOUT";
+  }
+  return "GEMM_ERR_UNKNOWN";
+}
+
+const char* gemm_last_cuda_error(void) { return g_last_cuda_error; }
+
+}  // extern "C"
+
+namespace {
+
+template <int CG, int EPI_WG>
+gemm_status_t launch_dense(const gemm_plan_s* pl, const CUtensorMap& tA, const CUtensorMap& tB, const CUtensorMap& tD,
+                           const DenseParams& p, cudaStream_t stream) {
+  auto kern = dense_gemm_kernel<CG, EPI_WG>;
+  static thread_local int configured_smem = 0;  // per instantiation
+  if (configured_smem < pl->smem_bytes) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl->smem_bytes) != cudaSuccess) {
+      note_cuda_error("cudaFuncSetAttribute", cudaGetErrorName(cudaGetLastError()));
+      return GEMM_ERR_CUDA;
+    }
+    configured_smem = pl->smem_bytes;
+  }
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof cfg);
+  cfg.gridDim = dim3(pl->grid, 1, 1);
+  cfg.blockDim = dim3(64 + 128 * EPI_WG, 1, 1);
+  cfg.dynamicSmemBytes = pl->smem_bytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = CG;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tA, tB, tD, p);
+  if (e != cudaSuccess) {
+    note_cuda_error("cudaLaunchKernelEx(dense)", cudaGetErrorName(e));
+    (void)cudaGetLastError();
+    return GEMM_ERR_CUDA;
+  }
+  return GEMM_OK;
+}
+
+gemm_status_t run_dense(gemm_plan_s* pl, const void* A, const void* B, void* C, const float* bias, float alpha, float beta,
+                        cudaStream_t stream) {
+  const gemm_desc_t& d = pl->d;
+  DenseParams p = pl->dense;
+  CUtensorMap tA, tB, tD;
+  const uint64_t batch = d.batch_count;
+  // A: K-major -> rows are M, inner K, box 64 x 128; M-major (stored K x M) -> rows are K, inner M, box 64 x 64
+  bool ok = p.a_kmajor ? encode_map(&tA, d.ab_dtype, A, d.K, d.M, batch, d.lda, d.stride_a, kBlockK, kCtaM)
+                       : encode_map(&tA, d.ab_dtype, A, d.M, d.K, batch, d.lda, d.stride_a, 64, kBlockK);
+  ok = ok && (p.b_kmajor ? encode_map(&tB, d.ab_dtype, B, d.K, d.N, batch, d.ldb, d.stride_b, kBlockK, p.b_rows)
+                         : encode_map(&tB, d.ab_dtype, B, d.N, d.K, batch, d.ldb, d.stride_b, 64, kBlockK));
+  const uint32_t slab_cols = d.c_dtype == GEMM_F32 ? 32 : 64;
+  ok = ok && encode_map(&tD, d.c_dtype, C, d.N, d.M, batch, d.ldc, d.stride_c, slab_cols, 32);
+  if (!ok) return GEMM_ERR_CUDA;
+  p.alpha = alpha;
+  p.beta = beta;
+  p.bias = bias;
+  p.c_in = C;
+  p.status = pl->d_status;
+  p.timeout_ns = static_cast<unsigned long long>(pl->timeout_ms) * 1000000ull;
+  if (pl->cg == 1) return launch_dense<1, 1>(pl, tA, tB, tD, p, stream);
+  return launch_dense<2, 1>(pl, tA, tB, tD, p, stream);
+}
+
+gemm_status_t run_skinny(gemm_plan_s* pl, const void* A, const void* B, void* C, const float* bias, float alpha, float beta,
+                         void* workspace, cudaStream_t stream) {
+  const gemm_desc_t& d = pl->d;
+  const SkinnyPlan& s = pl->skinny;
+  CUtensorMap tW, tX;
+  // weights W = B stored N x K (K contiguous): box 64 x 128; activations X = A stored M x K: box 64 x m_pad
+  bool ok = encode_map(&tW, d.ab_dtype, B, d.K, d.N, 1, d.ldb, 0, kBlockK, kSkinnyTileN);
+  ok = ok && encode_map(&tX, d.ab_dtype, A, d.K, d.M, 1, d.lda, 0, kBlockK, s.m_pad);
+  if (!ok) return GEMM_ERR_CUDA;
+  SkinnyParams p;
+  memset(&p, 0, sizeof p);
+  p.plan = s;
+  p.M = static_cast<int>(d.M);
+  p.N = static_cast<int>(d.N);
+  p.K = static_cast<int>(d.K);
+  p.idesc = make_idesc(d.ab_dtype == GEMM_BF16, 0, 0, kSkinnyTileN, s.m_pad);
+  p.out_dtype = d.c_dtype;
+  p.epilogue = d.epilogue;
+  p.alpha = alpha;
+  p.beta = beta;
+  p.bias = bias;
+  p.c = C;
+  p.ldc = d.ldc;
+  p.partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + s.counters_bytes);
+  p.counters = reinterpret_cast<uint32_t*>(workspace);
+  p.status = pl->d_status;
+  p.timeout_ns = static_cast<unsigned long long>(pl->timeout_ms) * 1000000ull;
+  return static_cast<gemm_status_t>(skinny_launch(p, tW, tX, stream, g_last_cuda_error, sizeof g_last_cuda_error));
+}
+
+}  // namespace
+
+extern "C" gemm_status_t gemm_run(gemm_plan_t plan, const void* A, const void* B, void* C, const float* bias, float alpha,
+                                  float beta, void* workspace, size_t workspace_bytes, gemm_stream_t stream) {
+  if (!plan || !A || !B || !C) return GEMM_ERR_NULL;
+  if (has_bias(plan->d.epilogue) && !bias) return GEMM_ERR_NULL;
+  auto misaligned = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; };
+  if (misaligned(A) || misaligned(B) || misaligned(C) || (bias && misaligned(bias))) return GEMM_ERR_ALIGNMENT;
+  const size_t need = plan->info.workspace_bytes;
+  if (need > 0) {
+    if (!workspace || workspace_bytes < need) return GEMM_ERR_WORKSPACE;
+    if (misaligned(workspace)) return GEMM_ERR_ALIGNMENT;
+  }
+  if (!plan->has_device || !plan->arch_ok || !plan->d_status) return GEMM_ERR_ARCH;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (plan->variant == GEMM_VARIANT_SKINNY_STREAMK) return run_skinny(plan, A, B, C, bias, alpha, beta, workspace, s);
+  return run_dense(plan, A, B, C, bias, alpha, beta, s);
+}

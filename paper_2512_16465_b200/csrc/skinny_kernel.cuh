@@ -1,0 +1,301 @@
+// Skinny (memory-bound) GEMM for sm_100a: D[M x N] = act(alpha * X[M x K] * W[N x K]^T + beta * C + bias)
+// with a handful of rows M.  The whole cost is streaming W from HBM once, so the kernel is built
+// around the TMA stream, not around the tensor core:
+//
+//   * operands are swapped: a 128-row slab of W is the tcgen05.mma "A" operand (M_mma = 128), the
+//     activations X, zero-padded by TMA to m_pad rows, are the "B" operand (N_mma = m_pad >= 16);
+//     the accumulator is D^T: 128 TMEM lanes (output columns) x m_pad TMEM columns (output rows);
+//   * stream-K: the (n-tile, k-block) work units, n-tile major, are cut into `grid` equal contiguous
+//     ranges, one per CTA (one CTA per SM), so every SM streams the same number of bytes;
+//   * a CTA whose range covers only part of a tile's K writes its fp32 partial to the workspace and
+//     bumps the tile's arrival counter; the CTA that arrives last adds the partials in contributor
+//     order (deterministic, no floating-point atomics), applies the epilogue and writes D.
+//     Nobody ever waits for another CTA.
+//
+// Roles per CTA (192 threads): warp 0 lane 0 = TMA producer, warp 1 lane 0 = MMA issuer (warp 1 owns
+// the TMEM allocation), warps 2-5 = epilogue / fix-up.
+#pragma once
+#include <cuda_runtime.h>
+
+#include "dense_kernel.cuh"
+
+namespace b200 {
+
+constexpr int kSkinnyTileN = 128;   // output columns (rows of W) per tile = TMEM lanes
+constexpr int kSkinnyMaxM = 64;     // largest M the skinny path takes
+constexpr int kSkinnyThreads = 192;
+
+struct SkinnyPlan {
+  int m_pad;             // M rounded up to a multiple of 16 (the MMA's N extent)
+  int n_tiles;           // ceil(N / 128)
+  int kbs;               // k-blocks per tile = ceil(K / 64)
+  long long total_units; // n_tiles * kbs
+  int grid;              // CTAs = min(SM count, total_units)
+  int stages;
+  int stage_bytes;       // 16 KB of W + m_pad * 128 bytes of X
+  int smem_bytes;
+  int max_contributors;  // upper bound on CTAs touching one tile
+  size_t counters_bytes; // workspace: [counters (n_tiles x u32, padded)] [partials: grid * 2 slots]
+  size_t workspace_bytes;
+};
+
+// First work unit of CTA c, and the CTA that owns unit u, for T units over G CTAs.
+__host__ __device__ inline long long sk_begin(long long c, long long T, long long G) { return c * T / G; }
+__host__ __device__ inline int sk_owner(long long u, long long T, long long G) { return static_cast<int>(((u + 1) * G - 1) / T); }
+
+inline bool skinny_make_plan(SkinnyPlan* s, int M, int N, int K, int sm_count, int forced_stages, int max_smem) {
+  if (M < 1 || M > kSkinnyMaxM) return false;
+  s->m_pad = ((M + 15) / 16) * 16;
+  s->n_tiles = (N + kSkinnyTileN - 1) / kSkinnyTileN;
+  s->kbs = (K + kBlockK - 1) / kBlockK;
+  s->total_units = static_cast<long long>(s->n_tiles) * s->kbs;
+  s->grid = static_cast<int>(s->total_units < sm_count ? s->total_units : sm_count);
+  s->stage_bytes = kSkinnyTileN * 128 + s->m_pad * 128;
+  const int fixed = 1024 + 16 * kMaxStages + 64;
+  int stages = forced_stages ? forced_stages : (max_smem - fixed) / s->stage_bytes;
+  if (stages > kMaxStages) stages = kMaxStages;
+  if (stages < 2) return false;
+  s->stages = stages;
+  s->smem_bytes = fixed + stages * s->stage_bytes;
+  if (s->smem_bytes > max_smem) return false;
+  const long long per_cta = s->total_units / s->grid;  // >= 1
+  s->max_contributors = static_cast<int>((s->kbs + per_cta - 1) / per_cta + 1);
+  s->counters_bytes = (static_cast<size_t>(s->n_tiles) * 4 + 255) / 256 * 256;
+  s->workspace_bytes = s->counters_bytes + static_cast<size_t>(s->grid) * 2 * kSkinnyTileN * s->m_pad * 4;
+  return true;
+}
+
+struct SkinnyParams {
+  SkinnyPlan plan;
+  int M, N, K;
+  uint32_t idesc;
+  int out_dtype;
+  int epilogue;
+  float alpha, beta;
+  const float* bias;
+  void* c;                // D buffer (also C_in when beta != 0), row-major M x N
+  long long ldc;
+  float* partials;        // workspace: slot-major, each slot [m_pad][128] floats
+  uint32_t* counters;     // workspace: one arrival counter per n-tile, zero at launch
+  uint32_t* status;
+  unsigned long long timeout_ns;
+};
+
+__device__ __forceinline__ float sk_load_c(const SkinnyParams& p, long long idx) {
+  if (p.out_dtype == 2) return static_cast<const float*>(p.c)[idx];
+  if (p.out_dtype == 0) return __bfloat162float(static_cast<const __nv_bfloat16*>(p.c)[idx]);
+  return __half2float(static_cast<const __half*>(p.c)[idx]);
+}
+__device__ __forceinline__ void sk_store_d(const SkinnyParams& p, long long idx, float v) {
+  if (p.out_dtype == 2) static_cast<float*>(p.c)[idx] = v;
+  else if (p.out_dtype == 0) static_cast<__nv_bfloat16*>(p.c)[idx] = __float2bfloat16_rn(v);
+  else static_cast<__half*>(p.c)[idx] = __float2half_rn(v);
+}
+__device__ __forceinline__ void sk_finish(const SkinnyParams& p, int m, int n, float acc) {
+  const long long idx = static_cast<long long>(m) * p.ldc + n;
+  float v = p.alpha * acc;
+  if (p.beta != 0.0f) v += p.beta * sk_load_c(p, idx);
+  if (p.epilogue & 1) v += __ldg(p.bias + n);
+  if (p.epilogue == 2 || p.epilogue == 3) v = fmaxf(v, 0.0f);
+  else if (p.epilogue >= 4) v = gelu_erf(v);
+  sk_store_d(p, idx, v);
+}
+
+__global__ void __launch_bounds__(kSkinnyThreads, 1)
+skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, const SkinnyParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_addr(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* gen = smem_raw + (base - raw);
+  const uint32_t warp = threadIdx.x >> 5;
+  const uint32_t lane = lane_id();
+  const SkinnyPlan& sp = p.plan;
+
+  const uint32_t bars_off = static_cast<uint32_t>(sp.stages) * sp.stage_bytes;
+  const uint32_t full0 = base + bars_off;
+  const uint32_t empty0 = full0 + 8u * kMaxStages;
+  const uint32_t tfull0 = empty0 + 8u * kMaxStages;
+  const uint32_t tempty0 = tfull0 + 16u;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + bars_off + 16u * kMaxStages + 32u);
+  volatile uint32_t* s_abort = tmem_slot + 1;
+  volatile uint32_t* s_last = tmem_slot + 2;
+  const WaitCtx w{s_abort, p.status, p.timeout_ns};
+  const uint32_t tmem_cols = sp.m_pad * 2 <= 32 ? 32u : (sp.m_pad * 2 <= 64 ? 64u : 128u);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < sp.stages; ++s) {
+      mbar_init(full0 + 8u * s, 1);
+      mbar_init(empty0 + 8u * s, 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(tfull0 + 8u * b, 1);
+      mbar_init(tempty0 + 8u * b, 4);
+    }
+    *s_abort = 0u;
+    fence_mbar_init();
+    prefetch_tensormap(&tmW);
+    prefetch_tensormap(&tmX);
+  }
+  if (warp == 1) {
+    tmem_alloc<1>(smem_addr(const_cast<uint32_t*>(tmem_slot)), tmem_cols);
+    tmem_relinquish<1>();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const long long T = sp.total_units, G = gridDim.x;
+  const long long u_begin = sk_begin(blockIdx.x, T, G);
+  const long long u_end = sk_begin(blockIdx.x + 1, T, G);
+
+  if (warp == 0) {
+    if (lane == 0) {
+      uint32_t kc = 0;
+      for (long long u = u_begin; u < u_end; ++u, ++kc) {
+        const int tile = static_cast<int>(u / sp.kbs);
+        const int kb = static_cast<int>(u - static_cast<long long>(tile) * sp.kbs);
+        const uint32_t s = kc % static_cast<uint32_t>(sp.stages);
+        const uint32_t ph = (kc / static_cast<uint32_t>(sp.stages)) & 1u;
+        if (!mbar_wait(empty0 + 8u * s, ph ^ 1u, w, (1u << 8) | s)) break;
+        mbar_arrive_expect_tx(full0 + 8u * s, sp.stage_bytes);
+        const uint32_t sw_ = base + s * sp.stage_bytes;
+        tma_load_3d(sw_, &tmW, full0 + 8u * s, kb * kBlockK, tile * kSkinnyTileN, 0);
+        tma_load_3d(sw_ + kSkinnyTileN * 128u, &tmX, full0 + 8u * s, kb * kBlockK, 0, 0);
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint64_t desc_hi = make_smem_desc_hi(16, 1024);
+      uint32_t kc = 0, seg = 0;
+      long long u = u_begin;
+      bool ok = true;
+      while (ok && u < u_end) {
+        const long long tile = u / sp.kbs;
+        const long long seg_end = min(u_end, (tile + 1) * sp.kbs);
+        const uint32_t buf = seg & 1u;
+        if (!mbar_wait(tempty0 + 8u * buf, ((seg >> 1) & 1u) ^ 1u, w, (2u << 8) | 0x80u | buf)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * static_cast<uint32_t>(sp.m_pad);
+        for (long long uu = u; uu < seg_end; ++uu, ++kc) {
+          const uint32_t s = kc % static_cast<uint32_t>(sp.stages);
+          const uint32_t ph = (kc / static_cast<uint32_t>(sp.stages)) & 1u;
+          if (!mbar_wait(full0 + 8u * s, ph, w, (2u << 8) | s)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t sw_ = base + s * sp.stage_bytes;
+          const uint32_t sx = sw_ + kSkinnyTileN * 128u;
+#pragma unroll
+          for (int k = 0; k < kBlockK / kUmmaK; ++k)
+            umma_f16<1>(d_tmem, smem_desc(desc_hi, sw_ + k * 32u), smem_desc(desc_hi, sx + k * 32u), p.idesc,
+                        static_cast<uint32_t>(uu != u || k != 0));
+          umma_commit<1>(empty0 + 8u * s);
+        }
+        if (ok) umma_commit<1>(tfull0 + 8u * buf);
+        u = seg_end;
+        ++seg;
+      }
+    }
+    __syncwarp();
+  } else {
+    const uint32_t q = warp & 3u;
+    const int n_local = static_cast<int>(q * 32u + lane);
+    const bool leader = (warp == 2 && lane == 0);
+    uint32_t seg = 0;
+    long long u = u_begin;
+    while (u < u_end) {
+      const long long tile = u / sp.kbs;
+      const long long tile_u0 = tile * sp.kbs;
+      const long long seg_end = min(u_end, tile_u0 + sp.kbs);
+      const uint32_t buf = seg & 1u;
+      if (!mbar_wait(tfull0 + 8u * buf, (seg >> 1) & 1u, w, (3u << 8) | buf)) break;
+      tc_fence_after();
+      const int n = static_cast<int>(tile) * kSkinnyTileN + n_local;
+      const bool whole = (u == tile_u0) && (seg_end == tile_u0 + sp.kbs);  // this CTA owns the tile's whole K
+      const uint32_t t_row = tmem_base + ((q * 32u) << 16) + buf * static_cast<uint32_t>(sp.m_pad);
+      float* my_partial = p.partials + (static_cast<size_t>(blockIdx.x) * 2 + (seg == 0 ? 0 : 1)) * (kSkinnyTileN * sp.m_pad);
+      for (int c0 = 0; c0 < sp.m_pad; c0 += 16) {
+        uint32_t acc[16];
+        tmem_ld_32x16(t_row + static_cast<uint32_t>(c0), acc);
+        tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const int m = c0 + j;
+          if (m < p.M) {
+            if (whole) {
+              if (n < p.N) sk_finish(p, m, n, __uint_as_float(acc[j]));
+            } else {
+              my_partial[m * kSkinnyTileN + n_local] = __uint_as_float(acc[j]);
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty0 + 8u * buf);
+      if (!whole) {
+        // publish the partial, then count arrivals; the last contributor reduces
+        const int c_first = sk_owner(tile_u0, T, G);
+        const int c_last = sk_owner(tile_u0 + sp.kbs - 1, T, G);
+        __threadfence();
+        named_barrier_sync(1, 128);
+        if (leader) {
+          const uint32_t old = atomicAdd(p.counters + tile, 1u);
+          *s_last = (old == static_cast<uint32_t>(c_last - c_first)) ? 1u : 0u;
+        }
+        named_barrier_sync(1, 128);
+        const bool last = *s_last != 0u;
+        if (last) {
+          __threadfence();
+          for (int m = 0; m < p.M; ++m) {
+            float sum = 0.0f;
+            for (int c = c_first; c <= c_last; ++c) {
+              const int slot = (sk_begin(c, T, G) / sp.kbs == tile) ? 0 : 1;  // tile is c's first segment?
+              const float* part = p.partials + (static_cast<size_t>(c) * 2 + slot) * (kSkinnyTileN * sp.m_pad);
+              sum += __ldcg(part + m * kSkinnyTileN + n_local);
+            }
+            if (n < p.N) sk_finish(p, m, n, sum);
+          }
+          if (leader) p.counters[tile] = 0u;  // leave the counter clean for the next launch
+        }
+        named_barrier_sync(1, 128);  // s_last is reused by the next segment
+      }
+      u = seg_end;
+      ++seg;
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc<1>(tmem_base, tmem_cols);
+  }
+}
+
+// Zero the arrival counters and launch.  Returns a gemm_status_t value (0 = ok, 7 = CUDA failure).
+inline int skinny_launch(const SkinnyParams& p, const CUtensorMap& tW, const CUtensorMap& tX, cudaStream_t stream, char* err,
+                         size_t err_len) {
+  static thread_local int configured_smem = 0;
+  cudaError_t e = cudaSuccess;
+  if (configured_smem < p.plan.smem_bytes) {
+    e = cudaFuncSetAttribute(skinny_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, p.plan.smem_bytes);
+    if (e == cudaSuccess) configured_smem = p.plan.smem_bytes;
+  }
+  if (e == cudaSuccess) e = cudaMemsetAsync(p.counters, 0, p.plan.counters_bytes, stream);
+  if (e == cudaSuccess) {
+    skinny_gemm_kernel<<<p.plan.grid, kSkinnyThreads, p.plan.smem_bytes, stream>>>(tW, tX, p);
+    e = cudaGetLastError();
+  }
+  if (e != cudaSuccess) {
+    snprintf(err, err_len, "skinny launch: %s", cudaGetErrorName(e));
+    (void)cudaGetLastError();
+    return 7;
+  }
+  return 0;
+}
+
+}  // namespace b200

@@ -1,0 +1,161 @@
+"""Shared plumbing of the GPU parity tests: upload a seeded workload, run it through the
+C-ABI binding, evaluate the oracle on the checked rows / columns and compare.
+
+Acceptance (per checked element, against the UNROUNDED fp64 oracle value y):
+    |D_gpu - y| <= 2e-3 * (|alpha| * sum_k |a||b| + |beta| * |C_in| + |bias_j|) + 1e-5
+and, over each checked block, the relative Frobenius error
+    ||D_gpu - ref||_F / ||ref||_F <= 1e-4
+where ref = y for fp32 output and ref = RNE(y -> output dtype) for 16-bit outputs (rounding
+y to bf16 alone moves it by ~1.7e-3 relative, fp16 by ~2e-4, so the 1e-4 bar can only be
+applied against the rounded oracle there; the accumulator itself is held to 1e-4 against
+y by re-running the same plan with fp32 output).
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle
+import paper_2512_16465_b200 as bg
+import workloads as wl
+
+REL_TOL, ABS_TOL, FROB_TOL = 2e-3, 1e-5, 1e-4
+_TORCH_DT = {wl.BF16: torch.bfloat16, wl.F16: torch.float16, wl.F32: torch.float32}
+
+
+def to_device(arr: np.ndarray, dtype: int) -> torch.Tensor:
+    if dtype == wl.F32:
+        return torch.from_numpy(arr).cuda()
+    return torch.from_numpy(arr.view(np.int16)).cuda().view(_TORCH_DT[dtype])
+
+
+def to_host_bits(t: torch.Tensor, dtype: int) -> np.ndarray:
+    if dtype == wl.F32:
+        return t.cpu().numpy()
+    return t.view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def desc_of(w: wl.Workload, flags: int = 0, c_dtype=None) -> bg.Desc:
+    cd = w.c_dtype if c_dtype is None else c_dtype
+    return bg.make_desc(w.M, w.N, w.K, w.transa, w.transb, w.ab_dtype, cd, w.lda, w.ldb, w.ldc, w.batch,
+                        w.stride_a, w.stride_b, w.stride_c, w.epilogue, flags)
+
+
+def problem_of(w: wl.Workload, c_dtype=None) -> oracle.Problem:
+    cd = w.c_dtype if c_dtype is None else c_dtype
+    return oracle.Problem(w.M, w.N, w.K, w.transa, w.transb, w.ab_dtype, cd, w.lda, w.ldb, w.ldc, w.batch,
+                          w.stride_a, w.stride_b, w.stride_c, w.epilogue)
+
+
+def c_in_as(inputs: dict, w: wl.Workload, c_dtype: int):
+    """C_in converted to another output dtype (for the fp32-output re-run of a 16-bit config)."""
+    c = inputs["C"]
+    if c is None or c_dtype == w.c_dtype:
+        return c
+    vals = oracle.decode(c, w.c_dtype)
+    return oracle.round_to(vals, c_dtype)
+
+
+def run_gpu(w: wl.Workload, inputs: dict, flags: int = 0, c_dtype=None, poison: bool = True, repeats: int = 1):
+    """Run the workload through the binding; returns (host bit array of the whole C buffer, plan info)."""
+    cd = w.c_dtype if c_dtype is None else c_dtype
+    plan = bg.Plan(desc_of(w, flags, cd))
+    try:
+        A = to_device(inputs["A"], w.ab_dtype)
+        B = to_device(inputs["B"], w.ab_dtype)
+        bias = None if inputs["bias"] is None else to_device(inputs["bias"], wl.F32)
+        cin = c_in_as(inputs, w, cd)
+        outs = []
+        for _ in range(repeats):
+            if cin is not None:
+                C = to_device(cin, cd).clone()
+            else:
+                C = torch.empty(w.elems_c(), dtype=_TORCH_DT[cd], device="cuda")
+                if poison:   # beta == 0 must never read C: NaN would propagate
+                    C.fill_(float("nan"))
+            plan.run(A, B, C, bias, w.alpha, w.beta)
+            torch.cuda.synchronize()
+            st = plan.status()
+            if st != bg.OK:
+                raise bg.GemmError(st, "gemm_plan_status")
+            outs.append(to_host_bits(C, cd))
+        for o in outs[1:]:
+            assert np.array_equal(o, outs[0]), "run-to-run results differ bitwise"
+        return outs[0], plan.info
+    finally:
+        plan.close()
+
+
+def gather(cbits: np.ndarray, w: wl.Workload, batches, rows, cols) -> np.ndarray:
+    idx = (np.asarray(batches)[:, None, None] * w.stride_c + np.asarray(rows)[None, :, None] * w.ldc +
+           np.asarray(cols)[None, None, :])
+    return cbits[idx]
+
+
+def compare_block(got_bits: np.ndarray, y: np.ndarray, bound: np.ndarray, c_dtype: int) -> dict:
+    got = oracle.decode(got_bits, c_dtype)
+    err = np.abs(got - y)
+    tol = REL_TOL * bound + ABS_TOL
+    ref_bits = oracle.round_to(y, c_dtype)
+    ref = oracle.decode(ref_bits, c_dtype) if c_dtype != wl.F32 else y
+    denom = float(np.linalg.norm(ref.ravel()))
+    frob = float(np.linalg.norm((got - ref).ravel())) / max(denom, 1e-300)
+    frob_unrounded = float(np.linalg.norm((got - y).ravel())) / max(float(np.linalg.norm(y.ravel())), 1e-300)
+    exact = float(np.mean(got_bits == ref_bits))
+    finite = bool(np.all(np.isfinite(got)))
+    worst = float(np.max(err / tol)) if err.size else 0.0
+    return {"max_err_over_tol": worst, "frob": frob, "frob_unrounded": frob_unrounded, "bit_identical": exact,
+            "finite": finite, "n": int(err.size), "argmax": np.unravel_index(int(np.argmax(err / tol)), err.shape) if err.size else None}
+
+
+def check_blocks(w: wl.Workload, inputs: dict, cbits: np.ndarray, blocks, c_dtype=None) -> list:
+    """blocks: list of (batches, rows, cols) index arrays.  Returns one report per block."""
+    cd = w.c_dtype if c_dtype is None else c_dtype
+    p = problem_of(w, cd)
+    cin = c_in_as(inputs, w, cd)
+    reports = []
+    for batches, rows, cols in blocks:
+        y, bound = oracle.gemm(p, inputs["A"], inputs["B"], C_in=cin, bias=inputs["bias"], alpha=w.alpha, beta=w.beta,
+                               batches=batches, rows=rows, cols=cols)
+        reports.append(compare_block(gather(cbits, w, batches, rows, cols), y, bound, cd))
+    return reports
+
+
+def default_blocks(w: wl.Workload) -> list:
+    """Everything for small problems; seeded rows x all columns and all rows x seeded columns
+    (plus whole batches where the config asks) for the large ones."""
+    allb = np.arange(w.batch, dtype=np.int64)
+    allr = np.arange(w.M, dtype=np.int64)
+    allc = np.arange(w.N, dtype=np.int64)
+    if not w.sample_rows and not w.sample_cols:
+        return [(allb, allr, allc)]
+    blocks = []
+    if w.full_batches:
+        fb = sorted(set([0, w.batch - 1] + wl.sample_indices(w.batch, w.full_batches, w.seed, 3)[:w.full_batches].tolist()))
+        fb = fb[:max(w.full_batches, 2)]
+        blocks.append((np.array(fb, dtype=np.int64), allr, allc))
+    rows = wl.sample_indices(w.M, w.sample_rows, w.seed, 1)
+    cols = wl.sample_indices(w.N, w.sample_cols, w.seed, 2)
+    blocks.append((allb, rows, allc))
+    blocks.append((allb, allr, cols))
+    return blocks
+
+
+def assert_reports(reports, frob_tol=FROB_TOL, what=""):
+    for r in reports:
+        assert r["finite"], f"{what}: non-finite output {r}"
+        assert r["max_err_over_tol"] <= 1.0, f"{what}: per-element tolerance exceeded {r}"
+        assert r["frob"] <= frob_tol, f"{what}: Frobenius error {r}"
+
+
+def check_workload(w: wl.Workload, flags: int = 0, exact: bool = False, c_dtype=None, repeats: int = 1, inputs=None):
+    """Run + compare.  exact=True additionally requires bit equality with the rounded oracle
+    (for integer-valued inputs whose every partial sum is exactly representable)."""
+    inputs = wl.make_inputs(w) if inputs is None else inputs
+    cbits, info = run_gpu(w, inputs, flags, c_dtype, repeats=repeats)
+    reports = check_blocks(w, inputs, cbits, default_blocks(w), c_dtype)
+    assert_reports(reports, what=w.name)
+    if exact:
+        for r in reports:
+            assert r["bit_identical"] == 1.0, f"{w.name}: not bit-exact {r} {info}"
+    return reports, info
