@@ -1,0 +1,408 @@
+#!/usr/bin/env python
+"""Benchmark of the b200 GEMM hot path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config c1..c5]
+
+A step is one pass of the whole hot path (plan already made; tensor-map encode, tile scheduling,
+TMA/tcgen05 main loop, epilogue) over one batch of synthetic input.  The headline workload is
+config c2 (8192^3 bf16, A row-major, B column-major, bf16 output), the configuration the
+metric is quoted on; ``--all`` (default on) adds one entry per benchmark configuration under
+``configs_measured``.  Prints ONE JSON line on rank 0.
+
+Timing: CUDA events on the launching stream around K back-to-back steps, after W >= 3 warm-up
+steps; inputs rotate through enough seeded buffer sets to exceed twice the L2 capacity, so no
+step finds its operands in cache.  ``e2e`` repeats the measurement with host-resident pinned
+inputs and output: every step copies A and B to the device, runs the GEMM and copies D back.
+
+``--impl reference`` times the CPU oracle (the fp64 triple loop) on a bounded sample of the same
+workload; it is a deliberately slow program and only a reported baseline.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+import workloads as wl  # noqa: E402
+
+L2_BYTES = 126 * 1024 * 1024
+NOMINAL = {"tensor_tflops": 2250.0, "hbm_gbs": 8000.0}
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
+# summarised under profiles/ (file named there); None until a capture exists for the config.
+NCU_TRAFFIC_BYTES = {"c1": None, "c2": None, "c3": None, "c4": None, "c5": None}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"]))}, "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.index, self.samples, self.reasons, self.max_mhz = index, [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {nv.nvmlClocksThrottleReasonSwPowerCap: "sw_power_cap",
+                 nv.nvmlClocksThrottleReasonHwSlowdown: "hw_slowdown",
+                 nv.nvmlClocksThrottleReasonHwThermalSlowdown: "hw_thermal_slowdown",
+                 nv.nvmlClocksThrottleReasonSwThermalSlowdown: "sw_thermal_slowdown"}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.005)
+
+    def __enter__(self):
+        if self.nv:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+
+    def summary(self):
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def roofline_for(w: wl.Workload, key: str, seconds: float, peaks: dict, peak_kind: str) -> dict:
+    """Roofline entry of the step's single kernel: the bound is whichever of (flops / tensor peak)
+    and (compulsory bytes / HBM bandwidth) is slower."""
+    t_tensor = w.flops / (peaks["bf16_tflops"] * 1e12)
+    t_hbm = w.min_bytes / (peaks["hbm_gbs"] * 1e9)
+    if t_tensor >= t_hbm:
+        achieved, peak, unit, bound = w.flops / seconds / 1e12, peaks["bf16_tflops"], "TFLOP/s", "tensor"
+    else:
+        achieved, peak, unit, bound = w.min_bytes / seconds / 1e9, peaks["hbm_gbs"], "GB/s", "hbm"
+    return {"bound": bound, "achieved": round(achieved, 2), "peak": peak, "unit": unit, "frac": round(achieved / peak, 4),
+            "traffic": NCU_TRAFFIC_BYTES.get(key), "peak_source": f"of {peak_kind}",
+            "frac_of_nominal": round(achieved / (NOMINAL["tensor_tflops"] if bound == "tensor" else NOMINAL["hbm_gbs"]), 4),
+            "algorithmic_flops": w.flops, "algorithmic_bytes": w.min_bytes}
+
+
+# --------------------------------------------------------------------------- our arm
+
+def _torch_dt(torch, code):
+    return {wl.BF16: torch.bfloat16, wl.F16: torch.float16, wl.F32: torch.float32}[code]
+
+
+def _to_torch(torch, arr, code, device=None, pin=False):
+    t = torch.from_numpy(arr) if code == wl.F32 else torch.from_numpy(arr.view(np.int16)).view(_torch_dt(torch, code))
+    if pin:
+        t = t.pin_memory()
+    return t.to(device) if device is not None else t
+
+
+class DeviceCase:
+    """One benchmark configuration resident in HBM: R rotating input sets and a plan."""
+
+    def __init__(self, torch, bg, key: str, w: wl.Workload, flags: int, device):
+        self.torch, self.bg, self.key, self.w, self.device = torch, bg, key, w, device
+        footprint = w.min_bytes
+        self.nsets = int(max(1, min(160, -(-2 * L2_BYTES // int(footprint))))) if footprint < 2 * L2_BYTES else 1
+        self.sets = []
+        for r in range(self.nsets):
+            inp = wl.make_inputs(w, seed_offset=1000 * r)
+            A = _to_torch(torch, inp["A"], w.ab_dtype, device)
+            B = _to_torch(torch, inp["B"], w.ab_dtype, device)
+            if inp["C"] is not None:
+                C = _to_torch(torch, inp["C"], w.c_dtype, device)
+            else:
+                C = torch.empty(w.elems_c(), dtype=_torch_dt(torch, w.c_dtype), device=device)
+            bias = None if inp["bias"] is None else _to_torch(torch, inp["bias"], wl.F32, device)
+            self.sets.append((A, B, C, bias))
+            if r == 0:
+                self.host_inputs = inp
+        d = bg.make_desc(w.M, w.N, w.K, w.transa, w.transb, w.ab_dtype, w.c_dtype, w.lda, w.ldb, w.ldc, w.batch,
+                         w.stride_a, w.stride_b, w.stride_c, w.epilogue, flags)
+        self.plan = bg.Plan(d)
+        self.plan.workspace(device)
+        self.i = 0
+
+    def step(self):
+        A, B, C, bias = self.sets[self.i % self.nsets]
+        self.i += 1
+        self.plan.run(A, B, C, bias, self.w.alpha, self.w.beta)
+
+    def time_steps(self, steps: int, warmup: int) -> float:
+        """Seconds per step over `steps` back-to-back steps (CUDA events on the launching stream)."""
+        torch = self.torch
+        for _ in range(warmup):
+            self.step()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            self.step()
+        e1.record()
+        torch.cuda.synchronize()
+        st = self.plan.status()
+        if st != self.bg.OK:
+            raise RuntimeError(f"device status {self.bg.status_string(st)} after timing {self.key}")
+        return e0.elapsed_time(e1) * 1e-3 / steps
+
+    def time_e2e(self, steps: int, warmup: int):
+        """Same metric with host-resident inputs and output: H2D of A, B (and C_in, bias), the GEMM,
+        D2H of D, every step.  Returns (seconds per step, h2d bytes, d2h bytes)."""
+        torch, w = self.torch, self.w
+        inp = self.host_inputs
+        hA = _to_torch(torch, inp["A"], w.ab_dtype, pin=True)
+        hB = _to_torch(torch, inp["B"], w.ab_dtype, pin=True)
+        hC = None if inp["C"] is None else _to_torch(torch, inp["C"], w.c_dtype, pin=True)
+        hbias = None if inp["bias"] is None else _to_torch(torch, inp["bias"], wl.F32, pin=True)
+        A, B, C, bias = self.sets[0]
+        hD = torch.empty(C.shape, dtype=C.dtype).pin_memory()
+        h2d = hA.numel() * hA.element_size() + hB.numel() * hB.element_size()
+        h2d += 0 if hC is None else hC.numel() * hC.element_size()
+        h2d += 0 if hbias is None else hbias.numel() * 4
+        d2h = hD.numel() * hD.element_size()
+
+        def one():
+            A.copy_(hA, non_blocking=True)
+            B.copy_(hB, non_blocking=True)
+            if hC is not None:
+                C.copy_(hC, non_blocking=True)
+            if hbias is not None:
+                bias.copy_(hbias, non_blocking=True)
+            self.plan.run(A, B, C, bias, w.alpha, w.beta)
+            hD.copy_(C, non_blocking=True)
+
+        for _ in range(warmup):
+            one()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            one()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e-3 / steps, h2d, d2h
+
+    def close(self):
+        self.plan.close()
+        self.sets = []
+
+
+def metric_value(w: wl.Workload, seconds: float) -> float:
+    return w.flops / seconds / 1e12
+
+
+def time_oracle_sample(w: wl.Workload, inputs: dict, target_seconds: float):
+    """Time the oracle, as it stands, on the first rows of batch 0 of the workload; the row count
+    is calibrated so the run takes about `target_seconds`.  Returns (TFLOP/s, cores, description)."""
+    import oracle
+    p = oracle.Problem(w.M, w.N, w.K, w.transa, w.transb, w.ab_dtype, w.c_dtype, w.lda, w.ldb, w.ldc, w.batch,
+                       w.stride_a, w.stride_b, w.stride_c, w.epilogue)
+    cores = oracle.max_threads()
+    cols = np.arange(w.N, dtype=np.int64)
+
+    def run(nrows):
+        rows = np.arange(nrows, dtype=np.int64)
+        t0 = time.perf_counter()
+        oracle.gemm(p, inputs["A"], inputs["B"], C_in=inputs["C"], bias=inputs["bias"], alpha=w.alpha, beta=w.beta,
+                    batches=[0], rows=rows, cols=cols)
+        return time.perf_counter() - t0
+
+    probe_rows = min(w.M, 2)
+    t_probe = max(run(probe_rows), 1e-4)
+    nrows = int(max(probe_rows, min(w.M, round(probe_rows * target_seconds / t_probe))))
+    t = run(nrows)
+    flops = 2.0 * nrows * w.N * w.K
+    return flops / t / 1e12, cores, f"rows 0..{nrows - 1} x all {w.N} columns of batch 0 ({flops / 1e9:.1f} GFLOP in {t:.1f} s)"
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2512_16465_b200 as bg
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+    peaks, peak_kind = load_peaks()
+    cfgs = wl.configs()
+    flags = int(args.flags, 0)
+    steps, warmup = args.steps, max(3, args.warmup)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    key = args.config
+    w = cfgs[key]
+    case = DeviceCase(torch, bg, key, w, flags, device)
+    barrier()
+    with ClockSampler(local_rank) as clocks:
+        sec = case.time_steps(steps, warmup)
+        barrier()
+    sec = max_over_ranks(sec)
+    e2e_steps = max(2, min(steps, args.e2e_steps))
+    barrier()
+    if args.e2e_steps > 0:
+        e2e_sec, h2d, d2h = case.time_e2e(e2e_steps, 2)
+    else:  # profiling runs skip the host-buffer leg
+        e2e_sec, h2d, d2h = float("nan"), 0, 0
+    barrier()
+    e2e_sec = max_over_ranks(e2e_sec)
+
+    out = {
+        "metric": "GEMM TFLOP/s at 1 B200 and % of dense bf16 roofline (HBM GB/s for skinny)",
+        "value": round(metric_value(w, sec) * world, 2), "unit": "TFLOP/s", "n_gpus": world, "steps": steps, "warmup": warmup,
+        "ms_per_step": round(sec * 1e3, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 x bf16 -> fp32 accumulate", "data": "synthetic",
+        "config": {"workload": w.name, "M": w.M, "N": w.N, "K": w.K, "batch": w.batch,
+                   "layout": "A row-major, B stored N x K", "out_dtype": ["bf16", "f16", "f32"][w.c_dtype],
+                   "l2": f"inputs larger than L2: {case.nsets} rotating seeded input set(s), {w.min_bytes / 1e6:.0f} MB each",
+                   "multi_gpu": "replicas only (independent GEMMs, no collective)", "plan": case.plan.info},
+        "e2e": None if args.e2e_steps <= 0 else {"value": round(metric_value(w, e2e_sec) * world, 3), "unit": "TFLOP/s", "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": round(e2e_sec * 1e3, 3), "steps": e2e_steps},
+        "gpu_launches": steps,
+        "clocks": clocks.summary(),
+        "roofline": roofline_for(w, key, sec, peaks, peak_kind),
+    }
+    out["roofline"]["frac_of_sustained_peak"] = round(metric_value(w, sec) / peaks["bf16_tflops_sustained"], 4)
+    host_inputs = case.host_inputs
+    case.close()
+
+    if args.all:
+        measured = []
+        for k2, w2 in cfgs.items():
+            if k2 == key:
+                measured.append({"config": k2, "workload": w2.name, "ms_per_step": out["ms_per_step"], "tflops": out["value"] / world,
+                                 "roofline": out["roofline"]})
+                continue
+            c2 = DeviceCase(torch, bg, k2, w2, 0, device)
+            s2 = max_over_ranks(c2.time_steps(steps, warmup))
+            measured.append({"config": k2, "workload": w2.name, "ms_per_step": round(s2 * 1e3, 5),
+                             "tflops": round(metric_value(w2, s2), 2), "gbs": round(w2.min_bytes / s2 / 1e9, 1),
+                             "input_sets": c2.nsets, "plan": c2.plan.info, "roofline": roofline_for(w2, k2, s2, peaks, peak_kind)})
+            c2.close()
+        out["configs_measured"] = measured
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, cores, sample = time_oracle_sample(w, host_inputs, args.cpu_seconds)
+        out["cpu_baseline"] = {"value": round(v, 6), "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample}
+    if rank == 0:
+        print(json.dumps(out), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_reference(args):
+    """The reference arm of this build is the CPU oracle: K steps, each a bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    w = wl.configs()[args.config]
+    inputs = wl.make_inputs(w)
+    steps, warmup = args.steps, args.warmup
+    # size each step so that the whole run stays within a few minutes
+    per_step = max(0.5, min(10.0, 120.0 / max(1, steps + warmup)))
+    p = oracle.Problem(w.M, w.N, w.K, w.transa, w.transb, w.ab_dtype, w.c_dtype, w.lda, w.ldb, w.ldc, w.batch,
+                       w.stride_a, w.stride_b, w.stride_c, w.epilogue)
+    cols = np.arange(w.N, dtype=np.int64)
+
+    def run(nrows):
+        t0 = time.perf_counter()
+        oracle.gemm(p, inputs["A"], inputs["B"], C_in=inputs["C"], bias=inputs["bias"], alpha=w.alpha, beta=w.beta,
+                    batches=[0], rows=np.arange(nrows, dtype=np.int64), cols=cols)
+        return time.perf_counter() - t0
+
+    t1 = max(run(1), 1e-4)
+    nrows = int(max(1, min(w.M, round(per_step / t1))))
+    for _ in range(warmup):
+        run(nrows)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        run(nrows)
+    sec = (time.perf_counter() - t0) / steps
+    flops = 2.0 * nrows * w.N * w.K
+    v = flops / sec / 1e12
+    cores = oracle.max_threads()
+    sample = f"each step: rows 0..{nrows - 1} x all {w.N} columns of batch 0 ({flops / 1e9:.2f} GFLOP)"
+    print(json.dumps({
+        "impl": "reference", "metric": "GEMM TFLOP/s at 1 B200 and % of dense bf16 roofline (HBM GB/s for skinny)",
+        "value": round(v, 6), "unit": "TFLOP/s", "n_gpus": args.gpus, "steps": steps, "warmup": warmup,
+        "ms_per_step": round(sec * 1e3, 3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "M": w.M, "N": w.N, "K": w.K, "batch": w.batch, "sample": sample},
+        "cpu_baseline": {"value": round(v, 6), "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": round(v, 6), "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--config", default="c2", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--flags", default="0", help="gemm_desc_t.flags override for the headline config (tuning)")
+    ap.add_argument("--all", dest="all", action="store_true", default=True)
+    ap.add_argument("--only", dest="all", action="store_false", help="time only --config (used for profiling)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,252 @@
+"""GPU parity tests: the CUDA path, called through the C-ABI binding, against the CPU oracle
+on the same seeded inputs.  Run with ``-m gpu`` on a B200."""
+import numpy as np
+import pytest
+import torch
+
+import harness as H
+import oracle
+import paper_2512_16465_b200 as bg
+import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+INT = wl.Dist("integer", -4, 4)
+V1, V2, VS = bg.VARIANT_DENSE_1CTA, bg.VARIANT_DENSE_2CTA, bg.VARIANT_SKINNY_STREAMK
+
+
+def int_workload(name, M, N, K, ta=0, tb=1, ab=wl.BF16, cd=wl.F32, batch=1, epi=0, alpha=1.0, beta=0.0, **kw):
+    """Integer-valued inputs in [-4, 4]: every product and partial sum is an exactly representable
+    integer (< 2^24), so fp32 accumulation is exact in any order and the result must be bit-identical."""
+    return wl.Workload(name, M, N, K, transa=ta, transb=tb, ab_dtype=ab, c_dtype=cd, batch=batch, epilogue=epi,
+                       alpha=alpha, beta=beta, dist_a=INT, dist_b=INT, dist_c=INT, dist_bias=INT, seed=4242, **kw)
+
+
+# ----------------------------------------------------------------------------- exact regime
+
+EXACT_CASES = [
+    # name, M, N, K, kwargs, flags
+    ("one_tile", 128, 128, 64, {}, dict(variant=V1, tile_n=128)),
+    ("one_kblock_ragged_k", 128, 64, 40, {}, dict(variant=V1, tile_n=64)),
+    ("tile_n_256", 256, 512, 192, {}, dict(variant=V1, tile_n=256)),
+    ("tile_n_192", 256, 576, 192, {}, dict(variant=V1, tile_n=192)),
+    ("ragged_all", 200, 328, 200, {}, dict(variant=V1, tile_n=128)),
+    ("tiny", 1, 8, 8, {}, dict(variant=V1)),
+    ("m1_n_ragged", 1, 1000, 72, {}, dict(variant=V1)),
+    ("n_small", 300, 8, 136, {}, dict(variant=V1)),
+    ("persistent_many_tiles", 1536, 2560, 128, {}, dict(variant=V1, tile_n=64)),
+    ("raster_1", 1024, 1024, 64, {}, dict(variant=V1, tile_n=128, raster=1)),
+    ("raster_3", 1100, 1024, 64, {}, dict(variant=V1, tile_n=128, raster=3)),
+    ("stages_2", 256, 256, 1024, {}, dict(variant=V1, tile_n=128, stages=2)),
+    ("stages_3_long_k", 128, 256, 8192, {}, dict(variant=V1, tile_n=256, stages=3)),
+    ("nn", 264, 328, 200, dict(ta=0, tb=0), dict(variant=V1, tile_n=128)),
+    ("nn_wide", 256, 512, 128, dict(ta=0, tb=0), dict(variant=V1, tile_n=256)),
+    ("tn", 264, 328, 200, dict(ta=1, tb=1), dict(variant=V1, tile_n=128)),
+    ("tt", 264, 328, 200, dict(ta=1, tb=0), dict(variant=V1, tile_n=64)),
+    ("f16_in_f16_out", 200, 328, 136, dict(ab=wl.F16, cd=wl.F16), dict(variant=V1)),
+    ("bf16_out", 200, 328, 136, dict(cd=wl.BF16), dict(variant=V1)),
+    ("f16_in_f32_out", 200, 328, 136, dict(ab=wl.F16), dict(variant=V1)),
+    ("alpha_beta_f32", 200, 328, 136, dict(alpha=0.5, beta=2.0), dict(variant=V1)),
+    ("beta_bf16_c", 200, 328, 136, dict(cd=wl.BF16, beta=1.0), dict(variant=V1)),
+    ("beta_f16_c", 200, 328, 136, dict(ab=wl.F16, cd=wl.F16, beta=-1.0), dict(variant=V1)),
+    ("bias", 200, 328, 136, dict(epi=bg.EPI_BIAS), dict(variant=V1)),
+    ("relu", 200, 328, 136, dict(epi=bg.EPI_RELU, cd=wl.BF16), dict(variant=V1)),
+    ("bias_relu_beta", 200, 328, 136, dict(epi=bg.EPI_BIAS_RELU, beta=1.0, alpha=2.0), dict(variant=V1)),
+    ("batched_tight", 200, 328, 72, dict(batch=5, ab=wl.F16, cd=wl.F16, alpha=0.25), dict(variant=V1)),
+    ("batched_nn", 136, 200, 72, dict(batch=3, ta=0, tb=0), dict(variant=V1)),
+    ("pair_one_tile", 256, 128, 64, {}, dict(variant=V2, tile_n=128)),
+    ("pair_256x256", 512, 512, 256, {}, dict(variant=V2, tile_n=256)),
+    ("pair_ragged", 600, 712, 200, {}, dict(variant=V2, tile_n=128)),
+    ("pair_m_below_tile", 100, 300, 136, {}, dict(variant=V2, tile_n=64)),
+    ("pair_nn", 520, 512, 200, dict(ta=0, tb=0), dict(variant=V2, tile_n=128)),
+    ("pair_tn", 520, 512, 200, dict(ta=1, tb=1), dict(variant=V2, tile_n=256)),
+    ("pair_tt", 520, 512, 200, dict(ta=1, tb=0), dict(variant=V2, tile_n=256)),
+    ("pair_batched_bias_bf16", 300, 264, 136, dict(batch=3, epi=bg.EPI_BIAS, cd=wl.BF16), dict(variant=V2, tile_n=128)),
+    ("pair_persistent_beta", 2048, 4096, 128, dict(beta=1.0), dict(variant=V2, tile_n=256)),
+    ("skinny_one_unit", 8, 128, 64, {}, dict(variant=VS)),
+    ("skinny_split_k", 8, 256, 4096, {}, dict(variant=VS)),
+    ("skinny_ragged_beta", 8, 1864, 2136, dict(beta=1.0), dict(variant=VS)),
+    ("skinny_gemv", 1, 4096, 4096, {}, dict(variant=VS)),
+    ("skinny_m16_whole_tiles", 16, 28672, 1024, {}, dict(variant=VS)),
+    ("skinny_m33_bias_bf16", 33, 1000, 520, dict(cd=wl.BF16, epi=bg.EPI_BIAS), dict(variant=VS)),
+    ("skinny_m64_f16", 64, 520, 1032, dict(ab=wl.F16, cd=wl.F16, alpha=0.5, beta=1.0), dict(variant=VS)),
+    ("skinny_stages_2", 8, 384, 1024, {}, dict(variant=VS, stages=2)),
+]
+
+
+@pytest.mark.parametrize("case", EXACT_CASES, ids=[c[0] for c in EXACT_CASES])
+def test_exact_integer_inputs(case):
+    name, M, N, K, kw, fl = case
+    w = int_workload(name, M, N, K, **kw)
+    H.check_workload(w, bg.make_flags(**fl), exact=True, repeats=2)
+
+
+def test_padded_leading_dimensions_and_strides():
+    w = int_workload("padded", 200, 328, 136, batch=3, cd=wl.BF16, beta=1.0,
+                     lda=136 + 8, ldb=136 + 24, ldc=328 + 16,
+                     stride_a=200 * 144 + 64, stride_b=328 * 160 + 8, stride_c=200 * 344 + 128)
+    inputs = wl.make_inputs(w)
+    cbits, _ = H.run_gpu(w, inputs, bg.make_flags(V1))
+    reports = H.check_blocks(w, inputs, cbits, H.default_blocks(w))
+    assert all(r["bit_identical"] == 1.0 for r in reports)
+    # the padding of C must be untouched
+    mask = np.ones(w.elems_c(), bool)
+    idx = (np.arange(w.batch)[:, None, None] * w.stride_c + np.arange(w.M)[None, :, None] * w.ldc + np.arange(w.N)[None, None, :])
+    mask[idx.ravel()] = False
+    assert np.array_equal(cbits[mask], inputs["C"][mask])
+
+
+def test_beta_zero_never_reads_c():
+    # run_gpu pre-fills C with NaN when beta == 0; a finite, exact result proves C was not read
+    for fl in (dict(variant=V1), dict(variant=V2, tile_n=128), dict(variant=VS)):
+        M = 8 if fl["variant"] == VS else 300
+        w = int_workload("nan_c", M, 264, 136)
+        H.check_workload(w, bg.make_flags(**fl), exact=True)
+
+
+def test_automatic_plan_choices_run():
+    for M, N, K in [(512, 512, 512), (8, 4096, 2048), (96, 96, 96), (1000, 3000, 520)]:
+        w = int_workload(f"auto_{M}x{N}x{K}", M, N, K)
+        H.check_workload(w, 0, exact=True)
+
+
+# ----------------------------------------------------------------------------- tolerance regime
+
+@pytest.mark.parametrize("key", ["c2s", "c3s", "c4s", "c5s"])
+@pytest.mark.parametrize("variant", [0, V1, V2])
+def test_small_replicas_of_the_configs(key, variant):
+    w = wl.small_replicas()[key]
+    if key == "c5s" and variant == V2:
+        pytest.skip("M = 8 has no second tile row")
+    H.check_workload(w, bg.make_flags(variant), repeats=2)
+    if w.c_dtype != wl.F32:     # accumulator-domain check: same plan, fp32 output, Frobenius vs the unrounded oracle
+        H.check_workload(w, bg.make_flags(variant), c_dtype=wl.F32)
+
+
+def test_config_c1_full():
+    w = wl.configs()["c1"]
+    reports, info = H.check_workload(w, 0, repeats=3)
+    assert reports[0]["n"] == 512 * 512
+    assert reports[0]["max_err_over_tol"] < 1e-2      # fp32 accumulation sits orders of magnitude inside the bound
+
+
+def _full_config(key, flags=0):
+    w = wl.configs()[key]
+    inputs = wl.make_inputs(w)
+    cbits, info = H.run_gpu(w, inputs, flags)
+    blocks = H.default_blocks(w)
+    reports = H.check_blocks(w, inputs, cbits, blocks)
+    H.assert_reports(reports, what=key)
+    if w.c_dtype != wl.F32:
+        for r in reports:
+            assert r["bit_identical"] >= 0.99, r     # rest is within one ulp (covered by the Frobenius bound)
+        # accumulator-domain check on the sampled rows only (fp32 output of the same plan)
+        cb32, _ = H.run_gpu(w, inputs, flags, c_dtype=wl.F32)
+        rows_block = blocks[-2]
+        rep32 = H.check_blocks(w, inputs, cb32, [rows_block], c_dtype=wl.F32)
+        H.assert_reports(rep32, what=key + " fp32 output")
+        assert rep32[0]["max_err_over_tol"] < 1e-2
+    return reports, info
+
+
+def test_config_c2_sampled_rows_and_columns():
+    reports, info = _full_config("c2")
+    assert info["tile_n"] == 256
+
+
+def test_config_c2_paired_ctas():
+    _full_config("c2", bg.make_flags(V2, 256))
+
+
+def test_config_c3_bias_gelu():
+    _full_config("c3")
+
+
+def test_config_c4_batched_fp16():
+    reports, _ = _full_config("c4")
+    assert len(reports) == 3      # whole batches, sampled rows, sampled columns
+
+
+def test_config_c5_skinny_full():
+    w = wl.configs()["c5"]
+    reports, info = H.check_workload(w, 0, repeats=2)
+    assert info["variant"] == VS and info["grid"] >= 100
+    assert reports[0]["n"] == 8 * 28672
+    assert reports[0]["max_err_over_tol"] < 1e-2
+
+
+def test_gelu_epilogue_values():
+    w = wl.Workload("gelu_probe", 256, 264, 136, transb=1, epilogue=bg.EPI_BIAS_GELU_ERF, c_dtype=wl.F32,
+                    dist_a=wl.Dist("normal", 0, 1), dist_b=wl.Dist("normal", 0, 0.2), seed=99)
+    reports, _ = H.check_workload(w, bg.make_flags(V1))
+    assert reports[0]["frob"] < 1e-5
+
+
+# ----------------------------------------------------------------------------- boundary behaviour on a device
+
+def test_run_argument_errors_launch_nothing():
+    plan = bg.Plan(bg.make_desc(256, 256, 64, epilogue=bg.EPI_BIAS))
+    A = torch.zeros(256 * 64 + 8, dtype=torch.bfloat16, device="cuda")
+    B = torch.zeros(256 * 64, dtype=torch.bfloat16, device="cuda")
+    C = torch.zeros(256 * 256, dtype=torch.float32, device="cuda")
+    bias = torch.zeros(256, dtype=torch.float32, device="cuda")
+    s = torch.cuda.current_stream().cuda_stream
+    with pytest.raises(bg.GemmError) as e:
+        bg.gemm_run(plan.handle, A.data_ptr(), B.data_ptr(), C.data_ptr(), 0, 1.0, 0.0, 0, 0, s)
+    assert e.value.status == bg.ERR_NULL            # bias missing
+    with pytest.raises(bg.GemmError) as e:
+        bg.gemm_run(plan.handle, A.data_ptr() + 2, B.data_ptr(), C.data_ptr(), bias.data_ptr(), 1.0, 0.0, 0, 0, s)
+    assert e.value.status == bg.ERR_ALIGNMENT
+    with pytest.raises(bg.GemmError) as e:
+        bg.gemm_run(plan.handle, 0, B.data_ptr(), C.data_ptr(), bias.data_ptr(), 1.0, 0.0, 0, 0, s)
+    assert e.value.status == bg.ERR_NULL
+    plan.close()
+    sk = bg.Plan(bg.make_desc(8, 1024, 1024, flags=bg.make_flags(VS)))
+    assert sk.workspace_bytes > 0
+    X = torch.zeros(8 * 1024, dtype=torch.bfloat16, device="cuda")
+    Wt = torch.zeros(1024 * 1024, dtype=torch.bfloat16, device="cuda")
+    D = torch.zeros(8 * 1024, dtype=torch.float32, device="cuda")
+    with pytest.raises(bg.GemmError) as e:
+        bg.gemm_run(sk.handle, X.data_ptr(), Wt.data_ptr(), D.data_ptr(), 0, 1.0, 0.0, 0, 0, s)
+    assert e.value.status == bg.ERR_WORKSPACE
+    small = torch.zeros(64, dtype=torch.uint8, device="cuda")
+    with pytest.raises(bg.GemmError) as e:
+        bg.gemm_run(sk.handle, X.data_ptr(), Wt.data_ptr(), D.data_ptr(), 0, 1.0, 0.0, small.data_ptr(), 64, s)
+    assert e.value.status == bg.ERR_WORKSPACE
+    torch.cuda.synchronize()
+    assert sk.status() == bg.OK
+    sk.close()
+
+
+def test_runs_on_a_side_stream():
+    w = int_workload("side_stream", 300, 264, 136)
+    inputs = wl.make_inputs(w)
+    plan = bg.Plan(H.desc_of(w, bg.make_flags(V1)))
+    A, B = H.to_device(inputs["A"], w.ab_dtype), H.to_device(inputs["B"], w.ab_dtype)
+    C = torch.empty(w.elems_c(), dtype=torch.float32, device="cuda")
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        plan.run(A, B, C)
+    side.synchronize()
+    reports = H.check_blocks(w, inputs, H.to_host_bits(C, wl.F32), H.default_blocks(w))
+    assert reports[0]["bit_identical"] == 1.0
+    plan.close()
+
+
+@pytest.mark.parametrize("variant", [V1, V2])
+def test_bounded_wait_reports_timeout_and_context_survives(variant):
+    """A producer arrival is withheld by a test flag, so a device-side wait runs into its limit; the
+    kernel must return on its own, the plan must report GEMM_ERR_TIMEOUT and later work must run."""
+    w = int_workload("stall", 512, 512, 256)
+    inputs = wl.make_inputs(w)
+    plan = bg.Plan(H.desc_of(w, bg.make_flags(variant, 128, debug_stall=True)))
+    plan.set_timeout_ms(20)
+    A, B = H.to_device(inputs["A"], w.ab_dtype), H.to_device(inputs["B"], w.ab_dtype)
+    C = torch.zeros(w.elems_c(), dtype=torch.float32, device="cuda")
+    plan.run(A, B, C)
+    torch.cuda.synchronize()
+    assert plan.status() == bg.ERR_TIMEOUT
+    assert plan.status() == bg.OK          # reading clears the word
+    plan.close()
+    H.check_workload(w, bg.make_flags(variant, 128), exact=True)

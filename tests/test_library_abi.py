@@ -1,0 +1,153 @@
+"""Host-side tests of the C-ABI library: it loads, exports every symbol the header declares,
+validates arguments synchronously and plans the benchmark configurations as documented.
+No GPU needed: nothing here launches a kernel."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2512_16465_b200 as bg
+import workloads as wl
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "gemm.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(gemm_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported():
+    names = declared_functions()
+    assert {"gemm_plan", "gemm_run", "gemm_destroy", "gemm_workspace_bytes"} <= set(names)
+    lib = ctypes.CDLL(bg.LIB_PATH)
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in include/gemm.h but not exported"
+    assert set(bg.EXPORTS) <= set(names)
+
+
+def test_struct_layouts_match_the_header():
+    # 2 x u32, 3 x i64, 4 x i32, 3 x i64, 2 x i32, 3 x i64
+    assert ctypes.sizeof(bg.Desc) == 8 + 24 + 16 + 24 + 8 + 24
+    assert bg.Desc.M.offset == 8 and bg.Desc.lda.offset == 48 and bg.Desc.batch_count.offset == 72
+    assert bg.Desc.stride_a.offset == 80
+    assert bg.Info.num_tiles.offset == 48 and bg.Info.flops.offset == 56
+
+
+def plan_status(**kw):
+    d = bg.make_desc(**kw)
+    try:
+        h = bg.gemm_plan(d)
+    except bg.GemmError as e:
+        return e.status
+    bg.gemm_destroy(h)
+    return bg.OK
+
+
+def test_plan_validation_codes():
+    ok = dict(M=256, N=256, K=256)
+    assert plan_status(**ok) == bg.OK
+    assert plan_status(M=0, N=256, K=256) == bg.ERR_INVALID_ARG
+    assert plan_status(M=256, N=-1, K=256) == bg.ERR_INVALID_ARG
+    assert plan_status(**ok, batch=0) == bg.ERR_INVALID_ARG
+    assert plan_status(**ok, lda=128) == bg.ERR_INVALID_ARG          # lda < K
+    assert plan_status(**ok, ldc=255) == bg.ERR_INVALID_ARG
+    assert plan_status(**ok, transa=2) == bg.ERR_INVALID_ARG
+    assert plan_status(**ok, epilogue=6) == bg.ERR_INVALID_ARG
+    assert plan_status(**ok, c_dtype=3) == bg.ERR_INVALID_ARG
+    assert plan_status(**ok, ab_dtype=bg.F32) == bg.ERR_UNSUPPORTED
+    assert plan_status(M=256, N=256, K=100, lda=100) == bg.ERR_ALIGNMENT     # 200-byte rows
+    assert plan_status(M=256, N=250, K=256, c_dtype=bg.BF16) == bg.ERR_ALIGNMENT  # ldc = 250 -> 500-byte rows
+    assert plan_status(M=256, N=250, K=256, c_dtype=bg.BF16, ldc=256) == bg.OK
+    assert plan_status(**ok, batch=2, stride_c=100) == bg.ERR_INVALID_ARG    # outputs would overlap
+    assert plan_status(**ok, batch=2, stride_a=256 * 256 + 4) == bg.ERR_ALIGNMENT
+    assert plan_status(M=200, N=256, K=256, flags=bg.make_flags(bg.VARIANT_SKINNY_STREAMK)) == bg.ERR_UNSUPPORTED
+    assert plan_status(**ok, flags=bg.make_flags(bg.VARIANT_DENSE_1CTA, tile_n=272)) == bg.ERR_UNSUPPORTED
+    d = bg.make_desc(**ok)
+    d.struct_size = 12
+    with pytest.raises(bg.GemmError) as e:
+        bg.gemm_plan(d)
+    assert e.value.status == bg.ERR_INVALID_ARG
+    assert bg._lib.gemm_plan(None, None) == bg.ERR_NULL
+    assert bg._lib.gemm_destroy(None) == bg.OK
+    assert bg._lib.gemm_workspace_bytes(None) == 0
+    assert bg._lib.gemm_plan_status(None) == bg.ERR_NULL
+
+
+def test_status_strings():
+    names = [bg.status_string(i) for i in range(9)]
+    assert names[0] == "GEMM_OK" and names[8] == "GEMM_ERR_TIMEOUT" and len(set(names)) == 9
+    assert bg.status_string(99) == "GEMM_ERR_UNKNOWN"
+
+
+def info_for(w: wl.Workload, flags=0):
+    h = bg.gemm_plan(bg.make_desc(w.M, w.N, w.K, w.transa, w.transb, w.ab_dtype, w.c_dtype, batch=w.batch,
+                                  epilogue=w.epilogue, flags=flags))
+    info = bg.gemm_plan_info(h)
+    bg.gemm_destroy(h)
+    return info
+
+
+def test_roofline_classification_of_the_five_configs():
+    c = wl.configs()
+    i1, i2, i3, i4, i5 = (info_for(c[k]) for k in ("c1", "c2", "c3", "c4", "c5"))
+    # arithmetic intensities of the configurations (flops / compulsory bytes)
+    assert i1["intensity"] == pytest.approx(128.0)
+    assert i2["intensity"] == pytest.approx(2730.67, rel=1e-4)
+    assert i3["intensity"] == pytest.approx(2667.0, rel=1e-3)
+    assert i4["intensity"] == pytest.approx(113.78, rel=1e-3)
+    assert i5["intensity"] == pytest.approx(7.98, rel=1e-2)       # C read for beta is a run-time matter
+    assert [i["regime"] for i in (i1, i2, i3, i4, i5)] == [1, 2, 2, 1, 0]
+    assert i5["variant"] == bg.VARIANT_SKINNY_STREAMK and i5["workspace_bytes"] > 0
+    for i in (i1, i2, i3, i4):
+        assert i["variant"] in (bg.VARIANT_DENSE_1CTA, bg.VARIANT_DENSE_2CTA) and i["workspace_bytes"] == 0
+        assert i["smem_bytes"] <= 232448 and i["stages"] >= 2
+    assert i2["flops"] == 2.0 * 8192 ** 3 and i2["min_bytes"] == 3 * 8192 * 8192 * 2
+    for k, i in zip(("c1", "c2", "c3", "c4", "c5"), (i1, i2, i3, i4, i5)):
+        assert i["flops"] == c[k].flops
+
+
+def test_stream_k_plan_geometry():
+    i5 = info_for(wl.configs()["c5"])
+    assert i5["num_tiles"] == 224 * 128              # (n-tile, k-block) work units
+    assert i5["grid"] == 148 and i5["tile_m"] == 128 and i5["tile_n"] == 16
+    assert i5["split"] >= 2
+    # counters (224 x 4 bytes padded to 256) + 2 partial slots of 128 x 16 fp32 per CTA
+    assert i5["workspace_bytes"] == 1024 + 148 * 2 * 128 * 16 * 4
+    tiny = info_for(wl.Workload("t", 4, 100, 64), bg.make_flags(bg.VARIANT_SKINNY_STREAMK))
+    assert tiny["grid"] == 1 and tiny["num_tiles"] == 1
+
+
+def test_forced_variants_and_tiles():
+    w = wl.configs()["c2"]
+    i = info_for(w, bg.make_flags(bg.VARIANT_DENSE_2CTA, tile_n=256))
+    assert (i["variant"], i["cluster_size"], i["tile_m"], i["tile_n"]) == (2, 2, 256, 256)
+    assert i["num_tiles"] == 32 * 32 and i["grid"] == 148
+    i = info_for(w, bg.make_flags(bg.VARIANT_DENSE_1CTA, tile_n=128, raster=5, stages=3))
+    assert (i["tile_m"], i["tile_n"], i["raster_group"], i["stages"]) == (128, 128, 5, 3)
+    assert i["num_tiles"] == 64 * 64
+
+
+def test_run_without_a_device_is_an_error_not_a_fallback():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a device is present")
+    h = bg.gemm_plan(bg.make_desc(128, 128, 64))
+    buf = (ctypes.c_char * 65536)()
+    addr = (ctypes.addressof(buf) + 15) & ~15
+    with pytest.raises(bg.GemmError) as e:
+        bg.gemm_run(h, addr, addr, addr, 0, 1.0, 0.0, 0, 0, 0)
+    assert e.value.status == bg.ERR_ARCH
+    assert bg.gemm_plan_status(h) == bg.ERR_ARCH
+    bg.gemm_destroy(h)
+
+
+def test_product_package_does_not_import_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2512_16465_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert "oracle" not in text.lower(), f"{f} mentions the oracle"

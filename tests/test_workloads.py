@@ -1,0 +1,76 @@
+"""Seeded input generators and the benchmark configurations (CPU only)."""
+import numpy as np
+
+import workloads as wl
+
+
+def f32_of_bf16(bits):
+    return np.frombuffer((bits.astype(np.uint32) << 16).tobytes(), np.float32)
+
+
+def test_generators_are_deterministic_and_counter_based():
+    a = wl.normal(7, 1, 10000, 0.0, 1.0, wl.BF16)
+    b = wl.normal(7, 1, 10000, 0.0, 1.0, wl.BF16)
+    assert np.array_equal(a, b)
+    assert np.array_equal(wl.normal(7, 1, 5000, 0.0, 1.0, wl.BF16), a[:5000])   # element i depends on i only
+    assert not np.array_equal(wl.normal(8, 1, 10000, 0.0, 1.0, wl.BF16), a)     # seed matters
+    assert not np.array_equal(wl.normal(7, 2, 10000, 0.0, 1.0, wl.BF16), a)     # tensor id matters
+
+
+def test_distributions():
+    n = 400000
+    u = wl.uniform(1, 1, n, -2.0, 2.0, wl.F16).view(np.float16).astype(np.float64)
+    assert u.min() >= -2.0 and u.max() <= 2.0
+    assert abs(u.mean()) < 0.01 and abs(u.var() - 16.0 / 12.0) < 0.01
+    z = f32_of_bf16(wl.normal(1, 2, n, 0.0, 0.02, wl.BF16)).astype(np.float64)
+    assert abs(z.mean()) < 2e-4 and abs(z.std() - 0.02) < 2e-4
+    assert abs(np.mean(np.abs(z) < 0.02) - 0.6827) < 0.005
+    b = wl.normal(1, 4, n, 0.0, 0.1, wl.F32)
+    assert b.dtype == np.float32 and abs(b.std() - 0.1) < 1e-3
+    k = f32_of_bf16(wl.integer(1, 3, n, -4, 4, wl.BF16))
+    assert set(np.unique(k).tolist()) == set(range(-4, 5))
+    assert np.all(np.bincount((k + 4).astype(int)) > n / 9 * 0.95)
+
+
+def test_configs_match_the_benchmark_definition():
+    c = wl.configs()
+    assert [(w.M, w.N, w.K, w.batch) for w in c.values()] == [
+        (512, 512, 512, 1), (8192, 8192, 8192, 1), (16384, 14336, 4096, 1), (2048, 2048, 128, 64), (8, 28672, 8192, 1)]
+    assert (c["c1"].transa, c["c1"].transb) == (0, 0)
+    assert all((c[k].transa, c[k].transb) == (0, 1) for k in ("c2", "c3", "c4", "c5"))
+    assert c["c3"].epilogue == wl.EPI_BIAS_GELU_ERF and c["c3"].c_dtype == wl.BF16
+    assert c["c4"].ab_dtype == wl.F16 and c["c4"].c_dtype == wl.F16
+    assert c["c4"].alpha == float(np.float32(1.0) / np.sqrt(np.float32(128)))
+    assert (c["c4"].stride_a, c["c4"].stride_b, c["c4"].stride_c) == (262144, 262144, 4194304)
+    assert c["c5"].beta == 1.0 and c["c5"].c_dtype == wl.F32
+    # work and compulsory traffic
+    assert c["c2"].flops == 2 * 8192.0 ** 3 and c["c2"].min_bytes == 3 * 128 * 2 ** 20
+    assert abs(c["c3"].min_bytes - 721.5e6) < 0.1e6
+    assert abs(c["c4"].min_bytes - 604.0e6) < 0.1e6
+    assert abs(c["c5"].min_bytes - 471.7e6) < 0.1e6
+    assert c["c1"].min_bytes == 2 * 2 ** 20
+
+
+def test_make_inputs_shapes_and_rotation():
+    w = wl.small_replicas()["c4s"]
+    a = wl.make_inputs(w)
+    assert a["A"].size == w.batch * w.M * w.K and a["B"].size == w.batch * w.N * w.K
+    assert a["C"] is None and a["bias"] is None
+    b = wl.make_inputs(w, seed_offset=1000)
+    assert not np.array_equal(a["A"], b["A"])
+    w5 = wl.small_replicas()["c5s"]
+    i5 = wl.make_inputs(w5)
+    assert i5["C"].dtype == np.float32 and i5["C"].size == w5.M * w5.N
+    w3 = wl.small_replicas()["c3s"]
+    assert wl.make_inputs(w3)["bias"].size == w3.N
+
+
+def test_sample_indices():
+    s = wl.sample_indices(8192, 256, 5, 1)
+    assert np.array_equal(s, np.unique(s)) and 256 <= s.size <= 256 + 8
+    for e in (0, 1, 127, 128, 255, 256, 8190, 8191):
+        assert e in s
+    assert np.array_equal(s, wl.sample_indices(8192, 256, 5, 1))
+    assert not np.array_equal(s, wl.sample_indices(8192, 256, 5, 2))
+    assert np.array_equal(wl.sample_indices(40, 0, 1, 1), np.arange(40))
+    assert np.array_equal(wl.sample_indices(40, 64, 1, 1), np.arange(40))
