@@ -4,11 +4,20 @@ C-ABI binding, evaluate the oracle on the checked rows / columns and compare.
 Acceptance (per checked element, against the UNROUNDED fp64 oracle value y):
     |D_gpu - y| <= 2e-3 * (|alpha| * sum_k |a||b| + |beta| * |C_in| + |bias_j|) + 1e-5
 and, over each checked block, the relative Frobenius error
-    ||D_gpu - ref||_F / ||ref||_F <= 1e-4
-where ref = y for fp32 output and ref = RNE(y -> output dtype) for 16-bit outputs (rounding
-y to bf16 alone moves it by ~1.7e-3 relative, fp16 by ~2e-4, so the 1e-4 bar can only be
-applied against the rounded oracle there; the accumulator itself is held to 1e-4 against
-y by re-running the same plan with fp32 output).
+    fp32 output  : ||D_gpu - y||_F / ||y||_F <= 1e-4
+    16-bit output: every element within one unit in the last place of RNE(y -> output dtype)
+                   (or within the absolute 1e-5 of y: values that small are governed by the
+                   absolute term), at least 99 % of the elements with |y| >= 1e-4 bit-identical
+                   to it, and
+                   ||D_gpu - RNE(y)||_F / ||RNE(y)||_F <= max(1e-4, 0.1 * u_out),
+                   u_out = 2^-8 (bf16) or 2^-11 (fp16).
+Rounding y to bf16 alone moves it by ~1.7e-3 relative (fp16: ~2e-4), so the 1e-4 bar cannot be
+applied to a 16-bit output against y; against the rounded oracle the only differences are
+elements whose fp32 accumulator landed on the other side of a rounding boundary.  With a
+fraction f of such one-ulp flips the Frobenius distance is about u_out * sqrt(f); fp32
+accumulation over K = 8192 terms with heavy cancellation (config c2) flips about 0.5 % of the
+elements, so the bar is set at f = 1 %, i.e. 0.1 * u_out.  The accumulator itself is held to 1e-4
+against y by re-running the same plan with fp32 output.
 """
 from __future__ import annotations
 
@@ -20,6 +29,19 @@ import paper_2512_16465_b200 as bg
 import workloads as wl
 
 REL_TOL, ABS_TOL, FROB_TOL = 2e-3, 1e-5, 1e-4
+U_OUT = {wl.BF16: 2.0 ** -8, wl.F16: 2.0 ** -11, wl.F32: 0.0}
+
+
+def frob_tol_for(c_dtype: int) -> float:
+    return max(FROB_TOL, 0.1 * U_OUT[c_dtype])
+
+
+def ulp_distance(a_bits: np.ndarray, b_bits: np.ndarray) -> np.ndarray:
+    """Distance in representable values between two arrays of 16-bit float patterns."""
+    def key(x):
+        x = x.astype(np.int32)
+        return np.where(x & 0x8000, -(x & 0x7FFF), x)
+    return np.abs(key(a_bits) - key(b_bits))
 _TORCH_DT = {wl.BF16: torch.bfloat16, wl.F16: torch.float16, wl.F32: torch.float32}
 
 
@@ -101,11 +123,18 @@ def compare_block(got_bits: np.ndarray, y: np.ndarray, bound: np.ndarray, c_dtyp
     denom = float(np.linalg.norm(ref.ravel()))
     frob = float(np.linalg.norm((got - ref).ravel())) / max(denom, 1e-300)
     frob_unrounded = float(np.linalg.norm((got - y).ravel())) / max(float(np.linalg.norm(y.ravel())), 1e-300)
-    exact = float(np.mean(got_bits == ref_bits))
+    same = got_bits == ref_bits
+    big = np.abs(y) >= 1e-4
+    exact = float(np.mean(same[big])) if big.any() else 1.0
     finite = bool(np.all(np.isfinite(got)))
+    max_ulp = 0
+    if c_dtype != wl.F32 and err.size:
+        ulps = ulp_distance(got_bits, ref_bits)
+        ulps = np.where(err <= ABS_TOL, np.minimum(ulps, 1), ulps)
+        max_ulp = int(ulps.max())
     worst = float(np.max(err / tol)) if err.size else 0.0
     return {"max_err_over_tol": worst, "frob": frob, "frob_unrounded": frob_unrounded, "bit_identical": exact,
-            "finite": finite, "n": int(err.size), "argmax": np.unravel_index(int(np.argmax(err / tol)), err.shape) if err.size else None}
+            "finite": finite, "n": int(err.size), "max_ulp": max_ulp, "c_dtype": c_dtype, "argmax": np.unravel_index(int(np.argmax(err / tol)), err.shape) if err.size else None}
 
 
 def check_blocks(w: wl.Workload, inputs: dict, cbits: np.ndarray, blocks, c_dtype=None) -> list:
@@ -141,11 +170,14 @@ def default_blocks(w: wl.Workload) -> list:
     return blocks
 
 
-def assert_reports(reports, frob_tol=FROB_TOL, what=""):
+def assert_reports(reports, what=""):
     for r in reports:
         assert r["finite"], f"{what}: non-finite output {r}"
         assert r["max_err_over_tol"] <= 1.0, f"{what}: per-element tolerance exceeded {r}"
-        assert r["frob"] <= frob_tol, f"{what}: Frobenius error {r}"
+        assert r["frob"] <= frob_tol_for(r["c_dtype"]), f"{what}: Frobenius error {r}"
+        if r["c_dtype"] != wl.F32:
+            assert r["max_ulp"] <= 1, f"{what}: more than one ulp from the rounded oracle {r}"
+            assert r["bit_identical"] >= 0.99, f"{what}: too many one-ulp flips {r}"
 
 
 def check_workload(w: wl.Workload, flags: int = 0, exact: bool = False, c_dtype=None, repeats: int = 1, inputs=None):
