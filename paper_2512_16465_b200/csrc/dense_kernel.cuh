@@ -89,6 +89,33 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const W
   return mbar_wait_slow(bar, parity, w, code);
 }
 
+// Warp-uniform variant: every lane of a fully active warp polls, and all lanes leave with the same answer.
+__device__ __noinline__ bool mbar_wait_warp_slow(uint32_t bar, uint32_t parity, const WaitCtx& w, uint32_t code) {
+  const uint64_t t0 = globaltimer_ns();
+  uint32_t it = 0;
+  while (true) {
+    if (__all_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
+    if ((++it & 31u) == 0u) {
+      bool give_up = false;
+      if (lane_id() == 0) {
+        if (*w.s_abort || *reinterpret_cast<volatile uint32_t*>(w.g_status) != 0u) {
+          *w.s_abort = 1u;
+          give_up = true;
+        } else if (globaltimer_ns() - t0 > w.timeout_ns) {
+          *w.s_abort = 1u;
+          atomicCAS(w.g_status, 0u, kStatusTimeout | code);
+          give_up = true;
+        }
+      }
+      if (__any_sync(0xffffffffu, give_up)) return false;
+    }
+  }
+}
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, const WaitCtx& w, uint32_t code) {
+  if (__all_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
+  return mbar_wait_warp_slow(bar, parity, w, code);
+}
+
 struct TileCoord {
   int batch, tm, tn;
 };
@@ -199,45 +226,56 @@ __device__ __forceinline__ void epilogue_math(float (&v)[32], const uint32_t (&a
   }
 }
 
+// Both single-issuer roles are run by a whole warp in uniform control flow; only the instructions that
+// must be issued once (TMA, tcgen05.mma, commits, barrier arrivals) sit under elect_one().  That keeps
+// addresses, descriptors and coordinates in uniform registers, which is what those instructions read.
 template <int CG>
 __device__ __forceinline__ void producer_role(const DenseParams& p, const CUtensorMap* tmA, const CUtensorMap* tmB,
                                               uint32_t tiles_base, uint32_t full0, uint32_t empty0, uint32_t cta_rank,
                                               int cluster_id, int num_clusters, const WaitCtx& w) {
   const uint32_t stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
-  uint32_t kc = 0;
+  const uint32_t nstages = static_cast<uint32_t>(p.stages);
+  const bool expects = (CG == 1) || (cta_rank == 0);  // in a pair only the leader's barrier counts bytes
+  const int b_groups = p.b_rows / 64;
+  uint32_t s = 0, ph = 0;                             // ring slot and its phase, advanced incrementally
   bool stall_pending = (p.debug_flags & 1u) != 0u;
   for (int tile = cluster_id; tile < p.num_tiles; tile += num_clusters) {
     const TileCoord tc = decode_tile(tile, p.tiles_m, p.tiles_n, p.raster_group);
     const int m0 = tc.tm * (kCtaM * CG) + static_cast<int>(cta_rank) * kCtaM;
     const int n0 = tc.tn * p.bn + (CG == 2 ? static_cast<int>(cta_rank) * p.b_rows : 0);
-    for (int kb = 0; kb < p.num_kb; ++kb, ++kc) {
-      const uint32_t s = kc % static_cast<uint32_t>(p.stages);
-      const uint32_t ph = (kc / static_cast<uint32_t>(p.stages)) & 1u;
-      if (!mbar_wait(empty0 + 8u * s, ph ^ 1u, w, (1u << 8) | s)) return;
+    int k0 = 0;
+    for (int kb = 0; kb < p.num_kb; ++kb, k0 += kBlockK) {
+      if (!mbar_wait_warp(empty0 + 8u * s, ph ^ 1u, w, (1u << 8) | s)) return;
       if (stall_pending) {  // test hook: this stage is never filled nor signalled
         stall_pending = false;
-        continue;
-      }
-      const uint32_t full_local = full0 + 8u * s;
-      if (CG == 1 || cta_rank == 0) mbar_arrive_expect_tx(full_local, stage_bytes * CG);
-      const uint32_t bar = (CG == 1) ? full_local : mapa(full_local, 0);
-      const uint32_t sa = tiles_base + s * stage_bytes;
-      const uint32_t sb = sa + p.a_stage_bytes;
-      const int k0 = kb * kBlockK;
-      auto load = [&](uint32_t dst, const CUtensorMap* map, int x, int y) {
-        if constexpr (CG == 1) tma_load_3d(dst, map, bar, x, y, tc.batch);
-        else tma_load_3d_pair(dst, map, bar, x, y, tc.batch);
-      };
-      if (p.a_kmajor) {
-        load(sa, tmA, k0, m0);
       } else {
-        load(sa, tmA, m0, k0);
-        load(sa + 8192u, tmA, m0 + 64, k0);
+        const uint32_t full_local = full0 + 8u * s;
+        const uint32_t bar = (CG == 1) ? full_local : mapa(full_local, 0);
+        const uint32_t sa = tiles_base + s * stage_bytes;
+        const uint32_t sb = sa + p.a_stage_bytes;
+        if (elect_one()) {
+          if (expects) mbar_arrive_expect_tx(full_local, stage_bytes * CG);
+          auto load = [&](uint32_t dst, const CUtensorMap* map, int x, int y) {
+            if constexpr (CG == 1) tma_load_3d(dst, map, bar, x, y, tc.batch);
+            else tma_load_3d_pair(dst, map, bar, x, y, tc.batch);
+          };
+          if (p.a_kmajor) {
+            load(sa, tmA, k0, m0);
+          } else {
+            load(sa, tmA, m0, k0);
+            load(sa + 8192u, tmA, m0 + 64, k0);
+          }
+          if (p.b_kmajor) {
+            load(sb, tmB, k0, n0);
+          } else {
+            for (int g = 0; g < b_groups; ++g) load(sb + 8192u * g, tmB, n0 + 64 * g, k0);
+          }
+        }
+        __syncwarp();
       }
-      if (p.b_kmajor) {
-        load(sb, tmB, k0, n0);
-      } else {
-        for (int g = 0; g < p.b_rows / 64; ++g) load(sb + 8192u * g, tmB, n0 + 64 * g, k0);
+      if (++s == nstages) {
+        s = 0;
+        ph ^= 1u;
       }
     }
   }
@@ -248,30 +286,46 @@ __device__ __forceinline__ void mma_role(const DenseParams& p, uint32_t tiles_ba
                                          uint32_t tfull0, uint32_t tempty0, uint32_t tmem_base, int cluster_id,
                                          int num_clusters, const WaitCtx& w) {
   const uint32_t stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
-  uint32_t kc = 0, it = 0;
+  const uint32_t nstages = static_cast<uint32_t>(p.stages);
+  const uint32_t stage16 = stage_bytes >> 4, ak16 = p.a_kstep >> 4, bk16 = p.b_kstep >> 4;
+  const uint64_t adesc0 = smem_desc(p.a_desc_hi, tiles_base);
+  const uint64_t bdesc0 = smem_desc(p.b_desc_hi, tiles_base + p.a_stage_bytes);
+  const uint32_t idesc = p.idesc;
+  const int num_kb = p.num_kb;
+  uint32_t s = 0, ph = 0, it = 0;
+  uint64_t adesc = adesc0, bdesc = bdesc0;
   for (int tile = cluster_id; tile < p.num_tiles; tile += num_clusters, ++it) {
     const uint32_t buf = it & 1u;
     const uint32_t aph = (it >> 1) & 1u;
-    if (!mbar_wait(tempty0 + 8u * buf, aph ^ 1u, w, (2u << 8) | 0x80u | buf)) return;
+    if (!mbar_wait_warp(tempty0 + 8u * buf, aph ^ 1u, w, (2u << 8) | 0x80u | buf)) return;
     tc_fence_after();
     const uint32_t d_tmem = tmem_base + buf * static_cast<uint32_t>(p.bn);
-    for (int kb = 0; kb < p.num_kb; ++kb, ++kc) {
-      const uint32_t s = kc % static_cast<uint32_t>(p.stages);
-      const uint32_t ph = (kc / static_cast<uint32_t>(p.stages)) & 1u;
-      if (!mbar_wait(full0 + 8u * s, ph, w, (2u << 8) | s)) return;
+    for (int kb = 0; kb < num_kb; ++kb) {
+      if (!mbar_wait_warp(full0 + 8u * s, ph, w, (2u << 8) | s)) return;
       tc_fence_after();
-      const uint32_t sa = tiles_base + s * stage_bytes;
-      const uint32_t sb = sa + p.a_stage_bytes;
+      const uint32_t empty_bar = empty0 + 8u * s;
+      if (elect_one()) {
+        umma_f16<CG>(d_tmem, adesc, bdesc, idesc, static_cast<uint32_t>(kb != 0));
 #pragma unroll
-      for (int k = 0; k < kBlockK / kUmmaK; ++k) {
-        umma_f16<CG>(d_tmem, smem_desc(p.a_desc_hi, sa + k * p.a_kstep), smem_desc(p.b_desc_hi, sb + k * p.b_kstep),
-                     p.idesc, static_cast<uint32_t>((kb | k) != 0));
+        for (uint32_t k = 1; k < kBlockK / kUmmaK; ++k) umma_f16<CG>(d_tmem, adesc + k * ak16, bdesc + k * bk16, idesc, 1u);
+        umma_commit<CG>(empty_bar);  // ring slot reusable once these MMAs have read it
+        if constexpr (CG == 2) umma_commit<CG>(mapa(empty_bar, 1));
       }
-      umma_commit<CG>(empty0 + 8u * s);  // ring slot reusable once these MMAs have read it
-      if constexpr (CG == 2) umma_commit<CG>(mapa(empty0 + 8u * s, 1));
+      __syncwarp();
+      adesc += stage16;
+      bdesc += stage16;
+      if (++s == nstages) {
+        s = 0;
+        ph ^= 1u;
+        adesc = adesc0;
+        bdesc = bdesc0;
+      }
     }
-    umma_commit<CG>(tfull0 + 8u * buf);  // accumulator complete
-    if constexpr (CG == 2) umma_commit<CG>(mapa(tfull0 + 8u * buf, 1));
+    if (elect_one()) {
+      umma_commit<CG>(tfull0 + 8u * buf);  // accumulator complete
+      if constexpr (CG == 2) umma_commit<CG>(mapa(tfull0 + 8u * buf, 1));
+    }
+    __syncwarp();
   }
 }
 
@@ -405,12 +459,9 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
-    if (lane_id() == 0) producer_role<CG>(p, &tmA, &tmB, base, full0, empty0, cta_rank, cluster_id, num_clusters, w);
-    __syncwarp();
+    producer_role<CG>(p, &tmA, &tmB, base, full0, empty0, cta_rank, cluster_id, num_clusters, w);
   } else if (warp == 1) {
-    if (lane_id() == 0 && cta_rank == 0)
-      mma_role<CG>(p, base, full0, empty0, tfull0, tempty0, tmem_base, cluster_id, num_clusters, w);
-    __syncwarp();
+    if (cta_rank == 0) mma_role<CG>(p, base, full0, empty0, tfull0, tempty0, tmem_base, cluster_id, num_clusters, w);
   } else {
     epilogue_role<CG, EPI_WG>(p, &tmD, base + staging_off, tfull0, tempty0, tmem_base, cta_rank, cluster_id, num_clusters, w);
   }
