@@ -38,10 +38,12 @@ struct DenseParams {
   int raster_group;      // tile rows swept together (column-wise inside the group)
   int bn;                // tile N (multiple of 64, <= 256)
   int stages;            // ring depth
-  int num_kb;            // ceil(K / 64)
+  int num_kb;            // ring stages per tile = ceil(K / (64 * atoms))
+  int atoms;             // 64-wide K slices ("swizzle atoms") per ring stage: 1 or 2
   uint32_t tmem_cols;    // power of two >= 2 * bn
   uint32_t idesc;        // tcgen05 instruction descriptor
-  uint32_t a_stage_bytes, b_stage_bytes;  // per CTA, per stage
+  uint32_t a_stage_bytes, b_stage_bytes;  // per CTA, per stage (all atoms)
+  uint32_t a_atom_bytes, b_atom_bytes;    // per CTA, one 64-wide K slice
   int a_kmajor, b_kmajor;                 // 1: K contiguous in memory; 0: M (resp. N) contiguous
   int b_rows;                             // rows of B (N extent) this CTA loads per stage
   uint64_t a_desc_hi, b_desc_hi;          // descriptor bits above the start address
@@ -55,6 +57,7 @@ struct DenseParams {
   uint32_t* status;                       // device status word
   unsigned long long timeout_ns;
   uint32_t debug_flags;                   // bit 0: withhold one producer arrival (timeout test hook)
+  int l2_hint_a, l2_hint_b;               // L2 eviction priority of operand loads: 0 normal, 1 evict-first, 2 evict-last
 };
 
 struct WaitCtx {
@@ -239,12 +242,14 @@ __device__ __forceinline__ void producer_role(const DenseParams& p, const CUtens
   const int b_groups = p.b_rows / 64;
   uint32_t s = 0, ph = 0;                             // ring slot and its phase, advanced incrementally
   bool stall_pending = (p.debug_flags & 1u) != 0u;
+  const uint64_t pol_a = p.l2_hint_a == 2 ? l2_policy_evict_last() : (p.l2_hint_a == 1 ? l2_policy_evict_first() : l2_policy_evict_normal());
+  const uint64_t pol_b = p.l2_hint_b == 2 ? l2_policy_evict_last() : (p.l2_hint_b == 1 ? l2_policy_evict_first() : l2_policy_evict_normal());
   for (int tile = cluster_id; tile < p.num_tiles; tile += num_clusters) {
     const TileCoord tc = decode_tile(tile, p.tiles_m, p.tiles_n, p.raster_group);
     const int m0 = tc.tm * (kCtaM * CG) + static_cast<int>(cta_rank) * kCtaM;
     const int n0 = tc.tn * p.bn + (CG == 2 ? static_cast<int>(cta_rank) * p.b_rows : 0);
     int k0 = 0;
-    for (int kb = 0; kb < p.num_kb; ++kb, k0 += kBlockK) {
+    for (int kb = 0; kb < p.num_kb; ++kb, k0 += kBlockK * p.atoms) {
       if (!mbar_wait_warp(empty0 + 8u * s, ph ^ 1u, w, (1u << 8) | s)) return;
       if (stall_pending) {  // test hook: this stage is never filled nor signalled
         stall_pending = false;
@@ -255,20 +260,24 @@ __device__ __forceinline__ void producer_role(const DenseParams& p, const CUtens
         const uint32_t sb = sa + p.a_stage_bytes;
         if (elect_one()) {
           if (expects) mbar_arrive_expect_tx(full_local, stage_bytes * CG);
-          auto load = [&](uint32_t dst, const CUtensorMap* map, int x, int y) {
-            if constexpr (CG == 1) tma_load_3d(dst, map, bar, x, y, tc.batch);
-            else tma_load_3d_pair(dst, map, bar, x, y, tc.batch);
+          auto load = [&](uint32_t dst, const CUtensorMap* map, int x, int y, uint64_t pol) {
+            if constexpr (CG == 1) tma_load_3d(dst, map, bar, x, y, tc.batch, pol);
+            else tma_load_3d_pair(dst, map, bar, x, y, tc.batch, pol);
           };
-          if (p.a_kmajor) {
-            load(sa, tmA, k0, m0);
-          } else {
-            load(sa, tmA, m0, k0);
-            load(sa + 8192u, tmA, m0 + 64, k0);
-          }
-          if (p.b_kmajor) {
-            load(sb, tmB, k0, n0);
-          } else {
-            for (int g = 0; g < b_groups; ++g) load(sb + 8192u * g, tmB, n0 + 64 * g, k0);
+          for (int a = 0; a < p.atoms; ++a) {  // slices past K are zero-filled by the copy engine
+            const int ka = k0 + a * kBlockK;
+            const uint32_t saa = sa + a * p.a_atom_bytes, sba = sb + a * p.b_atom_bytes;
+            if (p.a_kmajor) {
+              load(saa, tmA, ka, m0, pol_a);
+            } else {
+              load(saa, tmA, m0, ka, pol_a);
+              load(saa + 8192u, tmA, m0 + 64, ka, pol_a);
+            }
+            if (p.b_kmajor) {
+              load(sba, tmB, ka, n0, pol_b);
+            } else {
+              for (int g = 0; g < b_groups; ++g) load(sba + 8192u * g, tmB, n0 + 64 * g, ka, pol_b);
+            }
           }
         }
         __syncwarp();
@@ -292,6 +301,9 @@ __device__ __forceinline__ void mma_role(const DenseParams& p, uint32_t tiles_ba
   const uint64_t bdesc0 = smem_desc(p.b_desc_hi, tiles_base + p.a_stage_bytes);
   const uint32_t idesc = p.idesc;
   const int num_kb = p.num_kb;
+  const uint32_t aatom16 = p.a_atom_bytes >> 4, batom16 = p.b_atom_bytes >> 4;
+  // atoms of the last stage that still hold part of K (the rest is zero fill and is skipped)
+  const int last_atoms = (p.K - (num_kb - 1) * kBlockK * p.atoms + kBlockK - 1) / kBlockK;
   uint32_t s = 0, ph = 0, it = 0;
   uint64_t adesc = adesc0, bdesc = bdesc0;
   for (int tile = cluster_id; tile < p.num_tiles; tile += num_clusters, ++it) {
@@ -304,12 +316,19 @@ __device__ __forceinline__ void mma_role(const DenseParams& p, uint32_t tiles_ba
       if (!mbar_wait_warp(full0 + 8u * s, ph, w, (2u << 8) | s)) return;
       tc_fence_after();
       const uint32_t empty_bar = empty0 + 8u * s;
+      const bool two = (p.atoms == 2) && (kb + 1 < num_kb || last_atoms == 2);
       if (elect_one()) {
         umma_f16<CG>(d_tmem, adesc, bdesc, idesc, static_cast<uint32_t>(kb != 0));
 #pragma unroll
         for (uint32_t k = 1; k < kBlockK / kUmmaK; ++k) umma_f16<CG>(d_tmem, adesc + k * ak16, bdesc + k * bk16, idesc, 1u);
-        umma_commit<CG>(empty_bar);  // ring slot reusable once these MMAs have read it
-        if constexpr (CG == 2) umma_commit<CG>(mapa(empty_bar, 1));
+        if (two) {
+#pragma unroll
+          for (uint32_t k = 0; k < kBlockK / kUmmaK; ++k)
+            umma_f16<CG>(d_tmem, adesc + aatom16 + k * ak16, bdesc + batom16 + k * bk16, idesc, 1u);
+        }
+        // ring slot reusable once these MMAs have read it (both CTAs of a pair are told at once)
+        if constexpr (CG == 1) umma_commit<1>(empty_bar);
+        else umma_commit_pair_mcast(empty_bar, 3);
       }
       __syncwarp();
       adesc += stage16;
@@ -321,9 +340,9 @@ __device__ __forceinline__ void mma_role(const DenseParams& p, uint32_t tiles_ba
         bdesc = bdesc0;
       }
     }
-    if (elect_one()) {
-      umma_commit<CG>(tfull0 + 8u * buf);  // accumulator complete
-      if constexpr (CG == 2) umma_commit<CG>(mapa(tfull0 + 8u * buf, 1));
+    if (elect_one()) {  // accumulator complete
+      if constexpr (CG == 1) umma_commit<1>(tfull0 + 8u * buf);
+      else umma_commit_pair_mcast(tfull0 + 8u * buf, 3);
     }
     __syncwarp();
   }

@@ -141,12 +141,12 @@ gemm_status_t validate(const gemm_desc_t* d) {
   return GEMM_OK;
 }
 
-int dense_smem_bytes(int stages, int a_stage, int b_stage, int epi_wg) {
+int dense_smem_bytes(int stages, int a_stage, int b_stage, int epi_wg) {  // a_stage, b_stage: all atoms of a stage
   return 1024 /*alignment slack*/ + stages * (a_stage + b_stage) + 4 * epi_wg * 2 * kSlabBytes + 16 * kMaxStages + 64;
 }
 
 // Fill plan->dense and the launch geometry for a dense variant.
-gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_raster, int forced_stages) {
+gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_raster, int forced_stages, int forced_atoms) {
   const gemm_desc_t& d = pl->d;
   const int a_kmajor = d.transa == GEMM_OP_N;
   const int b_kmajor = d.transb == GEMM_OP_T;
@@ -169,8 +169,15 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   if (bn < bn_step || bn > 256 || bn % bn_step) return GEMM_ERR_UNSUPPORTED;
   const int tiles_n = ceil_div(d.N, bn);
   const int b_rows = bn / cg;
-  const int a_stage = kCtaM * kBlockK * 2;
-  const int b_stage = b_rows * kBlockK * 2;
+  const int a_atom = kCtaM * kBlockK * 2;
+  const int b_atom = b_rows * kBlockK * 2;
+  // Each ring stage ends with one tcgen05.commit, which costs tensor-pipe time; a stage of two 64-wide K slices
+  // halves that cost.  Worth it when the ring still has at least three such stages (pairs; narrow 1-CTA tiles).
+  int atoms = forced_atoms;
+  if (atoms == 0) atoms = (d.K > kBlockK && 3 * 2 * (a_atom + b_atom) + dense_smem_bytes(0, 0, 0, 1) <= kMaxSmemOptin) ? 2 : 1;
+  if (atoms < 1 || atoms > 2) return GEMM_ERR_UNSUPPORTED;
+  const int a_stage = atoms * a_atom;
+  const int b_stage = atoms * b_atom;
   const int epi_wg = 1;
   int stages = forced_stages;
   if (stages == 0) {
@@ -204,7 +211,10 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   p.raster_group = raster;
   p.bn = bn;
   p.stages = stages;
-  p.num_kb = ceil_div(d.K, kBlockK);
+  p.num_kb = ceil_div(d.K, kBlockK * atoms);
+  p.atoms = atoms;
+  p.a_atom_bytes = a_atom;
+  p.b_atom_bytes = b_atom;
   uint32_t cols = 32;
   while (cols < 2u * bn) cols <<= 1;
   p.tmem_cols = cols;
@@ -226,6 +236,11 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   p.ldc = d.ldc;
   p.stride_c = d.batch_count > 1 ? d.stride_c : 0;
   p.debug_flags = (d.flags & GEMM_FLAG_DEBUG_STALL) ? 1u : 0u;
+  // The scheduler keeps a band of `raster` tile rows of A live across several waves while B panels stream past;
+  // on request, L2 is asked to hold on to A and to let B go first (measured neutral on 8192^3, so off by default).
+  const bool hints = (d.flags & GEMM_FLAG_L2_HINTS) != 0;
+  p.l2_hint_a = hints ? 2 : 0;
+  p.l2_hint_b = hints ? 1 : 0;
 
   pl->cg = cg;
   pl->epi_wg = epi_wg;
@@ -241,7 +256,7 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   info.variant = pl->variant;
   info.tile_m = tile_m;
   info.tile_n = bn;
-  info.tile_k = kBlockK;
+  info.tile_k = kBlockK * atoms;
   info.stages = stages;
   info.cluster_size = cg;
   info.grid = pl->grid;
@@ -328,16 +343,20 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
   const int forced_bn = static_cast<int>((d.flags & GEMM_FLAG_TILE_N_MASK) >> GEMM_FLAG_TILE_N_SHIFT) * 16;
   const int forced_raster = (d.flags & GEMM_FLAG_RASTER_MASK) >> GEMM_FLAG_RASTER_SHIFT;
   const int forced_stages = (d.flags & GEMM_FLAG_STAGES_MASK) >> GEMM_FLAG_STAGES_SHIFT;
+  const int forced_atoms = (d.flags & GEMM_FLAG_KSLICES_MASK) >> GEMM_FLAG_KSLICES_SHIFT;
   int variant = forced_variant;
   if (variant == 0) {
     // memory-bound problems with a handful of rows stream the weight matrix once: stream-K path;
     // everything else is a dense tiled GEMM, paired CTAs when there are at least two tile rows
     const bool skinny_ok = d.M <= kSkinnyMaxM && d.batch_count == 1 && d.transa == GEMM_OP_N && d.transb == GEMM_OP_T;
+    // a CTA pair halves the B traffic per SM; it pays once there are enough 256-row tiles to occupy every pair
+    const long long pair_tiles = static_cast<long long>(ceil_div(d.M, 2 * kCtaM)) * ceil_div(d.N, 256) * d.batch_count;
     if (skinny_ok && info.intensity < 4.0 * kRidgeCudaCore) variant = GEMM_VARIANT_SKINNY_STREAMK;
+    else if (d.M > kCtaM && pair_tiles >= pl->sm_count / 2) variant = GEMM_VARIANT_DENSE_2CTA;
     else variant = GEMM_VARIANT_DENSE_1CTA;
   }
-  if (variant == GEMM_VARIANT_DENSE_1CTA) st = plan_dense(pl, 1, forced_bn, forced_raster, forced_stages);
-  else if (variant == GEMM_VARIANT_DENSE_2CTA) st = plan_dense(pl, 2, forced_bn, forced_raster, forced_stages);
+  if (variant == GEMM_VARIANT_DENSE_1CTA) st = plan_dense(pl, 1, forced_bn, forced_raster, forced_stages, forced_atoms);
+  else if (variant == GEMM_VARIANT_DENSE_2CTA) st = plan_dense(pl, 2, forced_bn, forced_raster, forced_stages, forced_atoms);
   else if (variant == GEMM_VARIANT_SKINNY_STREAMK) st = plan_skinny(pl, forced_stages);
   else st = GEMM_ERR_INVALID_ARG;
   if (st != GEMM_OK) {

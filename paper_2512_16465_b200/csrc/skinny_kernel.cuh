@@ -151,6 +151,8 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
 
   if (warp == 0) {
     if (lane == 0) {
+      const uint64_t pol_w = l2_policy_evict_first();  // weights are read exactly once
+      const uint64_t pol_x = l2_policy_evict_last();   // the activation slab is re-read by every CTA
       uint32_t kc = 0;
       for (long long u = u_begin; u < u_end; ++u, ++kc) {
         const int tile = static_cast<int>(u / sp.kbs);
@@ -160,8 +162,8 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         if (!mbar_wait(empty0 + 8u * s, ph ^ 1u, w, (1u << 8) | s)) break;
         mbar_arrive_expect_tx(full0 + 8u * s, sp.stage_bytes);
         const uint32_t sw_ = base + s * sp.stage_bytes;
-        tma_load_3d(sw_, &tmW, full0 + 8u * s, kb * kBlockK, tile * kSkinnyTileN, 0);
-        tma_load_3d(sw_ + kSkinnyTileN * 128u, &tmX, full0 + 8u * s, kb * kBlockK, 0, 0);
+        tma_load_3d(sw_, &tmW, full0 + 8u * s, kb * kBlockK, tile * kSkinnyTileN, 0, pol_w);
+        tma_load_3d(sw_ + kSkinnyTileN * 128u, &tmX, full0 + 8u * s, kb * kBlockK, 0, 0, pol_x);
       }
     }
     __syncwarp();
