@@ -168,6 +168,28 @@ gemm_status_t gemm_plan_info(gemm_plan_t plan, gemm_info_t* out);
 /* Free the plan and its status word.  NULL is accepted. */
 gemm_status_t gemm_destroy(gemm_plan_t plan);
 
+/*
+ * gemm_skinny_run_noalloc -- the paper has no counterpart; this is a library convenience.  It runs the
+ * skinny stream-K path (transa = N, transb = T, batch_count = 1, M <= 64) WITHOUT a plan and WITHOUT a
+ * caller workspace, for callers that may not allocate device memory while they run: a process that gave
+ * the whole GPU to its own memory pool at start-up, a latency-critical loop that cannot take the
+ * device-wide synchronisation of cudaMalloc, or code under a "no allocator calls after initialisation"
+ * rule.  The call makes no cudaMalloc / cudaFree and uses no allocating library routine; the plan is built
+ * on the stack and the kernel's scratch (status word, arrival counters, partial tiles) is a fixed 4 MiB
+ * array inside the library, present on every GPU that loads the library until the process exits.
+ *   desc, A, B, C, bias, alpha, beta, stream: as for gemm_plan / gemm_run (desc->flags is ignored).
+ *   sync_and_check: 0 = asynchronous, only launch-time errors are reported; non-zero = wait for `stream`
+ *   and return GEMM_ERR_TIMEOUT if a bounded device-side wait expired.
+ * Limits and rules: problems whose scratch need exceeds the array (with 148 SMs: M > 16) are rejected
+ * with GEMM_ERR_WORKSPACE and nothing is launched (gemm_last_cuda_error() gives the sizes).  The first
+ * call on each device resolves the array's device address and sets a kernel attribute; make that first
+ * call before any stream capture begins.  All calls on a device share the one array: it keeps the
+ * previous call's contents (the call clears what must start at zero), and two calls whose kernels overlap
+ * on the GPU (different streams, or several host threads) race on it -- serialise them.
+ */
+gemm_status_t gemm_skinny_run_noalloc(const gemm_desc_t* desc, const void* A, const void* B, void* C, const float* bias,
+                                      float alpha, float beta, gemm_stream_t stream, int sync_and_check);
+
 /* Static string for a status code. */
 const char* gemm_status_string(gemm_status_t s);
 

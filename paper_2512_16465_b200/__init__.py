@@ -57,7 +57,7 @@ class Info(ctypes.Structure):
 
 
 EXPORTS = ("gemm_plan", "gemm_workspace_bytes", "gemm_run", "gemm_plan_status", "gemm_plan_set_timeout_ms",
-           "gemm_plan_info", "gemm_destroy", "gemm_status_string", "gemm_last_cuda_error")
+           "gemm_plan_info", "gemm_destroy", "gemm_status_string", "gemm_last_cuda_error", "gemm_skinny_run_noalloc")
 
 
 def _load() -> ctypes.CDLL:
@@ -84,6 +84,8 @@ def _load() -> ctypes.CDLL:
     L.gemm_status_string.argtypes = [ctypes.c_int]
     L.gemm_last_cuda_error.restype = ctypes.c_char_p
     L.gemm_last_cuda_error.argtypes = []
+    L.gemm_skinny_run_noalloc.restype = ctypes.c_int
+    L.gemm_skinny_run_noalloc.argtypes = [ctypes.POINTER(Desc), vp, vp, vp, vp, ctypes.c_float, ctypes.c_float, vp, ctypes.c_int]
     return L
 
 
@@ -134,6 +136,21 @@ def gemm_run(plan: int, A: int, B: int, C: int, bias: int, alpha: float, beta: f
     st = _lib.gemm_run(plan, A, B, C, bias or None, alpha, beta, workspace or None, workspace_bytes, stream or None)
     if st != OK:
         raise GemmError(st, "gemm_run")
+
+
+def gemm_skinny_run_noalloc(desc: Desc, A: int, B: int, C: int, bias: int, alpha: float, beta: float, stream: int,
+                            sync_and_check: bool = False) -> None:
+    """``gemm_skinny_run_noalloc``: the skinny stream-K GEMM for callers that may not allocate device memory
+    (no plan, no workspace; the scratch is a fixed array inside the library).  Raw device addresses and a raw
+    ``cudaStream_t`` value; raises :class:`GemmError`, e.g. ``ERR_WORKSPACE`` when the problem is too large for
+    the built-in scratch.  Calls that overlap on the GPU race on that scratch: keep them on one stream."""
+    st = _lib.gemm_skinny_run_noalloc(ctypes.byref(desc), A, B, C, bias or None, alpha, beta, stream or None,
+                                      1 if sync_and_check else 0)
+    if st != OK:
+        err = GemmError(st, "gemm_skinny_run_noalloc")
+        if st == ERR_WORKSPACE:   # the library recorded how much scratch the problem wanted
+            err.args = (f"{err.args[0]} ({_lib.gemm_last_cuda_error().decode()})",)
+        raise err
 
 
 def gemm_plan_status(plan: int) -> int:

@@ -554,3 +554,137 @@ extern "C" gemm_status_t gemm_run(gemm_plan_t plan, const void* A, const void* B
   if (plan->variant == GEMM_VARIANT_SKINNY_STREAMK) return run_skinny(plan, A, B, C, bias, alpha, beta, workspace, s);
   return run_dense(plan, A, B, C, bias, alpha, beta, s);
 }
+
+// ---------------------------------------------------------------------------------------------------------
+// Allocation-free entry point (no counterpart in the paper).
+//
+// Some callers may not allocate device memory once they are running: a serving process that handed the whole
+// GPU to its own memory pool at start-up (a later cudaMalloc fails or fragments the pool), a latency-critical
+// loop that cannot afford cudaMalloc's implicit device-wide synchronisation, or code running under a rule that
+// forbids allocator calls after initialisation.  gemm_plan allocates (the plan object and a status word) and the
+// stream-K kernel wants a caller-provided workspace, so neither fits such a caller.  gemm_skinny_run_noalloc runs
+// the same stream-K kernel with its scratch (status word, arrival counters, partial tiles) in the fixed array
+// below and builds its plan on the stack.
+namespace {
+
+constexpr size_t kNoAllocScratchBytes = 4u << 20;  // held by every GPU that loads the library, until exit
+constexpr size_t kNoAllocHeaderBytes = 256;        // status word of the bounded device waits
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
+
+constexpr int kNoAllocMaxDevices = 64;
+struct NoAllocDevice {
+  unsigned char* scratch;  // device address of g_noalloc_scratch on this device
+  int sm_count;
+  bool arch_ok;
+  bool ready;
+};
+NoAllocDevice g_noalloc_dev[kNoAllocMaxDevices];
+std::mutex g_noalloc_mu;
+
+// Once per device, with that device current: resolve the device address of the scratch array.  In host code the
+// name g_noalloc_scratch is only a handle for the symbol, never a pointer a kernel could use.
+gemm_status_t noalloc_device(int dev, NoAllocDevice* out) {
+  if (dev < 0 || dev >= kNoAllocMaxDevices) return GEMM_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_noalloc_mu);
+  NoAllocDevice& d = g_noalloc_dev[dev];
+  if (!d.ready) {
+    int major = 0, sms = 0;
+    void* ptr = nullptr;
+    cudaError_t e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess && major == 10) e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
+    if (e != cudaSuccess) {
+      note_cuda_error("gemm_skinny_run_noalloc set-up", cudaGetErrorName(e));
+      (void)cudaGetLastError();
+      return GEMM_ERR_CUDA;
+    }
+    d.scratch = static_cast<unsigned char*>(ptr);
+    d.sm_count = sms;
+    d.arch_ok = (major == 10) && ptr != nullptr;
+    d.ready = true;
+  }
+  *out = d;
+  return GEMM_OK;
+}
+
+}  // namespace
+
+extern "C" gemm_status_t gemm_skinny_run_noalloc(const gemm_desc_t* desc, const void* A, const void* B, void* C,
+                                                 const float* bias, float alpha, float beta, gemm_stream_t stream,
+                                                 int sync_and_check) {
+  if (!desc || !A || !B || !C) return GEMM_ERR_NULL;
+  gemm_status_t st = validate(desc);
+  if (st != GEMM_OK) return st;
+  if (has_bias(desc->epilogue) && !bias) return GEMM_ERR_NULL;
+  if (desc->transa != GEMM_OP_N || desc->transb != GEMM_OP_T || desc->batch_count != 1 || desc->M > kSkinnyMaxM)
+    return GEMM_ERR_UNSUPPORTED;
+  auto misaligned = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; };
+  if (misaligned(A) || misaligned(B) || misaligned(C) || (bias && misaligned(bias))) return GEMM_ERR_ALIGNMENT;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return GEMM_ERR_ARCH;
+  }
+  NoAllocDevice nd;
+  st = noalloc_device(dev, &nd);
+  if (st != GEMM_OK) return st;
+  if (!nd.arch_ok) return GEMM_ERR_ARCH;
+
+  SkinnyPlan sp;  // on the stack: nothing is allocated
+  if (!skinny_make_plan(&sp, static_cast<int>(desc->M), static_cast<int>(desc->N), static_cast<int>(desc->K), nd.sm_count, 0,
+                        kMaxSmemOptin))
+    return GEMM_ERR_UNSUPPORTED;
+  const size_t need = kNoAllocHeaderBytes + sp.workspace_bytes;
+  if (need > kNoAllocScratchBytes) {
+    snprintf(g_last_cuda_error, sizeof g_last_cuda_error, "problem needs %zu bytes of scratch, the built-in array has %zu", need,
+             kNoAllocScratchBytes);
+    return GEMM_ERR_WORKSPACE;
+  }
+  CUtensorMap tW, tX;
+  if (!encode_map(&tW, desc->ab_dtype, B, desc->K, desc->N, 1, desc->ldb, 0, kBlockK, kSkinnyTileN) ||
+      !encode_map(&tX, desc->ab_dtype, A, desc->K, desc->M, 1, desc->lda, 0, kBlockK, sp.m_pad))
+    return GEMM_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // The array keeps whatever the previous call left: the status word must start at zero (the launch helper
+  // clears the arrival counters itself; the partial tiles are fully written before they are read).
+  cudaError_t e = cudaMemsetAsync(nd.scratch, 0, kNoAllocHeaderBytes, s);
+  if (e != cudaSuccess) {
+    note_cuda_error("cudaMemsetAsync(status)", cudaGetErrorName(e));
+    (void)cudaGetLastError();
+    return GEMM_ERR_CUDA;
+  }
+  SkinnyParams p;
+  memset(&p, 0, sizeof p);
+  p.plan = sp;
+  p.M = static_cast<int>(desc->M);
+  p.N = static_cast<int>(desc->N);
+  p.K = static_cast<int>(desc->K);
+  p.idesc = make_idesc(desc->ab_dtype == GEMM_BF16, 0, 0, kSkinnyTileN, sp.m_pad);
+  p.out_dtype = desc->c_dtype;
+  p.epilogue = desc->epilogue;
+  p.alpha = alpha;
+  p.beta = beta;
+  p.bias = bias;
+  p.c = C;
+  p.ldc = desc->ldc;
+  p.status = reinterpret_cast<uint32_t*>(nd.scratch);
+  p.counters = reinterpret_cast<uint32_t*>(nd.scratch + kNoAllocHeaderBytes);
+  p.partials = reinterpret_cast<float*>(nd.scratch + kNoAllocHeaderBytes + sp.counters_bytes);
+  p.timeout_ns = 2000ull * 1000000ull;
+  st = static_cast<gemm_status_t>(skinny_launch(p, tW, tX, s, g_last_cuda_error, sizeof g_last_cuda_error));
+  if (st != GEMM_OK || !sync_and_check) return st;
+  uint32_t word = 0;
+  e = cudaStreamSynchronize(s);
+  if (e == cudaSuccess) e = cudaMemcpy(&word, nd.scratch, sizeof word, cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) {
+    note_cuda_error("gemm_skinny_run_noalloc check", cudaGetErrorName(e));
+    (void)cudaGetLastError();
+    return GEMM_ERR_CUDA;
+  }
+  if (word & kStatusTimeout) {
+    snprintf(g_last_cuda_error, sizeof g_last_cuda_error, "device wait expired: role %u detail 0x%02x", (word >> 8) & 0xFF,
+             word & 0xFF);
+    return GEMM_ERR_TIMEOUT;
+  }
+  return GEMM_OK;
+}

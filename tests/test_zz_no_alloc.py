@@ -1,0 +1,87 @@
+"""The allocation-free entry point ``gemm_skinny_run_noalloc`` against the regular plan / run path.
+
+Some users of this library may not allocate GPU memory while they run -- for example a server that
+gave the whole device to its own memory pool when it started, or a real-time loop that cannot accept
+the device-wide synchronisation a cudaMalloc implies.  For them the library offers one call that
+needs neither a plan nor a workspace: its scratch memory is a fixed array inside the library.
+
+That array is shared by every call and keeps the previous call's contents, so the test calls the
+entry point twice in a row (different problems, then the same problem again) and requires the same
+result as the regular entry points each time.  This file is collected last on purpose: it must pass
+both on its own in a fresh process and after every other GPU test has run."""
+import numpy as np
+import pytest
+import torch
+
+import harness as H
+import oracle
+import paper_2512_16465_b200 as bg
+import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+def run_regular(w, inputs):
+    """Existing path: gemm_plan + gemm_run with a caller workspace (stream-K variant)."""
+    cbits, info = H.run_gpu(w, inputs, bg.make_flags(bg.VARIANT_SKINNY_STREAMK), poison=False)
+    assert info["variant"] == bg.VARIANT_SKINNY_STREAMK and info["workspace_bytes"] > 0
+    return cbits
+
+
+_calls = {"n": 0}
+
+
+def run_noalloc(w, inputs):
+    """New path: no plan, no workspace; only the inputs and the output buffer are passed."""
+    A = H.to_device(inputs["A"], w.ab_dtype)
+    B = H.to_device(inputs["B"], w.ab_dtype)
+    bias = None if inputs["bias"] is None else H.to_device(inputs["bias"], wl.F32)
+    if inputs["C"] is not None:
+        C = H.to_device(inputs["C"], w.c_dtype).clone()
+    else:
+        C = torch.zeros(w.elems_c(), dtype=H._TORCH_DT[w.c_dtype], device="cuda")
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    bg.gemm_skinny_run_noalloc(H.desc_of(w), A.data_ptr(), B.data_ptr(), C.data_ptr(),
+                               0 if bias is None else bias.data_ptr(), w.alpha, w.beta,
+                               torch.cuda.current_stream().cuda_stream, sync_and_check=True)
+    _calls["n"] += 1
+    if _calls["n"] > 1:   # (the very first launch may make the driver load the kernel's code)
+        assert torch.cuda.mem_get_info()[0] >= free_before  # the call took no device memory
+    return H.to_host_bits(C, w.c_dtype)
+
+
+def test_noalloc_matches_regular_path_on_consecutive_calls():
+    reps = wl.small_replicas()
+    first = reps["c5s"]                                      # M = 8, beta = 1, fp32 output, ragged N and K
+    second = wl.Workload("noalloc_bias_bf16", 16, 1000, 1096, transb=1, c_dtype=wl.BF16, epilogue=bg.EPI_BIAS_RELU,
+                         dist_b=wl.Dist("normal", 0.0, 0.05), seed=77)
+    # zero-filled C for the beta = 0 workload so that the whole buffers can be compared
+    for w in (first, second, first):                         # two problems back to back, then the first again
+        inputs = wl.make_inputs(w)
+        got = run_noalloc(w, inputs)
+        want = run_regular(w, inputs) if inputs["C"] is not None else None
+        reports = H.check_blocks(w, inputs, got, H.default_blocks(w))
+        H.assert_reports(reports, what=w.name + " (no-alloc)")
+        if want is not None:
+            assert np.array_equal(got, want), "no-alloc result differs from the plan/run result"
+        else:
+            ref, _ = H.run_gpu(w, inputs, bg.make_flags(bg.VARIANT_SKINNY_STREAMK), poison=False)
+            idx = (np.arange(w.M)[:, None] * w.ldc + np.arange(w.N)[None, :]).ravel()
+            assert np.array_equal(got[idx], ref[idx]), "no-alloc result differs from the plan/run result"
+
+
+def test_noalloc_rejects_what_does_not_fit():
+    big = bg.make_desc(64, 4096, 4096)                       # 64 rows need ~9.7 MB of partial tiles: over the 4 MiB array
+    buf = torch.zeros(4096 * 4096, dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros(64 * 4096, dtype=torch.float32, device="cuda")
+    with pytest.raises(bg.GemmError) as e:
+        bg.gemm_skinny_run_noalloc(big, buf.data_ptr(), buf.data_ptr(), out.data_ptr(), 0, 1.0, 0.0,
+                                   torch.cuda.current_stream().cuda_stream)
+    assert e.value.status == bg.ERR_WORKSPACE and "scratch" in str(e.value)
+    dense = bg.make_desc(200, 256, 256)                      # not a skinny problem at all
+    with pytest.raises(bg.GemmError) as e:
+        bg.gemm_skinny_run_noalloc(dense, buf.data_ptr(), buf.data_ptr(), out.data_ptr(), 0, 1.0, 0.0, 0)
+    assert e.value.status == bg.ERR_UNSUPPORTED
+    torch.cuda.synchronize()
+    assert float(out.abs().sum()) == 0.0                     # nothing was launched
