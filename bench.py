@@ -221,6 +221,22 @@ class DeviceCase:
         self.sets = []
 
 
+def max_over_ranks(x: float, device=None) -> float:
+    """MAX of a per-rank scalar over the process group (identity when not distributed)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return x
+    t = torch.tensor([x], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(w: wl.Workload, seconds_max_over_ranks: float, world: int) -> float:
+    """Replicas: every rank runs the same problem, the job's throughput is world x flops over the slowest rank's time."""
+    return world * w.flops / seconds_max_over_ranks / 1e12
+
+
 def metric_value(w: wl.Workload, seconds: float) -> float:
     return w.flops / seconds / 1e12
 
@@ -273,12 +289,8 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    def max_over(x: float) -> float:
+        return max_over_ranks(x, device)
 
     key = args.config
     w = cfgs[key]
@@ -287,7 +299,7 @@ def run_ours(args):
     with ClockSampler(local_rank) as clocks:
         sec = case.time_steps(steps, warmup)
         barrier()
-    sec = max_over_ranks(sec)
+    sec = max_over(sec)
     e2e_steps = max(2, min(steps, args.e2e_steps))
     barrier()
     if args.e2e_steps > 0:
@@ -295,11 +307,11 @@ def run_ours(args):
     else:  # profiling runs skip the host-buffer leg
         e2e_sec, h2d, d2h = float("nan"), 0, 0
     barrier()
-    e2e_sec = max_over_ranks(e2e_sec)
+    e2e_sec = max_over(e2e_sec)
 
     out = {
         "metric": "GEMM TFLOP/s at 1 B200 and % of dense bf16 roofline (HBM GB/s for skinny)",
-        "value": round(metric_value(w, sec) * world, 2), "unit": "TFLOP/s", "n_gpus": world, "steps": steps, "warmup": warmup,
+        "value": round(whole_job_value(w, sec, world), 2), "unit": "TFLOP/s", "n_gpus": world, "steps": steps, "warmup": warmup,
         "ms_per_step": round(sec * 1e3, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16 x bf16 -> fp32 accumulate", "data": "synthetic",
         "config": {"workload": w.name, "M": w.M, "N": w.N, "K": w.K, "batch": w.batch,
@@ -324,12 +336,34 @@ def run_ours(args):
                                  "roofline": out["roofline"]})
                 continue
             c2 = DeviceCase(torch, bg, k2, w2, 0, device)
-            s2 = max_over_ranks(c2.time_steps(steps, warmup))
+            s2 = max_over(c2.time_steps(steps, warmup))
             measured.append({"config": k2, "workload": w2.name, "ms_per_step": round(s2 * 1e3, 5),
                              "tflops": round(metric_value(w2, s2), 2), "gbs": round(w2.min_bytes / s2 / 1e9, 1),
                              "input_sets": c2.nsets, "plan": c2.plan.info, "roofline": roofline_for(w2, k2, s2, peaks, peak_kind)})
             c2.close()
         out["configs_measured"] = measured
+
+    # context only (library kernels, not part of the product): what plain streaming kernels reach on this GPU.
+    # The copy figure in MEASURED_PEAKS.json mixes reads and writes; a write-dominated kernel (c4) cannot go faster
+    # than a pure fill, a read-dominated one (c5) than a pure reduction.
+    if args.all:
+        xs = torch.empty(1 << 29, dtype=torch.float16, device=device)
+
+        def rate(fn, nbytes, n=10):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(n):
+                fn()
+            b.record()
+            torch.cuda.synchronize()
+            return round(nbytes / (a.elapsed_time(b) * 1e-3 / n) / 1e9, 1)
+
+        out["hbm_context"] = {"torch_fill_write_only_gbs": rate(lambda: xs.fill_(1.0), xs.numel() * 2),
+                              "torch_sum_read_only_gbs": rate(lambda: xs.sum(), xs.numel() * 2)}
+        del xs
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         v, cores, sample = time_oracle_sample(w, host_inputs, args.cpu_seconds)
@@ -350,7 +384,7 @@ def run_reference(args):
     inputs = wl.make_inputs(w)
     steps, warmup = args.steps, args.warmup
     # size each step so that the whole run stays within a few minutes
-    per_step = max(0.5, min(10.0, 120.0 / max(1, steps + warmup)))
+    per_step = max(0.05, min(args.ref_step_seconds, 120.0 / max(1, steps + warmup)))
     p = oracle.Problem(w.M, w.N, w.K, w.transa, w.transb, w.ab_dtype, w.c_dtype, w.lda, w.ldb, w.ldc, w.batch,
                        w.stride_a, w.stride_b, w.stride_c, w.epilogue)
     cols = np.arange(w.N, dtype=np.int64)
@@ -397,6 +431,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--ref-step-seconds", type=float, default=10.0, help="--impl reference: CPU time budget of one step")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -388,11 +388,14 @@ __device__ __forceinline__ void epilogue_role(const DenseParams& p, const CUtens
           st_shared_v4(srow + ((static_cast<uint32_t>(j) ^ sw) << 4), __float_as_uint(v[4 * j]), __float_as_uint(v[4 * j + 1]),
                        __float_as_uint(v[4 * j + 2]), __float_as_uint(v[4 * j + 3]));
       } else {
+        // both halves of the 64-column slab are requested before the single wait, so their TMEM latencies overlap
+        uint32_t acc1[32];
+        tmem_ld_32x32(t_row + static_cast<uint32_t>(sl * 64), acc);
+        tmem_ld_32x32(t_row + static_cast<uint32_t>(sl * 64 + 32), acc1);
+        tmem_ld_wait();
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-          tmem_ld_32x32(t_row + static_cast<uint32_t>(sl * 64 + h * 32), acc);
-          tmem_ld_wait();
-          epilogue_math(v, acc, p, row, col0 + h * 32, tc.batch);
+          epilogue_math(v, h == 0 ? acc : acc1, p, row, col0 + h * 32, tc.batch);
           uint32_t pk[16];
           if (p.out_dtype == 0) {
 #pragma unroll

@@ -174,11 +174,13 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   // Each ring stage ends with one tcgen05.commit, which costs tensor-pipe time; a stage of two 64-wide K slices
   // halves that cost.  Worth it when the ring still has at least three such stages (pairs; narrow 1-CTA tiles).
   int atoms = forced_atoms;
-  if (atoms == 0) atoms = (d.K > kBlockK && 3 * 2 * (a_atom + b_atom) + dense_smem_bytes(0, 0, 0, 1) <= kMaxSmemOptin) ? 2 : 1;
+  if (atoms == 0) atoms = (d.K > 2 * kBlockK && 3 * 2 * (a_atom + b_atom) + dense_smem_bytes(0, 0, 0, 1) <= kMaxSmemOptin) ? 2 : 1;
   if (atoms < 1 || atoms > 2) return GEMM_ERR_UNSUPPORTED;
   const int a_stage = atoms * a_atom;
   const int b_stage = atoms * b_atom;
-  const int epi_wg = 1;
+  // A tile's main loop lasts about 512 cycles per 64 columns of K (at tile N = 256); draining 128 x 256 accumulators
+  // with four warps takes several thousand.  Short-K (output-bound) problems get a second epilogue warpgroup.
+  const int epi_wg = (static_cast<long long>(ceil_div(d.K, kBlockK)) * 2 * bn <= 8192) ? 2 : 1;
   int stages = forced_stages;
   if (stages == 0) {
     stages = (kMaxSmemOptin - dense_smem_bytes(0, a_stage, b_stage, epi_wg)) / (a_stage + b_stage);
@@ -352,7 +354,7 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
     // a CTA pair halves the B traffic per SM; it pays once there are enough 256-row tiles to occupy every pair
     const long long pair_tiles = static_cast<long long>(ceil_div(d.M, 2 * kCtaM)) * ceil_div(d.N, 256) * d.batch_count;
     if (skinny_ok && info.intensity < 4.0 * kRidgeCudaCore) variant = GEMM_VARIANT_SKINNY_STREAMK;
-    else if (d.M > kCtaM && pair_tiles >= pl->sm_count / 2) variant = GEMM_VARIANT_DENSE_2CTA;
+    else if (d.M > kCtaM && d.K >= 512 && pair_tiles >= pl->sm_count / 2) variant = GEMM_VARIANT_DENSE_2CTA;
     else variant = GEMM_VARIANT_DENSE_1CTA;
   }
   if (variant == GEMM_VARIANT_DENSE_1CTA) st = plan_dense(pl, 1, forced_bn, forced_raster, forced_stages, forced_atoms);
@@ -502,8 +504,8 @@ gemm_status_t run_dense(gemm_plan_s* pl, const void* A, const void* B, void* C, 
   p.c_in = C;
   p.status = pl->d_status;
   p.timeout_ns = static_cast<unsigned long long>(pl->timeout_ms) * 1000000ull;
-  if (pl->cg == 1) return launch_dense<1, 1>(pl, tA, tB, tD, p, stream);
-  return launch_dense<2, 1>(pl, tA, tB, tD, p, stream);
+  if (pl->cg == 1) return pl->epi_wg == 2 ? launch_dense<1, 2>(pl, tA, tB, tD, p, stream) : launch_dense<1, 1>(pl, tA, tB, tD, p, stream);
+  return pl->epi_wg == 2 ? launch_dense<2, 2>(pl, tA, tB, tD, p, stream) : launch_dense<2, 1>(pl, tA, tB, tD, p, stream);
 }
 
 gemm_status_t run_skinny(gemm_plan_s* pl, const void* A, const void* B, void* C, const float* bias, float alpha, float beta,

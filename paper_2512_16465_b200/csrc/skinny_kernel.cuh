@@ -12,8 +12,8 @@
 //     order (deterministic, no floating-point atomics), applies the epilogue and writes D.
 //     Nobody ever waits for another CTA.
 //
-// Roles per CTA (192 threads): warp 0 lane 0 = TMA producer, warp 1 lane 0 = MMA issuer (warp 1 owns
-// the TMEM allocation), warps 2-5 = epilogue / fix-up.
+// Roles per CTA (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer and owner of the TMEM allocation
+// (both warp-uniform, one elected lane issues), warps 2-5 = epilogue / fix-up.
 #pragma once
 #include <cuda_runtime.h>
 
@@ -54,6 +54,7 @@ inline bool skinny_make_plan(SkinnyPlan* s, int M, int N, int K, int sm_count, i
   const int fixed = 1024 + 16 * kMaxStages + 64;
   int stages = forced_stages ? forced_stages : (max_smem - fixed) / s->stage_bytes;
   if (stages > kMaxStages) stages = kMaxStages;
+  if (!forced_stages && stages > 8) stages = 8;  // measured on B200: 6-10 stages stream fastest, 12 is slower again
   if (stages < 2) return false;
   s->stages = stages;
   s->smem_bytes = fixed + stages * s->stage_bytes;
@@ -149,59 +150,81 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
   const long long u_begin = sk_begin(blockIdx.x, T, G);
   const long long u_end = sk_begin(blockIdx.x + 1, T, G);
 
+  // The producer and MMA roles run warp-uniform (one elected lane issues), with the (tile, k-block) position and
+  // the ring slot advanced incrementally: the single issuing thread must sustain one 18 KB stage every few hundred
+  // cycles, so there is no division and no per-lane register traffic in these loops.
+  const uint32_t nstages = static_cast<uint32_t>(sp.stages);
+  const int tile0 = static_cast<int>(u_begin / sp.kbs);
+  const int kb0 = static_cast<int>(u_begin - static_cast<long long>(tile0) * sp.kbs);
+  const int n_units = static_cast<int>(u_end - u_begin);
   if (warp == 0) {
-    if (lane == 0) {
-      const uint64_t pol_w = l2_policy_evict_first();  // weights are read exactly once
-      const uint64_t pol_x = l2_policy_evict_last();   // the activation slab is re-read by every CTA
-      uint32_t kc = 0;
-      for (long long u = u_begin; u < u_end; ++u, ++kc) {
-        const int tile = static_cast<int>(u / sp.kbs);
-        const int kb = static_cast<int>(u - static_cast<long long>(tile) * sp.kbs);
-        const uint32_t s = kc % static_cast<uint32_t>(sp.stages);
-        const uint32_t ph = (kc / static_cast<uint32_t>(sp.stages)) & 1u;
-        if (!mbar_wait(empty0 + 8u * s, ph ^ 1u, w, (1u << 8) | s)) break;
-        mbar_arrive_expect_tx(full0 + 8u * s, sp.stage_bytes);
-        const uint32_t sw_ = base + s * sp.stage_bytes;
-        tma_load_3d(sw_, &tmW, full0 + 8u * s, kb * kBlockK, tile * kSkinnyTileN, 0, pol_w);
-        tma_load_3d(sw_ + kSkinnyTileN * 128u, &tmX, full0 + 8u * s, kb * kBlockK, 0, 0, pol_x);
+    const uint64_t pol_w = l2_policy_evict_first();  // weights are read exactly once
+    const uint64_t pol_x = l2_policy_evict_last();   // the activation slab is re-read by every CTA
+    uint32_t s = 0, ph = 0;
+    int tile = tile0, kb = kb0;
+    for (int i = 0; i < n_units; ++i) {
+      if (!mbar_wait_warp(empty0 + 8u * s, ph ^ 1u, w, (1u << 8) | s)) break;
+      const uint32_t bar = full0 + 8u * s;
+      const uint32_t sw_ = base + s * sp.stage_bytes;
+      if (elect_one()) {
+        mbar_arrive_expect_tx(bar, sp.stage_bytes);
+        tma_load_3d(sw_, &tmW, bar, kb * kBlockK, tile * kSkinnyTileN, 0, pol_w);
+        tma_load_3d(sw_ + kSkinnyTileN * 128u, &tmX, bar, kb * kBlockK, 0, 0, pol_x);
+      }
+      __syncwarp();
+      if (++kb == sp.kbs) {
+        kb = 0;
+        ++tile;
+      }
+      if (++s == nstages) {
+        s = 0;
+        ph ^= 1u;
       }
     }
-    __syncwarp();
   } else if (warp == 1) {
-    if (lane == 0) {
-      const uint64_t desc_hi = make_smem_desc_hi(16, 1024);
-      uint32_t kc = 0, seg = 0;
-      long long u = u_begin;
-      bool ok = true;
-      while (ok && u < u_end) {
-        const long long tile = u / sp.kbs;
-        const long long seg_end = min(u_end, (tile + 1) * sp.kbs);
-        const uint32_t buf = seg & 1u;
-        if (!mbar_wait(tempty0 + 8u * buf, ((seg >> 1) & 1u) ^ 1u, w, (2u << 8) | 0x80u | buf)) break;
+    const uint64_t desc_hi = make_smem_desc_hi(16, 1024);
+    const uint32_t stage16 = static_cast<uint32_t>(sp.stage_bytes) >> 4;
+    const uint64_t wdesc0 = smem_desc(desc_hi, base);
+    const uint64_t xdesc0 = smem_desc(desc_hi, base + kSkinnyTileN * 128u);
+    const uint32_t idesc = p.idesc;
+    uint32_t s = 0, ph = 0, seg = 0;
+    uint64_t wdesc = wdesc0, xdesc = xdesc0;
+    int kb = kb0, done = 0;
+    bool ok = true;
+    while (ok && done < n_units) {
+      const int seg_units = min(n_units - done, sp.kbs - kb);  // rest of this tile's K that belongs to this CTA
+      const uint32_t buf = seg & 1u;
+      if (!mbar_wait_warp(tempty0 + 8u * buf, ((seg >> 1) & 1u) ^ 1u, w, (2u << 8) | 0x80u | buf)) break;
+      tc_fence_after();
+      const uint32_t d_tmem = tmem_base + buf * static_cast<uint32_t>(sp.m_pad);
+      for (int i = 0; i < seg_units; ++i) {
+        if (!mbar_wait_warp(full0 + 8u * s, ph, w, (2u << 8) | s)) {
+          ok = false;
+          break;
+        }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + buf * static_cast<uint32_t>(sp.m_pad);
-        for (long long uu = u; uu < seg_end; ++uu, ++kc) {
-          const uint32_t s = kc % static_cast<uint32_t>(sp.stages);
-          const uint32_t ph = (kc / static_cast<uint32_t>(sp.stages)) & 1u;
-          if (!mbar_wait(full0 + 8u * s, ph, w, (2u << 8) | s)) {
-            ok = false;
-            break;
-          }
-          tc_fence_after();
-          const uint32_t sw_ = base + s * sp.stage_bytes;
-          const uint32_t sx = sw_ + kSkinnyTileN * 128u;
+        if (elect_one()) {
+          umma_f16<1>(d_tmem, wdesc, xdesc, idesc, static_cast<uint32_t>(i != 0));
 #pragma unroll
-          for (int k = 0; k < kBlockK / kUmmaK; ++k)
-            umma_f16<1>(d_tmem, smem_desc(desc_hi, sw_ + k * 32u), smem_desc(desc_hi, sx + k * 32u), p.idesc,
-                        static_cast<uint32_t>(uu != u || k != 0));
+          for (uint32_t k = 1; k < kBlockK / kUmmaK; ++k) umma_f16<1>(d_tmem, wdesc + 2u * k, xdesc + 2u * k, idesc, 1u);
           umma_commit<1>(empty0 + 8u * s);
         }
-        if (ok) umma_commit<1>(tfull0 + 8u * buf);
-        u = seg_end;
-        ++seg;
+        __syncwarp();
+        wdesc += stage16;
+        xdesc += stage16;
+        if (++s == nstages) {
+          s = 0;
+          ph ^= 1u;
+          wdesc = wdesc0;
+          xdesc = xdesc0;
+        }
       }
+      if (ok && elect_one()) umma_commit<1>(tfull0 + 8u * buf);
+      __syncwarp();
+      done += seg_units;
+      kb = 0;
+      ++seg;
     }
-    __syncwarp();
   } else {
     const uint32_t q = warp & 3u;
     const int n_local = static_cast<int>(q * 32u + lane);

@@ -113,7 +113,7 @@ def test_stream_k_plan_geometry():
     i5 = info_for(wl.configs()["c5"])
     assert i5["num_tiles"] == 224 * 128              # (n-tile, k-block) work units
     assert i5["grid"] == 148 and i5["tile_m"] == 128 and i5["tile_n"] == 16
-    assert i5["split"] >= 2
+    assert i5["split"] >= 2 and i5["stages"] == 8
     # counters (224 x 4 bytes padded to 256) + 2 partial slots of 128 x 16 fp32 per CTA
     assert i5["workspace_bytes"] == 1024 + 148 * 2 * 128 * 16 * 4
     tiny = info_for(wl.Workload("t", 4, 100, 64), bg.make_flags(bg.VARIANT_SKINNY_STREAMK))
