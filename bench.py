@@ -38,9 +38,9 @@ L2_BYTES = 126 * 1024 * 1024
 NOMINAL = {"tensor_tflops": 2250.0, "hbm_gbs": 8000.0}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
-# summarised under profiles/ (file named there); None until a capture exists for the config.
-NCU_TRAFFIC_BYTES = {"c1": None, "c2": None, "c3": None, "c4": None, "c5": None}
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the full-size ncu captures
+# summarised under profiles/ (dense_*_cN_*.txt, skinny_streamk_c5_*.txt; last line of each file).
+NCU_TRAFFIC_BYTES = {"c1": 1122048, "c2": 1245954376, "c3": 1549778496, "c4": 545224448, "c5": 476862208}
 
 
 def load_peaks():
