@@ -83,6 +83,8 @@ typedef enum { GEMM_VARIANT_DENSE_1CTA = 1, GEMM_VARIANT_DENSE_2CTA = 2, GEMM_VA
 #define GEMM_FLAG_STAGES_MASK 0xF000000u
 #define GEMM_FLAG_KSLICES_SHIFT 28         /* bits 28-29: force 64-wide K slices per pipeline stage, 1 or 2 (0 = automatic) */
 #define GEMM_FLAG_KSLICES_MASK 0x30000000u
+#define GEMM_FLAG_NO_K_SERPENTINE 0x8u      /* walk K forwards in every tile (default: alternate tiles walk it backwards,
+                                              which re-uses the operand lines L2 touched last) */
 #define GEMM_FLAG_L2_HINTS 0x40000000u     /* load A with evict-last and B with evict-first L2 priority (default: normal) */
 #define GEMM_FLAG_DEBUG_STALL 0x80000000u  /* test hook: one producer arrival is withheld so that a bounded
                                               wait expires and GEMM_ERR_TIMEOUT is reported */

@@ -94,11 +94,11 @@ LIB_PATH = _build.LIB
 
 
 def make_flags(variant: int = 0, tile_n: int = 0, raster: int = 0, stages: int = 0, debug_stall: bool = False,
-               kslices: int = 0, l2_hints: bool = False) -> int:
+               kslices: int = 0, l2_hints: bool = False, no_k_serpentine: bool = False) -> int:
     """Pack the GEMM_FLAG_* fields of ``gemm_desc_t.flags`` (0 everywhere = automatic)."""
     assert tile_n % 16 == 0
     return ((variant & 0xF) << 4) | (((tile_n // 16) & 0xFF) << 8) | ((raster & 0xFF) << 16) | ((stages & 0xF) << 24) | \
-        ((kslices & 0x3) << 28) | (0x40000000 if l2_hints else 0) | \
+        ((kslices & 0x3) << 28) | (0x40000000 if l2_hints else 0) | (0x8 if no_k_serpentine else 0) | \
         (FLAG_DEBUG_STALL if debug_stall else 0)
 
 

@@ -58,6 +58,7 @@ struct DenseParams {
   unsigned long long timeout_ns;
   uint32_t debug_flags;                   // bit 0: withhold one producer arrival (timeout test hook)
   int l2_hint_a, l2_hint_b;               // L2 eviction priority of operand loads: 0 normal, 1 evict-first, 2 evict-last
+  int k_serpentine;                       // 1: every second tile of a CTA walks K from the far end back to 0
 };
 
 struct WaitCtx {
@@ -73,6 +74,7 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, const
   uint32_t it = 0;
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
+    if (it > 64u) __nanosleep(256);  // long waits (an epilogue warp during a main loop) should not burn issue slots
     if ((++it & 31u) == 0u) {
       if (*w.s_abort) return false;
       if (*reinterpret_cast<volatile uint32_t*>(w.g_status) != 0u) {
@@ -244,12 +246,18 @@ __device__ __forceinline__ void producer_role(const DenseParams& p, const CUtens
   bool stall_pending = (p.debug_flags & 1u) != 0u;
   const uint64_t pol_a = p.l2_hint_a == 2 ? l2_policy_evict_last() : (p.l2_hint_a == 1 ? l2_policy_evict_first() : l2_policy_evict_normal());
   const uint64_t pol_b = p.l2_hint_b == 2 ? l2_policy_evict_last() : (p.l2_hint_b == 1 ? l2_policy_evict_first() : l2_policy_evict_normal());
-  for (int tile = cluster_id; tile < p.num_tiles; tile += num_clusters) {
+  const int kstep = kBlockK * p.atoms;
+  uint32_t it = 0;
+  for (int tile = cluster_id; tile < p.num_tiles; tile += num_clusters, ++it) {
     const TileCoord tc = decode_tile(tile, p.tiles_m, p.tiles_n, p.raster_group);
     const int m0 = tc.tm * (kCtaM * CG) + static_cast<int>(cta_rank) * kCtaM;
     const int n0 = tc.tn * p.bn + (CG == 2 ? static_cast<int>(cta_rank) * p.b_rows : 0);
-    int k0 = 0;
-    for (int kb = 0; kb < p.num_kb; ++kb, k0 += kBlockK * p.atoms) {
+    // Serpentine K: all CTAs advance through K roughly in step, so the K range a wave touched last is what L2
+    // still holds when the next wave starts; walking it backwards re-uses those lines of the shared A band.
+    const bool rev = p.k_serpentine && (it & 1u);
+    int k0 = rev ? (p.num_kb - 1) * kstep : 0;
+    const int dk = rev ? -kstep : kstep;
+    for (int kb = 0; kb < p.num_kb; ++kb, k0 += dk) {
       if (!mbar_wait_warp(empty0 + 8u * s, ph ^ 1u, w, (1u << 8) | s)) return;
       if (stall_pending) {  // test hook: this stage is never filled nor signalled
         stall_pending = false;
@@ -312,11 +320,13 @@ __device__ __forceinline__ void mma_role(const DenseParams& p, uint32_t tiles_ba
     if (!mbar_wait_warp(tempty0 + 8u * buf, aph ^ 1u, w, (2u << 8) | 0x80u | buf)) return;
     tc_fence_after();
     const uint32_t d_tmem = tmem_base + buf * static_cast<uint32_t>(p.bn);
+    const bool rev = p.k_serpentine && (it & 1u);
     for (int kb = 0; kb < num_kb; ++kb) {
       if (!mbar_wait_warp(full0 + 8u * s, ph, w, (2u << 8) | s)) return;
       tc_fence_after();
       const uint32_t empty_bar = empty0 + 8u * s;
-      const bool two = (p.atoms == 2) && (kb + 1 < num_kb || last_atoms == 2);
+      const bool ragged_stage = rev ? (kb == 0) : (kb + 1 == num_kb);  // the stage that holds the end of K
+      const bool two = (p.atoms == 2) && (!ragged_stage || last_atoms == 2);
       if (elect_one()) {
         umma_f16<CG>(d_tmem, adesc, bdesc, idesc, static_cast<uint32_t>(kb != 0));
 #pragma unroll
@@ -425,7 +435,7 @@ __device__ __forceinline__ void epilogue_role(const DenseParams& p, const CUtens
       else mbar_arrive_cluster(mapa(tempty0 + 8u * buf, 0));
     }
   }
-  if (lane == 0) bulk_wait_group<0>();
+  if (lane == 0) bulk_wait_group_read<0>();  // staging may be released; the writes themselves complete with the grid
 }
 
 template <int CG, int EPI_WG>

@@ -173,14 +173,21 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   const int b_atom = b_rows * kBlockK * 2;
   // Each ring stage ends with one tcgen05.commit, which costs tensor-pipe time; a stage of two 64-wide K slices
   // halves that cost.  Worth it when the ring still has at least three such stages (pairs; narrow 1-CTA tiles).
+  const int units = pl->sm_count / cg;
+  const long long tiles_total = static_cast<long long>(tiles_m) * ceil_div(d.N, bn) * d.batch_count;
+  const bool single_wave = tiles_total <= units;  // every CTA (pair) computes at most one tile: pure latency
   int atoms = forced_atoms;
-  if (atoms == 0) atoms = (d.K > 2 * kBlockK && 3 * 2 * (a_atom + b_atom) + dense_smem_bytes(0, 0, 0, 1) <= kMaxSmemOptin) ? 2 : 1;
+  if (atoms == 0) {
+    const bool fits3 = 3 * 2 * (a_atom + b_atom) + dense_smem_bytes(0, 0, 0, 1) <= kMaxSmemOptin;
+    atoms = (d.K > 2 * kBlockK && fits3 && !single_wave) ? 2 : 1;  // one-tile problems want every K slice in flight at once
+  }
   if (atoms < 1 || atoms > 2) return GEMM_ERR_UNSUPPORTED;
   const int a_stage = atoms * a_atom;
   const int b_stage = atoms * b_atom;
   // A tile's main loop lasts about 512 cycles per 64 columns of K (at tile N = 256); draining 128 x 256 accumulators
-  // with four warps takes several thousand.  Short-K (output-bound) problems get a second epilogue warpgroup.
-  const int epi_wg = (static_cast<long long>(ceil_div(d.K, kBlockK)) * 2 * bn <= 8192) ? 2 : 1;
+  // with four warps takes several thousand.  Short-K (output-bound) problems with several tiles per CTA get a second
+  // epilogue warpgroup.
+  const int epi_wg = (!single_wave && static_cast<long long>(ceil_div(d.K, kBlockK)) * 2 * bn <= 8192) ? 2 : 1;
   int stages = forced_stages;
   if (stages == 0) {
     stages = (kMaxSmemOptin - dense_smem_bytes(0, a_stage, b_stage, epi_wg)) / (a_stage + b_stage);
@@ -241,6 +248,7 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   // The scheduler keeps a band of `raster` tile rows of A live across several waves while B panels stream past;
   // on request, L2 is asked to hold on to A and to let B go first (measured neutral on 8192^3, so off by default).
   const bool hints = (d.flags & GEMM_FLAG_L2_HINTS) != 0;
+  p.k_serpentine = ((d.flags & GEMM_FLAG_NO_K_SERPENTINE) || p.num_kb < 4) ? 0 : 1;  // pointless for a couple of stages
   p.l2_hint_a = hints ? 2 : 0;
   p.l2_hint_b = hints ? 1 : 0;
 
@@ -250,7 +258,6 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   pl->stages = stages;
   pl->raster_group = raster;
   pl->smem_bytes = smem;
-  const int units = pl->sm_count / cg;
   pl->grid = static_cast<int>(std::min<long long>(num_tiles, units)) * cg;
   pl->variant = cg == 2 ? GEMM_VARIANT_DENSE_2CTA : GEMM_VARIANT_DENSE_1CTA;
 

@@ -63,6 +63,12 @@ EXACT_CASES = [
     ("pair_tt", 520, 512, 200, dict(ta=1, tb=0), dict(variant=V2, tile_n=256)),
     ("pair_batched_bias_bf16", 300, 264, 136, dict(batch=3, epi=bg.EPI_BIAS, cd=wl.BF16), dict(variant=V2, tile_n=128)),
     ("pair_persistent_beta", 2048, 4096, 128, dict(beta=1.0), dict(variant=V2, tile_n=256)),
+    ("pair_forward_k_only", 512, 512, 1000, {}, dict(variant=V2, tile_n=256, no_k_serpentine=True)),
+    ("pair_serpentine_many_tiles_odd_stages", 1024, 2048, 712, {}, dict(variant=V2, tile_n=128)),
+    ("pair_one_slice_stages", 1024, 1024, 712, {}, dict(variant=V2, tile_n=256, kslices=1)),
+    ("single_serpentine_ragged_k", 1100, 1100, 456, {}, dict(variant=V1, tile_n=128, kslices=2)),
+    ("single_l2_hints", 600, 600, 520, {}, dict(variant=V1, tile_n=64, l2_hints=True)),
+    ("pair_l2_hints", 600, 600, 520, {}, dict(variant=V2, tile_n=128, l2_hints=True)),
     ("skinny_one_unit", 8, 128, 64, {}, dict(variant=VS)),
     ("skinny_split_k", 8, 256, 4096, {}, dict(variant=VS)),
     ("skinny_ragged_beta", 8, 1864, 2136, dict(beta=1.0), dict(variant=VS)),
