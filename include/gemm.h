@@ -70,7 +70,12 @@ typedef enum {
 /* Roofline class of a problem (Section 4.3 of the paper, applied at plan time). */
 typedef enum { GEMM_REGIME_MEMORY = 0, GEMM_REGIME_MIDDLE = 1, GEMM_REGIME_COMPUTE = 2 } gemm_regime_t;
 /* Kernel family a plan selected. */
-typedef enum { GEMM_VARIANT_DENSE_1CTA = 1, GEMM_VARIANT_DENSE_2CTA = 2, GEMM_VARIANT_SKINNY_STREAMK = 3 } gemm_variant_t;
+typedef enum {
+  GEMM_VARIANT_DENSE_1CTA = 1,      /* 128 x N tile per CTA, accumulator double buffered */
+  GEMM_VARIANT_DENSE_2CTA = 2,      /* CTA pair, 256 x N pair tile, accumulator double buffered */
+  GEMM_VARIANT_SKINNY_STREAMK = 3,  /* M <= 64: stream-K over the weight matrix */
+  GEMM_VARIANT_DENSE_2CTA_WIDE = 4  /* CTA pair, 512 x 256 pair tile: least operand traffic per FLOP */
+} gemm_variant_t;
 
 /* gemm_desc_t.flags: 0 = let the plan decide everything. */
 #define GEMM_FLAG_VARIANT_SHIFT 4          /* bits 4-7: force a gemm_variant_t (0 = automatic) */

@@ -20,7 +20,7 @@ from . import build as _build
 BF16, F16, F32 = 0, 1, 2
 OP_N, OP_T = 0, 1
 EPI_NONE, EPI_BIAS, EPI_RELU, EPI_BIAS_RELU, EPI_GELU_ERF, EPI_BIAS_GELU_ERF = range(6)
-VARIANT_AUTO, VARIANT_DENSE_1CTA, VARIANT_DENSE_2CTA, VARIANT_SKINNY_STREAMK = 0, 1, 2, 3
+VARIANT_AUTO, VARIANT_DENSE_1CTA, VARIANT_DENSE_2CTA, VARIANT_SKINNY_STREAMK, VARIANT_DENSE_2CTA_WIDE = 0, 1, 2, 3, 4
 REGIME_NAMES = {0: "memory-bound", 1: "middle-zone", 2: "compute-bound"}
 FLAG_DEBUG_STALL = 0x80000000
 

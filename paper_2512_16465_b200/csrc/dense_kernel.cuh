@@ -74,7 +74,6 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, const
   uint32_t it = 0;
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (it > 64u) __nanosleep(256);  // long waits (an epilogue warp during a main loop) should not burn issue slots
     if ((++it & 31u) == 0u) {
       if (*w.s_abort) return false;
       if (*reinterpret_cast<volatile uint32_t*>(w.g_status) != 0u) {
@@ -95,11 +94,13 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const W
 }
 
 // Warp-uniform variant: every lane of a fully active warp polls, and all lanes leave with the same answer.
-__device__ __noinline__ bool mbar_wait_warp_slow(uint32_t bar, uint32_t parity, const WaitCtx& w, uint32_t code) {
+__device__ __noinline__ bool mbar_wait_warp_slow(uint32_t bar, uint32_t parity, const WaitCtx& w, uint32_t code,
+                                                 uint32_t backoff_ns) {
   const uint64_t t0 = globaltimer_ns();
   uint32_t it = 0;
   while (true) {
     if (__all_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
+    if (backoff_ns != 0u && it > 16u) __nanosleep(backoff_ns);  // long waits should not burn issue slots
     if ((++it & 31u) == 0u) {
       bool give_up = false;
       if (lane_id() == 0) {
@@ -116,9 +117,11 @@ __device__ __noinline__ bool mbar_wait_warp_slow(uint32_t bar, uint32_t parity, 
     }
   }
 }
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, const WaitCtx& w, uint32_t code) {
+// backoff_ns > 0: the warp sleeps between polls once the wait has proved long (an epilogue warp during a main loop).
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, const WaitCtx& w, uint32_t code,
+                                               uint32_t backoff_ns = 0u) {
   if (__all_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
-  return mbar_wait_warp_slow(bar, parity, w, code);
+  return mbar_wait_warp_slow(bar, parity, w, code, backoff_ns);
 }
 
 struct TileCoord {
@@ -375,7 +378,7 @@ __device__ __forceinline__ void epilogue_role(const DenseParams& p, const CUtens
     const TileCoord tc = decode_tile(tile, p.tiles_m, p.tiles_n, p.raster_group);
     const uint32_t buf = it & 1u;
     const uint32_t ph = (it >> 1) & 1u;
-    if (!mbar_wait(tfull0 + 8u * buf, ph, w, (3u << 8) | buf)) return;
+    if (!mbar_wait_warp(tfull0 + 8u * buf, ph, w, (3u << 8) | buf, 64u)) return;  // whole warp leaves the wait together
     tc_fence_after();
     const int row0 = tc.tm * (kCtaM * CG) + static_cast<int>(cta_rank) * kCtaM + static_cast<int>(q) * 32;
     const long long row = row0 + static_cast<int>(lane);

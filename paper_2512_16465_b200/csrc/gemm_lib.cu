@@ -17,6 +17,7 @@
 
 #include "dense_kernel.cuh"
 #include "skinny_kernel.cuh"
+#include "wide_kernel.cuh"
 
 using namespace b200;
 
@@ -277,6 +278,84 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   return GEMM_OK;
 }
 
+// Wide pair variant: 512 x 256 cluster tiles, one 64-wide K slice per stage, 3-deep ring, 8 epilogue warps.
+gemm_status_t plan_wide(gemm_plan_s* pl, int forced_raster, int forced_stages) {
+  const gemm_desc_t& d = pl->d;
+  const int a_kmajor = d.transa == GEMM_OP_N;
+  const int b_kmajor = d.transb == GEMM_OP_T;
+  const int tile_m = 2 * kWideCtaM, bn = kWideTileN;
+  const int tiles_m = ceil_div(d.M, tile_m), tiles_n = ceil_div(d.N, bn);
+  const int a_stage = kWideCtaM * kBlockK * 2, b_stage = (bn / 2) * kBlockK * 2;
+  const int fixed = 1024 + 16 * kSlabBytes + 16 * kMaxStages + 64;
+  int stages = forced_stages ? forced_stages : std::min(3, (kMaxSmemOptin - fixed) / (a_stage + b_stage));
+  if (stages < 2 || stages > kMaxStages) return GEMM_ERR_UNSUPPORTED;
+  const int smem = fixed + stages * (a_stage + b_stage);
+  if (smem > kMaxSmemOptin) return GEMM_ERR_UNSUPPORTED;
+  const long long num_tiles = static_cast<long long>(tiles_m) * tiles_n * d.batch_count;
+  if (num_tiles > 0x7FFFFFFFll) return GEMM_ERR_UNSUPPORTED;
+  const int units = pl->sm_count / 2;
+  int raster = forced_raster;
+  if (raster == 0) raster = std::max(1, static_cast<int>(std::lround(std::sqrt(static_cast<double>(units) * bn / tile_m))));
+  raster = std::max(1, std::min(raster, tiles_m));
+
+  DenseParams& p = pl->dense;
+  memset(&p, 0, sizeof p);
+  p.M = static_cast<int>(d.M);
+  p.N = static_cast<int>(d.N);
+  p.K = static_cast<int>(d.K);
+  p.batch = d.batch_count;
+  p.tiles_m = tiles_m;
+  p.tiles_n = tiles_n;
+  p.num_tiles = static_cast<int>(num_tiles);
+  p.raster_group = raster;
+  p.bn = bn;
+  p.stages = stages;
+  p.num_kb = ceil_div(d.K, kBlockK);
+  p.atoms = 1;
+  p.tmem_cols = 512;
+  p.idesc = make_idesc(d.ab_dtype == GEMM_BF16, !a_kmajor, !b_kmajor, 256, bn);
+  p.a_stage_bytes = a_stage;
+  p.b_stage_bytes = b_stage;
+  p.a_atom_bytes = a_stage;
+  p.b_atom_bytes = b_stage;
+  p.a_kmajor = a_kmajor;
+  p.b_kmajor = b_kmajor;
+  p.b_rows = bn / 2;
+  p.a_desc_hi = a_kmajor ? make_smem_desc_hi(16, 1024) : make_smem_desc_hi(8192, 1024);
+  p.b_desc_hi = b_kmajor ? make_smem_desc_hi(16, 1024) : make_smem_desc_hi(8192, 1024);
+  p.a_kstep = a_kmajor ? kUmmaK * 2 : kUmmaK * 128;
+  p.b_kstep = b_kmajor ? kUmmaK * 2 : kUmmaK * 128;
+  p.out_dtype = d.c_dtype;
+  p.epilogue = d.epilogue;
+  p.ldc = d.ldc;
+  p.stride_c = d.batch_count > 1 ? d.stride_c : 0;
+  p.debug_flags = (d.flags & GEMM_FLAG_DEBUG_STALL) ? 1u : 0u;
+  p.k_serpentine = ((d.flags & GEMM_FLAG_NO_K_SERPENTINE) || p.num_kb < 4) ? 0 : 1;
+
+  pl->cg = 2;
+  pl->epi_wg = 2;
+  pl->bn = bn;
+  pl->stages = stages;
+  pl->raster_group = raster;
+  pl->smem_bytes = smem;
+  pl->grid = static_cast<int>(std::min<long long>(num_tiles, units)) * 2;
+  pl->variant = GEMM_VARIANT_DENSE_2CTA_WIDE;
+  gemm_info_t& info = pl->info;
+  info.variant = pl->variant;
+  info.tile_m = tile_m;
+  info.tile_n = bn;
+  info.tile_k = kBlockK;
+  info.stages = stages;
+  info.cluster_size = 2;
+  info.grid = pl->grid;
+  info.raster_group = raster;
+  info.split = 1;
+  info.smem_bytes = smem;
+  info.num_tiles = num_tiles;
+  info.workspace_bytes = 0;
+  return GEMM_OK;
+}
+
 gemm_status_t plan_skinny(gemm_plan_s* pl, int forced_stages) {
   const gemm_desc_t& d = pl->d;
   if (d.transa != GEMM_OP_N || d.transb != GEMM_OP_T) return GEMM_ERR_UNSUPPORTED;  // both operands K-contiguous
@@ -361,19 +440,31 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
     // a CTA pair halves the B traffic per SM; it pays once there are enough 256-row tiles to occupy every pair
     const long long pair_tiles = static_cast<long long>(ceil_div(d.M, 2 * kCtaM)) * ceil_div(d.N, 256) * d.batch_count;
     if (skinny_ok && info.intensity < 4.0 * kRidgeCudaCore) variant = GEMM_VARIANT_SKINNY_STREAMK;
-    else if (d.M > kCtaM && d.K >= 512 && pair_tiles >= pl->sm_count / 2) variant = GEMM_VARIANT_DENSE_2CTA;
+    else if (d.M > kCtaM && d.K >= 512 && pair_tiles >= pl->sm_count / 2) {
+      variant = GEMM_VARIANT_DENSE_2CTA;
+      // The 512 x 256 variant moves a quarter less operand data per FLOP (it runs ~4 % faster at the power cap) but
+      // exposes part of its epilogue: taken for long K, cheap epilogues and when its last wave is about as full.
+      const int pairs = pl->sm_count / 2;
+      const long long wide_tiles = static_cast<long long>(ceil_div(d.M, 2 * kWideCtaM)) * ceil_div(d.N, kWideTileN) * d.batch_count;
+      const double eff_pair = static_cast<double>(pair_tiles) / (static_cast<double>(ceil_div(pair_tiles, pairs)) * pairs);
+      const double eff_wide = static_cast<double>(wide_tiles) / (static_cast<double>(ceil_div(wide_tiles, pairs)) * pairs);
+      const bool cheap_epilogue = d.epilogue < GEMM_EPI_GELU_ERF;
+      if (cheap_epilogue && d.K >= 4096 && d.M >= 2 * kWideCtaM && wide_tiles >= pairs && eff_wide >= eff_pair - 0.02)
+        variant = GEMM_VARIANT_DENSE_2CTA_WIDE;
+    }
     else variant = GEMM_VARIANT_DENSE_1CTA;
   }
   if (variant == GEMM_VARIANT_DENSE_1CTA) st = plan_dense(pl, 1, forced_bn, forced_raster, forced_stages, forced_atoms);
   else if (variant == GEMM_VARIANT_DENSE_2CTA) st = plan_dense(pl, 2, forced_bn, forced_raster, forced_stages, forced_atoms);
   else if (variant == GEMM_VARIANT_SKINNY_STREAMK) st = plan_skinny(pl, forced_stages);
+  else if (variant == GEMM_VARIANT_DENSE_2CTA_WIDE) st = plan_wide(pl, forced_raster, forced_stages);
   else st = GEMM_ERR_INVALID_ARG;
   if (st != GEMM_OK) {
     delete pl;
     return st;
   }
   if (pl->has_device && pl->arch_ok) {
-    if (cudaMalloc(&pl->d_status, 16) != cudaSuccess || cudaMemset(pl->d_status, 0, 16) != cudaSuccess) {
+    if (cudaMalloc(&pl->d_status, 256) != cudaSuccess || cudaMemset(pl->d_status, 0, 256) != cudaSuccess) {
       note_cuda_error("cudaMalloc(status word)", cudaGetErrorName(cudaGetLastError()));
       delete pl;
       return GEMM_ERR_CUDA;
@@ -491,6 +582,38 @@ gemm_status_t launch_dense(const gemm_plan_s* pl, const CUtensorMap& tA, const C
   return GEMM_OK;
 }
 
+gemm_status_t launch_wide(const gemm_plan_s* pl, const CUtensorMap& tA, const CUtensorMap& tB, const CUtensorMap& tD,
+                          const DenseParams& p, cudaStream_t stream) {
+  static thread_local int configured_smem = 0;
+  if (configured_smem < pl->smem_bytes) {
+    if (cudaFuncSetAttribute(wide_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, pl->smem_bytes) != cudaSuccess) {
+      note_cuda_error("cudaFuncSetAttribute", cudaGetErrorName(cudaGetLastError()));
+      return GEMM_ERR_CUDA;
+    }
+    configured_smem = pl->smem_bytes;
+  }
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof cfg);
+  cfg.gridDim = dim3(pl->grid, 1, 1);
+  cfg.blockDim = dim3(kWideThreads, 1, 1);
+  cfg.dynamicSmemBytes = pl->smem_bytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, wide_gemm_kernel, tA, tB, tD, p);
+  if (e != cudaSuccess) {
+    note_cuda_error("cudaLaunchKernelEx(wide)", cudaGetErrorName(e));
+    (void)cudaGetLastError();
+    return GEMM_ERR_CUDA;
+  }
+  return GEMM_OK;
+}
+
 gemm_status_t run_dense(gemm_plan_s* pl, const void* A, const void* B, void* C, const float* bias, float alpha, float beta,
                         cudaStream_t stream) {
   const gemm_desc_t& d = pl->d;
@@ -498,7 +621,8 @@ gemm_status_t run_dense(gemm_plan_s* pl, const void* A, const void* B, void* C, 
   CUtensorMap tA, tB, tD;
   const uint64_t batch = d.batch_count;
   // A: K-major -> rows are M, inner K, box 64 x 128; M-major (stored K x M) -> rows are K, inner M, box 64 x 64
-  bool ok = p.a_kmajor ? encode_map(&tA, d.ab_dtype, A, d.K, d.M, batch, d.lda, d.stride_a, kBlockK, kCtaM)
+  const uint32_t a_box_rows = pl->variant == GEMM_VARIANT_DENSE_2CTA_WIDE ? kWideCtaM : kCtaM;
+  bool ok = p.a_kmajor ? encode_map(&tA, d.ab_dtype, A, d.K, d.M, batch, d.lda, d.stride_a, kBlockK, a_box_rows)
                        : encode_map(&tA, d.ab_dtype, A, d.M, d.K, batch, d.lda, d.stride_a, 64, kBlockK);
   ok = ok && (p.b_kmajor ? encode_map(&tB, d.ab_dtype, B, d.K, d.N, batch, d.ldb, d.stride_b, kBlockK, p.b_rows)
                          : encode_map(&tB, d.ab_dtype, B, d.N, d.K, batch, d.ldb, d.stride_b, 64, kBlockK));
@@ -511,6 +635,7 @@ gemm_status_t run_dense(gemm_plan_s* pl, const void* A, const void* B, void* C, 
   p.c_in = C;
   p.status = pl->d_status;
   p.timeout_ns = static_cast<unsigned long long>(pl->timeout_ms) * 1000000ull;
+  if (pl->variant == GEMM_VARIANT_DENSE_2CTA_WIDE) return launch_wide(pl, tA, tB, tD, p, stream);
   if (pl->cg == 1) return pl->epi_wg == 2 ? launch_dense<1, 2>(pl, tA, tB, tD, p, stream) : launch_dense<1, 1>(pl, tA, tB, tD, p, stream);
   return pl->epi_wg == 2 ? launch_dense<2, 2>(pl, tA, tB, tD, p, stream) : launch_dense<2, 1>(pl, tA, tB, tD, p, stream);
 }

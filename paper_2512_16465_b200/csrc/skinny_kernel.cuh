@@ -236,7 +236,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
       const long long tile_u0 = tile * sp.kbs;
       const long long seg_end = min(u_end, tile_u0 + sp.kbs);
       const uint32_t buf = seg & 1u;
-      if (!mbar_wait(tfull0 + 8u * buf, (seg >> 1) & 1u, w, (3u << 8) | buf)) break;
+      if (!mbar_wait_warp(tfull0 + 8u * buf, (seg >> 1) & 1u, w, (3u << 8) | buf, 64u)) break;
       tc_fence_after();
       const int n = static_cast<int>(tile) * kSkinnyTileN + n_local;
       const bool whole = (u == tile_u0) && (seg_end == tile_u0 + sp.kbs);  // this CTA owns the tile's whole K

@@ -13,6 +13,7 @@ pytestmark = pytest.mark.gpu
 
 INT = wl.Dist("integer", -4, 4)
 V1, V2, VS = bg.VARIANT_DENSE_1CTA, bg.VARIANT_DENSE_2CTA, bg.VARIANT_SKINNY_STREAMK
+VW = bg.VARIANT_DENSE_2CTA_WIDE
 
 
 def int_workload(name, M, N, K, ta=0, tb=1, ab=wl.BF16, cd=wl.F32, batch=1, epi=0, alpha=1.0, beta=0.0, **kw):
@@ -69,6 +70,15 @@ EXACT_CASES = [
     ("single_serpentine_ragged_k", 1100, 1100, 456, {}, dict(variant=V1, tile_n=128, kslices=2)),
     ("single_l2_hints", 600, 600, 520, {}, dict(variant=V1, tile_n=64, l2_hints=True)),
     ("pair_l2_hints", 600, 600, 520, {}, dict(variant=V2, tile_n=128, l2_hints=True)),
+    ("wide_one_tile", 512, 256, 64, {}, dict(variant=VW)),
+    ("wide_ragged", 1100, 712, 456, {}, dict(variant=VW)),
+    ("wide_m_below_tile", 100, 300, 136, {}, dict(variant=VW)),
+    ("wide_persistent_bf16", 4096, 4096, 320, dict(cd=wl.BF16), dict(variant=VW)),
+    ("wide_beta_bias_f32", 1100, 712, 200, dict(beta=1.0, epi=bg.EPI_BIAS), dict(variant=VW)),
+    ("wide_nn", 1024, 520, 264, dict(ta=0, tb=0), dict(variant=VW)),
+    ("wide_tn", 1024, 520, 264, dict(ta=1, tb=1), dict(variant=VW)),
+    ("wide_tt_batched_f16", 600, 520, 136, dict(ta=1, tb=0, batch=3, ab=wl.F16, cd=wl.F16, alpha=0.5), dict(variant=VW)),
+    ("wide_two_stage_ring_forward_k", 1024, 512, 1000, {}, dict(variant=VW, stages=2, no_k_serpentine=True)),
     ("skinny_one_unit", 8, 128, 64, {}, dict(variant=VS)),
     ("skinny_split_k", 8, 256, 4096, {}, dict(variant=VS)),
     ("skinny_ragged_beta", 8, 1864, 2136, dict(beta=1.0), dict(variant=VS)),
@@ -119,10 +129,10 @@ def test_automatic_plan_choices_run():
 # ----------------------------------------------------------------------------- tolerance regime
 
 @pytest.mark.parametrize("key", ["c2s", "c3s", "c4s", "c5s"])
-@pytest.mark.parametrize("variant", [0, V1, V2])
+@pytest.mark.parametrize("variant", [0, V1, V2, VW])
 def test_small_replicas_of_the_configs(key, variant):
     w = wl.small_replicas()[key]
-    if key == "c5s" and variant == V2:
+    if key == "c5s" and variant in (V2, VW):
         pytest.skip("M = 8 has no second tile row")
     H.check_workload(w, bg.make_flags(variant), repeats=2)
     if w.c_dtype != wl.F32:     # accumulator-domain check: same plan, fp32 output, Frobenius vs the unrounded oracle
@@ -157,7 +167,7 @@ def _full_config(key, flags=0):
 
 def test_config_c2_sampled_rows_and_columns():
     reports, info = _full_config("c2")
-    assert info["tile_n"] == 256
+    assert info["tile_n"] == 256 and info["variant"] == VW     # the automatic choice for this shape
 
 
 def test_config_c2_paired_ctas():
@@ -240,13 +250,14 @@ def test_runs_on_a_side_stream():
     plan.close()
 
 
-@pytest.mark.parametrize("variant", [V1, V2])
+@pytest.mark.parametrize("variant", [V1, V2, VW])
 def test_bounded_wait_reports_timeout_and_context_survives(variant):
     """A producer arrival is withheld by a test flag, so a device-side wait runs into its limit; the
     kernel must return on its own, the plan must report GEMM_ERR_TIMEOUT and later work must run."""
     w = int_workload("stall", 512, 512, 256)
     inputs = wl.make_inputs(w)
-    plan = bg.Plan(H.desc_of(w, bg.make_flags(variant, 128, debug_stall=True)))
+    tile_n = 0 if variant == VW else 128
+    plan = bg.Plan(H.desc_of(w, bg.make_flags(variant, tile_n, debug_stall=True)))
     plan.set_timeout_ms(20)
     A, B = H.to_device(inputs["A"], w.ab_dtype), H.to_device(inputs["B"], w.ab_dtype)
     C = torch.zeros(w.elems_c(), dtype=torch.float32, device="cuda")
@@ -255,4 +266,4 @@ def test_bounded_wait_reports_timeout_and_context_survives(variant):
     assert plan.status() == bg.ERR_TIMEOUT
     assert plan.status() == bg.OK          # reading clears the word
     plan.close()
-    H.check_workload(w, bg.make_flags(variant, 128), exact=True)
+    H.check_workload(w, bg.make_flags(variant, tile_n), exact=True)

@@ -102,9 +102,13 @@ def test_roofline_classification_of_the_five_configs():
     assert [i["regime"] for i in (i1, i2, i3, i4, i5)] == [1, 2, 2, 1, 0]
     assert i5["variant"] == bg.VARIANT_SKINNY_STREAMK and i5["workspace_bytes"] > 0
     for i in (i1, i2, i3, i4):
-        assert i["variant"] in (bg.VARIANT_DENSE_1CTA, bg.VARIANT_DENSE_2CTA) and i["workspace_bytes"] == 0
+        assert i["variant"] in (bg.VARIANT_DENSE_1CTA, bg.VARIANT_DENSE_2CTA, bg.VARIANT_DENSE_2CTA_WIDE)
+        assert i["workspace_bytes"] == 0
         assert i["smem_bytes"] <= 232448 and i["stages"] >= 2
     assert i2["flops"] == 2.0 * 8192 ** 3 and i2["min_bytes"] == 3 * 8192 * 8192 * 2
+    assert i2["variant"] == bg.VARIANT_DENSE_2CTA_WIDE and (i2["tile_m"], i2["tile_n"], i2["stages"]) == (512, 256, 3)
+    assert i3["variant"] == bg.VARIANT_DENSE_2CTA          # erf-GELU epilogue: keep the double-buffered accumulator
+    assert i4["variant"] == bg.VARIANT_DENSE_1CTA and i1["variant"] == bg.VARIANT_DENSE_1CTA
     for k, i in zip(("c1", "c2", "c3", "c4", "c5"), (i1, i2, i3, i4, i5)):
         assert i["flops"] == c[k].flops
 
