@@ -9,13 +9,14 @@
 // Each CTA owns 256 rows (two 128-row halves, one TMEM lane set each) x 256 columns: the accumulator
 // fills all 512 TMEM columns (half h in columns [256 h, 256 h + 256)), so there is no second accumulator
 // buffer.  Overlap with the next tile comes from releasing early instead: the eight epilogue warps drain half 0
-// first (64 columns per thread at a time: read, convert, stage, TMA store) and hand its TMEM columns back as
-// soon as they are read; the MMA issuer starts the next tile on half 0 while half 1 is still being drained.
+// first (per thread 128 columns: read, convert and pack in registers) and hand its TMEM columns back as soon as
+// they are read; the MMA issuer starts the next tile on half 0 while half 1 is still being drained.
 //
 // Ring stage = 64 columns of K: A 256 x 64 (32 KB) + this CTA's half of B, 128 x 64 (16 KB); per stage the
 // leader issues 8 tcgen05.mma.cta_group::2 (M 256, N 256, K 16: four per half) and one multicast commit.
 // Three ring stages (144 KB) and two 4 KB staging slabs per epilogue warp (64 KB).
-// Roles: warp 0 producer, warp 1 MMA issuer (leader CTA) and TMEM owner, warps 2-9 epilogue.
+// Roles: warp 0 producer, warp 1 MMA issuer (leader CTA) and TMEM owner, warps 4-11 epilogue (two whole
+// warpgroups; warps 2-3 only take part in the CTA-wide barriers).
 #pragma once
 #include "dense_kernel.cuh"
 
@@ -23,7 +24,22 @@ namespace b200 {
 
 constexpr int kWideCtaM = 256;      // rows per CTA (two TMEM-lane halves)
 constexpr int kWideTileN = 256;     // tile columns = columns of one accumulator half
-constexpr int kWideThreads = 64 + 256;
+constexpr int kWideThreads = 128 + 256;  // warps 0-1: producer, MMA issuer; warps 2-3: idle; warps 4-11: epilogue
+
+// Conversions pinned in program order (volatile): the packed values of one 64-column part must exist before the
+// next part's accumulators are loaded, otherwise both parts' raw accumulators are live at once.  (A 320-thread CTA
+// gets at most 168 registers per thread; the epilogue below fits without spilling, and spills here cost
+// microseconds per tile because their cache lines are long gone when the next tile ends.)
+__device__ __forceinline__ uint32_t pack_bf16x2_pinned(float lo, float hi) {
+  uint32_t d;
+  asm volatile("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+__device__ __forceinline__ uint32_t pack_f16x2_pinned(float lo, float hi) {
+  uint32_t d;
+  asm volatile("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
 
 __device__ __forceinline__ void wide_producer_role(const DenseParams& p, const CUtensorMap* tmA, const CUtensorMap* tmB,
                                                    uint32_t tiles_base, uint32_t full0, uint32_t empty0, uint32_t cta_rank,
@@ -90,6 +106,7 @@ __device__ __forceinline__ void wide_mma_role(const DenseParams& p, uint32_t til
   // starts on half 1), so the first `lead` stages are issued for half 0 only, without releasing their ring slots;
   // half 1 then catches up on the same stages and releases them.  From there on both halves go stage by stage.
   const int lead = min(p.stages, num_kb);
+  const int tail = min(p.stages, num_kb - lead);
   auto advance = [&](uint32_t& cs, uint32_t& cph, uint64_t& ca, uint64_t& cb) {
     ca += stage16;
     cb += stage16;
@@ -131,7 +148,7 @@ __device__ __forceinline__ void wide_mma_role(const DenseParams& p, uint32_t til
         advance(s, ph, adesc, bdesc);
       }
     }
-    for (int kb = lead; kb < num_kb; ++kb) {
+    for (int kb = lead; kb < num_kb - tail; ++kb) {
       if (!mbar_wait_warp(full0 + 8u * s, ph, w, (2u << 8) | s)) return;
       tc_fence_after();
       if (elect_one()) {
@@ -145,8 +162,36 @@ __device__ __forceinline__ void wide_mma_role(const DenseParams& p, uint32_t til
       __syncwarp();
       advance(s, ph, adesc, bdesc);
     }
-    if (elect_one()) umma_commit_pair_mcast(tfull, 3);  // both halves of the accumulator are complete
-    __syncwarp();
+    // Mirror image at the end of the tile: the last `tail` stages are issued for half 0 first, so half 0 completes
+    // (and its read-out starts) while the tensor pipe is still busy with half 1's share of those stages.
+    {
+      uint32_t s0 = s, ph0 = ph;
+      uint64_t a0 = adesc, b0 = bdesc;
+      for (int kb = 0; kb < tail; ++kb) {
+        if (!mbar_wait_warp(full0 + 8u * s0, ph0, w, (2u << 8) | s0)) return;
+        tc_fence_after();
+        if (elect_one()) {
+#pragma unroll
+          for (uint32_t k = 0; k < kBlockK / kUmmaK; ++k) umma_f16<2>(tmem_base, a0 + k * ak16, b0 + k * bk16, idesc, 1u);
+        }
+        __syncwarp();
+        advance(s0, ph0, a0, b0);
+      }
+      if (elect_one()) umma_commit_pair_mcast(tfull, 3);  // half 0 of the accumulator is complete
+      __syncwarp();
+      for (int kb = 0; kb < tail; ++kb) {
+        if (elect_one()) {
+#pragma unroll
+          for (uint32_t k = 0; k < kBlockK / kUmmaK; ++k)
+            umma_f16<2>(tmem_base + kWideTileN, adesc + half16 + k * ak16, bdesc + k * bk16, idesc, 1u);
+          umma_commit_pair_mcast(empty0 + 8u * s, 3);
+        }
+        __syncwarp();
+        advance(s, ph, adesc, bdesc);
+      }
+      if (elect_one()) umma_commit_pair_mcast(tfull + 8u, 3);  // half 1 is complete
+      __syncwarp();
+    }
   }
 }
 
@@ -156,38 +201,38 @@ __device__ __forceinline__ void wide_epilogue_role(const DenseParams& p, const C
   const uint32_t warp = threadIdx.x >> 5;
   const uint32_t lane = lane_id();
   const uint32_t q = warp & 3u;          // TMEM lane quarter this warp may read
-  const uint32_t ch = (warp - 2u) >> 2;  // which 128 columns of each half this warpgroup drains
-  const uint32_t stg = staging + (warp - 2u) * (2u * kSlabBytes);  // two slabs per warp, used alternately
+  const uint32_t ch = (warp - 4u) >> 2;  // which 128 columns of each half this warpgroup drains
+  const uint32_t stg = staging + (warp - 4u) * (2u * kSlabBytes);  // two slabs per warp, used alternately
   const uint32_t sw = lane & 7u;
   uint32_t it = 0, nstore = 0;
   for (int tile = cluster_id; tile < p.num_tiles; tile += num_clusters, ++it) {
     const TileCoord tc = decode_tile(tile, p.tiles_m, p.tiles_n, p.raster_group);
     const int row_cta = tc.tm * (2 * kWideCtaM) + static_cast<int>(cta_rank) * kWideCtaM + static_cast<int>(q) * 32;
     const int colbase = tc.tn * kWideTileN + static_cast<int>(ch) * 128;
-    if (!mbar_wait_warp(tfull, it & 1u, w, (3u << 8), 64u)) return;
-    tc_fence_after();
 #pragma unroll 1
     for (uint32_t h = 0; h < 2; ++h) {
+      if (!mbar_wait_warp(tfull + 8u * h, it & 1u, w, (3u << 8) | h, 64u)) return;
+      tc_fence_after();
       const int row0 = row_cta + static_cast<int>(h) * 128;
       const long long row = row0 + static_cast<int>(lane);
       const uint32_t t_row = tmem_base + ((q * 32u) << 16) + h * kWideTileN + ch * 128u;
+      float v[32];
+      if (p.out_dtype == 2) {
+        // fp32 output: 64 accumulator columns at a time; the half is handed back once its second part is read
 #pragma unroll 1
-      for (uint32_t part = 0; part < 2; ++part) {  // 64 accumulator columns at a time: 64 live registers, no spills
-        uint32_t acc0[32], acc1[32];
-        tmem_ld_32x32(t_row + 64u * part, acc0);
-        tmem_ld_32x32(t_row + 64u * part + 32u, acc1);
-        tmem_ld_wait();
-        if (part == 1) {  // this thread's share of half h is in registers: hand the TMEM columns back
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive_cluster(mapa(tempty0 + 8u * h, 0));
-        }
-        const int col64 = colbase + 64 * static_cast<int>(part);
-        float v[32];
-        if (p.out_dtype == 2) {
+        for (uint32_t part = 0; part < 2; ++part) {
+          uint32_t acc0[32], acc1[32];
+          tmem_ld_32x32(t_row + 64u * part, acc0);
+          tmem_ld_32x32(t_row + 64u * part + 32u, acc1);
+          tmem_ld_wait();
+          if (part == 1) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(mapa(tempty0 + 8u * h, 0));
+          }
 #pragma unroll
           for (int u = 0; u < 2; ++u, ++nstore) {
-            const int col0 = col64 + 32 * u;
+            const int col0 = colbase + 64 * static_cast<int>(part) + 32 * u;
             const uint32_t sbuf = stg + (nstore & 1u) * kSlabBytes;
             const uint32_t srow = sbuf + lane * 128u;
             if (lane == 0) bulk_wait_group_read<1>();  // the store that last read this slab has finished with it
@@ -204,27 +249,49 @@ __device__ __forceinline__ void wide_epilogue_role(const DenseParams& p, const C
               bulk_commit_group();
             }
           }
-        } else {
+        }
+      } else {
+        // 16-bit output: both 64-column parts are read, converted and packed (2 x 32 registers) before anything is
+        // staged, so the half goes back to the MMA issuer a few hundred cycles after the accumulator is complete;
+        // the two slabs are then written out without waiting on each other.
+        uint32_t pk0[32], pk1[32];
+        auto read_part = [&](const uint32_t part, uint32_t (&pk)[32]) {
+          uint32_t acc0[32], acc1[32];
+          tmem_ld_32x32(t_row + 64u * part, acc0);
+          tmem_ld_32x32(t_row + 64u * part + 32u, acc1);
+          tmem_ld_wait();
+          if (part == 1u) {  // this thread's share of half h is in registers: hand the TMEM columns back
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(mapa(tempty0 + 8u * h, 0));
+          }
+          const int col64 = colbase + 64 * static_cast<int>(part);
+          epilogue_math(v, acc0, p, row, col64, tc.batch);
+          if (p.out_dtype == 0) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) pk[j] = pack_bf16x2_pinned(v[2 * j], v[2 * j + 1]);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) pk[j] = pack_f16x2_pinned(v[2 * j], v[2 * j + 1]);
+          }
+          epilogue_math(v, acc1, p, row, col64 + 32, tc.batch);
+          if (p.out_dtype == 0) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) pk[16 + j] = pack_bf16x2_pinned(v[2 * j], v[2 * j + 1]);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) pk[16 + j] = pack_f16x2_pinned(v[2 * j], v[2 * j + 1]);
+          }
+        };
+        auto store_part = [&](const uint32_t part, const uint32_t (&pk)[32]) {
+          const int col64 = colbase + 64 * static_cast<int>(part);
           const uint32_t sbuf = stg + (nstore & 1u) * kSlabBytes;
           const uint32_t srow = sbuf + lane * 128u;
-          if (lane == 0) bulk_wait_group_read<1>();
+          if (lane == 0) bulk_wait_group_read<1>();  // the store that last read this slab has finished with it
           __syncwarp();
 #pragma unroll
-          for (int hh = 0; hh < 2; ++hh) {
-            epilogue_math(v, hh == 0 ? acc0 : acc1, p, row, col64 + 32 * hh, tc.batch);
-            uint32_t pk[16];
-            if (p.out_dtype == 0) {
-#pragma unroll
-              for (int j = 0; j < 16; ++j) pk[j] = pack_bf16x2(v[2 * j], v[2 * j + 1]);
-            } else {
-#pragma unroll
-              for (int j = 0; j < 16; ++j) pk[j] = pack_f16x2(v[2 * j], v[2 * j + 1]);
-            }
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-              st_shared_v4(srow + ((static_cast<uint32_t>(4 * hh + j) ^ sw) << 4), pk[4 * j], pk[4 * j + 1], pk[4 * j + 2],
-                           pk[4 * j + 3]);
-          }
+          for (int j = 0; j < 8; ++j)
+            st_shared_v4(srow + ((static_cast<uint32_t>(j) ^ sw) << 4), pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
           fence_proxy_async_smem();
           __syncwarp();
           if (lane == 0) {
@@ -232,7 +299,11 @@ __device__ __forceinline__ void wide_epilogue_role(const DenseParams& p, const C
             bulk_commit_group();
           }
           ++nstore;
-        }
+        };
+        read_part(0u, pk0);
+        read_part(1u, pk1);
+        store_part(0u, pk0);
+        store_part(1u, pk1);
       }
     }
   }
@@ -266,7 +337,8 @@ wide_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       mbar_init(full0 + 8u * s, 1);
       mbar_init(empty0 + 8u * s, 1);
     }
-    mbar_init(tfull, 1);
+    mbar_init(tfull, 1);          // accumulator half 0 complete
+    mbar_init(tfull + 8u, 1);     // accumulator half 1 complete
     mbar_init(tempty0, 16);       // 8 epilogue warps in each CTA of the pair, per accumulator half
     mbar_init(tempty0 + 8u, 16);
     *s_abort = 0u;
@@ -290,7 +362,7 @@ wide_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     wide_producer_role(p, &tmA, &tmB, base, full0, empty0, cta_rank, cluster_id, num_clusters, w);
   } else if (warp == 1) {
     if (cta_rank == 0) wide_mma_role(p, base, full0, empty0, tfull, tempty0, tmem_base, cluster_id, num_clusters, w);
-  } else {
+  } else if (warp >= 4) {
     wide_epilogue_role(p, &tmD, base + staging_off, tfull, tempty0, tmem_base, cta_rank, cluster_id, num_clusters, w);
   }
 
