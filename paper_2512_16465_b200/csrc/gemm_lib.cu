@@ -439,7 +439,7 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
     const bool skinny_ok = d.M <= kSkinnyMaxM && d.batch_count == 1 && d.transa == GEMM_OP_N && d.transb == GEMM_OP_T;
     // a CTA pair halves the B traffic per SM; it pays once there are enough 256-row tiles to occupy every pair
     const long long pair_tiles = static_cast<long long>(ceil_div(d.M, 2 * kCtaM)) * ceil_div(d.N, 256) * d.batch_count;
-    if (skinny_ok && info.intensity < 4.0 * kRidgeCudaCore) variant = GEMM_VARIANT_SKINNY_STREAMK;
+    if (skinny_ok && info.intensity < 5.2 * kRidgeCudaCore) variant = GEMM_VARIANT_SKINNY_STREAMK;  // measured: wins up to M ~ 48
     else if (d.M > kCtaM && d.K >= 512 && pair_tiles >= pl->sm_count / 2) {
       variant = GEMM_VARIANT_DENSE_2CTA;
       // The 512 x 256 variant moves a quarter less operand data per FLOP (it runs ~4 % faster at the power cap) but

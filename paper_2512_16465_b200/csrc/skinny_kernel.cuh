@@ -92,14 +92,24 @@ __device__ __forceinline__ void sk_store_d(const SkinnyParams& p, long long idx,
   else if (p.out_dtype == 0) static_cast<__nv_bfloat16*>(p.c)[idx] = __float2bfloat16_rn(v);
   else static_cast<__half*>(p.c)[idx] = __float2half_rn(v);
 }
-__device__ __forceinline__ void sk_finish(const SkinnyParams& p, int m, int n, float acc) {
-  const long long idx = static_cast<long long>(m) * p.ldc + n;
-  float v = p.alpha * acc;
-  if (p.beta != 0.0f) v += p.beta * sk_load_c(p, idx);
-  if (p.epilogue & 1) v += __ldg(p.bias + n);
-  if (p.epilogue == 2 || p.epilogue == 3) v = fmaxf(v, 0.0f);
-  else if (p.epilogue >= 4) v = gelu_erf(v);
-  sk_store_d(p, idx, v);
+// Finish up to 16 rows of one output column: all C_in values are fetched first and only then is D stored.
+// (C_in and D are the same buffer, so a load placed after a store could not be moved ahead of it and the rows
+// would cost one global-memory round trip each.)
+__device__ __forceinline__ void sk_finish16(const SkinnyParams& p, int m0, int n, const float (&acc)[16]) {
+  float cin[16];
+  const float bias = (p.epilogue & 1) ? __ldg(p.bias + n) : 0.0f;
+#pragma unroll
+  for (int j = 0; j < 16; ++j)
+    cin[j] = (p.beta != 0.0f && m0 + j < p.M) ? sk_load_c(p, static_cast<long long>(m0 + j) * p.ldc + n) : 0.0f;
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    if (m0 + j < p.M) {
+      float v = p.alpha * acc[j] + p.beta * cin[j] + bias;
+      if (p.epilogue == 2 || p.epilogue == 3) v = fmaxf(v, 0.0f);
+      else if (p.epilogue >= 4) v = gelu_erf(v);
+      sk_store_d(p, static_cast<long long>(m0 + j) * p.ldc + n, v);
+    }
+  }
 }
 
 __global__ void __launch_bounds__(kSkinnyThreads, 1)
@@ -246,16 +256,15 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         uint32_t acc[16];
         tmem_ld_32x16(t_row + static_cast<uint32_t>(c0), acc);
         tmem_ld_wait();
+        if (whole) {
+          float accf[16];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const int m = c0 + j;
-          if (m < p.M) {
-            if (whole) {
-              if (n < p.N) sk_finish(p, m, n, __uint_as_float(acc[j]));
-            } else {
-              my_partial[m * kSkinnyTileN + n_local] = __uint_as_float(acc[j]);
-            }
-          }
+          for (int j = 0; j < 16; ++j) accf[j] = __uint_as_float(acc[j]);
+          if (n < p.N) sk_finish16(p, c0, n, accf);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            if (c0 + j < p.M) my_partial[(c0 + j) * kSkinnyTileN + n_local] = __uint_as_float(acc[j]);
         }
       }
       tc_fence_before();
@@ -275,14 +284,18 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         const bool last = *s_last != 0u;
         if (last) {
           __threadfence();
-          for (int m = 0; m < p.M; ++m) {
-            float sum = 0.0f;
-            for (int c = c_first; c <= c_last; ++c) {
+          for (int m0 = 0; m0 < p.M; m0 += 16) {
+            float sum[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) sum[j] = 0.0f;
+            for (int c = c_first; c <= c_last; ++c) {  // contributor order: the result does not depend on arrival order
               const int slot = (sk_begin(c, T, G) / sp.kbs == tile) ? 0 : 1;  // tile is c's first segment?
               const float* part = p.partials + (static_cast<size_t>(c) * 2 + slot) * (kSkinnyTileN * sp.m_pad);
-              sum += __ldcg(part + m * kSkinnyTileN + n_local);
+#pragma unroll
+              for (int j = 0; j < 16; ++j)
+                if (m0 + j < p.M) sum[j] += __ldcg(part + (m0 + j) * kSkinnyTileN + n_local);
             }
-            if (n < p.N) sk_finish(p, m, n, sum);
+            if (n < p.N) sk_finish16(p, m0, n, sum);
           }
           if (leader) p.counters[tile] = 0u;  // leave the counter clean for the next launch
         }
