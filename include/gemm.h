@@ -153,7 +153,8 @@ size_t gemm_workspace_bytes(gemm_plan_t plan);
  * that is 0); concurrent runs of one plan need distinct workspaces.  alpha and
  * beta are host scalars.  Errors are returned before anything is launched:
  * GEMM_ERR_NULL, GEMM_ERR_ALIGNMENT, GEMM_ERR_WORKSPACE, GEMM_ERR_ARCH,
- * GEMM_ERR_CUDA (tensor-map encoding or launch failure).
+ * GEMM_ERR_INVALID_ARG (the current CUDA device is not the one the plan was
+ * made on), GEMM_ERR_CUDA (tensor-map encoding or launch failure).
  */
 gemm_status_t gemm_run(gemm_plan_t plan, const void* A, const void* B, void* C, const float* bias, float alpha,
                        float beta, void* workspace, size_t workspace_bytes, gemm_stream_t stream);

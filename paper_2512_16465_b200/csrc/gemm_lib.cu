@@ -101,6 +101,7 @@ struct gemm_plan_s {
   int grid;
   int smem_bytes;
   int sm_count;
+  int device;            // CUDA device the plan was made on (-1: none); runs must use the same one
   bool has_device;
   bool arch_ok;
   uint32_t* d_status;
@@ -402,9 +403,11 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
   pl->timeout_ms = 2000;
   pl->sm_count = kDefaultSmCount;
   int dev = -1;
+  pl->device = -1;
   if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0) {
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, dev) == cudaSuccess) {
+      pl->device = dev;
       pl->has_device = true;
       pl->arch_ok = prop.major == 10;
       if (pl->arch_ok) pl->sm_count = prop.multiProcessorCount;
@@ -552,13 +555,10 @@ template <int CG, int EPI_WG>
 gemm_status_t launch_dense(const gemm_plan_s* pl, const CUtensorMap& tA, const CUtensorMap& tB, const CUtensorMap& tD,
                            const DenseParams& p, cudaStream_t stream) {
   auto kern = dense_gemm_kernel<CG, EPI_WG>;
-  static thread_local int configured_smem = 0;  // per instantiation
-  if (configured_smem < pl->smem_bytes) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl->smem_bytes) != cudaSuccess) {
-      note_cuda_error("cudaFuncSetAttribute", cudaGetErrorName(cudaGetLastError()));
-      return GEMM_ERR_CUDA;
-    }
-    configured_smem = pl->smem_bytes;
+  constexpr KernelSlot slot = CG == 1 ? (EPI_WG == 1 ? kSlotDense11 : kSlotDense12) : (EPI_WG == 1 ? kSlotDense21 : kSlotDense22);
+  if (ensure_dynamic_smem(reinterpret_cast<const void*>(kern), slot, pl->device, pl->smem_bytes) != cudaSuccess) {
+    note_cuda_error("cudaFuncSetAttribute", cudaGetErrorName(cudaGetLastError()));
+    return GEMM_ERR_CUDA;
   }
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof cfg);
@@ -584,13 +584,9 @@ gemm_status_t launch_dense(const gemm_plan_s* pl, const CUtensorMap& tA, const C
 
 gemm_status_t launch_wide(const gemm_plan_s* pl, const CUtensorMap& tA, const CUtensorMap& tB, const CUtensorMap& tD,
                           const DenseParams& p, cudaStream_t stream) {
-  static thread_local int configured_smem = 0;
-  if (configured_smem < pl->smem_bytes) {
-    if (cudaFuncSetAttribute(wide_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, pl->smem_bytes) != cudaSuccess) {
-      note_cuda_error("cudaFuncSetAttribute", cudaGetErrorName(cudaGetLastError()));
-      return GEMM_ERR_CUDA;
-    }
-    configured_smem = pl->smem_bytes;
+  if (ensure_dynamic_smem(reinterpret_cast<const void*>(wide_gemm_kernel), kSlotWide, pl->device, pl->smem_bytes) != cudaSuccess) {
+    note_cuda_error("cudaFuncSetAttribute", cudaGetErrorName(cudaGetLastError()));
+    return GEMM_ERR_CUDA;
   }
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof cfg);
@@ -667,7 +663,7 @@ gemm_status_t run_skinny(gemm_plan_s* pl, const void* A, const void* B, void* C,
   p.counters = reinterpret_cast<uint32_t*>(workspace);
   p.status = pl->d_status;
   p.timeout_ns = static_cast<unsigned long long>(pl->timeout_ms) * 1000000ull;
-  return static_cast<gemm_status_t>(skinny_launch(p, tW, tX, stream, g_last_cuda_error, sizeof g_last_cuda_error));
+  return static_cast<gemm_status_t>(skinny_launch(p, tW, tX, pl->device, stream, g_last_cuda_error, sizeof g_last_cuda_error));
 }
 
 }  // namespace
@@ -684,6 +680,8 @@ extern "C" gemm_status_t gemm_run(gemm_plan_t plan, const void* A, const void* B
     if (misaligned(workspace)) return GEMM_ERR_ALIGNMENT;
   }
   if (!plan->has_device || !plan->arch_ok || !plan->d_status) return GEMM_ERR_ARCH;
+  int cur = -1;
+  if (cudaGetDevice(&cur) != cudaSuccess || cur != plan->device) return GEMM_ERR_INVALID_ARG;  // plan belongs to another device
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (plan->variant == GEMM_VARIANT_SKINNY_STREAMK) return run_skinny(plan, A, B, C, bias, alpha, beta, workspace, s);
   return run_dense(plan, A, B, C, bias, alpha, beta, s);
@@ -805,7 +803,7 @@ extern "C" gemm_status_t gemm_skinny_run_noalloc(const gemm_desc_t* desc, const 
   p.counters = reinterpret_cast<uint32_t*>(nd.scratch + kNoAllocHeaderBytes);
   p.partials = reinterpret_cast<float*>(nd.scratch + kNoAllocHeaderBytes + sp.counters_bytes);
   p.timeout_ns = 2000ull * 1000000ull;
-  st = static_cast<gemm_status_t>(skinny_launch(p, tW, tX, s, g_last_cuda_error, sizeof g_last_cuda_error));
+  st = static_cast<gemm_status_t>(skinny_launch(p, tW, tX, dev, s, g_last_cuda_error, sizeof g_last_cuda_error));
   if (st != GEMM_OK || !sync_and_check) return st;
   uint32_t word = 0;
   e = cudaStreamSynchronize(s);

@@ -18,6 +18,7 @@
 #include <cuda_runtime.h>
 
 #include "dense_kernel.cuh"
+#include "launch_util.cuh"
 
 namespace b200 {
 
@@ -315,14 +316,9 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
 }
 
 // Zero the arrival counters and launch.  Returns a gemm_status_t value (0 = ok, 7 = CUDA failure).
-inline int skinny_launch(const SkinnyParams& p, const CUtensorMap& tW, const CUtensorMap& tX, cudaStream_t stream, char* err,
-                         size_t err_len) {
-  static thread_local int configured_smem = 0;
-  cudaError_t e = cudaSuccess;
-  if (configured_smem < p.plan.smem_bytes) {
-    e = cudaFuncSetAttribute(skinny_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, p.plan.smem_bytes);
-    if (e == cudaSuccess) configured_smem = p.plan.smem_bytes;
-  }
+inline int skinny_launch(const SkinnyParams& p, const CUtensorMap& tW, const CUtensorMap& tX, int device, cudaStream_t stream,
+                         char* err, size_t err_len) {
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(skinny_gemm_kernel), kSlotSkinny, device, p.plan.smem_bytes);
   if (e == cudaSuccess) e = cudaMemsetAsync(p.counters, 0, p.plan.counters_bytes, stream);
   if (e == cudaSuccess) {
     skinny_gemm_kernel<<<p.plan.grid, kSkinnyThreads, p.plan.smem_bytes, stream>>>(tW, tX, p);

@@ -2,7 +2,9 @@
 C-ABI binding, evaluate the oracle on the checked rows / columns and compare.
 
 Acceptance (per checked element, against the UNROUNDED fp64 oracle value y):
-    |D_gpu - y| <= 2e-3 * (|alpha| * sum_k |a||b| + |beta| * |C_in| + |bias_j|) + 1e-5
+    |D_gpu - y| <= 2e-3 * (|alpha| * sum_k |a||b| + |beta| * |C_in| + |bias_j|) + 1e-5  (+ u_out * |y| for a 16-bit
+    output: when there is no cancellation, |y| equals the sum in the first term and rounding y to bf16 alone can
+    move it by 2^-8 |y| = 3.9e-3 |y|, more than the 2e-3 allows)
 and, over each checked block, the relative Frobenius error
     fp32 output  : ||D_gpu - y||_F / ||y||_F <= 1e-4
     16-bit output: every element within one unit in the last place of RNE(y -> output dtype)
@@ -102,7 +104,7 @@ def run_gpu(w: wl.Workload, inputs: dict, flags: int = 0, c_dtype=None, poison: 
                 raise bg.GemmError(st, "gemm_plan_status")
             outs.append(to_host_bits(C, cd))
         for o in outs[1:]:
-            assert np.array_equal(o, outs[0]), "run-to-run results differ bitwise"
+            assert o.tobytes() == outs[0].tobytes(), "run-to-run results differ bitwise"   # (NaN-poisoned padding included)
         return outs[0], plan.info
     finally:
         plan.close()
@@ -117,7 +119,8 @@ def gather(cbits: np.ndarray, w: wl.Workload, batches, rows, cols) -> np.ndarray
 def compare_block(got_bits: np.ndarray, y: np.ndarray, bound: np.ndarray, c_dtype: int) -> dict:
     got = oracle.decode(got_bits, c_dtype)
     err = np.abs(got - y)
-    tol = REL_TOL * bound + ABS_TOL
+    # a 16-bit output may sit half an ulp (relative 2^-8 / 2^-11 at the bottom of a binade) from y by rounding alone
+    tol = REL_TOL * bound + ABS_TOL + U_OUT[c_dtype] * np.abs(y)
     ref_bits = oracle.round_to(y, c_dtype)
     ref = oracle.decode(ref_bits, c_dtype) if c_dtype != wl.F32 else y
     denom = float(np.linalg.norm(ref.ravel()))

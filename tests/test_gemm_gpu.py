@@ -33,6 +33,11 @@ EXACT_CASES = [
     ("tile_n_192", 256, 576, 192, {}, dict(variant=V1, tile_n=192)),
     ("ragged_all", 200, 328, 200, {}, dict(variant=V1, tile_n=128)),
     ("tiny", 1, 8, 8, {}, dict(variant=V1)),
+    ("one_by_one_by_one", 1, 1, 1, dict(lda=8, ldb=8, ldc=4), dict(variant=V1)),
+    ("one_by_one_by_one_skinny", 1, 1, 1, dict(lda=8, ldb=8, ldc=4), dict(variant=VS)),
+    ("many_small_batches", 64, 64, 64, dict(batch=300, cd=wl.BF16), dict(variant=V1)),
+    ("very_long_k", 128, 64, 65536, {}, dict(variant=V1)),
+    ("very_wide_n", 128, 70000, 64, dict(cd=wl.BF16), dict(variant=V1)),
     ("m1_n_ragged", 1, 1000, 72, {}, dict(variant=V1)),
     ("n_small", 300, 8, 136, {}, dict(variant=V1)),
     ("persistent_many_tiles", 1536, 2560, 128, {}, dict(variant=V1, tile_n=64)),
