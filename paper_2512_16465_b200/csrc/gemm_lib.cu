@@ -467,7 +467,7 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
     return st;
   }
   if (pl->has_device && pl->arch_ok) {
-    if (cudaMalloc(&pl->d_status, 256) != cudaSuccess || cudaMemset(pl->d_status, 0, 256) != cudaSuccess) {
+    if (cudaMalloc(&pl->d_status, 16) != cudaSuccess || cudaMemset(pl->d_status, 0, 16) != cudaSuccess) {
       note_cuda_error("cudaMalloc(status word)", cudaGetErrorName(cudaGetLastError()));
       delete pl;
       return GEMM_ERR_CUDA;
@@ -661,6 +661,7 @@ gemm_status_t run_skinny(gemm_plan_s* pl, const void* A, const void* B, void* C,
   p.ldc = d.ldc;
   p.partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + s.counters_bytes);
   p.counters = reinterpret_cast<uint32_t*>(workspace);
+  p.debug_flags = (d.flags & GEMM_FLAG_DEBUG_STALL) ? 1u : 0u;
   p.status = pl->d_status;
   p.timeout_ns = static_cast<unsigned long long>(pl->timeout_ms) * 1000000ull;
   return static_cast<gemm_status_t>(skinny_launch(p, tW, tX, pl->device, stream, g_last_cuda_error, sizeof g_last_cuda_error));

@@ -81,6 +81,7 @@ struct SkinnyParams {
   uint32_t* counters;     // workspace: one arrival counter per n-tile, zero at launch
   uint32_t* status;
   unsigned long long timeout_ns;
+  uint32_t debug_flags;   // bit 0: withhold one producer arrival (timeout test hook)
 };
 
 __device__ __forceinline__ float sk_load_c(const SkinnyParams& p, long long idx) {
@@ -177,7 +178,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
       if (!mbar_wait_warp(empty0 + 8u * s, ph ^ 1u, w, (1u << 8) | s)) break;
       const uint32_t bar = full0 + 8u * s;
       const uint32_t sw_ = base + s * sp.stage_bytes;
-      if (elect_one()) {
+      if (elect_one() && !((p.debug_flags & 1u) && i == 0)) {  // test hook: the first stage is never filled nor signalled
         mbar_arrive_expect_tx(bar, sp.stage_bytes);
         tma_load_3d(sw_, &tmW, bar, kb * kBlockK, tile * kSkinnyTileN, 0, pol_w);
         tma_load_3d(sw_ + kSkinnyTileN * 128u, &tmX, bar, kb * kBlockK, 0, 0, pol_x);

@@ -255,13 +255,13 @@ def test_runs_on_a_side_stream():
     plan.close()
 
 
-@pytest.mark.parametrize("variant", [V1, V2, VW])
+@pytest.mark.parametrize("variant", [V1, V2, VW, VS])
 def test_bounded_wait_reports_timeout_and_context_survives(variant):
     """A producer arrival is withheld by a test flag, so a device-side wait runs into its limit; the
     kernel must return on its own, the plan must report GEMM_ERR_TIMEOUT and later work must run."""
-    w = int_workload("stall", 512, 512, 256)
+    w = int_workload("stall", 8 if variant == VS else 512, 512, 256)
     inputs = wl.make_inputs(w)
-    tile_n = 0 if variant == VW else 128
+    tile_n = 0 if variant in (VW, VS) else 128
     plan = bg.Plan(H.desc_of(w, bg.make_flags(variant, tile_n, debug_stall=True)))
     plan.set_timeout_ms(20)
     A, B = H.to_device(inputs["A"], w.ab_dtype), H.to_device(inputs["B"], w.ab_dtype)
