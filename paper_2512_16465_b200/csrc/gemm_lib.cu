@@ -147,6 +147,41 @@ int dense_smem_bytes(int stages, int a_stage, int b_stage, int epi_wg) {  // a_s
   return 1024 /*alignment slack*/ + stages * (a_stage + b_stage) + 4 * epi_wg * 2 * kSlabBytes + 16 * kMaxStages + 64;
 }
 
+// Plan-time roofline estimate (Section 4.3 applied per kernel candidate): cycles one SM spends on its share of the
+// problem with a given kernel family and tile width.  Per tile the slowest of three resources decides -- the tensor
+// pipe (with the family's measured streaming efficiency), the L2 -> SM operand feed and the HBM write share -- plus
+// what the family leaves exposed per tile; tiles are dealt out in waves over the SMs (or SM pairs).
+struct DenseCandidate {
+  int variant;
+  int bn;
+  double cycles;
+};
+double estimate_dense_cycles(const gemm_desc_t& d, int sm_count, int variant, int bn) {
+  const bool wide = variant == GEMM_VARIANT_DENSE_2CTA_WIDE;
+  const int cg = variant == GEMM_VARIANT_DENSE_1CTA ? 1 : 2;
+  const int rows_cta = wide ? kWideCtaM : kCtaM;
+  const int rows_tile = rows_cta * cg;
+  const int units = std::max(1, sm_count / cg);
+  const long long tiles = static_cast<long long>(ceil_div(d.M, rows_tile)) * ceil_div(d.N, bn) * d.batch_count;
+  const long long waves = (tiles + units - 1) / units;
+  const double kblocks = static_cast<double>(ceil_div(d.K, kBlockK));
+  // tensor pipe: one 128 x bn x 16 MMA per CTA takes bn / 2 cycles; four per k-block and 128-row half
+  static const double eff1[3] = {0.45, 0.68, 0.88}, eff2[3] = {0.55, 0.80, 0.95};  // bn = 64, 128, 256 (measured, 8192^3)
+  const int bi = bn <= 64 ? 0 : (bn <= 128 ? 1 : 2);
+  const double eff = wide ? 1.0 : (cg == 1 ? eff1[bi] : eff2[bi]);
+  const double mma = kblocks * 4.0 * (bn / 2.0) * (rows_cta / 128.0) / eff;
+  // operand feed: bytes this SM receives per k-block at ~90 B/clk
+  const double feed = kblocks * (rows_cta + static_cast<double>(bn) / cg) * 128.0 / 90.0;
+  // output: this SM's share of the HBM write bandwidth is ~16 B/clk
+  const double out = static_cast<double>(rows_cta) * bn * elem_bytes(d.c_dtype) / 16.0;
+  const bool gelu = d.epilogue >= GEMM_EPI_GELU_ERF;
+  double exposed = 400.0;                       // barrier round trips per tile that nothing hides
+  if (wide) exposed = gelu ? 9000.0 : 3000.0;   // no second accumulator: read-out (and conversion) of half 0
+  else if (cg == 2) exposed = 1000.0;           // pair hand-shakes cross the SM-to-SM network
+  const double per_tile = std::max(mma, std::max(feed, out)) + exposed;
+  return static_cast<double>(waves) * per_tile + 3000.0;  // + pipeline fill and drain
+}
+
 // Fill plan->dense and the launch geometry for a dense variant.
 gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_raster, int forced_stages, int forced_atoms) {
   const gemm_desc_t& d = pl->d;
@@ -189,7 +224,7 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   // A tile's main loop lasts about 512 cycles per 64 columns of K (at tile N = 256); draining 128 x 256 accumulators
   // with four warps takes several thousand.  Short-K (output-bound) problems with several tiles per CTA get a second
   // epilogue warpgroup.
-  const int epi_wg = (!single_wave && static_cast<long long>(ceil_div(d.K, kBlockK)) * 2 * bn <= 8192) ? 2 : 1;
+  const int epi_wg = (!single_wave && static_cast<long long>(ceil_div(d.K, kBlockK)) * 2 * bn <= 4096) ? 2 : 1;
   int stages = forced_stages;
   if (stages == 0) {
     stages = (kMaxSmemOptin - dense_smem_bytes(0, a_stage, b_stage, epi_wg)) / (a_stage + b_stage);
@@ -436,29 +471,33 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
   const int forced_stages = (d.flags & GEMM_FLAG_STAGES_MASK) >> GEMM_FLAG_STAGES_SHIFT;
   const int forced_atoms = (d.flags & GEMM_FLAG_KSLICES_MASK) >> GEMM_FLAG_KSLICES_SHIFT;
   int variant = forced_variant;
+  int auto_bn = 0;  // tile width chosen together with the variant
   if (variant == 0) {
     // memory-bound problems with a handful of rows stream the weight matrix once: stream-K path;
     // everything else is a dense tiled GEMM, paired CTAs when there are at least two tile rows
     const bool skinny_ok = d.M <= kSkinnyMaxM && d.batch_count == 1 && d.transa == GEMM_OP_N && d.transb == GEMM_OP_T;
-    // a CTA pair halves the B traffic per SM; it pays once there are enough 256-row tiles to occupy every pair
-    const long long pair_tiles = static_cast<long long>(ceil_div(d.M, 2 * kCtaM)) * ceil_div(d.N, 256) * d.batch_count;
-    if (skinny_ok && info.intensity < 5.2 * kRidgeCudaCore) variant = GEMM_VARIANT_SKINNY_STREAMK;  // measured: wins up to M ~ 48
-    else if (d.M > kCtaM && d.K >= 512 && pair_tiles >= pl->sm_count / 2) {
-      variant = GEMM_VARIANT_DENSE_2CTA;
-      // The 512 x 256 variant moves a quarter less operand data per FLOP (it runs ~4 % faster at the power cap) but
-      // exposes part of its epilogue: taken for long K, cheap epilogues and when its last wave is about as full.
-      const int pairs = pl->sm_count / 2;
-      const long long wide_tiles = static_cast<long long>(ceil_div(d.M, 2 * kWideCtaM)) * ceil_div(d.N, kWideTileN) * d.batch_count;
-      const double eff_pair = static_cast<double>(pair_tiles) / (static_cast<double>(ceil_div(pair_tiles, pairs)) * pairs);
-      const double eff_wide = static_cast<double>(wide_tiles) / (static_cast<double>(ceil_div(wide_tiles, pairs)) * pairs);
-      const bool cheap_epilogue = d.epilogue < GEMM_EPI_GELU_ERF;
-      if (cheap_epilogue && d.K >= 4096 && d.M >= 2 * kWideCtaM && wide_tiles >= pairs && eff_wide >= eff_pair - 0.02)
-        variant = GEMM_VARIANT_DENSE_2CTA_WIDE;
+    if (skinny_ok && info.intensity < 5.2 * kRidgeCudaCore) {
+      variant = GEMM_VARIANT_SKINNY_STREAMK;  // measured: wins up to M ~ 48
+    } else {
+      // score every dense family and tile width with the roofline estimate and take the cheapest
+      const bool b_kmajor = d.transb == GEMM_OP_T;
+      DenseCandidate best{GEMM_VARIANT_DENSE_1CTA, 64, 1e300};
+      for (int v : {GEMM_VARIANT_DENSE_1CTA, GEMM_VARIANT_DENSE_2CTA, GEMM_VARIANT_DENSE_2CTA_WIDE}) {
+        for (int bn : {256, 128, 64}) {
+          if (v == GEMM_VARIANT_DENSE_2CTA_WIDE && bn != kWideTileN) continue;
+          if (v == GEMM_VARIANT_DENSE_2CTA && !b_kmajor && bn % 128) continue;  // 64-column boxes per CTA
+          if (v != GEMM_VARIANT_DENSE_1CTA && d.M <= kCtaM) continue;           // a pair needs two tile rows
+          if (forced_bn && bn != forced_bn) continue;
+          const double c = estimate_dense_cycles(d, pl->sm_count, v, bn);
+          if (c < best.cycles * 0.995) best = DenseCandidate{v, bn, c};          // ties go to the earlier, simpler one
+        }
+      }
+      variant = best.variant;
+      auto_bn = best.bn;
     }
-    else variant = GEMM_VARIANT_DENSE_1CTA;
   }
-  if (variant == GEMM_VARIANT_DENSE_1CTA) st = plan_dense(pl, 1, forced_bn, forced_raster, forced_stages, forced_atoms);
-  else if (variant == GEMM_VARIANT_DENSE_2CTA) st = plan_dense(pl, 2, forced_bn, forced_raster, forced_stages, forced_atoms);
+  if (variant == GEMM_VARIANT_DENSE_1CTA) st = plan_dense(pl, 1, forced_bn ? forced_bn : auto_bn, forced_raster, forced_stages, forced_atoms);
+  else if (variant == GEMM_VARIANT_DENSE_2CTA) st = plan_dense(pl, 2, forced_bn ? forced_bn : auto_bn, forced_raster, forced_stages, forced_atoms);
   else if (variant == GEMM_VARIANT_SKINNY_STREAMK) st = plan_skinny(pl, forced_stages);
   else if (variant == GEMM_VARIANT_DENSE_2CTA_WIDE) st = plan_wide(pl, forced_raster, forced_stages);
   else st = GEMM_ERR_INVALID_ARG;
