@@ -155,3 +155,21 @@ def test_product_package_does_not_import_the_oracle():
             if f.endswith((".py", ".cu", ".cuh", ".h")):
                 text = open(os.path.join(dirpath, f)).read()
                 assert "oracle" not in text.lower(), f"{f} mentions the oracle"
+
+
+def test_cost_model_choices_follow_the_measurements():
+    """The plan scores (family, tile width) candidates with a roofline estimate; these are shapes whose best
+    family was measured on a B200."""
+    def choice(M, N, K, **kw):
+        h = bg.gemm_plan(bg.make_desc(M, N, K, c_dtype=bg.BF16, **kw))
+        i = bg.gemm_plan_info(h)
+        bg.gemm_destroy(h)
+        return i["variant"], i["tile_n"]
+    assert choice(2048, 2048, 2048) == (bg.VARIANT_DENSE_2CTA, 256)          # 64 pair tiles on 74 pairs beat 256 small ones
+    assert choice(4096, 4096, 4096) == (bg.VARIANT_DENSE_2CTA_WIDE, 256)
+    assert choice(128, 28672, 8192) == (bg.VARIANT_DENSE_1CTA, 256)          # one tile row: no pair
+    assert choice(16384, 14336, 4096, epilogue=bg.EPI_BIAS_GELU_ERF)[0] == bg.VARIANT_DENSE_2CTA
+    assert choice(16, 28672, 8192)[0] == bg.VARIANT_SKINNY_STREAMK
+    assert choice(64, 28672, 8192)[0] == bg.VARIANT_DENSE_1CTA               # stream-K stops paying near M = 48
+    v, bn = choice(2048, 2048, 128, batch=64)
+    assert (v, bn) == (bg.VARIANT_DENSE_1CTA, 256)                           # output-bound: widest tile, fewest hand-shakes
