@@ -40,7 +40,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the full-size ncu captures
 # summarised under profiles/ (dense_*_cN_*.txt, skinny_streamk_c5_*.txt; last line of each file).
-NCU_TRAFFIC_BYTES = {"c1": 1122304, "c2": 871786752, "c3": 1633176128, "c4": 544957440, "c5": 476399616}
+NCU_TRAFFIC_BYTES = {"c1": 1122048, "c2": 882350848, "c3": 1645141584, "c4": 545059072, "c5": 476179200}
 
 
 def load_peaks():
