@@ -383,6 +383,83 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def parse_shape(spec: str) -> wl.Workload:
+    """'MxNxK' followed by optional ':key=value' fields: batch, ta, tb (1 = stored transposed), ab/cd (bf16|f16|f32),
+    epi (none|bias|relu|bias_relu|gelu|bias_gelu), alpha, beta, lda, ldb, ldc.  Example: 28672x8x8192:beta=1:cd=f32."""
+    head, *fields = spec.split(":")
+    M, N, K = (int(x) for x in head.lower().split("x"))
+    dt = {"bf16": wl.BF16, "f16": wl.F16, "f32": wl.F32}
+    epi = {"none": wl.EPI_NONE, "bias": wl.EPI_BIAS, "relu": wl.EPI_RELU, "bias_relu": wl.EPI_BIAS_RELU,
+           "gelu": wl.EPI_GELU_ERF, "bias_gelu": wl.EPI_BIAS_GELU_ERF}
+    kw = dict(c_dtype=wl.BF16, dist_a=wl.Dist("normal", 0.0, 0.02), dist_b=wl.Dist("normal", 0.0, 0.02))
+    for f in fields:
+        k, v = f.split("=")
+        if k == "batch":
+            kw["batch"] = int(v)
+        elif k in ("ta", "tb"):
+            kw["transa" if k == "ta" else "transb"] = int(v)
+        elif k in ("ab", "cd"):
+            kw["ab_dtype" if k == "ab" else "c_dtype"] = dt[v]
+        elif k == "epi":
+            kw["epilogue"] = epi[v]
+        elif k in ("alpha", "beta"):
+            kw[k] = float(v)
+        elif k in ("lda", "ldb", "ldc"):  # leading dimensions in elements (each must span a multiple of 16 bytes)
+            kw[k] = int(v)
+        else:
+            raise SystemExit(f"unknown field {k!r} in --shapes")
+    return wl.Workload(spec, M, N, K, **kw)
+
+
+def run_shapes(args):
+    """Time arbitrary problem shapes with the automatic plan (sweeps beyond the five configurations): one JSON line
+    whose `shapes_measured` holds, per shape, the plan taken, the time per launch and the roofline entry."""
+    import torch
+    import paper_2512_16465_b200 as bg
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+        raise SystemExit("--shapes is a single-GPU sweep")
+    torch.cuda.set_device(0)
+    device = torch.device("cuda", 0)
+    peaks, peak_kind = load_peaks()
+    steps, warmup = args.steps, max(3, args.warmup)
+    rows = []
+    with ClockSampler(0) as clocks:
+        for spec in args.shapes.split(";"):
+            w = parse_shape(spec.strip())
+            case = DeviceCase(torch, bg, spec, w, int(args.flags, 0), device)
+            torch.cuda.synchronize()
+            time.sleep(0.3)
+            sec = case.time_steps(steps, warmup)
+            row = {"shape": spec, "ms_per_step": round(sec * 1e3, 5), "tflops": round(metric_value(w, sec), 2),
+                   "gbs": round(w.min_bytes / sec / 1e9, 1), "input_sets": case.nsets,
+                   "plan": {k: case.plan.info[k] for k in ("variant", "tile_m", "tile_n", "stages", "cluster_size", "grid", "split")},
+                   "roofline": roofline_for(w, spec, sec, peaks, peak_kind)}
+            if args.library_reference and w.batch == 1 and w.epilogue == wl.EPI_NONE and w.beta == 0.0 and w.alpha == 1.0:
+                # context only: the vendor library on the same operands (no part of the product)
+                A, B, _, _ = case.sets[0]
+                a2 = A[: (w.K if w.transa else w.M) * w.lda].view(-1, w.lda)
+                b2 = B[: (w.N if w.transb else w.K) * w.ldb].view(-1, w.ldb)
+                opa = a2[:, : w.M].t() if w.transa else a2[:, : w.K]
+                opb = b2[:, : w.K].t() if w.transb else b2[:, : w.N]
+                for _ in range(warmup):
+                    torch.matmul(opa, opb)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                e0.record()
+                for _ in range(steps):
+                    torch.matmul(opa, opb)
+                e1.record()
+                torch.cuda.synchronize()
+                row["library_reference_ms"] = round(e0.elapsed_time(e1) / steps, 5)
+            rows.append(row)
+            case.close()
+    print(json.dumps({"shapes_measured": rows, "steps": steps, "warmup": warmup, "clocks": clocks.summary(),
+                      "timing": "CUDA events around back-to-back launches; inputs rotate so that each step's footprint exceeds L2"}), flush=True)
+
+
 def run_reference(args):
     """The reference arm of this build is the CPU oracle: K steps, each a bounded sample."""
     rank = int(os.environ.get("RANK", "0"))
@@ -441,9 +518,13 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--ref-step-seconds", type=float, default=10.0, help="--impl reference: CPU time budget of one step")
+    ap.add_argument("--shapes", default="", help="';'-separated MxNxK[:key=value...] problems to time instead of the five configurations")
+    ap.add_argument("--library-reference", action="store_true", help="--shapes: also time torch.matmul on the same operands (context)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.shapes:
+        run_shapes(args)
     else:
         run_ours(args)
 

@@ -73,7 +73,7 @@ typedef enum { GEMM_REGIME_MEMORY = 0, GEMM_REGIME_MIDDLE = 1, GEMM_REGIME_COMPU
 typedef enum {
   GEMM_VARIANT_DENSE_1CTA = 1,      /* 128 x N tile per CTA, accumulator double buffered */
   GEMM_VARIANT_DENSE_2CTA = 2,      /* CTA pair, 256 x N pair tile, accumulator double buffered */
-  GEMM_VARIANT_SKINNY_STREAMK = 3,  /* M <= 64: stream-K over the weight matrix */
+  GEMM_VARIANT_SKINNY_STREAMK = 3,  /* M <= 64 or N <= 64 (transa = N, transb = T, no batch): stream-K over the long operand */
   GEMM_VARIANT_DENSE_2CTA_WIDE = 4  /* CTA pair, 512 x 256 pair tile: least operand traffic per FLOP */
 } gemm_variant_t;
 
@@ -111,7 +111,7 @@ typedef struct {
   uint32_t struct_size;  /* = sizeof(gemm_info_t), set by the caller */
   int32_t variant;       /* gemm_variant_t */
   int32_t regime;        /* gemm_regime_t */
-  int32_t tile_m, tile_n, tile_k; /* output tile of one CTA (1-CTA) or CTA pair (2-CTA); skinny: tile over N, M-pad, K */
+  int32_t tile_m, tile_n, tile_k; /* output tile of one CTA (1-CTA) or CTA pair (2-CTA); skinny: tile over the long extent, padded short extent, K */
   int32_t stages;        /* depth of the shared-memory ring */
   int32_t cluster_size;  /* 1 or 2 */
   int32_t grid;          /* CTAs launched */

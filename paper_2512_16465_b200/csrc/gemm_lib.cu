@@ -108,6 +108,7 @@ struct gemm_plan_s {
   uint32_t timeout_ms;
   DenseParams dense;     // filled at plan time except pointers / scalars
   SkinnyPlan skinny;     // stream-K decomposition of the skinny variant
+  bool skinny_tall = false;  // the short output extent is N (A is the streamed operand), not M
 };
 
 namespace {
@@ -392,13 +393,15 @@ gemm_status_t plan_wide(gemm_plan_s* pl, int forced_raster, int forced_stages) {
   return GEMM_OK;
 }
 
-gemm_status_t plan_skinny(gemm_plan_s* pl, int forced_stages) {
+gemm_status_t plan_skinny(gemm_plan_s* pl, int forced_stages, int forced_atoms) {
   const gemm_desc_t& d = pl->d;
   if (d.transa != GEMM_OP_N || d.transb != GEMM_OP_T) return GEMM_ERR_UNSUPPORTED;  // both operands K-contiguous
-  if (d.M > kSkinnyMaxM || d.batch_count != 1) return GEMM_ERR_UNSUPPORTED;
+  if ((d.M > kSkinnyMaxM && d.N > kSkinnyMaxM) || d.batch_count != 1) return GEMM_ERR_UNSUPPORTED;
   SkinnyPlan& s = pl->skinny;
-  if (!skinny_make_plan(&s, static_cast<int>(d.M), static_cast<int>(d.N), static_cast<int>(d.K), pl->sm_count, forced_stages,
-                        kMaxSmemOptin))
+  pl->skinny_tall = d.M > kSkinnyMaxM;  // the short extent is N: A is streamed, B is the resident slab
+  const int small_extent = static_cast<int>(pl->skinny_tall ? d.N : d.M), big_extent = static_cast<int>(pl->skinny_tall ? d.M : d.N);
+  if (forced_atoms > 3) return GEMM_ERR_UNSUPPORTED;
+  if (!skinny_make_plan(&s, small_extent, big_extent, static_cast<int>(d.K), pl->sm_count, forced_stages, kMaxSmemOptin, forced_atoms))
     return GEMM_ERR_UNSUPPORTED;
   pl->variant = GEMM_VARIANT_SKINNY_STREAMK;
   pl->cg = 1;
@@ -407,9 +410,10 @@ gemm_status_t plan_skinny(gemm_plan_s* pl, int forced_stages) {
   pl->smem_bytes = s.smem_bytes;
   gemm_info_t& info = pl->info;
   info.variant = pl->variant;
-  info.tile_m = kSkinnyTileN;  // rows of the weight matrix (output columns) per tile
+  // 128 rows of the streamed operand per tile; the short extent padded to a multiple of 16
+  info.tile_m = kSkinnyTileN;
   info.tile_n = s.m_pad;
-  info.tile_k = kBlockK;
+  info.tile_k = kBlockK * s.atoms;
   info.stages = s.stages;
   info.cluster_size = 1;
   info.grid = s.grid;
@@ -475,7 +479,7 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
   if (variant == 0) {
     // memory-bound problems with a handful of rows stream the weight matrix once: stream-K path;
     // everything else is a dense tiled GEMM, paired CTAs when there are at least two tile rows
-    const bool skinny_ok = d.M <= kSkinnyMaxM && d.batch_count == 1 && d.transa == GEMM_OP_N && d.transb == GEMM_OP_T;
+    const bool skinny_ok = (d.M <= kSkinnyMaxM || d.N <= kSkinnyMaxM) && d.batch_count == 1 && d.transa == GEMM_OP_N && d.transb == GEMM_OP_T;
     if (skinny_ok && info.intensity < 5.2 * kRidgeCudaCore) {
       variant = GEMM_VARIANT_SKINNY_STREAMK;  // measured: wins up to M ~ 48
     } else {
@@ -498,7 +502,7 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
   }
   if (variant == GEMM_VARIANT_DENSE_1CTA) st = plan_dense(pl, 1, forced_bn ? forced_bn : auto_bn, forced_raster, forced_stages, forced_atoms);
   else if (variant == GEMM_VARIANT_DENSE_2CTA) st = plan_dense(pl, 2, forced_bn ? forced_bn : auto_bn, forced_raster, forced_stages, forced_atoms);
-  else if (variant == GEMM_VARIANT_SKINNY_STREAMK) st = plan_skinny(pl, forced_stages);
+  else if (variant == GEMM_VARIANT_SKINNY_STREAMK) st = plan_skinny(pl, forced_stages, forced_atoms);
   else if (variant == GEMM_VARIANT_DENSE_2CTA_WIDE) st = plan_wide(pl, forced_raster, forced_stages);
   else st = GEMM_ERR_INVALID_ARG;
   if (st != GEMM_OK) {
@@ -680,9 +684,16 @@ gemm_status_t run_skinny(gemm_plan_s* pl, const void* A, const void* B, void* C,
   const gemm_desc_t& d = pl->d;
   const SkinnyPlan& s = pl->skinny;
   CUtensorMap tW, tX;
-  // weights W = B stored N x K (K contiguous): box 64 x 128; activations X = A stored M x K: box 64 x m_pad
-  bool ok = encode_map(&tW, d.ab_dtype, B, d.K, d.N, 1, d.ldb, 0, kBlockK, kSkinnyTileN);
-  ok = ok && encode_map(&tX, d.ab_dtype, A, d.K, d.M, 1, d.lda, 0, kBlockK, s.m_pad);
+  // weights W = B stored N x K (K contiguous): box 64 x 128; activations X = A stored M x K: box 64 x m_pad;
+  // a tall problem streams A in W's place and keeps B as the slab
+  bool ok;
+  if (pl->skinny_tall) {
+    ok = encode_map(&tW, d.ab_dtype, A, d.K, d.M, 1, d.lda, 0, kBlockK, kSkinnyTileN);
+    ok = ok && encode_map(&tX, d.ab_dtype, B, d.K, d.N, 1, d.ldb, 0, kBlockK, s.m_pad);
+  } else {
+    ok = encode_map(&tW, d.ab_dtype, B, d.K, d.N, 1, d.ldb, 0, kBlockK, kSkinnyTileN);
+    ok = ok && encode_map(&tX, d.ab_dtype, A, d.K, d.M, 1, d.lda, 0, kBlockK, s.m_pad);
+  }
   if (!ok) return GEMM_ERR_CUDA;
   SkinnyParams p;
   memset(&p, 0, sizeof p);
@@ -703,7 +714,8 @@ gemm_status_t run_skinny(gemm_plan_s* pl, const void* A, const void* B, void* C,
   p.debug_flags = (d.flags & GEMM_FLAG_DEBUG_STALL) ? 1u : 0u;
   p.status = pl->d_status;
   p.timeout_ns = static_cast<unsigned long long>(pl->timeout_ms) * 1000000ull;
-  return static_cast<gemm_status_t>(skinny_launch(p, tW, tX, pl->device, stream, g_last_cuda_error, sizeof g_last_cuda_error));
+  return static_cast<gemm_status_t>(
+      skinny_launch(p, tW, tX, pl->device, stream, g_last_cuda_error, sizeof g_last_cuda_error, pl->skinny_tall));
 }
 
 }  // namespace

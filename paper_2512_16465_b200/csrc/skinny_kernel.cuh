@@ -12,6 +12,10 @@
 //     order (deterministic, no floating-point atomics), applies the epilogue and writes D.
 //     Nobody ever waits for another CTA.
 //
+// The same kernel serves the mirrored case, a tall output with a handful of columns (N <= 64 < M, kTall): the long
+// operand A[M x K] then takes W's place and B[N x K] takes X's; only the addressing of C, D and the bias differs.
+// Below, "big" is the long output extent (128 per tile, on the TMEM lanes) and "small" the short one.
+//
 // Roles per CTA (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer and owner of the TMEM allocation
 // (both warp-uniform, one elected lane issues), warps 2-5 = epilogue / fix-up.
 #pragma once
@@ -27,13 +31,14 @@ constexpr int kSkinnyMaxM = 64;     // largest M the skinny path takes
 constexpr int kSkinnyThreads = 192;
 
 struct SkinnyPlan {
-  int m_pad;             // M rounded up to a multiple of 16 (the MMA's N extent)
-  int n_tiles;           // ceil(N / 128)
-  int kbs;               // k-blocks per tile = ceil(K / 64)
+  int m_pad;             // small extent rounded up to a multiple of 16 (the MMA's N extent)
+  int n_tiles;           // ceil(big extent / 128)
+  int atoms;             // 64-wide K slices per pipeline stage (each slice is one 128-byte swizzle atom per row)
+  int kbs;               // work units per tile = ceil(K / (64 * atoms))
   long long total_units; // n_tiles * kbs
   int grid;              // CTAs = min(SM count, total_units)
   int stages;
-  int stage_bytes;       // 16 KB of W + m_pad * 128 bytes of X
+  int stage_bytes;       // atoms x (16 KB of W + m_pad * 128 bytes of X)
   int smem_bytes;
   int max_contributors;  // upper bound on CTAs touching one tile
   size_t counters_bytes; // workspace: [counters (n_tiles x u32, padded)] [partials: grid * 2 slots]
@@ -44,18 +49,22 @@ struct SkinnyPlan {
 __host__ __device__ inline long long sk_begin(long long c, long long T, long long G) { return c * T / G; }
 __host__ __device__ inline int sk_owner(long long u, long long T, long long G) { return static_cast<int>(((u + 1) * G - 1) / T); }
 
-inline bool skinny_make_plan(SkinnyPlan* s, int M, int N, int K, int sm_count, int forced_stages, int max_smem) {
+// M is the small output extent and N the big one (for a tall problem the caller passes them swapped).
+inline bool skinny_make_plan(SkinnyPlan* s, int M, int N, int K, int sm_count, int forced_stages, int max_smem, int forced_atoms = 0) {
   if (M < 1 || M > kSkinnyMaxM) return false;
   s->m_pad = ((M + 15) / 16) * 16;
   s->n_tiles = (N + kSkinnyTileN - 1) / kSkinnyTileN;
-  s->kbs = (K + kBlockK - 1) / kBlockK;
+  // Two adjacent 128-byte pieces of every weight row are requested together when K is long enough: DRAM then serves
+  // both from one open row.
+  s->atoms = forced_atoms ? forced_atoms : (K >= 1024 ? 2 : 1);
+  s->kbs = (K + kBlockK * s->atoms - 1) / (kBlockK * s->atoms);
   s->total_units = static_cast<long long>(s->n_tiles) * s->kbs;
   s->grid = static_cast<int>(s->total_units < sm_count ? s->total_units : sm_count);
-  s->stage_bytes = kSkinnyTileN * 128 + s->m_pad * 128;
+  s->stage_bytes = s->atoms * (kSkinnyTileN * 128 + s->m_pad * 128);
   const int fixed = 1024 + 16 * kMaxStages + 64;
   int stages = forced_stages ? forced_stages : (max_smem - fixed) / s->stage_bytes;
   if (stages > kMaxStages) stages = kMaxStages;
-  if (!forced_stages && stages > 8) stages = 8;  // measured on B200: 6-10 stages stream fastest, 12 is slower again
+  if (!forced_stages && stages * s->atoms > 8) stages = 8 / s->atoms > 3 ? 8 / s->atoms : 3;  // measured on B200: ~144 KB in flight per SM streams fastest
   if (stages < 2) return false;
   s->stages = stages;
   s->smem_bytes = fixed + stages * s->stage_bytes;
@@ -97,23 +106,31 @@ __device__ __forceinline__ void sk_store_d(const SkinnyParams& p, long long idx,
 // Finish up to 16 rows of one output column: all C_in values are fetched first and only then is D stored.
 // (C_in and D are the same buffer, so a load placed after a store could not be moved ahead of it and the rows
 // would cost one global-memory round trip each.)
-__device__ __forceinline__ void sk_finish16(const SkinnyParams& p, int m0, int n, const float (&acc)[16]) {
+// `big` is this thread's index along the long output extent, s0 the first of its 16 indices along the short one.
+template <bool kTall>
+__device__ __forceinline__ void sk_finish16(const SkinnyParams& p, int s0, int big, const float (&acc)[16]) {
+  const int small_extent = kTall ? p.N : p.M;
+  auto at = [&](int j) {  // D is row-major M x N: the short extent is M (rows) unless kTall
+    return kTall ? static_cast<long long>(big) * p.ldc + (s0 + j) : static_cast<long long>(s0 + j) * p.ldc + big;
+  };
   float cin[16];
-  const float bias = (p.epilogue & 1) ? __ldg(p.bias + n) : 0.0f;
+  const bool has_bias = (p.epilogue & 1) != 0;
+  const float bias_big = (!kTall && has_bias) ? __ldg(p.bias + big) : 0.0f;  // the bias runs along N
 #pragma unroll
-  for (int j = 0; j < 16; ++j)
-    cin[j] = (p.beta != 0.0f && m0 + j < p.M) ? sk_load_c(p, static_cast<long long>(m0 + j) * p.ldc + n) : 0.0f;
+  for (int j = 0; j < 16; ++j) cin[j] = (p.beta != 0.0f && s0 + j < small_extent) ? sk_load_c(p, at(j)) : 0.0f;
 #pragma unroll
   for (int j = 0; j < 16; ++j) {
-    if (m0 + j < p.M) {
+    if (s0 + j < small_extent) {
+      const float bias = (kTall && has_bias) ? __ldg(p.bias + s0 + j) : bias_big;
       float v = p.alpha * acc[j] + p.beta * cin[j] + bias;
       if (p.epilogue == 2 || p.epilogue == 3) v = fmaxf(v, 0.0f);
       else if (p.epilogue >= 4) v = gelu_erf(v);
-      sk_store_d(p, static_cast<long long>(m0 + j) * p.ldc + n, v);
+      sk_store_d(p, at(j), v);
     }
   }
 }
 
+template <bool kTall>
 __global__ void __launch_bounds__(kSkinnyThreads, 1)
 skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, const SkinnyParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -123,6 +140,8 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
   const uint32_t warp = threadIdx.x >> 5;
   const uint32_t lane = lane_id();
   const SkinnyPlan& sp = p.plan;
+  const int small_extent = kTall ? p.N : p.M;
+  const int big_extent = kTall ? p.M : p.N;
 
   const uint32_t bars_off = static_cast<uint32_t>(sp.stages) * sp.stage_bytes;
   const uint32_t full0 = base + bars_off;
@@ -166,6 +185,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
   // the ring slot advanced incrementally: the single issuing thread must sustain one 18 KB stage every few hundred
   // cycles, so there is no division and no per-lane register traffic in these loops.
   const uint32_t nstages = static_cast<uint32_t>(sp.stages);
+  const uint32_t atom_bytes = kSkinnyTileN * 128u + static_cast<uint32_t>(sp.m_pad) * 128u;
   const int tile0 = static_cast<int>(u_begin / sp.kbs);
   const int kb0 = static_cast<int>(u_begin - static_cast<long long>(tile0) * sp.kbs);
   const int n_units = static_cast<int>(u_end - u_begin);
@@ -180,8 +200,11 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
       const uint32_t sw_ = base + s * sp.stage_bytes;
       if (elect_one() && !((p.debug_flags & 1u) && i == 0)) {  // test hook: the first stage is never filled nor signalled
         mbar_arrive_expect_tx(bar, sp.stage_bytes);
-        tma_load_3d(sw_, &tmW, bar, kb * kBlockK, tile * kSkinnyTileN, 0, pol_w);
-        tma_load_3d(sw_ + kSkinnyTileN * 128u, &tmX, bar, kb * kBlockK, 0, 0, pol_x);
+        for (int a = 0; a < sp.atoms; ++a) {  // slices past K are zero-filled by TMA and still count their bytes
+          const int k0 = (kb * sp.atoms + a) * kBlockK;
+          tma_load_3d(sw_ + a * atom_bytes, &tmW, bar, k0, tile * kSkinnyTileN, 0, pol_w);
+          tma_load_3d(sw_ + a * atom_bytes + kSkinnyTileN * 128u, &tmX, bar, k0, 0, 0, pol_x);
+        }
       }
       __syncwarp();
       if (++kb == sp.kbs) {
@@ -216,9 +239,12 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         }
         tc_fence_after();
         if (elect_one()) {
-          umma_f16<1>(d_tmem, wdesc, xdesc, idesc, static_cast<uint32_t>(i != 0));
+          for (uint32_t a = 0; a < static_cast<uint32_t>(sp.atoms); ++a) {
+            const uint64_t wd = wdesc + a * (atom_bytes >> 4), xd = xdesc + a * (atom_bytes >> 4);
+            umma_f16<1>(d_tmem, wd, xd, idesc, static_cast<uint32_t>(i != 0 || a != 0));
 #pragma unroll
-          for (uint32_t k = 1; k < kBlockK / kUmmaK; ++k) umma_f16<1>(d_tmem, wdesc + 2u * k, xdesc + 2u * k, idesc, 1u);
+            for (uint32_t k = 1; k < kBlockK / kUmmaK; ++k) umma_f16<1>(d_tmem, wd + 2u * k, xd + 2u * k, idesc, 1u);
+          }
           umma_commit<1>(empty0 + 8u * s);
         }
         __syncwarp();
@@ -262,11 +288,11 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
           float accf[16];
 #pragma unroll
           for (int j = 0; j < 16; ++j) accf[j] = __uint_as_float(acc[j]);
-          if (n < p.N) sk_finish16(p, c0, n, accf);
+          if (n < big_extent) sk_finish16<kTall>(p, c0, n, accf);
         } else {
 #pragma unroll
           for (int j = 0; j < 16; ++j)
-            if (c0 + j < p.M) my_partial[(c0 + j) * kSkinnyTileN + n_local] = __uint_as_float(acc[j]);
+            if (c0 + j < small_extent) my_partial[(c0 + j) * kSkinnyTileN + n_local] = __uint_as_float(acc[j]);
         }
       }
       tc_fence_before();
@@ -286,7 +312,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         const bool last = *s_last != 0u;
         if (last) {
           __threadfence();
-          for (int m0 = 0; m0 < p.M; m0 += 16) {
+          for (int m0 = 0; m0 < small_extent; m0 += 16) {
             float sum[16];
 #pragma unroll
             for (int j = 0; j < 16; ++j) sum[j] = 0.0f;
@@ -295,9 +321,9 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
               const float* part = p.partials + (static_cast<size_t>(c) * 2 + slot) * (kSkinnyTileN * sp.m_pad);
 #pragma unroll
               for (int j = 0; j < 16; ++j)
-                if (m0 + j < p.M) sum[j] += __ldcg(part + (m0 + j) * kSkinnyTileN + n_local);
+                if (m0 + j < small_extent) sum[j] += __ldcg(part + (m0 + j) * kSkinnyTileN + n_local);
             }
-            if (n < p.N) sk_finish16(p, m0, n, sum);
+            if (n < big_extent) sk_finish16<kTall>(p, m0, n, sum);
           }
           if (leader) p.counters[tile] = 0u;  // leave the counter clean for the next launch
         }
@@ -317,12 +343,15 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
 }
 
 // Zero the arrival counters and launch.  Returns a gemm_status_t value (0 = ok, 7 = CUDA failure).
+// `tall` selects the mirrored addressing (tW then maps A, tX maps B).
 inline int skinny_launch(const SkinnyParams& p, const CUtensorMap& tW, const CUtensorMap& tX, int device, cudaStream_t stream,
-                         char* err, size_t err_len) {
-  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(skinny_gemm_kernel), kSlotSkinny, device, p.plan.smem_bytes);
+                         char* err, size_t err_len, bool tall = false) {
+  cudaError_t e = tall ? ensure_dynamic_smem(reinterpret_cast<const void*>(skinny_gemm_kernel<true>), kSlotSkinnyTall, device, p.plan.smem_bytes)
+                       : ensure_dynamic_smem(reinterpret_cast<const void*>(skinny_gemm_kernel<false>), kSlotSkinny, device, p.plan.smem_bytes);
   if (e == cudaSuccess) e = cudaMemsetAsync(p.counters, 0, p.plan.counters_bytes, stream);
   if (e == cudaSuccess) {
-    skinny_gemm_kernel<<<p.plan.grid, kSkinnyThreads, p.plan.smem_bytes, stream>>>(tW, tX, p);
+    if (tall) skinny_gemm_kernel<true><<<p.plan.grid, kSkinnyThreads, p.plan.smem_bytes, stream>>>(tW, tX, p);
+    else skinny_gemm_kernel<false><<<p.plan.grid, kSkinnyThreads, p.plan.smem_bytes, stream>>>(tW, tX, p);
     e = cudaGetLastError();
   }
   if (e != cudaSuccess) {

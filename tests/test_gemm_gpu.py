@@ -92,6 +92,18 @@ EXACT_CASES = [
     ("skinny_m33_bias_bf16", 33, 1000, 520, dict(cd=wl.BF16, epi=bg.EPI_BIAS), dict(variant=VS)),
     ("skinny_m64_f16", 64, 520, 1032, dict(ab=wl.F16, cd=wl.F16, alpha=0.5, beta=1.0), dict(variant=VS)),
     ("skinny_stages_2", 8, 384, 1024, {}, dict(variant=VS, stages=2)),
+    ("skinny_one_slice_stages", 8, 256, 4096, {}, dict(variant=VS, kslices=1)),
+    ("skinny_three_slice_stages", 8, 384, 1100 - 4, {}, dict(variant=VS, kslices=3)),
+    ("skinny_k_slice_past_the_end", 8, 256, 1080, {}, dict(variant=VS)),
+    # mirrored stream-K: a tall output with a handful of columns (A is the streamed operand)
+    ("tall_one_unit", 128, 8, 64, {}, dict(variant=VS)),
+    ("tall_split_k", 256, 8, 4096, {}, dict(variant=VS)),
+    ("tall_ragged_beta", 1864, 8, 2136, dict(beta=1.0), dict(variant=VS)),
+    ("tall_matrix_vector", 4096, 1, 4096, dict(ldb=4096, ldc=4), dict(variant=VS)),
+    ("tall_n16_whole_tiles", 28672, 16, 1024, {}, dict(variant=VS)),
+    ("tall_n33_bias_bf16", 1000, 33, 520, dict(cd=wl.BF16, epi=bg.EPI_BIAS, ldc=40), dict(variant=VS)),
+    ("tall_n64_f16_bias_relu", 520, 64, 1032, dict(ab=wl.F16, cd=wl.F16, alpha=0.5, beta=1.0, epi=bg.EPI_BIAS_RELU), dict(variant=VS)),
+    ("tall_auto_plan", 8192, 8, 2048, dict(beta=1.0), dict()),
 ]
 
 

@@ -115,9 +115,9 @@ def test_roofline_classification_of_the_five_configs():
 
 def test_stream_k_plan_geometry():
     i5 = info_for(wl.configs()["c5"])
-    assert i5["num_tiles"] == 224 * 128              # (n-tile, k-block) work units
-    assert i5["grid"] == 148 and i5["tile_m"] == 128 and i5["tile_n"] == 16
-    assert i5["split"] >= 2 and i5["stages"] == 8
+    assert i5["num_tiles"] == 224 * 64               # (n-tile, 128-wide k-block) work units
+    assert i5["grid"] == 148 and i5["tile_m"] == 128 and i5["tile_n"] == 16 and i5["tile_k"] == 128
+    assert i5["split"] >= 2 and i5["stages"] == 4    # 4 stages of two 64-wide K slices: 144 KB in flight per SM
     # counters (224 x 4 bytes padded to 256) + 2 partial slots of 128 x 16 fp32 per CTA
     assert i5["workspace_bytes"] == 1024 + 148 * 2 * 128 * 16 * 4
     tiny = info_for(wl.Workload("t", 4, 100, 64), bg.make_flags(bg.VARIANT_SKINNY_STREAMK))
@@ -170,6 +170,8 @@ def test_cost_model_choices_follow_the_measurements():
     assert choice(128, 28672, 8192) == (bg.VARIANT_DENSE_1CTA, 256)          # one tile row: no pair
     assert choice(16384, 14336, 4096, epilogue=bg.EPI_BIAS_GELU_ERF)[0] == bg.VARIANT_DENSE_2CTA
     assert choice(16, 28672, 8192)[0] == bg.VARIANT_SKINNY_STREAMK
+    assert choice(28672, 16, 8192)[0] == bg.VARIANT_SKINNY_STREAMK            # mirrored: the long operand is A
+    assert choice(28672, 16, 8192, transb=bg.OP_N)[0] != bg.VARIANT_SKINNY_STREAMK   # needs both operands K-contiguous
     assert choice(64, 28672, 8192)[0] == bg.VARIANT_DENSE_1CTA               # stream-K stops paying near M = 48
     v, bn = choice(2048, 2048, 128, batch=64)
     assert (v, bn) == (bg.VARIANT_DENSE_1CTA, 256)                           # output-bound: widest tile, fewest hand-shakes
