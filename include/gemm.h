@@ -91,8 +91,8 @@ typedef enum {
 #define GEMM_FLAG_NO_K_SERPENTINE 0x8u      /* walk K forwards in every tile (default: alternate tiles walk it backwards,
                                               which re-uses the operand lines L2 touched last) */
 #define GEMM_FLAG_L2_HINTS 0x40000000u     /* load A with evict-last and B with evict-first L2 priority (default: normal) */
-#define GEMM_FLAG_DEBUG_STALL 0x80000000u  /* test hook: one producer arrival is withheld so that a bounded
-                                              wait expires and GEMM_ERR_TIMEOUT is reported */
+#define GEMM_FLAG_DEBUG_STALL 0x80000000u  /* test hook: in the plan's first run one producer arrival is withheld so that
+                                              a bounded wait expires and GEMM_ERR_TIMEOUT is reported; later runs are normal */
 
 typedef struct {
   uint32_t struct_size;  /* = sizeof(gemm_desc_t) */
@@ -130,7 +130,8 @@ typedef struct {
  * roofline (Section 4.3), choose the kernel variant, tile shape, pipeline depth,
  * cluster size, raster order and stream-K split, and return a plan (host
  * memory).  If a CUDA device is current, also allocates the plan's 16-byte
- * device status word and reads the SM count; without a device the plan is still
+ * device status word (and, for the stream-K variant, its arrival counters, one
+ * word per output tile) and reads the SM count; without a device the plan is still
  * created (148 SMs assumed) so that planning can be inspected, and gemm_run
  * reports GEMM_ERR_ARCH.  Errors: NULL -> GEMM_ERR_NULL; extents < 1, leading
  * dimension smaller than the row length, unknown enum, wrong struct_size ->
@@ -141,7 +142,7 @@ typedef struct {
 gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan);
 
 /* Bytes of device workspace gemm_run needs for this plan (0 for the dense variants;
- * stream-K partial tiles and arrival counters for the skinny variant).  0 on a NULL plan. */
+ * stream-K partial tiles for the skinny variant).  0 on a NULL plan. */
 size_t gemm_workspace_bytes(gemm_plan_t plan);
 
 /*
@@ -150,8 +151,10 @@ size_t gemm_workspace_bytes(gemm_plan_t plan);
  * aligned, laid out as `desc` said.  bias: device fp32[N], required iff the
  * epilogue has a bias.  C is read only when beta != 0.  workspace: device
  * memory of at least gemm_workspace_bytes(plan) bytes, 16-byte aligned (may be NULL when
- * that is 0); concurrent runs of one plan need distinct workspaces.  alpha and
- * beta are host scalars.  Errors are returned before anything is launched:
+ * that is 0).  Runs of one dense plan may overlap on the GPU; runs of one
+ * stream-K plan must not (they share the plan's arrival counters, which every
+ * run leaves at zero): order them on one stream or with events, or make one
+ * plan per stream.  alpha and beta are host scalars.  Errors are returned before anything is launched:
  * GEMM_ERR_NULL, GEMM_ERR_ALIGNMENT, GEMM_ERR_WORKSPACE, GEMM_ERR_ARCH,
  * GEMM_ERR_INVALID_ARG (the current CUDA device is not the one the plan was
  * made on), GEMM_ERR_CUDA (tensor-map encoding or launch failure).
@@ -162,8 +165,10 @@ gemm_status_t gemm_run(gemm_plan_t plan, const void* A, const void* B, void* C, 
 /*
  * gemm_plan_status -- synchronise the device and read the plan's status word:
  * GEMM_OK, or GEMM_ERR_TIMEOUT if a bounded device-side wait of an earlier run
- * expired (the kernel then returned early and its output is undefined).  The
- * word is cleared by the read.
+ * expired (the kernel then returned early and its output is undefined; until
+ * the word has been read, later runs of the plan may give up early as well,
+ * and a stream-K plan does not finish split tiles).  The read clears the word
+ * and puts the plan back in order.
  */
 gemm_status_t gemm_plan_status(gemm_plan_t plan);
 

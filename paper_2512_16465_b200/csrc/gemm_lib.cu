@@ -104,7 +104,9 @@ struct gemm_plan_s {
   int device;            // CUDA device the plan was made on (-1: none); runs must use the same one
   bool has_device;
   bool arch_ok;
-  uint32_t* d_status;
+  uint32_t* d_status;       // device: 16-byte status word, followed (256 bytes on) by the stream-K arrival counters
+  size_t d_counters_bytes = 0;  // 0 unless the plan is a stream-K plan
+  unsigned long long runs = 0;  // launches so far (the timeout test hook acts on the first one only)
   uint32_t timeout_ms;
   DenseParams dense;     // filled at plan time except pointers / scalars
   SkinnyPlan skinny;     // stream-K decomposition of the skinny variant
@@ -282,7 +284,7 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   p.epilogue = d.epilogue;
   p.ldc = d.ldc;
   p.stride_c = d.batch_count > 1 ? d.stride_c : 0;
-  p.debug_flags = (d.flags & GEMM_FLAG_DEBUG_STALL) ? 1u : 0u;
+  p.debug_flags = 0u;  // set per run
   // The scheduler keeps a band of `raster` tile rows of A live across several waves while B panels stream past;
   // on request, L2 is asked to hold on to A and to let B go first (measured neutral on 8192^3, so off by default).
   const bool hints = (d.flags & GEMM_FLAG_L2_HINTS) != 0;
@@ -366,7 +368,7 @@ gemm_status_t plan_wide(gemm_plan_s* pl, int forced_raster, int forced_stages) {
   p.epilogue = d.epilogue;
   p.ldc = d.ldc;
   p.stride_c = d.batch_count > 1 ? d.stride_c : 0;
-  p.debug_flags = (d.flags & GEMM_FLAG_DEBUG_STALL) ? 1u : 0u;
+  p.debug_flags = 0u;  // set per run
   p.k_serpentine = ((d.flags & GEMM_FLAG_NO_K_SERPENTINE) || p.num_kb < 4) ? 0 : 1;
 
   pl->cg = 2;
@@ -510,7 +512,10 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
     return st;
   }
   if (pl->has_device && pl->arch_ok) {
-    if (cudaMalloc(&pl->d_status, 16) != cudaSuccess || cudaMemset(pl->d_status, 0, 16) != cudaSuccess) {
+    // the counters start at zero here and every run leaves them at zero again (gemm_plan_status cleans up after a timeout)
+    pl->d_counters_bytes = pl->variant == GEMM_VARIANT_SKINNY_STREAMK ? pl->skinny.counters_bytes : 0;
+    const size_t dev_bytes = pl->d_counters_bytes ? 256 + pl->d_counters_bytes : 16;
+    if (cudaMalloc(&pl->d_status, dev_bytes) != cudaSuccess || cudaMemset(pl->d_status, 0, dev_bytes) != cudaSuccess) {
       note_cuda_error("cudaMalloc(status word)", cudaGetErrorName(cudaGetLastError()));
       delete pl;
       return GEMM_ERR_CUDA;
@@ -550,6 +555,8 @@ gemm_status_t gemm_plan_status(gemm_plan_t plan) {
   cudaError_t e = cudaDeviceSynchronize();
   if (e == cudaSuccess) e = cudaMemcpy(h, plan->d_status, 16, cudaMemcpyDeviceToHost);
   if (e == cudaSuccess) e = cudaMemset(plan->d_status, 0, 16);
+  if (e == cudaSuccess && h[0] != 0 && plan->d_counters_bytes)  // a run that gave up may have left arrivals half counted
+    e = cudaMemset(reinterpret_cast<char*>(plan->d_status) + 256, 0, plan->d_counters_bytes);
   if (e != cudaSuccess) {
     note_cuda_error("gemm_plan_status", cudaGetErrorName(e));
     return GEMM_ERR_CUDA;
@@ -654,7 +661,7 @@ gemm_status_t launch_wide(const gemm_plan_s* pl, const CUtensorMap& tA, const CU
 }
 
 gemm_status_t run_dense(gemm_plan_s* pl, const void* A, const void* B, void* C, const float* bias, float alpha, float beta,
-                        cudaStream_t stream) {
+                        cudaStream_t stream, bool stall) {
   const gemm_desc_t& d = pl->d;
   DenseParams p = pl->dense;
   CUtensorMap tA, tB, tD;
@@ -672,6 +679,7 @@ gemm_status_t run_dense(gemm_plan_s* pl, const void* A, const void* B, void* C, 
   p.beta = beta;
   p.bias = bias;
   p.c_in = C;
+  p.debug_flags = stall ? 1u : 0u;
   p.status = pl->d_status;
   p.timeout_ns = static_cast<unsigned long long>(pl->timeout_ms) * 1000000ull;
   if (pl->variant == GEMM_VARIANT_DENSE_2CTA_WIDE) return launch_wide(pl, tA, tB, tD, p, stream);
@@ -680,7 +688,7 @@ gemm_status_t run_dense(gemm_plan_s* pl, const void* A, const void* B, void* C, 
 }
 
 gemm_status_t run_skinny(gemm_plan_s* pl, const void* A, const void* B, void* C, const float* bias, float alpha, float beta,
-                         void* workspace, cudaStream_t stream) {
+                         void* workspace, cudaStream_t stream, bool stall) {
   const gemm_desc_t& d = pl->d;
   const SkinnyPlan& s = pl->skinny;
   CUtensorMap tW, tX;
@@ -709,13 +717,13 @@ gemm_status_t run_skinny(gemm_plan_s* pl, const void* A, const void* B, void* C,
   p.bias = bias;
   p.c = C;
   p.ldc = d.ldc;
-  p.partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + s.counters_bytes);
-  p.counters = reinterpret_cast<uint32_t*>(workspace);
-  p.debug_flags = (d.flags & GEMM_FLAG_DEBUG_STALL) ? 1u : 0u;
+  p.partials = static_cast<float*>(workspace);
+  p.counters = reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(pl->d_status) + 256);
+  p.debug_flags = stall ? 1u : 0u;
   p.status = pl->d_status;
   p.timeout_ns = static_cast<unsigned long long>(pl->timeout_ms) * 1000000ull;
   return static_cast<gemm_status_t>(
-      skinny_launch(p, tW, tX, pl->device, stream, g_last_cuda_error, sizeof g_last_cuda_error, pl->skinny_tall));
+      skinny_launch(p, tW, tX, pl->device, stream, g_last_cuda_error, sizeof g_last_cuda_error, pl->skinny_tall, /*zero_counters=*/false));
 }
 
 }  // namespace
@@ -735,8 +743,10 @@ extern "C" gemm_status_t gemm_run(gemm_plan_t plan, const void* A, const void* B
   int cur = -1;
   if (cudaGetDevice(&cur) != cudaSuccess || cur != plan->device) return GEMM_ERR_INVALID_ARG;  // plan belongs to another device
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (plan->variant == GEMM_VARIANT_SKINNY_STREAMK) return run_skinny(plan, A, B, C, bias, alpha, beta, workspace, s);
-  return run_dense(plan, A, B, C, bias, alpha, beta, s);
+  const bool stall = (plan->d.flags & GEMM_FLAG_DEBUG_STALL) && plan->runs == 0;  // test hook: the plan's first run only
+  ++plan->runs;
+  if (plan->variant == GEMM_VARIANT_SKINNY_STREAMK) return run_skinny(plan, A, B, C, bias, alpha, beta, workspace, s, stall);
+  return run_dense(plan, A, B, C, bias, alpha, beta, s, stall);
 }
 
 // ---------------------------------------------------------------------------------------------------------
@@ -818,7 +828,7 @@ extern "C" gemm_status_t gemm_skinny_run_noalloc(const gemm_desc_t* desc, const 
   if (!skinny_make_plan(&sp, static_cast<int>(desc->M), static_cast<int>(desc->N), static_cast<int>(desc->K), nd.sm_count, 0,
                         kMaxSmemOptin))
     return GEMM_ERR_UNSUPPORTED;
-  const size_t need = kNoAllocHeaderBytes + sp.workspace_bytes;
+  const size_t need = kNoAllocHeaderBytes + sp.counters_bytes + sp.workspace_bytes;
   if (need > kNoAllocScratchBytes) {
     snprintf(g_last_cuda_error, sizeof g_last_cuda_error, "problem needs %zu bytes of scratch, the built-in array has %zu", need,
              kNoAllocScratchBytes);
@@ -855,7 +865,8 @@ extern "C" gemm_status_t gemm_skinny_run_noalloc(const gemm_desc_t* desc, const 
   p.counters = reinterpret_cast<uint32_t*>(nd.scratch + kNoAllocHeaderBytes);
   p.partials = reinterpret_cast<float*>(nd.scratch + kNoAllocHeaderBytes + sp.counters_bytes);
   p.timeout_ns = 2000ull * 1000000ull;
-  st = static_cast<gemm_status_t>(skinny_launch(p, tW, tX, dev, s, g_last_cuda_error, sizeof g_last_cuda_error));
+  st = static_cast<gemm_status_t>(
+      skinny_launch(p, tW, tX, dev, s, g_last_cuda_error, sizeof g_last_cuda_error, /*tall=*/false, /*zero_counters=*/true));
   if (st != GEMM_OK || !sync_and_check) return st;
   uint32_t word = 0;
   e = cudaStreamSynchronize(s);

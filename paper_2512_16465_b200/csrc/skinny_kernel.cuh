@@ -9,7 +9,8 @@
 //     ranges, one per CTA (one CTA per SM), so every SM streams the same number of bytes;
 //   * a CTA whose range covers only part of a tile's K writes its fp32 partial to the workspace and
 //     bumps the tile's arrival counter; the CTA that arrives last adds the partials in contributor
-//     order (deterministic, no floating-point atomics), applies the epilogue and writes D.
+//     order (deterministic, no floating-point atomics), applies the epilogue, writes D and puts the
+//     counter back to zero, so the counters are clean again when the kernel ends.
 //     Nobody ever waits for another CTA.
 //
 // The same kernel serves the mirrored case, a tall output with a handful of columns (N <= 64 < M, kTall): the long
@@ -35,19 +36,23 @@ struct SkinnyPlan {
   int n_tiles;           // ceil(big extent / 128)
   int atoms;             // 64-wide K slices per pipeline stage (each slice is one 128-byte swizzle atom per row)
   int kbs;               // work units per tile = ceil(K / (64 * atoms))
-  long long total_units; // n_tiles * kbs
+  long long total_units; // n_tiles * kbs (< 2^31)
+  int units_q, units_r;  // total_units = grid * units_q + units_r: the first units_r CTAs take units_q + 1 units
   int grid;              // CTAs = min(SM count, total_units)
   int stages;
   int stage_bytes;       // atoms x (16 KB of W + m_pad * 128 bytes of X)
   int smem_bytes;
   int max_contributors;  // upper bound on CTAs touching one tile
-  size_t counters_bytes; // workspace: [counters (n_tiles x u32, padded)] [partials: grid * 2 slots]
-  size_t workspace_bytes;
+  size_t counters_bytes; // arrival counters: n_tiles x u32, padded to 256 bytes
+  size_t workspace_bytes;  // partial tiles: grid * 2 slots of [m_pad][128] floats
 };
 
-// First work unit of CTA c, and the CTA that owns unit u, for T units over G CTAs.
-__host__ __device__ inline long long sk_begin(long long c, long long T, long long G) { return c * T / G; }
-__host__ __device__ inline int sk_owner(long long u, long long T, long long G) { return static_cast<int>(((u + 1) * G - 1) / T); }
+// First work unit of CTA c, and the CTA that owns unit u (32-bit arithmetic: these run on the device's critical path).
+__host__ __device__ inline int sk_begin(int c, int q, int r) { return c * q + (c < r ? c : r); }
+__host__ __device__ inline int sk_owner(int u, int q, int r) {
+  const int head = r * (q + 1);
+  return u < head ? u / (q + 1) : r + (u - head) / q;
+}
 
 // M is the small output extent and N the big one (for a tall problem the caller passes them swapped).
 inline bool skinny_make_plan(SkinnyPlan* s, int M, int N, int K, int sm_count, int forced_stages, int max_smem, int forced_atoms = 0) {
@@ -59,7 +64,10 @@ inline bool skinny_make_plan(SkinnyPlan* s, int M, int N, int K, int sm_count, i
   s->atoms = forced_atoms ? forced_atoms : (K >= 1024 ? 2 : 1);
   s->kbs = (K + kBlockK * s->atoms - 1) / (kBlockK * s->atoms);
   s->total_units = static_cast<long long>(s->n_tiles) * s->kbs;
+  if (s->total_units > 0x7fffffffll) return false;
   s->grid = static_cast<int>(s->total_units < sm_count ? s->total_units : sm_count);
+  s->units_q = static_cast<int>(s->total_units / s->grid);
+  s->units_r = static_cast<int>(s->total_units % s->grid);
   s->stage_bytes = s->atoms * (kSkinnyTileN * 128 + s->m_pad * 128);
   const int fixed = 1024 + 16 * kMaxStages + 64;
   int stages = forced_stages ? forced_stages : (max_smem - fixed) / s->stage_bytes;
@@ -69,10 +77,10 @@ inline bool skinny_make_plan(SkinnyPlan* s, int M, int N, int K, int sm_count, i
   s->stages = stages;
   s->smem_bytes = fixed + stages * s->stage_bytes;
   if (s->smem_bytes > max_smem) return false;
-  const long long per_cta = s->total_units / s->grid;  // >= 1
-  s->max_contributors = static_cast<int>((s->kbs + per_cta - 1) / per_cta + 1);
+  const int per_cta = s->units_q;  // >= 1
+  s->max_contributors = (s->kbs + per_cta - 1) / per_cta + 1;
   s->counters_bytes = (static_cast<size_t>(s->n_tiles) * 4 + 255) / 256 * 256;
-  s->workspace_bytes = s->counters_bytes + static_cast<size_t>(s->grid) * 2 * kSkinnyTileN * s->m_pad * 4;
+  s->workspace_bytes = static_cast<size_t>(s->grid) * 2 * kSkinnyTileN * s->m_pad * 4;
   return true;
 }
 
@@ -87,7 +95,7 @@ struct SkinnyParams {
   void* c;                // D buffer (also C_in when beta != 0), row-major M x N
   long long ldc;
   float* partials;        // workspace: slot-major, each slot [m_pad][128] floats
-  uint32_t* counters;     // workspace: one arrival counter per n-tile, zero at launch
+  uint32_t* counters;     // one arrival counter per n-tile, zero at launch and zero again at the end
   uint32_t* status;
   unsigned long long timeout_ns;
   uint32_t debug_flags;   // bit 0: withhold one producer arrival (timeout test hook)
@@ -103,21 +111,27 @@ __device__ __forceinline__ void sk_store_d(const SkinnyParams& p, long long idx,
   else if (p.out_dtype == 0) static_cast<__nv_bfloat16*>(p.c)[idx] = __float2bfloat16_rn(v);
   else static_cast<__half*>(p.c)[idx] = __float2half_rn(v);
 }
-// Finish up to 16 rows of one output column: all C_in values are fetched first and only then is D stored.
-// (C_in and D are the same buffer, so a load placed after a store could not be moved ahead of it and the rows
-// would cost one global-memory round trip each.)
 // `big` is this thread's index along the long output extent, s0 the first of its 16 indices along the short one.
+// D is row-major M x N: the short extent is M (rows) unless kTall.
 template <bool kTall>
-__device__ __forceinline__ void sk_finish16(const SkinnyParams& p, int s0, int big, const float (&acc)[16]) {
+__device__ __forceinline__ long long sk_index(const SkinnyParams& p, int small, int big) {
+  return kTall ? static_cast<long long>(big) * p.ldc + small : static_cast<long long>(small) * p.ldc + big;
+}
+// Fetch the 16 C_in values (zeros when beta == 0).  Kept apart from sk_finish16 so that the loads can be issued
+// before other long-latency loads, and before any store to the same buffer (C_in and D are one buffer: a load
+// placed after a store could not be moved ahead of it and the rows would cost one round trip each).
+template <bool kTall>
+__device__ __forceinline__ void sk_load_cin16(const SkinnyParams& p, int s0, int big, float (&cin)[16]) {
   const int small_extent = kTall ? p.N : p.M;
-  auto at = [&](int j) {  // D is row-major M x N: the short extent is M (rows) unless kTall
-    return kTall ? static_cast<long long>(big) * p.ldc + (s0 + j) : static_cast<long long>(s0 + j) * p.ldc + big;
-  };
-  float cin[16];
+#pragma unroll
+  for (int j = 0; j < 16; ++j)
+    cin[j] = (p.beta != 0.0f && s0 + j < small_extent) ? sk_load_c(p, sk_index<kTall>(p, s0 + j, big)) : 0.0f;
+}
+template <bool kTall>
+__device__ __forceinline__ void sk_finish16(const SkinnyParams& p, int s0, int big, const float (&acc)[16], const float (&cin)[16]) {
+  const int small_extent = kTall ? p.N : p.M;
   const bool has_bias = (p.epilogue & 1) != 0;
   const float bias_big = (!kTall && has_bias) ? __ldg(p.bias + big) : 0.0f;  // the bias runs along N
-#pragma unroll
-  for (int j = 0; j < 16; ++j) cin[j] = (p.beta != 0.0f && s0 + j < small_extent) ? sk_load_c(p, at(j)) : 0.0f;
 #pragma unroll
   for (int j = 0; j < 16; ++j) {
     if (s0 + j < small_extent) {
@@ -125,7 +139,7 @@ __device__ __forceinline__ void sk_finish16(const SkinnyParams& p, int s0, int b
       float v = p.alpha * acc[j] + p.beta * cin[j] + bias;
       if (p.epilogue == 2 || p.epilogue == 3) v = fmaxf(v, 0.0f);
       else if (p.epilogue >= 4) v = gelu_erf(v);
-      sk_store_d(p, at(j), v);
+      sk_store_d(p, sk_index<kTall>(p, s0 + j, big), v);
     }
   }
 }
@@ -151,7 +165,19 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + bars_off + 16u * kMaxStages + 32u);
   volatile uint32_t* s_abort = tmem_slot + 1;
   volatile uint32_t* s_last = tmem_slot + 2;
+  volatile uint32_t* s_early = tmem_slot + 3;  // two words: a CTA has at most two partial segments (its first and its last)
   const WaitCtx w{s_abort, p.status, p.timeout_ns};
+  // This CTA's contiguous range of work units (computed while the barriers and tensor memory are being set up).
+  const int uq = sp.units_q, ur = sp.units_r;
+  const int u_begin = sk_begin(static_cast<int>(blockIdx.x), uq, ur);
+  const int u_end = sk_begin(static_cast<int>(blockIdx.x) + 1, uq, ur);
+  const int tile0 = u_begin / sp.kbs;
+  const int kb0 = u_begin - tile0 * sp.kbs;
+  const int n_units = u_end - u_begin;
+  // An earlier run of this plan that timed out may have left arrival counters half counted; the status word stays
+  // set until the host has read it (and cleaned the counters), and until then no run trusts them.  The load is
+  // issued here and consumed only by the fix-up, long after it has landed.
+  const uint32_t stale_status = *reinterpret_cast<volatile const uint32_t*>(p.status);
   const uint32_t tmem_cols = sp.m_pad * 2 <= 32 ? 32u : (sp.m_pad * 2 <= 64 ? 64u : 128u);
 
   if (threadIdx.x == 0) {
@@ -177,18 +203,11 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  const long long T = sp.total_units, G = gridDim.x;
-  const long long u_begin = sk_begin(blockIdx.x, T, G);
-  const long long u_end = sk_begin(blockIdx.x + 1, T, G);
-
   // The producer and MMA roles run warp-uniform (one elected lane issues), with the (tile, k-block) position and
   // the ring slot advanced incrementally: the single issuing thread must sustain one 18 KB stage every few hundred
   // cycles, so there is no division and no per-lane register traffic in these loops.
   const uint32_t nstages = static_cast<uint32_t>(sp.stages);
   const uint32_t atom_bytes = kSkinnyTileN * 128u + static_cast<uint32_t>(sp.m_pad) * 128u;
-  const int tile0 = static_cast<int>(u_begin / sp.kbs);
-  const int kb0 = static_cast<int>(u_begin - static_cast<long long>(tile0) * sp.kbs);
-  const int n_units = static_cast<int>(u_end - u_begin);
   if (warp == 0) {
     const uint64_t pol_w = l2_policy_evict_first();  // weights are read exactly once
     const uint64_t pol_x = l2_policy_evict_last();   // the activation slab is re-read by every CTA
@@ -268,16 +287,46 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
     const int n_local = static_cast<int>(q * 32u + lane);
     const bool leader = (warp == 2 && lane == 0);
     uint32_t seg = 0;
-    long long u = u_begin;
+    int u = u_begin;
     while (u < u_end) {
-      const long long tile = u / sp.kbs;
-      const long long tile_u0 = tile * sp.kbs;
-      const long long seg_end = min(u_end, tile_u0 + sp.kbs);
+      const int tile = u / sp.kbs;
+      const int tile_u0 = tile * sp.kbs;
+      const int seg_end = min(u_end, tile_u0 + sp.kbs);
       const uint32_t buf = seg & 1u;
+      const int n = tile * kSkinnyTileN + n_local;
+      const bool whole = (u == tile_u0) && (seg_end == tile_u0 + sp.kbs);  // this CTA owns the tile's whole K
+      // contributors of a split tile: c_first reaches it at the end of its range (second slot) unless its range starts
+      // exactly here; every later contributor starts inside the tile (first slot)
+      const int c_first = whole ? 0 : sk_owner(tile_u0, uq, ur);
+      const int c_last = whole ? 0 : sk_owner(tile_u0 + sp.kbs - 1, uq, ur);
+      const int first_slot = (whole || sk_begin(c_first, uq, ur) == tile_u0) ? 0 : 1;
+      auto partial_of = [&](int c) {
+        return p.partials + (static_cast<size_t>(c) * 2 + (c == c_first ? first_slot : 0)) * (kSkinnyTileN * sp.m_pad);
+      };
+      // While the main loop of this segment runs, these warps have nothing to do.  The usual case for the CTA that
+      // computes the head of a split tile is that all other contributors finished long ago; if the count says so,
+      // their partials (and C_in) are fetched now, this CTA never publishes its own partial and the tail of the kernel
+      // is one tensor-memory read, a few adds and the stores.  (One chunk of 16 and at most four contributors, so that
+      // everything fits in registers; other shapes take the general path below.)  Both paths add the same values in
+      // the same order, so the result does not depend on which one ran.
+      bool early = false;
+      float pre[4][16], cin0[16];
+      if (!whole && sp.m_pad == 16 && c_last - c_first <= 3) {
+        if (leader) s_early[seg == 0 ? 0 : 1] = (stale_status == 0u && ld_acquire_gpu(p.counters + tile) == static_cast<uint32_t>(c_last - c_first)) ? 1u : 0u;
+        named_barrier_sync(1, 128);
+        early = s_early[seg == 0 ? 0 : 1] != 0u;
+        if (early) {
+#pragma unroll
+          for (int b = 0; b < 4; ++b) {
+            const float* part = partial_of(min(c_first + b, c_last));  // (this CTA's own slot is read too and not used)
+#pragma unroll
+            for (int j = 0; j < 16; ++j) pre[b][j] = __ldcg(part + j * kSkinnyTileN + n_local);
+          }
+          if (n < big_extent) sk_load_cin16<kTall>(p, 0, n, cin0);
+        }
+      }
       if (!mbar_wait_warp(tfull0 + 8u * buf, (seg >> 1) & 1u, w, (3u << 8) | buf, 64u)) break;
       tc_fence_after();
-      const int n = static_cast<int>(tile) * kSkinnyTileN + n_local;
-      const bool whole = (u == tile_u0) && (seg_end == tile_u0 + sp.kbs);  // this CTA owns the tile's whole K
       const uint32_t t_row = tmem_base + ((q * 32u) << 16) + buf * static_cast<uint32_t>(sp.m_pad);
       float* my_partial = p.partials + (static_cast<size_t>(blockIdx.x) * 2 + (seg == 0 ? 0 : 1)) * (kSkinnyTileN * sp.m_pad);
       for (int c0 = 0; c0 < sp.m_pad; c0 += 16) {
@@ -285,10 +334,26 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         tmem_ld_32x16(t_row + static_cast<uint32_t>(c0), acc);
         tmem_ld_wait();
         if (whole) {
-          float accf[16];
+          float accf[16], cin[16];
 #pragma unroll
           for (int j = 0; j < 16; ++j) accf[j] = __uint_as_float(acc[j]);
-          if (n < big_extent) sk_finish16<kTall>(p, c0, n, accf);
+          if (n < big_extent) {
+            sk_load_cin16<kTall>(p, c0, n, cin);
+            sk_finish16<kTall>(p, c0, n, accf, cin);
+          }
+        } else if (early) {
+          float sum[16];
+#pragma unroll
+          for (int j = 0; j < 16; ++j) sum[j] = 0.0f;
+#pragma unroll
+          for (int b = 0; b < 4; ++b) {
+            const int cc = c_first + b;
+            if (cc <= c_last) {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) sum[j] += (cc == static_cast<int>(blockIdx.x)) ? __uint_as_float(acc[j]) : pre[b][j];
+            }
+          }
+          if (n < big_extent) sk_finish16<kTall>(p, 0, n, sum, cin0);
         } else {
 #pragma unroll
           for (int j = 0; j < 16; ++j)
@@ -298,32 +363,44 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty0 + 8u * buf);
-      if (!whole) {
-        // publish the partial, then count arrivals; the last contributor reduces
-        const int c_first = sk_owner(tile_u0, T, G);
-        const int c_last = sk_owner(tile_u0 + sp.kbs - 1, T, G);
-        __threadfence();
+      if (early) {
+        if (leader) p.counters[tile] = 0u;  // the others counted themselves in; leave the counter clean for the next launch
+      } else if (!whole) {
+        // Publish the partial and count the arrival; the last contributor reduces.  The barrier orders the four
+        // warps' partial stores before the leader's atomic, whose release makes them visible to whoever reads the
+        // count later and whose acquire, passed on by the second barrier, lets this CTA read the earlier partials.
         named_barrier_sync(1, 128);
         if (leader) {
-          const uint32_t old = atomicAdd(p.counters + tile, 1u);
+          const uint32_t old = stale_status == 0u ? atom_add_acq_rel_gpu(p.counters + tile, 1u) : 0xffffffffu;
           *s_last = (old == static_cast<uint32_t>(c_last - c_first)) ? 1u : 0u;
         }
         named_barrier_sync(1, 128);
         const bool last = *s_last != 0u;
         if (last) {
-          __threadfence();
           for (int m0 = 0; m0 < small_extent; m0 += 16) {
-            float sum[16];
+            float sum[16], cin[16];
 #pragma unroll
             for (int j = 0; j < 16; ++j) sum[j] = 0.0f;
-            for (int c = c_first; c <= c_last; ++c) {  // contributor order: the result does not depend on arrival order
-              const int slot = (sk_begin(c, T, G) / sp.kbs == tile) ? 0 : 1;  // tile is c's first segment?
-              const float* part = p.partials + (static_cast<size_t>(c) * 2 + slot) * (kSkinnyTileN * sp.m_pad);
+            if (n < big_extent) sk_load_cin16<kTall>(p, m0, n, cin);  // in flight together with the partials
+            // Contributor order, so that the result does not depend on arrival order; four contributors' loads are in
+            // flight at a time.  The loads are unconditional (past the last contributor they repeat it) because loads
+            // under a condition were scheduled one contributor, and one round trip to memory, after the other.
+            for (int c = c_first; c <= c_last; c += 4) {
+              float v[4][16];
 #pragma unroll
-              for (int j = 0; j < 16; ++j)
-                if (m0 + j < small_extent) sum[j] += __ldcg(part + (m0 + j) * kSkinnyTileN + n_local);
+              for (int b = 0; b < 4; ++b) {
+                const float* part = partial_of(min(c + b, c_last));
+#pragma unroll
+                for (int j = 0; j < 16; ++j) v[b][j] = __ldcg(part + (m0 + j) * kSkinnyTileN + n_local);  // m0 + j < m_pad
+              }
+#pragma unroll
+              for (int b = 0; b < 4; ++b)
+                if (c + b <= c_last) {
+#pragma unroll
+                  for (int j = 0; j < 16; ++j) sum[j] += v[b][j];
+                }
             }
-            if (n < big_extent) sk_finish16<kTall>(p, m0, n, sum);
+            if (n < big_extent) sk_finish16<kTall>(p, m0, n, sum, cin);
           }
           if (leader) p.counters[tile] = 0u;  // leave the counter clean for the next launch
         }
@@ -342,13 +419,15 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
   }
 }
 
-// Zero the arrival counters and launch.  Returns a gemm_status_t value (0 = ok, 7 = CUDA failure).
+// Launch, after zeroing the arrival counters when the caller cannot vouch for them (`zero_counters`; a plan's own
+// counters are zero from their allocation on, since every run puts them back).  Returns a gemm_status_t value
+// (0 = ok, 7 = CUDA failure).
 // `tall` selects the mirrored addressing (tW then maps A, tX maps B).
 inline int skinny_launch(const SkinnyParams& p, const CUtensorMap& tW, const CUtensorMap& tX, int device, cudaStream_t stream,
-                         char* err, size_t err_len, bool tall = false) {
+                         char* err, size_t err_len, bool tall, bool zero_counters) {
   cudaError_t e = tall ? ensure_dynamic_smem(reinterpret_cast<const void*>(skinny_gemm_kernel<true>), kSlotSkinnyTall, device, p.plan.smem_bytes)
                        : ensure_dynamic_smem(reinterpret_cast<const void*>(skinny_gemm_kernel<false>), kSlotSkinny, device, p.plan.smem_bytes);
-  if (e == cudaSuccess) e = cudaMemsetAsync(p.counters, 0, p.plan.counters_bytes, stream);
+  if (e == cudaSuccess && zero_counters) e = cudaMemsetAsync(p.counters, 0, p.plan.counters_bytes, stream);
   if (e == cudaSuccess) {
     if (tall) skinny_gemm_kernel<true><<<p.plan.grid, kSkinnyThreads, p.plan.smem_bytes, stream>>>(tW, tX, p);
     else skinny_gemm_kernel<false><<<p.plan.grid, kSkinnyThreads, p.plan.smem_bytes, stream>>>(tW, tX, p);

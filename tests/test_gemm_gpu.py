@@ -271,7 +271,7 @@ def test_runs_on_a_side_stream():
 def test_bounded_wait_reports_timeout_and_context_survives(variant):
     """A producer arrival is withheld by a test flag, so a device-side wait runs into its limit; the
     kernel must return on its own, the plan must report GEMM_ERR_TIMEOUT and later work must run."""
-    w = int_workload("stall", 8 if variant == VS else 512, 512, 256)
+    w = int_workload("stall", 8 if variant == VS else 512, 512, 256 if variant != VS else 8192)  # stream-K: split tiles
     inputs = wl.make_inputs(w)
     tile_n = 0 if variant in (VW, VS) else 128
     plan = bg.Plan(H.desc_of(w, bg.make_flags(variant, tile_n, debug_stall=True)))
@@ -280,7 +280,18 @@ def test_bounded_wait_reports_timeout_and_context_survives(variant):
     C = torch.zeros(w.elems_c(), dtype=torch.float32, device="cuda")
     plan.run(A, B, C)
     torch.cuda.synchronize()
+    plan.run(A, B, C)                      # before the status has been read: may give up early, must not hang or fault
+    torch.cuda.synchronize()
     assert plan.status() == bg.ERR_TIMEOUT
     assert plan.status() == bg.OK          # reading clears the word
+    # the hook acts on the first run only: the same plan must now give the exact result (for stream-K this needs the
+    # arrival counters of the abandoned runs to have been put back to zero)
+    for _ in range(2):
+        C.fill_(float("nan"))
+        plan.run(A, B, C)
+        torch.cuda.synchronize()
+        assert plan.status() == bg.OK
+        reports = H.check_blocks(w, inputs, H.to_host_bits(C, w.c_dtype), H.default_blocks(w))
+        assert all(r["bit_identical"] == 1.0 for r in reports)
     plan.close()
     H.check_workload(w, bg.make_flags(variant, tile_n), exact=True)

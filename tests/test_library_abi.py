@@ -118,8 +118,8 @@ def test_stream_k_plan_geometry():
     assert i5["num_tiles"] == 224 * 64               # (n-tile, 128-wide k-block) work units
     assert i5["grid"] == 148 and i5["tile_m"] == 128 and i5["tile_n"] == 16 and i5["tile_k"] == 128
     assert i5["split"] >= 2 and i5["stages"] == 4    # 4 stages of two 64-wide K slices: 144 KB in flight per SM
-    # counters (224 x 4 bytes padded to 256) + 2 partial slots of 128 x 16 fp32 per CTA
-    assert i5["workspace_bytes"] == 1024 + 148 * 2 * 128 * 16 * 4
+    # 2 partial slots of 128 x 16 fp32 per CTA (the arrival counters belong to the plan, not to the workspace)
+    assert i5["workspace_bytes"] == 148 * 2 * 128 * 16 * 4
     tiny = info_for(wl.Workload("t", 4, 100, 64), bg.make_flags(bg.VARIANT_SKINNY_STREAMK))
     assert tiny["grid"] == 1 and tiny["num_tiles"] == 1
 
