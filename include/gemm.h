@@ -90,6 +90,10 @@ typedef enum {
 #define GEMM_FLAG_KSLICES_MASK 0x30000000u
 #define GEMM_FLAG_NO_K_SERPENTINE 0x8u      /* walk K forwards in every tile (default: alternate tiles walk it backwards,
                                               which re-uses the operand lines L2 touched last) */
+#define GEMM_FLAG_NO_EARLY_LAUNCH 0x4u       /* launch without programmatic dependent launch (default: the kernel may be
+                                              scheduled while the previous kernel of the stream is finishing and does
+                                              its set-up then; it waits for that kernel to complete before it reads or
+                                              writes global memory) */
 #define GEMM_FLAG_L2_HINTS 0x40000000u     /* load A with evict-last and B with evict-first L2 priority (default: normal) */
 #define GEMM_FLAG_DEBUG_STALL 0x80000000u  /* test hook: in the plan's first run one producer arrival is withheld so that
                                               a bounded wait expires and GEMM_ERR_TIMEOUT is reported; later runs are normal */

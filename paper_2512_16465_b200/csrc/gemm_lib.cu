@@ -616,13 +616,15 @@ gemm_status_t launch_dense(const gemm_plan_s* pl, const CUtensorMap& tA, const C
   cfg.blockDim = dim3(64 + 128 * EPI_WG, 1, 1);
   cfg.dynamicSmemBytes = pl->smem_bytes;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = CG;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // set-up may overlap the previous kernel's tail
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = (pl->d.flags & GEMM_FLAG_NO_EARLY_LAUNCH) ? 1 : 2;
   cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tA, tB, tD, p);
   if (e != cudaSuccess) {
     note_cuda_error("cudaLaunchKernelEx(dense)", cudaGetErrorName(e));
@@ -644,13 +646,15 @@ gemm_status_t launch_wide(const gemm_plan_s* pl, const CUtensorMap& tA, const CU
   cfg.blockDim = dim3(kWideThreads, 1, 1);
   cfg.dynamicSmemBytes = pl->smem_bytes;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // set-up may overlap the previous kernel's tail
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = (pl->d.flags & GEMM_FLAG_NO_EARLY_LAUNCH) ? 1 : 2;
   cudaError_t e = cudaLaunchKernelEx(&cfg, wide_gemm_kernel, tA, tB, tD, p);
   if (e != cudaSuccess) {
     note_cuda_error("cudaLaunchKernelEx(wide)", cudaGetErrorName(e));
@@ -723,7 +727,8 @@ gemm_status_t run_skinny(gemm_plan_s* pl, const void* A, const void* B, void* C,
   p.status = pl->d_status;
   p.timeout_ns = static_cast<unsigned long long>(pl->timeout_ms) * 1000000ull;
   return static_cast<gemm_status_t>(
-      skinny_launch(p, tW, tX, pl->device, stream, g_last_cuda_error, sizeof g_last_cuda_error, pl->skinny_tall, /*zero_counters=*/false));
+      skinny_launch(p, tW, tX, pl->device, stream, g_last_cuda_error, sizeof g_last_cuda_error, pl->skinny_tall, /*zero_counters=*/false,
+                    /*early_launch=*/!(d.flags & GEMM_FLAG_NO_EARLY_LAUNCH)));
 }
 
 }  // namespace
@@ -866,7 +871,8 @@ extern "C" gemm_status_t gemm_skinny_run_noalloc(const gemm_desc_t* desc, const 
   p.partials = reinterpret_cast<float*>(nd.scratch + kNoAllocHeaderBytes + sp.counters_bytes);
   p.timeout_ns = 2000ull * 1000000ull;
   st = static_cast<gemm_status_t>(
-      skinny_launch(p, tW, tX, dev, s, g_last_cuda_error, sizeof g_last_cuda_error, /*tall=*/false, /*zero_counters=*/true));
+      skinny_launch(p, tW, tX, dev, s, g_last_cuda_error, sizeof g_last_cuda_error, /*tall=*/false, /*zero_counters=*/true,
+                    /*early_launch=*/false));
   if (st != GEMM_OK || !sync_and_check) return st;
   uint32_t word = 0;
   e = cudaStreamSynchronize(s);

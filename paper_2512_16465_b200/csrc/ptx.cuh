@@ -83,6 +83,12 @@ __device__ __forceinline__ uint32_t atom_add_acq_rel_gpu(uint32_t* addr, uint32_
   asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(old) : "l"(addr), "r"(v) : "memory");
   return old;
 }
+// Programmatic dependent launch.  launch_dependents lets the next kernel of the stream (if it was launched with the
+// programmatic-serialisation attribute) be scheduled before this grid has finished; wait blocks until every grid this
+// one depends on has completed and its memory operations are visible.  Everything before the wait must touch
+// nothing but this CTA's own shared and tensor memory.  Both are no-ops in a launch without the attribute.
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ uint32_t ld_acquire_gpu(const uint32_t* addr) {
   uint32_t v;
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(addr) : "memory");

@@ -22,6 +22,8 @@
 #pragma once
 #include <cuda_runtime.h>
 
+#include <cstring>
+
 #include "dense_kernel.cuh"
 #include "launch_util.cuh"
 
@@ -148,6 +150,7 @@ template <bool kTall>
 __global__ void __launch_bounds__(kSkinnyThreads, 1)
 skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, const SkinnyParams p) {
   extern __shared__ uint8_t smem_raw[];
+  griddep_launch_dependents();  // the next kernel's set-up may overlap this one; it waits below before touching global memory
   const uint32_t raw = smem_addr(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* gen = smem_raw + (base - raw);
@@ -174,10 +177,6 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
   const int tile0 = u_begin / sp.kbs;
   const int kb0 = u_begin - tile0 * sp.kbs;
   const int n_units = u_end - u_begin;
-  // An earlier run of this plan that timed out may have left arrival counters half counted; the status word stays
-  // set until the host has read it (and cleaned the counters), and until then no run trusts them.  The load is
-  // issued here and consumed only by the fix-up, long after it has landed.
-  const uint32_t stale_status = *reinterpret_cast<volatile const uint32_t*>(p.status);
   const uint32_t tmem_cols = sp.m_pad * 2 <= 32 ? 32u : (sp.m_pad * 2 <= 64 ? 64u : 128u);
 
   if (threadIdx.x == 0) {
@@ -202,6 +201,11 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  griddep_wait();  // barriers and tensor memory are set up; from here on global memory is read and written
+  // An earlier run of this plan that timed out may have left arrival counters half counted; the status word stays
+  // set until the host has read it (and cleaned the counters), and until then no run trusts them.  The load is
+  // issued here and consumed only by the fix-up, long after it has landed.
+  const uint32_t stale_status = *reinterpret_cast<volatile const uint32_t*>(p.status);
 
   // The producer and MMA roles run warp-uniform (one elected lane issues), with the (tile, k-block) position and
   // the ring slot advanced incrementally: the single issuing thread must sustain one 18 KB stage every few hundred
@@ -424,14 +428,23 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
 // (0 = ok, 7 = CUDA failure).
 // `tall` selects the mirrored addressing (tW then maps A, tX maps B).
 inline int skinny_launch(const SkinnyParams& p, const CUtensorMap& tW, const CUtensorMap& tX, int device, cudaStream_t stream,
-                         char* err, size_t err_len, bool tall, bool zero_counters) {
+                         char* err, size_t err_len, bool tall, bool zero_counters, bool early_launch) {
   cudaError_t e = tall ? ensure_dynamic_smem(reinterpret_cast<const void*>(skinny_gemm_kernel<true>), kSlotSkinnyTall, device, p.plan.smem_bytes)
                        : ensure_dynamic_smem(reinterpret_cast<const void*>(skinny_gemm_kernel<false>), kSlotSkinny, device, p.plan.smem_bytes);
   if (e == cudaSuccess && zero_counters) e = cudaMemsetAsync(p.counters, 0, p.plan.counters_bytes, stream);
   if (e == cudaSuccess) {
-    if (tall) skinny_gemm_kernel<true><<<p.plan.grid, kSkinnyThreads, p.plan.smem_bytes, stream>>>(tW, tX, p);
-    else skinny_gemm_kernel<false><<<p.plan.grid, kSkinnyThreads, p.plan.smem_bytes, stream>>>(tW, tX, p);
-    e = cudaGetLastError();
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(p.plan.grid, 1, 1);
+    cfg.blockDim = dim3(kSkinnyThreads, 1, 1);
+    cfg.dynamicSmemBytes = p.plan.smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // set-up may overlap the previous kernel's tail
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = early_launch ? 1 : 0;
+    e = tall ? cudaLaunchKernelEx(&cfg, skinny_gemm_kernel<true>, tW, tX, p) : cudaLaunchKernelEx(&cfg, skinny_gemm_kernel<false>, tW, tX, p);
   }
   if (e != cudaSuccess) {
     snprintf(err, err_len, "skinny launch: %s", cudaGetErrorName(e));

@@ -313,6 +313,7 @@ __global__ void __launch_bounds__(kWideThreads, 1)
 wide_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const __grid_constant__ CUtensorMap tmD, const DenseParams p) {
   extern __shared__ uint8_t smem_raw[];
+  griddep_launch_dependents();  // the next kernel's set-up may overlap this one; it waits below before touching global memory
   const uint32_t raw = smem_addr(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* gen = smem_raw + (base - raw);
@@ -357,6 +358,7 @@ wide_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   cluster_wait();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  griddep_wait();  // barriers and tensor memory are set up; from here on global memory is read and written
 
   if (warp == 0) {
     wide_producer_role(p, &tmA, &tmB, base, full0, empty0, cta_rank, cluster_id, num_clusters, w);

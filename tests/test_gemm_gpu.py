@@ -95,6 +95,8 @@ EXACT_CASES = [
     ("skinny_one_slice_stages", 8, 256, 4096, {}, dict(variant=VS, kslices=1)),
     ("skinny_three_slice_stages", 8, 384, 1100 - 4, {}, dict(variant=VS, kslices=3)),
     ("skinny_k_slice_past_the_end", 8, 256, 1080, {}, dict(variant=VS)),
+    ("no_early_launch_1cta", 264, 328, 200, {}, dict(variant=V1, tile_n=128, no_early_launch=True)),
+    ("no_early_launch_skinny", 8, 256, 4096, dict(beta=1.0), dict(variant=VS, no_early_launch=True)),
     # mirrored stream-K: a tall output with a handful of columns (A is the streamed operand)
     ("tall_one_unit", 128, 8, 64, {}, dict(variant=VS)),
     ("tall_split_k", 256, 8, 4096, {}, dict(variant=VS)),
