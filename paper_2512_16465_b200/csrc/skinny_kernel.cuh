@@ -310,19 +310,24 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
       // While the main loop of this segment runs, these warps have nothing to do.  The usual case for the CTA that
       // computes the head of a split tile is that all other contributors finished long ago; if the count says so,
       // their partials (and C_in) are fetched now, this CTA never publishes its own partial and the tail of the kernel
-      // is one tensor-memory read, a few adds and the stores.  (One chunk of 16 and at most four contributors, so that
-      // everything fits in registers; other shapes take the general path below.)  Both paths add the same values in
-      // the same order, so the result does not depend on which one ran.
+      // is one tensor-memory read, a few adds and the stores.  The 64 prefetch registers hold either one chunk of 16
+      // from up to four contributors (short extent <= 16) or up to four chunks from the one other contributor; other
+      // shapes take the general path below.  Both paths add the same values in the same order, so the result does
+      // not depend on which one ran.
       bool early = false;
       float pre[4][16], cin0[16];
-      if (!whole && sp.m_pad == 16 && c_last - c_first <= 3) {
+      const bool by_chunk = sp.m_pad > 16;  // pre[b] = chunk b of the other contributor (else: chunk 0 of contributor b)
+      if (!whole && (by_chunk ? c_last - c_first == 1 : c_last - c_first <= 3)) {
         if (leader) s_early[seg == 0 ? 0 : 1] = (stale_status == 0u && ld_acquire_gpu(p.counters + tile) == static_cast<uint32_t>(c_last - c_first)) ? 1u : 0u;
         named_barrier_sync(1, 128);
         early = s_early[seg == 0 ? 0 : 1] != 0u;
         if (early) {
 #pragma unroll
+          const int other = c_first == static_cast<int>(blockIdx.x) ? c_last : c_first;
           for (int b = 0; b < 4; ++b) {
-            const float* part = partial_of(min(c_first + b, c_last));  // (this CTA's own slot is read too and not used)
+            // (by contributor: this CTA's own slot is read too and not used; by chunk: chunks past m_pad repeat the last)
+            const float* part = by_chunk ? partial_of(other) + min(b * 16, sp.m_pad - 16) * kSkinnyTileN
+                                         : partial_of(min(c_first + b, c_last));
 #pragma unroll
             for (int j = 0; j < 16; ++j) pre[b][j] = __ldcg(part + j * kSkinnyTileN + n_local);
           }
@@ -346,18 +351,27 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
             sk_finish16<kTall>(p, c0, n, accf, cin);
           }
         } else if (early) {
-          float sum[16];
+          float sum[16], cin[16];
 #pragma unroll
           for (int j = 0; j < 16; ++j) sum[j] = 0.0f;
 #pragma unroll
+          for (int j = 0; j < 16; ++j) cin[j] = cin0[j];
+          if (c0 != 0 && n < big_extent) sk_load_cin16<kTall>(p, c0, n, cin);
+#pragma unroll
           for (int b = 0; b < 4; ++b) {
+            // by contributor: b-th contributor; by chunk: the two contributors in order, the other one's chunk c0 / 16
             const int cc = c_first + b;
             if (cc <= c_last) {
+              const bool own = cc == static_cast<int>(blockIdx.x);
 #pragma unroll
-              for (int j = 0; j < 16; ++j) sum[j] += (cc == static_cast<int>(blockIdx.x)) ? __uint_as_float(acc[j]) : pre[b][j];
+              for (int j = 0; j < 16; ++j) {
+                float other_v = pre[b][j];
+                if (by_chunk) other_v = c0 == 0 ? pre[0][j] : (c0 == 16 ? pre[1][j] : (c0 == 32 ? pre[2][j] : pre[3][j]));
+                sum[j] += own ? __uint_as_float(acc[j]) : other_v;
+              }
             }
           }
-          if (n < big_extent) sk_finish16<kTall>(p, 0, n, sum, cin0);
+          if (n < big_extent) sk_finish16<kTall>(p, c0, n, sum, cin);
         } else {
 #pragma unroll
           for (int j = 0; j < 16; ++j)
