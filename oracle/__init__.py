@@ -21,7 +21,8 @@ _SRC = os.path.join(_HERE, "gemm_oracle.c")
 _LIB = os.path.join(_HERE, "libgemm_oracle.so")
 
 BF16, F16, F32 = 0, 1, 2
-EPI_NONE, EPI_BIAS, EPI_RELU, EPI_BIAS_RELU, EPI_GELU_ERF, EPI_BIAS_GELU_ERF = range(6)
+(EPI_NONE, EPI_BIAS, EPI_RELU, EPI_BIAS_RELU, EPI_GELU_ERF, EPI_BIAS_GELU_ERF, EPI_GELU_TANH, EPI_BIAS_GELU_TANH,
+ EPI_SILU, EPI_BIAS_SILU) = range(10)
 
 
 def build(force: bool = False) -> str:
@@ -40,7 +41,7 @@ class _Desc(ctypes.Structure):
                 ("lda", ctypes.c_int64), ("ldb", ctypes.c_int64), ("ldc", ctypes.c_int64),
                 ("stride_a", ctypes.c_int64), ("stride_b", ctypes.c_int64),
                 ("stride_c", ctypes.c_int64),
-                ("epilogue", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+                ("epilogue", ctypes.c_int32), ("bias_per_row", ctypes.c_int32)]
 
 
 _lib = None
@@ -62,6 +63,9 @@ def lib() -> ctypes.CDLL:
         L.oracle_gelu_erf.argtypes = [ctypes.c_double]
         L.oracle_gelu_erf_alt.restype = ctypes.c_double
         L.oracle_gelu_erf_alt.argtypes = [ctypes.c_double]
+        for name in ("oracle_logistic", "oracle_silu", "oracle_gelu_tanh"):
+            getattr(L, name).restype = ctypes.c_double
+            getattr(L, name).argtypes = [ctypes.c_double]
         L.oracle_gemm.restype = ctypes.c_int
         L.oracle_gemm.argtypes = [ctypes.POINTER(_Desc), ctypes.c_void_p, ctypes.c_void_p,
                                   ctypes.c_void_p, ctypes.c_void_p, ctypes.c_float, ctypes.c_float,
@@ -95,6 +99,7 @@ class Problem:
     stride_b: int = 0
     stride_c: int = 0
     epilogue: int = EPI_NONE
+    bias_per_row: bool = False   # bias has M entries, one per output row (default: N entries, one per column)
 
     def finalize(self) -> "Problem":
         if not self.lda:
@@ -114,7 +119,7 @@ class Problem:
     def _cdesc(self) -> _Desc:
         return _Desc(self.M, self.N, self.K, self.transa, self.transb, self.ab_dtype, self.c_dtype,
                      self.lda, self.ldb, self.ldc, self.stride_a, self.stride_b, self.stride_c,
-                     self.epilogue, 0)
+                     self.epilogue, 1 if self.bias_per_row else 0)
 
 
 def _ptr(a):
@@ -127,7 +132,7 @@ def gemm(p: Problem, A, B, C_in=None, bias=None, alpha=1.0, beta=0.0,
 
     Returns ``(y, bound)``, fp64 arrays of shape ``[len(batches), len(rows), len(cols)]``:
     the unrounded result and the tolerance scale
-    ``|alpha| sum|a||b| + |beta||C_in| + |bias_j|``.
+    ``|alpha| sum|a||b| + |beta||C_in| + |bias|``.
     """
     p.finalize()
     batches = np.arange(p.batch, dtype=np.int64) if batches is None else np.ascontiguousarray(batches, np.int64)

@@ -9,7 +9,9 @@
  * ("GEMM", Section 5.4) written out as a plain triple loop:
  *
  *     y(b,i,j) = act( alpha * sum_{k=0}^{K-1} opA(b,i,k) * opB(b,k,j)
- *                     + beta * C_in(b,i,j) + bias[j] )
+ *                     + beta * C_in(b,i,j) + bias[j] )        (bias[i] when bias_per_row)
+ *
+ * act: identity, ReLU, GELU (exact erf form), GELU (tanh form) or SiLU;
  *
  * evaluated in IEEE double, k ascending, one output at a time, no blocking,
  * no reassociation (build without -ffast-math).  Inputs arrive as the very bit
@@ -29,7 +31,9 @@
  * Parity pins (tests/test_oracle_pins.py): exhaustive codec round trips and
  * hand values, identity / permutation matrices, all-ones inputs (= K), rank-1
  * closed form, hand-computed tiny cases, alpha/beta special cases, batched ==
- * loop of singles, textbook values of the normal CDF for GELU, and numpy's
+ * loop of singles, textbook values of the normal CDF for GELU, closed forms of
+ * the logistic function for SiLU and the tanh GELU (plus the library's fp64
+ * routines), row bias == column bias of the transposed product, and numpy's
  * fp64 matmul on small shapes.
  */
 #include <math.h>
@@ -37,8 +41,10 @@
 #include <string.h>
 
 enum { OR_BF16 = 0, OR_F16 = 1, OR_F32 = 2 };
+/* even values: no bias; odd values: the same activation with a bias added first */
 enum { OR_EPI_NONE = 0, OR_EPI_BIAS = 1, OR_EPI_RELU = 2, OR_EPI_BIAS_RELU = 3,
-       OR_EPI_GELU_ERF = 4, OR_EPI_BIAS_GELU_ERF = 5 };
+       OR_EPI_GELU_ERF = 4, OR_EPI_BIAS_GELU_ERF = 5, OR_EPI_GELU_TANH = 6, OR_EPI_BIAS_GELU_TANH = 7,
+       OR_EPI_SILU = 8, OR_EPI_BIAS_SILU = 9 };
 
 typedef struct {
   int64_t M, N, K;
@@ -48,7 +54,7 @@ typedef struct {
   int64_t lda, ldb, ldc;
   int64_t stride_a, stride_b, stride_c;
   int32_t epilogue;
-  int32_t reserved;
+  int32_t bias_per_row;  /* 0: bias[N], one value per output column; 1: bias[M], one value per output row */
 } oracle_desc_t;
 
 /* ---- codecs: bit pattern -> double (exact) ------------------------------ */
@@ -119,6 +125,22 @@ double oracle_gelu_erf(double t) { return 0.5 * t * erfc(-t * 0.7071067811865475
 /* The same function through erf; the pins require both forms to agree. */
 double oracle_gelu_erf_alt(double t) { return 0.5 * t * (1.0 + erf(t * 0.70710678118654752440)); }
 
+/* The logistic function 1 / (1 + e^-t), evaluated on the side where the exponential cannot overflow. */
+double oracle_logistic(double t) {
+  if (t >= 0.0) return 1.0 / (1.0 + exp(-t));
+  double e = exp(t);
+  return e / (1.0 + e);
+}
+/* SiLU (swish): t * logistic(t). */
+double oracle_silu(double t) { return t * oracle_logistic(t); }
+/* GELU, tanh form: 0.5 t (1 + tanh u) with u = sqrt(2/pi) (t + 0.044715 t^3).  Evaluated as t * logistic(2u),
+ * the same function (0.5 (1 + tanh u) = 1 / (1 + e^-2u)) without the cancellation of 1 + tanh u in the negative
+ * tail; the pins compare it with the tanh expression. */
+double oracle_gelu_tanh(double t) {
+  double u = 0.79788456080286535588 * (t + 0.044715 * t * t * t);
+  return t * oracle_logistic(2.0 * u);
+}
+
 int oracle_max_threads(void);
 
 static double load_ab(const void* p, int dtype, int64_t idx) {
@@ -135,7 +157,7 @@ static double load_c(const void* p, int dtype, int64_t idx) {
  * Evaluate the definition on the cross product batches x rows x cols.
  * Outputs (each nb*nr*nc doubles, [batch][row][col] order):
  *   y      unrounded fp64 result
- *   bound  |alpha| * sum_k |a||b| + |beta| * |C_in| + |bias_j|   (tolerance scale)
+ *   bound  |alpha| * sum_k |a||b| + |beta| * |C_in| + |bias|   (tolerance scale)
  * `bound` may be NULL.  `threads` <= 0 lets OpenMP decide.  Returns 0, or -1
  * on a bad argument.
  */
@@ -144,10 +166,12 @@ int oracle_gemm(const oracle_desc_t* d, const void* A, const void* B, const void
                 const int64_t* batches, int64_t nb, const int64_t* rows, int64_t nr,
                 const int64_t* cols, int64_t nc, double* y, double* bound, int threads) {
   if (!d || !A || !B || !y || !batches || !rows || !cols) return -1;
-  int has_bias = d->epilogue == OR_EPI_BIAS || d->epilogue == OR_EPI_BIAS_RELU ||
-                 d->epilogue == OR_EPI_BIAS_GELU_ERF;
+  if (d->epilogue < OR_EPI_NONE || d->epilogue > OR_EPI_BIAS_SILU) return -1;
+  int has_bias = d->epilogue & 1;
   int relu = d->epilogue == OR_EPI_RELU || d->epilogue == OR_EPI_BIAS_RELU;
   int gelu = d->epilogue == OR_EPI_GELU_ERF || d->epilogue == OR_EPI_BIAS_GELU_ERF;
+  int gelu_tanh = d->epilogue == OR_EPI_GELU_TANH || d->epilogue == OR_EPI_BIAS_GELU_TANH;
+  int silu = d->epilogue == OR_EPI_SILU || d->epilogue == OR_EPI_BIAS_SILU;
   if (has_bias && !bias) return -1;
   if (beta != 0.0f && !C_in) return -1;
   const int64_t K = d->K;
@@ -178,11 +202,14 @@ int oracle_gemm(const oracle_desc_t* d, const void* A, const void* B, const void
       bnd += fabs(dbeta) * fabs(cv);
     }
     if (has_bias) {
-      t += (double)bias[j];
-      bnd += fabs((double)bias[j]);
+      double bv = (double)bias[d->bias_per_row ? i : j];
+      t += bv;
+      bnd += fabs(bv);
     }
     if (relu) t = t > 0.0 ? t : 0.0;
     if (gelu) t = oracle_gelu_erf(t);
+    if (gelu_tanh) t = oracle_gelu_tanh(t);
+    if (silu) t = oracle_silu(t);
     y[o] = t;
     if (bound) bound[o] = bnd;
   }

@@ -252,6 +252,62 @@ def test_gelu_textbook_values_and_identities(golden_dir):
     assert g(12.0) == 12.0 and abs(g(-12.0)) < 1e-30
 
 
+def test_logistic_silu_and_tanh_gelu(golden_dir):
+    L = oracle.lib()
+    sg, silu, gt, ge = L.oracle_logistic, L.oracle_silu, L.oracle_gelu_tanh, L.oracle_gelu_erf
+    for line in open(os.path.join(golden_dir, "logistic_values.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        x, want = map(float, line.split())
+        assert abs(sg(x) - want) < 2e-16 * 4, x
+        assert abs(silu(x) - x * want) < 1e-15 * max(1.0, abs(x)), x
+    xs = np.linspace(-30, 30, 481)
+    for x in xs:
+        assert abs(sg(x) + sg(-x) - 1.0) < 3e-16                          # s(x) + s(-x) = 1
+        assert abs((silu(x) - silu(-x)) - x) < 1e-15 * max(1.0, abs(x))   # hence silu(x) - silu(-x) = x
+        assert abs((gt(x) - gt(-x)) - x) < 1e-15 * max(1.0, abs(x))       # tanh is odd: the same identity
+        u = math.sqrt(2.0 / math.pi) * (x + 0.044715 * x ** 3)
+        assert abs(gt(x) - 0.5 * x * (1.0 + math.tanh(u))) < 4e-16 * max(1.0, abs(x))   # the tanh expression itself
+    assert sg(800.0) == 1.0 and sg(-800.0) == 0.0 and silu(-800.0) == 0.0   # no overflow on either side
+    assert silu(0.0) == 0.0 and gt(0.0) == 0.0 and gt(10.0) == 10.0 and abs(gt(-10.0)) < 1e-30
+    # the tanh form approximates x Phi(x): the two differ, but by less than 5e-4 anywhere
+    dev = max(abs(gt(x) - ge(x)) for x in np.linspace(-6, 6, 2401))
+    assert 1e-4 < dev < 5e-4
+    # library routines in fp64
+    import torch
+    t = torch.linspace(-12, 12, 1001, dtype=torch.float64)
+    assert np.allclose([silu(float(v)) for v in t], torch.nn.functional.silu(t).numpy(), rtol=1e-14, atol=1e-300)
+    assert np.allclose([gt(float(v)) for v in t], torch.nn.functional.gelu(t, approximate="tanh").numpy(), rtol=1e-13, atol=1e-14)
+
+
+def test_new_activations_and_row_bias_in_the_gemm():
+    M, N, K = 6, 9, 16
+    a = ints((M, K), -2, 2, 41)
+    b = ints((K, N), -2, 2, 42)
+    bias_n = (np.arange(N, dtype=np.float32) - 3.25) / 4
+    bias_m = (np.arange(M, dtype=np.float32) * 0.5 - 1.0)
+    y0, b0 = oracle.gemm(Problem(M, N, K), a, b)
+    L = oracle.lib()
+    for epi, f in ((oracle.EPI_BIAS_SILU, L.oracle_silu), (oracle.EPI_BIAS_GELU_TANH, L.oracle_gelu_tanh)):
+        y, _ = oracle.gemm(Problem(M, N, K, epilogue=epi), a, b, bias=bias_n, alpha=0.25)
+        want = np.vectorize(f)(0.25 * y0[0] + bias_n[None, :])
+        assert np.array_equal(y[0], want)
+        y, _ = oracle.gemm(Problem(M, N, K, epilogue=epi - 1), a, b, alpha=0.25)     # the bias-free twin
+        assert np.array_equal(y[0], np.vectorize(f)(0.25 * y0[0]))
+    # a per-row bias: one value per output row, also in the tolerance scale
+    y, bd = oracle.gemm(Problem(M, N, K, epilogue=oracle.EPI_BIAS, bias_per_row=True), a, b, bias=bias_m)
+    assert np.array_equal(y[0], y0[0] + bias_m[:, None])
+    assert np.array_equal(bd[0], b0[0] + np.abs(bias_m)[:, None])
+    # ... which is the per-column bias of the transposed product (A B)^T = B^T A^T
+    at = np.ascontiguousarray(a.T)
+    bt = np.ascontiguousarray(b.T)
+    yt, _ = oracle.gemm(Problem(N, M, K, epilogue=oracle.EPI_BIAS_RELU), bt, at, bias=bias_m)
+    y, _ = oracle.gemm(Problem(M, N, K, epilogue=oracle.EPI_BIAS_RELU, bias_per_row=True), a, b, bias=bias_m)
+    assert np.array_equal(y[0], yt[0].T)
+    with pytest.raises(ValueError):
+        oracle.gemm(Problem(M, N, K, epilogue=10), a, b)                              # unknown epilogue
+
+
 def test_batched_equals_loop_of_singles():
     w = wl.Workload("t", 9, 7, 12, transa=0, transb=1, ab_dtype=F16, batch=4, beta=0.5, c_dtype=F16,
                     dist_a=wl.Dist("uniform", -2, 2), dist_b=wl.Dist("uniform", -2, 2), alpha=0.25,
