@@ -152,7 +152,8 @@ class DeviceCase:
             if r == 0:
                 self.host_inputs = inp
         d = bg.make_desc(w.M, w.N, w.K, w.transa, w.transb, w.ab_dtype, w.c_dtype, w.lda, w.ldb, w.ldc, w.batch,
-                         w.stride_a, w.stride_b, w.stride_c, w.epilogue, flags)
+                         w.stride_a, w.stride_b, w.stride_c, w.epilogue,
+                         flags | (bg.make_flags(bias_per_row=True) if w.bias_per_row else 0))
         self.plan = bg.Plan(d)
         self.plan.workspace(device)
         self.i = 0
@@ -385,12 +386,14 @@ def run_ours(args):
 
 def parse_shape(spec: str) -> wl.Workload:
     """'MxNxK' followed by optional ':key=value' fields: batch, ta, tb (1 = stored transposed), ab/cd (bf16|f16|f32),
-    epi (none|bias|relu|bias_relu|gelu|bias_gelu), alpha, beta, lda, ldb, ldc.  Example: 28672x8x8192:beta=1:cd=f32."""
+    epi (none|bias|relu|bias_relu|gelu|bias_gelu|gelu_tanh|bias_gelu_tanh|silu|bias_silu), rowbias (0|1), alpha, beta,
+    lda, ldb, ldc.  Example: 28672x8x8192:beta=1:cd=f32."""
     head, *fields = spec.split(":")
     M, N, K = (int(x) for x in head.lower().split("x"))
     dt = {"bf16": wl.BF16, "f16": wl.F16, "f32": wl.F32}
     epi = {"none": wl.EPI_NONE, "bias": wl.EPI_BIAS, "relu": wl.EPI_RELU, "bias_relu": wl.EPI_BIAS_RELU,
-           "gelu": wl.EPI_GELU_ERF, "bias_gelu": wl.EPI_BIAS_GELU_ERF}
+           "gelu": wl.EPI_GELU_ERF, "bias_gelu": wl.EPI_BIAS_GELU_ERF, "gelu_tanh": wl.EPI_GELU_TANH,
+           "bias_gelu_tanh": wl.EPI_BIAS_GELU_TANH, "silu": wl.EPI_SILU, "bias_silu": wl.EPI_BIAS_SILU}
     kw = dict(c_dtype=wl.BF16, dist_a=wl.Dist("normal", 0.0, 0.02), dist_b=wl.Dist("normal", 0.0, 0.02))
     for f in fields:
         k, v = f.split("=")
@@ -404,6 +407,8 @@ def parse_shape(spec: str) -> wl.Workload:
             kw["epilogue"] = epi[v]
         elif k in ("alpha", "beta"):
             kw[k] = float(v)
+        elif k == "rowbias":
+            kw["bias_per_row"] = bool(int(v))
         elif k in ("lda", "ldb", "ldc"):  # leading dimensions in elements (each must span a multiple of 16 bytes)
             kw[k] = int(v)
         else:

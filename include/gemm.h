@@ -64,7 +64,11 @@ typedef enum {
   GEMM_EPI_RELU = 2,
   GEMM_EPI_BIAS_RELU = 3,
   GEMM_EPI_GELU_ERF = 4,     /* x * Phi(x) with the exact error function */
-  GEMM_EPI_BIAS_GELU_ERF = 5
+  GEMM_EPI_BIAS_GELU_ERF = 5,
+  GEMM_EPI_GELU_TANH = 6,    /* 0.5 x (1 + tanh(sqrt(2/pi) (x + 0.044715 x^3))) */
+  GEMM_EPI_BIAS_GELU_TANH = 7,
+  GEMM_EPI_SILU = 8,         /* x / (1 + e^-x) */
+  GEMM_EPI_BIAS_SILU = 9     /* odd values: the bias is added before the activation */
 } gemm_epilogue_t;
 
 /* Roofline class of a problem (Section 4.3 of the paper, applied at plan time). */
@@ -90,6 +94,8 @@ typedef enum {
 #define GEMM_FLAG_KSLICES_MASK 0x30000000u
 #define GEMM_FLAG_NO_K_SERPENTINE 0x8u      /* walk K forwards in every tile (default: alternate tiles walk it backwards,
                                               which re-uses the operand lines L2 touched last) */
+#define GEMM_FLAG_BIAS_PER_ROW 0x1u         /* the bias is fp32[M], one value per output row (default: fp32[N], one per
+                                              column); not a tuning knob: it changes what is computed */
 #define GEMM_FLAG_NO_EARLY_LAUNCH 0x4u       /* launch without programmatic dependent launch (default: the kernel may be
                                               scheduled while the previous kernel of the stream is finishing and does
                                               its set-up then; it waits for that kernel to complete before it reads or
@@ -152,8 +158,9 @@ size_t gemm_workspace_bytes(gemm_plan_t plan);
 /*
  * gemm_run -- enqueue D = act(alpha*op(A)*op(B) + beta*C + bias) on `stream`
  * (asynchronous; the hot path of Section 5.4).  A, B, C: device pointers, 16-byte
- * aligned, laid out as `desc` said.  bias: device fp32[N], required iff the
- * epilogue has a bias.  C is read only when beta != 0.  workspace: device
+ * aligned, laid out as `desc` said.  bias: device fp32[N] (fp32[M] with
+ * GEMM_FLAG_BIAS_PER_ROW), shared by all batches, required iff the epilogue
+ * has a bias.  C is read only when beta != 0.  workspace: device
  * memory of at least gemm_workspace_bytes(plan) bytes, 16-byte aligned (may be NULL when
  * that is 0).  Runs of one dense plan may overlap on the GPU; runs of one
  * stream-K plan must not (they share the plan's arrival counters, which every

@@ -50,6 +50,7 @@ struct DenseParams {
   uint32_t a_kstep, b_kstep;              // start-address advance per K = 16 slice, bytes
   int out_dtype;                          // 0 bf16, 1 f16, 2 f32
   int epilogue;                           // gemm_epilogue_t
+  int bias_per_row;                       // the bias has M entries (one per output row) instead of N
   float alpha, beta;
   const float* bias;
   const void* c_in;                       // = D buffer; read when beta != 0
@@ -179,7 +180,38 @@ __device__ __forceinline__ float gelu_erf(float t) {
   return 0.5f * t * (t < 0.0f ? g : 2.0f - g);
 }
 
-// alpha/beta/bias/activation on 32 consecutive columns of one output row, in fp32.
+// x * logistic(x): one ex2 and one reciprocal.  Far in the negative tail e^-x overflows to +inf, the reciprocal is 0
+// and the result -0, the limit.
+__device__ __forceinline__ float silu(float t) {
+  float e, r;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(-1.4426950408889634f * t));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.0f + e));
+  return t * r;
+}
+// GELU, tanh form: 0.5 t (1 + tanh u) = t * logistic(2u), u = sqrt(2/pi) (t + 0.044715 t^3).  The constants are
+// 2 sqrt(2/pi) log2(e) and that times 0.044715.
+__device__ __forceinline__ float gelu_tanh(float t) {
+  const float a = t * fmaf(0.10294324f * t, t, 2.3022082f);
+  float e, r;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(-a));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.0f + e));
+  return t * r;
+}
+// The activation of gemm_epilogue_t value `epilogue` (value >> 1: none, ReLU, erf GELU, tanh GELU, SiLU).
+__device__ __forceinline__ float activate(float v, int act) {
+  if (act == 1) return fmaxf(v, 0.0f);
+  if (act == 2) return gelu_erf(v);
+  if (act == 3) return gelu_tanh(v);
+  if (act == 4) return silu(v);
+  return v;
+}
+
+// alpha/beta/bias/activation on 32 consecutive columns of one output row, in fp32.  kAll = false is the wide pair
+// kernel's subset (bias per column, ReLU, erf GELU): its epilogue runs at the 168-register ceiling, and of the code
+// shapes tried only this one, with erf GELU through erff(), was allocated without spills (the polynomial GELU, the
+// further activations, and even no GELU at all spilled 16 to 48 bytes).  The plan never picks that kernel for a
+// transcendental epilogue, so the slower erff() is not on any automatic path.
+template <bool kAll = true>
 __device__ __forceinline__ void epilogue_math(float (&v)[32], const uint32_t (&acc)[32], const DenseParams& p, long long row,
                                               int col0, int batch) {
 #pragma unroll
@@ -231,7 +263,11 @@ __device__ __forceinline__ void epilogue_math(float (&v)[32], const uint32_t (&a
       }
     }
   }
-  if (p.epilogue & 1) {  // bias variants are the odd enum values
+  if (kAll && (p.epilogue & 1) && p.bias_per_row) {  // bias variants are the odd enum values
+    const float b = row < p.M ? __ldg(p.bias + row) : 0.0f;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] += b;
+  } else if (p.epilogue & 1) {
     if (col0 + 32 <= p.N) {
       const float4* b4 = reinterpret_cast<const float4*>(p.bias + col0);
 #pragma unroll
@@ -247,12 +283,22 @@ __device__ __forceinline__ void epilogue_math(float (&v)[32], const uint32_t (&a
         if (col0 + j < p.N) v[j] += __ldg(p.bias + col0 + j);
     }
   }
+  const int act = p.epilogue >> 1;
   if (p.epilogue == 2 || p.epilogue == 3) {
 #pragma unroll
     for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.0f);
-  } else if (p.epilogue >= 4) {
+  } else if (!kAll && p.epilogue >= 4) {  // (only erf GELU reaches the wide kernel)
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = 0.5f * v[j] * (1.0f + erff(v[j] * 0.70710678118654752f));
+  } else if (kAll && act == 2) {
 #pragma unroll
     for (int j = 0; j < 32; ++j) v[j] = gelu_erf(v[j]);
+  } else if (kAll && act == 3) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = gelu_tanh(v[j]);
+  } else if (kAll && act == 4) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = silu(v[j]);
   }
 }
 

@@ -115,7 +115,7 @@ struct gemm_plan_s {
 
 namespace {
 
-bool has_bias(int epi) { return epi == GEMM_EPI_BIAS || epi == GEMM_EPI_BIAS_RELU || epi == GEMM_EPI_BIAS_GELU_ERF; }
+bool has_bias(int epi) { return (epi & 1) != 0; }  // the odd gemm_epilogue_t values
 
 gemm_status_t validate(const gemm_desc_t* d) {
   if (d->struct_size != sizeof(gemm_desc_t)) return GEMM_ERR_INVALID_ARG;
@@ -125,7 +125,7 @@ gemm_status_t validate(const gemm_desc_t* d) {
     return GEMM_ERR_INVALID_ARG;
   if (d->ab_dtype < GEMM_BF16 || d->ab_dtype > GEMM_F32 || d->c_dtype < GEMM_BF16 || d->c_dtype > GEMM_F32)
     return GEMM_ERR_INVALID_ARG;
-  if (d->epilogue < GEMM_EPI_NONE || d->epilogue > GEMM_EPI_BIAS_GELU_ERF) return GEMM_ERR_INVALID_ARG;
+  if (d->epilogue < GEMM_EPI_NONE || d->epilogue > GEMM_EPI_BIAS_SILU) return GEMM_ERR_INVALID_ARG;
   if (d->ab_dtype == GEMM_F32) return GEMM_ERR_UNSUPPORTED;
   const int64_t a_row = d->transa == GEMM_OP_N ? d->K : d->M;
   const int64_t b_row = d->transb == GEMM_OP_N ? d->N : d->K;
@@ -177,7 +177,7 @@ double estimate_dense_cycles(const gemm_desc_t& d, int sm_count, int variant, in
   const double feed = kblocks * (rows_cta + static_cast<double>(bn) / cg) * 128.0 / 90.0;
   // output: this SM's share of the HBM write bandwidth is ~16 B/clk
   const double out = static_cast<double>(rows_cta) * bn * elem_bytes(d.c_dtype) / 16.0;
-  const bool gelu = d.epilogue >= GEMM_EPI_GELU_ERF;
+  const bool gelu = d.epilogue >= GEMM_EPI_GELU_ERF;  // any transcendental activation
   double exposed = 400.0;                       // barrier round trips per tile that nothing hides
   if (wide) exposed = gelu ? 9000.0 : 3000.0;   // no second accumulator: read-out (and conversion) of half 0
   else if (cg == 2) exposed = 1000.0;           // pair hand-shakes cross the SM-to-SM network
@@ -282,6 +282,7 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   p.b_kstep = b_kmajor ? kUmmaK * 2 : kUmmaK * 128;
   p.out_dtype = d.c_dtype;
   p.epilogue = d.epilogue;
+  p.bias_per_row = (d.flags & GEMM_FLAG_BIAS_PER_ROW) ? 1 : 0;
   p.ldc = d.ldc;
   p.stride_c = d.batch_count > 1 ? d.stride_c : 0;
   p.debug_flags = 0u;  // set per run
@@ -320,6 +321,8 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
 // Wide pair variant: 512 x 256 cluster tiles, one 64-wide K slice per stage, 3-deep ring, 8 epilogue warps.
 gemm_status_t plan_wide(gemm_plan_s* pl, int forced_raster, int forced_stages) {
   const gemm_desc_t& d = pl->d;
+  // its epilogue covers the bias per column, ReLU and erf GELU only
+  if (d.epilogue > GEMM_EPI_BIAS_GELU_ERF || (d.flags & GEMM_FLAG_BIAS_PER_ROW)) return GEMM_ERR_UNSUPPORTED;
   const int a_kmajor = d.transa == GEMM_OP_N;
   const int b_kmajor = d.transb == GEMM_OP_T;
   const int tile_m = 2 * kWideCtaM, bn = kWideTileN;
@@ -366,6 +369,7 @@ gemm_status_t plan_wide(gemm_plan_s* pl, int forced_raster, int forced_stages) {
   p.b_kstep = b_kmajor ? kUmmaK * 2 : kUmmaK * 128;
   p.out_dtype = d.c_dtype;
   p.epilogue = d.epilogue;
+  p.bias_per_row = (d.flags & GEMM_FLAG_BIAS_PER_ROW) ? 1 : 0;
   p.ldc = d.ldc;
   p.stride_c = d.batch_count > 1 ? d.stride_c : 0;
   p.debug_flags = 0u;  // set per run
@@ -462,7 +466,7 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
   const double flops = 2.0 * d.M * d.N * d.K * d.batch_count;
   double bytes = d.batch_count * (static_cast<double>(d.M) * d.K + static_cast<double>(d.K) * d.N) * eb +
                  d.batch_count * static_cast<double>(d.M) * d.N * ec;
-  if (has_bias(d.epilogue)) bytes += 4.0 * d.N;
+  if (has_bias(d.epilogue)) bytes += 4.0 * ((d.flags & GEMM_FLAG_BIAS_PER_ROW) ? d.M : d.N);
   gemm_info_t& info = pl->info;
   info.struct_size = sizeof(gemm_info_t);
   info.flops = flops;
@@ -491,6 +495,7 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
       for (int v : {GEMM_VARIANT_DENSE_1CTA, GEMM_VARIANT_DENSE_2CTA, GEMM_VARIANT_DENSE_2CTA_WIDE}) {
         for (int bn : {256, 128, 64}) {
           if (v == GEMM_VARIANT_DENSE_2CTA_WIDE && bn != kWideTileN) continue;
+          if (v == GEMM_VARIANT_DENSE_2CTA_WIDE && (d.epilogue > GEMM_EPI_BIAS_GELU_ERF || (d.flags & GEMM_FLAG_BIAS_PER_ROW))) continue;
           if (v == GEMM_VARIANT_DENSE_2CTA && !b_kmajor && bn % 128) continue;  // 64-column boxes per CTA
           if (v != GEMM_VARIANT_DENSE_1CTA && d.M <= kCtaM) continue;           // a pair needs two tile rows
           if (forced_bn && bn != forced_bn) continue;
@@ -716,6 +721,7 @@ gemm_status_t run_skinny(gemm_plan_s* pl, const void* A, const void* B, void* C,
   p.idesc = make_idesc(d.ab_dtype == GEMM_BF16, 0, 0, kSkinnyTileN, s.m_pad);
   p.out_dtype = d.c_dtype;
   p.epilogue = d.epilogue;
+  p.bias_per_row = (d.flags & GEMM_FLAG_BIAS_PER_ROW) ? 1 : 0;
   p.alpha = alpha;
   p.beta = beta;
   p.bias = bias;
@@ -861,6 +867,7 @@ extern "C" gemm_status_t gemm_skinny_run_noalloc(const gemm_desc_t* desc, const 
   p.idesc = make_idesc(desc->ab_dtype == GEMM_BF16, 0, 0, kSkinnyTileN, sp.m_pad);
   p.out_dtype = desc->c_dtype;
   p.epilogue = desc->epilogue;
+  p.bias_per_row = 0;  // desc->flags is ignored by this entry point
   p.alpha = alpha;
   p.beta = beta;
   p.bias = bias;

@@ -92,6 +92,7 @@ struct SkinnyParams {
   uint32_t idesc;
   int out_dtype;
   int epilogue;
+  int bias_per_row;       // the bias has M entries (one per output row) instead of N
   float alpha, beta;
   const float* bias;
   void* c;                // D buffer (also C_in when beta != 0), row-major M x N
@@ -133,14 +134,15 @@ template <bool kTall>
 __device__ __forceinline__ void sk_finish16(const SkinnyParams& p, int s0, int big, const float (&acc)[16], const float (&cin)[16]) {
   const int small_extent = kTall ? p.N : p.M;
   const bool has_bias = (p.epilogue & 1) != 0;
-  const float bias_big = (!kTall && has_bias) ? __ldg(p.bias + big) : 0.0f;  // the bias runs along N
+  // the bias runs along N (the long extent unless kTall) or, per row, along M
+  const bool bias_along_big = kTall ? p.bias_per_row != 0 : p.bias_per_row == 0;
+  const float bias_big = (bias_along_big && has_bias) ? __ldg(p.bias + big) : 0.0f;
+  const int act = p.epilogue >> 1;
 #pragma unroll
   for (int j = 0; j < 16; ++j) {
     if (s0 + j < small_extent) {
-      const float bias = (kTall && has_bias) ? __ldg(p.bias + s0 + j) : bias_big;
-      float v = p.alpha * acc[j] + p.beta * cin[j] + bias;
-      if (p.epilogue == 2 || p.epilogue == 3) v = fmaxf(v, 0.0f);
-      else if (p.epilogue >= 4) v = gelu_erf(v);
+      const float bias = (!bias_along_big && has_bias) ? __ldg(p.bias + s0 + j) : bias_big;
+      const float v = activate(p.alpha * acc[j] + p.beta * cin[j] + bias, act);
       sk_store_d(p, sk_index<kTall>(p, s0 + j, big), v);
     }
   }

@@ -237,7 +237,7 @@ __device__ __forceinline__ void wide_epilogue_role(const DenseParams& p, const C
             const uint32_t srow = sbuf + lane * 128u;
             if (lane == 0) bulk_wait_group_read<1>();  // the store that last read this slab has finished with it
             __syncwarp();
-            epilogue_math(v, u == 0 ? acc0 : acc1, p, row, col0, tc.batch);
+            epilogue_math<false>(v, u == 0 ? acc0 : acc1, p, row, col0, tc.batch);
 #pragma unroll
             for (int j = 0; j < 8; ++j)
               st_shared_v4(srow + ((static_cast<uint32_t>(j) ^ sw) << 4), __float_as_uint(v[4 * j]), __float_as_uint(v[4 * j + 1]),
@@ -266,7 +266,7 @@ __device__ __forceinline__ void wide_epilogue_role(const DenseParams& p, const C
             if (lane == 0) mbar_arrive_cluster(mapa(tempty0 + 8u * h, 0));
           }
           const int col64 = colbase + 64 * static_cast<int>(part);
-          epilogue_math(v, acc0, p, row, col64, tc.batch);
+          epilogue_math<false>(v, acc0, p, row, col64, tc.batch);
           if (p.out_dtype == 0) {
 #pragma unroll
             for (int j = 0; j < 16; ++j) pk[j] = pack_bf16x2_pinned(v[2 * j], v[2 * j + 1]);
@@ -274,7 +274,7 @@ __device__ __forceinline__ void wide_epilogue_role(const DenseParams& p, const C
 #pragma unroll
             for (int j = 0; j < 16; ++j) pk[j] = pack_f16x2_pinned(v[2 * j], v[2 * j + 1]);
           }
-          epilogue_math(v, acc1, p, row, col64 + 32, tc.batch);
+          epilogue_math<false>(v, acc1, p, row, col64 + 32, tc.batch);
           if (p.out_dtype == 0) {
 #pragma unroll
             for (int j = 0; j < 16; ++j) pk[16 + j] = pack_bf16x2_pinned(v[2 * j], v[2 * j + 1]);

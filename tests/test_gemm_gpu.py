@@ -217,6 +217,48 @@ def test_gelu_epilogue_values():
     assert reports[0]["frob"] < 1e-5
 
 
+ACTIVATIONS = [bg.EPI_GELU_ERF, bg.EPI_BIAS_GELU_ERF, bg.EPI_GELU_TANH, bg.EPI_BIAS_GELU_TANH, bg.EPI_SILU, bg.EPI_BIAS_SILU]
+
+
+@pytest.mark.parametrize("epi", ACTIVATIONS)
+@pytest.mark.parametrize("shape", ["dense_1cta", "dense_pair", "stream_k", "stream_k_tall"])
+def test_activation_epilogues(epi, shape):
+    """Every transcendental activation on every kernel family, wide value range (|t| up to ~15), fp32 output:
+    the stated per-element tolerance and a relative Frobenius error far below it."""
+    M, N, K, fl = {"dense_1cta": (200, 264, 136, dict(variant=V1)), "dense_pair": (300, 264, 136, dict(variant=V2, tile_n=128)),
+                   "stream_k": (8, 520, 1032, dict(variant=VS)), "stream_k_tall": (520, 8, 1032, dict(variant=VS))}[shape]
+    w = wl.Workload(f"act_{shape}", M, N, K, transb=1, epilogue=epi, c_dtype=wl.F32, beta=0.5,
+                    dist_a=wl.Dist("normal", 0, 1), dist_b=wl.Dist("normal", 0, 0.15), dist_bias=wl.Dist("normal", 0, 1.0), seed=7)
+    reports, _ = H.check_workload(w, bg.make_flags(**fl))
+    assert reports[0]["frob"] < 1e-5 and reports[0]["max_err_over_tol"] < 0.05
+
+
+@pytest.mark.parametrize("case", [
+    ("row_bias_1cta", 200, 328, 136, dict(epi=bg.EPI_BIAS), dict(variant=V1)),
+    ("row_bias_pair_relu_bf16", 300, 264, 136, dict(epi=bg.EPI_BIAS_RELU, cd=wl.BF16), dict(variant=V2, tile_n=128)),
+    ("row_bias_ragged_rows", 130, 64, 72, dict(epi=bg.EPI_BIAS, beta=1.0), dict(variant=V1)),
+    ("row_bias_batched", 96, 72, 64, dict(epi=bg.EPI_BIAS, batch=3), dict(variant=V1)),
+    ("row_bias_stream_k", 8, 520, 1032, dict(epi=bg.EPI_BIAS_RELU), dict(variant=VS)),
+    ("row_bias_stream_k_tall", 520, 8, 1032, dict(epi=bg.EPI_BIAS, beta=1.0), dict(variant=VS)),
+    ("row_bias_auto", 1024, 512, 256, dict(epi=bg.EPI_BIAS), dict()),
+], ids=lambda c: c[0])
+def test_bias_per_row_exact(case):
+    name, M, N, K, kw, fl = case
+    w = int_workload(name, M, N, K, bias_per_row=True, **kw)
+    H.check_workload(w, bg.make_flags(**fl), exact=True, repeats=2)
+
+
+def test_wide_kernel_refuses_what_its_epilogue_lacks():
+    for kw in (dict(epilogue=bg.EPI_SILU), dict(epilogue=bg.EPI_BIAS_GELU_TANH), dict(epilogue=bg.EPI_BIAS, flags_extra=dict(bias_per_row=True))):
+        extra = kw.pop("flags_extra", {})
+        with pytest.raises(bg.GemmError) as e:
+            bg.gemm_plan(bg.make_desc(1024, 1024, 4096, flags=bg.make_flags(VW, **extra), **kw))
+        assert e.value.status == bg.ERR_UNSUPPORTED
+    h = bg.gemm_plan(bg.make_desc(8192, 8192, 8192, c_dtype=bg.BF16, epilogue=bg.EPI_BIAS_SILU))   # the automatic plan goes elsewhere
+    assert bg.gemm_plan_info(h)["variant"] == V2
+    bg.gemm_destroy(h)
+
+
 # ----------------------------------------------------------------------------- boundary behaviour on a device
 
 def test_run_argument_errors_launch_nothing():

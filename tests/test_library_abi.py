@@ -55,7 +55,8 @@ def test_plan_validation_codes():
     assert plan_status(**ok, lda=128) == bg.ERR_INVALID_ARG          # lda < K
     assert plan_status(**ok, ldc=255) == bg.ERR_INVALID_ARG
     assert plan_status(**ok, transa=2) == bg.ERR_INVALID_ARG
-    assert plan_status(**ok, epilogue=6) == bg.ERR_INVALID_ARG
+    assert plan_status(**ok, epilogue=10) == bg.ERR_INVALID_ARG
+    assert plan_status(**ok, epilogue=bg.EPI_BIAS_SILU) == bg.OK
     assert plan_status(**ok, c_dtype=3) == bg.ERR_INVALID_ARG
     assert plan_status(**ok, ab_dtype=bg.F32) == bg.ERR_UNSUPPORTED
     assert plan_status(M=256, N=256, K=100, lda=100) == bg.ERR_ALIGNMENT     # 200-byte rows

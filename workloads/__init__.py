@@ -25,7 +25,8 @@ _SRC = os.path.join(_HERE, "gen.c")
 _LIB = os.path.join(_HERE, "libworkloads_gen.so")
 
 BF16, F16, F32 = 0, 1, 2
-EPI_NONE, EPI_BIAS, EPI_RELU, EPI_BIAS_RELU, EPI_GELU_ERF, EPI_BIAS_GELU_ERF = range(6)
+(EPI_NONE, EPI_BIAS, EPI_RELU, EPI_BIAS_RELU, EPI_GELU_ERF, EPI_BIAS_GELU_ERF, EPI_GELU_TANH, EPI_BIAS_GELU_TANH,
+ EPI_SILU, EPI_BIAS_SILU) = range(10)
 ELEM_BYTES = {BF16: 2, F16: 2, F32: 4}
 TENSOR_A, TENSOR_B, TENSOR_C, TENSOR_BIAS = 1, 2, 3, 4
 BASE_SEED = 0x5EED0000
@@ -108,6 +109,7 @@ class Workload:
     c_dtype: int = F32
     batch: int = 1
     epilogue: int = EPI_NONE
+    bias_per_row: bool = False   # the bias has M entries (one per output row) instead of N
     alpha: float = 1.0
     beta: float = 0.0
     dist_a: Dist = field(default_factory=lambda: Dist("normal", 0.0, 1.0))
@@ -143,7 +145,7 @@ class Workload:
 
     @property
     def has_bias(self) -> bool:
-        return self.epilogue in (EPI_BIAS, EPI_BIAS_RELU, EPI_BIAS_GELU_ERF)
+        return bool(self.epilogue & 1)   # the odd epilogue values
 
     @property
     def flops(self) -> float:
@@ -158,7 +160,7 @@ class Workload:
         if self.beta != 0.0:
             n += self.batch * self.M * self.N * cb
         if self.has_bias:
-            n += self.N * 4
+            n += (self.M if self.bias_per_row else self.N) * 4
         return float(n)
 
     def elems_a(self) -> int:
@@ -191,7 +193,7 @@ def make_inputs(w: Workload, seed_offset: int = 0) -> dict:
     if w.beta != 0.0:
         out["C"] = _draw(w.dist_c, s, TENSOR_C, w.elems_c(), w.c_dtype)
     if w.has_bias:
-        out["bias"] = _draw(w.dist_bias, s, TENSOR_BIAS, w.N, F32)
+        out["bias"] = _draw(w.dist_bias, s, TENSOR_BIAS, w.M if w.bias_per_row else w.N, F32)
     return out
 
 
