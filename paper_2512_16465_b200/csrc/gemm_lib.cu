@@ -169,7 +169,7 @@ double estimate_dense_cycles(const gemm_desc_t& d, int sm_count, int variant, in
   const long long waves = (tiles + units - 1) / units;
   const double kblocks = static_cast<double>(ceil_div(d.K, kBlockK));
   // tensor pipe: one 128 x bn x 16 MMA per CTA takes bn / 2 cycles; four per k-block and 128-row half
-  static const double eff1[3] = {0.45, 0.68, 0.88}, eff2[3] = {0.55, 0.80, 0.95};  // bn = 64, 128, 256 (measured, 8192^3)
+  static const double eff1[3] = {0.45, 0.68, 0.88}, eff2[3] = {0.55, 0.80, 0.938};  // bn = 64, 128, 256 (measured, 8192^3)
   const int bi = bn <= 64 ? 0 : (bn <= 128 ? 1 : 2);
   const double eff = wide ? 1.0 : (cg == 1 ? eff1[bi] : eff2[bi]);
   const double mma = kblocks * 4.0 * (bn / 2.0) * (rows_cta / 128.0) / eff;
@@ -179,7 +179,9 @@ double estimate_dense_cycles(const gemm_desc_t& d, int sm_count, int variant, in
   const double out = static_cast<double>(rows_cta) * bn * elem_bytes(d.c_dtype) / 16.0;
   const bool gelu = d.epilogue >= GEMM_EPI_GELU_ERF;  // any transcendental activation
   double exposed = 400.0;                       // barrier round trips per tile that nothing hides
-  if (wide) exposed = gelu ? 9000.0 : 3000.0;   // no second accumulator: read-out (and conversion) of half 0
+  // no second accumulator: read-out (and bias fetch, conversion) of half 0; fitted, like the pair efficiency above, to
+  // measured pair-vs-wide time ratios at K = 4096 ... 16384 on 8192 x 8192 and 16384 x 14336 outputs
+  if (wide) exposed = (gelu ? 13000.0 : 5100.0) + (has_bias(d.epilogue) ? 1300.0 : 0.0);
   else if (cg == 2) exposed = 1000.0;           // pair hand-shakes cross the SM-to-SM network
   const double per_tile = std::max(mma, std::max(feed, out)) + exposed;
   return static_cast<double>(waves) * per_tile + 3000.0;  // + pipeline fill and drain
