@@ -459,6 +459,23 @@ def run_shapes(args):
                 e1.record()
                 torch.cuda.synchronize()
                 row["library_reference_ms"] = round(e0.elapsed_time(e1) / steps, 5)
+            if args.tune:
+                # measured plan selection on the first input set (its C is scratch from here on), then the same timing
+                # loop again: the new plan picks the remembered choice up by itself
+                A, B, C, bias = case.sets[0]
+                tuned, rep = bg.Plan.tuned(case.plan.desc, A, B, C, bias, w.alpha, w.beta, iterations=10)
+                tuned.close()
+                case.close()
+                case = DeviceCase(torch, bg, spec, w, 0, device)
+                torch.cuda.synchronize()
+                time.sleep(0.3)
+                sec2 = case.time_steps(steps, warmup)
+                row["tuned"] = {"ms_per_step": round(sec2 * 1e3, 5), "flags": hex(rep["best_flags"]),
+                                "plan": {k: case.plan.info[k] for k in ("variant", "tile_m", "tile_n", "tile_k", "stages", "raster_group")},
+                                "candidates_tried": rep["candidates_tried"], "candidates_skipped": rep["candidates_skipped"],
+                                "tuner_auto_ms": round(rep["auto_ms"], 5), "tuner_best_ms": round(rep["best_ms"], 5),
+                                "roofline_frac": roofline_for(w, spec, sec2, peaks, peak_kind)["frac"]}
+                bg.gemm_tune_cache_clear()
             rows.append(row)
             case.close()
     print(json.dumps({"shapes_measured": rows, "steps": steps, "warmup": warmup, "clocks": clocks.summary(),
@@ -524,6 +541,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--ref-step-seconds", type=float, default=10.0, help="--impl reference: CPU time budget of one step")
     ap.add_argument("--shapes", default="", help="';'-separated MxNxK[:key=value...] problems to time instead of the five configurations")
+    ap.add_argument("--tune", action="store_true", help="--shapes: also plan by measurement (gemm_tune) and time the tuned plan")
     ap.add_argument("--library-reference", action="store_true", help="--shapes: also time torch.matmul on the same operands (context)")
     args = ap.parse_args()
     if args.impl == "reference":

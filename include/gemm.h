@@ -214,6 +214,48 @@ gemm_status_t gemm_destroy(gemm_plan_t plan);
 gemm_status_t gemm_skinny_run_noalloc(const gemm_desc_t* desc, const void* A, const void* B, void* C, const float* bias,
                                       float alpha, float beta, gemm_stream_t stream, int sync_and_check);
 
+/*
+ * Measured plan selection.  The paper's search (Section 4.3: the roofline class of a kernel steers which
+ * optimisations are tried, and candidates are kept by measured time) has one part that needs no language
+ * model: among the handful of kernel families, tile widths, ring shapes and raster heights this library
+ * has, try the ones the problem's roofline class makes plausible, time them on the caller's buffers, keep
+ * the fastest and remember it for the shape.
+ *
+ * GEMM_TUNE_MAX_CANDIDATES bounds the report arrays.
+ */
+#define GEMM_TUNE_MAX_CANDIDATES 32
+typedef struct {
+  uint32_t struct_size;         /* = sizeof(gemm_tune_report_t) */
+  int32_t candidates_tried;     /* plans that ran and were timed (entries of tried_*) */
+  int32_t candidates_skipped;   /* refused by gemm_plan for this problem, or needing more workspace than given */
+  uint32_t best_flags;          /* gemm_desc_t.flags of the winner (tuning fields filled in) */
+  float best_ms;                /* its mean device time per launch */
+  float auto_ms;                /* the same for the untuned automatic plan, for comparison */
+  uint32_t tried_flags[GEMM_TUNE_MAX_CANDIDATES];
+  float tried_ms[GEMM_TUNE_MAX_CANDIDATES];
+} gemm_tune_report_t;
+
+/* Workspace that lets gemm_tune try every candidate of this problem (0 if none needs any). */
+size_t gemm_tune_workspace_bytes(const gemm_desc_t* desc);
+
+/*
+ * gemm_tune -- plan `desc` by measurement.  A, B, C, bias, alpha, beta, workspace, stream: as for gemm_run;
+ * every candidate is RUN on them (2 warm-up launches, then `iterations` timed launches between CUDA events
+ * on `stream`; iterations < 1 means 10), so C is overwritten again and again (and, with beta != 0, keeps
+ * accumulating): pass scratch data.  The call synchronises `stream` several times.  Tuning fields of
+ * desc->flags (variant, tile, raster, stages, K slices) are ignored; the other flags are kept.
+ * On success *out_plan is the winner, ready for gemm_run, and the winner's flags are remembered for this
+ * device and shape: later gemm_plan calls with the same shape and no tuning fields set use them.
+ * report may be NULL.  Errors: as gemm_plan and gemm_run; GEMM_ERR_TIMEOUT if a candidate's device-side
+ * wait expired (nothing is remembered then); GEMM_ERR_UNSUPPORTED if no candidate could run.
+ */
+gemm_status_t gemm_tune(const gemm_desc_t* desc, const void* A, const void* B, void* C, const float* bias, float alpha,
+                        float beta, void* workspace, size_t workspace_bytes, gemm_stream_t stream, int iterations,
+                        gemm_plan_t* out_plan, gemm_tune_report_t* report);
+
+/* Forget every remembered tuning result (all devices). */
+void gemm_tune_cache_clear(void);
+
 /* Static string for a status code. */
 const char* gemm_status_string(gemm_status_t s);
 

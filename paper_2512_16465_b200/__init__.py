@@ -57,8 +57,24 @@ class Info(ctypes.Structure):
         return {k: getattr(self, k) for k, _ in self._fields_ if k != "struct_size"}
 
 
+TUNE_MAX_CANDIDATES = 32
+
+
+class TuneReport(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_uint32), ("candidates_tried", ctypes.c_int32), ("candidates_skipped", ctypes.c_int32),
+                ("best_flags", ctypes.c_uint32), ("best_ms", ctypes.c_float), ("auto_ms", ctypes.c_float),
+                ("tried_flags", ctypes.c_uint32 * TUNE_MAX_CANDIDATES), ("tried_ms", ctypes.c_float * TUNE_MAX_CANDIDATES)]
+
+    def as_dict(self) -> dict:
+        n = self.candidates_tried
+        return {"candidates_tried": n, "candidates_skipped": self.candidates_skipped, "best_flags": self.best_flags,
+                "best_ms": self.best_ms, "auto_ms": self.auto_ms,
+                "tried": [(self.tried_flags[i], self.tried_ms[i]) for i in range(n)]}
+
+
 EXPORTS = ("gemm_plan", "gemm_workspace_bytes", "gemm_run", "gemm_plan_status", "gemm_plan_set_timeout_ms",
-           "gemm_plan_info", "gemm_destroy", "gemm_status_string", "gemm_last_cuda_error", "gemm_skinny_run_noalloc")
+           "gemm_plan_info", "gemm_destroy", "gemm_status_string", "gemm_last_cuda_error", "gemm_skinny_run_noalloc",
+           "gemm_tune", "gemm_tune_workspace_bytes", "gemm_tune_cache_clear")
 
 
 def _load() -> ctypes.CDLL:
@@ -87,6 +103,13 @@ def _load() -> ctypes.CDLL:
     L.gemm_last_cuda_error.argtypes = []
     L.gemm_skinny_run_noalloc.restype = ctypes.c_int
     L.gemm_skinny_run_noalloc.argtypes = [ctypes.POINTER(Desc), vp, vp, vp, vp, ctypes.c_float, ctypes.c_float, vp, ctypes.c_int]
+    L.gemm_tune.restype = ctypes.c_int
+    L.gemm_tune.argtypes = [ctypes.POINTER(Desc), vp, vp, vp, vp, ctypes.c_float, ctypes.c_float, vp, ctypes.c_size_t, vp,
+                            ctypes.c_int, ctypes.POINTER(vp), ctypes.POINTER(TuneReport)]
+    L.gemm_tune_workspace_bytes.restype = ctypes.c_size_t
+    L.gemm_tune_workspace_bytes.argtypes = [ctypes.POINTER(Desc)]
+    L.gemm_tune_cache_clear.restype = None
+    L.gemm_tune_cache_clear.argtypes = []
     return L
 
 
@@ -155,6 +178,28 @@ def gemm_skinny_run_noalloc(desc: Desc, A: int, B: int, C: int, bias: int, alpha
         raise err
 
 
+def gemm_tune_workspace_bytes(desc: Desc) -> int:
+    return int(_lib.gemm_tune_workspace_bytes(ctypes.byref(desc)))
+
+
+def gemm_tune(desc: Desc, A: int, B: int, C: int, bias: int, alpha: float, beta: float, workspace: int, workspace_bytes: int,
+              stream: int, iterations: int = 10):
+    """``gemm_tune``: time the plausible plans of ``desc`` on the given device buffers (C is overwritten repeatedly) and
+    return ``(plan handle of the fastest, report dict)``.  The choice is remembered for later ``gemm_plan`` calls."""
+    h = ctypes.c_void_p()
+    rep = TuneReport()
+    rep.struct_size = ctypes.sizeof(TuneReport)
+    st = _lib.gemm_tune(ctypes.byref(desc), A, B, C, bias or None, alpha, beta, workspace or None, workspace_bytes, stream or None,
+                        iterations, ctypes.byref(h), ctypes.byref(rep))
+    if st != OK:
+        raise GemmError(st, "gemm_tune")
+    return h.value, rep.as_dict()
+
+
+def gemm_tune_cache_clear() -> None:
+    _lib.gemm_tune_cache_clear()
+
+
 def gemm_plan_status(plan: int) -> int:
     return int(_lib.gemm_plan_status(plan))
 
@@ -186,12 +231,23 @@ def _torch_dtype_code(t) -> int:
 class Plan:
     """A planned GEMM bound to torch tensors.  ``run`` enqueues on the current torch stream."""
 
-    def __init__(self, desc: Desc):
+    def __init__(self, desc: Desc, handle: Optional[int] = None):
         self.desc = desc
-        self.handle = gemm_plan(desc)
+        self.handle = gemm_plan(desc) if handle is None else handle
         self.info = gemm_plan_info(self.handle)
         self.workspace_bytes = gemm_workspace_bytes(self.handle)
         self._ws = None
+
+    @classmethod
+    def tuned(cls, desc: Desc, A, B, C, bias=None, alpha: float = 1.0, beta: float = 0.0, iterations: int = 10):
+        """Plan by measurement on these tensors (C is overwritten repeatedly); returns ``(Plan, report)``."""
+        import torch
+        nbytes = gemm_tune_workspace_bytes(desc)
+        ws = torch.empty(max(nbytes, 16), dtype=torch.uint8, device=A.device)
+        s = torch.cuda.current_stream(A.device).cuda_stream
+        h, rep = gemm_tune(desc, A.data_ptr(), B.data_ptr(), C.data_ptr(), 0 if bias is None else bias.data_ptr(), float(alpha),
+                           float(beta), ws.data_ptr(), ws.numel(), s, iterations)
+        return cls(desc, handle=h), rep
 
     def workspace(self, device=None):
         import torch

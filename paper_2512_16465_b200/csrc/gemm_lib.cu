@@ -17,6 +17,7 @@
 
 #include "dense_kernel.cuh"
 #include "skinny_kernel.cuh"
+#include "tune_cache.h"
 #include "wide_kernel.cuh"
 
 using namespace b200;
@@ -461,6 +462,10 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
     }
   }
   (void)cudaGetLastError();
+  if (pl->has_device && (pl->d.flags & kTuningFlagMask) == 0) {  // a measured choice for this shape, if gemm_tune made one
+    uint32_t tuned = 0;
+    if (tune_cache_lookup(pl->d, pl->device, &tuned)) pl->d.flags |= tuned;
+  }
 
   // roofline class (Section 4.3): compulsory traffic vs. work
   const gemm_desc_t& d = pl->d;

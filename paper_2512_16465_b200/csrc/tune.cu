@@ -1,0 +1,258 @@
+// Measured plan selection (gemm_tune) on top of the library's own public calls: candidates are ordinary plans with
+// forced tuning fields, timed with CUDA events on the caller's buffers.  Which candidates are worth trying follows
+// from the problem's roofline class (Section 4.3 of the paper: memory-bound kernels are tuned for streaming, compute-
+// bound ones for tensor-pipe occupancy); the winner is remembered per device and shape.
+#include <cuda_runtime.h>
+
+#include <cstring>
+#include <map>
+#include <mutex>
+#include <tuple>
+#include <vector>
+
+#include "../../include/gemm.h"
+#include "tune_cache.h"
+
+namespace b200 {
+namespace {
+
+using Key = std::tuple<int, int64_t, int64_t, int64_t, int32_t, int32_t, int32_t, int32_t, int64_t, int64_t, int64_t, int32_t, int32_t,
+                       int64_t, int64_t, int64_t, uint32_t>;
+
+Key key_of(const gemm_desc_t& d, int device) {
+  const bool batched = d.batch_count > 1;
+  return Key(device, d.M, d.N, d.K, d.transa, d.transb, d.ab_dtype, d.c_dtype, d.lda, d.ldb, d.ldc, d.batch_count, d.epilogue,
+             batched ? d.stride_a : 0, batched ? d.stride_b : 0, batched ? d.stride_c : 0, d.flags & ~kTuningFlagMask);
+}
+
+std::mutex g_mu;
+std::map<Key, uint32_t>& cache() {
+  static std::map<Key, uint32_t> m;
+  return m;
+}
+
+uint32_t pack(int variant, int tile_n, int raster, int stages, int kslices) {
+  return (static_cast<uint32_t>(variant) << GEMM_FLAG_VARIANT_SHIFT) | (static_cast<uint32_t>(tile_n / 16) << GEMM_FLAG_TILE_N_SHIFT) |
+         (static_cast<uint32_t>(raster) << GEMM_FLAG_RASTER_SHIFT) | (static_cast<uint32_t>(stages) << GEMM_FLAG_STAGES_SHIFT) |
+         (static_cast<uint32_t>(kslices) << GEMM_FLAG_KSLICES_SHIFT);
+}
+
+bool short_extent(const gemm_desc_t& d) {
+  return (d.M <= 64 || d.N <= 64) && d.batch_count == 1 && d.transa == GEMM_OP_N && d.transb == GEMM_OP_T;
+}
+
+// First round: one candidate per kernel family and tile width that the roofline class makes plausible.
+std::vector<uint32_t> first_round(const gemm_desc_t& d, const gemm_info_t& automatic) {
+  std::vector<uint32_t> c;
+  const bool streaming = automatic.regime == GEMM_REGIME_MEMORY || automatic.intensity < 64.0;  // HBM-bound or close to it
+  if (short_extent(d)) {
+    for (int ks = 1; ks <= 3; ++ks) c.push_back(pack(GEMM_VARIANT_SKINNY_STREAMK, 0, 0, 0, ks));
+  }
+  if (streaming) {
+    for (int bn : {64, 128, 256}) c.push_back(pack(GEMM_VARIANT_DENSE_1CTA, bn, 0, 0, 0));
+  } else {
+    for (int bn : {256, 128}) c.push_back(pack(GEMM_VARIANT_DENSE_1CTA, bn, 0, 0, 0));
+    for (int bn : {256, 128}) c.push_back(pack(GEMM_VARIANT_DENSE_2CTA, bn, 0, 0, 0));
+    c.push_back(pack(GEMM_VARIANT_DENSE_2CTA_WIDE, 0, 0, 0, 0));
+  }
+  return c;
+}
+
+// Second round: neighbours of the first-round winner (its plan `w`) in raster height and ring shape.
+std::vector<uint32_t> second_round(uint32_t best, const gemm_info_t& w) {
+  std::vector<uint32_t> c;
+  if (w.variant == GEMM_VARIANT_SKINNY_STREAMK) {
+    for (int st : {w.stages - 1, w.stages + 1})
+      if (st >= 2 && st <= 8) c.push_back((best & ~GEMM_FLAG_STAGES_MASK) | (static_cast<uint32_t>(st) << GEMM_FLAG_STAGES_SHIFT));
+    return c;
+  }
+  for (int rg : {w.raster_group / 2, w.raster_group * 2})
+    if (rg >= 1 && rg <= 64 && rg != w.raster_group)
+      c.push_back((best & ~GEMM_FLAG_RASTER_MASK) | (static_cast<uint32_t>(rg) << GEMM_FLAG_RASTER_SHIFT));
+  if (w.variant != GEMM_VARIANT_DENSE_2CTA_WIDE) {
+    const int ks = w.tile_k / 64;  // 64-wide K slices per stage of the winner
+    c.push_back((best & ~GEMM_FLAG_KSLICES_MASK) | (static_cast<uint32_t>(ks == 1 ? 2 : 1) << GEMM_FLAG_KSLICES_SHIFT));
+  }
+  return c;
+}
+
+struct Timer {
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  bool ok() { return cudaEventCreate(&e0) == cudaSuccess && cudaEventCreate(&e1) == cudaSuccess; }
+  ~Timer() {
+    if (e0) cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+  }
+};
+
+struct Args {
+  const void *A, *B;
+  void* C;
+  const float* bias;
+  float alpha, beta;
+  void* ws;
+  size_t ws_bytes;
+  cudaStream_t stream;
+  int iterations;
+};
+
+// Plan `d` (flags already set), run and time it.  GEMM_OK with *ms < 0 means "not applicable here" (the plan was
+// refused or needs more workspace than given); any other status is an error that ends the tuning.
+gemm_status_t time_candidate(const gemm_desc_t& d, const Args& a, Timer& t, float* ms, gemm_info_t* info) {
+  *ms = -1.0f;
+  gemm_plan_t plan = nullptr;
+  gemm_status_t st = gemm_plan(&d, &plan);
+  if (st == GEMM_ERR_UNSUPPORTED || st == GEMM_ERR_INVALID_ARG) return GEMM_OK;
+  if (st != GEMM_OK) return st;
+  info->struct_size = sizeof *info;
+  (void)gemm_plan_info(plan, info);
+  if (gemm_workspace_bytes(plan) > a.ws_bytes) {
+    gemm_destroy(plan);
+    return GEMM_OK;
+  }
+  for (int i = 0; i < 2 && st == GEMM_OK; ++i) st = gemm_run(plan, a.A, a.B, a.C, a.bias, a.alpha, a.beta, a.ws, a.ws_bytes, a.stream);
+  if (st == GEMM_OK && cudaEventRecord(t.e0, a.stream) != cudaSuccess) st = GEMM_ERR_CUDA;
+  for (int i = 0; i < a.iterations && st == GEMM_OK; ++i) st = gemm_run(plan, a.A, a.B, a.C, a.bias, a.alpha, a.beta, a.ws, a.ws_bytes, a.stream);
+  if (st == GEMM_OK && (cudaEventRecord(t.e1, a.stream) != cudaSuccess || cudaEventSynchronize(t.e1) != cudaSuccess)) st = GEMM_ERR_CUDA;
+  float total = 0.0f;
+  if (st == GEMM_OK && cudaEventElapsedTime(&total, t.e0, t.e1) != cudaSuccess) st = GEMM_ERR_CUDA;
+  if (st == GEMM_OK) st = gemm_plan_status(plan);  // a candidate whose device-side wait expired is an error, not a slow plan
+  gemm_destroy(plan);
+  if (st == GEMM_OK) *ms = total / static_cast<float>(a.iterations);
+  (void)cudaGetLastError();
+  return st;
+}
+
+}  // namespace
+
+bool tune_cache_lookup(const gemm_desc_t& d, int device, uint32_t* flags) {
+  std::lock_guard<std::mutex> lock(g_mu);
+  auto it = cache().find(key_of(d, device));
+  if (it == cache().end()) return false;
+  *flags = it->second;
+  return true;
+}
+
+void tune_cache_store(const gemm_desc_t& d, int device, uint32_t flags) {
+  std::lock_guard<std::mutex> lock(g_mu);
+  cache()[key_of(d, device)] = flags & kTuningFlagMask;
+}
+
+}  // namespace b200
+
+using namespace b200;
+
+extern "C" void gemm_tune_cache_clear(void) {
+  std::lock_guard<std::mutex> lock(g_mu);
+  cache().clear();
+}
+
+extern "C" size_t gemm_tune_workspace_bytes(const gemm_desc_t* desc) {
+  if (!desc || !short_extent(*desc)) return 0;
+  size_t need = 0;
+  for (int ks = 1; ks <= 3; ++ks) {  // only the stream-K candidates use a workspace
+    gemm_desc_t d = *desc;
+    d.flags = (d.flags & ~kTuningFlagMask) | pack(GEMM_VARIANT_SKINNY_STREAMK, 0, 0, 0, ks);
+    gemm_plan_t plan = nullptr;
+    if (gemm_plan(&d, &plan) != GEMM_OK) continue;
+    const size_t b = gemm_workspace_bytes(plan);
+    if (b > need) need = b;
+    gemm_destroy(plan);
+  }
+  return need;
+}
+
+extern "C" gemm_status_t gemm_tune(const gemm_desc_t* desc, const void* A, const void* B, void* C, const float* bias, float alpha,
+                                   float beta, void* workspace, size_t workspace_bytes, gemm_stream_t stream, int iterations,
+                                   gemm_plan_t* out_plan, gemm_tune_report_t* report) {
+  if (!desc || !out_plan || !A || !B || !C) return GEMM_ERR_NULL;
+  *out_plan = nullptr;
+  if (report && report->struct_size != sizeof(gemm_tune_report_t)) return GEMM_ERR_INVALID_ARG;
+  int device = -1;
+  if (cudaGetDevice(&device) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return GEMM_ERR_ARCH;
+  }
+  Timer timer;
+  if (!timer.ok()) {
+    (void)cudaGetLastError();
+    return GEMM_ERR_CUDA;
+  }
+  const Args args{A, B, C, bias, alpha, beta, workspace, workspace ? workspace_bytes : 0, static_cast<cudaStream_t>(stream),
+                  iterations < 1 ? 10 : iterations};
+  gemm_desc_t base = *desc;
+  base.flags &= ~kTuningFlagMask;
+
+  // The untuned automatic plan is the yardstick and the fallback.  (A remembered result must not answer for it.)
+  {
+    std::lock_guard<std::mutex> lock(g_mu);
+    cache().erase(key_of(base, device));
+  }
+  gemm_tune_report_t rep;
+  memset(&rep, 0, sizeof rep);
+  rep.struct_size = sizeof rep;
+  gemm_info_t auto_info, info;
+  float ms = -1.0f;
+  gemm_status_t st = time_candidate(base, args, timer, &ms, &auto_info);
+  if (st != GEMM_OK) return st;
+  if (ms < 0.0f) {  // the automatic plan itself could not run: report why
+    gemm_plan_t probe = nullptr;
+    st = gemm_plan(&base, &probe);
+    if (st != GEMM_OK) return st;
+    const bool ws_short = gemm_workspace_bytes(probe) > args.ws_bytes;
+    gemm_destroy(probe);
+    return ws_short ? GEMM_ERR_WORKSPACE : GEMM_ERR_UNSUPPORTED;
+  }
+  rep.auto_ms = ms;
+  uint32_t best_flags = 0;  // 0 = the automatic plan
+  float best_ms = ms;
+  gemm_info_t best_info = auto_info;
+  auto consider = [&](uint32_t f) -> gemm_status_t {
+    for (int i = 0; i < rep.candidates_tried; ++i)
+      if (rep.tried_flags[i] == f) return GEMM_OK;  // already timed
+    if (rep.candidates_tried >= GEMM_TUNE_MAX_CANDIDATES) return GEMM_OK;
+    gemm_desc_t d = base;
+    d.flags |= f;
+    float t = -1.0f;
+    const gemm_status_t s = time_candidate(d, args, timer, &t, &info);
+    if (s != GEMM_OK) return s;
+    if (t < 0.0f) {
+      ++rep.candidates_skipped;
+      return GEMM_OK;
+    }
+    rep.tried_flags[rep.candidates_tried] = f;
+    rep.tried_ms[rep.candidates_tried] = t;
+    ++rep.candidates_tried;
+    if (t < best_ms) {
+      best_ms = t;
+      best_flags = f;
+      best_info = info;
+    }
+    return GEMM_OK;
+  };
+  rep.tried_flags[0] = 0;
+  rep.tried_ms[0] = ms;
+  rep.candidates_tried = 1;
+  for (uint32_t f : first_round(base, auto_info)) {
+    st = consider(f);
+    if (st != GEMM_OK) return st;
+  }
+  // neighbours of the winner; if the winner is the automatic plan, pin its own choices down first
+  uint32_t pinned = best_flags;
+  if (pinned == 0)
+    pinned = pack(best_info.variant, (best_info.variant == GEMM_VARIANT_DENSE_1CTA || best_info.variant == GEMM_VARIANT_DENSE_2CTA) ? best_info.tile_n : 0, 0, 0, 0);
+  for (uint32_t f : second_round(pinned, best_info)) {
+    st = consider(f);
+    if (st != GEMM_OK) return st;
+  }
+
+  gemm_desc_t win = base;
+  win.flags |= best_flags;
+  st = gemm_plan(&win, out_plan);
+  if (st != GEMM_OK) return st;
+  tune_cache_store(base, device, best_flags);
+  rep.best_flags = win.flags;
+  rep.best_ms = best_ms;
+  if (report) *report = rep;
+  return GEMM_OK;
+}

@@ -339,3 +339,78 @@ def test_bounded_wait_reports_timeout_and_context_survives(variant):
         assert all(r["bit_identical"] == 1.0 for r in reports)
     plan.close()
     H.check_workload(w, bg.make_flags(variant, tile_n), exact=True)
+
+
+# ----------------------------------------------------------------------------- measured plan selection
+
+def _tune_case(w, iterations=5):
+    inputs = wl.make_inputs(w)
+    A, B = H.to_device(inputs["A"], w.ab_dtype), H.to_device(inputs["B"], w.ab_dtype)
+    C = torch.zeros(w.elems_c(), dtype=H._TORCH_DT[w.c_dtype], device="cuda")
+    desc = H.desc_of(w)
+    plan, rep = bg.Plan.tuned(desc, A, B, C, iterations=iterations)
+    return inputs, A, B, C, desc, plan, rep
+
+
+def test_tune_times_candidates_keeps_the_fastest_and_remembers_it():
+    bg.gemm_tune_cache_clear()
+    w = int_workload("tune_dense", 1024, 1536, 512, cd=wl.BF16)
+    inputs, A, B, C, desc, plan, rep = _tune_case(w)
+    times = [t for _, t in rep["tried"]]
+    assert rep["candidates_tried"] >= 5 and all(t > 0 for t in times)
+    assert rep["tried"][0][0] == 0 and abs(rep["auto_ms"] - times[0]) < 1e-9          # the automatic plan is the yardstick
+    assert abs(rep["best_ms"] - min(times)) < 1e-9 and rep["best_ms"] <= rep["auto_ms"]
+    variants = {(f >> 4) & 0xF for f, _ in rep["tried"]}
+    assert {V1, V2} <= variants                                                     # compute-side families were tried
+    C.fill_(float("nan"))
+    plan.run(A, B, C)
+    torch.cuda.synchronize()
+    assert plan.status() == bg.OK
+    reports = H.check_blocks(w, inputs, H.to_host_bits(C, w.c_dtype), H.default_blocks(w))
+    assert all(r["bit_identical"] == 1.0 for r in reports)
+    keys = ("variant", "tile_m", "tile_n", "tile_k", "stages", "raster_group", "grid")
+    again = bg.Plan(desc)                                                           # no tuning fields: the remembered choice
+    assert {k: again.info[k] for k in keys} == {k: plan.info[k] for k in keys}
+    forced = bg.Plan(H.desc_of(w, bg.make_flags(V1, 64)))                           # explicit fields still win
+    assert forced.info["tile_n"] == 64
+    for p in (again, forced, plan):
+        p.close()
+    bg.gemm_tune_cache_clear()
+
+
+def test_tune_short_extent_tries_stream_k_and_dense():
+    bg.gemm_tune_cache_clear()
+    w = int_workload("tune_skinny", 8, 4096, 2048, beta=0.0)
+    inputs, A, B, C, desc, plan, rep = _tune_case(w)
+    variants = {(f >> 4) & 0xF for f, _ in rep["tried"]}
+    assert VS in variants and V1 in variants
+    C.fill_(float("nan"))
+    plan.run(A, B, C)
+    torch.cuda.synchronize()
+    reports = H.check_blocks(w, inputs, H.to_host_bits(C, w.c_dtype), H.default_blocks(w))
+    assert all(r["bit_identical"] == 1.0 for r in reports)
+    plan.close()
+    # without a workspace the stream-K candidates are skipped, not failed
+    s = torch.cuda.current_stream().cuda_stream
+    A64 = torch.zeros(64 * 2048, dtype=torch.bfloat16, device="cuda")
+    C64 = torch.zeros(64 * 4096, device="cuda")
+    h, rep2 = bg.gemm_tune(bg.make_desc(64, 4096, 2048, flags=bg.make_flags(no_early_launch=True)), A64.data_ptr(), B.data_ptr(),
+                           C64.data_ptr(), 0, 1.0, 0.0, 0, 0, s, 3)
+    assert rep2["candidates_skipped"] >= 1 and rep2["best_flags"] & 0x4               # the caller's own flag is kept
+    bg.gemm_destroy(h)
+    bg.gemm_tune_cache_clear()
+
+
+def test_tune_argument_errors():
+    d = bg.make_desc(256, 256, 64)
+    with pytest.raises(bg.GemmError) as e:
+        bg.gemm_tune(d, 0, 16, 16, 0, 1.0, 0.0, 0, 0, 0)
+    assert e.value.status == bg.ERR_NULL
+    A = torch.zeros(256 * 64, dtype=torch.bfloat16, device="cuda")
+    C = torch.zeros(256 * 256, device="cuda")
+    with pytest.raises(bg.GemmError) as e:                                          # bias epilogue without a bias
+        bg.gemm_tune(bg.make_desc(256, 256, 64, epilogue=bg.EPI_BIAS), A.data_ptr(), A.data_ptr(), C.data_ptr(), 0, 1.0, 0.0, 0, 0, 0)
+    assert e.value.status == bg.ERR_NULL
+    with pytest.raises(bg.GemmError) as e:                                          # short-extent shape whose automatic plan needs a workspace
+        bg.gemm_tune(bg.make_desc(8, 256, 4096), A.data_ptr(), A.data_ptr(), C.data_ptr(), 0, 1.0, 0.0, 0, 0, 0)
+    assert e.value.status == bg.ERR_WORKSPACE

@@ -176,3 +176,17 @@ def test_cost_model_choices_follow_the_measurements():
     assert choice(64, 28672, 8192)[0] == bg.VARIANT_DENSE_1CTA               # stream-K stops paying near M = 48
     v, bn = choice(2048, 2048, 128, batch=64)
     assert (v, bn) == (bg.VARIANT_DENSE_1CTA, 256)                           # output-bound: widest tile, fewest hand-shakes
+
+
+def test_tuning_entry_points_on_the_host():
+    # the workspace bound needs no device: only the stream-K candidates of a short-extent problem use one
+    assert bg.gemm_tune_workspace_bytes(bg.make_desc(1024, 1024, 512)) == 0
+    need = bg.gemm_tune_workspace_bytes(bg.make_desc(8, 4096, 2048))
+    assert need >= 148 * 2 * 128 * 16 * 4
+    assert bg.gemm_tune_workspace_bytes(bg.make_desc(4096, 8, 2048)) == need      # mirrored
+    bg.gemm_tune_cache_clear()                                                    # harmless when empty
+    import torch
+    if not torch.cuda.is_available():
+        with pytest.raises(bg.GemmError) as e:
+            bg.gemm_tune(bg.make_desc(256, 256, 64), 16, 16, 16, 0, 1.0, 0.0, 0, 0, 0)
+        assert e.value.status in (bg.ERR_ARCH, bg.ERR_CUDA)                       # no device: an error, never a fallback
