@@ -40,7 +40,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the full-size ncu captures
 # summarised under profiles/ (dense_*_cN_*.txt, skinny_streamk_c5_*.txt; last line of each file).
-NCU_TRAFFIC_BYTES = {"c1": 1122048, "c2": 882350848, "c3": 1645141584, "c4": 545059072, "c5": 476179200}
+NCU_TRAFFIC_BYTES = {"c1": 1122560, "c2": 872922624, "c3": 1641893432, "c4": 545672704, "c5": 477679872}
 
 
 def load_peaks():
@@ -345,7 +345,7 @@ def run_ours(args):
                 continue
             c2 = DeviceCase(torch, bg, k2, w2, 0, device)
             torch.cuda.synchronize()
-            time.sleep(0.5)  # let clocks and the power governor recover from the previous configuration's load
+            time.sleep(1.5)  # let clocks and the power governor recover from the previous configuration's load
             s2 = max_over(c2.time_steps(steps, warmup))
             measured.append({"config": k2, "workload": w2.name, "ms_per_step": round(s2 * 1e3, 5),
                              "tflops": round(metric_value(w2, s2), 2), "gbs": round(w2.min_bytes / s2 / 1e9, 1),

@@ -170,7 +170,7 @@ double estimate_dense_cycles(const gemm_desc_t& d, int sm_count, int variant, in
   const long long waves = (tiles + units - 1) / units;
   const double kblocks = static_cast<double>(ceil_div(d.K, kBlockK));
   // tensor pipe: one 128 x bn x 16 MMA per CTA takes bn / 2 cycles; four per k-block and 128-row half
-  static const double eff1[3] = {0.45, 0.68, 0.88}, eff2[3] = {0.55, 0.80, 0.938};  // bn = 64, 128, 256 (measured, 8192^3)
+  static const double eff1[3] = {0.45, 0.68, 0.82}, eff2[3] = {0.55, 0.80, 0.938};  // bn = 64, 128, 256 (measured: 8192^3, and K = 512 ... 4096)
   const int bi = bn <= 64 ? 0 : (bn <= 128 ? 1 : 2);
   const double eff = wide ? 1.0 : (cg == 1 ? eff1[bi] : eff2[bi]);
   const double mma = kblocks * 4.0 * (bn / 2.0) * (rows_cta / 128.0) / eff;
@@ -179,12 +179,14 @@ double estimate_dense_cycles(const gemm_desc_t& d, int sm_count, int variant, in
   // output: this SM's share of the HBM write bandwidth is ~16 B/clk
   const double out = static_cast<double>(rows_cta) * bn * elem_bytes(d.c_dtype) / 16.0;
   const bool gelu = d.epilogue >= GEMM_EPI_GELU_ERF;  // any transcendental activation
-  double exposed = 400.0;                       // barrier round trips per tile that nothing hides
+  double exposed = 900.0;                       // barrier round trips per tile that nothing hides (fitted at K = 512, 1024)
   // no second accumulator: read-out (and bias fetch, conversion) of half 0; fitted, like the pair efficiency above, to
   // measured pair-vs-wide time ratios at K = 4096 ... 16384 on 8192 x 8192 and 16384 x 14336 outputs
   if (wide) exposed = (gelu ? 13000.0 : 5100.0) + (has_bias(d.epilogue) ? 1300.0 : 0.0);
   else if (cg == 2) exposed = 1000.0;           // pair hand-shakes cross the SM-to-SM network
-  const double per_tile = std::max(mma, std::max(feed, out)) + exposed;
+  // what is exposed stalls the tensor pipe, so it adds to the compute side; an output-bound tile instead pays a small
+  // switch-over per tile (measured on the batched short-K shape: fewer, larger tiles win)
+  const double per_tile = std::max(std::max(mma, feed) + exposed, out + 300.0);
   return static_cast<double>(waves) * per_tile + 3000.0;  // + pipeline fill and drain
 }
 
@@ -219,18 +221,18 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   const int units = pl->sm_count / cg;
   const long long tiles_total = static_cast<long long>(tiles_m) * ceil_div(d.N, bn) * d.batch_count;
   const bool single_wave = tiles_total <= units;  // every CTA (pair) computes at most one tile: pure latency
+  // A tile's main loop lasts about 512 cycles per 64 columns of K (at tile N = 256); draining 128 x 256 accumulators
+  // with four warps takes several thousand.  Short-K (output-bound) problems with several tiles per CTA get a second
+  // epilogue warpgroup (measured: a gain only up to K = 512 at tile N = 256; 7-14 % slower beyond).
+  const int epi_wg = (!single_wave && static_cast<long long>(ceil_div(d.K, kBlockK)) * 2 * bn <= 4096) ? 2 : 1;
   int atoms = forced_atoms;
   if (atoms == 0) {
-    const bool fits3 = 3 * 2 * (a_atom + b_atom) + dense_smem_bytes(0, 0, 0, 1) <= kMaxSmemOptin;
-    atoms = (d.K > 2 * kBlockK && fits3 && !single_wave) ? 2 : 1;  // one-tile problems want every K slice in flight at once
+    const bool fits3 = 3 * 2 * (a_atom + b_atom) + dense_smem_bytes(0, 0, 0, epi_wg) <= kMaxSmemOptin;
+    atoms = (d.K > 2 * kBlockK && fits3) ? 2 : 1;  // (measured by gemm_tune: also faster for one-tile-per-CTA problems)
   }
   if (atoms < 1 || atoms > 2) return GEMM_ERR_UNSUPPORTED;
   const int a_stage = atoms * a_atom;
   const int b_stage = atoms * b_atom;
-  // A tile's main loop lasts about 512 cycles per 64 columns of K (at tile N = 256); draining 128 x 256 accumulators
-  // with four warps takes several thousand.  Short-K (output-bound) problems with several tiles per CTA get a second
-  // epilogue warpgroup.
-  const int epi_wg = (!single_wave && static_cast<long long>(ceil_div(d.K, kBlockK)) * 2 * bn <= 4096) ? 2 : 1;
   int stages = forced_stages;
   if (stages == 0) {
     stages = (kMaxSmemOptin - dense_smem_bytes(0, a_stage, b_stage, epi_wg)) / (a_stage + b_stage);

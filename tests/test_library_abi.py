@@ -109,7 +109,8 @@ def test_roofline_classification_of_the_five_configs():
     assert i2["flops"] == 2.0 * 8192 ** 3 and i2["min_bytes"] == 3 * 8192 * 8192 * 2
     assert i2["variant"] == bg.VARIANT_DENSE_2CTA_WIDE and (i2["tile_m"], i2["tile_n"], i2["stages"]) == (512, 256, 3)
     assert i3["variant"] == bg.VARIANT_DENSE_2CTA          # erf-GELU epilogue: keep the double-buffered accumulator
-    assert i4["variant"] == bg.VARIANT_DENSE_1CTA and i1["variant"] == bg.VARIANT_DENSE_1CTA
+    assert i4["variant"] == bg.VARIANT_DENSE_2CTA_WIDE   # output-bound: the largest tiles, fewest tile switches (measured)
+    assert i1["variant"] == bg.VARIANT_DENSE_1CTA
     for k, i in zip(("c1", "c2", "c3", "c4", "c5"), (i1, i2, i3, i4, i5)):
         assert i["flops"] == c[k].flops
 
@@ -175,7 +176,8 @@ def test_cost_model_choices_follow_the_measurements():
     assert choice(28672, 16, 8192, transb=bg.OP_N)[0] != bg.VARIANT_SKINNY_STREAMK   # needs both operands K-contiguous
     assert choice(64, 28672, 8192)[0] == bg.VARIANT_DENSE_1CTA               # stream-K stops paying near M = 48
     v, bn = choice(2048, 2048, 128, batch=64)
-    assert (v, bn) == (bg.VARIANT_DENSE_1CTA, 256)                           # output-bound: widest tile, fewest hand-shakes
+    assert (v, bn) == (bg.VARIANT_DENSE_2CTA_WIDE, 256)                      # output-bound: largest tile, fewest tile switches
+    assert choice(8192, 8192, 1024)[0] == bg.VARIANT_DENSE_2CTA              # the pair beats the single CTA at every K measured
 
 
 def test_tuning_entry_points_on_the_host():
