@@ -32,6 +32,7 @@ namespace b200 {
 constexpr int kSkinnyTileN = 128;   // output columns (rows of W) per tile = TMEM lanes
 constexpr int kSkinnyMaxM = 64;     // largest M the skinny path takes
 constexpr int kSkinnyThreads = 192;
+constexpr int kSkinnyParkBytes = 80 * 128 * 4;  // 80 prefetched floats for each of the 128 epilogue threads
 
 struct SkinnyPlan {
   int m_pad;             // small extent rounded up to a multiple of 16 (the MMA's N extent)
@@ -71,7 +72,7 @@ inline bool skinny_make_plan(SkinnyPlan* s, int M, int N, int K, int sm_count, i
   s->units_q = static_cast<int>(s->total_units / s->grid);
   s->units_r = static_cast<int>(s->total_units % s->grid);
   s->stage_bytes = s->atoms * (kSkinnyTileN * 128 + s->m_pad * 128);
-  const int fixed = 1024 + 16 * kMaxStages + 64;
+  const int fixed = 1024 + 16 * kMaxStages + 64 + kSkinnyParkBytes;
   int stages = forced_stages ? forced_stages : (max_smem - fixed) / s->stage_bytes;
   if (stages > kMaxStages) stages = kMaxStages;
   if (!forced_stages && stages * s->atoms > 8) stages = 8 / s->atoms > 3 ? 8 / s->atoms : 3;  // measured on B200: ~144 KB in flight per SM streams fastest
@@ -312,20 +313,23 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
       // While the main loop of this segment runs, these warps have nothing to do.  The usual case for the CTA that
       // computes the head of a split tile is that all other contributors finished long ago; if the count says so,
       // their partials (and C_in) are fetched now, this CTA never publishes its own partial and the tail of the kernel
-      // is one tensor-memory read, a few adds and the stores.  The 64 prefetch registers hold either one chunk of 16
-      // from up to four contributors (short extent <= 16) or up to four chunks from the one other contributor; other
-      // shapes take the general path below.  Both paths add the same values in the same order, so the result does
-      // not depend on which one ran.
+      // is one tensor-memory read, a few adds and the stores.  The fetched values are parked in shared memory: the
+      // store cannot issue before its load has landed, which pins the loads to this side of the wait (left in
+      // registers, the loads were scheduled after the wait, next to their use, and the tail paid their latency).
+      // Room for 64 floats per thread: one chunk of 16 from up to four contributors (short extent <= 16) or up to
+      // four chunks from the one other contributor; other shapes take the general path below.  Both paths add the
+      // same values in the same order, so the result does not depend on which one ran.
       bool early = false;
-      float pre[4][16], cin0[16];
-      const bool by_chunk = sp.m_pad > 16;  // pre[b] = chunk b of the other contributor (else: chunk 0 of contributor b)
+      const bool by_chunk = sp.m_pad > 16;  // parked value 16 b + j = chunk b of the other contributor (else: chunk 0 of contributor b)
+      const uint32_t park = base + bars_off + 16u * kMaxStages + 64u + (threadIdx.x - 64u) * 4u;  // value v lives at park + 512 v
       if (!whole && (by_chunk ? c_last - c_first == 1 : c_last - c_first <= 3)) {
         if (leader) s_early[seg == 0 ? 0 : 1] = (stale_status == 0u && ld_acquire_gpu(p.counters + tile) == static_cast<uint32_t>(c_last - c_first)) ? 1u : 0u;
         named_barrier_sync(1, 128);
         early = s_early[seg == 0 ? 0 : 1] != 0u;
         if (early) {
-#pragma unroll
           const int other = c_first == static_cast<int>(blockIdx.x) ? c_last : c_first;
+          float pre[4][16], cin0[16];
+#pragma unroll
           for (int b = 0; b < 4; ++b) {
             // (by contributor: this CTA's own slot is read too and not used; by chunk: chunks past m_pad repeat the last)
             const float* part = by_chunk ? partial_of(other) + min(b * 16, sp.m_pad - 16) * kSkinnyTileN
@@ -333,7 +337,16 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
 #pragma unroll
             for (int j = 0; j < 16; ++j) pre[b][j] = __ldcg(part + j * kSkinnyTileN + n_local);
           }
+#pragma unroll
+          for (int j = 0; j < 16; ++j) cin0[j] = 0.0f;
           if (n < big_extent) sk_load_cin16<kTall>(p, 0, n, cin0);
+#pragma unroll
+          for (int b = 0; b < 4; ++b) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) st_shared_b32(park + 512u * (16 * b + j), __float_as_uint(pre[b][j]));
+          }
+#pragma unroll
+          for (int j = 0; j < 16; ++j) st_shared_b32(park + 512u * (64 + j), __float_as_uint(cin0[j]));
         }
       }
       if (!mbar_wait_warp(tfull0 + 8u * buf, (seg >> 1) & 1u, w, (3u << 8) | buf, 64u)) break;
@@ -357,7 +370,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
 #pragma unroll
           for (int j = 0; j < 16; ++j) sum[j] = 0.0f;
 #pragma unroll
-          for (int j = 0; j < 16; ++j) cin[j] = cin0[j];
+          for (int j = 0; j < 16; ++j) cin[j] = __uint_as_float(ld_shared_b32(park + 512u * (64 + j)));
           if (c0 != 0 && n < big_extent) sk_load_cin16<kTall>(p, c0, n, cin);
 #pragma unroll
           for (int b = 0; b < 4; ++b) {
@@ -367,8 +380,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
               const bool own = cc == static_cast<int>(blockIdx.x);
 #pragma unroll
               for (int j = 0; j < 16; ++j) {
-                float other_v = pre[b][j];
-                if (by_chunk) other_v = c0 == 0 ? pre[0][j] : (c0 == 16 ? pre[1][j] : (c0 == 32 ? pre[2][j] : pre[3][j]));
+                const float other_v = __uint_as_float(ld_shared_b32(park + 512u * ((by_chunk ? c0 : 16 * b) + j)));
                 sum[j] += own ? __uint_as_float(acc[j]) : other_v;
               }
             }
