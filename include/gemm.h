@@ -86,14 +86,20 @@ typedef enum {
 #define GEMM_FLAG_VARIANT_MASK 0xF0u
 #define GEMM_FLAG_TILE_N_SHIFT 8           /* bits 8-15: force tile N / 16 (0 = automatic) */
 #define GEMM_FLAG_TILE_N_MASK 0xFF00u
-#define GEMM_FLAG_RASTER_SHIFT 16          /* bits 16-23: force the raster group height in tiles (0 = automatic) */
-#define GEMM_FLAG_RASTER_MASK 0xFF0000u
+#define GEMM_FLAG_RASTER_SHIFT 16          /* bits 16-22: force the raster group height in tiles (0 = automatic) */
+#define GEMM_FLAG_RASTER_MASK 0x7F0000u
 #define GEMM_FLAG_STAGES_SHIFT 24          /* bits 24-27: force the pipeline depth (0 = automatic) */
 #define GEMM_FLAG_STAGES_MASK 0xF000000u
 #define GEMM_FLAG_KSLICES_SHIFT 28         /* bits 28-29: force 64-wide K slices per pipeline stage, 1 or 2 (0 = automatic) */
 #define GEMM_FLAG_KSLICES_MASK 0x30000000u
 #define GEMM_FLAG_NO_K_SERPENTINE 0x8u      /* walk K forwards in every tile (default: alternate tiles walk it backwards,
                                               which re-uses the operand lines L2 touched last) */
+/* Structure of op(A) (M x K), a promise by the caller, not a mask: with A_LOWER every element with k > i IS zero in
+ * memory, with A_UPPER every element with k < i.  The result is that of the plain GEMM; the library skips the K
+ * ranges that can only contribute zeros (about half the work for a square A).  Dense variants only; at most one
+ * of the two.  (The paper lists symmetric and triangular operands among its operator cases, Section 5.1.) */
+#define GEMM_FLAG_A_LOWER 0x2u
+#define GEMM_FLAG_A_UPPER 0x800000u
 #define GEMM_FLAG_BIAS_PER_ROW 0x1u         /* the bias is fp32[M], one value per output row (default: fp32[N], one per
                                               column); not a tuning knob: it changes what is computed */
 #define GEMM_FLAG_NO_EARLY_LAUNCH 0x4u       /* launch without programmatic dependent launch (default: the kernel may be

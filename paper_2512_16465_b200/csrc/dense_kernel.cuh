@@ -51,6 +51,7 @@ struct DenseParams {
   int out_dtype;                          // 0 bf16, 1 f16, 2 f32
   int epilogue;                           // gemm_epilogue_t
   int bias_per_row;                       // the bias has M entries (one per output row) instead of N
+  int a_tri;                              // structure of op(A): 0 dense, 1 lower triangular (zero for k > i), 2 upper (zero for k < i)
   float alpha, beta;
   const float* bias;
   const void* c_in;                       // = D buffer; read when beta != 0
@@ -144,6 +145,21 @@ __device__ __forceinline__ TileCoord decode_tile(int t, int tiles_m, int tiles_n
   c.tn = within / gm;
   c.tm = first_m + (within - c.tn * gm);
   return c;
+}
+
+// The ring stages [lo, hi) of K that a tile with output rows [row0, row0 + rows) has to visit.  A triangular op(A)
+// (zero beyond the diagonal by the caller's word) makes every stage that lies wholly in the zero part a no-op, so
+// it is skipped; the stages that the diagonal crosses are computed in full.  At least one stage is always kept
+// so that the accumulator gets written.
+struct KRange {
+  int lo, hi;
+};
+__device__ __forceinline__ KRange k_range(const DenseParams& p, int row0, int rows) {
+  KRange r{0, p.num_kb};
+  const int kstep = kBlockK * p.atoms;
+  if (p.a_tri == 1) r.hi = min(p.num_kb, (min(row0 + rows, p.M) - 1) / kstep + 1);
+  else if (p.a_tri == 2) r.lo = min(row0 / kstep, p.num_kb - 1);
+  return r;
 }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -326,9 +342,10 @@ __device__ __forceinline__ void producer_role(const DenseParams& p, const CUtens
     // Serpentine K: all CTAs advance through K roughly in step, so the K range a wave touched last is what L2
     // still holds when the next wave starts; walking it backwards re-uses those lines of the shared A band.
     const bool rev = p.k_serpentine && (it & 1u);
-    int k0 = rev ? (p.num_kb - 1) * kstep : 0;
+    const KRange kr = k_range(p, tc.tm * (kCtaM * CG), kCtaM * CG);
+    int k0 = rev ? (kr.hi - 1) * kstep : kr.lo * kstep;
     const int dk = rev ? -kstep : kstep;
-    for (int kb = 0; kb < p.num_kb; ++kb, k0 += dk) {
+    for (int kb = kr.lo; kb < kr.hi; ++kb, k0 += dk) {
       if (!mbar_wait_warp(empty0 + 8u * s, ph ^ 1u, w, (1u << 8) | s)) return;
       if (stall_pending) {  // test hook: this stage is never filled nor signalled
         stall_pending = false;
@@ -392,11 +409,14 @@ __device__ __forceinline__ void mma_role(const DenseParams& p, uint32_t tiles_ba
     tc_fence_after();
     const uint32_t d_tmem = tmem_base + buf * static_cast<uint32_t>(p.bn);
     const bool rev = p.k_serpentine && (it & 1u);
-    for (int kb = 0; kb < num_kb; ++kb) {
+    KRange kr{0, num_kb};
+    if (p.a_tri != 0) kr = k_range(p, decode_tile(tile, p.tiles_m, p.tiles_n, p.raster_group).tm * (kCtaM * CG), kCtaM * CG);
+    const int n_kb = kr.hi - kr.lo;
+    for (int kb = 0; kb < n_kb; ++kb) {
       if (!mbar_wait_warp(full0 + 8u * s, ph, w, (2u << 8) | s)) return;
       tc_fence_after();
       const uint32_t empty_bar = empty0 + 8u * s;
-      const bool ragged_stage = rev ? (kb == 0) : (kb + 1 == num_kb);  // the stage that holds the end of K
+      const bool ragged_stage = (rev ? kr.hi - 1 - kb : kr.lo + kb) == num_kb - 1;  // the stage that holds the end of K
       const bool two = (p.atoms == 2) && (!ragged_stage || last_atoms == 2);
       if (elect_one()) {
         umma_f16<CG>(d_tmem, adesc, bdesc, idesc, static_cast<uint32_t>(kb != 0));

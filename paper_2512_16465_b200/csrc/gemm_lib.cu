@@ -127,6 +127,7 @@ gemm_status_t validate(const gemm_desc_t* d) {
   if (d->ab_dtype < GEMM_BF16 || d->ab_dtype > GEMM_F32 || d->c_dtype < GEMM_BF16 || d->c_dtype > GEMM_F32)
     return GEMM_ERR_INVALID_ARG;
   if (d->epilogue < GEMM_EPI_NONE || d->epilogue > GEMM_EPI_BIAS_SILU) return GEMM_ERR_INVALID_ARG;
+  if ((d->flags & GEMM_FLAG_A_LOWER) && (d->flags & GEMM_FLAG_A_UPPER)) return GEMM_ERR_INVALID_ARG;
   if (d->ab_dtype == GEMM_F32) return GEMM_ERR_UNSUPPORTED;
   const int64_t a_row = d->transa == GEMM_OP_N ? d->K : d->M;
   const int64_t b_row = d->transb == GEMM_OP_N ? d->N : d->K;
@@ -288,6 +289,7 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   p.out_dtype = d.c_dtype;
   p.epilogue = d.epilogue;
   p.bias_per_row = (d.flags & GEMM_FLAG_BIAS_PER_ROW) ? 1 : 0;
+  p.a_tri = (d.flags & GEMM_FLAG_A_LOWER) ? 1 : ((d.flags & GEMM_FLAG_A_UPPER) ? 2 : 0);
   p.ldc = d.ldc;
   p.stride_c = d.batch_count > 1 ? d.stride_c : 0;
   p.debug_flags = 0u;  // set per run
@@ -326,8 +328,8 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
 // Wide pair variant: 512 x 256 cluster tiles, one 64-wide K slice per stage, 3-deep ring, 8 epilogue warps.
 gemm_status_t plan_wide(gemm_plan_s* pl, int forced_raster, int forced_stages) {
   const gemm_desc_t& d = pl->d;
-  // its epilogue covers the bias per column, ReLU and erf GELU only
-  if (d.epilogue > GEMM_EPI_BIAS_GELU_ERF || (d.flags & GEMM_FLAG_BIAS_PER_ROW)) return GEMM_ERR_UNSUPPORTED;
+  // its epilogue covers the bias per column, ReLU and erf GELU only; its MMA schedule has no K-range skipping
+  if (d.epilogue > GEMM_EPI_BIAS_GELU_ERF || (d.flags & (GEMM_FLAG_BIAS_PER_ROW | GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER))) return GEMM_ERR_UNSUPPORTED;
   const int a_kmajor = d.transa == GEMM_OP_N;
   const int b_kmajor = d.transb == GEMM_OP_T;
   const int tile_m = 2 * kWideCtaM, bn = kWideTileN;
@@ -375,6 +377,7 @@ gemm_status_t plan_wide(gemm_plan_s* pl, int forced_raster, int forced_stages) {
   p.out_dtype = d.c_dtype;
   p.epilogue = d.epilogue;
   p.bias_per_row = (d.flags & GEMM_FLAG_BIAS_PER_ROW) ? 1 : 0;
+  p.a_tri = (d.flags & GEMM_FLAG_A_LOWER) ? 1 : ((d.flags & GEMM_FLAG_A_UPPER) ? 2 : 0);
   p.ldc = d.ldc;
   p.stride_c = d.batch_count > 1 ? d.stride_c : 0;
   p.debug_flags = 0u;  // set per run
@@ -408,6 +411,7 @@ gemm_status_t plan_skinny(gemm_plan_s* pl, int forced_stages, int forced_atoms) 
   const gemm_desc_t& d = pl->d;
   if (d.transa != GEMM_OP_N || d.transb != GEMM_OP_T) return GEMM_ERR_UNSUPPORTED;  // both operands K-contiguous
   if ((d.M > kSkinnyMaxM && d.N > kSkinnyMaxM) || d.batch_count != 1) return GEMM_ERR_UNSUPPORTED;
+  if (d.flags & (GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER)) return GEMM_ERR_UNSUPPORTED;  // no K-range skipping in stream-K
   SkinnyPlan& s = pl->skinny;
   pl->skinny_tall = d.M > kSkinnyMaxM;  // the short extent is N: A is streamed, B is the resident slab
   const int small_extent = static_cast<int>(pl->skinny_tall ? d.N : d.M), big_extent = static_cast<int>(pl->skinny_tall ? d.M : d.N);
@@ -494,7 +498,8 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
   if (variant == 0) {
     // memory-bound problems with a handful of rows stream the weight matrix once: stream-K path;
     // everything else is a dense tiled GEMM, paired CTAs when there are at least two tile rows
-    const bool skinny_ok = (d.M <= kSkinnyMaxM || d.N <= kSkinnyMaxM) && d.batch_count == 1 && d.transa == GEMM_OP_N && d.transb == GEMM_OP_T;
+    const bool skinny_ok = (d.M <= kSkinnyMaxM || d.N <= kSkinnyMaxM) && d.batch_count == 1 && d.transa == GEMM_OP_N &&
+                           d.transb == GEMM_OP_T && !(d.flags & (GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER));
     if (skinny_ok && info.intensity < 5.2 * kRidgeCudaCore) {
       variant = GEMM_VARIANT_SKINNY_STREAMK;  // measured: wins up to M ~ 48
     } else {
@@ -504,7 +509,9 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
       for (int v : {GEMM_VARIANT_DENSE_1CTA, GEMM_VARIANT_DENSE_2CTA, GEMM_VARIANT_DENSE_2CTA_WIDE}) {
         for (int bn : {256, 128, 64}) {
           if (v == GEMM_VARIANT_DENSE_2CTA_WIDE && bn != kWideTileN) continue;
-          if (v == GEMM_VARIANT_DENSE_2CTA_WIDE && (d.epilogue > GEMM_EPI_BIAS_GELU_ERF || (d.flags & GEMM_FLAG_BIAS_PER_ROW))) continue;
+          if (v == GEMM_VARIANT_DENSE_2CTA_WIDE &&
+              (d.epilogue > GEMM_EPI_BIAS_GELU_ERF || (d.flags & (GEMM_FLAG_BIAS_PER_ROW | GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER))))
+            continue;
           if (v == GEMM_VARIANT_DENSE_2CTA && !b_kmajor && bn % 128) continue;  // 64-column boxes per CTA
           if (v != GEMM_VARIANT_DENSE_1CTA && d.M <= kCtaM) continue;           // a pair needs two tile rows
           if (forced_bn && bn != forced_bn) continue;

@@ -97,6 +97,18 @@ EXACT_CASES = [
     ("skinny_k_slice_past_the_end", 8, 256, 1080, {}, dict(variant=VS)),
     ("no_early_launch_1cta", 264, 328, 200, {}, dict(variant=V1, tile_n=128, no_early_launch=True)),
     ("no_early_launch_skinny", 8, 256, 4096, dict(beta=1.0), dict(variant=VS, no_early_launch=True)),
+    # triangular op(A): K ranges that can only contribute zeros are skipped
+    ("tri_lower_1cta", 512, 264, 512, dict(a_tri=1), dict(variant=V1, tile_n=128)),
+    ("tri_upper_1cta", 512, 264, 512, dict(a_tri=2), dict(variant=V1, tile_n=128)),
+    ("tri_lower_pair_ragged", 600, 328, 520, dict(a_tri=1), dict(variant=V2, tile_n=128)),
+    ("tri_upper_pair_k_longer", 300, 264, 1000, dict(a_tri=2), dict(variant=V2, tile_n=128)),
+    ("tri_lower_m_longer", 1000, 136, 200, dict(a_tri=1), dict(variant=V1)),
+    ("tri_upper_m_longer", 1000, 136, 200, dict(a_tri=2), dict(variant=V1)),
+    ("tri_lower_a_stored_transposed", 512, 264, 512, dict(a_tri=1, ta=1), dict(variant=V1, tile_n=128)),
+    ("tri_upper_one_slice_stages", 512, 264, 512, dict(a_tri=2), dict(variant=V2, tile_n=128, kslices=1)),
+    ("tri_lower_no_serpentine", 512, 264, 512, dict(a_tri=1), dict(variant=V1, tile_n=64, no_k_serpentine=True)),
+    ("tri_lower_batched_beta", 256, 136, 256, dict(a_tri=1, batch=3, beta=1.0, cd=wl.BF16), dict(variant=V1)),
+    ("tri_lower_auto", 2048, 512, 2048, dict(a_tri=1, cd=wl.BF16), dict()),
     # mirrored stream-K: a tall output with a handful of columns (A is the streamed operand)
     ("tall_one_unit", 128, 8, 64, {}, dict(variant=VS)),
     ("tall_split_k", 256, 8, 4096, {}, dict(variant=VS)),
@@ -339,6 +351,26 @@ def test_bounded_wait_reports_timeout_and_context_survives(variant):
         assert all(r["bit_identical"] == 1.0 for r in reports)
     plan.close()
     H.check_workload(w, bg.make_flags(variant, tile_n), exact=True)
+
+
+def test_triangular_a_really_skips():
+    """Lower-triangular A, 512 x 512: every kernel variant works on tile rows of at most 256 and ring stages of at most
+    128 columns, so element (i, k) with k >= 256 (i // 256 + 1) lies in a stage no tile may visit.  NaN there must
+    not reach the output; the diagonal stages are computed in full, so the zeros next to the diagonal are real zeros."""
+    w = int_workload("tri_skip", 512, 264, 512, a_tri=1)
+    inputs = wl.make_inputs(w)
+    a = inputs["A"].reshape(512, 512)
+    for i in range(512):
+        a[i, 256 * (i // 256 + 1):] = 0x7FC0          # bf16 NaN
+    for fl in (dict(variant=V1, tile_n=128), dict(variant=V2, tile_n=128), dict()):
+        cbits, info = H.run_gpu(w, inputs, bg.make_flags(**fl))
+        clean = wl.make_inputs(w)
+        reports = H.check_blocks(w, clean, cbits, H.default_blocks(w))
+        assert all(r["bit_identical"] == 1.0 and r["finite"] for r in reports), info
+    for bad in (dict(variant=VS), dict(variant=VW)):     # these kernels have no K-range skipping: refused, not ignored
+        with pytest.raises(bg.GemmError) as e:
+            bg.gemm_plan(H.desc_of(int_workload("tri_refused", 8 if bad["variant"] == VS else 1024, 1024, 4096, a_tri=1), bg.make_flags(**bad)))
+        assert e.value.status == bg.ERR_UNSUPPORTED
 
 
 # ----------------------------------------------------------------------------- measured plan selection

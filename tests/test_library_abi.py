@@ -56,6 +56,9 @@ def test_plan_validation_codes():
     assert plan_status(**ok, ldc=255) == bg.ERR_INVALID_ARG
     assert plan_status(**ok, transa=2) == bg.ERR_INVALID_ARG
     assert plan_status(**ok, epilogue=10) == bg.ERR_INVALID_ARG
+    assert plan_status(**ok, flags=bg.make_flags(a_lower=True, a_upper=True)) == bg.ERR_INVALID_ARG
+    assert plan_status(**ok, flags=bg.make_flags(a_lower=True)) == bg.OK
+    assert plan_status(M=8, N=4096, K=4096, flags=bg.make_flags(a_upper=True)) == bg.OK      # planned dense, not stream-K
     assert plan_status(**ok, epilogue=bg.EPI_BIAS_SILU) == bg.OK
     assert plan_status(**ok, c_dtype=3) == bg.ERR_INVALID_ARG
     assert plan_status(**ok, ab_dtype=bg.F32) == bg.ERR_UNSUPPORTED

@@ -74,3 +74,20 @@ def test_sample_indices():
     assert not np.array_equal(s, wl.sample_indices(8192, 256, 5, 2))
     assert np.array_equal(wl.sample_indices(40, 0, 1, 1), np.arange(40))
     assert np.array_equal(wl.sample_indices(40, 64, 1, 1), np.arange(40))
+
+
+def test_triangular_structure_of_a():
+    for ta in (0, 1):
+        for tri, keep in ((1, np.tril), (2, np.triu)):
+            w = wl.Workload("t", 7, 5, 9, transa=ta, a_tri=tri, batch=2, lda=12)
+            dense = wl.make_inputs(wl.Workload("t", 7, 5, 9, transa=ta, batch=2, lda=12))["A"]
+            got = wl.make_inputs(w)["A"]
+            rows, cols = (9, 7) if ta else (7, 9)
+            for b in range(2):
+                g = got[b * w.stride_a: b * w.stride_a + rows * 12].reshape(rows, 12)[:, :cols]
+                d = dense[b * w.stride_a: b * w.stride_a + rows * 12].reshape(rows, 12)[:, :cols]
+                op_g, op_d = (g.T, d.T) if ta else (g, d)          # op(A) is M x K = 7 x 9
+                assert np.array_equal(op_g, keep(op_d))
+    # useful work: non-zeros of op(A) times N, two flops each
+    assert wl.Workload("t", 4, 3, 4, a_tri=1).flops == 2.0 * 10 * 3
+    assert wl.Workload("t", 4, 3, 6, a_tri=2).flops == 2.0 * (6 + 5 + 4 + 3) * 3

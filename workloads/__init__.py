@@ -110,6 +110,7 @@ class Workload:
     batch: int = 1
     epilogue: int = EPI_NONE
     bias_per_row: bool = False   # the bias has M entries (one per output row) instead of N
+    a_tri: int = 0               # structure of op(A): 0 dense, 1 lower triangular (zero for k > i), 2 upper (zero for k < i)
     alpha: float = 1.0
     beta: float = 0.0
     dist_a: Dist = field(default_factory=lambda: Dist("normal", 0.0, 1.0))
@@ -149,7 +150,14 @@ class Workload:
 
     @property
     def flops(self) -> float:
-        return 2.0 * self.M * self.N * self.K * self.batch
+        """Useful work: two flops per (non-zero element of op(A)) x (output column)."""
+        if self.a_tri == 1:
+            nz = sum(min(i + 1, self.K) for i in range(self.M))
+        elif self.a_tri == 2:
+            nz = sum(max(self.K - i, 0) for i in range(self.M))
+        else:
+            nz = self.M * self.K
+        return 2.0 * nz * self.N * self.batch
 
     @property
     def min_bytes(self) -> float:
@@ -183,6 +191,20 @@ def _draw(dist: Dist, seed, tensor_id, n, dtype):
     raise ValueError(dist.kind)
 
 
+def _zero_triangle(a: np.ndarray, w: Workload) -> None:
+    """Store zeros in the part of op(A) that a triangular workload declares empty (input structure, no arithmetic)."""
+    for b in range(w.batch):
+        off = b * w.stride_a
+        if not w.transa:          # stored M x K: row i holds op(A)[i, :]
+            for i in range(w.M):
+                lo, hi = (min(i + 1, w.K), w.K) if w.a_tri == 1 else (0, min(i, w.K))
+                a[off + i * w.lda + lo: off + i * w.lda + hi] = 0
+        else:                     # stored K x M: row k holds op(A)[:, k]
+            for k in range(w.K):
+                lo, hi = (0, min(k, w.M)) if w.a_tri == 1 else (min(k + 1, w.M), w.M)
+                a[off + k * w.lda + lo: off + k * w.lda + hi] = 0
+
+
 def make_inputs(w: Workload, seed_offset: int = 0) -> dict:
     """Draw A, B and, when used, C_in and bias for ``w``.  ``seed_offset`` gives the
     benchmark its rotating "different random inputs" sets."""
@@ -190,6 +212,8 @@ def make_inputs(w: Workload, seed_offset: int = 0) -> dict:
     out = {"A": _draw(w.dist_a, s, TENSOR_A, w.elems_a(), w.ab_dtype),
            "B": _draw(w.dist_b, s, TENSOR_B, w.elems_b(), w.ab_dtype),
            "C": None, "bias": None}
+    if w.a_tri:
+        _zero_triangle(out["A"], w)
     if w.beta != 0.0:
         out["C"] = _draw(w.dist_c, s, TENSOR_C, w.elems_c(), w.c_dtype)
     if w.has_bias:
