@@ -40,7 +40,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the full-size ncu captures
 # summarised under profiles/ (dense_*_cN_*.txt, skinny_streamk_c5_*.txt; last line of each file).
-NCU_TRAFFIC_BYTES = {"c1": 1122560, "c2": 872922624, "c3": 1641893432, "c4": 545672704, "c5": 477679872}
+NCU_TRAFFIC_BYTES = {"c1": 1123584, "c2": 873626624, "c3": 1637930408, "c4": 545520896, "c5": 478118656}
 
 
 def load_peaks():
