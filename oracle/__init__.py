@@ -5,7 +5,7 @@ The oracle is the fp64 triple-loop definition of
 Section 5.4 case study).  Nothing in the product package imports this module:
 only the tests, the smoke check and the benchmark's CPU-baseline legs do.
 
-Arrays are numpy: ``uint16`` bit patterns for bf16 / fp16, ``float32`` for fp32.
+Arrays are numpy: ``uint16`` bit patterns for bf16 / fp16, ``uint8`` for the 8-bit floats, ``float32`` for fp32.
 """
 from __future__ import annotations
 
@@ -20,7 +20,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "gemm_oracle.c")
 _LIB = os.path.join(_HERE, "libgemm_oracle.so")
 
-BF16, F16, F32 = 0, 1, 2
+BF16, F16, F32, FP8_E4M3, FP8_E5M2 = 0, 1, 2, 3, 4
 (EPI_NONE, EPI_BIAS, EPI_RELU, EPI_BIAS_RELU, EPI_GELU_ERF, EPI_BIAS_GELU_ERF, EPI_GELU_TANH, EPI_BIAS_GELU_TANH,
  EPI_SILU, EPI_BIAS_SILU) = range(10)
 
@@ -59,6 +59,9 @@ def lib() -> ctypes.CDLL:
         L.oracle_f64_to_bf16.argtypes = [ctypes.c_double]
         L.oracle_f64_to_f16.restype = ctypes.c_uint16
         L.oracle_f64_to_f16.argtypes = [ctypes.c_double]
+        for name in ("oracle_e4m3_to_f64", "oracle_e5m2_to_f64"):
+            getattr(L, name).restype = ctypes.c_double
+            getattr(L, name).argtypes = [ctypes.c_uint8]
         L.oracle_gelu_erf.restype = ctypes.c_double
         L.oracle_gelu_erf.argtypes = [ctypes.c_double]
         L.oracle_gelu_erf_alt.restype = ctypes.c_double
@@ -143,7 +146,8 @@ def gemm(p: Problem, A, B, C_in=None, bias=None, alpha=1.0, beta=0.0,
     assert cols.size == 0 or (cols.min() >= 0 and cols.max() < p.N)
     for arr in (A, B, C_in, bias):
         assert arr is None or arr.flags["C_CONTIGUOUS"]
-    assert A.dtype == np.uint16 and B.dtype == np.uint16
+    ab_np = np.uint8 if p.ab_dtype in (FP8_E4M3, FP8_E5M2) else np.uint16
+    assert A.dtype == ab_np and B.dtype == ab_np
     if C_in is not None:
         assert C_in.dtype == (np.float32 if p.c_dtype == F32 else np.uint16)
     if bias is not None:

@@ -16,7 +16,7 @@
  * evaluated in IEEE double, k ascending, one output at a time, no blocking,
  * no reassociation (build without -ffast-math).  Inputs arrive as the very bit
  * patterns the GPU receives (uint16 for bf16 / fp16, float for fp32) and are
- * decoded exactly; a product of two 8- or 11-bit significands is exact in
+ * decoded exactly; a product of two significands of at most 11 bits is exact in
  * double, so the only rounding is the fp64 summation (relative error about
  * K * 2^-53 of sum |a||b|).
  *
@@ -40,7 +40,7 @@
 #include <stdint.h>
 #include <string.h>
 
-enum { OR_BF16 = 0, OR_F16 = 1, OR_F32 = 2 };
+enum { OR_BF16 = 0, OR_F16 = 1, OR_F32 = 2, OR_FP8_E4M3 = 3, OR_FP8_E5M2 = 4 };
 /* even values: no bias; odd values: the same activation with a bias added first */
 enum { OR_EPI_NONE = 0, OR_EPI_BIAS = 1, OR_EPI_RELU = 2, OR_EPI_BIAS_RELU = 3,
        OR_EPI_GELU_ERF = 4, OR_EPI_BIAS_GELU_ERF = 5, OR_EPI_GELU_TANH = 6, OR_EPI_BIAS_GELU_TANH = 7,
@@ -49,7 +49,7 @@ enum { OR_EPI_NONE = 0, OR_EPI_BIAS = 1, OR_EPI_RELU = 2, OR_EPI_BIAS_RELU = 3,
 typedef struct {
   int64_t M, N, K;
   int32_t transa, transb;
-  int32_t ab_dtype;      /* OR_BF16 or OR_F16 */
+  int32_t ab_dtype;      /* OR_BF16, OR_F16 (uint16 patterns) or OR_FP8_E4M3, OR_FP8_E5M2 (uint8 patterns) */
   int32_t c_dtype;       /* dtype of C_in (read only when beta != 0) */
   int64_t lda, ldb, ldc;
   int64_t stride_a, stride_b, stride_c;
@@ -78,6 +78,27 @@ double oracle_f16_to_f64(uint16_t h) {
   } else {
     v = ldexp((double)(m | 0x400), e - 25);    /* (1.m) * 2^(e-15) */
   }
+  return sign ? -v : v;
+}
+
+/* 8-bit floats (the OCP FP8 formats the fifth-generation tensor cores take).
+ * E4M3: 1 sign, 4 exponent (bias 7), 3 mantissa bits; no infinities: exponent field 15 is an ordinary binade
+ * (largest finite value 1.75 * 2^8 = 448) except that mantissa 7 there is NaN.
+ * E5M2: 1 sign, 5 exponent (bias 15), 2 mantissa bits; IEEE-like, exponent field 31 is infinity / NaN. */
+double oracle_e4m3_to_f64(uint8_t h) {
+  int sign = (h >> 7) & 1, e = (h >> 3) & 0xF, m = h & 0x7;
+  double v;
+  if (e == 15 && m == 7) v = NAN;
+  else if (e == 0) v = ldexp((double)m, -9);            /* subnormal: m/8 * 2^-6 */
+  else v = ldexp((double)(m | 0x8), e - 10);           /* (1.m) * 2^(e-7) */
+  return sign ? -v : v;
+}
+double oracle_e5m2_to_f64(uint8_t h) {
+  int sign = (h >> 7) & 1, e = (h >> 2) & 0x1F, m = h & 0x3;
+  double v;
+  if (e == 31) v = m ? NAN : INFINITY;
+  else if (e == 0) v = ldexp((double)m, -16);           /* subnormal: m/4 * 2^-14 */
+  else v = ldexp((double)(m | 0x4), e - 17);           /* (1.m) * 2^(e-15) */
   return sign ? -v : v;
 }
 
@@ -144,6 +165,8 @@ double oracle_gelu_tanh(double t) {
 int oracle_max_threads(void);
 
 static double load_ab(const void* p, int dtype, int64_t idx) {
+  if (dtype == OR_FP8_E4M3) return oracle_e4m3_to_f64(((const uint8_t*)p)[idx]);
+  if (dtype == OR_FP8_E5M2) return oracle_e5m2_to_f64(((const uint8_t*)p)[idx]);
   const uint16_t* h = (const uint16_t*)p;
   return dtype == OR_BF16 ? oracle_bf16_to_f64(h[idx]) : oracle_f16_to_f64(h[idx]);
 }

@@ -252,6 +252,29 @@ def test_gelu_textbook_values_and_identities(golden_dir):
     assert g(12.0) == 12.0 and abs(g(-12.0)) < 1e-30
 
 
+def test_fp8_decoders_exhaustively():
+    """All 256 patterns of both 8-bit formats against the library's conversion, plus the values the format
+    definitions fix (1.0, largest finite, smallest subnormal, the NaN / infinity encodings)."""
+    import torch
+    L = oracle.lib()
+    codes = torch.arange(256, dtype=torch.int32).to(torch.uint8)
+    for fn, tdt in ((L.oracle_e4m3_to_f64, torch.float8_e4m3fn), (L.oracle_e5m2_to_f64, torch.float8_e5m2)):
+        want = codes.view(tdt).to(torch.float64).numpy()
+        got = np.array([fn(int(c)) for c in range(256)])
+        assert np.array_equal(np.isnan(got), np.isnan(want))
+        assert np.array_equal(got[~np.isnan(got)], want[~np.isnan(want)])
+        assert np.array_equal(np.signbit(got), np.signbit(want))
+    e4, e5 = L.oracle_e4m3_to_f64, L.oracle_e5m2_to_f64
+    assert e4(0x38) == 1.0 and e4(0x7E) == 448.0 and e4(0x01) == 2.0 ** -9 and e4(0xC0) == -2.0 and math.isnan(e4(0x7F))
+    assert e4(0x78) == 256.0                                    # exponent field 15 is an ordinary binade: no infinity
+    assert e5(0x3C) == 1.0 and e5(0x7B) == 57344.0 and e5(0x01) == 2.0 ** -16 and e5(0x7C) == math.inf and math.isnan(e5(0x7E))
+    # in the GEMM: 2 x 2 by hand, e4m3 operands {1, 2; -0.5, 448} . {3; 0.25}
+    a = np.array([0x38, 0x40, 0xB0, 0x7E], np.uint8)             # [[1, 2], [-0.5, 448]]
+    b = np.array([0x44, 0x28], np.uint8)                         # stored N x K: [[3, 0.25]]
+    y, bound = oracle.gemm(Problem(2, 1, 2, transb=1, ab_dtype=oracle.FP8_E4M3), a, b)
+    assert y[0, :, 0].tolist() == [3.5, 110.5] and bound[0, :, 0].tolist() == [3.5, 113.5]
+
+
 def test_logistic_silu_and_tanh_gelu(golden_dir):
     L = oracle.lib()
     sg, silu, gt, ge = L.oracle_logistic, L.oracle_silu, L.oracle_gelu_tanh, L.oracle_gelu_erf
