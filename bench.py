@@ -106,15 +106,18 @@ class ClockSampler:
 def roofline_for(w: wl.Workload, key: str, seconds: float, peaks: dict, peak_kind: str) -> dict:
     """Roofline entry of the step's single kernel: the bound is whichever of (flops / tensor peak)
     and (compulsory bytes / HBM bandwidth) is slower."""
-    t_tensor = w.flops / (peaks["bf16_tflops"] * 1e12)
+    fp8 = w.ab_dtype in (wl.FP8_E4M3, wl.FP8_E5M2)
+    # a contraction takes the peak of its own operand type: the measured bf16 figure times the nominal fp8 : bf16 ratio
+    tensor_peak = peaks["bf16_tflops"] * (2.0 if fp8 else 1.0)
+    t_tensor = w.flops / (tensor_peak * 1e12)
     t_hbm = w.min_bytes / (peaks["hbm_gbs"] * 1e9)
     if t_tensor >= t_hbm:
-        achieved, peak, unit, bound = w.flops / seconds / 1e12, peaks["bf16_tflops"], "TFLOP/s", "tensor"
+        achieved, peak, unit, bound = w.flops / seconds / 1e12, tensor_peak, "TFLOP/s", "tensor"
     else:
         achieved, peak, unit, bound = w.min_bytes / seconds / 1e9, peaks["hbm_gbs"], "GB/s", "hbm"
     return {"bound": bound, "achieved": round(achieved, 2), "peak": peak, "unit": unit, "frac": round(achieved / peak, 4),
-            "traffic": NCU_TRAFFIC_BYTES.get(key), "peak_source": f"of {peak_kind}",
-            "frac_of_nominal": round(achieved / (NOMINAL["tensor_tflops"] if bound == "tensor" else NOMINAL["hbm_gbs"]), 4),
+            "traffic": NCU_TRAFFIC_BYTES.get(key), "peak_source": f"of {peak_kind}" + (" bf16 x 2 (nominal fp8 ratio)" if fp8 and bound == "tensor" else ""),
+            "frac_of_nominal": round(achieved / (NOMINAL["tensor_tflops"] * (2.0 if fp8 else 1.0) if bound == "tensor" else NOMINAL["hbm_gbs"]), 4),
             "algorithmic_flops": w.flops, "algorithmic_bytes": w.min_bytes}
 
 
@@ -125,7 +128,10 @@ def _torch_dt(torch, code):
 
 
 def _to_torch(torch, arr, code, device=None, pin=False):
-    t = torch.from_numpy(arr) if code == wl.F32 else torch.from_numpy(arr.view(np.int16)).view(_torch_dt(torch, code))
+    if code == wl.F32 or arr.dtype == np.uint8:   # fp32 values, or the bytes of 8-bit floats
+        t = torch.from_numpy(arr)
+    else:
+        t = torch.from_numpy(arr.view(np.int16)).view(_torch_dt(torch, code))
     if pin:
         t = t.pin_memory()
     return t.to(device) if device is not None else t
@@ -385,12 +391,12 @@ def run_ours(args):
 
 
 def parse_shape(spec: str) -> wl.Workload:
-    """'MxNxK' followed by optional ':key=value' fields: batch, ta, tb (1 = stored transposed), ab/cd (bf16|f16|f32),
+    """'MxNxK' followed by optional ':key=value' fields: batch, ta, tb (1 = stored transposed), ab (bf16|f16|e4m3|e5m2), cd (bf16|f16|f32),
     epi (none|bias|relu|bias_relu|gelu|bias_gelu|gelu_tanh|bias_gelu_tanh|silu|bias_silu), rowbias (0|1), tri (lower|upper: op(A) triangular), alpha, beta,
     lda, ldb, ldc.  Example: 28672x8x8192:beta=1:cd=f32."""
     head, *fields = spec.split(":")
     M, N, K = (int(x) for x in head.lower().split("x"))
-    dt = {"bf16": wl.BF16, "f16": wl.F16, "f32": wl.F32}
+    dt = {"bf16": wl.BF16, "f16": wl.F16, "f32": wl.F32, "e4m3": wl.FP8_E4M3, "e5m2": wl.FP8_E5M2}
     epi = {"none": wl.EPI_NONE, "bias": wl.EPI_BIAS, "relu": wl.EPI_RELU, "bias_relu": wl.EPI_BIAS_RELU,
            "gelu": wl.EPI_GELU_ERF, "bias_gelu": wl.EPI_BIAS_GELU_ERF, "gelu_tanh": wl.EPI_GELU_TANH,
            "bias_gelu_tanh": wl.EPI_BIAS_GELU_TANH, "silu": wl.EPI_SILU, "bias_silu": wl.EPI_BIAS_SILU}
@@ -444,7 +450,8 @@ def run_shapes(args):
                    "gbs": round(w.min_bytes / sec / 1e9, 1), "input_sets": case.nsets,
                    "plan": {k: case.plan.info[k] for k in ("variant", "tile_m", "tile_n", "stages", "cluster_size", "grid", "split")},
                    "roofline": roofline_for(w, spec, sec, peaks, peak_kind)}
-            if args.library_reference and w.batch == 1 and w.epilogue == wl.EPI_NONE and w.beta == 0.0 and w.alpha == 1.0:
+            if args.library_reference and w.batch == 1 and w.epilogue == wl.EPI_NONE and w.beta == 0.0 and w.alpha == 1.0 and \
+                    w.ab_dtype in (wl.BF16, wl.F16):
                 # context only: the vendor library on the same operands (no part of the product)
                 A, B, _, _ = case.sets[0]
                 a2 = A[: (w.K if w.transa else w.M) * w.lda].view(-1, w.lda)

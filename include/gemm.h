@@ -56,7 +56,13 @@ typedef enum {
   GEMM_ERR_TIMEOUT = 8      /* a bounded device-side wait expired (see gemm_plan_status) */
 } gemm_status_t;
 
-typedef enum { GEMM_BF16 = 0, GEMM_F16 = 1, GEMM_F32 = 2 } gemm_dtype_t;
+typedef enum {
+  GEMM_BF16 = 0,
+  GEMM_F16 = 1,
+  GEMM_F32 = 2,
+  GEMM_FP8_E4M3 = 3, /* 8-bit float, 4 exponent / 3 mantissa bits, no infinities (largest finite 448); operands only */
+  GEMM_FP8_E5M2 = 4  /* 8-bit float, 5 exponent / 2 mantissa bits, IEEE-like; operands only */
+} gemm_dtype_t;
 typedef enum { GEMM_OP_N = 0, GEMM_OP_T = 1 } gemm_op_t;
 typedef enum {
   GEMM_EPI_NONE = 0,
@@ -115,7 +121,8 @@ typedef struct {
   uint32_t flags;        /* GEMM_FLAG_* */
   int64_t M, N, K;       /* op(A) is M x K, op(B) is K x N, C/D is M x N; all >= 1 */
   int32_t transa, transb;     /* gemm_op_t */
-  int32_t ab_dtype;           /* gemm_dtype_t: GEMM_BF16 or GEMM_F16, for both A and B */
+  int32_t ab_dtype;           /* gemm_dtype_t: GEMM_BF16, GEMM_F16, or an 8-bit float (then transa = N, transb = T and the
+                                 dense variants only), for both A and B */
   int32_t c_dtype;            /* gemm_dtype_t of C/D */
   int64_t lda, ldb, ldc;      /* leading dimensions in elements */
   int32_t batch_count;        /* >= 1 */

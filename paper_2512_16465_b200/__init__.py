@@ -17,7 +17,7 @@ from typing import Optional
 
 from . import build as _build
 
-BF16, F16, F32 = 0, 1, 2
+BF16, F16, F32, FP8_E4M3, FP8_E5M2 = 0, 1, 2, 3, 4
 OP_N, OP_T = 0, 1
 (EPI_NONE, EPI_BIAS, EPI_RELU, EPI_BIAS_RELU, EPI_GELU_ERF, EPI_BIAS_GELU_ERF, EPI_GELU_TANH, EPI_BIAS_GELU_TANH,
  EPI_SILU, EPI_BIAS_SILU) = range(10)
@@ -225,7 +225,16 @@ def status_string(st: int) -> str:
 
 def _torch_dtype_code(t) -> int:
     import torch
-    return {torch.bfloat16: BF16, torch.float16: F16, torch.float32: F32}[t]
+    return {torch.bfloat16: BF16, torch.float16: F16, torch.float32: F32, torch.float8_e4m3fn: FP8_E4M3,
+            torch.float8_e5m2: FP8_E5M2}[t]
+
+
+def _operand_matches(t, code: int) -> bool:
+    """8-bit float operands may also be handed over as plain bytes (``torch.uint8``)."""
+    import torch
+    if t == torch.uint8:
+        return code in (FP8_E4M3, FP8_E5M2)
+    return _torch_dtype_code(t) == code
 
 
 class Plan:
@@ -259,7 +268,7 @@ class Plan:
         import torch
         if not (A.is_cuda and B.is_cuda and C.is_cuda):
             raise ValueError("A, B and C must be CUDA tensors")
-        if _torch_dtype_code(A.dtype) != self.desc.ab_dtype or _torch_dtype_code(B.dtype) != self.desc.ab_dtype or \
+        if not _operand_matches(A.dtype, self.desc.ab_dtype) or not _operand_matches(B.dtype, self.desc.ab_dtype) or \
                 _torch_dtype_code(C.dtype) != self.desc.c_dtype:
             raise ValueError("tensor dtypes do not match the plan")
         ws = workspace if workspace is not None else self.workspace(A.device)

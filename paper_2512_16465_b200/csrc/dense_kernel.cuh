@@ -51,6 +51,8 @@ struct DenseParams {
   int out_dtype;                          // 0 bf16, 1 f16, 2 f32
   int epilogue;                           // gemm_epilogue_t
   int bias_per_row;                       // the bias has M entries (one per output row) instead of N
+  int ab_fp8;                             // operands are 8-bit floats (tcgen05 kind::f8f6f4), else 16-bit (kind::f16)
+  int kblk;                               // elements of K in one 128-byte slice: 64 (16-bit operands) or 128 (8-bit)
   int a_tri;                              // structure of op(A): 0 dense, 1 lower triangular (zero for k > i), 2 upper (zero for k < i)
   float alpha, beta;
   const float* bias;
@@ -156,7 +158,7 @@ struct KRange {
 };
 __device__ __forceinline__ KRange k_range(const DenseParams& p, int row0, int rows) {
   KRange r{0, p.num_kb};
-  const int kstep = kBlockK * p.atoms;
+  const int kstep = p.kblk * p.atoms;
   if (p.a_tri == 1) r.hi = min(p.num_kb, (min(row0 + rows, p.M) - 1) / kstep + 1);
   else if (p.a_tri == 2) r.lo = min(row0 / kstep, p.num_kb - 1);
   return r;
@@ -333,7 +335,7 @@ __device__ __forceinline__ void producer_role(const DenseParams& p, const CUtens
   bool stall_pending = (p.debug_flags & 1u) != 0u;
   const uint64_t pol_a = p.l2_hint_a == 2 ? l2_policy_evict_last() : (p.l2_hint_a == 1 ? l2_policy_evict_first() : l2_policy_evict_normal());
   const uint64_t pol_b = p.l2_hint_b == 2 ? l2_policy_evict_last() : (p.l2_hint_b == 1 ? l2_policy_evict_first() : l2_policy_evict_normal());
-  const int kstep = kBlockK * p.atoms;
+  const int kstep = p.kblk * p.atoms;
   uint32_t it = 0;
   for (int tile = cluster_id; tile < p.num_tiles; tile += num_clusters, ++it) {
     const TileCoord tc = decode_tile(tile, p.tiles_m, p.tiles_n, p.raster_group);
@@ -361,7 +363,7 @@ __device__ __forceinline__ void producer_role(const DenseParams& p, const CUtens
             else tma_load_3d_pair(dst, map, bar, x, y, tc.batch, pol);
           };
           for (int a = 0; a < p.atoms; ++a) {  // slices past K are zero-filled by the copy engine
-            const int ka = k0 + a * kBlockK;
+            const int ka = k0 + a * p.kblk;
             const uint32_t saa = sa + a * p.a_atom_bytes, sba = sb + a * p.b_atom_bytes;
             if (p.a_kmajor) {
               load(saa, tmA, ka, m0, pol_a);
@@ -399,7 +401,7 @@ __device__ __forceinline__ void mma_role(const DenseParams& p, uint32_t tiles_ba
   const int num_kb = p.num_kb;
   const uint32_t aatom16 = p.a_atom_bytes >> 4, batom16 = p.b_atom_bytes >> 4;
   // atoms of the last stage that still hold part of K (the rest is zero fill and is skipped)
-  const int last_atoms = (p.K - (num_kb - 1) * kBlockK * p.atoms + kBlockK - 1) / kBlockK;
+  const int last_atoms = (p.K - (num_kb - 1) * p.kblk * p.atoms + p.kblk - 1) / p.kblk;
   uint32_t s = 0, ph = 0, it = 0;
   uint64_t adesc = adesc0, bdesc = bdesc0;
   for (int tile = cluster_id; tile < p.num_tiles; tile += num_clusters, ++it) {
@@ -419,13 +421,23 @@ __device__ __forceinline__ void mma_role(const DenseParams& p, uint32_t tiles_ba
       const bool ragged_stage = (rev ? kr.hi - 1 - kb : kr.lo + kb) == num_kb - 1;  // the stage that holds the end of K
       const bool two = (p.atoms == 2) && (!ragged_stage || last_atoms == 2);
       if (elect_one()) {
-        umma_f16<CG>(d_tmem, adesc, bdesc, idesc, static_cast<uint32_t>(kb != 0));
+        if (!p.ab_fp8) {
+          umma_f16<CG>(d_tmem, adesc, bdesc, idesc, static_cast<uint32_t>(kb != 0));
 #pragma unroll
-        for (uint32_t k = 1; k < kBlockK / kUmmaK; ++k) umma_f16<CG>(d_tmem, adesc + k * ak16, bdesc + k * bk16, idesc, 1u);
-        if (two) {
+          for (uint32_t k = 1; k < kBlockK / kUmmaK; ++k) umma_f16<CG>(d_tmem, adesc + k * ak16, bdesc + k * bk16, idesc, 1u);
+          if (two) {
 #pragma unroll
-          for (uint32_t k = 0; k < kBlockK / kUmmaK; ++k)
-            umma_f16<CG>(d_tmem, adesc + aatom16 + k * ak16, bdesc + batom16 + k * bk16, idesc, 1u);
+            for (uint32_t k = 0; k < kBlockK / kUmmaK; ++k)
+              umma_f16<CG>(d_tmem, adesc + aatom16 + k * ak16, bdesc + batom16 + k * bk16, idesc, 1u);
+          }
+        } else {  // four 32-byte steps per 128-byte slice, as above
+          umma_f8<CG>(d_tmem, adesc, bdesc, idesc, static_cast<uint32_t>(kb != 0));
+#pragma unroll
+          for (uint32_t k = 1; k < 4; ++k) umma_f8<CG>(d_tmem, adesc + k * ak16, bdesc + k * bk16, idesc, 1u);
+          if (two) {
+#pragma unroll
+            for (uint32_t k = 0; k < 4; ++k) umma_f8<CG>(d_tmem, adesc + aatom16 + k * ak16, bdesc + batom16 + k * bk16, idesc, 1u);
+          }
         }
         // ring slot reusable once these MMAs have read it (both CTAs of a pair are told at once)
         if constexpr (CG == 1) umma_commit<1>(empty_bar);

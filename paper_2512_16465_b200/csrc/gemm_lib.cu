@@ -54,9 +54,15 @@ EncodeFn get_encode_fn() {
   return fn;
 }
 
-int elem_bytes(int dtype) { return dtype == GEMM_F32 ? 4 : 2; }
+bool is_fp8(int dtype) { return dtype == GEMM_FP8_E4M3 || dtype == GEMM_FP8_E5M2; }
+int elem_bytes(int dtype) { return dtype == GEMM_F32 ? 4 : (is_fp8(dtype) ? 1 : 2); }
+// elements of K in one 128-byte swizzle row of an operand
+int kblk_of(int ab_dtype) { return is_fp8(ab_dtype) ? 2 * kBlockK : kBlockK; }
+// format code of the instruction descriptor: kind::f16 0 = f16, 1 = bf16; kind::f8f6f4 0 = E4M3, 1 = E5M2
+int ab_format(int ab_dtype) { return (ab_dtype == GEMM_BF16 || ab_dtype == GEMM_FP8_E5M2) ? 1 : 0; }
 
 CUtensorMapDataType tm_dtype(int dtype) {
+  if (is_fp8(dtype)) return CU_TENSOR_MAP_DATA_TYPE_UINT8;  // the copy engine only moves the bytes
   return dtype == GEMM_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16
                             : (dtype == GEMM_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32);
 }
@@ -124,11 +130,13 @@ gemm_status_t validate(const gemm_desc_t* d) {
   if (d->M > 0x7FFFFFFFll || d->N > 0x7FFFFFFFll || d->K > 0x7FFFFFFFll) return GEMM_ERR_INVALID_ARG;
   if ((d->transa != GEMM_OP_N && d->transa != GEMM_OP_T) || (d->transb != GEMM_OP_N && d->transb != GEMM_OP_T))
     return GEMM_ERR_INVALID_ARG;
-  if (d->ab_dtype < GEMM_BF16 || d->ab_dtype > GEMM_F32 || d->c_dtype < GEMM_BF16 || d->c_dtype > GEMM_F32)
+  if (d->ab_dtype < GEMM_BF16 || d->ab_dtype > GEMM_FP8_E5M2 || d->c_dtype < GEMM_BF16 || d->c_dtype > GEMM_F32)
     return GEMM_ERR_INVALID_ARG;
   if (d->epilogue < GEMM_EPI_NONE || d->epilogue > GEMM_EPI_BIAS_SILU) return GEMM_ERR_INVALID_ARG;
   if ((d->flags & GEMM_FLAG_A_LOWER) && (d->flags & GEMM_FLAG_A_UPPER)) return GEMM_ERR_INVALID_ARG;
   if (d->ab_dtype == GEMM_F32) return GEMM_ERR_UNSUPPORTED;
+  // 8-bit operands: K-contiguous storage only (A stored M x K, B stored N x K)
+  if (is_fp8(d->ab_dtype) && (d->transa != GEMM_OP_N || d->transb != GEMM_OP_T)) return GEMM_ERR_UNSUPPORTED;
   const int64_t a_row = d->transa == GEMM_OP_N ? d->K : d->M;
   const int64_t b_row = d->transb == GEMM_OP_N ? d->N : d->K;
   if (d->lda < a_row || d->ldb < b_row || d->ldc < d->N) return GEMM_ERR_INVALID_ARG;
@@ -141,7 +149,7 @@ gemm_status_t validate(const gemm_desc_t* d) {
     (void)a_rows;
     (void)b_rows;
   }
-  const int eab = 2, ec = elem_bytes(d->c_dtype);
+  const int eab = elem_bytes(d->ab_dtype), ec = elem_bytes(d->c_dtype);
   if ((d->lda * eab) % 16 || (d->ldb * eab) % 16 || (d->ldc * ec) % 16) return GEMM_ERR_ALIGNMENT;
   if (d->batch_count > 1 && ((d->stride_a * eab) % 16 || (d->stride_b * eab) % 16 || (d->stride_c * ec) % 16))
     return GEMM_ERR_ALIGNMENT;
@@ -169,7 +177,7 @@ double estimate_dense_cycles(const gemm_desc_t& d, int sm_count, int variant, in
   const int units = std::max(1, sm_count / cg);
   const long long tiles = static_cast<long long>(ceil_div(d.M, rows_tile)) * ceil_div(d.N, bn) * d.batch_count;
   const long long waves = (tiles + units - 1) / units;
-  const double kblocks = static_cast<double>(ceil_div(d.K, kBlockK));
+  const double kblocks = static_cast<double>(ceil_div(d.K, kblk_of(d.ab_dtype)));  // 128-byte slices: same pipe time for either width
   // tensor pipe: one 128 x bn x 16 MMA per CTA takes bn / 2 cycles; four per k-block and 128-row half
   static const double eff1[3] = {0.45, 0.68, 0.82}, eff2[3] = {0.55, 0.80, 0.938};  // bn = 64, 128, 256 (measured: 8192^3, and K = 512 ... 4096)
   const int bi = bn <= 64 ? 0 : (bn <= 128 ? 1 : 2);
@@ -225,11 +233,12 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   // A tile's main loop lasts about 512 cycles per 64 columns of K (at tile N = 256); draining 128 x 256 accumulators
   // with four warps takes several thousand.  Short-K (output-bound) problems with several tiles per CTA get a second
   // epilogue warpgroup (measured: a gain only up to K = 512 at tile N = 256; 7-14 % slower beyond).
-  const int epi_wg = (!single_wave && static_cast<long long>(ceil_div(d.K, kBlockK)) * 2 * bn <= 4096) ? 2 : 1;
+  const int kblk = kblk_of(d.ab_dtype);
+  const int epi_wg = (!single_wave && static_cast<long long>(ceil_div(d.K, kblk)) * 2 * bn <= 4096) ? 2 : 1;
   int atoms = forced_atoms;
   if (atoms == 0) {
     const bool fits3 = 3 * 2 * (a_atom + b_atom) + dense_smem_bytes(0, 0, 0, epi_wg) <= kMaxSmemOptin;
-    atoms = (d.K > 2 * kBlockK && fits3) ? 2 : 1;  // (measured by gemm_tune: also faster for one-tile-per-CTA problems)
+    atoms = (d.K > 2 * kblk && fits3) ? 2 : 1;  // (measured by gemm_tune: also faster for one-tile-per-CTA problems)
   }
   if (atoms < 1 || atoms > 2) return GEMM_ERR_UNSUPPORTED;
   const int a_stage = atoms * a_atom;
@@ -266,14 +275,16 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   p.raster_group = raster;
   p.bn = bn;
   p.stages = stages;
-  p.num_kb = ceil_div(d.K, kBlockK * atoms);
+  p.num_kb = ceil_div(d.K, kblk * atoms);
   p.atoms = atoms;
+  p.kblk = kblk;
+  p.ab_fp8 = is_fp8(d.ab_dtype) ? 1 : 0;
   p.a_atom_bytes = a_atom;
   p.b_atom_bytes = b_atom;
   uint32_t cols = 32;
   while (cols < 2u * bn) cols <<= 1;
   p.tmem_cols = cols;
-  p.idesc = make_idesc(d.ab_dtype == GEMM_BF16, !a_kmajor, !b_kmajor, tile_m, bn);
+  p.idesc = make_idesc(ab_format(d.ab_dtype), !a_kmajor, !b_kmajor, tile_m, bn);
   p.a_stage_bytes = a_stage;
   p.b_stage_bytes = b_stage;
   p.a_kmajor = a_kmajor;
@@ -313,7 +324,7 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   info.variant = pl->variant;
   info.tile_m = tile_m;
   info.tile_n = bn;
-  info.tile_k = kBlockK * atoms;
+  info.tile_k = kblk * atoms;
   info.stages = stages;
   info.cluster_size = cg;
   info.grid = pl->grid;
@@ -328,6 +339,7 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
 // Wide pair variant: 512 x 256 cluster tiles, one 64-wide K slice per stage, 3-deep ring, 8 epilogue warps.
 gemm_status_t plan_wide(gemm_plan_s* pl, int forced_raster, int forced_stages) {
   const gemm_desc_t& d = pl->d;
+  if (is_fp8(d.ab_dtype)) return GEMM_ERR_UNSUPPORTED;  // 16-bit operands only
   // its epilogue covers the bias per column, ReLU and erf GELU only; its MMA schedule has no K-range skipping
   if (d.epilogue > GEMM_EPI_BIAS_GELU_ERF || (d.flags & (GEMM_FLAG_BIAS_PER_ROW | GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER))) return GEMM_ERR_UNSUPPORTED;
   const int a_kmajor = d.transa == GEMM_OP_N;
@@ -360,6 +372,8 @@ gemm_status_t plan_wide(gemm_plan_s* pl, int forced_raster, int forced_stages) {
   p.bn = bn;
   p.stages = stages;
   p.num_kb = ceil_div(d.K, kBlockK);
+  p.kblk = kBlockK;
+  p.ab_fp8 = 0;
   p.atoms = 1;
   p.tmem_cols = 512;
   p.idesc = make_idesc(d.ab_dtype == GEMM_BF16, !a_kmajor, !b_kmajor, 256, bn);
@@ -412,6 +426,7 @@ gemm_status_t plan_skinny(gemm_plan_s* pl, int forced_stages, int forced_atoms) 
   if (d.transa != GEMM_OP_N || d.transb != GEMM_OP_T) return GEMM_ERR_UNSUPPORTED;  // both operands K-contiguous
   if ((d.M > kSkinnyMaxM && d.N > kSkinnyMaxM) || d.batch_count != 1) return GEMM_ERR_UNSUPPORTED;
   if (d.flags & (GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER)) return GEMM_ERR_UNSUPPORTED;  // no K-range skipping in stream-K
+  if (is_fp8(d.ab_dtype)) return GEMM_ERR_UNSUPPORTED;  // 16-bit operands only
   SkinnyPlan& s = pl->skinny;
   pl->skinny_tall = d.M > kSkinnyMaxM;  // the short extent is N: A is streamed, B is the resident slab
   const int small_extent = static_cast<int>(pl->skinny_tall ? d.N : d.M), big_extent = static_cast<int>(pl->skinny_tall ? d.M : d.N);
@@ -475,7 +490,7 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
 
   // roofline class (Section 4.3): compulsory traffic vs. work
   const gemm_desc_t& d = pl->d;
-  const double eb = 2.0, ec = elem_bytes(d.c_dtype);
+  const double eb = elem_bytes(d.ab_dtype), ec = elem_bytes(d.c_dtype);
   const double flops = 2.0 * d.M * d.N * d.K * d.batch_count;
   double bytes = d.batch_count * (static_cast<double>(d.M) * d.K + static_cast<double>(d.K) * d.N) * eb +
                  d.batch_count * static_cast<double>(d.M) * d.N * ec;
@@ -499,7 +514,7 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
     // memory-bound problems with a handful of rows stream the weight matrix once: stream-K path;
     // everything else is a dense tiled GEMM, paired CTAs when there are at least two tile rows
     const bool skinny_ok = (d.M <= kSkinnyMaxM || d.N <= kSkinnyMaxM) && d.batch_count == 1 && d.transa == GEMM_OP_N &&
-                           d.transb == GEMM_OP_T && !(d.flags & (GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER));
+                           d.transb == GEMM_OP_T && !(d.flags & (GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER)) && !is_fp8(d.ab_dtype);
     if (skinny_ok && info.intensity < 5.2 * kRidgeCudaCore) {
       variant = GEMM_VARIANT_SKINNY_STREAMK;  // measured: wins up to M ~ 48
     } else {
@@ -509,6 +524,7 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
       for (int v : {GEMM_VARIANT_DENSE_1CTA, GEMM_VARIANT_DENSE_2CTA, GEMM_VARIANT_DENSE_2CTA_WIDE}) {
         for (int bn : {256, 128, 64}) {
           if (v == GEMM_VARIANT_DENSE_2CTA_WIDE && bn != kWideTileN) continue;
+          if (v == GEMM_VARIANT_DENSE_2CTA_WIDE && is_fp8(d.ab_dtype)) continue;
           if (v == GEMM_VARIANT_DENSE_2CTA_WIDE &&
               (d.epilogue > GEMM_EPI_BIAS_GELU_ERF || (d.flags & (GEMM_FLAG_BIAS_PER_ROW | GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER))))
             continue;
@@ -693,9 +709,9 @@ gemm_status_t run_dense(gemm_plan_s* pl, const void* A, const void* B, void* C, 
   const uint64_t batch = d.batch_count;
   // A: K-major -> rows are M, inner K, box 64 x 128; M-major (stored K x M) -> rows are K, inner M, box 64 x 64
   const uint32_t a_box_rows = pl->variant == GEMM_VARIANT_DENSE_2CTA_WIDE ? kWideCtaM : kCtaM;
-  bool ok = p.a_kmajor ? encode_map(&tA, d.ab_dtype, A, d.K, d.M, batch, d.lda, d.stride_a, kBlockK, a_box_rows)
+  bool ok = p.a_kmajor ? encode_map(&tA, d.ab_dtype, A, d.K, d.M, batch, d.lda, d.stride_a, p.kblk, a_box_rows)
                        : encode_map(&tA, d.ab_dtype, A, d.M, d.K, batch, d.lda, d.stride_a, 64, kBlockK);
-  ok = ok && (p.b_kmajor ? encode_map(&tB, d.ab_dtype, B, d.K, d.N, batch, d.ldb, d.stride_b, kBlockK, p.b_rows)
+  ok = ok && (p.b_kmajor ? encode_map(&tB, d.ab_dtype, B, d.K, d.N, batch, d.ldb, d.stride_b, p.kblk, p.b_rows)
                          : encode_map(&tB, d.ab_dtype, B, d.N, d.K, batch, d.ldb, d.stride_b, 64, kBlockK));
   const uint32_t slab_cols = d.c_dtype == GEMM_F32 ? 32 : 64;
   ok = ok && encode_map(&tD, d.c_dtype, C, d.N, d.M, batch, d.ldc, d.stride_c, slab_cols, 32);

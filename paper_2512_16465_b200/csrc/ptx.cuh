@@ -190,6 +190,23 @@ __device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t adesc, uint64
         ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// The same with 8-bit float inputs (E4M3 or E5M2, named by the instruction descriptor): 32 elements of K per instruction,
+// which is again 32 bytes of every operand row, so descriptors step exactly as for the 16-bit kinds.
+template <int CG>
+__device__ __forceinline__ void umma_f8(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  if constexpr (CG == 1)
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n}\n"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  else
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n}\n"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
 // arrive on `bar` (shared::cluster address; a shared::cta address names the own CTA) once every
 // tcgen05.mma issued so far by this thread has finished
 template <int CG>
@@ -249,11 +266,12 @@ __host__ __device__ constexpr uint64_t make_smem_desc_hi(uint32_t lbo_bytes, uin
 }
 __device__ __forceinline__ uint64_t smem_desc(uint64_t hi, uint32_t saddr) { return hi | ((saddr >> 4) & 0x3FFF); }
 
-// 32-bit instruction descriptor of tcgen05.mma.kind::f16 with fp32 accumulation:
-//   bits 4-5 D format (1 = f32)   bits 7-9 A format, 10-12 B format (0 = f16, 1 = bf16)
+// 32-bit instruction descriptor of tcgen05.mma with fp32 accumulation:
+//   bits 4-5 D format (1 = f32)   bits 7-9 A format, 10-12 B format (kind::f16: 0 = f16, 1 = bf16;
+//   kind::f8f6f4: 0 = E4M3, 1 = E5M2)
 //   bit 15 / 16: A / B is MN-major   bits 17-22 N >> 3   bits 24-28 M >> 4
-__host__ __device__ constexpr uint32_t make_idesc(int ab_is_bf16, int a_mn_major, int b_mn_major, int umma_m, int umma_n) {
-  return (1u << 4) | (static_cast<uint32_t>(ab_is_bf16) << 7) | (static_cast<uint32_t>(ab_is_bf16) << 10) |
+__host__ __device__ constexpr uint32_t make_idesc(int ab_format, int a_mn_major, int b_mn_major, int umma_m, int umma_n) {
+  return (1u << 4) | (static_cast<uint32_t>(ab_format) << 7) | (static_cast<uint32_t>(ab_format) << 10) |
          (static_cast<uint32_t>(a_mn_major) << 15) | (static_cast<uint32_t>(b_mn_major) << 16) |
          (static_cast<uint32_t>(umma_n >> 3) << 17) | (static_cast<uint32_t>(umma_m >> 4) << 24);
 }

@@ -48,7 +48,7 @@ _TORCH_DT = {wl.BF16: torch.bfloat16, wl.F16: torch.float16, wl.F32: torch.float
 
 
 def to_device(arr: np.ndarray, dtype: int) -> torch.Tensor:
-    if dtype == wl.F32:
+    if dtype == wl.F32 or arr.dtype == np.uint8:      # fp32 values, or the bytes of 8-bit floats
         return torch.from_numpy(arr).cuda()
     return torch.from_numpy(arr.view(np.int16)).cuda().view(_TORCH_DT[dtype])
 

@@ -109,6 +109,17 @@ EXACT_CASES = [
     ("tri_lower_no_serpentine", 512, 264, 512, dict(a_tri=1), dict(variant=V1, tile_n=64, no_k_serpentine=True)),
     ("tri_lower_batched_beta", 256, 136, 256, dict(a_tri=1, batch=3, beta=1.0, cd=wl.BF16), dict(variant=V1)),
     ("tri_lower_auto", 2048, 512, 2048, dict(a_tri=1, cd=wl.BF16), dict()),
+    # 8-bit float operands (tcgen05 kind::f8f6f4): 128 elements of K per 128-byte slice
+    ("fp8_e4m3_one_tile", 128, 128, 128, dict(ab=wl.FP8_E4M3), dict(variant=V1, tile_n=128)),
+    ("fp8_e5m2_ragged", 200, 328, 208, dict(ab=wl.FP8_E5M2), dict(variant=V1, tile_n=128)),
+    ("fp8_e4m3_pair_long_k", 300, 264, 4096 + 64, dict(ab=wl.FP8_E4M3), dict(variant=V2, tile_n=128)),
+    ("fp8_e5m2_pair_256", 512, 512, 1024, dict(ab=wl.FP8_E5M2, cd=wl.BF16), dict(variant=V2, tile_n=256)),
+    ("fp8_e4m3_bias_relu_f16_out", 200, 328, 272, dict(ab=wl.FP8_E4M3, cd=wl.F16, epi=bg.EPI_BIAS_RELU, beta=1.0), dict(variant=V1)),
+    ("fp8_e4m3_batched", 96, 72, 256, dict(ab=wl.FP8_E4M3, batch=3), dict(variant=V1)),
+    ("fp8_e4m3_one_slice_stages", 256, 256, 1040, dict(ab=wl.FP8_E4M3), dict(variant=V1, tile_n=128, kslices=1)),
+    ("fp8_e4m3_tiny_k", 128, 64, 16, dict(ab=wl.FP8_E4M3), dict(variant=V1, tile_n=64)),
+    ("fp8_e4m3_lower_triangular", 512, 264, 512, dict(ab=wl.FP8_E4M3, a_tri=1), dict(variant=V2, tile_n=128)),
+    ("fp8_e4m3_auto", 1024, 1024, 2048, dict(ab=wl.FP8_E4M3, cd=wl.BF16), dict()),
     # mirrored stream-K: a tall output with a handful of columns (A is the streamed operand)
     ("tall_one_unit", 128, 8, 64, {}, dict(variant=VS)),
     ("tall_split_k", 256, 8, 4096, {}, dict(variant=VS)),
@@ -371,6 +382,31 @@ def test_triangular_a_really_skips():
         with pytest.raises(bg.GemmError) as e:
             bg.gemm_plan(H.desc_of(int_workload("tri_refused", 8 if bad["variant"] == VS else 1024, 1024, 4096, a_tri=1), bg.make_flags(**bad)))
         assert e.value.status == bg.ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("ab", [wl.FP8_E4M3, wl.FP8_E5M2])
+def test_fp8_operands_general_values(ab):
+    """Normally distributed 8-bit operands (every product is exact in fp32; the sums are not): the stated per-element
+    tolerance and a small Frobenius error against the fp64 oracle, on both dense families."""
+    for fl in (dict(variant=V1), dict(variant=V2, tile_n=128)):
+        w = wl.Workload("fp8_normal", 300, 264, 1040, transb=1, ab_dtype=ab, c_dtype=wl.F32, epilogue=bg.EPI_BIAS_GELU_TANH,
+                        dist_a=wl.Dist("normal", 0, 1), dist_b=wl.Dist("normal", 0, 0.1), seed=11)
+        reports, _ = H.check_workload(w, bg.make_flags(**fl))
+        assert reports[0]["frob"] < 1e-5 and reports[0]["max_err_over_tol"] < 0.05
+
+
+def test_fp8_refusals():
+    for kw in (dict(transb=bg.OP_N), dict(transa=bg.OP_T)):                       # K-contiguous storage only
+        with pytest.raises(bg.GemmError) as e:
+            bg.gemm_plan(bg.make_desc(256, 256, 256, ab_dtype=bg.FP8_E4M3, **kw))
+        assert e.value.status == bg.ERR_UNSUPPORTED
+    for v in (VS, VW):                                                            # 16-bit kernels: refused, not ignored
+        with pytest.raises(bg.GemmError) as e:
+            bg.gemm_plan(bg.make_desc(8 if v == VS else 1024, 1024, 4096, ab_dtype=bg.FP8_E5M2, flags=bg.make_flags(v)))
+        assert e.value.status == bg.ERR_UNSUPPORTED
+    h = bg.gemm_plan(bg.make_desc(8, 4096, 4096, ab_dtype=bg.FP8_E4M3))             # the automatic plan goes to a dense kernel
+    assert bg.gemm_plan_info(h)["variant"] == V1 and bg.gemm_plan_info(h)["tile_k"] in (128, 256)
+    bg.gemm_destroy(h)
 
 
 # ----------------------------------------------------------------------------- measured plan selection

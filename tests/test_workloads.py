@@ -91,3 +91,16 @@ def test_triangular_structure_of_a():
     # useful work: non-zeros of op(A) times N, two flops each
     assert wl.Workload("t", 4, 3, 4, a_tri=1).flops == 2.0 * 10 * 3
     assert wl.Workload("t", 4, 3, 6, a_tri=2).flops == 2.0 * (6 + 5 + 4 + 3) * 3
+
+
+def test_fp8_encoding_matches_the_library_conversion():
+    import torch
+    rng = np.random.default_rng(0)
+    x = np.concatenate([rng.normal(0, 3, 20000), rng.normal(0, 1e-3, 5000),
+                        [0.0, -0.0, 1.0, 447.9, 500.0, -1e9, 2.0 ** -9, 2.0 ** -10, 3 * 2.0 ** -10, 2.0 ** -17, 1.0625, 1.1875]]).astype(np.float32)
+    for dt, tdt, lim in ((wl.FP8_E4M3, torch.float8_e4m3fn, 448.0), (wl.FP8_E5M2, torch.float8_e5m2, 57344.0)):
+        got = wl.encode(x, dt)
+        want = torch.from_numpy(np.clip(x, -lim, lim)).to(tdt).view(torch.uint8).numpy()    # saturating, ties to even
+        assert got.dtype == np.uint8 and np.array_equal(got, want)
+        ints = wl.integer(1, 1, 4096, -4, 4, dt)
+        assert set(torch.from_numpy(ints).view(tdt).float().tolist()) == set(float(v) for v in range(-4, 5))

@@ -24,10 +24,10 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "gen.c")
 _LIB = os.path.join(_HERE, "libworkloads_gen.so")
 
-BF16, F16, F32 = 0, 1, 2
+BF16, F16, F32, FP8_E4M3, FP8_E5M2 = 0, 1, 2, 3, 4
 (EPI_NONE, EPI_BIAS, EPI_RELU, EPI_BIAS_RELU, EPI_GELU_ERF, EPI_BIAS_GELU_ERF, EPI_GELU_TANH, EPI_BIAS_GELU_TANH,
  EPI_SILU, EPI_BIAS_SILU) = range(10)
-ELEM_BYTES = {BF16: 2, F16: 2, F32: 4}
+ELEM_BYTES = {BF16: 2, F16: 2, F32: 4, FP8_E4M3: 1, FP8_E5M2: 1}
 TENSOR_A, TENSOR_B, TENSOR_C, TENSOR_BIAS = 1, 2, 3, 4
 BASE_SEED = 0x5EED0000
 
@@ -60,7 +60,7 @@ def _gen():
 
 
 def _alloc(n: int, dtype: int) -> np.ndarray:
-    return np.empty(n, np.float32 if dtype == F32 else np.uint16)
+    return np.empty(n, {F32: np.float32, FP8_E4M3: np.uint8, FP8_E5M2: np.uint8}.get(dtype, np.uint16))
 
 
 def uniform(seed, tensor_id, n, lo, hi, dtype) -> np.ndarray:

@@ -17,7 +17,7 @@
 #include <stdint.h>
 #include <string.h>
 
-enum { G_BF16 = 0, G_F16 = 1, G_F32 = 2 };
+enum { G_BF16 = 0, G_F16 = 1, G_F32 = 2, G_FP8_E4M3 = 3, G_FP8_E5M2 = 4 };
 
 static inline uint64_t mix(uint64_t seed, uint64_t tensor_id, uint64_t c) {
   uint64_t z = seed + tensor_id * 0x9E3779B97F4A7C15ull + c;
@@ -44,7 +44,29 @@ static inline uint16_t f32_to_f16_bits(float f) {
   return b;
 }
 
+/* Nearest 8-bit float (ties to even) with `mbits` mantissa bits and exponent bias `bias`; magnitudes beyond the
+ * largest finite value saturate to it, NaN becomes zero: the generators only ever emit finite numbers. */
+static inline uint8_t f64_to_fp8_bits(double v, int mbits, int bias, double max_finite) {
+  uint8_t sign = signbit(v) ? 0x80 : 0;
+  double a = fabs(v);
+  if (!(a == a) || a == 0.0) return sign;
+  if (a > max_finite) a = max_finite;
+  int ex;
+  (void)frexp(a, &ex);
+  int e = ex - 1, emin = 1 - bias;
+  int q = (e < emin ? emin : e) - mbits;            /* exponent of one unit in the last place here */
+  double r = ldexp(nearbyint(ldexp(a, -q)), q);     /* default rounding mode: to nearest, ties to even */
+  if (r == 0.0) return sign;
+  (void)frexp(r, &ex);
+  e = ex - 1;
+  if (e < emin) return (uint8_t)(sign | (unsigned)ldexp(r, mbits - emin));                 /* subnormal */
+  unsigned mant = (unsigned)ldexp(r, mbits - e) - (1u << mbits);
+  return (uint8_t)(sign | ((unsigned)(e + bias) << mbits) | mant);
+}
+
 static inline void store(void* out, int64_t i, int dtype, double v) {
+  if (dtype == G_FP8_E4M3) { ((uint8_t*)out)[i] = f64_to_fp8_bits(v, 3, 7, 448.0); return; }
+  if (dtype == G_FP8_E5M2) { ((uint8_t*)out)[i] = f64_to_fp8_bits(v, 2, 15, 57344.0); return; }
   float f = (float)v;
   if (dtype == G_BF16) ((uint16_t*)out)[i] = f32_to_bf16_bits(f);
   else if (dtype == G_F16) ((uint16_t*)out)[i] = f32_to_f16_bits(f);
