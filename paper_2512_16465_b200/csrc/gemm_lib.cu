@@ -426,12 +426,12 @@ gemm_status_t plan_skinny(gemm_plan_s* pl, int forced_stages, int forced_atoms) 
   if (d.transa != GEMM_OP_N || d.transb != GEMM_OP_T) return GEMM_ERR_UNSUPPORTED;  // both operands K-contiguous
   if ((d.M > kSkinnyMaxM && d.N > kSkinnyMaxM) || d.batch_count != 1) return GEMM_ERR_UNSUPPORTED;
   if (d.flags & (GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER)) return GEMM_ERR_UNSUPPORTED;  // no K-range skipping in stream-K
-  if (is_fp8(d.ab_dtype)) return GEMM_ERR_UNSUPPORTED;  // 16-bit operands only
   SkinnyPlan& s = pl->skinny;
   pl->skinny_tall = d.M > kSkinnyMaxM;  // the short extent is N: A is streamed, B is the resident slab
   const int small_extent = static_cast<int>(pl->skinny_tall ? d.N : d.M), big_extent = static_cast<int>(pl->skinny_tall ? d.M : d.N);
   if (forced_atoms > 3) return GEMM_ERR_UNSUPPORTED;
-  if (!skinny_make_plan(&s, small_extent, big_extent, static_cast<int>(d.K), pl->sm_count, forced_stages, kMaxSmemOptin, forced_atoms))
+  if (!skinny_make_plan(&s, small_extent, big_extent, static_cast<int>(d.K), pl->sm_count, forced_stages, kMaxSmemOptin, forced_atoms,
+                        kblk_of(d.ab_dtype)))
     return GEMM_ERR_UNSUPPORTED;
   pl->variant = GEMM_VARIANT_SKINNY_STREAMK;
   pl->cg = 1;
@@ -443,7 +443,7 @@ gemm_status_t plan_skinny(gemm_plan_s* pl, int forced_stages, int forced_atoms) 
   // 128 rows of the streamed operand per tile; the short extent padded to a multiple of 16
   info.tile_m = kSkinnyTileN;
   info.tile_n = s.m_pad;
-  info.tile_k = kBlockK * s.atoms;
+  info.tile_k = s.kblk * s.atoms;
   info.stages = s.stages;
   info.cluster_size = 1;
   info.grid = s.grid;
@@ -514,7 +514,7 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
     // memory-bound problems with a handful of rows stream the weight matrix once: stream-K path;
     // everything else is a dense tiled GEMM, paired CTAs when there are at least two tile rows
     const bool skinny_ok = (d.M <= kSkinnyMaxM || d.N <= kSkinnyMaxM) && d.batch_count == 1 && d.transa == GEMM_OP_N &&
-                           d.transb == GEMM_OP_T && !(d.flags & (GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER)) && !is_fp8(d.ab_dtype);
+                           d.transb == GEMM_OP_T && !(d.flags & (GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER));
     if (skinny_ok && info.intensity < 5.2 * kRidgeCudaCore) {
       variant = GEMM_VARIANT_SKINNY_STREAMK;  // measured: wins up to M ~ 48
     } else {
@@ -737,11 +737,11 @@ gemm_status_t run_skinny(gemm_plan_s* pl, const void* A, const void* B, void* C,
   // a tall problem streams A in W's place and keeps B as the slab
   bool ok;
   if (pl->skinny_tall) {
-    ok = encode_map(&tW, d.ab_dtype, A, d.K, d.M, 1, d.lda, 0, kBlockK, kSkinnyTileN);
-    ok = ok && encode_map(&tX, d.ab_dtype, B, d.K, d.N, 1, d.ldb, 0, kBlockK, s.m_pad);
+    ok = encode_map(&tW, d.ab_dtype, A, d.K, d.M, 1, d.lda, 0, s.kblk, kSkinnyTileN);
+    ok = ok && encode_map(&tX, d.ab_dtype, B, d.K, d.N, 1, d.ldb, 0, s.kblk, s.m_pad);
   } else {
-    ok = encode_map(&tW, d.ab_dtype, B, d.K, d.N, 1, d.ldb, 0, kBlockK, kSkinnyTileN);
-    ok = ok && encode_map(&tX, d.ab_dtype, A, d.K, d.M, 1, d.lda, 0, kBlockK, s.m_pad);
+    ok = encode_map(&tW, d.ab_dtype, B, d.K, d.N, 1, d.ldb, 0, s.kblk, kSkinnyTileN);
+    ok = ok && encode_map(&tX, d.ab_dtype, A, d.K, d.M, 1, d.lda, 0, s.kblk, s.m_pad);
   }
   if (!ok) return GEMM_ERR_CUDA;
   SkinnyParams p;
@@ -750,7 +750,8 @@ gemm_status_t run_skinny(gemm_plan_s* pl, const void* A, const void* B, void* C,
   p.M = static_cast<int>(d.M);
   p.N = static_cast<int>(d.N);
   p.K = static_cast<int>(d.K);
-  p.idesc = make_idesc(d.ab_dtype == GEMM_BF16, 0, 0, kSkinnyTileN, s.m_pad);
+  p.idesc = make_idesc(ab_format(d.ab_dtype), 0, 0, kSkinnyTileN, s.m_pad);
+  p.ab_fp8 = is_fp8(d.ab_dtype) ? 1 : 0;
   p.out_dtype = d.c_dtype;
   p.epilogue = d.epilogue;
   p.bias_per_row = (d.flags & GEMM_FLAG_BIAS_PER_ROW) ? 1 : 0;
@@ -853,7 +854,7 @@ extern "C" gemm_status_t gemm_skinny_run_noalloc(const gemm_desc_t* desc, const 
   gemm_status_t st = validate(desc);
   if (st != GEMM_OK) return st;
   if (has_bias(desc->epilogue) && !bias) return GEMM_ERR_NULL;
-  if (desc->transa != GEMM_OP_N || desc->transb != GEMM_OP_T || desc->batch_count != 1 || desc->M > kSkinnyMaxM)
+  if (desc->transa != GEMM_OP_N || desc->transb != GEMM_OP_T || desc->batch_count != 1 || desc->M > kSkinnyMaxM || is_fp8(desc->ab_dtype))
     return GEMM_ERR_UNSUPPORTED;
   auto misaligned = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; };
   if (misaligned(A) || misaligned(B) || misaligned(C) || (bias && misaligned(bias))) return GEMM_ERR_ALIGNMENT;

@@ -37,8 +37,9 @@ constexpr int kSkinnyParkBytes = 80 * 128 * 4;  // 80 prefetched floats for each
 struct SkinnyPlan {
   int m_pad;             // small extent rounded up to a multiple of 16 (the MMA's N extent)
   int n_tiles;           // ceil(big extent / 128)
-  int atoms;             // 64-wide K slices per pipeline stage (each slice is one 128-byte swizzle atom per row)
-  int kbs;               // work units per tile = ceil(K / (64 * atoms))
+  int kblk;              // elements of K in one 128-byte slice: 64 (16-bit operands) or 128 (8-bit floats)
+  int atoms;             // K slices per pipeline stage (each slice is one 128-byte swizzle atom per row)
+  int kbs;               // work units per tile = ceil(K / (kblk * atoms))
   long long total_units; // n_tiles * kbs (< 2^31)
   int units_q, units_r;  // total_units = grid * units_q + units_r: the first units_r CTAs take units_q + 1 units
   int grid;              // CTAs = min(SM count, total_units)
@@ -58,14 +59,16 @@ __host__ __device__ inline int sk_owner(int u, int q, int r) {
 }
 
 // M is the small output extent and N the big one (for a tall problem the caller passes them swapped).
-inline bool skinny_make_plan(SkinnyPlan* s, int M, int N, int K, int sm_count, int forced_stages, int max_smem, int forced_atoms = 0) {
+inline bool skinny_make_plan(SkinnyPlan* s, int M, int N, int K, int sm_count, int forced_stages, int max_smem, int forced_atoms = 0,
+                             int kblk = kBlockK) {
   if (M < 1 || M > kSkinnyMaxM) return false;
   s->m_pad = ((M + 15) / 16) * 16;
   s->n_tiles = (N + kSkinnyTileN - 1) / kSkinnyTileN;
   // Two adjacent 128-byte pieces of every weight row are requested together when K is long enough: DRAM then serves
   // both from one open row.
-  s->atoms = forced_atoms ? forced_atoms : (K >= 1024 ? 2 : 1);
-  s->kbs = (K + kBlockK * s->atoms - 1) / (kBlockK * s->atoms);
+  s->kblk = kblk;
+  s->atoms = forced_atoms ? forced_atoms : (K >= 16 * kblk ? 2 : 1);
+  s->kbs = (K + kblk * s->atoms - 1) / (kblk * s->atoms);
   s->total_units = static_cast<long long>(s->n_tiles) * s->kbs;
   if (s->total_units > 0x7fffffffll) return false;
   s->grid = static_cast<int>(s->total_units < sm_count ? s->total_units : sm_count);
@@ -103,6 +106,7 @@ struct SkinnyParams {
   uint32_t* status;
   unsigned long long timeout_ns;
   uint32_t debug_flags;   // bit 0: withhold one producer arrival (timeout test hook)
+  int ab_fp8;             // operands are 8-bit floats (tcgen05 kind::f8f6f4)
 };
 
 __device__ __forceinline__ float sk_load_c(const SkinnyParams& p, long long idx) {
@@ -227,7 +231,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
       if (elect_one() && !((p.debug_flags & 1u) && i == 0)) {  // test hook: the first stage is never filled nor signalled
         mbar_arrive_expect_tx(bar, sp.stage_bytes);
         for (int a = 0; a < sp.atoms; ++a) {  // slices past K are zero-filled by TMA and still count their bytes
-          const int k0 = (kb * sp.atoms + a) * kBlockK;
+          const int k0 = (kb * sp.atoms + a) * sp.kblk;
           tma_load_3d(sw_ + a * atom_bytes, &tmW, bar, k0, tile * kSkinnyTileN, 0, pol_w);
           tma_load_3d(sw_ + a * atom_bytes + kSkinnyTileN * 128u, &tmX, bar, k0, 0, 0, pol_x);
         }
@@ -267,9 +271,15 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         if (elect_one()) {
           for (uint32_t a = 0; a < static_cast<uint32_t>(sp.atoms); ++a) {
             const uint64_t wd = wdesc + a * (atom_bytes >> 4), xd = xdesc + a * (atom_bytes >> 4);
-            umma_f16<1>(d_tmem, wd, xd, idesc, static_cast<uint32_t>(i != 0 || a != 0));
+            if (!p.ab_fp8) {
+              umma_f16<1>(d_tmem, wd, xd, idesc, static_cast<uint32_t>(i != 0 || a != 0));
 #pragma unroll
-            for (uint32_t k = 1; k < kBlockK / kUmmaK; ++k) umma_f16<1>(d_tmem, wd + 2u * k, xd + 2u * k, idesc, 1u);
+              for (uint32_t k = 1; k < kBlockK / kUmmaK; ++k) umma_f16<1>(d_tmem, wd + 2u * k, xd + 2u * k, idesc, 1u);
+            } else {  // 8-bit floats: again four 32-byte steps per 128-byte slice
+              umma_f8<1>(d_tmem, wd, xd, idesc, static_cast<uint32_t>(i != 0 || a != 0));
+#pragma unroll
+              for (uint32_t k = 1; k < 4; ++k) umma_f8<1>(d_tmem, wd + 2u * k, xd + 2u * k, idesc, 1u);
+            }
           }
           umma_commit<1>(empty0 + 8u * s);
         }
