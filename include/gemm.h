@@ -269,6 +269,30 @@ gemm_status_t gemm_tune(const gemm_desc_t* desc, const void* A, const void* B, v
 /* Forget every remembered tuning result (all devices). */
 void gemm_tune_cache_clear(void);
 
+/*
+ * GEMM on HOST-resident operands (the end-to-end path of a caller whose matrices live in host memory; the
+ * paper's measurements start with the data on the GPU, so this has no counterpart there).  The output rows are cut
+ * into `panels` row panels; panel p's slice of A is copied in while panel p-1 is multiplied and panel p-2's result is
+ * copied out, on three streams owned by the handle, so the whole call costs little more than the longer of the two
+ * copy directions.  B (and the bias) go to the device once per run.
+ *
+ * gemm_host_create: desc as for gemm_plan, with transa = N and batch_count = 1 (row panels of A and C must be
+ * contiguous row ranges); panels = 0 picks a count (about 8, fewer for small M).  Allocates the device staging
+ * buffers (B, two A panels, two C panels, a workspace if the panel plan wants one), the streams and the events, on
+ * the current device.  Errors: as gemm_plan; GEMM_ERR_UNSUPPORTED for transa = T, a batch or a triangular op(A); GEMM_ERR_CUDA if an
+ * allocation fails (nothing is leaked).
+ * gemm_host_run: hA, hB, hC (and hbias, iff the epilogue has a bias): HOST pointers laid out as desc says; page-locked
+ * memory is what makes the copies overlap (pageable memory works, without overlap).  hC is read only when beta != 0
+ * and receives D.  Blocks until D is complete in hC.  Returns GEMM_ERR_TIMEOUT if a device-side wait expired.
+ * One run at a time per handle.  gemm_host_destroy frees everything; NULL is accepted.
+ */
+typedef struct gemm_host_s* gemm_host_t;
+gemm_status_t gemm_host_create(const gemm_desc_t* desc, int panels, gemm_host_t* out);
+gemm_status_t gemm_host_run(gemm_host_t h, const void* hA, const void* hB, void* hC, const float* hbias, float alpha, float beta);
+/* Row panels the handle uses (0 on NULL). */
+int gemm_host_panels(gemm_host_t h);
+gemm_status_t gemm_host_destroy(gemm_host_t h);
+
 /* Static string for a status code. */
 const char* gemm_status_string(gemm_status_t s);
 

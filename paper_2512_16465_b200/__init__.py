@@ -74,7 +74,8 @@ class TuneReport(ctypes.Structure):
 
 EXPORTS = ("gemm_plan", "gemm_workspace_bytes", "gemm_run", "gemm_plan_status", "gemm_plan_set_timeout_ms",
            "gemm_plan_info", "gemm_destroy", "gemm_status_string", "gemm_last_cuda_error", "gemm_skinny_run_noalloc",
-           "gemm_tune", "gemm_tune_workspace_bytes", "gemm_tune_cache_clear")
+           "gemm_tune", "gemm_tune_workspace_bytes", "gemm_tune_cache_clear",
+           "gemm_host_create", "gemm_host_run", "gemm_host_panels", "gemm_host_destroy")
 
 
 def _load() -> ctypes.CDLL:
@@ -110,6 +111,14 @@ def _load() -> ctypes.CDLL:
     L.gemm_tune_workspace_bytes.argtypes = [ctypes.POINTER(Desc)]
     L.gemm_tune_cache_clear.restype = None
     L.gemm_tune_cache_clear.argtypes = []
+    L.gemm_host_create.restype = ctypes.c_int
+    L.gemm_host_create.argtypes = [ctypes.POINTER(Desc), ctypes.c_int, ctypes.POINTER(vp)]
+    L.gemm_host_run.restype = ctypes.c_int
+    L.gemm_host_run.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, ctypes.c_float]
+    L.gemm_host_panels.restype = ctypes.c_int
+    L.gemm_host_panels.argtypes = [vp]
+    L.gemm_host_destroy.restype = ctypes.c_int
+    L.gemm_host_destroy.argtypes = [vp]
     return L
 
 
@@ -198,6 +207,30 @@ def gemm_tune(desc: Desc, A: int, B: int, C: int, bias: int, alpha: float, beta:
 
 def gemm_tune_cache_clear() -> None:
     _lib.gemm_tune_cache_clear()
+
+
+def gemm_host_create(desc: Desc, panels: int = 0) -> int:
+    """``gemm_host_create``: a handle for GEMMs whose operands live in host memory (row panels pipelined over three streams)."""
+    h = ctypes.c_void_p()
+    st = _lib.gemm_host_create(ctypes.byref(desc), panels, ctypes.byref(h))
+    if st != OK:
+        raise GemmError(st, "gemm_host_create")
+    return h.value
+
+
+def gemm_host_run(handle: int, hA: int, hB: int, hC: int, hbias: int, alpha: float, beta: float) -> None:
+    """``gemm_host_run`` on raw HOST addresses; returns when D is complete in the host C buffer."""
+    st = _lib.gemm_host_run(handle, hA, hB, hC, hbias or None, alpha, beta)
+    if st != OK:
+        raise GemmError(st, "gemm_host_run")
+
+
+def gemm_host_panels(handle: int) -> int:
+    return int(_lib.gemm_host_panels(handle))
+
+
+def gemm_host_destroy(handle: int) -> None:
+    _lib.gemm_host_destroy(handle)
 
 
 def gemm_plan_status(plan: int) -> int:

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libb200gemm.so")
-SOURCES = ["gemm_lib.cu", "tune.cu"]
+SOURCES = ["gemm_lib.cu", "tune.cu", "host_pipeline.cu"]
 HEADERS = ["ptx.cuh", "dense_kernel.cuh", "skinny_kernel.cuh", "wide_kernel.cuh", "launch_util.cuh", "tune_cache.h", os.path.join("..", "..", "include", "gemm.h")]
 
 

@@ -485,3 +485,55 @@ def test_tune_argument_errors():
     with pytest.raises(bg.GemmError) as e:                                          # short-extent shape whose automatic plan needs a workspace
         bg.gemm_tune(bg.make_desc(8, 256, 4096), A.data_ptr(), A.data_ptr(), C.data_ptr(), 0, 1.0, 0.0, 0, 0, 0)
     assert e.value.status == bg.ERR_WORKSPACE
+
+
+# ----------------------------------------------------------------------------- host-resident operands
+
+@pytest.mark.parametrize("case", [
+    ("host_three_panels_beta_bias", 700, 328, 136, dict(beta=1.0, epi=bg.EPI_BIAS_RELU, cd=wl.BF16, ldc=328 + 24, lda=136 + 8), 3),
+    ("host_default_panels_small", 100, 264, 72, dict(), 0),
+    ("host_row_bias_nn", 1000, 136, 200, dict(epi=bg.EPI_BIAS, bias_per_row=True, tb=0), 4),
+    ("host_skinny_panel", 40, 520, 1032, dict(beta=1.0), 1),
+    ("host_fp8", 600, 264, 272, dict(ab=wl.FP8_E4M3, cd=wl.F16), 2),
+], ids=lambda c: c[0])
+def test_host_resident_gemm_exact(case):
+    """gemm_host_run on pinned host buffers: bit-exact against the oracle, padding of the host C buffer untouched,
+    and the same again on a second run of the same handle."""
+    name, M, N, K, kw, panels = case
+    w = int_workload(name, M, N, K, **kw)
+    inputs = wl.make_inputs(w)
+    pin = lambda a: None if a is None else torch.from_numpy(a).pin_memory()
+    hA, hB, hbias = pin(inputs["A"]), pin(inputs["B"]), pin(inputs["bias"])
+    c_np = np.float32 if w.c_dtype == wl.F32 else np.uint16
+    sentinel = np.full(w.elems_c(), 0x4321 if c_np == np.uint16 else 1234.5, c_np)
+    handle = bg.gemm_host_create(H.desc_of(w), panels)
+    try:
+        want_panels = {3: 3, 0: 1, 4: 4, 1: 1, 2: 2}[panels]
+        assert bg.gemm_host_panels(handle) == want_panels
+        for _ in range(2):
+            hC = pin(inputs["C"].copy() if inputs["C"] is not None else sentinel.copy())
+            bg.gemm_host_run(handle, hA.data_ptr(), hB.data_ptr(), hC.data_ptr(), 0 if hbias is None else hbias.data_ptr(),
+                             float(w.alpha), float(w.beta))
+            got = hC.numpy()
+            reports = H.check_blocks(w, inputs, got, H.default_blocks(w))
+            assert all(r["bit_identical"] == 1.0 for r in reports)
+            before = inputs["C"] if inputs["C"] is not None else sentinel
+            mask = np.ones(w.elems_c(), bool)
+            mask[(np.arange(w.M)[:, None] * w.ldc + np.arange(w.N)[None, :]).ravel()] = False
+            assert np.array_equal(got[mask], before[mask])           # row padding of the host buffer is not written
+    finally:
+        bg.gemm_host_destroy(handle)
+
+
+def test_host_resident_gemm_refusals():
+    for kw in (dict(transa=bg.OP_T), dict(batch=2), dict(flags=bg.make_flags(a_lower=True))):
+        with pytest.raises(bg.GemmError) as e:
+            bg.gemm_host_create(bg.make_desc(256, 256, 256, **kw))
+        assert e.value.status == bg.ERR_UNSUPPORTED
+    h = bg.gemm_host_create(bg.make_desc(256, 256, 64, epilogue=bg.EPI_BIAS))
+    buf = torch.zeros(256 * 256, dtype=torch.float32).pin_memory()
+    with pytest.raises(bg.GemmError) as e:
+        bg.gemm_host_run(h, buf.data_ptr(), buf.data_ptr(), buf.data_ptr(), 0, 1.0, 0.0)
+    assert e.value.status == bg.ERR_NULL
+    bg.gemm_host_destroy(h)
+    bg.gemm_host_destroy(0)
