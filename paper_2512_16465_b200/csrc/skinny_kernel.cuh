@@ -109,16 +109,6 @@ struct SkinnyParams {
   int ab_fp8;             // operands are 8-bit floats (tcgen05 kind::f8f6f4)
 };
 
-__device__ __forceinline__ float sk_load_c(const SkinnyParams& p, long long idx) {
-  if (p.out_dtype == 2) return static_cast<const float*>(p.c)[idx];
-  if (p.out_dtype == 0) return __bfloat162float(static_cast<const __nv_bfloat16*>(p.c)[idx]);
-  return __half2float(static_cast<const __half*>(p.c)[idx]);
-}
-__device__ __forceinline__ void sk_store_d(const SkinnyParams& p, long long idx, float v) {
-  if (p.out_dtype == 2) static_cast<float*>(p.c)[idx] = v;
-  else if (p.out_dtype == 0) static_cast<__nv_bfloat16*>(p.c)[idx] = __float2bfloat16_rn(v);
-  else static_cast<__half*>(p.c)[idx] = __float2half_rn(v);
-}
 // `big` is this thread's index along the long output extent, s0 the first of its 16 indices along the short one.
 // D is row-major M x N: the short extent is M (rows) unless kTall.
 template <bool kTall>
@@ -132,24 +122,78 @@ template <bool kTall>
 __device__ __forceinline__ void sk_load_cin16(const SkinnyParams& p, int s0, int big, float (&cin)[16]) {
   const int small_extent = kTall ? p.N : p.M;
 #pragma unroll
-  for (int j = 0; j < 16; ++j)
-    cin[j] = (p.beta != 0.0f && s0 + j < small_extent) ? sk_load_c(p, sk_index<kTall>(p, s0 + j, big)) : 0.0f;
+  for (int j = 0; j < 16; ++j) cin[j] = 0.0f;
+  if (p.beta == 0.0f) return;
+  const long long i0 = sk_index<kTall>(p, s0, big);
+  const long long step = kTall ? 1 : p.ldc;
+  if (p.out_dtype == 2) {  // (the type switch stays outside the loop, see sk_finish16)
+    const float* c = static_cast<const float*>(p.c) + i0;
+#pragma unroll
+    for (int j = 0; j < 16; ++j)
+      if (s0 + j < small_extent) cin[j] = c[j * step];
+  } else if (p.out_dtype == 0) {
+    const __nv_bfloat16* c = static_cast<const __nv_bfloat16*>(p.c) + i0;
+#pragma unroll
+    for (int j = 0; j < 16; ++j)
+      if (s0 + j < small_extent) cin[j] = __bfloat162float(c[j * step]);
+  } else {
+    const __half* c = static_cast<const __half*>(p.c) + i0;
+#pragma unroll
+    for (int j = 0; j < 16; ++j)
+      if (s0 + j < small_extent) cin[j] = __half2float(c[j * step]);
+  }
 }
+// The switches on activation and output type sit outside the loops over the 16 values: this code runs once per
+// kernel, from a cold instruction cache, and a branch per value (each jumping over the inlined bodies of the other
+// cases) cost hundreds of cycles per value in instruction fetches.
 template <bool kTall>
 __device__ __forceinline__ void sk_finish16(const SkinnyParams& p, int s0, int big, const float (&acc)[16], const float (&cin)[16]) {
   const int small_extent = kTall ? p.N : p.M;
   const bool has_bias = (p.epilogue & 1) != 0;
   // the bias runs along N (the long extent unless kTall) or, per row, along M
   const bool bias_along_big = kTall ? p.bias_per_row != 0 : p.bias_per_row == 0;
-  const float bias_big = (bias_along_big && has_bias) ? __ldg(p.bias + big) : 0.0f;
-  const int act = p.epilogue >> 1;
+  float v[16];
+  if (has_bias && !bias_along_big) {
 #pragma unroll
-  for (int j = 0; j < 16; ++j) {
-    if (s0 + j < small_extent) {
-      const float bias = (!bias_along_big && has_bias) ? __ldg(p.bias + s0 + j) : bias_big;
-      const float v = activate(p.alpha * acc[j] + p.beta * cin[j] + bias, act);
-      sk_store_d(p, sk_index<kTall>(p, s0 + j, big), v);
-    }
+    for (int j = 0; j < 16; ++j) v[j] = (s0 + j < small_extent) ? __ldg(p.bias + s0 + j) : 0.0f;
+  } else {
+    const float bias_big = has_bias ? __ldg(p.bias + big) : 0.0f;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) v[j] = bias_big;
+  }
+#pragma unroll
+  for (int j = 0; j < 16; ++j) v[j] += p.alpha * acc[j] + p.beta * cin[j];
+  const int act = p.epilogue >> 1;
+  if (act == 1) {
+#pragma unroll
+    for (int j = 0; j < 16; ++j) v[j] = fmaxf(v[j], 0.0f);
+  } else if (act == 2) {
+#pragma unroll
+    for (int j = 0; j < 16; ++j) v[j] = gelu_erf(v[j]);
+  } else if (act == 3) {
+#pragma unroll
+    for (int j = 0; j < 16; ++j) v[j] = gelu_tanh(v[j]);
+  } else if (act == 4) {
+#pragma unroll
+    for (int j = 0; j < 16; ++j) v[j] = silu(v[j]);
+  }
+  const long long i0 = sk_index<kTall>(p, s0, big);
+  const long long step = kTall ? 1 : p.ldc;  // from one of the 16 values to the next
+  if (p.out_dtype == 2) {
+    float* d = static_cast<float*>(p.c) + i0;
+#pragma unroll
+    for (int j = 0; j < 16; ++j)
+      if (s0 + j < small_extent) d[j * step] = v[j];
+  } else if (p.out_dtype == 0) {
+    __nv_bfloat16* d = static_cast<__nv_bfloat16*>(p.c) + i0;
+#pragma unroll
+    for (int j = 0; j < 16; ++j)
+      if (s0 + j < small_extent) d[j * step] = __float2bfloat16_rn(v[j]);
+  } else {
+    __half* d = static_cast<__half*>(p.c) + i0;
+#pragma unroll
+    for (int j = 0; j < 16; ++j)
+      if (s0 + j < small_extent) d[j * step] = __float2half_rn(v[j]);
   }
 }
 
