@@ -515,8 +515,8 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
     // everything else is a dense tiled GEMM, paired CTAs when there are at least two tile rows
     const bool skinny_ok = (d.M <= kSkinnyMaxM || d.N <= kSkinnyMaxM) && d.batch_count == 1 && d.transa == GEMM_OP_N &&
                            d.transb == GEMM_OP_T && !(d.flags & (GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER));
-    if (skinny_ok && info.intensity < 5.2 * kRidgeCudaCore) {
-      variant = GEMM_VARIANT_SKINNY_STREAMK;  // measured: wins up to M ~ 48
+    if (skinny_ok && info.intensity < 7.0 * kRidgeCudaCore) {
+      variant = GEMM_VARIANT_SKINNY_STREAMK;  // measured: level with the dense kernels at a short extent of 64 on the largest shapes, far ahead elsewhere
     } else {
       // score every dense family and tile width with the roofline estimate and take the cheapest
       const bool b_kmajor = d.transb == GEMM_OP_T;

@@ -67,15 +67,18 @@ inline bool skinny_make_plan(SkinnyPlan* s, int M, int N, int K, int sm_count, i
   // Two adjacent 128-byte pieces of every weight row are requested together when K is long enough: DRAM then serves
   // both from one open row.
   s->kblk = kblk;
-  s->atoms = forced_atoms ? forced_atoms : (K >= 16 * kblk ? 2 : 1);
+  const int fixed = 1024 + 16 * kMaxStages + 64 + kSkinnyParkBytes;
+  const int slice_bytes = kSkinnyTileN * 128 + s->m_pad * 128;
+  // ... as long as four such double stages fit (a short extent of 64 leaves room for three only: single slices, seven deep,
+  // measured faster there)
+  s->atoms = forced_atoms ? forced_atoms : ((K >= 16 * kblk && (max_smem - fixed) / (2 * slice_bytes) >= 4) ? 2 : 1);
   s->kbs = (K + kblk * s->atoms - 1) / (kblk * s->atoms);
   s->total_units = static_cast<long long>(s->n_tiles) * s->kbs;
   if (s->total_units > 0x7fffffffll) return false;
   s->grid = static_cast<int>(s->total_units < sm_count ? s->total_units : sm_count);
   s->units_q = static_cast<int>(s->total_units / s->grid);
   s->units_r = static_cast<int>(s->total_units % s->grid);
-  s->stage_bytes = s->atoms * (kSkinnyTileN * 128 + s->m_pad * 128);
-  const int fixed = 1024 + 16 * kMaxStages + 64 + kSkinnyParkBytes;
+  s->stage_bytes = s->atoms * slice_bytes;
   int stages = forced_stages ? forced_stages : (max_smem - fixed) / s->stage_bytes;
   if (stages > kMaxStages) stages = kMaxStages;
   if (!forced_stages && stages * s->atoms > 8) stages = 8 / s->atoms > 3 ? 8 / s->atoms : 3;  // measured on B200: ~144 KB in flight per SM streams fastest

@@ -177,7 +177,8 @@ def test_cost_model_choices_follow_the_measurements():
     assert choice(16, 28672, 8192)[0] == bg.VARIANT_SKINNY_STREAMK
     assert choice(28672, 16, 8192)[0] == bg.VARIANT_SKINNY_STREAMK            # mirrored: the long operand is A
     assert choice(28672, 16, 8192, transb=bg.OP_N)[0] != bg.VARIANT_SKINNY_STREAMK   # needs both operands K-contiguous
-    assert choice(64, 28672, 8192)[0] == bg.VARIANT_DENSE_1CTA               # stream-K stops paying near M = 48
+    assert choice(64, 28672, 8192)[0] == bg.VARIANT_SKINNY_STREAMK            # up to the largest short extent the path takes
+    assert choice(128, 28672, 8192)[0] == bg.VARIANT_DENSE_1CTA
     v, bn = choice(2048, 2048, 128, batch=64)
     assert (v, bn) == (bg.VARIANT_DENSE_2CTA_WIDE, 256)                      # output-bound: largest tile, fewest tile switches
     assert choice(8192, 8192, 1024)[0] == bg.VARIANT_DENSE_2CTA              # the pair beats the single CTA at every K measured
