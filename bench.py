@@ -40,7 +40,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the full-size ncu captures
 # summarised under profiles/ (dense_*_cN_*.txt, skinny_streamk_c5_*.txt; last line of each file).
-NCU_TRAFFIC_BYTES = {"c1": 1123584, "c2": 873626624, "c3": 1637930408, "c4": 545520896, "c5": 478118656}
+NCU_TRAFFIC_BYTES = {"c1": 1125632, "c2": 871944960, "c3": 1644200816, "c4": 544876800, "c5": 478002688}
 
 
 def load_peaks():
@@ -182,6 +182,13 @@ class DeviceCase:
         for _ in range(warmup):
             self.step()
         torch.cuda.synchronize()
+        # a configuration whose launches take microseconds would otherwise be timed while the clocks are still
+        # ramping up from idle: keep warming up (untimed) until 30 ms have passed
+        t_warm = time.perf_counter()
+        while time.perf_counter() - t_warm < 0.03:
+            for _ in range(16):
+                self.step()
+            torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for _ in range(steps):
