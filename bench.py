@@ -179,13 +179,14 @@ class DeviceCase:
     def time_steps(self, steps: int, warmup: int) -> float:
         """Seconds per step over `steps` back-to-back steps (CUDA events on the launching stream)."""
         torch = self.torch
+        t_warm = time.perf_counter()
         for _ in range(warmup):
             self.step()
         torch.cuda.synchronize()
         # a configuration whose launches take microseconds would otherwise be timed while the clocks are still
-        # ramping up from idle: keep warming up (untimed) until 30 ms have passed
-        t_warm = time.perf_counter()
-        while time.perf_counter() - t_warm < 0.03:
+        # ramping up from idle: such a one keeps warming up (untimed) until 30 ms have passed
+        short_steps = (time.perf_counter() - t_warm) / warmup < 100e-6
+        while short_steps and time.perf_counter() - t_warm < 0.03:
             for _ in range(16):
                 self.step()
             torch.cuda.synchronize()
