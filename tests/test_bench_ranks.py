@@ -69,3 +69,20 @@ def test_reference_arm_under_torchrun_prints_one_line_from_rank0():
     assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["value"] == d["value"] > 0
     assert d["e2e"] == {"value": d["value"], "unit": d["unit"], "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
     assert d["unit"] == "TFLOP/s" and d["higher_is_better"] is True and d["config"]["workload"].startswith("c1")
+
+
+def test_shape_specifications_of_the_sweep_mode():
+    import pytest
+    import bench
+    import workloads as wl
+    w = bench.parse_shape("28672x8x8192:beta=1:cd=f32:epi=bias_silu:rowbias=1")
+    assert (w.M, w.N, w.K, w.beta, w.c_dtype, w.epilogue, w.bias_per_row) == (28672, 8, 8192, 1.0, wl.F32, wl.EPI_BIAS_SILU, True)
+    w = bench.parse_shape("256x128x512:ab=e4m3:tri=upper:batch=3:ta=0:tb=1:lda=520")
+    assert (w.ab_dtype, w.a_tri, w.batch, w.lda, w.c_dtype) == (wl.FP8_E4M3, 2, 3, 520, wl.BF16)
+    assert w.min_bytes == 3 * (256 * 512 + 512 * 128) * 1 + 3 * 256 * 128 * 2       # 8-bit operands, 16-bit output
+    with pytest.raises(SystemExit):
+        bench.parse_shape("8x8x8:nonsense=1")
+    # an 8-bit problem is held against the measured bf16 peak times the nominal fp8 : bf16 ratio
+    peaks = {"bf16_tflops": 1000.0, "bf16_tflops_sustained": 900.0, "hbm_gbs": 6000.0}
+    r = bench.roofline_for(bench.parse_shape("8192x8192x8192:ab=e4m3"), "x", 1e-3, peaks, "measured")
+    assert r["bound"] == "tensor" and r["peak"] == 2000.0 and abs(r["frac"] - 2 * 8192 ** 3 / 1e-3 / 1e12 / 2000.0) < 1e-3
