@@ -87,7 +87,9 @@ typedef enum {
   GEMM_VARIANT_DENSE_2CTA_WIDE = 4  /* CTA pair, 512 x 256 pair tile: least operand traffic per FLOP */
 } gemm_variant_t;
 
-/* gemm_desc_t.flags: 0 = let the plan decide everything. */
+/* gemm_desc_t.flags: 0 = the plain problem, every choice left to the plan.  The first group are tuning fields (they
+ * never change the result; gemm_tune chooses them by measurement), the second group changes what is computed or how
+ * it is launched. */
 #define GEMM_FLAG_VARIANT_SHIFT 4          /* bits 4-7: force a gemm_variant_t (0 = automatic) */
 #define GEMM_FLAG_VARIANT_MASK 0xF0u
 #define GEMM_FLAG_TILE_N_SHIFT 8           /* bits 8-15: force tile N / 16 (0 = automatic) */
@@ -96,7 +98,8 @@ typedef enum {
 #define GEMM_FLAG_RASTER_MASK 0x7F0000u
 #define GEMM_FLAG_STAGES_SHIFT 24          /* bits 24-27: force the pipeline depth (0 = automatic) */
 #define GEMM_FLAG_STAGES_MASK 0xF000000u
-#define GEMM_FLAG_KSLICES_SHIFT 28         /* bits 28-29: force 64-wide K slices per pipeline stage, 1 or 2 (0 = automatic) */
+#define GEMM_FLAG_KSLICES_SHIFT 28         /* bits 28-29: force the number of 128-byte K slices (64 elements of 16 bits, 128 of 8)
+                                              per pipeline stage: 1 or 2, stream-K also 3 (0 = automatic) */
 #define GEMM_FLAG_KSLICES_MASK 0x30000000u
 #define GEMM_FLAG_NO_K_SERPENTINE 0x8u      /* walk K forwards in every tile (default: alternate tiles walk it backwards,
                                               which re-uses the operand lines L2 touched last) */
