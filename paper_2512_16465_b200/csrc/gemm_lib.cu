@@ -184,7 +184,10 @@ double estimate_dense_cycles(const gemm_desc_t& d, int sm_count, int variant, in
   const double eff = wide ? 1.0 : (cg == 1 ? eff1[bi] : eff2[bi]);
   const double mma = kblocks * 4.0 * (bn / 2.0) * (rows_cta / 128.0) / eff;
   // operand feed: bytes this SM receives per k-block at ~90 B/clk
-  const double feed = kblocks * (rows_cta + static_cast<double>(bn) / cg) * 128.0 / 90.0;
+  // ... and half that rate when an operand's row pitch is not a multiple of 128 bytes: every row of a TMA box then
+  // straddles two memory lines (measured: the families rank by loads per FLOP there, wide > pair > single CTA)
+  const bool straddling = (d.lda * elem_bytes(d.ab_dtype)) % 128 != 0 || (d.ldb * elem_bytes(d.ab_dtype)) % 128 != 0;
+  const double feed = kblocks * (rows_cta + static_cast<double>(bn) / cg) * 128.0 / (straddling ? 45.0 : 90.0);
   // output: this SM's share of the HBM write bandwidth is ~16 B/clk
   const double out = static_cast<double>(rows_cta) * bn * elem_bytes(d.c_dtype) / 16.0;
   const bool gelu = d.epilogue >= GEMM_EPI_GELU_ERF;  // any transcendental activation
