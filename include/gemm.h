@@ -124,8 +124,8 @@ typedef struct {
   uint32_t flags;        /* GEMM_FLAG_* */
   int64_t M, N, K;       /* op(A) is M x K, op(B) is K x N, C/D is M x N; all >= 1 */
   int32_t transa, transb;     /* gemm_op_t */
-  int32_t ab_dtype;           /* gemm_dtype_t: GEMM_BF16, GEMM_F16, or an 8-bit float (then transa = N, transb = T; not the wide
-                                 pair variant), for both A and B */
+  int32_t ab_dtype;           /* gemm_dtype_t: GEMM_BF16, GEMM_F16, or an 8-bit float (then transa = N and transb = T), for both A
+                                 and B */
   int32_t c_dtype;            /* gemm_dtype_t of C/D */
   int64_t lda, ldb, ldc;      /* leading dimensions in elements */
   int32_t batch_count;        /* >= 1 */

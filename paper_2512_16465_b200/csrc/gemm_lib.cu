@@ -342,7 +342,6 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
 // Wide pair variant: 512 x 256 cluster tiles, one 64-wide K slice per stage, 3-deep ring, 8 epilogue warps.
 gemm_status_t plan_wide(gemm_plan_s* pl, int forced_raster, int forced_stages) {
   const gemm_desc_t& d = pl->d;
-  if (is_fp8(d.ab_dtype)) return GEMM_ERR_UNSUPPORTED;  // 16-bit operands only
   // its epilogue covers the bias per column, ReLU and erf GELU only; its MMA schedule has no K-range skipping
   if (d.epilogue > GEMM_EPI_BIAS_GELU_ERF || (d.flags & (GEMM_FLAG_BIAS_PER_ROW | GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER))) return GEMM_ERR_UNSUPPORTED;
   const int a_kmajor = d.transa == GEMM_OP_N;
@@ -374,12 +373,12 @@ gemm_status_t plan_wide(gemm_plan_s* pl, int forced_raster, int forced_stages) {
   p.raster_group = raster;
   p.bn = bn;
   p.stages = stages;
-  p.num_kb = ceil_div(d.K, kBlockK);
-  p.kblk = kBlockK;
-  p.ab_fp8 = 0;
+  p.num_kb = ceil_div(d.K, kblk_of(d.ab_dtype));
+  p.kblk = kblk_of(d.ab_dtype);
+  p.ab_fp8 = is_fp8(d.ab_dtype) ? 1 : 0;
   p.atoms = 1;
   p.tmem_cols = 512;
-  p.idesc = make_idesc(d.ab_dtype == GEMM_BF16, !a_kmajor, !b_kmajor, 256, bn);
+  p.idesc = make_idesc(ab_format(d.ab_dtype), !a_kmajor, !b_kmajor, 256, bn);
   p.a_stage_bytes = a_stage;
   p.b_stage_bytes = b_stage;
   p.a_atom_bytes = a_stage;
@@ -412,7 +411,7 @@ gemm_status_t plan_wide(gemm_plan_s* pl, int forced_raster, int forced_stages) {
   info.variant = pl->variant;
   info.tile_m = tile_m;
   info.tile_n = bn;
-  info.tile_k = kBlockK;
+  info.tile_k = kblk_of(d.ab_dtype);
   info.stages = stages;
   info.cluster_size = 2;
   info.grid = pl->grid;
@@ -527,7 +526,6 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
       for (int v : {GEMM_VARIANT_DENSE_1CTA, GEMM_VARIANT_DENSE_2CTA, GEMM_VARIANT_DENSE_2CTA_WIDE}) {
         for (int bn : {256, 128, 64}) {
           if (v == GEMM_VARIANT_DENSE_2CTA_WIDE && bn != kWideTileN) continue;
-          if (v == GEMM_VARIANT_DENSE_2CTA_WIDE && is_fp8(d.ab_dtype)) continue;
           if (v == GEMM_VARIANT_DENSE_2CTA_WIDE &&
               (d.epilogue > GEMM_EPI_BIAS_GELU_ERF || (d.flags & (GEMM_FLAG_BIAS_PER_ROW | GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER))))
             continue;
@@ -676,7 +674,9 @@ gemm_status_t launch_dense(const gemm_plan_s* pl, const CUtensorMap& tA, const C
 
 gemm_status_t launch_wide(const gemm_plan_s* pl, const CUtensorMap& tA, const CUtensorMap& tB, const CUtensorMap& tD,
                           const DenseParams& p, cudaStream_t stream) {
-  if (ensure_dynamic_smem(reinterpret_cast<const void*>(wide_gemm_kernel), kSlotWide, pl->device, pl->smem_bytes) != cudaSuccess) {
+  const bool fp8 = is_fp8(pl->d.ab_dtype);
+  const void* kern = fp8 ? reinterpret_cast<const void*>(wide_gemm_kernel<true>) : reinterpret_cast<const void*>(wide_gemm_kernel<false>);
+  if (ensure_dynamic_smem(kern, fp8 ? kSlotWideFp8 : kSlotWide, pl->device, pl->smem_bytes) != cudaSuccess) {
     note_cuda_error("cudaFuncSetAttribute", cudaGetErrorName(cudaGetLastError()));
     return GEMM_ERR_CUDA;
   }
@@ -695,7 +695,7 @@ gemm_status_t launch_wide(const gemm_plan_s* pl, const CUtensorMap& tA, const CU
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = (pl->d.flags & GEMM_FLAG_NO_EARLY_LAUNCH) ? 1 : 2;
-  cudaError_t e = cudaLaunchKernelEx(&cfg, wide_gemm_kernel, tA, tB, tD, p);
+  cudaError_t e = fp8 ? cudaLaunchKernelEx(&cfg, wide_gemm_kernel<true>, tA, tB, tD, p) : cudaLaunchKernelEx(&cfg, wide_gemm_kernel<false>, tA, tB, tD, p);
   if (e != cudaSuccess) {
     note_cuda_error("cudaLaunchKernelEx(wide)", cudaGetErrorName(e));
     (void)cudaGetLastError();

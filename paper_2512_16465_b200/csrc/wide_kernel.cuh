@@ -41,6 +41,8 @@ __device__ __forceinline__ uint32_t pack_f16x2_pinned(float lo, float hi) {
   return d;
 }
 
+// kFp8: 8-bit float operands (128 elements of K per 128-byte slice, tcgen05 kind::f8f6f4); otherwise 16-bit.
+template <bool kFp8>
 __device__ __forceinline__ void wide_producer_role(const DenseParams& p, const CUtensorMap* tmA, const CUtensorMap* tmB,
                                                    uint32_t tiles_base, uint32_t full0, uint32_t empty0, uint32_t cta_rank,
                                                    int cluster_id, int num_clusters, const WaitCtx& w) {
@@ -55,8 +57,9 @@ __device__ __forceinline__ void wide_producer_role(const DenseParams& p, const C
     const int m0 = tc.tm * (2 * kWideCtaM) + static_cast<int>(cta_rank) * kWideCtaM;
     const int n0 = tc.tn * kWideTileN + static_cast<int>(cta_rank) * p.b_rows;
     const bool rev = p.k_serpentine && (it & 1u);  // see dense_kernel.cuh: re-use what L2 touched last
-    int k0 = rev ? (p.num_kb - 1) * kBlockK : 0;
-    const int dk = rev ? -kBlockK : kBlockK;
+    constexpr int kSliceK = kFp8 ? 2 * kBlockK : kBlockK;
+    int k0 = rev ? (p.num_kb - 1) * kSliceK : 0;
+    const int dk = rev ? -kSliceK : kSliceK;
     for (int kb = 0; kb < p.num_kb; ++kb, k0 += dk) {
       if (!mbar_wait_warp(empty0 + 8u * s, ph ^ 1u, w, (1u << 8) | s)) return;
       if (stall_pending) {  // test hook: this stage is never filled nor signalled
@@ -89,6 +92,13 @@ __device__ __forceinline__ void wide_producer_role(const DenseParams& p, const C
   }
 }
 
+template <bool kFp8>
+__device__ __forceinline__ void wide_umma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  if constexpr (kFp8) umma_f8<2>(tmem_d, adesc, bdesc, idesc, accumulate);
+  else umma_f16<2>(tmem_d, adesc, bdesc, idesc, accumulate);
+}
+
+template <bool kFp8>
 __device__ __forceinline__ void wide_mma_role(const DenseParams& p, uint32_t tiles_base, uint32_t full0, uint32_t empty0,
                                               uint32_t tfull, uint32_t tempty0, uint32_t tmem_base, int cluster_id,
                                               int num_clusters, const WaitCtx& w) {
@@ -127,9 +137,9 @@ __device__ __forceinline__ void wide_mma_role(const DenseParams& p, uint32_t til
         if (!mbar_wait_warp(full0 + 8u * s0, ph0, w, (2u << 8) | s0)) return;
         tc_fence_after();
         if (elect_one()) {
-          umma_f16<2>(tmem_base, a0, b0, idesc, static_cast<uint32_t>(kb != 0));
+          wide_umma<kFp8>(tmem_base, a0, b0, idesc, static_cast<uint32_t>(kb != 0));
 #pragma unroll
-          for (uint32_t k = 1; k < kBlockK / kUmmaK; ++k) umma_f16<2>(tmem_base, a0 + k * ak16, b0 + k * bk16, idesc, 1u);
+          for (uint32_t k = 1; k < kBlockK / kUmmaK; ++k) wide_umma<kFp8>(tmem_base, a0 + k * ak16, b0 + k * bk16, idesc, 1u);
         }
         __syncwarp();
         advance(s0, ph0, a0, b0);
@@ -138,10 +148,10 @@ __device__ __forceinline__ void wide_mma_role(const DenseParams& p, uint32_t til
       tc_fence_after();
       for (int kb = 0; kb < lead; ++kb) {
         if (elect_one()) {
-          umma_f16<2>(tmem_base + kWideTileN, adesc + half16, bdesc, idesc, static_cast<uint32_t>(kb != 0));
+          wide_umma<kFp8>(tmem_base + kWideTileN, adesc + half16, bdesc, idesc, static_cast<uint32_t>(kb != 0));
 #pragma unroll
           for (uint32_t k = 1; k < kBlockK / kUmmaK; ++k)
-            umma_f16<2>(tmem_base + kWideTileN, adesc + half16 + k * ak16, bdesc + k * bk16, idesc, 1u);
+            wide_umma<kFp8>(tmem_base + kWideTileN, adesc + half16 + k * ak16, bdesc + k * bk16, idesc, 1u);
           umma_commit_pair_mcast(empty0 + 8u * s, 3);  // ring slot free in both CTAs once both halves have read it
         }
         __syncwarp();
@@ -153,10 +163,10 @@ __device__ __forceinline__ void wide_mma_role(const DenseParams& p, uint32_t til
       tc_fence_after();
       if (elect_one()) {
 #pragma unroll
-        for (uint32_t k = 0; k < kBlockK / kUmmaK; ++k) umma_f16<2>(tmem_base, adesc + k * ak16, bdesc + k * bk16, idesc, 1u);
+        for (uint32_t k = 0; k < kBlockK / kUmmaK; ++k) wide_umma<kFp8>(tmem_base, adesc + k * ak16, bdesc + k * bk16, idesc, 1u);
 #pragma unroll
         for (uint32_t k = 0; k < kBlockK / kUmmaK; ++k)
-          umma_f16<2>(tmem_base + kWideTileN, adesc + half16 + k * ak16, bdesc + k * bk16, idesc, 1u);
+          wide_umma<kFp8>(tmem_base + kWideTileN, adesc + half16 + k * ak16, bdesc + k * bk16, idesc, 1u);
         umma_commit_pair_mcast(empty0 + 8u * s, 3);
       }
       __syncwarp();
@@ -172,7 +182,7 @@ __device__ __forceinline__ void wide_mma_role(const DenseParams& p, uint32_t til
         tc_fence_after();
         if (elect_one()) {
 #pragma unroll
-          for (uint32_t k = 0; k < kBlockK / kUmmaK; ++k) umma_f16<2>(tmem_base, a0 + k * ak16, b0 + k * bk16, idesc, 1u);
+          for (uint32_t k = 0; k < kBlockK / kUmmaK; ++k) wide_umma<kFp8>(tmem_base, a0 + k * ak16, b0 + k * bk16, idesc, 1u);
         }
         __syncwarp();
         advance(s0, ph0, a0, b0);
@@ -183,7 +193,7 @@ __device__ __forceinline__ void wide_mma_role(const DenseParams& p, uint32_t til
         if (elect_one()) {
 #pragma unroll
           for (uint32_t k = 0; k < kBlockK / kUmmaK; ++k)
-            umma_f16<2>(tmem_base + kWideTileN, adesc + half16 + k * ak16, bdesc + k * bk16, idesc, 1u);
+            wide_umma<kFp8>(tmem_base + kWideTileN, adesc + half16 + k * ak16, bdesc + k * bk16, idesc, 1u);
           umma_commit_pair_mcast(empty0 + 8u * s, 3);
         }
         __syncwarp();
@@ -309,6 +319,7 @@ __device__ __forceinline__ void wide_epilogue_role(const DenseParams& p, const C
   }
   if (lane == 0) bulk_wait_group_read<0>();
 }
+template <bool kFp8>
 __global__ void __launch_bounds__(kWideThreads, 1)
 wide_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const __grid_constant__ CUtensorMap tmD, const DenseParams p) {
@@ -361,9 +372,9 @@ wide_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   griddep_wait();  // barriers and tensor memory are set up; from here on global memory is read and written
 
   if (warp == 0) {
-    wide_producer_role(p, &tmA, &tmB, base, full0, empty0, cta_rank, cluster_id, num_clusters, w);
+    wide_producer_role<kFp8>(p, &tmA, &tmB, base, full0, empty0, cta_rank, cluster_id, num_clusters, w);
   } else if (warp == 1) {
-    if (cta_rank == 0) wide_mma_role(p, base, full0, empty0, tfull, tempty0, tmem_base, cluster_id, num_clusters, w);
+    if (cta_rank == 0) wide_mma_role<kFp8>(p, base, full0, empty0, tfull, tempty0, tmem_base, cluster_id, num_clusters, w);
   } else if (warp >= 4) {
     wide_epilogue_role(p, &tmD, base + staging_off, tfull, tempty0, tmem_base, cta_rank, cluster_id, num_clusters, w);
   }

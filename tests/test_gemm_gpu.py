@@ -120,6 +120,9 @@ EXACT_CASES = [
     ("fp8_e4m3_tiny_k", 128, 64, 16, dict(ab=wl.FP8_E4M3), dict(variant=V1, tile_n=64)),
     ("fp8_e4m3_lower_triangular", 512, 264, 512, dict(ab=wl.FP8_E4M3, a_tri=1), dict(variant=V2, tile_n=128)),
     ("fp8_e4m3_auto", 1024, 1024, 2048, dict(ab=wl.FP8_E4M3, cd=wl.BF16), dict()),
+    ("fp8_e4m3_wide", 1024, 512, 2048, dict(ab=wl.FP8_E4M3, cd=wl.BF16), dict(variant=VW)),
+    ("fp8_e5m2_wide_ragged_bias_relu", 700, 328, 1040, dict(ab=wl.FP8_E5M2, epi=bg.EPI_BIAS_RELU, beta=1.0), dict(variant=VW)),
+    ("fp8_e4m3_wide_short_k", 600, 264, 128, dict(ab=wl.FP8_E4M3), dict(variant=VW)),
     ("fp8_e4m3_stream_k", 8, 520, 4096 + 128, dict(ab=wl.FP8_E4M3, beta=1.0), dict(variant=VS)),
     ("fp8_e5m2_stream_k_tall_bias", 1000, 33, 1040, dict(ab=wl.FP8_E5M2, cd=wl.BF16, epi=bg.EPI_BIAS, ldc=40), dict(variant=VS)),
     ("fp8_e4m3_stream_k_one_slice", 16, 384, 2048, dict(ab=wl.FP8_E4M3), dict(variant=VS, kslices=1)),
@@ -404,9 +407,6 @@ def test_fp8_refusals():
         with pytest.raises(bg.GemmError) as e:
             bg.gemm_plan(bg.make_desc(256, 256, 256, ab_dtype=bg.FP8_E4M3, **kw))
         assert e.value.status == bg.ERR_UNSUPPORTED
-    with pytest.raises(bg.GemmError) as e:                                        # the wide pair kernel is 16-bit only: refused
-        bg.gemm_plan(bg.make_desc(1024, 1024, 4096, ab_dtype=bg.FP8_E5M2, flags=bg.make_flags(VW)))
-    assert e.value.status == bg.ERR_UNSUPPORTED
     h = bg.gemm_plan(bg.make_desc(8, 4096, 4096, ab_dtype=bg.FP8_E4M3))             # short extent: stream-K with 128-wide K slices
     assert bg.gemm_plan_info(h)["variant"] == VS and bg.gemm_plan_info(h)["tile_k"] == 256
     bg.gemm_destroy(h)
