@@ -235,9 +235,11 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   const bool single_wave = tiles_total <= units;  // every CTA (pair) computes at most one tile: pure latency
   // A tile's main loop lasts about 512 cycles per 64 columns of K (at tile N = 256); draining 128 x 256 accumulators
   // with four warps takes several thousand.  Short-K (output-bound) problems with several tiles per CTA get a second
-  // epilogue warpgroup (measured: a gain only up to K = 512 at tile N = 256; 7-14 % slower beyond).
+  // epilogue warpgroup (measured: a gain only up to K = 512 at tile N = 256; 7-14 % slower beyond).  A problem of one
+  // 256-wide tile per CTA has nothing to hide its epilogue behind: there too eight warps drain the accumulator
+  // (2048^3: 19.6 -> 18.0 us; narrower tiles measured slower with them).
   const int kblk = kblk_of(d.ab_dtype);
-  const int epi_wg = (!single_wave && static_cast<long long>(ceil_div(d.K, kblk)) * 2 * bn <= 4096) ? 2 : 1;
+  const int epi_wg = ((!single_wave && static_cast<long long>(ceil_div(d.K, kblk)) * 2 * bn <= 4096) || (single_wave && bn == 256)) ? 2 : 1;
   int atoms = forced_atoms;
   if (atoms == 0) {
     const bool fits3 = 3 * 2 * (a_atom + b_atom) + dense_smem_bytes(0, 0, 0, epi_wg) <= kMaxSmemOptin;
