@@ -341,6 +341,34 @@ def test_runs_on_a_side_stream():
     plan.close()
 
 
+def test_one_dense_plan_on_two_streams_and_stream_k_plans_per_stream():
+    """Runs of one dense plan may overlap on the GPU (they share nothing but the status word); stream-K plans share
+    their arrival counters between runs, so concurrent streams get one plan each."""
+    wd = int_workload("two_streams_dense", 1024, 1024, 512, cd=wl.BF16)
+    ws = int_workload("two_streams_stream_k", 8, 4096, 4096, beta=0.0)
+    streams = [torch.cuda.Stream() for _ in range(2)]
+    for w, plans in ((wd, None), (ws, "per stream")):
+        inputs = wl.make_inputs(w)
+        A, B = H.to_device(inputs["A"], w.ab_dtype), H.to_device(inputs["B"], w.ab_dtype)
+        outs = [torch.empty(w.elems_c(), dtype=H._TORCH_DT[w.c_dtype], device="cuda") for _ in streams]
+        shared = bg.Plan(H.desc_of(w))
+        per = [shared, shared] if plans is None else [shared, bg.Plan(H.desc_of(w))]
+        wss = [pl.workspace_bytes and torch.empty(pl.workspace_bytes, dtype=torch.uint8, device="cuda") for pl in per]
+        torch.cuda.synchronize()
+        for rep in range(4):                       # interleaved launches: the kernels of the two streams overlap
+            for st, pl, out, wsb in zip(streams, per, outs, wss):
+                with torch.cuda.stream(st):
+                    pl.run(A, B, out, workspace=wsb if pl.workspace_bytes else None)
+        torch.cuda.synchronize()
+        for pl in set(per):
+            assert pl.status() == bg.OK
+        for out in outs:
+            reports = H.check_blocks(w, inputs, H.to_host_bits(out, w.c_dtype), H.default_blocks(w))
+            assert all(r["bit_identical"] == 1.0 for r in reports)
+        for pl in set(per):
+            pl.close()
+
+
 @pytest.mark.parametrize("variant", [V1, V2, VW, VS])
 def test_bounded_wait_reports_timeout_and_context_survives(variant):
     """A producer arrival is withheld by a test flag, so a device-side wait runs into its limit; the
