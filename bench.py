@@ -179,14 +179,19 @@ class DeviceCase:
     def time_steps(self, steps: int, warmup: int) -> float:
         """Seconds per step over `steps` back-to-back steps (CUDA events on the launching stream)."""
         torch = self.torch
-        t_warm = time.perf_counter()
         for _ in range(warmup):
             self.step()
         torch.cuda.synchronize()
-        # a configuration whose launches take microseconds would otherwise be timed while the clocks are still
-        # ramping up from idle: such a one keeps warming up (untimed) until 30 ms have passed
-        short_steps = (time.perf_counter() - t_warm) / warmup < 100e-6
-        while short_steps and time.perf_counter() - t_warm < 0.03:
+        # A configuration whose whole timed region lasts well under a millisecond would otherwise be measured while the
+        # clocks are still ramping up from idle (the pause between configurations lets them drop): such a one keeps
+        # warming up, untimed, until 30 ms have passed.  (The first launches carry one-off costs, so the step time is
+        # estimated from a second small batch.)
+        t_warm = time.perf_counter()
+        for _ in range(8):
+            self.step()
+        torch.cuda.synchronize()
+        short_region = (time.perf_counter() - t_warm) / 8 * steps < 0.03
+        while short_region and time.perf_counter() - t_warm < 0.03:
             for _ in range(16):
                 self.step()
             torch.cuda.synchronize()

@@ -54,6 +54,11 @@ struct DenseParams {
   int ab_fp8;                             // operands are 8-bit floats (tcgen05 kind::f8f6f4), else 16-bit (kind::f16)
   int kblk;                               // elements of K in one 128-byte slice: 64 (16-bit operands) or 128 (8-bit)
   int a_tri;                              // structure of op(A): 0 dense, 1 lower triangular (zero for k > i), 2 upper (zero for k < i)
+  // Tail split (kernels built with kSplit): the tiles from split_first_tile on, which would leave most CTAs idle in
+  // the last wave, are cut into `split` slices of K each, one work item per slice; num_items counts whole tiles + slices.
+  int split, split_first_tile, num_items;
+  float* partials;                        // workspace: raw fp32 accumulators of slices 1..split-1, [tile][rank][slice-1][128][bn]
+  uint32_t* split_flags;                  // one word per such partial: 1 = written (reset to 0 by the reducing CTA)
   float alpha, beta;
   const float* bias;
   const void* c_in;                       // = D buffer; read when beta != 0
@@ -162,6 +167,53 @@ __device__ __forceinline__ KRange k_range(const DenseParams& p, int row0, int ro
   if (p.a_tri == 1) r.hi = min(p.num_kb, (min(row0 + rows, p.M) - 1) / kstep + 1);
   else if (p.a_tri == 2) r.lo = min(row0 / kstep, p.num_kb - 1);
   return r;
+}
+
+// A work item of a CTA (pair): a whole tile (slice = -1) or one K slice of a split tile, with the ring stages it covers.
+struct WorkItem {
+  int tile, slice;
+  KRange kr;
+};
+template <bool kSplit>
+__device__ __forceinline__ int item_tile(const DenseParams& p, int item) {
+  if (!kSplit || item < p.split_first_tile) return item;
+  return p.split_first_tile + (item - p.split_first_tile) / p.split;
+}
+template <bool kSplit>
+__device__ __forceinline__ WorkItem work_item(const DenseParams& p, int item, int tile, int row0, int rows) {
+  WorkItem wi{tile, -1, k_range(p, row0, rows)};
+  if (kSplit && item >= p.split_first_tile) {
+    wi.slice = (item - p.split_first_tile) - (tile - p.split_first_tile) * p.split;
+    wi.kr.lo = wi.slice * p.num_kb / p.split;
+    wi.kr.hi = (wi.slice + 1) * p.num_kb / p.split;
+  }
+  return wi;
+}
+// Bounded wait for a flag word another CTA of this launch sets (all CTAs of these persistent kernels are resident,
+// and the CTA that sets the flag never waits for anybody).  Warp-uniform; false = gave up (timeout or abort elsewhere).
+__device__ __noinline__ bool flag_wait_warp(const uint32_t* flag, const WaitCtx& w, uint32_t code) {
+  const uint64_t t0 = globaltimer_ns();
+  uint32_t it = 0;
+  while (true) {
+    uint32_t v = 0;
+    if (lane_id() == 0) v = ld_acquire_gpu(flag);
+    if (__shfl_sync(0xffffffffu, v, 0) != 0u) return true;
+    __nanosleep(64);
+    if ((++it & 31u) == 0u) {
+      bool give_up = false;
+      if (lane_id() == 0) {
+        if (*w.s_abort || *reinterpret_cast<volatile uint32_t*>(w.g_status) != 0u) {
+          *w.s_abort = 1u;
+          give_up = true;
+        } else if (globaltimer_ns() - t0 > w.timeout_ns) {
+          *w.s_abort = 1u;
+          atomicCAS(w.g_status, 0u, kStatusTimeout | code);
+          give_up = true;
+        }
+      }
+      if (__any_sync(0xffffffffu, give_up)) return false;
+    }
+  }
 }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -323,7 +375,7 @@ __device__ __forceinline__ void epilogue_math(float (&v)[32], const uint32_t (&a
 // Both single-issuer roles are run by a whole warp in uniform control flow; only the instructions that
 // must be issued once (TMA, tcgen05.mma, commits, barrier arrivals) sit under elect_one().  That keeps
 // addresses, descriptors and coordinates in uniform registers, which is what those instructions read.
-template <int CG>
+template <int CG, bool kSplit = false>
 __device__ __forceinline__ void producer_role(const DenseParams& p, const CUtensorMap* tmA, const CUtensorMap* tmB,
                                               uint32_t tiles_base, uint32_t full0, uint32_t empty0, uint32_t cta_rank,
                                               int cluster_id, int num_clusters, const WaitCtx& w) {
@@ -337,14 +389,16 @@ __device__ __forceinline__ void producer_role(const DenseParams& p, const CUtens
   const uint64_t pol_b = p.l2_hint_b == 2 ? l2_policy_evict_last() : (p.l2_hint_b == 1 ? l2_policy_evict_first() : l2_policy_evict_normal());
   const int kstep = p.kblk * p.atoms;
   uint32_t it = 0;
-  for (int tile = cluster_id; tile < p.num_tiles; tile += num_clusters, ++it) {
+  const int n_items = kSplit ? p.num_items : p.num_tiles;
+  for (int item = cluster_id; item < n_items; item += num_clusters, ++it) {
+    const int tile = item_tile<kSplit>(p, item);
     const TileCoord tc = decode_tile(tile, p.tiles_m, p.tiles_n, p.raster_group);
     const int m0 = tc.tm * (kCtaM * CG) + static_cast<int>(cta_rank) * kCtaM;
     const int n0 = tc.tn * p.bn + (CG == 2 ? static_cast<int>(cta_rank) * p.b_rows : 0);
     // Serpentine K: all CTAs advance through K roughly in step, so the K range a wave touched last is what L2
     // still holds when the next wave starts; walking it backwards re-uses those lines of the shared A band.
     const bool rev = p.k_serpentine && (it & 1u);
-    const KRange kr = k_range(p, tc.tm * (kCtaM * CG), kCtaM * CG);
+    const KRange kr = work_item<kSplit>(p, item, tile, tc.tm * (kCtaM * CG), kCtaM * CG).kr;
     int k0 = rev ? (kr.hi - 1) * kstep : kr.lo * kstep;
     const int dk = rev ? -kstep : kstep;
     for (int kb = kr.lo; kb < kr.hi; ++kb, k0 += dk) {
@@ -388,7 +442,7 @@ __device__ __forceinline__ void producer_role(const DenseParams& p, const CUtens
   }
 }
 
-template <int CG>
+template <int CG, bool kSplit = false>
 __device__ __forceinline__ void mma_role(const DenseParams& p, uint32_t tiles_base, uint32_t full0, uint32_t empty0,
                                          uint32_t tfull0, uint32_t tempty0, uint32_t tmem_base, int cluster_id,
                                          int num_clusters, const WaitCtx& w) {
@@ -404,7 +458,9 @@ __device__ __forceinline__ void mma_role(const DenseParams& p, uint32_t tiles_ba
   const int last_atoms = (p.K - (num_kb - 1) * p.kblk * p.atoms + p.kblk - 1) / p.kblk;
   uint32_t s = 0, ph = 0, it = 0;
   uint64_t adesc = adesc0, bdesc = bdesc0;
-  for (int tile = cluster_id; tile < p.num_tiles; tile += num_clusters, ++it) {
+  const int n_items = kSplit ? p.num_items : p.num_tiles;
+  for (int item = cluster_id; item < n_items; item += num_clusters, ++it) {
+    const int tile = item_tile<kSplit>(p, item);
     const uint32_t buf = it & 1u;
     const uint32_t aph = (it >> 1) & 1u;
     if (!mbar_wait_warp(tempty0 + 8u * buf, aph ^ 1u, w, (2u << 8) | 0x80u | buf)) return;
@@ -412,7 +468,8 @@ __device__ __forceinline__ void mma_role(const DenseParams& p, uint32_t tiles_ba
     const uint32_t d_tmem = tmem_base + buf * static_cast<uint32_t>(p.bn);
     const bool rev = p.k_serpentine && (it & 1u);
     KRange kr{0, num_kb};
-    if (p.a_tri != 0) kr = k_range(p, decode_tile(tile, p.tiles_m, p.tiles_n, p.raster_group).tm * (kCtaM * CG), kCtaM * CG);
+    if (p.a_tri != 0 || (kSplit && item >= p.split_first_tile))
+      kr = work_item<kSplit>(p, item, tile, decode_tile(tile, p.tiles_m, p.tiles_n, p.raster_group).tm * (kCtaM * CG), kCtaM * CG).kr;
     const int n_kb = kr.hi - kr.lo;
     for (int kb = 0; kb < n_kb; ++kb) {
       if (!mbar_wait_warp(full0 + 8u * s, ph, w, (2u << 8) | s)) return;
@@ -461,7 +518,28 @@ __device__ __forceinline__ void mma_role(const DenseParams& p, uint32_t tiles_ba
   }
 }
 
-template <int CG, int EPI_WG>
+// Partial tiles travel through the workspace in the order the epilogue threads hold them, not row-major: the 32
+// accumulator columns of TMEM lane quarter q, column group g are eight 512-byte rows, one float4 per lane, so that
+// every warp-wide store and load is one contiguous 512-byte access.  Offset (in float4) of row j of group (q, g):
+__device__ __forceinline__ size_t partial_f4(uint32_t q, int g, int groups, int j) {
+  return (static_cast<size_t>(q) * groups + g) * 256 + static_cast<size_t>(j) * 32;
+}
+// Fetch the eight float4 of one (q, g) group of one partial tile (issued together: one round trip to L2).
+__device__ __forceinline__ void load_partial(float4 (&v)[8], const float4* tile, uint32_t q, int g, int groups, uint32_t lane) {
+#pragma unroll
+  for (int j = 0; j < 8; ++j) v[j] = __ldcg(tile + partial_f4(q, g, groups, j) + lane);
+}
+__device__ __forceinline__ void add_partial(uint32_t (&acc)[32], const float4 (&v)[8]) {
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    acc[4 * j + 0] = __float_as_uint(__uint_as_float(acc[4 * j + 0]) + v[j].x);
+    acc[4 * j + 1] = __float_as_uint(__uint_as_float(acc[4 * j + 1]) + v[j].y);
+    acc[4 * j + 2] = __float_as_uint(__uint_as_float(acc[4 * j + 2]) + v[j].z);
+    acc[4 * j + 3] = __float_as_uint(__uint_as_float(acc[4 * j + 3]) + v[j].w);
+  }
+}
+
+template <int CG, int EPI_WG, bool kSplit = false>
 __device__ __forceinline__ void epilogue_role(const DenseParams& p, const CUtensorMap* tmD, uint32_t staging, uint32_t tfull0,
                                               uint32_t tempty0, uint32_t tmem_base, uint32_t cta_rank, int cluster_id,
                                               int num_clusters, const WaitCtx& w) {
@@ -474,12 +552,54 @@ __device__ __forceinline__ void epilogue_role(const DenseParams& p, const CUtens
   const int slab_cols = (p.out_dtype == 2) ? 32 : 64;
   const int nslabs = p.bn / slab_cols;
   uint32_t it = 0, nstore = 0;
-  for (int tile = cluster_id; tile < p.num_tiles; tile += num_clusters, ++it) {
+  const int n_items = kSplit ? p.num_items : p.num_tiles;
+  const size_t partial_elems = static_cast<size_t>(kCtaM) * p.bn;
+  for (int item = cluster_id; item < n_items; item += num_clusters, ++it) {
+    const int tile = item_tile<kSplit>(p, item);
     const TileCoord tc = decode_tile(tile, p.tiles_m, p.tiles_n, p.raster_group);
     const uint32_t buf = it & 1u;
     const uint32_t ph = (it >> 1) & 1u;
     if (!mbar_wait_warp(tfull0 + 8u * buf, ph, w, (3u << 8) | buf, 64u)) return;  // whole warp leaves the wait together
     tc_fence_after();
+    // split tile: slice `slice` of `p.split`; the partials of slices 1.. live at part0, flags at flag0
+    int slice = -1;
+    float* part0 = nullptr;
+    uint32_t* flag0 = nullptr;
+    if (kSplit && item >= p.split_first_tile) {
+      slice = (item - p.split_first_tile) - (tile - p.split_first_tile) * p.split;
+      const size_t first = (static_cast<size_t>(tile - p.split_first_tile) * CG + cta_rank) * (p.split - 1);
+      part0 = p.partials + first * partial_elems;
+      flag0 = p.split_flags + first;
+    }
+    if (kSplit && slice > 0) {
+      // contributor: the raw accumulators go to the workspace, 32 columns at a time, then the flag is raised
+      const uint32_t t_rowc = tmem_base + ((q * 32u) << 16) + buf * static_cast<uint32_t>(p.bn);
+      float4* dst = reinterpret_cast<float4*>(part0 + static_cast<size_t>(slice - 1) * partial_elems);
+      const int groups = p.bn / 32;
+      for (int g = static_cast<int>(wg); g < p.bn / 32; g += EPI_WG) {
+        uint32_t acc[32];
+        tmem_ld_32x32(t_rowc + static_cast<uint32_t>(g * 32), acc);
+        tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          __stcg(dst + partial_f4(q, g, groups, j) + lane, make_float4(__uint_as_float(acc[4 * j]), __uint_as_float(acc[4 * j + 1]), __uint_as_float(acc[4 * j + 2]),
+                                     __uint_as_float(acc[4 * j + 3])));
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) {
+        if constexpr (CG == 1) mbar_arrive(tempty0 + 8u * buf);
+        else mbar_arrive_cluster(mapa(tempty0 + 8u * buf, 0));
+      }
+      // the barrier orders every epilogue warp's stores before the one releasing increment of the flag
+      named_barrier_sync(2, 128 * EPI_WG);
+      if (ew == 0 && lane == 0) (void)atom_add_acq_rel_gpu(flag0 + (slice - 1), 1u);
+      continue;
+    }
+    if (kSplit && slice == 0) {  // reducer: the other slices of this tile run in the same wave; wait for their partials
+      for (int sidx = 0; sidx < p.split - 1; ++sidx)
+        if (!flag_wait_warp(flag0 + sidx, w, (3u << 8) | 0x40u | static_cast<uint32_t>(sidx))) return;
+    }
     const int row0 = tc.tm * (kCtaM * CG) + static_cast<int>(cta_rank) * kCtaM + static_cast<int>(q) * 32;
     const long long row = row0 + static_cast<int>(lane);
     const uint32_t t_row = tmem_base + ((q * 32u) << 16) + buf * static_cast<uint32_t>(p.bn);
@@ -494,7 +614,18 @@ __device__ __forceinline__ void epilogue_role(const DenseParams& p, const CUtens
       float v[32];
       if (p.out_dtype == 2) {
         tmem_ld_32x32(t_row + static_cast<uint32_t>(sl * 32), acc);
-        tmem_ld_wait();
+        if (kSplit && slice == 0) {  // the partials are requested while the tensor-memory read is in flight
+          float4 pv[8];
+          load_partial(pv, reinterpret_cast<const float4*>(part0), q, sl, p.bn / 32, lane);
+          tmem_ld_wait();
+          add_partial(acc, pv);
+          for (int sidx = 1; sidx < p.split - 1; ++sidx) {  // further slices, in slice order
+            load_partial(pv, reinterpret_cast<const float4*>(part0 + sidx * partial_elems), q, sl, p.bn / 32, lane);
+            add_partial(acc, pv);
+          }
+        } else {
+          tmem_ld_wait();
+        }
         epilogue_math(v, acc, p, row, col0, tc.batch);
 #pragma unroll
         for (int j = 0; j < 8; ++j)
@@ -505,7 +636,22 @@ __device__ __forceinline__ void epilogue_role(const DenseParams& p, const CUtens
         uint32_t acc1[32];
         tmem_ld_32x32(t_row + static_cast<uint32_t>(sl * 64), acc);
         tmem_ld_32x32(t_row + static_cast<uint32_t>(sl * 64 + 32), acc1);
-        tmem_ld_wait();
+        if (kSplit && slice == 0) {
+          float4 pv[8], pv1[8];
+          load_partial(pv, reinterpret_cast<const float4*>(part0), q, 2 * sl, p.bn / 32, lane);
+          load_partial(pv1, reinterpret_cast<const float4*>(part0), q, 2 * sl + 1, p.bn / 32, lane);
+          tmem_ld_wait();
+          add_partial(acc, pv);
+          add_partial(acc1, pv1);
+          for (int sidx = 1; sidx < p.split - 1; ++sidx) {
+            load_partial(pv, reinterpret_cast<const float4*>(part0 + sidx * partial_elems), q, 2 * sl, p.bn / 32, lane);
+            load_partial(pv1, reinterpret_cast<const float4*>(part0 + sidx * partial_elems), q, 2 * sl + 1, p.bn / 32, lane);
+            add_partial(acc, pv);
+            add_partial(acc1, pv1);
+          }
+        } else {
+          tmem_ld_wait();
+        }
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
           epilogue_math(v, h == 0 ? acc : acc1, p, row, col0 + h * 32, tc.batch);
@@ -537,11 +683,16 @@ __device__ __forceinline__ void epilogue_role(const DenseParams& p, const CUtens
       if constexpr (CG == 1) mbar_arrive(tempty0 + 8u * buf);
       else mbar_arrive_cluster(mapa(tempty0 + 8u * buf, 0));
     }
+    if (kSplit && slice == 0) {  // every epilogue warp has read the partials: lower the flags for the next launch
+      named_barrier_sync(2, 128 * EPI_WG);
+      if (ew == 0 && lane == 0)
+        for (int sidx = 0; sidx < p.split - 1; ++sidx) flag0[sidx] = 0u;
+    }
   }
   if (lane == 0) bulk_wait_group_read<0>();  // staging may be released; the writes themselves complete with the grid
 }
 
-template <int CG, int EPI_WG>
+template <int CG, int EPI_WG, bool kSplit = false>
 __global__ void __launch_bounds__(64 + 128 * EPI_WG, 1)
 dense_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                   const __grid_constant__ CUtensorMap tmD, const DenseParams p) {
@@ -596,11 +747,11 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   griddep_wait();  // barriers and tensor memory are set up; from here on global memory is read and written
 
   if (warp == 0) {
-    producer_role<CG>(p, &tmA, &tmB, base, full0, empty0, cta_rank, cluster_id, num_clusters, w);
+    producer_role<CG, kSplit>(p, &tmA, &tmB, base, full0, empty0, cta_rank, cluster_id, num_clusters, w);
   } else if (warp == 1) {
-    if (cta_rank == 0) mma_role<CG>(p, base, full0, empty0, tfull0, tempty0, tmem_base, cluster_id, num_clusters, w);
+    if (cta_rank == 0) mma_role<CG, kSplit>(p, base, full0, empty0, tfull0, tempty0, tmem_base, cluster_id, num_clusters, w);
   } else {
-    epilogue_role<CG, EPI_WG>(p, &tmD, base + staging_off, tfull0, tempty0, tmem_base, cta_rank, cluster_id, num_clusters, w);
+    epilogue_role<CG, EPI_WG, kSplit>(p, &tmD, base + staging_off, tfull0, tempty0, tmem_base, cta_rank, cluster_id, num_clusters, w);
   }
 
   tc_fence_before();

@@ -112,7 +112,9 @@ struct gemm_plan_s {
   bool has_device;
   bool arch_ok;
   uint32_t* d_status;       // device: 16-byte status word, followed (256 bytes on) by the stream-K arrival counters
-  size_t d_counters_bytes = 0;  // 0 unless the plan is a stream-K plan
+  size_t d_counters_bytes = 0;  // plan-owned words after the status word: stream-K arrival counters or tail-split flags
+  int split = 1;                // tail split factor of a dense plan
+  size_t split_flag_bytes = 0;
   unsigned long long runs = 0;  // launches so far (the timeout test hook acts on the first one only)
   uint32_t timeout_ms;
   DenseParams dense;     // filled at plan time except pointers / scalars
@@ -160,6 +162,19 @@ int dense_smem_bytes(int stages, int a_stage, int b_stage, int epi_wg) {  // a_s
   return 1024 /*alignment slack*/ + stages * (a_stage + b_stage) + 4 * epi_wg * 2 * kSlabBytes + 16 * kMaxStages + 64;
 }
 
+// Tail split of the double-buffered dense kernels (on request, GEMM_FLAG_TAIL_SPLIT): when the tiles left over after the
+// full waves occupy at most half of the CTAs (pairs), each of them is cut into this many K slices, one per CTA (pair); the slice that
+// starts at K = 0 adds the others' raw accumulators from the workspace and finishes the tile.  1 = no split.
+int tail_split(long long tiles, int units, int num_kb, const gemm_desc_t& d) {
+  if (!(d.flags & GEMM_FLAG_TAIL_SPLIT) || (d.flags & (GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER))) return 1;
+  const long long rem = tiles % units;
+  if (rem == 0 || rem * 2 > units) return 1;
+  if (tiles / units >= 8) return 1;  // many full waves: the last one is a few per cent at most; keep the plain kernel
+  int split = static_cast<int>(std::min<long long>(units / rem, 2));  // more slices cost the reducing CTA one pass over a partial tile each
+  split = std::min(split, num_kb / 4);  // a slice of fewer than four ring stages is all pipeline fill
+  return std::max(split, 1);
+}
+
 // Plan-time roofline estimate (Section 4.3 applied per kernel candidate): cycles one SM spends on its share of the
 // problem with a given kernel family and tile width.  Per tile the slowest of three resources decides -- the tensor
 // pipe (with the family's measured streaming efficiency), the L2 -> SM operand feed and the HBM write share -- plus
@@ -176,8 +191,12 @@ double estimate_dense_cycles(const gemm_desc_t& d, int sm_count, int variant, in
   const int rows_tile = rows_cta * cg;
   const int units = std::max(1, sm_count / cg);
   const long long tiles = static_cast<long long>(ceil_div(d.M, rows_tile)) * ceil_div(d.N, bn) * d.batch_count;
-  const long long waves = (tiles + units - 1) / units;
   const double kblocks = static_cast<double>(ceil_div(d.K, kblk_of(d.ab_dtype)));  // 128-byte slices: same pipe time for either width
+  double waves = static_cast<double>((tiles + units - 1) / units);
+  if (!wide) {  // a thinly filled last wave is split along K (two slices per stage assumed, as plan_dense will choose for long K)
+    const int split = tail_split(tiles, units, static_cast<int>(kblocks) / 2, d);
+    if (split > 1) waves += 1.0 / split - 1.0 + 0.08;  // + hand-over of the partial accumulators
+  }
   // tensor pipe: one 128 x bn x 16 MMA per CTA takes bn / 2 cycles; four per k-block and 128-row half
   static const double eff1[3] = {0.45, 0.68, 0.82}, eff2[3] = {0.55, 0.80, 0.938};  // bn = 64, 128, 256 (measured: 8192^3, and K = 512 ... 4096)
   const int bi = bn <= 64 ? 0 : (bn <= 128 ? 1 : 2);
@@ -199,7 +218,7 @@ double estimate_dense_cycles(const gemm_desc_t& d, int sm_count, int variant, in
   // what is exposed stalls the tensor pipe, so it adds to the compute side; an output-bound tile instead pays a small
   // switch-over per tile (measured on the batched short-K shape: fewer, larger tiles win)
   const double per_tile = std::max(std::max(mma, feed) + exposed, out + 300.0);
-  return static_cast<double>(waves) * per_tile + 3000.0;  // + pipeline fill and drain
+  return waves * per_tile + 3000.0;  // + pipeline fill and drain
 }
 
 // Fill plan->dense and the launch geometry for a dense variant.
@@ -334,10 +353,20 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   info.cluster_size = cg;
   info.grid = pl->grid;
   info.raster_group = raster;
-  info.split = 1;
+  const int units_i = pl->sm_count / cg;
+  const int split = tail_split(num_tiles, units_i, p.num_kb, d);
+  const long long rem = num_tiles % units_i;
+  p.split = split;
+  p.split_first_tile = static_cast<int>(split > 1 ? num_tiles - rem : num_tiles);
+  p.num_items = static_cast<int>(split > 1 ? num_tiles - rem + rem * split : num_tiles);
+  pl->split = split;
+  pl->split_flag_bytes = split > 1 ? (static_cast<size_t>(rem) * cg * (split - 1) * 4 + 255) / 256 * 256 : 0;
+  if (split > 1) pl->grid = static_cast<int>(std::min<long long>(p.num_items, units_i)) * cg;
+  info.grid = pl->grid;
+  info.split = split;
   info.smem_bytes = smem;
   info.num_tiles = num_tiles;
-  info.workspace_bytes = 0;
+  info.workspace_bytes = split > 1 ? static_cast<size_t>(rem) * cg * (split - 1) * kCtaM * bn * 4 : 0;
   return GEMM_OK;
 }
 
@@ -553,7 +582,7 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
   }
   if (pl->has_device && pl->arch_ok) {
     // the counters start at zero here and every run leaves them at zero again (gemm_plan_status cleans up after a timeout)
-    pl->d_counters_bytes = pl->variant == GEMM_VARIANT_SKINNY_STREAMK ? pl->skinny.counters_bytes : 0;
+    pl->d_counters_bytes = pl->variant == GEMM_VARIANT_SKINNY_STREAMK ? pl->skinny.counters_bytes : pl->split_flag_bytes;
     const size_t dev_bytes = pl->d_counters_bytes ? 256 + pl->d_counters_bytes : 16;
     if (cudaMalloc(&pl->d_status, dev_bytes) != cudaSuccess || cudaMemset(pl->d_status, 0, dev_bytes) != cudaSuccess) {
       note_cuda_error("cudaMalloc(status word)", cudaGetErrorName(cudaGetLastError()));
@@ -641,11 +670,12 @@ const char* gemm_last_cuda_error(void) { return g_last_cuda_error; }
 
 namespace {
 
-template <int CG, int EPI_WG>
+template <int CG, int EPI_WG, bool kSplit>
 gemm_status_t launch_dense(const gemm_plan_s* pl, const CUtensorMap& tA, const CUtensorMap& tB, const CUtensorMap& tD,
                            const DenseParams& p, cudaStream_t stream) {
-  auto kern = dense_gemm_kernel<CG, EPI_WG>;
-  constexpr KernelSlot slot = CG == 1 ? (EPI_WG == 1 ? kSlotDense11 : kSlotDense12) : (EPI_WG == 1 ? kSlotDense21 : kSlotDense22);
+  auto kern = dense_gemm_kernel<CG, EPI_WG, kSplit>;
+  constexpr KernelSlot slot = static_cast<KernelSlot>((CG == 1 ? (EPI_WG == 1 ? kSlotDense11 : kSlotDense12) : (EPI_WG == 1 ? kSlotDense21 : kSlotDense22)) +
+                                                      (kSplit ? kSlotDenseSplit11 - kSlotDense11 : 0));
   if (ensure_dynamic_smem(reinterpret_cast<const void*>(kern), slot, pl->device, pl->smem_bytes) != cudaSuccess) {
     note_cuda_error("cudaFuncSetAttribute", cudaGetErrorName(cudaGetLastError()));
     return GEMM_ERR_CUDA;
@@ -707,7 +737,7 @@ gemm_status_t launch_wide(const gemm_plan_s* pl, const CUtensorMap& tA, const CU
 }
 
 gemm_status_t run_dense(gemm_plan_s* pl, const void* A, const void* B, void* C, const float* bias, float alpha, float beta,
-                        cudaStream_t stream, bool stall) {
+                        void* workspace, cudaStream_t stream, bool stall) {
   const gemm_desc_t& d = pl->d;
   DenseParams p = pl->dense;
   CUtensorMap tA, tB, tD;
@@ -729,8 +759,14 @@ gemm_status_t run_dense(gemm_plan_s* pl, const void* A, const void* B, void* C, 
   p.status = pl->d_status;
   p.timeout_ns = static_cast<unsigned long long>(pl->timeout_ms) * 1000000ull;
   if (pl->variant == GEMM_VARIANT_DENSE_2CTA_WIDE) return launch_wide(pl, tA, tB, tD, p, stream);
-  if (pl->cg == 1) return pl->epi_wg == 2 ? launch_dense<1, 2>(pl, tA, tB, tD, p, stream) : launch_dense<1, 1>(pl, tA, tB, tD, p, stream);
-  return pl->epi_wg == 2 ? launch_dense<2, 2>(pl, tA, tB, tD, p, stream) : launch_dense<2, 1>(pl, tA, tB, tD, p, stream);
+  if (pl->split > 1) {
+    p.partials = static_cast<float*>(workspace);
+    p.split_flags = reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(pl->d_status) + 256);
+    if (pl->cg == 1) return pl->epi_wg == 2 ? launch_dense<1, 2, true>(pl, tA, tB, tD, p, stream) : launch_dense<1, 1, true>(pl, tA, tB, tD, p, stream);
+    return pl->epi_wg == 2 ? launch_dense<2, 2, true>(pl, tA, tB, tD, p, stream) : launch_dense<2, 1, true>(pl, tA, tB, tD, p, stream);
+  }
+  if (pl->cg == 1) return pl->epi_wg == 2 ? launch_dense<1, 2, false>(pl, tA, tB, tD, p, stream) : launch_dense<1, 1, false>(pl, tA, tB, tD, p, stream);
+  return pl->epi_wg == 2 ? launch_dense<2, 2, false>(pl, tA, tB, tD, p, stream) : launch_dense<2, 1, false>(pl, tA, tB, tD, p, stream);
 }
 
 gemm_status_t run_skinny(gemm_plan_s* pl, const void* A, const void* B, void* C, const float* bias, float alpha, float beta,
@@ -795,7 +831,7 @@ extern "C" gemm_status_t gemm_run(gemm_plan_t plan, const void* A, const void* B
   const bool stall = (plan->d.flags & GEMM_FLAG_DEBUG_STALL) && plan->runs == 0;  // test hook: the plan's first run only
   ++plan->runs;
   if (plan->variant == GEMM_VARIANT_SKINNY_STREAMK) return run_skinny(plan, A, B, C, bias, alpha, beta, workspace, s, stall);
-  return run_dense(plan, A, B, C, bias, alpha, beta, s, stall);
+  return run_dense(plan, A, B, C, bias, alpha, beta, workspace, s, stall);
 }
 
 // ---------------------------------------------------------------------------------------------------------

@@ -70,6 +70,7 @@ std::vector<uint32_t> second_round(uint32_t best, const gemm_info_t& w) {
     if (rg >= 1 && rg <= 64 && rg != w.raster_group)
       c.push_back((best & ~GEMM_FLAG_RASTER_MASK) | (static_cast<uint32_t>(rg) << GEMM_FLAG_RASTER_SHIFT));
   if (w.variant != GEMM_VARIANT_DENSE_2CTA_WIDE) {
+    c.push_back(best | GEMM_FLAG_TAIL_SPLIT);  // has an effect only where the last wave is thinly filled
     const int ks = w.tile_k / 64;  // 64-wide K slices per stage of the winner
     c.push_back((best & ~GEMM_FLAG_KSLICES_MASK) | (static_cast<uint32_t>(ks == 1 ? 2 : 1) << GEMM_FLAG_KSLICES_SHIFT));
   }
@@ -148,17 +149,22 @@ extern "C" void gemm_tune_cache_clear(void) {
 }
 
 extern "C" size_t gemm_tune_workspace_bytes(const gemm_desc_t* desc) {
-  if (!desc || !short_extent(*desc)) return 0;
+  if (!desc) return 0;
   size_t need = 0;
-  for (int ks = 1; ks <= 3; ++ks) {  // only the stream-K candidates use a workspace
+  auto consider = [&](uint32_t f) {
     gemm_desc_t d = *desc;
-    d.flags = (d.flags & ~kTuningFlagMask) | pack(GEMM_VARIANT_SKINNY_STREAMK, 0, 0, 0, ks);
+    d.flags = (d.flags & ~kTuningFlagMask) | f;
     gemm_plan_t plan = nullptr;
-    if (gemm_plan(&d, &plan) != GEMM_OK) continue;
+    if (gemm_plan(&d, &plan) != GEMM_OK) return;
     const size_t b = gemm_workspace_bytes(plan);
     if (b > need) need = b;
     gemm_destroy(plan);
-  }
+  };
+  // the candidates that use a workspace: stream-K (partial tiles) and the dense kernels with a tail split (second slices)
+  if (short_extent(*desc))
+    for (int ks = 1; ks <= 3; ++ks) consider(pack(GEMM_VARIANT_SKINNY_STREAMK, 0, 0, 0, ks));
+  for (int v : {GEMM_VARIANT_DENSE_1CTA, GEMM_VARIANT_DENSE_2CTA})
+    for (int bn : {256, 128, 64}) consider(pack(v, bn, 0, 0, 0) | GEMM_FLAG_TAIL_SPLIT);
   return need;
 }
 

@@ -127,6 +127,17 @@ EXACT_CASES = [
     ("fp8_e5m2_stream_k_tall_bias", 1000, 33, 1040, dict(ab=wl.FP8_E5M2, cd=wl.BF16, epi=bg.EPI_BIAS, ldc=40), dict(variant=VS)),
     ("fp8_e4m3_stream_k_one_slice", 16, 384, 2048, dict(ab=wl.FP8_E4M3), dict(variant=VS, kslices=1)),
     ("fp8_e4m3_stream_k_auto", 8, 4096, 4096, dict(ab=wl.FP8_E4M3), dict()),
+    # tail split: the tiles of a thinly filled last wave are cut into K slices whose raw accumulators meet in the workspace
+    ("tail_split_pair_few_tiles", 1024, 1024, 2048, dict(cd=wl.BF16), dict(variant=V2, tile_n=256, tail_split=True)),
+    ("tail_split_pair_after_full_wave", 2560, 2560, 1032, dict(beta=1.0, epi=bg.EPI_BIAS_RELU, cd=wl.BF16), dict(variant=V2, tile_n=256, tail_split=True)),
+    ("tail_split_pair_narrow_f32", 1024, 1200, 1024, dict(epi=bg.EPI_BIAS), dict(variant=V2, tile_n=128, tail_split=True)),
+    ("tail_split_1cta", 512, 512, 2048, dict(), dict(variant=V1, tile_n=128, tail_split=True)),
+    ("tail_split_1cta_ragged_f16", 1000, 1000, 1096, dict(ab=wl.F16, cd=wl.F16, beta=-1.0), dict(variant=V1, tile_n=256, tail_split=True)),
+    ("tail_split_1cta_two_epilogue_groups", 1280, 4096, 512, dict(cd=wl.BF16), dict(variant=V1, tile_n=256, tail_split=True)),
+    ("tail_split_nn_layout", 1024, 1024, 2048, dict(ta=0, tb=0), dict(variant=V2, tile_n=128, tail_split=True)),
+    ("tail_split_fp8", 1024, 1024, 4096, dict(ab=wl.FP8_E4M3, cd=wl.BF16), dict(variant=V2, tile_n=256, tail_split=True)),
+    ("tail_split_switched_off", 1024, 1024, 2048, dict(cd=wl.BF16), dict(variant=V2, tile_n=256)),
+    ("tail_split_requested_auto_plan", 2304, 2304, 2304, dict(cd=wl.BF16), dict(tail_split=True)),
     # mirrored stream-K: a tall output with a handful of columns (A is the streamed operand)
     ("tall_one_unit", 128, 8, 64, {}, dict(variant=VS)),
     ("tall_split_k", 256, 8, 4096, {}, dict(variant=VS)),
@@ -397,6 +408,24 @@ def test_bounded_wait_reports_timeout_and_context_survives(variant):
         assert all(r["bit_identical"] == 1.0 for r in reports)
     plan.close()
     H.check_workload(w, bg.make_flags(variant, tile_n), exact=True)
+
+
+def test_tail_split_plans():
+    """Which plans split, what they ask for, and that the flag switches it off."""
+    def info(M, N, K, **fl):
+        h = bg.gemm_plan(bg.make_desc(M, N, K, c_dtype=bg.BF16, flags=bg.make_flags(**fl)))
+        i = bg.gemm_plan_info(h)
+        bg.gemm_destroy(h)
+        return i
+    i = info(1024, 1024, 2048, variant=V2, tile_n=256, tail_split=True)     # 16 pair tiles on 74 pairs: two slices each
+    assert i["split"] == 2 and i["grid"] == 64 and i["workspace_bytes"] == 16 * 2 * 1 * 128 * 256 * 4
+    i = info(1024, 1024, 2048, variant=V2, tile_n=256)                      # not asked for: whole tiles, no workspace
+    assert i["split"] == 1 and i["workspace_bytes"] == 0
+    assert info(1024, 1024, 256, variant=V2, tile_n=256, tail_split=True)["split"] == 1      # too little K to slice
+    assert info(3072, 3072, 3072, variant=V2, tile_n=256, tail_split=True)["split"] == 1     # 144 tiles: the last wave is 70 of 74
+    i = info(2560, 2560, 2560, variant=V2, tile_n=256, tail_split=True)                      # 100 tiles: 74 + 26, the 26 in two slices
+    assert i["split"] == 2 and i["workspace_bytes"] == 26 * 2 * 1 * 128 * 256 * 4
+    assert info(16384, 14336, 4096, variant=V2, tile_n=256, tail_split=True)["split"] == 1   # 48 full waves: not worth it
 
 
 def test_triangular_a_really_skips():

@@ -186,7 +186,8 @@ def test_cost_model_choices_follow_the_measurements():
 
 def test_tuning_entry_points_on_the_host():
     # the workspace bound needs no device: only the stream-K candidates of a short-extent problem use one
-    assert bg.gemm_tune_workspace_bytes(bg.make_desc(1024, 1024, 512)) == 0
+    assert bg.gemm_tune_workspace_bytes(bg.make_desc(8192, 8192, 512)) == 0          # nothing to split, no short extent
+    assert bg.gemm_tune_workspace_bytes(bg.make_desc(1024, 1024, 4096)) > 0           # a tail-split candidate wants room
     need = bg.gemm_tune_workspace_bytes(bg.make_desc(8, 4096, 2048))
     assert need >= 148 * 2 * 128 * 16 * 4
     assert bg.gemm_tune_workspace_bytes(bg.make_desc(4096, 8, 2048)) == need      # mirrored
