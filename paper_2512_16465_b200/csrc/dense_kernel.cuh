@@ -736,18 +736,30 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     tmem_alloc<CG>(smem_addr(const_cast<uint32_t*>(tmem_slot)), p.tmem_cols);
     tmem_relinquish<CG>();
   }
-  tc_fence_before();
-  __syncthreads();
-  if constexpr (CG == 2) {  // the peer's barriers must exist before anything signals them
-    cluster_arrive();
-    cluster_wait();
+  uint32_t tmem_base = 0;
+  if (CG == 1 && warp == 0) {
+    // A single CTA's producer needs the barriers (set up by its own lane 0) and nothing else: it announces them to
+    // the other warps and starts the loads while those are still waiting for the tensor-memory allocation.
+    __syncwarp();
+    named_barrier_arrive(3, blockDim.x);
+    griddep_wait();  // from here on global memory is read
+    producer_role<CG, kSplit>(p, &tmA, &tmB, base, full0, empty0, cta_rank, cluster_id, num_clusters, w);
+  } else {
+    tc_fence_before();
+    if constexpr (CG == 1) {
+      named_barrier_sync(3, blockDim.x);
+    } else {
+      __syncthreads();
+      cluster_arrive();  // the peer's barriers must exist before anything signals them
+      cluster_wait();
+    }
+    tc_fence_after();
+    tmem_base = *tmem_slot;
+    griddep_wait();  // barriers and tensor memory are set up; from here on global memory is read and written
   }
-  tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
-  griddep_wait();  // barriers and tensor memory are set up; from here on global memory is read and written
 
   if (warp == 0) {
-    producer_role<CG, kSplit>(p, &tmA, &tmB, base, full0, empty0, cta_rank, cluster_id, num_clusters, w);
+    if constexpr (CG == 2) producer_role<CG, kSplit>(p, &tmA, &tmB, base, full0, empty0, cta_rank, cluster_id, num_clusters, w);
   } else if (warp == 1) {
     if (cta_rank == 0) mma_role<CG, kSplit>(p, base, full0, empty0, tfull0, tempty0, tmem_base, cluster_id, num_clusters, w);
   } else {
