@@ -251,11 +251,19 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
     tmem_alloc<1>(smem_addr(const_cast<uint32_t*>(tmem_slot)), tmem_cols);
     tmem_relinquish<1>();
   }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
-  griddep_wait();  // barriers and tensor memory are set up; from here on global memory is read and written
+  // The producer needs the barriers (set up by its own lane 0) and nothing else: it announces them to the other
+  // warps and starts streaming while those still wait for the tensor-memory allocation.
+  uint32_t tmem_base = 0;
+  if (warp == 0) {
+    __syncwarp();
+    named_barrier_arrive(3, kSkinnyThreads);
+  } else {
+    tc_fence_before();
+    named_barrier_sync(3, kSkinnyThreads);
+    tc_fence_after();
+    tmem_base = *tmem_slot;
+  }
+  griddep_wait();  // from here on global memory is read and written
   // An earlier run of this plan that timed out may have left arrival counters half counted; the status word stays
   // set until the host has read it (and cleaned the counters), and until then no run trusts them.  The load is
   // issued here and consumed only by the fix-up, long after it has landed.
