@@ -40,7 +40,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the full-size ncu captures
 # summarised under profiles/ (dense_*_cN_*.txt, skinny_streamk_c5_*.txt; last line of each file).
-NCU_TRAFFIC_BYTES = {"c1": 1125632, "c2": 872594176, "c3": 1642422576, "c4": 545477888, "c5": 477278464}
+NCU_TRAFFIC_BYTES = {"c1": 1119744, "c2": 872149760, "c3": 1647279136, "c4": 545198848, "c5": 476800768}
 
 
 def load_peaks():
