@@ -187,7 +187,9 @@ size_t gemm_workspace_bytes(gemm_plan_t plan);
  * that is 0).  Runs of one dense plan may overlap on the GPU; runs of one
  * stream-K plan must not (they share the plan's arrival counters, which every
  * run leaves at zero): order them on one stream or with events, or make one
- * plan per stream.  alpha and beta are host scalars.  Errors are returned before anything is launched:
+ * plan per stream.  alpha and beta are host scalars.  The call only encodes tensor maps on the
+ * host and launches: once a plan has run once (which sets kernel attributes), further runs may be recorded by stream
+ * capture into a CUDA graph (tested).  Errors are returned before anything is launched:
  * GEMM_ERR_NULL, GEMM_ERR_ALIGNMENT, GEMM_ERR_WORKSPACE, GEMM_ERR_ARCH,
  * GEMM_ERR_INVALID_ARG (the current CUDA device is not the one the plan was
  * made on), GEMM_ERR_CUDA (tensor-map encoding or launch failure).

@@ -352,6 +352,42 @@ def test_runs_on_a_side_stream():
     plan.close()
 
 
+def test_runs_are_capturable_in_a_cuda_graph():
+    """gemm_run only encodes tensor maps on the host and launches: after one ordinary run (which sets the kernel
+    attributes) a chain of a dense and a stream-K GEMM is captured into a CUDA graph and replayed with new inputs."""
+    w1 = int_workload("graph_dense", 512, 384, 256, cd=wl.BF16)
+    w2 = int_workload("graph_stream_k", 8, 512, 4096, beta=0.0)
+    cases = []
+    for w in (w1, w2):
+        inputs = wl.make_inputs(w)
+        plan = bg.Plan(H.desc_of(w))
+        A, B = H.to_device(inputs["A"], w.ab_dtype), H.to_device(inputs["B"], w.ab_dtype)
+        C = torch.zeros(w.elems_c(), dtype=H._TORCH_DT[w.c_dtype], device="cuda")
+        plan.run(A, B, C)                      # sets attributes, allocates the workspace
+        cases.append((w, inputs, plan, A, B, C))
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for _, _, plan, A, B, C in cases:
+            plan.run(A, B, C)
+    for seed_offset in (0, 1000):              # replay on the same buffers with fresh contents
+        fresh = []
+        for w, _, plan, A, B, C in cases:
+            inp = wl.make_inputs(w, seed_offset=seed_offset)
+            A.copy_(H.to_device(inp["A"], w.ab_dtype))
+            B.copy_(H.to_device(inp["B"], w.ab_dtype))
+            C.fill_(float("nan"))
+            fresh.append(inp)
+        g.replay()
+        torch.cuda.synchronize()
+        for (w, _, plan, A, B, C), inp in zip(cases, fresh):
+            assert plan.status() == bg.OK
+            reports = H.check_blocks(w, inp, H.to_host_bits(C, w.c_dtype), H.default_blocks(w))
+            assert all(r["bit_identical"] == 1.0 for r in reports)
+    for _, _, plan, *_ in cases:
+        plan.close()
+
+
 def test_one_dense_plan_on_two_streams_and_stream_k_plans_per_stream():
     """Runs of one dense plan may overlap on the GPU (they share nothing but the status word); stream-K plans share
     their arrival counters between runs, so concurrent streams get one plan each."""
