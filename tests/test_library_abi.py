@@ -197,3 +197,17 @@ def test_tuning_entry_points_on_the_host():
         with pytest.raises(bg.GemmError) as e:
             bg.gemm_tune(bg.make_desc(256, 256, 64), 16, 16, 16, 0, 1.0, 0.0, 0, 0, 0)
         assert e.value.status in (bg.ERR_ARCH, bg.ERR_CUDA)                       # no device: an error, never a fallback
+
+
+def test_host_pipeline_entry_points_without_a_device():
+    import torch
+    for kw in (dict(transa=bg.OP_T), dict(batch=2), dict(flags=bg.make_flags(a_upper=True))):   # refused before any device work
+        with pytest.raises(bg.GemmError) as e:
+            bg.gemm_host_create(bg.make_desc(256, 256, 256, **kw))
+        assert e.value.status == bg.ERR_UNSUPPORTED
+    assert bg.gemm_host_panels(0) == 0
+    bg.gemm_host_destroy(0)                                                      # NULL is accepted
+    if not torch.cuda.is_available():
+        with pytest.raises(bg.GemmError) as e:
+            bg.gemm_host_create(bg.make_desc(256, 256, 256))
+        assert e.value.status in (bg.ERR_ARCH, bg.ERR_CUDA)                      # an error, never a CPU fallback
