@@ -95,11 +95,12 @@ typedef enum {
 #define GEMM_FLAG_TILE_N_SHIFT 8           /* bits 8-12: force tile N / 16 (0 = automatic) */
 #define GEMM_FLAG_TILE_N_MASK 0x1F00u
 #define GEMM_FLAG_TAIL_SPLIT 0x2000u       /* when the last wave of a 1-CTA or pair plan would fill at most half of the SMs, cut
-                                              its tiles into two K slices, one per CTA or pair (the plan then wants a workspace
-                                              for the raw accumulators of the second slices).  Off by default: under the power
-                                              cap idle SMs lend their budget to the busy ones, so it pays only on small
-                                              problems (measured: -10 % at 1024 x 1024 x 4096, nothing at 4096^3);
-                                              gemm_tune tries it */
+                                              its tiles into K slices, one per CTA or pair (the plan then wants a workspace for
+                                              the raw accumulators of the further slices).  Without the flag this happens only
+                                              for a handful of tiles with a very long K (three or more slices each); otherwise
+                                              it is left to the caller and to gemm_tune: under the power cap idle SMs lend
+                                              their budget to the busy ones, so it pays only on small problems (measured:
+                                              -10 % at 1024 x 1024 x 4096, nothing at 4096^3) */
 #define GEMM_FLAG_RASTER_SHIFT 16          /* bits 16-22: force the raster group height in tiles (0 = automatic) */
 #define GEMM_FLAG_RASTER_MASK 0x7F0000u
 #define GEMM_FLAG_STAGES_SHIFT 24          /* bits 24-27: force the pipeline depth (0 = automatic) */

@@ -166,13 +166,21 @@ int dense_smem_bytes(int stages, int a_stage, int b_stage, int epi_wg) {  // a_s
 // full waves occupy at most half of the CTAs (pairs), each of them is cut into this many K slices, one per CTA (pair); the slice that
 // starts at K = 0 adds the others' raw accumulators from the workspace and finishes the tile.  1 = no split.
 int tail_split(long long tiles, int units, int num_kb, const gemm_desc_t& d) {
-  if (!(d.flags & GEMM_FLAG_TAIL_SPLIT) || (d.flags & (GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER))) return 1;
+  if (d.flags & (GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER)) return 1;
   const long long rem = tiles % units;
   if (rem == 0 || rem * 2 > units) return 1;
   if (tiles / units >= 8) return 1;  // many full waves: the last one is a few per cent at most; keep the plain kernel
-  int split = static_cast<int>(std::min<long long>(units / rem, 2));  // more slices cost the reducing CTA one pass over a partial tile each
+  // The reducing CTA reads one partial tile per further slice (about 5000 cycles each), a ring stage takes about 1000:
+  // beyond sqrt(stages / 5) slices the reading costs more than the shorter main loop saves.
+  int by_length = 2;
+  while ((by_length + 1) * (by_length + 1) * 5 <= num_kb && by_length < 16) ++by_length;
+  int split = static_cast<int>(std::min<long long>(units / rem, by_length));
   split = std::min(split, num_kb / 4);  // a slice of fewer than four ring stages is all pipeline fill
-  return std::max(split, 1);
+  split = std::max(split, 1);
+  // Without the flag only the extreme case splits by itself: a handful of tiles (no full wave) whose K is long enough for
+  // three or more slices each, where whole tiles would leave most of the GPU idle for the whole run.
+  if (!(d.flags & GEMM_FLAG_TAIL_SPLIT) && !(tiles < units && split >= 3)) return 1;
+  return split;
 }
 
 // Plan-time roofline estimate (Section 4.3 applied per kernel candidate): cycles one SM spends on its share of the

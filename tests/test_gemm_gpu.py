@@ -136,6 +136,9 @@ EXACT_CASES = [
     ("tail_split_1cta_two_epilogue_groups", 1280, 4096, 512, dict(cd=wl.BF16), dict(variant=V1, tile_n=256, tail_split=True)),
     ("tail_split_nn_layout", 1024, 1024, 2048, dict(ta=0, tb=0), dict(variant=V2, tile_n=128, tail_split=True)),
     ("tail_split_fp8", 1024, 1024, 4096, dict(ab=wl.FP8_E4M3, cd=wl.BF16), dict(variant=V2, tile_n=256, tail_split=True)),
+    ("tail_split_seven_slices_long_k", 512, 512, 16384, dict(cd=wl.BF16, epi=bg.EPI_BIAS), dict(variant=V2, tile_n=256)),
+    ("tail_split_1cta_three_slices", 256, 384, 8192 + 64, dict(beta=1.0), dict(variant=V1, tile_n=128, tail_split=True)),
+    ("tail_split_automatic_for_few_tiles", 300, 264, 32768, dict(), dict()),
     ("tail_split_switched_off", 1024, 1024, 2048, dict(cd=wl.BF16), dict(variant=V2, tile_n=256)),
     ("tail_split_requested_auto_plan", 2304, 2304, 2304, dict(cd=wl.BF16), dict(tail_split=True)),
     # mirrored stream-K: a tall output with a handful of columns (A is the streamed operand)
@@ -462,6 +465,8 @@ def test_tail_split_plans():
     i = info(2560, 2560, 2560, variant=V2, tile_n=256, tail_split=True)                      # 100 tiles: 74 + 26, the 26 in two slices
     assert i["split"] == 2 and i["workspace_bytes"] == 26 * 2 * 1 * 128 * 256 * 4
     assert info(16384, 14336, 4096, variant=V2, tile_n=256, tail_split=True)["split"] == 1   # 48 full waves: not worth it
+    i = info(512, 512, 16384, variant=V2, tile_n=256)                                      # 4 tiles, 256 ring stages each: by itself
+    assert i["split"] == 7 and i["grid"] == 56 and i["workspace_bytes"] == 4 * 2 * 6 * 128 * 256 * 4
 
 
 def test_triangular_a_really_skips():
