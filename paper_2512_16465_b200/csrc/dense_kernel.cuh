@@ -67,6 +67,7 @@ struct DenseParams {
   unsigned long long timeout_ns;
   uint32_t debug_flags;                   // bit 0: withhold one producer arrival (timeout test hook)
   int l2_hint_a, l2_hint_b;               // L2 eviction priority of operand loads: 0 normal, 1 evict-first, 2 evict-last
+  int l2_hint_d;                          // 1: output stores ask L2 to evict them first (a large D would push the operands out)
   int k_serpentine;                       // 1: every second tile of a CTA walks K from the far end back to 0
 };
 
@@ -672,7 +673,10 @@ __device__ __forceinline__ void epilogue_role(const DenseParams& p, const CUtens
       fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) {
-        if (row0 < p.M && col0 < p.N) tma_store_3d(tmD, sbuf, col0, row0, tc.batch);
+        if (row0 < p.M && col0 < p.N) {
+          if (p.l2_hint_d) tma_store_3d_hint(tmD, sbuf, col0, row0, tc.batch, l2_policy_evict_first());
+          else tma_store_3d(tmD, sbuf, col0, row0, tc.batch);
+        }
         bulk_commit_group();
       }
     }

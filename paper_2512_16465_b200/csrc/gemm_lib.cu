@@ -332,6 +332,9 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   p.out_dtype = d.c_dtype;
   p.epilogue = d.epilogue;
   p.bias_per_row = (d.flags & GEMM_FLAG_BIAS_PER_ROW) ? 1 : 0;
+  // an output much larger than half the L2 is written with evict-first priority so that it does not push the operands
+  // out (measured: +0.5 to +2.5 % on the 470 MB output of the projection shape, neutral on 134 MB)
+  p.l2_hint_d = static_cast<double>(d.M) * d.N * d.batch_count * elem_bytes(d.c_dtype) > 64.0e6 ? 1 : 0;
   p.a_tri = (d.flags & GEMM_FLAG_A_LOWER) ? 1 : ((d.flags & GEMM_FLAG_A_UPPER) ? 2 : 0);
   p.ldc = d.ldc;
   p.stride_c = d.batch_count > 1 ? d.stride_c : 0;
@@ -432,6 +435,9 @@ gemm_status_t plan_wide(gemm_plan_s* pl, int forced_raster, int forced_stages) {
   p.out_dtype = d.c_dtype;
   p.epilogue = d.epilogue;
   p.bias_per_row = (d.flags & GEMM_FLAG_BIAS_PER_ROW) ? 1 : 0;
+  // an output much larger than half the L2 is written with evict-first priority so that it does not push the operands
+  // out (measured: +0.5 to +2.5 % on the 470 MB output of the projection shape, neutral on 134 MB)
+  p.l2_hint_d = static_cast<double>(d.M) * d.N * d.batch_count * elem_bytes(d.c_dtype) > 64.0e6 ? 1 : 0;
   p.a_tri = (d.flags & GEMM_FLAG_A_LOWER) ? 1 : ((d.flags & GEMM_FLAG_A_UPPER) ? 2 : 0);
   p.ldc = d.ldc;
   p.stride_c = d.batch_count > 1 ? d.stride_c : 0;

@@ -255,7 +255,10 @@ __device__ __forceinline__ void wide_epilogue_role(const DenseParams& p, const C
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) {
-              if (row0 < p.M && col0 < p.N) tma_store_3d(tmD, sbuf, col0, row0, tc.batch);
+              if (row0 < p.M && col0 < p.N) {
+                if (p.l2_hint_d) tma_store_3d_hint(tmD, sbuf, col0, row0, tc.batch, l2_policy_evict_first());
+                else tma_store_3d(tmD, sbuf, col0, row0, tc.batch);
+              }
               bulk_commit_group();
             }
           }
@@ -305,7 +308,10 @@ __device__ __forceinline__ void wide_epilogue_role(const DenseParams& p, const C
           fence_proxy_async_smem();
           __syncwarp();
           if (lane == 0) {
-            if (row0 < p.M && col64 < p.N) tma_store_3d(tmD, sbuf, col64, row0, tc.batch);
+            if (row0 < p.M && col64 < p.N) {
+              if (p.l2_hint_d) tma_store_3d_hint(tmD, sbuf, col64, row0, tc.batch, l2_policy_evict_first());
+              else tma_store_3d(tmD, sbuf, col64, row0, tc.batch);
+            }
             bulk_commit_group();
           }
           ++nstore;
