@@ -842,8 +842,9 @@ extern "C" gemm_status_t gemm_run(gemm_plan_t plan, const void* A, const void* B
   int cur = -1;
   if (cudaGetDevice(&cur) != cudaSuccess || cur != plan->device) return GEMM_ERR_INVALID_ARG;  // plan belongs to another device
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const bool stall = (plan->d.flags & GEMM_FLAG_DEBUG_STALL) && plan->runs == 0;  // test hook: the plan's first run only
-  ++plan->runs;
+  // (atomic: a dense plan may be run from several host threads at once)
+  const unsigned long long run_index = __atomic_fetch_add(&plan->runs, 1ull, __ATOMIC_RELAXED);
+  const bool stall = (plan->d.flags & GEMM_FLAG_DEBUG_STALL) && run_index == 0;  // test hook: the plan's first run only
   if (plan->variant == GEMM_VARIANT_SKINNY_STREAMK) return run_skinny(plan, A, B, C, bias, alpha, beta, workspace, s, stall);
   return run_dense(plan, A, B, C, bias, alpha, beta, workspace, s, stall);
 }
