@@ -116,6 +116,14 @@ typedef enum {
  * of the two.  (The paper lists symmetric and triangular operands among its operator cases, Section 5.1.) */
 #define GEMM_FLAG_A_LOWER 0x2u
 #define GEMM_FLAG_A_UPPER 0x800000u
+/* Symmetric results (D = A * A^T and the like; the paper's symmetric operator case, Section 5.1): only one triangle
+ * of D is wanted.  With D_LOWER the elements with row >= column are computed, with D_UPPER those with row <= column;
+ * output tiles that lie wholly in the other triangle are neither computed nor written (nor read, when beta != 0).
+ * The tiles the diagonal crosses are computed in full, so an element outside the wanted triangle is either left
+ * untouched or holds its value of the plain GEMM.  About half the work for a square D.  1-CTA and pair variants
+ * only (not the wide pair tile, not stream-K); at most one of the two; combines with A_LOWER / A_UPPER and batches. */
+#define GEMM_FLAG_D_LOWER 0x4000u
+#define GEMM_FLAG_D_UPPER 0x8000u
 #define GEMM_FLAG_BIAS_PER_ROW 0x1u         /* the bias is fp32[M], one value per output row (default: fp32[N], one per
                                               column); not a tuning knob: it changes what is computed */
 #define GEMM_FLAG_NO_EARLY_LAUNCH 0x4u       /* launch without programmatic dependent launch (default: the kernel may be

@@ -129,6 +129,20 @@ def _ptr(a):
     return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
 
 
+def wanted(rows, cols, d_tri: int) -> np.ndarray:
+    """Which outputs the triangular forms of the product define (the paper's symmetric operator case, Section 5.1):
+    ``d_tri`` = 0 all of D, 1 the lower triangle (row >= column, diagonal included), 2 the upper (row <= column).
+    Boolean array ``[len(rows), len(cols)]``; a wanted element's value is that of the plain product."""
+    r = np.asarray(rows, np.int64)[:, None]
+    c = np.asarray(cols, np.int64)[None, :]
+    if d_tri == 1:
+        return r >= c
+    if d_tri == 2:
+        return r <= c
+    assert d_tri == 0
+    return np.ones((r.shape[0], c.shape[1]), dtype=bool)
+
+
 def gemm(p: Problem, A, B, C_in=None, bias=None, alpha=1.0, beta=0.0,
          batches=None, rows=None, cols=None, threads: int = 0):
     """Evaluate the definition on ``batches x rows x cols`` (default: everything).

@@ -54,6 +54,10 @@ struct DenseParams {
   int ab_fp8;                             // operands are 8-bit floats (tcgen05 kind::f8f6f4), else 16-bit (kind::f16)
   int kblk;                               // elements of K in one 128-byte slice: 64 (16-bit operands) or 128 (8-bit)
   int a_tri;                              // structure of op(A): 0 dense, 1 lower triangular (zero for k > i), 2 upper (zero for k < i)
+  // One triangle of D wanted: the tiles that touch it, per matrix and in scheduling order, are listed in device memory
+  // (tile ids of the full tiles_m x tiles_n numbering); num_tiles then counts batch * list_len listed tiles.
+  const int* tile_list;                   // nullptr: every tile is computed
+  int list_len;
   // Tail split (kernels built with kSplit): the tiles from split_first_tile on, which would leave most CTAs idle in
   // the last wave, are cut into `split` slices of K each, one work item per slice; num_items counts whole tiles + slices.
   int split, split_first_tile, num_items;
@@ -177,6 +181,10 @@ struct WorkItem {
 };
 template <bool kSplit>
 __device__ __forceinline__ int item_tile(const DenseParams& p, int item) {
+  if (p.tile_list != nullptr) {  // (never together with a tail split)
+    const int b = item / p.list_len;
+    return b * (p.tiles_m * p.tiles_n) + __ldg(p.tile_list + (item - b * p.list_len));
+  }
   if (!kSplit || item < p.split_first_tile) return item;
   return p.split_first_tile + (item - p.split_first_tile) / p.split;
 }

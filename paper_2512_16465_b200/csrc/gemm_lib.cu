@@ -14,6 +14,7 @@
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <vector>
 
 #include "dense_kernel.cuh"
 #include "skinny_kernel.cuh"
@@ -114,6 +115,8 @@ struct gemm_plan_s {
   uint32_t* d_status;       // device: 16-byte status word, followed (256 bytes on) by the stream-K arrival counters
   size_t d_counters_bytes = 0;  // plan-owned words after the status word: stream-K arrival counters or tail-split flags
   int split = 1;                // tail split factor of a dense plan
+  int d_tri = 0;                // one triangle of D wanted: 1 lower, 2 upper (dense variants)
+  int* d_tile_list = nullptr;   // device: the tiles of one matrix that touch that triangle, in scheduling order
   size_t split_flag_bytes = 0;
   unsigned long long runs = 0;  // launches so far (the timeout test hook acts on the first one only)
   uint32_t timeout_ms;
@@ -136,6 +139,7 @@ gemm_status_t validate(const gemm_desc_t* d) {
     return GEMM_ERR_INVALID_ARG;
   if (d->epilogue < GEMM_EPI_NONE || d->epilogue > GEMM_EPI_BIAS_SILU) return GEMM_ERR_INVALID_ARG;
   if ((d->flags & GEMM_FLAG_A_LOWER) && (d->flags & GEMM_FLAG_A_UPPER)) return GEMM_ERR_INVALID_ARG;
+  if ((d->flags & GEMM_FLAG_D_LOWER) && (d->flags & GEMM_FLAG_D_UPPER)) return GEMM_ERR_INVALID_ARG;
   if (d->ab_dtype == GEMM_F32) return GEMM_ERR_UNSUPPORTED;
   // 8-bit operands: K-contiguous storage only (A stored M x K, B stored N x K)
   if (is_fp8(d->ab_dtype) && (d->transa != GEMM_OP_N || d->transb != GEMM_OP_T)) return GEMM_ERR_UNSUPPORTED;
@@ -162,11 +166,55 @@ int dense_smem_bytes(int stages, int a_stage, int b_stage, int epi_wg) {  // a_s
   return 1024 /*alignment slack*/ + stages * (a_stage + b_stage) + 4 * epi_wg * 2 * kSlabBytes + 16 * kMaxStages + 64;
 }
 
+int d_tri_of(const gemm_desc_t& d) { return (d.flags & GEMM_FLAG_D_LOWER) ? 1 : ((d.flags & GEMM_FLAG_D_UPPER) ? 2 : 0); }
+
+// Tile columns [*j0, *j1] of tile row i that touch the wanted triangle of D (empty when *j0 > *j1).
+// Lower (row >= column): the tile's last row must reach its first column; upper: its first row must not pass its last column.
+void tri_columns(int d_tri, long long i, int tile_m, int bn, long long M, long long N, int tiles_n, int* j0, int* j1) {
+  *j0 = 0;
+  *j1 = tiles_n - 1;
+  if (d_tri == 1) {
+    const long long last_row = std::min<long long>((i + 1) * tile_m, M) - 1;
+    *j1 = static_cast<int>(std::min<long long>(tiles_n - 1, last_row / bn));
+  } else if (d_tri == 2) {
+    const long long first_row = i * tile_m;
+    *j0 = first_row > N - 1 ? tiles_n : static_cast<int>(first_row / bn);
+  }
+}
+long long tri_tile_count(int d_tri, int tile_m, int bn, long long M, long long N) {
+  const int tiles_m = ceil_div(M, tile_m), tiles_n = ceil_div(N, bn);
+  if (d_tri == 0) return static_cast<long long>(tiles_m) * tiles_n;
+  long long n = 0;
+  for (int i = 0; i < tiles_m; ++i) {
+    int j0, j1;
+    tri_columns(d_tri, i, tile_m, bn, M, N, tiles_n, &j0, &j1);
+    if (j1 >= j0) n += j1 - j0 + 1;
+  }
+  return n;
+}
+// The listed tiles in the order the scheduler visits the full grid (groups of `raster` tile rows, inside a group
+// column by column with the row running fastest), so the resident tiles still share their A band and B panels.
+std::vector<int> tri_tile_list(int d_tri, int tile_m, int bn, long long M, long long N, int raster) {
+  const int tiles_m = ceil_div(M, tile_m), tiles_n = ceil_div(N, bn);
+  std::vector<int> list;
+  int t = 0;
+  for (int first = 0; first < tiles_m; first += raster) {
+    const int gm = std::min(raster, tiles_m - first);
+    for (int tn = 0; tn < tiles_n; ++tn)
+      for (int r = 0; r < gm; ++r, ++t) {
+        int j0, j1;
+        tri_columns(d_tri, first + r, tile_m, bn, M, N, tiles_n, &j0, &j1);
+        if (tn >= j0 && tn <= j1) list.push_back(t);
+      }
+  }
+  return list;
+}
+
 // Tail split of the double-buffered dense kernels (on request, GEMM_FLAG_TAIL_SPLIT): when the tiles left over after the
 // full waves occupy at most half of the CTAs (pairs), each of them is cut into this many K slices, one per CTA (pair); the slice that
 // starts at K = 0 adds the others' raw accumulators from the workspace and finishes the tile.  1 = no split.
 int tail_split(long long tiles, int units, int num_kb, const gemm_desc_t& d) {
-  if (d.flags & (GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER)) return 1;
+  if (d.flags & (GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER | GEMM_FLAG_D_LOWER | GEMM_FLAG_D_UPPER)) return 1;
   const long long rem = tiles % units;
   if (rem == 0 || rem * 2 > units) return 1;
   if (tiles / units >= 8) return 1;  // many full waves: the last one is a few per cent at most; keep the plain kernel
@@ -198,7 +246,7 @@ double estimate_dense_cycles(const gemm_desc_t& d, int sm_count, int variant, in
   const int rows_cta = wide ? kWideCtaM : kCtaM;
   const int rows_tile = rows_cta * cg;
   const int units = std::max(1, sm_count / cg);
-  const long long tiles = static_cast<long long>(ceil_div(d.M, rows_tile)) * ceil_div(d.N, bn) * d.batch_count;
+  const long long tiles = tri_tile_count(d_tri_of(d), rows_tile, bn, d.M, d.N) * d.batch_count;
   const double kblocks = static_cast<double>(ceil_div(d.K, kblk_of(d.ab_dtype)));  // 128-byte slices: same pipe time for either width
   double waves = static_cast<double>((tiles + units - 1) / units);
   if (!wide) {  // a thinly filled last wave is split along K (two slices per stage assumed, as plan_dense will choose for long K)
@@ -244,7 +292,7 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
     const int units = pl->sm_count / cg;
     bn = 256;
     while (bn > bn_step) {
-      const long long tiles = static_cast<long long>(tiles_m) * ceil_div(d.N, bn) * d.batch_count;
+      const long long tiles = tri_tile_count(d_tri_of(d), tile_m, bn, d.M, d.N) * d.batch_count;
       if (tiles >= units && d.N > bn / 2) break;
       bn -= bn_step;  // 256 -> 192 -> 128 -> 64
       if (bn == 192) bn = 128;
@@ -258,7 +306,8 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   // Each ring stage ends with one tcgen05.commit, which costs tensor-pipe time; a stage of two 64-wide K slices
   // halves that cost.  Worth it when the ring still has at least three such stages (pairs; narrow 1-CTA tiles).
   const int units = pl->sm_count / cg;
-  const long long tiles_total = static_cast<long long>(tiles_m) * ceil_div(d.N, bn) * d.batch_count;
+  const int d_tri = d_tri_of(d);
+  const long long tiles_total = tri_tile_count(d_tri, tile_m, bn, d.M, d.N) * d.batch_count;  // tiles that are computed
   const bool single_wave = tiles_total <= units;  // every CTA (pair) computes at most one tile: pure latency
   // A tile's main loop lasts about 512 cycles per 64 columns of K (at tile N = 256); draining 128 x 256 accumulators
   // with four warps takes several thousand.  Short-K (output-bound) problems with several tiles per CTA get a second
@@ -283,8 +332,8 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   if (stages < 2 || stages > kMaxStages) return GEMM_ERR_UNSUPPORTED;
   const int smem = dense_smem_bytes(stages, a_stage, b_stage, epi_wg);
   if (smem > kMaxSmemOptin) return GEMM_ERR_UNSUPPORTED;
-  const long long num_tiles = static_cast<long long>(tiles_m) * tiles_n * d.batch_count;
-  if (num_tiles > 0x7FFFFFFFll) return GEMM_ERR_UNSUPPORTED;
+  if (static_cast<long long>(tiles_m) * tiles_n * d.batch_count > 0x7FFFFFFFll) return GEMM_ERR_UNSUPPORTED;
+  const long long num_tiles = tiles_total;
   // raster group height G: the resident tiles cover G tile rows x (units / G) tile columns; operand traffic from L2
   // is smallest when that block is square in elements, G * tile_m ~ (units / G) * bn
   int raster = forced_raster;
@@ -336,6 +385,9 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   // out (measured: +0.5 to +2.5 % on the 470 MB output of the projection shape, neutral on 134 MB)
   p.l2_hint_d = static_cast<double>(d.M) * d.N * d.batch_count * elem_bytes(d.c_dtype) > 64.0e6 ? 1 : 0;
   p.a_tri = (d.flags & GEMM_FLAG_A_LOWER) ? 1 : ((d.flags & GEMM_FLAG_A_UPPER) ? 2 : 0);
+  p.tile_list = nullptr;  // the device copy of the list is made by gemm_plan
+  p.list_len = d_tri ? static_cast<int>(num_tiles / d.batch_count) : 0;
+  pl->d_tri = d_tri;
   p.ldc = d.ldc;
   p.stride_c = d.batch_count > 1 ? d.stride_c : 0;
   p.debug_flags = 0u;  // set per run
@@ -386,6 +438,7 @@ gemm_status_t plan_wide(gemm_plan_s* pl, int forced_raster, int forced_stages) {
   const gemm_desc_t& d = pl->d;
   // its epilogue covers the bias per column, ReLU and erf GELU only; its MMA schedule has no K-range skipping
   if (d.epilogue > GEMM_EPI_BIAS_GELU_ERF || (d.flags & (GEMM_FLAG_BIAS_PER_ROW | GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER))) return GEMM_ERR_UNSUPPORTED;
+  if (d_tri_of(d)) return GEMM_ERR_UNSUPPORTED;  // its scheduler has no tile list
   const int a_kmajor = d.transa == GEMM_OP_N;
   const int b_kmajor = d.transb == GEMM_OP_T;
   const int tile_m = 2 * kWideCtaM, bn = kWideTileN;
@@ -473,6 +526,7 @@ gemm_status_t plan_skinny(gemm_plan_s* pl, int forced_stages, int forced_atoms) 
   if (d.transa != GEMM_OP_N || d.transb != GEMM_OP_T) return GEMM_ERR_UNSUPPORTED;  // both operands K-contiguous
   if ((d.M > kSkinnyMaxM && d.N > kSkinnyMaxM) || d.batch_count != 1) return GEMM_ERR_UNSUPPORTED;
   if (d.flags & (GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER)) return GEMM_ERR_UNSUPPORTED;  // no K-range skipping in stream-K
+  if (d_tri_of(d)) return GEMM_ERR_UNSUPPORTED;  // a short extent of 64 has a single tile row or column: nothing to leave out
   SkinnyPlan& s = pl->skinny;
   pl->skinny_tall = d.M > kSkinnyMaxM;  // the short extent is N: A is streamed, B is the resident slab
   const int small_extent = static_cast<int>(pl->skinny_tall ? d.N : d.M), big_extent = static_cast<int>(pl->skinny_tall ? d.M : d.N);
@@ -538,9 +592,17 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
   // roofline class (Section 4.3): compulsory traffic vs. work
   const gemm_desc_t& d = pl->d;
   const double eb = elem_bytes(d.ab_dtype), ec = elem_bytes(d.c_dtype);
-  const double flops = 2.0 * d.M * d.N * d.K * d.batch_count;
+  // elements of D that are wanted: all of it, or one triangle (diagonal included)
+  double d_elems = static_cast<double>(d.M) * d.N;
+  if (d_tri_of(d)) {
+    const double s = static_cast<double>(std::min(d.M, d.N));  // the square part holds s (s + 1) / 2; what lies beside it is whole or empty
+    const double beside = d_tri_of(d) == 1 ? static_cast<double>(std::max<int64_t>(d.M - d.N, 0)) * d.N
+                                           : static_cast<double>(std::max<int64_t>(d.N - d.M, 0)) * d.M;
+    d_elems = s * (s + 1.0) / 2.0 + beside;
+  }
+  const double flops = 2.0 * d_elems * d.K * d.batch_count;
   double bytes = d.batch_count * (static_cast<double>(d.M) * d.K + static_cast<double>(d.K) * d.N) * eb +
-                 d.batch_count * static_cast<double>(d.M) * d.N * ec;
+                 d.batch_count * d_elems * ec;
   if (has_bias(d.epilogue)) bytes += 4.0 * ((d.flags & GEMM_FLAG_BIAS_PER_ROW) ? d.M : d.N);
   gemm_info_t& info = pl->info;
   info.struct_size = sizeof(gemm_info_t);
@@ -561,7 +623,7 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
     // memory-bound problems with a handful of rows stream the weight matrix once: stream-K path;
     // everything else is a dense tiled GEMM, paired CTAs when there are at least two tile rows
     const bool skinny_ok = (d.M <= kSkinnyMaxM || d.N <= kSkinnyMaxM) && d.batch_count == 1 && d.transa == GEMM_OP_N &&
-                           d.transb == GEMM_OP_T && !(d.flags & (GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER));
+                           d.transb == GEMM_OP_T && !(d.flags & (GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER)) && !d_tri_of(d);
     if (skinny_ok && info.intensity < 7.0 * kRidgeCudaCore) {
       variant = GEMM_VARIANT_SKINNY_STREAMK;  // measured: level with the dense kernels at a short extent of 64 on the largest shapes, far ahead elsewhere
     } else {
@@ -572,7 +634,8 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
         for (int bn : {256, 128, 64}) {
           if (v == GEMM_VARIANT_DENSE_2CTA_WIDE && bn != kWideTileN) continue;
           if (v == GEMM_VARIANT_DENSE_2CTA_WIDE &&
-              (d.epilogue > GEMM_EPI_BIAS_GELU_ERF || (d.flags & (GEMM_FLAG_BIAS_PER_ROW | GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER))))
+              (d.epilogue > GEMM_EPI_BIAS_GELU_ERF || d_tri_of(d) ||
+               (d.flags & (GEMM_FLAG_BIAS_PER_ROW | GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER))))
             continue;
           if (v == GEMM_VARIANT_DENSE_2CTA && !b_kmajor && bn % 128) continue;  // 64-column boxes per CTA
           if (v != GEMM_VARIANT_DENSE_1CTA && d.M <= kCtaM) continue;           // a pair needs two tile rows
@@ -603,6 +666,19 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
       delete pl;
       return GEMM_ERR_CUDA;
     }
+  }
+  if (pl->has_device && pl->arch_ok && pl->d_tri) {
+    const std::vector<int> list = tri_tile_list(pl->d_tri, pl->info.tile_m, pl->bn, d.M, d.N, pl->raster_group);
+    const size_t bytes = std::max<size_t>(list.size(), 1) * sizeof(int);
+    if (static_cast<int>(list.size()) != pl->dense.list_len || cudaMalloc(&pl->d_tile_list, bytes) != cudaSuccess ||
+        cudaMemcpy(pl->d_tile_list, list.data(), list.size() * sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) {
+      note_cuda_error("cudaMalloc(tile list)", cudaGetErrorName(cudaGetLastError()));
+      if (pl->d_tile_list) cudaFree(pl->d_tile_list);
+      cudaFree(pl->d_status);
+      delete pl;
+      return GEMM_ERR_CUDA;
+    }
+    pl->dense.tile_list = pl->d_tile_list;
   }
   if (getenv("B200GEMM_LOG")) {
     fprintf(stderr,
@@ -655,6 +731,10 @@ gemm_status_t gemm_plan_status(gemm_plan_t plan) {
 gemm_status_t gemm_destroy(gemm_plan_t plan) {
   if (!plan) return GEMM_OK;
   gemm_status_t st = GEMM_OK;
+  if (plan->d_tile_list && cudaFree(plan->d_tile_list) != cudaSuccess) {
+    note_cuda_error("cudaFree", cudaGetErrorName(cudaGetLastError()));
+    st = GEMM_ERR_CUDA;
+  }
   if (plan->d_status && cudaFree(plan->d_status) != cudaSuccess) {
     note_cuda_error("cudaFree", cudaGetErrorName(cudaGetLastError()));
     st = GEMM_ERR_CUDA;

@@ -62,7 +62,8 @@ def to_host_bits(t: torch.Tensor, dtype: int) -> np.ndarray:
 def desc_of(w: wl.Workload, flags: int = 0, c_dtype=None) -> bg.Desc:
     cd = w.c_dtype if c_dtype is None else c_dtype
     return bg.make_desc(w.M, w.N, w.K, w.transa, w.transb, w.ab_dtype, cd, w.lda, w.ldb, w.ldc, w.batch,
-                        w.stride_a, w.stride_b, w.stride_c, w.epilogue, flags | bg.make_flags(bias_per_row=w.bias_per_row, a_lower=w.a_tri == 1, a_upper=w.a_tri == 2))
+                        w.stride_a, w.stride_b, w.stride_c, w.epilogue, flags | bg.make_flags(bias_per_row=w.bias_per_row, a_lower=w.a_tri == 1, a_upper=w.a_tri == 2,
+                                                                                           d_lower=w.d_tri == 1, d_upper=w.d_tri == 2))
 
 
 def problem_of(w: wl.Workload, c_dtype=None) -> oracle.Problem:
@@ -149,7 +150,23 @@ def check_blocks(w: wl.Workload, inputs: dict, cbits: np.ndarray, blocks, c_dtyp
     for batches, rows, cols in blocks:
         y, bound = oracle.gemm(p, inputs["A"], inputs["B"], C_in=cin, bias=inputs["bias"], alpha=w.alpha, beta=w.beta,
                                batches=batches, rows=rows, cols=cols)
-        reports.append(compare_block(gather(cbits, w, batches, rows, cols), y, bound, cd))
+        got_bits = gather(cbits, w, batches, rows, cols)
+        if not w.d_tri:
+            reports.append(compare_block(got_bits, y, bound, cd))
+            continue
+        # one triangle of D wanted: its elements are held to the usual bars; every other element must either be
+        # untouched (still the NaN poison, or C_in when beta != 0) or hold its value of the plain product
+        keep = np.broadcast_to(oracle.wanted(rows, cols, w.d_tri)[None, :, :], y.shape)
+        rep = compare_block(got_bits[keep], y[keep], bound[keep], cd)
+        out_bits, out_y, out_bound = got_bits[~keep], y[~keep], bound[~keep]
+        out_val = oracle.decode(out_bits, cd)
+        untouched = np.isnan(out_val) if cin is None else out_bits == gather(cin, w, batches, rows, cols)[~keep]
+        with np.errstate(invalid="ignore"):
+            plain = np.abs(out_val - out_y) <= REL_TOL * out_bound + ABS_TOL + U_OUT[cd] * np.abs(out_y)
+        rep["outside_ok"] = bool(np.all(untouched | plain))
+        rep["outside_untouched"] = int(np.sum(untouched))
+        rep["outside_n"] = int(untouched.size)
+        reports.append(rep)
     return reports
 
 
@@ -176,6 +193,7 @@ def default_blocks(w: wl.Workload) -> list:
 def assert_reports(reports, what=""):
     for r in reports:
         assert r["finite"], f"{what}: non-finite output {r}"
+        assert r.get("outside_ok", True), f"{what}: an element outside the wanted triangle is neither untouched nor right {r}"
         assert r["max_err_over_tol"] <= 1.0, f"{what}: per-element tolerance exceeded {r}"
         assert r["frob"] <= frob_tol_for(r["c_dtype"]), f"{what}: Frobenius error {r}"
         if r["c_dtype"] != wl.F32:

@@ -80,6 +80,8 @@ def test_shape_specifications_of_the_sweep_mode():
     w = bench.parse_shape("256x128x512:ab=e4m3:tri=upper:batch=3:ta=0:tb=1:lda=520")
     assert (w.ab_dtype, w.a_tri, w.batch, w.lda, w.c_dtype) == (wl.FP8_E4M3, 2, 3, 520, wl.BF16)
     assert w.min_bytes == 3 * (256 * 512 + 512 * 128) * 1 + 3 * 256 * 128 * 2       # 8-bit operands, 16-bit output
+    w = bench.parse_shape("4096x4096x512:dtri=lower")
+    assert w.d_tri == 1 and w.flops == 2.0 * (4096 * 4097 // 2) * 512
     with pytest.raises(SystemExit):
         bench.parse_shape("8x8x8:nonsense=1")
     # an 8-bit problem is held against the measured bf16 peak times the nominal fp8 : bf16 ratio

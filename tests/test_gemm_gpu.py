@@ -1,5 +1,7 @@
 """GPU parity tests: the CUDA path, called through the C-ABI binding, against the CPU oracle
 on the same seeded inputs.  Run with ``-m gpu`` on a B200."""
+from dataclasses import replace
+
 import numpy as np
 import pytest
 import torch
@@ -141,6 +143,25 @@ EXACT_CASES = [
     ("tail_split_automatic_for_few_tiles", 300, 264, 32768, dict(), dict()),
     ("tail_split_switched_off", 1024, 1024, 2048, dict(cd=wl.BF16), dict(variant=V2, tile_n=256)),
     ("tail_split_requested_auto_plan", 2304, 2304, 2304, dict(cd=wl.BF16), dict(tail_split=True)),
+    # one triangle of D wanted (symmetric results): tiles wholly in the other triangle are left out of the schedule
+    ("d_lower_1cta", 700, 700, 200, dict(d_tri=1), dict(variant=V1, tile_n=128)),
+    ("d_upper_1cta", 700, 700, 200, dict(d_tri=2), dict(variant=V1, tile_n=128)),
+    ("d_lower_pair_wide_tiles", 1104, 1104, 264, dict(d_tri=1, cd=wl.BF16), dict(variant=V2, tile_n=256)),
+    ("d_upper_pair_narrow_tiles", 1104, 1104, 264, dict(d_tri=2), dict(variant=V2, tile_n=64)),
+    ("d_lower_tile_n_192_raster_2", 900, 1000, 136, dict(d_tri=1), dict(variant=V1, tile_n=192, raster=2)),
+    ("d_lower_m_longer", 1500, 400, 136, dict(d_tri=1), dict(variant=V1, tile_n=128)),
+    ("d_upper_m_longer", 1500, 400, 136, dict(d_tri=2), dict(variant=V2, tile_n=128)),
+    ("d_lower_n_longer", 400, 1500, 136, dict(d_tri=1), dict(variant=V2, tile_n=128)),
+    ("d_upper_n_longer", 400, 1500, 136, dict(d_tri=2), dict(variant=V1, tile_n=256)),
+    ("d_lower_batched_beta_bias", 304, 304, 136, dict(d_tri=1, batch=5, beta=1.0, epi=bg.EPI_BIAS_RELU, cd=wl.BF16), dict(variant=V1, tile_n=64)),
+    ("d_upper_batched_pair", 520, 520, 72, dict(d_tri=2, batch=3, ab=wl.F16, cd=wl.F16), dict(variant=V2, tile_n=128)),
+    ("d_lower_one_tile", 100, 100, 64, dict(d_tri=1), dict(variant=V1)),
+    ("d_lower_nn_layout", 704, 704, 200, dict(d_tri=1, ta=0, tb=0), dict(variant=V2, tile_n=128)),
+    ("d_lower_with_lower_a", 768, 768, 768, dict(d_tri=1, a_tri=1), dict(variant=V2, tile_n=128)),
+    ("d_lower_fp8", 704, 704, 528, dict(d_tri=1, ab=wl.FP8_E4M3, cd=wl.BF16), dict(variant=V2, tile_n=256)),
+    ("d_lower_two_epilogue_groups", 2048, 2048, 256, dict(d_tri=1, cd=wl.BF16), dict(variant=V1, tile_n=256)),
+    ("d_lower_auto", 2304, 2304, 520, dict(d_tri=1, cd=wl.BF16), dict()),
+    ("d_upper_auto_tail_split_requested", 1024, 1024, 2048, dict(d_tri=2), dict(tail_split=True)),
     # mirrored stream-K: a tall output with a handful of columns (A is the streamed operand)
     ("tall_one_unit", 128, 8, 64, {}, dict(variant=VS)),
     ("tall_split_k", 256, 8, 4096, {}, dict(variant=VS)),
@@ -487,6 +508,61 @@ def test_triangular_a_really_skips():
         with pytest.raises(bg.GemmError) as e:
             bg.gemm_plan(H.desc_of(int_workload("tri_refused", 8 if bad["variant"] == VS else 1024, 1024, 4096, a_tri=1), bg.make_flags(**bad)))
         assert e.value.status == bg.ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("d_tri", [1, 2])
+def test_triangular_d_leaves_the_other_tiles_alone(d_tri):
+    """One triangle of D wanted: every output tile that lies wholly in the other triangle stays as it was (NaN poison
+    here, and C_in when beta != 0), every wanted element is bit-exact, the plan reports fewer tiles than the full grid,
+    and the kernels without a tile list refuse the flag."""
+    for fl, M, N in ((dict(variant=V1, tile_n=128), 1000, 1000), (dict(variant=V2, tile_n=64), 1000, 1000), (dict(), 1300, 900)):
+        for beta in (0.0, 1.0):
+            w = int_workload("d_tri_skip", M, N, 200, d_tri=d_tri, beta=beta)
+            inputs = wl.make_inputs(w)
+            cbits, info = H.run_gpu(w, inputs, bg.make_flags(**fl))
+            reports = H.check_blocks(w, inputs, cbits, H.default_blocks(w))
+            H.assert_reports(reports, what=str(fl))
+            assert reports[0]["bit_identical"] == 1.0
+            tm, tn = info["tile_m"], info["tile_n"]
+            rows_t, cols_t = -(-M // tm), -(-N // tn)
+            got = cbits.reshape(M, N)
+            init = None if beta == 0.0 else inputs["C"].reshape(M, N)
+            skipped = 0
+            for ti in range(rows_t):
+                r0, r1 = ti * tm, min((ti + 1) * tm, M)
+                for tj in range(cols_t):
+                    c0, c1 = tj * tn, min((tj + 1) * tn, N)
+                    outside = c0 > r1 - 1 if d_tri == 1 else r0 > c1 - 1
+                    if outside:
+                        skipped += 1
+                        blk = got[r0:r1, c0:c1]
+                        assert np.all(np.isnan(blk)) if init is None else np.array_equal(blk, init[r0:r1, c0:c1]), (fl, ti, tj)
+            assert skipped > 0 and info["num_tiles"] == rows_t * cols_t - skipped, (info["num_tiles"], rows_t, cols_t, skipped)
+    for bad, M in ((dict(variant=VS), 8), (dict(variant=VW), 1024)):
+        with pytest.raises(bg.GemmError) as e:
+            bg.gemm_plan(H.desc_of(int_workload("d_tri_refused", M, 1024, 4096, d_tri=d_tri), bg.make_flags(**bad)))
+        assert e.value.status == bg.ERR_UNSUPPORTED
+    with pytest.raises(bg.GemmError) as e:
+        bg.gemm_plan(H.desc_of(int_workload("d_tri_both", 256, 256, 64), bg.make_flags(d_lower=True, d_upper=True)))
+    assert e.value.status == bg.ERR_INVALID_ARG
+
+
+def test_triangular_d_general_values_symmetric_product():
+    """D = A A^T with normally distributed A (the same buffer as both operands): the lower triangle meets the stated
+    tolerance, and mirrors the upper triangle of a second run bit for bit (the product is symmetric and, with K walked
+    forwards in every tile, both runs accumulate the same products in the same order)."""
+    w = wl.Workload("syrk", 900, 900, 520, transa=0, transb=1, c_dtype=wl.F32, d_tri=1, seed=5)
+    inputs = wl.make_inputs(w)
+    inputs["B"] = inputs["A"].copy()
+    fl = bg.make_flags(variant=V2, tile_n=256, no_k_serpentine=True)
+    lo, _ = H.run_gpu(w, inputs, fl)
+    H.assert_reports(H.check_blocks(w, inputs, lo, H.default_blocks(w)), what="lower")
+    wu = replace(w, d_tri=2)
+    up, _ = H.run_gpu(wu, inputs, fl)
+    H.assert_reports(H.check_blocks(wu, inputs, up, H.default_blocks(wu)), what="upper")
+    lo2, up2 = lo.reshape(900, 900), up.reshape(900, 900)
+    il = np.tril_indices(900)
+    assert np.array_equal(lo2[il], up2.T[il])
 
 
 @pytest.mark.parametrize("ab", [wl.FP8_E4M3, wl.FP8_E5M2])

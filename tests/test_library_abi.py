@@ -184,6 +184,34 @@ def test_cost_model_choices_follow_the_measurements():
     assert choice(8192, 8192, 1024)[0] == bg.VARIANT_DENSE_2CTA              # the pair beats the single CTA at every K measured
 
 
+def test_triangular_result_plans():
+    """One triangle of D wanted: the plan lists only the tiles that touch it, counts the useful work, and keeps to the
+    kernels that have a tile list."""
+    full = bg.Plan(bg.make_desc(8192, 8192, 8192, c_dtype=bg.F32)).info
+    for fl in (bg.make_flags(d_lower=True), bg.make_flags(d_upper=True)):
+        info = bg.Plan(bg.make_desc(8192, 8192, 8192, c_dtype=bg.F32, flags=fl)).info
+        assert info["variant"] == bg.VARIANT_DENSE_2CTA and (info["tile_m"], info["tile_n"]) == (256, 256)
+        assert info["num_tiles"] == 32 * 33 // 2                      # 32 x 32 square tiles, diagonal included
+        assert info["flops"] == 2.0 * (8192 * 8193 // 2) * 8192 and info["flops"] < 0.51 * full["flops"]
+    # non-square tiles and matrices: 1000 x 600 output, 128 x 64 tiles -> row i keeps columns 0 .. min(9, (128 (i + 1) - 1) // 64)
+    info = bg.Plan(bg.make_desc(1000, 600, 256, c_dtype=bg.F32, flags=bg.make_flags(variant=bg.VARIANT_DENSE_1CTA, tile_n=64, d_lower=True))).info
+    assert info["num_tiles"] == sum(min(9, (min(128 * (i + 1), 1000) - 1) // 64) + 1 for i in range(8))
+    info = bg.Plan(bg.make_desc(1000, 600, 256, c_dtype=bg.F32, flags=bg.make_flags(variant=bg.VARIANT_DENSE_1CTA, tile_n=64, d_upper=True))).info
+    assert info["num_tiles"] == sum(max(0, 10 - (128 * i) // 64) for i in range(8) if 128 * i <= 599)
+    # batches multiply the list
+    info = bg.Plan(bg.make_desc(512, 512, 256, c_dtype=bg.F32, batch=7, flags=bg.make_flags(variant=bg.VARIANT_DENSE_1CTA, tile_n=128, d_lower=True))).info
+    assert info["num_tiles"] == 7 * 10
+    for bad in (bg.make_flags(variant=bg.VARIANT_DENSE_2CTA_WIDE, d_lower=True), bg.make_flags(variant=bg.VARIANT_SKINNY_STREAMK, d_upper=True)):
+        with pytest.raises(bg.GemmError) as e:
+            bg.gemm_plan(bg.make_desc(64 if bad & 0x30 == 0x30 else 4096, 4096, 4096, flags=bad))
+        assert e.value.status == bg.ERR_UNSUPPORTED
+    with pytest.raises(bg.GemmError) as e:
+        bg.gemm_plan(bg.make_desc(512, 512, 512, flags=bg.make_flags(d_lower=True, d_upper=True)))
+    assert e.value.status == bg.ERR_INVALID_ARG
+    # a short output that would go to stream-K stays dense when a triangle is asked for
+    assert bg.Plan(bg.make_desc(64, 8192, 8192, flags=bg.make_flags(d_upper=True))).info["variant"] != bg.VARIANT_SKINNY_STREAMK
+
+
 def test_tuning_entry_points_on_the_host():
     # the workspace bound needs no device: only the stream-K candidates of a short-extent problem use one
     assert bg.gemm_tune_workspace_bytes(bg.make_desc(8192, 8192, 512)) == 0          # nothing to split, no short extent

@@ -331,6 +331,19 @@ def test_new_activations_and_row_bias_in_the_gemm():
         oracle.gemm(Problem(M, N, K, epilogue=10), a, b)                              # unknown epilogue
 
 
+def test_wanted_triangle_of_a_symmetric_result():
+    # the mask against numpy's own triangles, its element count in closed form, and the two triangles sharing only the diagonal
+    r, c = np.arange(6), np.arange(6)
+    lo, up = oracle.wanted(r, c, 1), oracle.wanted(r, c, 2)
+    assert np.array_equal(lo, np.tril(np.ones((6, 6), bool))) and np.array_equal(up, np.triu(np.ones((6, 6), bool)))
+    assert lo.sum() == 6 * 7 // 2 and np.array_equal(lo & up, np.eye(6, dtype=bool)) and np.all(lo | up)
+    assert np.array_equal(lo, up.T) and oracle.wanted(r, c, 0).all()
+    # arbitrary (sampled, unordered) rows and columns: the mask follows the indices, not the positions
+    rows, cols = np.array([5, 0, 3]), np.array([4, 4, 0, 5])
+    assert np.array_equal(oracle.wanted(rows, cols, 1), np.array([[1, 1, 1, 1], [0, 0, 1, 0], [0, 0, 1, 0]], bool))
+    assert oracle.wanted(np.arange(7), np.arange(3), 1).sum() == 6 + 4 * 3     # 7 x 3 lower: 1 + 2 + 3, then whole rows
+
+
 def test_batched_equals_loop_of_singles():
     w = wl.Workload("t", 9, 7, 12, transa=0, transb=1, ab_dtype=F16, batch=4, beta=0.5, c_dtype=F16,
                     dist_a=wl.Dist("uniform", -2, 2), dist_b=wl.Dist("uniform", -2, 2), alpha=0.25,

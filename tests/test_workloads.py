@@ -93,6 +93,19 @@ def test_triangular_structure_of_a():
     assert wl.Workload("t", 4, 3, 6, a_tri=2).flops == 2.0 * (6 + 5 + 4 + 3) * 3
 
 
+def test_useful_work_of_a_triangular_result():
+    # wanted elements of D, two flops per element and k: 4 x 4 lower = 10, 4 x 6 upper = 6 + 5 + 4 + 3, 6 x 4 lower = 10 + 2 * 4
+    assert wl.Workload("t", 4, 4, 5, d_tri=1).flops == 2.0 * 10 * 5
+    assert wl.Workload("t", 4, 6, 5, d_tri=2).flops == 2.0 * 18 * 5
+    assert wl.Workload("t", 6, 4, 5, d_tri=1, batch=3).flops == 2.0 * 18 * 5 * 3
+    # together with a lower-triangular op(A): row i has min(i + 1, K) non-zeros and i + 1 wanted columns
+    assert wl.Workload("t", 3, 3, 3, d_tri=1, a_tri=1).flops == 2.0 * (1 * 1 + 2 * 2 + 3 * 3)
+    # brute force against the definition of the mask
+    for d_tri, M, N in ((1, 7, 5), (2, 7, 5), (1, 5, 9), (2, 5, 9)):
+        cnt = sum(1 for i in range(M) for j in range(N) if (i >= j if d_tri == 1 else i <= j))
+        assert wl.Workload("t", M, N, 2, d_tri=d_tri).flops == 2.0 * cnt * 2
+
+
 def test_fp8_encoding_matches_the_library_conversion():
     import torch
     rng = np.random.default_rng(0)

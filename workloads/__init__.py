@@ -111,6 +111,7 @@ class Workload:
     epilogue: int = EPI_NONE
     bias_per_row: bool = False   # the bias has M entries (one per output row) instead of N
     a_tri: int = 0               # structure of op(A): 0 dense, 1 lower triangular (zero for k > i), 2 upper (zero for k < i)
+    d_tri: int = 0               # part of D that is wanted: 0 all, 1 lower triangle (row >= column), 2 upper (row <= column)
     alpha: float = 1.0
     beta: float = 0.0
     dist_a: Dist = field(default_factory=lambda: Dist("normal", 0.0, 1.0))
@@ -150,14 +151,21 @@ class Workload:
 
     @property
     def flops(self) -> float:
-        """Useful work: two flops per (non-zero element of op(A)) x (output column)."""
+        """Useful work: two flops per (non-zero element of op(A) in row i) x (wanted output column of row i)."""
+        i = np.arange(self.M, dtype=np.int64)
         if self.a_tri == 1:
-            nz = sum(min(i + 1, self.K) for i in range(self.M))
+            nz = np.minimum(i + 1, self.K)
         elif self.a_tri == 2:
-            nz = sum(max(self.K - i, 0) for i in range(self.M))
+            nz = np.maximum(self.K - i, 0)
         else:
-            nz = self.M * self.K
-        return 2.0 * nz * self.N * self.batch
+            nz = np.full(self.M, self.K, dtype=np.int64)
+        if self.d_tri == 1:
+            cols = np.minimum(i + 1, self.N)
+        elif self.d_tri == 2:
+            cols = np.maximum(self.N - i, 0)
+        else:
+            cols = np.full(self.M, self.N, dtype=np.int64)
+        return 2.0 * float(np.sum(nz * cols)) * self.batch
 
     @property
     def min_bytes(self) -> float:
