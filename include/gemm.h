@@ -124,6 +124,13 @@ typedef enum {
  * only (not the wide pair tile, not stream-K); at most one of the two; combines with A_LOWER / A_UPPER and batches. */
 #define GEMM_FLAG_D_LOWER 0x4000u
 #define GEMM_FLAG_D_UPPER 0x8000u
+/* gemm_desc_t.structure -- structure of op(B) (K x N), a promise like A_LOWER / A_UPPER: with B_LOWER every element
+ * with k < j IS zero in memory, with B_UPPER every element with k > j.  The K ranges that can only contribute zeros
+ * are skipped per output tile; together with A_UPPER and D_UPPER (or the three LOWER ones) this is the product of two
+ * triangular matrices, itself triangular, at about a sixth of the dense work.  Dense 1-CTA and pair variants only; at
+ * most one of the two. */
+#define GEMM_STRUCT_B_LOWER 0x1u
+#define GEMM_STRUCT_B_UPPER 0x2u
 #define GEMM_FLAG_BIAS_PER_ROW 0x1u         /* the bias is fp32[M], one value per output row (default: fp32[N], one per
                                               column); not a tuning knob: it changes what is computed */
 #define GEMM_FLAG_NO_EARLY_LAUNCH 0x4u       /* launch without programmatic dependent launch (default: the kernel may be
@@ -146,6 +153,8 @@ typedef struct {
   int32_t batch_count;        /* >= 1 */
   int32_t epilogue;           /* gemm_epilogue_t */
   int64_t stride_a, stride_b, stride_c; /* elements between consecutive matrices; ignored when batch_count == 1 */
+  uint32_t structure;         /* GEMM_STRUCT_*: further structure promises (flags has no bit left); 0 = none */
+  uint32_t reserved;          /* must be 0 */
 } gemm_desc_t;
 
 typedef struct {
@@ -299,7 +308,7 @@ void gemm_tune_cache_clear(void);
  * gemm_host_create: desc as for gemm_plan, with transa = N and batch_count = 1 (row panels of A and C must be
  * contiguous row ranges); panels = 0 picks a count (about 8, fewer for small M).  Allocates the device staging
  * buffers (B, two A panels, two C panels, a workspace if the panel plan wants one), the streams and the events, on
- * the current device.  Errors: as gemm_plan; GEMM_ERR_UNSUPPORTED for transa = T, a batch or a triangular op(A); GEMM_ERR_CUDA if an
+ * the current device.  Errors: as gemm_plan; GEMM_ERR_UNSUPPORTED for transa = T, a batch, a triangular op(A) or a wanted triangle of D; GEMM_ERR_CUDA if an
  * allocation fails (nothing is leaked).
  * gemm_host_run: hA, hB, hC (and hbias, iff the epilogue has a bias): HOST pointers laid out as desc says; page-locked
  * memory is what makes the copies overlap (pageable memory works, without overlap).  hC is read only when beta != 0

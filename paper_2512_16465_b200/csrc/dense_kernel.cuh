@@ -54,6 +54,7 @@ struct DenseParams {
   int ab_fp8;                             // operands are 8-bit floats (tcgen05 kind::f8f6f4), else 16-bit (kind::f16)
   int kblk;                               // elements of K in one 128-byte slice: 64 (16-bit operands) or 128 (8-bit)
   int a_tri;                              // structure of op(A): 0 dense, 1 lower triangular (zero for k > i), 2 upper (zero for k < i)
+  int b_tri;                              // structure of op(B): 0 dense, 1 lower triangular (zero for k < j), 2 upper (zero for k > j)
   // One triangle of D wanted: the tiles that touch it, per matrix and in scheduling order, are listed in device memory
   // (tile ids of the full tiles_m x tiles_n numbering); num_tiles then counts batch * list_len listed tiles.
   const int* tile_list;                   // nullptr: every tile is computed
@@ -159,18 +160,24 @@ __device__ __forceinline__ TileCoord decode_tile(int t, int tiles_m, int tiles_n
   return c;
 }
 
-// The ring stages [lo, hi) of K that a tile with output rows [row0, row0 + rows) has to visit.  A triangular op(A)
-// (zero beyond the diagonal by the caller's word) makes every stage that lies wholly in the zero part a no-op, so
-// it is skipped; the stages that the diagonal crosses are computed in full.  At least one stage is always kept
-// so that the accumulator gets written.
+// The ring stages [lo, hi) of K that a tile with output rows [row0, row0 + rows) and columns [col0, col0 + cols) has to
+// visit.  A triangular op(A) or op(B) (zero beyond the diagonal by the caller's word) makes every stage that lies
+// wholly in a zero part a no-op, so it is skipped; the stages that a diagonal crosses are computed in full.  At least
+// one stage is always kept so that the accumulator gets written (when nothing is left, any stage yields the zeros).
 struct KRange {
   int lo, hi;
 };
-__device__ __forceinline__ KRange k_range(const DenseParams& p, int row0, int rows) {
+__device__ __forceinline__ KRange k_range(const DenseParams& p, int row0, int rows, int col0, int cols) {
   KRange r{0, p.num_kb};
   const int kstep = p.kblk * p.atoms;
-  if (p.a_tri == 1) r.hi = min(p.num_kb, (min(row0 + rows, p.M) - 1) / kstep + 1);
-  else if (p.a_tri == 2) r.lo = min(row0 / kstep, p.num_kb - 1);
+  if (p.a_tri == 1) r.hi = min(r.hi, (min(row0 + rows, p.M) - 1) / kstep + 1);       // k <= last row
+  else if (p.a_tri == 2) r.lo = max(r.lo, row0 / kstep);                              // k >= first row
+  if (p.b_tri == 1) r.lo = max(r.lo, col0 / kstep);                                   // k >= first column
+  else if (p.b_tri == 2) r.hi = min(r.hi, (min(col0 + cols, p.N) - 1) / kstep + 1);   // k <= last column
+  if (r.lo >= r.hi) {
+    r.lo = min(r.lo, p.num_kb - 1);
+    r.hi = r.lo + 1;
+  }
   return r;
 }
 
@@ -189,8 +196,8 @@ __device__ __forceinline__ int item_tile(const DenseParams& p, int item) {
   return p.split_first_tile + (item - p.split_first_tile) / p.split;
 }
 template <bool kSplit>
-__device__ __forceinline__ WorkItem work_item(const DenseParams& p, int item, int tile, int row0, int rows) {
-  WorkItem wi{tile, -1, k_range(p, row0, rows)};
+__device__ __forceinline__ WorkItem work_item(const DenseParams& p, int item, int tile, int row0, int rows, int col0) {
+  WorkItem wi{tile, -1, k_range(p, row0, rows, col0, p.bn)};
   if (kSplit && item >= p.split_first_tile) {
     wi.slice = (item - p.split_first_tile) - (tile - p.split_first_tile) * p.split;
     wi.kr.lo = wi.slice * p.num_kb / p.split;
@@ -407,7 +414,7 @@ __device__ __forceinline__ void producer_role(const DenseParams& p, const CUtens
     // Serpentine K: all CTAs advance through K roughly in step, so the K range a wave touched last is what L2
     // still holds when the next wave starts; walking it backwards re-uses those lines of the shared A band.
     const bool rev = p.k_serpentine && (it & 1u);
-    const KRange kr = work_item<kSplit>(p, item, tile, tc.tm * (kCtaM * CG), kCtaM * CG).kr;
+    const KRange kr = work_item<kSplit>(p, item, tile, tc.tm * (kCtaM * CG), kCtaM * CG, tc.tn * p.bn).kr;
     int k0 = rev ? (kr.hi - 1) * kstep : kr.lo * kstep;
     const int dk = rev ? -kstep : kstep;
     for (int kb = kr.lo; kb < kr.hi; ++kb, k0 += dk) {
@@ -477,8 +484,10 @@ __device__ __forceinline__ void mma_role(const DenseParams& p, uint32_t tiles_ba
     const uint32_t d_tmem = tmem_base + buf * static_cast<uint32_t>(p.bn);
     const bool rev = p.k_serpentine && (it & 1u);
     KRange kr{0, num_kb};
-    if (p.a_tri != 0 || (kSplit && item >= p.split_first_tile))
-      kr = work_item<kSplit>(p, item, tile, decode_tile(tile, p.tiles_m, p.tiles_n, p.raster_group).tm * (kCtaM * CG), kCtaM * CG).kr;
+    if ((p.a_tri | p.b_tri) != 0 || (kSplit && item >= p.split_first_tile)) {
+      const TileCoord tc = decode_tile(tile, p.tiles_m, p.tiles_n, p.raster_group);
+      kr = work_item<kSplit>(p, item, tile, tc.tm * (kCtaM * CG), kCtaM * CG, tc.tn * p.bn).kr;
+    }
     const int n_kb = kr.hi - kr.lo;
     for (int kb = 0; kb < n_kb; ++kb) {
       if (!mbar_wait_warp(full0 + 8u * s, ph, w, (2u << 8) | s)) return;

@@ -140,6 +140,8 @@ gemm_status_t validate(const gemm_desc_t* d) {
   if (d->epilogue < GEMM_EPI_NONE || d->epilogue > GEMM_EPI_BIAS_SILU) return GEMM_ERR_INVALID_ARG;
   if ((d->flags & GEMM_FLAG_A_LOWER) && (d->flags & GEMM_FLAG_A_UPPER)) return GEMM_ERR_INVALID_ARG;
   if ((d->flags & GEMM_FLAG_D_LOWER) && (d->flags & GEMM_FLAG_D_UPPER)) return GEMM_ERR_INVALID_ARG;
+  if ((d->structure & ~(GEMM_STRUCT_B_LOWER | GEMM_STRUCT_B_UPPER)) || d->reserved != 0) return GEMM_ERR_INVALID_ARG;
+  if ((d->structure & GEMM_STRUCT_B_LOWER) && (d->structure & GEMM_STRUCT_B_UPPER)) return GEMM_ERR_INVALID_ARG;
   if (d->ab_dtype == GEMM_F32) return GEMM_ERR_UNSUPPORTED;
   // 8-bit operands: K-contiguous storage only (A stored M x K, B stored N x K)
   if (is_fp8(d->ab_dtype) && (d->transa != GEMM_OP_N || d->transb != GEMM_OP_T)) return GEMM_ERR_UNSUPPORTED;
@@ -214,7 +216,7 @@ std::vector<int> tri_tile_list(int d_tri, int tile_m, int bn, long long M, long 
 // full waves occupy at most half of the CTAs (pairs), each of them is cut into this many K slices, one per CTA (pair); the slice that
 // starts at K = 0 adds the others' raw accumulators from the workspace and finishes the tile.  1 = no split.
 int tail_split(long long tiles, int units, int num_kb, const gemm_desc_t& d) {
-  if (d.flags & (GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER | GEMM_FLAG_D_LOWER | GEMM_FLAG_D_UPPER)) return 1;
+  if ((d.flags & (GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER | GEMM_FLAG_D_LOWER | GEMM_FLAG_D_UPPER)) || d.structure) return 1;
   const long long rem = tiles % units;
   if (rem == 0 || rem * 2 > units) return 1;
   if (tiles / units >= 8) return 1;  // many full waves: the last one is a few per cent at most; keep the plain kernel
@@ -385,6 +387,7 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   // out (measured: +0.5 to +2.5 % on the 470 MB output of the projection shape, neutral on 134 MB)
   p.l2_hint_d = static_cast<double>(d.M) * d.N * d.batch_count * elem_bytes(d.c_dtype) > 64.0e6 ? 1 : 0;
   p.a_tri = (d.flags & GEMM_FLAG_A_LOWER) ? 1 : ((d.flags & GEMM_FLAG_A_UPPER) ? 2 : 0);
+  p.b_tri = (d.structure & GEMM_STRUCT_B_LOWER) ? 1 : ((d.structure & GEMM_STRUCT_B_UPPER) ? 2 : 0);
   p.tile_list = nullptr;  // the device copy of the list is made by gemm_plan
   p.list_len = d_tri ? static_cast<int>(num_tiles / d.batch_count) : 0;
   pl->d_tri = d_tri;
@@ -438,7 +441,7 @@ gemm_status_t plan_wide(gemm_plan_s* pl, int forced_raster, int forced_stages) {
   const gemm_desc_t& d = pl->d;
   // its epilogue covers the bias per column, ReLU and erf GELU only; its MMA schedule has no K-range skipping
   if (d.epilogue > GEMM_EPI_BIAS_GELU_ERF || (d.flags & (GEMM_FLAG_BIAS_PER_ROW | GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER))) return GEMM_ERR_UNSUPPORTED;
-  if (d_tri_of(d)) return GEMM_ERR_UNSUPPORTED;  // its scheduler has no tile list
+  if (d_tri_of(d) || d.structure) return GEMM_ERR_UNSUPPORTED;  // its scheduler has no tile list, its MMA schedule no K ranges
   const int a_kmajor = d.transa == GEMM_OP_N;
   const int b_kmajor = d.transb == GEMM_OP_T;
   const int tile_m = 2 * kWideCtaM, bn = kWideTileN;
@@ -526,7 +529,7 @@ gemm_status_t plan_skinny(gemm_plan_s* pl, int forced_stages, int forced_atoms) 
   if (d.transa != GEMM_OP_N || d.transb != GEMM_OP_T) return GEMM_ERR_UNSUPPORTED;  // both operands K-contiguous
   if ((d.M > kSkinnyMaxM && d.N > kSkinnyMaxM) || d.batch_count != 1) return GEMM_ERR_UNSUPPORTED;
   if (d.flags & (GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER)) return GEMM_ERR_UNSUPPORTED;  // no K-range skipping in stream-K
-  if (d_tri_of(d)) return GEMM_ERR_UNSUPPORTED;  // a short extent of 64 has a single tile row or column: nothing to leave out
+  if (d_tri_of(d) || d.structure) return GEMM_ERR_UNSUPPORTED;  // a short extent of 64 has a single tile row or column: nothing to leave out
   SkinnyPlan& s = pl->skinny;
   pl->skinny_tall = d.M > kSkinnyMaxM;  // the short extent is N: A is streamed, B is the resident slab
   const int small_extent = static_cast<int>(pl->skinny_tall ? d.N : d.M), big_extent = static_cast<int>(pl->skinny_tall ? d.M : d.N);
@@ -623,7 +626,7 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
     // memory-bound problems with a handful of rows stream the weight matrix once: stream-K path;
     // everything else is a dense tiled GEMM, paired CTAs when there are at least two tile rows
     const bool skinny_ok = (d.M <= kSkinnyMaxM || d.N <= kSkinnyMaxM) && d.batch_count == 1 && d.transa == GEMM_OP_N &&
-                           d.transb == GEMM_OP_T && !(d.flags & (GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER)) && !d_tri_of(d);
+                           d.transb == GEMM_OP_T && !(d.flags & (GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER)) && !d_tri_of(d) && !d.structure;
     if (skinny_ok && info.intensity < 7.0 * kRidgeCudaCore) {
       variant = GEMM_VARIANT_SKINNY_STREAMK;  // measured: level with the dense kernels at a short extent of 64 on the largest shapes, far ahead elsewhere
     } else {
@@ -634,7 +637,7 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
         for (int bn : {256, 128, 64}) {
           if (v == GEMM_VARIANT_DENSE_2CTA_WIDE && bn != kWideTileN) continue;
           if (v == GEMM_VARIANT_DENSE_2CTA_WIDE &&
-              (d.epilogue > GEMM_EPI_BIAS_GELU_ERF || d_tri_of(d) ||
+              (d.epilogue > GEMM_EPI_BIAS_GELU_ERF || d_tri_of(d) || d.structure ||
                (d.flags & (GEMM_FLAG_BIAS_PER_ROW | GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER))))
             continue;
           if (v == GEMM_VARIANT_DENSE_2CTA && !b_kmajor && bn % 128) continue;  // 64-column boxes per CTA

@@ -56,8 +56,8 @@ extern "C" gemm_status_t gemm_host_create(const gemm_desc_t* desc, int panels, g
   *out = nullptr;
   if (desc->struct_size != sizeof(gemm_desc_t) || panels < 0) return GEMM_ERR_INVALID_ARG;
   if (desc->transa != GEMM_OP_N || desc->batch_count != 1) return GEMM_ERR_UNSUPPORTED;
-  // a triangular op(A) would have a different diagonal position in every row panel
-  if (desc->flags & (GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER)) return GEMM_ERR_UNSUPPORTED;
+  // a triangular op(A), or a wanted triangle of D, would have a different diagonal position in every row panel
+  if ((desc->flags & (GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER | GEMM_FLAG_D_LOWER | GEMM_FLAG_D_UPPER)) || desc->structure) return GEMM_ERR_UNSUPPORTED;
   gemm_host_s* h = new (std::nothrow) gemm_host_s();
   if (!h) return GEMM_ERR_CUDA;
   memset(h, 0, sizeof *h);

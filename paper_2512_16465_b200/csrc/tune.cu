@@ -17,12 +17,12 @@ namespace b200 {
 namespace {
 
 using Key = std::tuple<int, int64_t, int64_t, int64_t, int32_t, int32_t, int32_t, int32_t, int64_t, int64_t, int64_t, int32_t, int32_t,
-                       int64_t, int64_t, int64_t, uint32_t>;
+                       int64_t, int64_t, int64_t, uint32_t, uint32_t>;
 
 Key key_of(const gemm_desc_t& d, int device) {
   const bool batched = d.batch_count > 1;
   return Key(device, d.M, d.N, d.K, d.transa, d.transb, d.ab_dtype, d.c_dtype, d.lda, d.ldb, d.ldc, d.batch_count, d.epilogue,
-             batched ? d.stride_a : 0, batched ? d.stride_b : 0, batched ? d.stride_c : 0, d.flags & ~kTuningFlagMask);
+             batched ? d.stride_a : 0, batched ? d.stride_b : 0, batched ? d.stride_c : 0, d.flags & ~kTuningFlagMask, d.structure);
 }
 
 std::mutex g_mu;

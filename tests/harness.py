@@ -63,7 +63,8 @@ def desc_of(w: wl.Workload, flags: int = 0, c_dtype=None) -> bg.Desc:
     cd = w.c_dtype if c_dtype is None else c_dtype
     return bg.make_desc(w.M, w.N, w.K, w.transa, w.transb, w.ab_dtype, cd, w.lda, w.ldb, w.ldc, w.batch,
                         w.stride_a, w.stride_b, w.stride_c, w.epilogue, flags | bg.make_flags(bias_per_row=w.bias_per_row, a_lower=w.a_tri == 1, a_upper=w.a_tri == 2,
-                                                                                           d_lower=w.d_tri == 1, d_upper=w.d_tri == 2))
+                                                                                           d_lower=w.d_tri == 1, d_upper=w.d_tri == 2),
+                        structure=w.b_tri)
 
 
 def problem_of(w: wl.Workload, c_dtype=None) -> oracle.Problem:

@@ -162,6 +162,20 @@ EXACT_CASES = [
     ("d_lower_two_epilogue_groups", 2048, 2048, 256, dict(d_tri=1, cd=wl.BF16), dict(variant=V1, tile_n=256)),
     ("d_lower_auto", 2304, 2304, 520, dict(d_tri=1, cd=wl.BF16), dict()),
     ("d_upper_auto_tail_split_requested", 1024, 1024, 2048, dict(d_tri=2), dict(tail_split=True)),
+    # triangular op(B): K ranges cut from the column side; with a triangular op(A) and the matching triangle of D this
+    # is the product of two triangular matrices
+    ("b_upper_1cta", 520, 700, 712, dict(b_tri=2), dict(variant=V1, tile_n=128)),
+    ("b_lower_1cta", 520, 700, 712, dict(b_tri=1), dict(variant=V1, tile_n=64)),
+    ("b_upper_pair_k_shorter", 520, 1000, 328, dict(b_tri=2), dict(variant=V2, tile_n=256)),
+    ("b_lower_pair_k_longer", 520, 456, 1000, dict(b_tri=1), dict(variant=V2, tile_n=128)),
+    ("b_lower_stored_k_by_n", 264, 712, 520, dict(b_tri=1, tb=0), dict(variant=V1, tile_n=128)),
+    ("b_upper_one_slice_stages_forward", 520, 712, 712, dict(b_tri=2), dict(variant=V2, tile_n=128, kslices=1, no_k_serpentine=True)),
+    ("upper_times_upper", 1104, 1104, 1104, dict(a_tri=2, b_tri=2, d_tri=2, cd=wl.BF16), dict(variant=V2, tile_n=128)),
+    ("lower_times_lower", 1104, 1104, 1104, dict(a_tri=1, b_tri=1, d_tri=1), dict(variant=V1, tile_n=128)),
+    ("upper_times_upper_full_d", 712, 712, 712, dict(a_tri=2, b_tri=2), dict(variant=V2, tile_n=256)),
+    ("lower_a_upper_b", 712, 712, 712, dict(a_tri=1, b_tri=2, epi=bg.EPI_BIAS, beta=1.0), dict(variant=V1, tile_n=128)),
+    ("upper_times_upper_batched_fp8", 384, 384, 384, dict(a_tri=2, b_tri=2, d_tri=2, batch=3, ab=wl.FP8_E4M3), dict(variant=V1, tile_n=64)),
+    ("upper_times_upper_auto", 2048, 2048, 2048, dict(a_tri=2, b_tri=2, d_tri=2, cd=wl.BF16), dict()),
     # mirrored stream-K: a tall output with a handful of columns (A is the streamed operand)
     ("tall_one_unit", 128, 8, 64, {}, dict(variant=VS)),
     ("tall_split_k", 256, 8, 4096, {}, dict(variant=VS)),
@@ -508,6 +522,27 @@ def test_triangular_a_really_skips():
         with pytest.raises(bg.GemmError) as e:
             bg.gemm_plan(H.desc_of(int_workload("tri_refused", 8 if bad["variant"] == VS else 1024, 1024, 4096, a_tri=1), bg.make_flags(**bad)))
         assert e.value.status == bg.ERR_UNSUPPORTED
+
+
+def test_triangular_b_really_skips():
+    """Upper-triangular op(B), 512 x 512 (stored N x K): every kernel variant works on tile columns of at most 256 and
+    ring stages of at most 128 elements of K, so element (k, j) with k >= 256 (j // 256 + 1) lies in a stage no tile
+    may visit.  NaN there must not reach the output.  Upper times upper with the lower tiles of D below the diagonal
+    computed all the same (full D): they come out as exact zeros."""
+    w = int_workload("b_tri_skip", 264, 512, 512, b_tri=2)
+    inputs = wl.make_inputs(w)
+    bm = inputs["B"].reshape(512, 512)                    # row j holds op(B)[:, j]
+    for j in range(512):
+        bm[j, 256 * (j // 256 + 1):] = 0x7FC0             # bf16 NaN
+    for fl in (dict(variant=V1, tile_n=128), dict(variant=V2, tile_n=128), dict()):
+        cbits, info = H.run_gpu(w, inputs, bg.make_flags(**fl))
+        clean = wl.make_inputs(w)
+        reports = H.check_blocks(w, clean, cbits, H.default_blocks(w))
+        assert all(r["bit_identical"] == 1.0 and r["finite"] for r in reports), info
+    w = int_workload("upper_upper_zero_tiles", 1024, 1024, 1024, a_tri=2, b_tri=2)
+    cbits, _ = H.run_gpu(w, wl.make_inputs(w), bg.make_flags(variant=V2, tile_n=128))
+    got = cbits.reshape(1024, 1024)
+    assert np.all(got[np.tril_indices(1024, -1)] == 0.0) and np.any(got[np.triu_indices(1024)] != 0.0)
 
 
 @pytest.mark.parametrize("d_tri", [1, 2])

@@ -29,8 +29,8 @@ def test_every_declared_symbol_is_exported():
 
 
 def test_struct_layouts_match_the_header():
-    # 2 x u32, 3 x i64, 4 x i32, 3 x i64, 2 x i32, 3 x i64
-    assert ctypes.sizeof(bg.Desc) == 8 + 24 + 16 + 24 + 8 + 24
+    # 2 x u32, 3 x i64, 4 x i32, 3 x i64, 2 x i32, 3 x i64, 2 x u32
+    assert ctypes.sizeof(bg.Desc) == 8 + 24 + 16 + 24 + 8 + 24 + 8 and bg.Desc.structure.offset == 104
     assert bg.Desc.M.offset == 8 and bg.Desc.lda.offset == 48 and bg.Desc.batch_count.offset == 72
     assert bg.Desc.stride_a.offset == 80
     assert bg.Info.num_tiles.offset == 48 and bg.Info.flops.offset == 56
@@ -208,6 +208,23 @@ def test_triangular_result_plans():
     with pytest.raises(bg.GemmError) as e:
         bg.gemm_plan(bg.make_desc(512, 512, 512, flags=bg.make_flags(d_lower=True, d_upper=True)))
     assert e.value.status == bg.ERR_INVALID_ARG
+    # structure of op(B): unknown bits, both triangles at once and a non-zero reserved word are invalid; the kernels
+    # without K ranges refuse it; it keeps a short output away from stream-K as well
+    for structure in (0x4, bg.STRUCT_B_LOWER | bg.STRUCT_B_UPPER):
+        with pytest.raises(bg.GemmError) as e:
+            bg.gemm_plan(bg.make_desc(512, 512, 512, structure=structure))
+        assert e.value.status == bg.ERR_INVALID_ARG
+    d = bg.make_desc(512, 512, 512)
+    d.reserved = 1
+    with pytest.raises(bg.GemmError) as e:
+        bg.gemm_plan(d)
+    assert e.value.status == bg.ERR_INVALID_ARG
+    for v, M in ((bg.VARIANT_DENSE_2CTA_WIDE, 4096), (bg.VARIANT_SKINNY_STREAMK, 64)):
+        with pytest.raises(bg.GemmError) as e:
+            bg.gemm_plan(bg.make_desc(M, 4096, 4096, flags=bg.make_flags(variant=v), structure=bg.STRUCT_B_UPPER))
+        assert e.value.status == bg.ERR_UNSUPPORTED
+    assert bg.Plan(bg.make_desc(8192, 8192, 8192, structure=bg.STRUCT_B_LOWER)).info["variant"] == bg.VARIANT_DENSE_2CTA
+    assert bg.Plan(bg.make_desc(64, 8192, 8192, structure=bg.STRUCT_B_UPPER)).info["variant"] != bg.VARIANT_SKINNY_STREAMK
     # a short output that would go to stream-K stays dense when a triangle is asked for
     assert bg.Plan(bg.make_desc(64, 8192, 8192, flags=bg.make_flags(d_upper=True))).info["variant"] != bg.VARIANT_SKINNY_STREAMK
 
@@ -229,7 +246,8 @@ def test_tuning_entry_points_on_the_host():
 
 def test_host_pipeline_entry_points_without_a_device():
     import torch
-    for kw in (dict(transa=bg.OP_T), dict(batch=2), dict(flags=bg.make_flags(a_upper=True))):   # refused before any device work
+    for kw in (dict(transa=bg.OP_T), dict(batch=2), dict(flags=bg.make_flags(a_upper=True)),
+               dict(flags=bg.make_flags(d_lower=True))):   # refused before any device work
         with pytest.raises(bg.GemmError) as e:
             bg.gemm_host_create(bg.make_desc(256, 256, 256, **kw))
         assert e.value.status == bg.ERR_UNSUPPORTED

@@ -93,6 +93,28 @@ def test_triangular_structure_of_a():
     assert wl.Workload("t", 4, 3, 6, a_tri=2).flops == 2.0 * (6 + 5 + 4 + 3) * 3
 
 
+def test_triangular_structure_of_b():
+    for tb in (0, 1):
+        for tri, keep in ((1, np.tril), (2, np.triu)):
+            w = wl.Workload("t", 5, 7, 9, transb=tb, b_tri=tri, batch=2, ldb=12)
+            dense = wl.make_inputs(wl.Workload("t", 5, 7, 9, transb=tb, batch=2, ldb=12))["B"]
+            got = wl.make_inputs(w)["B"]
+            rows, cols = (7, 9) if tb else (9, 7)
+            for b in range(2):
+                g = got[b * w.stride_b: b * w.stride_b + rows * 12].reshape(rows, 12)[:, :cols]
+                d = dense[b * w.stride_b: b * w.stride_b + rows * 12].reshape(rows, 12)[:, :cols]
+                op_g, op_d = (g.T, d.T) if tb else (g, d)          # op(B) is K x N = 9 x 7
+                assert np.array_equal(op_g, keep(op_d))
+    # useful work, brute force over (i, k, j): neither factor a structural zero, output wanted
+    for M, N, K, a, b, d in ((5, 6, 7, 2, 2, 2), (6, 6, 6, 1, 1, 1), (4, 9, 5, 2, 1, 0), (9, 4, 5, 0, 2, 1), (3, 3, 3, 0, 1, 0)):
+        cnt = sum(1 for i in range(M) for j in range(N) for k in range(K)
+                  if not (d == 1 and i < j) and not (d == 2 and i > j) and not (a == 1 and k > i) and not (a == 2 and k < i)
+                  and not (b == 1 and k < j) and not (b == 2 and k > j))
+        assert wl.Workload("t", M, N, K, a_tri=a, b_tri=b, d_tri=d).flops == 2.0 * cnt
+    # the product of two upper triangular n x n matrices costs n (n + 1) (n + 2) / 6 multiply-adds
+    assert wl.Workload("t", 50, 50, 50, a_tri=2, b_tri=2, d_tri=2).flops == 2.0 * 50 * 51 * 52 / 6
+
+
 def test_useful_work_of_a_triangular_result():
     # wanted elements of D, two flops per element and k: 4 x 4 lower = 10, 4 x 6 upper = 6 + 5 + 4 + 3, 6 x 4 lower = 10 + 2 * 4
     assert wl.Workload("t", 4, 4, 5, d_tri=1).flops == 2.0 * 10 * 5

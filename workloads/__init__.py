@@ -17,6 +17,7 @@ import ctypes
 import os
 import subprocess
 from dataclasses import dataclass, field, replace
+from functools import lru_cache
 
 import numpy as np
 
@@ -111,6 +112,7 @@ class Workload:
     epilogue: int = EPI_NONE
     bias_per_row: bool = False   # the bias has M entries (one per output row) instead of N
     a_tri: int = 0               # structure of op(A): 0 dense, 1 lower triangular (zero for k > i), 2 upper (zero for k < i)
+    b_tri: int = 0               # structure of op(B): 0 dense, 1 lower triangular (zero for k < j), 2 upper (zero for k > j)
     d_tri: int = 0               # part of D that is wanted: 0 all, 1 lower triangle (row >= column), 2 upper (row <= column)
     alpha: float = 1.0
     beta: float = 0.0
@@ -151,21 +153,9 @@ class Workload:
 
     @property
     def flops(self) -> float:
-        """Useful work: two flops per (non-zero element of op(A) in row i) x (wanted output column of row i)."""
-        i = np.arange(self.M, dtype=np.int64)
-        if self.a_tri == 1:
-            nz = np.minimum(i + 1, self.K)
-        elif self.a_tri == 2:
-            nz = np.maximum(self.K - i, 0)
-        else:
-            nz = np.full(self.M, self.K, dtype=np.int64)
-        if self.d_tri == 1:
-            cols = np.minimum(i + 1, self.N)
-        elif self.d_tri == 2:
-            cols = np.maximum(self.N - i, 0)
-        else:
-            cols = np.full(self.M, self.N, dtype=np.int64)
-        return 2.0 * float(np.sum(nz * cols)) * self.batch
+        """Useful work: two flops per product a(i,k) b(k,j) in which neither factor is a structural zero, over the
+        wanted outputs (i, j)."""
+        return 2.0 * _useful_products(self.M, self.N, self.K, self.a_tri, self.b_tri, self.d_tri) * self.batch
 
     @property
     def min_bytes(self) -> float:
@@ -187,6 +177,32 @@ class Workload:
 
     def elems_c(self) -> int:
         return (self.batch - 1) * self.stride_c + self.M * self.ldc
+
+
+@lru_cache(maxsize=256)
+def _useful_products(M: int, N: int, K: int, a_tri: int, b_tri: int, d_tri: int) -> float:
+    """Number of (i, k, j) with a(i,k) and b(k,j) not structurally zero and output (i, j) wanted.  Row i of op(A)
+    keeps k in [alo_i, ahi_i), column j of op(B) keeps k in [blo_j, bhi_j); the count is the summed overlap."""
+    i = np.arange(M, dtype=np.int64)
+    alo = np.minimum(i, K) if a_tri == 2 else np.zeros(M, np.int64)
+    ahi = np.minimum(i + 1, K) if a_tri == 1 else np.full(M, K, np.int64)
+    if not b_tri:   # every column keeps all of K: rows x wanted columns
+        cols = np.minimum(i + 1, N) if d_tri == 1 else (np.maximum(N - i, 0) if d_tri == 2 else np.full(M, N, np.int64))
+        return float(np.sum((ahi - alo) * cols))
+    j = np.arange(N, dtype=np.int64)
+    blo = np.minimum(j, K) if b_tri == 1 else np.zeros(N, np.int64)
+    bhi = np.minimum(j + 1, K) if b_tri == 2 else np.full(N, K, np.int64)
+    total = 0.0
+    for r0 in range(0, M, 512):          # row blocks keep the M x N intermediate small
+        r = slice(r0, min(r0 + 512, M))
+        ov = np.minimum(ahi[r, None], bhi[None, :]) - np.maximum(alo[r, None], blo[None, :])
+        np.maximum(ov, 0, out=ov)
+        if d_tri == 1:
+            ov[i[r, None] < j[None, :]] = 0
+        elif d_tri == 2:
+            ov[i[r, None] > j[None, :]] = 0
+        total += float(ov.sum())
+    return total
 
 
 def _draw(dist: Dist, seed, tensor_id, n, dtype):
@@ -213,6 +229,20 @@ def _zero_triangle(a: np.ndarray, w: Workload) -> None:
                 a[off + k * w.lda + lo: off + k * w.lda + hi] = 0
 
 
+def _zero_triangle_b(bm: np.ndarray, w: Workload) -> None:
+    """Same for op(B) (K x N): lower keeps k >= j, upper keeps k <= j."""
+    for b in range(w.batch):
+        off = b * w.stride_b
+        if not w.transb:          # stored K x N: row k holds op(B)[k, :]
+            for k in range(w.K):
+                lo, hi = (min(k + 1, w.N), w.N) if w.b_tri == 1 else (0, min(k, w.N))
+                bm[off + k * w.ldb + lo: off + k * w.ldb + hi] = 0
+        else:                     # stored N x K: row j holds op(B)[:, j]
+            for j in range(w.N):
+                lo, hi = (0, min(j, w.K)) if w.b_tri == 1 else (min(j + 1, w.K), w.K)
+                bm[off + j * w.ldb + lo: off + j * w.ldb + hi] = 0
+
+
 def make_inputs(w: Workload, seed_offset: int = 0) -> dict:
     """Draw A, B and, when used, C_in and bias for ``w``.  ``seed_offset`` gives the
     benchmark its rotating "different random inputs" sets."""
@@ -222,6 +252,8 @@ def make_inputs(w: Workload, seed_offset: int = 0) -> dict:
            "C": None, "bias": None}
     if w.a_tri:
         _zero_triangle(out["A"], w)
+    if w.b_tri:
+        _zero_triangle_b(out["B"], w)
     if w.beta != 0.0:
         out["C"] = _draw(w.dist_c, s, TENSOR_C, w.elems_c(), w.c_dtype)
     if w.has_bias:
