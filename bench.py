@@ -500,9 +500,13 @@ def run_shapes(args):
                                 "candidates_tried": rep["candidates_tried"], "candidates_skipped": rep["candidates_skipped"],
                                 "tuner_auto_ms": round(rep["auto_ms"], 5), "tuner_best_ms": round(rep["best_ms"], 5),
                                 "roofline_frac": roofline_for(w, spec, sec2, peaks, peak_kind)["frac"]}
-                bg.gemm_tune_cache_clear()
+                if not args.tune_file:
+                    bg.gemm_tune_cache_clear()
             rows.append(row)
             case.close()
+    if args.tune and args.tune_file:   # keep the measured choices: gemm_tune_cache_load brings them back in another process
+        print(f"[bench] {bg.gemm_tune_cache_save(args.tune_file)} tuning results written to {args.tune_file}", file=sys.stderr)
+        bg.gemm_tune_cache_clear()
     print(json.dumps({"shapes_measured": rows, "steps": steps, "warmup": warmup, "clocks": clocks.summary(),
                       "timing": "CUDA events around back-to-back launches; inputs rotate so that each step's footprint exceeds L2"}), flush=True)
 
@@ -566,6 +570,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--ref-step-seconds", type=float, default=10.0, help="--impl reference: CPU time budget of one step")
     ap.add_argument("--shapes", default="", help="';'-separated MxNxK[:key=value...] problems to time instead of the five configurations")
+    ap.add_argument("--tune-file", default="", help="--shapes --tune: write the measured choices to this file (gemm_tune_cache_save)")
     ap.add_argument("--tune", action="store_true", help="--shapes: also plan by measurement (gemm_tune) and time the tuned plan")
     ap.add_argument("--library-reference", action="store_true", help="--shapes: also time torch.matmul on the same operands (context)")
     args = ap.parse_args()

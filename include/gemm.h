@@ -299,6 +299,18 @@ gemm_status_t gemm_tune(const gemm_desc_t* desc, const void* A, const void* B, v
 void gemm_tune_cache_clear(void);
 
 /*
+ * Keep tuning results across processes (the paper's search runs once per operator and hardware, Section 4; this is the
+ * memory of that search).  gemm_tune_cache_save writes what was remembered for the CURRENT device to a text file
+ * (overwriting it); gemm_tune_cache_load adds the file's results to the current device's, after which gemm_plan picks
+ * them up like results of gemm_tune in this process.  path: host string.  *entries (may be NULL): results written /
+ * read.  Errors: GEMM_ERR_NULL; GEMM_ERR_ARCH without a CUDA device; GEMM_ERR_INVALID_ARG when the file cannot be
+ * opened or is malformed (nothing is loaded then); GEMM_ERR_UNSUPPORTED when the file was written on another GPU
+ * model or SM count.  A remembered choice that this version of the library cannot plan is ignored by gemm_plan.
+ */
+gemm_status_t gemm_tune_cache_save(const char* path, int* entries);
+gemm_status_t gemm_tune_cache_load(const char* path, int* entries);
+
+/*
  * GEMM on HOST-resident operands (the end-to-end path of a caller whose matrices live in host memory; the
  * paper's measurements start with the data on the GPU, so this has no counterpart there).  The output rows are cut
  * into `panels` row panels; panel p's slice of A is copied in while panel p-1 is multiplied and panel p-2's result is

@@ -76,7 +76,7 @@ class TuneReport(ctypes.Structure):
 
 EXPORTS = ("gemm_plan", "gemm_workspace_bytes", "gemm_run", "gemm_plan_status", "gemm_plan_set_timeout_ms",
            "gemm_plan_info", "gemm_destroy", "gemm_status_string", "gemm_last_cuda_error", "gemm_skinny_run_noalloc",
-           "gemm_tune", "gemm_tune_workspace_bytes", "gemm_tune_cache_clear",
+           "gemm_tune", "gemm_tune_workspace_bytes", "gemm_tune_cache_clear", "gemm_tune_cache_save", "gemm_tune_cache_load",
            "gemm_host_create", "gemm_host_run", "gemm_host_panels", "gemm_host_destroy")
 
 
@@ -113,6 +113,9 @@ def _load() -> ctypes.CDLL:
     L.gemm_tune_workspace_bytes.argtypes = [ctypes.POINTER(Desc)]
     L.gemm_tune_cache_clear.restype = None
     L.gemm_tune_cache_clear.argtypes = []
+    for fn in (L.gemm_tune_cache_save, L.gemm_tune_cache_load):
+        fn.restype = ctypes.c_int
+        fn.argtypes = [ctypes.c_char_p, ctypes.POINTER(ctypes.c_int)]
     L.gemm_host_create.restype = ctypes.c_int
     L.gemm_host_create.argtypes = [ctypes.POINTER(Desc), ctypes.c_int, ctypes.POINTER(vp)]
     L.gemm_host_run.restype = ctypes.c_int
@@ -211,6 +214,24 @@ def gemm_tune(desc: Desc, A: int, B: int, C: int, bias: int, alpha: float, beta:
 
 def gemm_tune_cache_clear() -> None:
     _lib.gemm_tune_cache_clear()
+
+
+def gemm_tune_cache_save(path: str) -> int:
+    """``gemm_tune_cache_save``: write the current device's remembered tuning results to ``path``; returns how many."""
+    n = ctypes.c_int(0)
+    st = _lib.gemm_tune_cache_save(os.fsencode(path), ctypes.byref(n))
+    if st != OK:
+        raise GemmError(st, "gemm_tune_cache_save")
+    return n.value
+
+
+def gemm_tune_cache_load(path: str) -> int:
+    """``gemm_tune_cache_load``: add the results in ``path`` to the current device's; returns how many were read."""
+    n = ctypes.c_int(0)
+    st = _lib.gemm_tune_cache_load(os.fsencode(path), ctypes.byref(n))
+    if st != OK:
+        raise GemmError(st, "gemm_tune_cache_load")
+    return n.value
 
 
 def gemm_host_create(desc: Desc, panels: int = 0) -> int:

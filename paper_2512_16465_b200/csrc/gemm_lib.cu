@@ -561,9 +561,12 @@ gemm_status_t plan_skinny(gemm_plan_s* pl, int forced_stages, int forced_atoms) 
 
 }  // namespace
 
-extern "C" {
+namespace {
 
-gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
+// gemm_plan proper.  use_cache: take the tuning fields gemm_tune remembered for this shape (when the caller set none);
+// *cache_used tells whether that happened.
+gemm_status_t plan_impl(const gemm_desc_t* desc, gemm_plan_t* out_plan, bool use_cache, bool* cache_used) {
+  *cache_used = false;
   if (!desc || !out_plan) return GEMM_ERR_NULL;
   *out_plan = nullptr;
   gemm_status_t st = validate(desc);
@@ -587,9 +590,12 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
     }
   }
   (void)cudaGetLastError();
-  if (pl->has_device && (pl->d.flags & kTuningFlagMask) == 0) {  // a measured choice for this shape, if gemm_tune made one
+  if (use_cache && pl->has_device && (pl->d.flags & kTuningFlagMask) == 0) {  // a measured choice for this shape, if gemm_tune made one
     uint32_t tuned = 0;
-    if (tune_cache_lookup(pl->d, pl->device, &tuned)) pl->d.flags |= tuned;
+    if (tune_cache_lookup(pl->d, pl->device, &tuned) && tuned != 0) {
+      pl->d.flags |= tuned;
+      *cache_used = true;
+    }
   }
 
   // roofline class (Section 4.3): compulsory traffic vs. work
@@ -693,6 +699,18 @@ gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
   }
   *out_plan = pl;
   return GEMM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan) {
+  bool cache_used = false;
+  gemm_status_t st = plan_impl(desc, out_plan, true, &cache_used);
+  // remembered tuning fields that do not plan (a file from another version of the library) must not break the problem
+  if (st != GEMM_OK && cache_used) st = plan_impl(desc, out_plan, false, &cache_used);
+  return st;
 }
 
 size_t gemm_workspace_bytes(gemm_plan_t plan) { return plan ? plan->info.workspace_bytes : 0; }

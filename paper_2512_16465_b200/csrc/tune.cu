@@ -4,10 +4,12 @@
 // bound ones for tensor-pipe occupancy); the winner is remembered per device and shape.
 #include <cuda_runtime.h>
 
+#include <cstdio>
 #include <cstring>
 #include <map>
 #include <mutex>
 #include <tuple>
+#include <utility>
 #include <vector>
 
 #include "../../include/gemm.h"
@@ -146,6 +148,98 @@ using namespace b200;
 extern "C" void gemm_tune_cache_clear(void) {
   std::lock_guard<std::mutex> lock(g_mu);
   cache().clear();
+}
+
+// ---- keeping tuning results across processes -------------------------------------------------------------------
+// A text file: one header line, then one line per remembered shape with the sixteen key fields after the device
+// and the chosen tuning flags.  Results are written for, and read into, the current device: a file made on one GPU
+// model means nothing on another, so the header carries the device name and the SM count and a mismatch is refused.
+namespace {
+
+constexpr const char* kTuneFileMagic = "b200gemm-tune-1";
+
+bool current_device_tag(int* device, char* name, size_t len, int* sms) {
+  cudaDeviceProp prop;
+  if (cudaGetDevice(device) != cudaSuccess || cudaGetDeviceProperties(&prop, *device) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return false;
+  }
+  snprintf(name, len, "%s", prop.name);
+  for (char* c = name; *c; ++c)
+    if (*c == ' ') *c = '_';
+  *sms = prop.multiProcessorCount;
+  return true;
+}
+
+}  // namespace
+
+extern "C" gemm_status_t gemm_tune_cache_save(const char* path, int* entries) {
+  if (!path) return GEMM_ERR_NULL;
+  if (entries) *entries = 0;
+  int device = -1, sms = 0;
+  char name[256];
+  if (!current_device_tag(&device, name, sizeof name, &sms)) return GEMM_ERR_ARCH;
+  FILE* f = fopen(path, "w");
+  if (!f) return GEMM_ERR_INVALID_ARG;
+  int n = 0;
+  bool ok = fprintf(f, "%s %s %d\n", kTuneFileMagic, name, sms) > 0;
+  {
+    std::lock_guard<std::mutex> lock(g_mu);
+    for (const auto& kv : cache()) {
+      const Key& k = kv.first;
+      if (std::get<0>(k) != device) continue;
+      ok = ok && fprintf(f, "%lld %lld %lld %d %d %d %d %lld %lld %lld %d %d %lld %lld %lld %u %u %u\n",
+                         (long long)std::get<1>(k), (long long)std::get<2>(k), (long long)std::get<3>(k), std::get<4>(k), std::get<5>(k),
+                         std::get<6>(k), std::get<7>(k), (long long)std::get<8>(k), (long long)std::get<9>(k), (long long)std::get<10>(k),
+                         std::get<11>(k), std::get<12>(k), (long long)std::get<13>(k), (long long)std::get<14>(k),
+                         (long long)std::get<15>(k), std::get<16>(k), std::get<17>(k), kv.second) > 0;
+      ++n;
+    }
+  }
+  ok = (fclose(f) == 0) && ok;
+  if (!ok) return GEMM_ERR_INVALID_ARG;
+  if (entries) *entries = n;
+  return GEMM_OK;
+}
+
+extern "C" gemm_status_t gemm_tune_cache_load(const char* path, int* entries) {
+  if (!path) return GEMM_ERR_NULL;
+  if (entries) *entries = 0;
+  int device = -1, sms = 0;
+  char name[256];
+  if (!current_device_tag(&device, name, sizeof name, &sms)) return GEMM_ERR_ARCH;
+  FILE* f = fopen(path, "r");
+  if (!f) return GEMM_ERR_INVALID_ARG;
+  char magic[64], file_name[256];
+  int file_sms = 0;
+  if (fscanf(f, "%63s %255s %d", magic, file_name, &file_sms) != 3 || strcmp(magic, kTuneFileMagic) != 0) {
+    fclose(f);
+    return GEMM_ERR_INVALID_ARG;
+  }
+  if (strcmp(file_name, name) != 0 || file_sms != sms) {  // measured on another kind of GPU
+    fclose(f);
+    return GEMM_ERR_UNSUPPORTED;
+  }
+  // read everything first: a malformed file changes nothing
+  std::vector<std::pair<Key, uint32_t>> read;
+  while (true) {
+    long long M, N, K, lda, ldb, ldc, sa, sb, sc;
+    int ta, tb, ab, cd, batch, epi;
+    unsigned flags, structure, tuned;
+    const int got = fscanf(f, "%lld %lld %lld %d %d %d %d %lld %lld %lld %d %d %lld %lld %lld %u %u %u", &M, &N, &K, &ta, &tb, &ab, &cd,
+                           &lda, &ldb, &ldc, &batch, &epi, &sa, &sb, &sc, &flags, &structure, &tuned);
+    if (got == EOF) break;
+    if (got != 18 || (tuned & ~kTuningFlagMask) || (flags & kTuningFlagMask) || M < 1 || N < 1 || K < 1 || batch < 1) {
+      fclose(f);
+      return GEMM_ERR_INVALID_ARG;
+    }
+    read.emplace_back(Key(device, M, N, K, ta, tb, ab, cd, lda, ldb, ldc, batch, epi, sa, sb, sc, flags, structure), tuned);
+  }
+  fclose(f);
+  std::lock_guard<std::mutex> lock(g_mu);
+  for (const auto& kv : read) cache()[kv.first] = kv.second;
+  if (entries) *entries = static_cast<int>(read.size());
+  return GEMM_OK;
 }
 
 extern "C" size_t gemm_tune_workspace_bytes(const gemm_desc_t* desc) {

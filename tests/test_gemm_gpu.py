@@ -682,6 +682,70 @@ def test_tune_short_extent_tries_stream_k_and_dense():
     bg.gemm_tune_cache_clear()
 
 
+def test_tuning_results_survive_in_a_file(tmp_path):
+    """Save after tuning, forget, load: gemm_plan makes the tuned plan again.  A file from another GPU model is refused,
+    a malformed one loads nothing, and a remembered choice that cannot be planned is ignored."""
+    bg.gemm_tune_cache_clear()
+    keys = ("variant", "tile_m", "tile_n", "tile_k", "stages", "raster_group", "grid")
+    w = int_workload("tune_file", 1024, 1536, 512, cd=wl.BF16)
+    inputs, A, B, C, desc, plan, rep = _tune_case(w)
+    # a second shape with a forced, distinctive winner: remember "1-CTA, tile N 64, raster 3" for it by hand
+    path = str(tmp_path / "tune.txt")
+    assert bg.gemm_tune_cache_save(path) == 1
+    lines = open(path).read().splitlines()
+    assert lines[0].startswith("b200gemm-tune-1 ") and len(lines) == 2 and len(lines[1].split()) == 18
+    odd = bg.make_flags(V1, 64, raster=3)
+    fields = lines[1].split()
+    fields[0:3] = ["640", "768", "256"]                        # M N K
+    fields[7:10] = ["256", "256", "768"]                       # lda ldb ldc (tight, transb = T)
+    fields[12:15] = ["0", "0", "0"]
+    fields[17] = str(odd)
+    with open(path, "a") as f:
+        f.write(" ".join(fields) + "\n")
+    bg.gemm_tune_cache_clear()
+    auto = bg.Plan(desc)
+    assert bg.gemm_tune_cache_load(path) == 2
+    again = bg.Plan(desc)
+    assert {k: again.info[k] for k in keys} == {k: plan.info[k] for k in keys}
+    hand = bg.Plan(bg.make_desc(640, 768, 256, c_dtype=bg.BF16))
+    assert (hand.info["variant"], hand.info["tile_n"], hand.info["raster_group"]) == (V1, 64, 3)
+    w2 = int_workload("tune_file_hand", 640, 768, 256, cd=wl.BF16)
+    H.check_workload(w2, exact=True)                           # runs through that remembered plan
+    for p in (auto, again, hand, plan):
+        p.close()
+    # another GPU model / SM count: refused; nothing changes
+    other = str(tmp_path / "other.txt")
+    head = lines[0].split()
+    open(other, "w").write(" ".join([head[0], head[1], str(int(head[2]) + 1)]) + "\n" + lines[1] + "\n")
+    bg.gemm_tune_cache_clear()
+    with pytest.raises(bg.GemmError) as e:
+        bg.gemm_tune_cache_load(other)
+    assert e.value.status == bg.ERR_UNSUPPORTED
+    # malformed: a short line, tuning bits outside the tuning fields, a wrong magic word, a missing file
+    for text in (lines[0] + "\n" + lines[1] + "\n1 2 3\n", lines[0] + "\n" + " ".join(fields[:17] + ["1"]) + "\n", "something else\n"):
+        bad = str(tmp_path / "bad.txt")
+        open(bad, "w").write(text)
+        with pytest.raises(bg.GemmError) as e:
+            bg.gemm_tune_cache_load(bad)
+        assert e.value.status == bg.ERR_INVALID_ARG
+    with pytest.raises(bg.GemmError) as e:
+        bg.gemm_tune_cache_load(str(tmp_path / "missing.txt"))
+    assert e.value.status == bg.ERR_INVALID_ARG
+    assert bg.gemm_tune_cache_save(str(tmp_path / "empty.txt")) == 0        # nothing was loaded by the failed attempts
+    # a remembered choice this library cannot plan for the shape (the wide pair kernel has no SiLU epilogue): ignored
+    fields[0:3] = ["1024", "1024", "512"]
+    fields[7:10] = ["512", "512", "1024"]
+    fields[11] = str(bg.EPI_SILU)
+    fields[17] = str(bg.make_flags(VW))
+    stale = str(tmp_path / "stale.txt")
+    open(stale, "w").write(lines[0] + "\n" + " ".join(fields) + "\n")
+    assert bg.gemm_tune_cache_load(stale) == 1
+    p = bg.Plan(bg.make_desc(1024, 1024, 512, c_dtype=bg.BF16, epilogue=bg.EPI_SILU))
+    assert p.info["variant"] != VW
+    p.close()
+    bg.gemm_tune_cache_clear()
+
+
 def test_tune_argument_errors():
     d = bg.make_desc(256, 256, 64)
     with pytest.raises(bg.GemmError) as e:

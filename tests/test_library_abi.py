@@ -242,6 +242,11 @@ def test_tuning_entry_points_on_the_host():
         with pytest.raises(bg.GemmError) as e:
             bg.gemm_tune(bg.make_desc(256, 256, 64), 16, 16, 16, 0, 1.0, 0.0, 0, 0, 0)
         assert e.value.status in (bg.ERR_ARCH, bg.ERR_CUDA)                       # no device: an error, never a fallback
+        for fn in (bg.gemm_tune_cache_save, bg.gemm_tune_cache_load):               # results belong to a device
+            with pytest.raises(bg.GemmError) as e:
+                fn("/nonexistent-directory/tune.txt")
+            assert e.value.status == bg.ERR_ARCH
+    assert bg._lib.gemm_tune_cache_save(None, None) == bg.ERR_NULL and bg._lib.gemm_tune_cache_load(None, None) == bg.ERR_NULL
 
 
 def test_host_pipeline_entry_points_without_a_device():
