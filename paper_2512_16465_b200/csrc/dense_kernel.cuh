@@ -55,9 +55,10 @@ struct DenseParams {
   int kblk;                               // elements of K in one 128-byte slice: 64 (16-bit operands) or 128 (8-bit)
   int a_tri;                              // structure of op(A): 0 dense, 1 lower triangular (zero for k > i), 2 upper (zero for k < i)
   int b_tri;                              // structure of op(B): 0 dense, 1 lower triangular (zero for k < j), 2 upper (zero for k > j)
-  // One triangle of D wanted: the tiles that touch it, per matrix and in scheduling order, are listed in device memory
-  // (tile ids of the full tiles_m x tiles_n numbering); num_tiles then counts batch * list_len listed tiles.
-  const int* tile_list;                   // nullptr: every tile is computed
+  // Structured problems (one triangle of D wanted, triangular operands) come with a schedule in device memory: per
+  // matrix, slot k * (CTAs or pairs) + c holds the k-th tile of CTA (pair) c as a tile id of the full tiles_m x tiles_n
+  // numbering, or -1 when it has none; num_tiles then counts batch * list_len slots.
+  const int* tile_list;                   // nullptr: every tile is computed, dealt round-robin
   int list_len;
   // Tail split (kernels built with kSplit): the tiles from split_first_tile on, which would leave most CTAs idle in
   // the last wave, are cut into `split` slices of K each, one work item per slice; num_items counts whole tiles + slices.
@@ -188,9 +189,10 @@ struct WorkItem {
 };
 template <bool kSplit>
 __device__ __forceinline__ int item_tile(const DenseParams& p, int item) {
-  if (p.tile_list != nullptr) {  // (never together with a tail split)
+  if (p.tile_list != nullptr) {  // (never together with a tail split); < 0: an empty slot
     const int b = item / p.list_len;
-    return b * (p.tiles_m * p.tiles_n) + __ldg(p.tile_list + (item - b * p.list_len));
+    const int t = __ldg(p.tile_list + (item - b * p.list_len));
+    return t < 0 ? -1 : b * (p.tiles_m * p.tiles_n) + t;
   }
   if (!kSplit || item < p.split_first_tile) return item;
   return p.split_first_tile + (item - p.split_first_tile) / p.split;
@@ -408,6 +410,10 @@ __device__ __forceinline__ void producer_role(const DenseParams& p, const CUtens
   const int n_items = kSplit ? p.num_items : p.num_tiles;
   for (int item = cluster_id; item < n_items; item += num_clusters, ++it) {
     const int tile = item_tile<kSplit>(p, item);
+    if (tile < 0) {  // an empty slot of a dealt schedule: every role skips it alike, and it does not count as a tile
+      --it;          // (the loop header adds the one back: buffer and phase bookkeeping follow the tiles actually computed)
+      continue;
+    }
     const TileCoord tc = decode_tile(tile, p.tiles_m, p.tiles_n, p.raster_group);
     const int m0 = tc.tm * (kCtaM * CG) + static_cast<int>(cta_rank) * kCtaM;
     const int n0 = tc.tn * p.bn + (CG == 2 ? static_cast<int>(cta_rank) * p.b_rows : 0);
@@ -477,6 +483,10 @@ __device__ __forceinline__ void mma_role(const DenseParams& p, uint32_t tiles_ba
   const int n_items = kSplit ? p.num_items : p.num_tiles;
   for (int item = cluster_id; item < n_items; item += num_clusters, ++it) {
     const int tile = item_tile<kSplit>(p, item);
+    if (tile < 0) {  // an empty slot of a dealt schedule: every role skips it alike, and it does not count as a tile
+      --it;          // (the loop header adds the one back: buffer and phase bookkeeping follow the tiles actually computed)
+      continue;
+    }
     const uint32_t buf = it & 1u;
     const uint32_t aph = (it >> 1) & 1u;
     if (!mbar_wait_warp(tempty0 + 8u * buf, aph ^ 1u, w, (2u << 8) | 0x80u | buf)) return;
@@ -574,6 +584,10 @@ __device__ __forceinline__ void epilogue_role(const DenseParams& p, const CUtens
   const size_t partial_elems = static_cast<size_t>(kCtaM) * p.bn;
   for (int item = cluster_id; item < n_items; item += num_clusters, ++it) {
     const int tile = item_tile<kSplit>(p, item);
+    if (tile < 0) {  // an empty slot of a dealt schedule: every role skips it alike, and it does not count as a tile
+      --it;          // (the loop header adds the one back: buffer and phase bookkeeping follow the tiles actually computed)
+      continue;
+    }
     const TileCoord tc = decode_tile(tile, p.tiles_m, p.tiles_n, p.raster_group);
     const uint32_t buf = it & 1u;
     const uint32_t ph = (it >> 1) & 1u;

@@ -14,6 +14,8 @@
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <queue>
+#include <utility>
 #include <vector>
 
 #include "dense_kernel.cuh"
@@ -116,7 +118,9 @@ struct gemm_plan_s {
   size_t d_counters_bytes = 0;  // plan-owned words after the status word: stream-K arrival counters or tail-split flags
   int split = 1;                // tail split factor of a dense plan
   int d_tri = 0;                // one triangle of D wanted: 1 lower, 2 upper (dense variants)
-  int* d_tile_list = nullptr;   // device: the tiles of one matrix that touch that triangle, in scheduling order
+  int* d_tile_list = nullptr;   // device: the dealt tile schedule of one matrix (structured problems)
+  int* h_tile_list = nullptr;   // host copy, kept from planning until it has been uploaded
+  ~gemm_plan_s() { free(h_tile_list); }
   size_t split_flag_bytes = 0;
   unsigned long long runs = 0;  // launches so far (the timeout test hook acts on the first one only)
   uint32_t timeout_ms;
@@ -194,22 +198,67 @@ long long tri_tile_count(int d_tri, int tile_m, int bn, long long M, long long N
   }
   return n;
 }
-// The listed tiles in the order the scheduler visits the full grid (groups of `raster` tile rows, inside a group
-// column by column with the row running fastest), so the resident tiles still share their A band and B panels.
-std::vector<int> tri_tile_list(int d_tri, int tile_m, int bn, long long M, long long N, int raster) {
-  const int tiles_m = ceil_div(M, tile_m), tiles_n = ceil_div(N, bn);
-  std::vector<int> list;
+// The schedule of a structured problem (one triangle of D wanted, triangular op(A) or op(B)): the tiles of one matrix
+// that are computed at all, dealt out to `units` CTAs (pairs) ahead of time.  The tiles are taken in the order the
+// scheduler visits the full grid (groups of `raster` tile rows, inside a group column by column with the row running
+// fastest, so that tiles in flight together share their A band and B panels) and each goes to the CTA with the least
+// work so far -- the K range of a tile under a triangular operand varies from one ring stage to all of K, and a
+// round-robin deal would leave the CTAs unevenly loaded.  Slot k * units + c holds the k-th tile of CTA c (tile id
+// of the full tiles_m x tiles_n numbering), -1 where that CTA has none; the kernels walk their slots in order.
+struct TileSchedule {
+  std::vector<int> slots;
+  int units = 0;        // CTAs (pairs) dealt to
+  long long tiles = 0;  // real tiles
+};
+TileSchedule deal_tiles(const gemm_desc_t& d, int tile_m, int bn, int raster, int kstep, int num_kb, int max_units) {
+  const int d_tri = d_tri_of(d);
+  const int a_tri = (d.flags & GEMM_FLAG_A_LOWER) ? 1 : ((d.flags & GEMM_FLAG_A_UPPER) ? 2 : 0);
+  const int b_tri = (d.structure & GEMM_STRUCT_B_LOWER) ? 1 : ((d.structure & GEMM_STRUCT_B_UPPER) ? 2 : 0);
+  const int tiles_m = ceil_div(d.M, tile_m), tiles_n = ceil_div(d.N, bn);
+  struct Item {
+    int tile;
+    long long work;
+  };
+  std::vector<Item> order;
   int t = 0;
   for (int first = 0; first < tiles_m; first += raster) {
     const int gm = std::min(raster, tiles_m - first);
     for (int tn = 0; tn < tiles_n; ++tn)
       for (int r = 0; r < gm; ++r, ++t) {
+        const long long tm = first + r;
         int j0, j1;
-        tri_columns(d_tri, first + r, tile_m, bn, M, N, tiles_n, &j0, &j1);
-        if (tn >= j0 && tn <= j1) list.push_back(t);
+        tri_columns(d_tri, tm, tile_m, bn, d.M, d.N, tiles_n, &j0, &j1);
+        if (tn < j0 || tn > j1) continue;
+        // ring stages this tile visits (the kernel's k_range) -> tensor-pipe cycles, plus what a tile costs besides
+        long long lo = 0, hi = num_kb;
+        const long long row0 = tm * tile_m, col0 = static_cast<long long>(tn) * bn;
+        if (a_tri == 1) hi = std::min<long long>(hi, (std::min<long long>(row0 + tile_m, d.M) - 1) / kstep + 1);
+        else if (a_tri == 2) lo = std::max<long long>(lo, row0 / kstep);
+        if (b_tri == 1) lo = std::max<long long>(lo, col0 / kstep);
+        else if (b_tri == 2) hi = std::min<long long>(hi, (std::min<long long>(col0 + bn, d.N) - 1) / kstep + 1);
+        const long long stages = std::max<long long>(1, hi - lo);
+        order.push_back(Item{t, stages * (kstep / 64) * 2 * bn + 1000});
       }
   }
-  return list;
+  TileSchedule sch;
+  sch.tiles = static_cast<long long>(order.size());
+  sch.units = static_cast<int>(std::max<long long>(1, std::min<long long>(max_units, sch.tiles)));
+  std::vector<std::vector<int>> mine(sch.units);
+  using Load = std::pair<long long, int>;  // (work so far, CTA): the least loaded CTA, the lowest index among equals
+  std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
+  for (int c = 0; c < sch.units; ++c) heap.push(Load(0, c));
+  for (const Item& it : order) {
+    Load l = heap.top();
+    heap.pop();
+    mine[l.second].push_back(it.tile);
+    heap.push(Load(l.first + it.work, l.second));
+  }
+  size_t rounds = 1;
+  for (const auto& v : mine) rounds = std::max(rounds, v.size());
+  sch.slots.assign(rounds * sch.units, -1);
+  for (int c = 0; c < sch.units; ++c)
+    for (size_t k = 0; k < mine[c].size(); ++k) sch.slots[k * sch.units + c] = mine[c][k];
+  return sch;
 }
 
 // Tail split of the double-buffered dense kernels (on request, GEMM_FLAG_TAIL_SPLIT): when the tiles left over after the
@@ -388,9 +437,21 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   p.l2_hint_d = static_cast<double>(d.M) * d.N * d.batch_count * elem_bytes(d.c_dtype) > 64.0e6 ? 1 : 0;
   p.a_tri = (d.flags & GEMM_FLAG_A_LOWER) ? 1 : ((d.flags & GEMM_FLAG_A_UPPER) ? 2 : 0);
   p.b_tri = (d.structure & GEMM_STRUCT_B_LOWER) ? 1 : ((d.structure & GEMM_STRUCT_B_UPPER) ? 2 : 0);
-  p.tile_list = nullptr;  // the device copy of the list is made by gemm_plan
-  p.list_len = d_tri ? static_cast<int>(num_tiles / d.batch_count) : 0;
+  p.tile_list = nullptr;  // the device copy of the schedule is made by gemm_plan
+  p.list_len = 0;
   pl->d_tri = d_tri;
+  int dealt_units = 0;
+  if (d_tri || p.a_tri || p.b_tri) {  // structured problem: tiles left out and / or unequal K ranges -> dealt ahead of time
+    const TileSchedule sch = deal_tiles(d, tile_m, bn, raster, kblk * atoms, p.num_kb, units);
+    if (static_cast<long long>(sch.slots.size()) * d.batch_count > 0x7FFFFFFFll) return GEMM_ERR_UNSUPPORTED;
+    free(pl->h_tile_list);
+    pl->h_tile_list = static_cast<int*>(malloc(sch.slots.size() * sizeof(int)));
+    if (!pl->h_tile_list) return GEMM_ERR_CUDA;
+    memcpy(pl->h_tile_list, sch.slots.data(), sch.slots.size() * sizeof(int));
+    p.list_len = static_cast<int>(sch.slots.size());
+    p.num_tiles = p.list_len * d.batch_count;  // slots, the empty ones included
+    dealt_units = sch.units;
+  }
   p.ldc = d.ldc;
   p.stride_c = d.batch_count > 1 ? d.stride_c : 0;
   p.debug_flags = 0u;  // set per run
@@ -407,7 +468,7 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   pl->stages = stages;
   pl->raster_group = raster;
   pl->smem_bytes = smem;
-  pl->grid = static_cast<int>(std::min<long long>(num_tiles, units)) * cg;
+  pl->grid = (dealt_units ? dealt_units : static_cast<int>(std::min<long long>(num_tiles, units))) * cg;
   pl->variant = cg == 2 ? GEMM_VARIANT_DENSE_2CTA : GEMM_VARIANT_DENSE_1CTA;
 
   gemm_info_t& info = pl->info;
@@ -676,18 +737,19 @@ gemm_status_t plan_impl(const gemm_desc_t* desc, gemm_plan_t* out_plan, bool use
       return GEMM_ERR_CUDA;
     }
   }
-  if (pl->has_device && pl->arch_ok && pl->d_tri) {
-    const std::vector<int> list = tri_tile_list(pl->d_tri, pl->info.tile_m, pl->bn, d.M, d.N, pl->raster_group);
-    const size_t bytes = std::max<size_t>(list.size(), 1) * sizeof(int);
-    if (static_cast<int>(list.size()) != pl->dense.list_len || cudaMalloc(&pl->d_tile_list, bytes) != cudaSuccess ||
-        cudaMemcpy(pl->d_tile_list, list.data(), list.size() * sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) {
-      note_cuda_error("cudaMalloc(tile list)", cudaGetErrorName(cudaGetLastError()));
+  if (pl->has_device && pl->arch_ok && pl->h_tile_list) {
+    const size_t bytes = static_cast<size_t>(pl->dense.list_len) * sizeof(int);
+    if (cudaMalloc(&pl->d_tile_list, bytes) != cudaSuccess ||
+        cudaMemcpy(pl->d_tile_list, pl->h_tile_list, bytes, cudaMemcpyHostToDevice) != cudaSuccess) {
+      note_cuda_error("cudaMalloc(tile schedule)", cudaGetErrorName(cudaGetLastError()));
       if (pl->d_tile_list) cudaFree(pl->d_tile_list);
       cudaFree(pl->d_status);
       delete pl;
       return GEMM_ERR_CUDA;
     }
     pl->dense.tile_list = pl->d_tile_list;
+    free(pl->h_tile_list);
+    pl->h_tile_list = nullptr;
   }
   if (getenv("B200GEMM_LOG")) {
     fprintf(stderr,
