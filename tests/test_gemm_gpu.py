@@ -176,6 +176,10 @@ EXACT_CASES = [
     ("lower_a_upper_b", 712, 712, 712, dict(a_tri=1, b_tri=2, epi=bg.EPI_BIAS, beta=1.0), dict(variant=V1, tile_n=128)),
     ("upper_times_upper_batched_fp8", 384, 384, 384, dict(a_tri=2, b_tri=2, d_tri=2, batch=3, ab=wl.FP8_E4M3), dict(variant=V1, tile_n=64)),
     ("upper_times_upper_auto", 2048, 2048, 2048, dict(a_tri=2, b_tri=2, d_tri=2, cd=wl.BF16), dict()),
+    # dealt schedules with empty slots in the middle of a CTA's sequence: more tiles than CTAs, not a multiple, batched
+    ("d_lower_batched_two_rounds", 2304, 2304, 136, dict(d_tri=1, batch=2, cd=wl.BF16, sample_rows=96, sample_cols=96), dict(variant=V1, tile_n=128)),
+    ("tri_upper_batched_two_rounds", 2304, 1152, 1160, dict(a_tri=2, batch=3, sample_rows=96, sample_cols=96), dict(variant=V1, tile_n=128)),
+    ("upper_times_upper_pair_batched_rounds", 2560, 2560, 1288, dict(a_tri=2, b_tri=2, d_tri=2, batch=2, cd=wl.BF16, sample_rows=96, sample_cols=96), dict(variant=V2, tile_n=128)),
     # mirrored stream-K: a tall output with a handful of columns (A is the streamed operand)
     ("tall_one_unit", 128, 8, 64, {}, dict(variant=VS)),
     ("tall_split_k", 256, 8, 4096, {}, dict(variant=VS)),
