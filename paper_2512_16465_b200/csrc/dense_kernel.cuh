@@ -31,11 +31,38 @@ constexpr int kSlabBytes = 32 * 128;  // epilogue staging slab of one warp: 32 r
 // device status word values (also used by the skinny kernel)
 constexpr uint32_t kStatusTimeout = 0x80000000u;  // | role << 8 | detail
 
+// Division by a divisor fixed at plan time (Granlund-Montgomery): n / d for every 32-bit n in a multiply and two shifts.
+// The tile scheduler divides by run-time tile counts several times per tile and role; a hardware-emulated 32-bit
+// division is a chain of some twenty dependent instructions, most felt in front of a CTA's first load.
+struct FastDiv {
+  uint32_t mul, sh1, sh2;
+};
+inline FastDiv make_fastdiv(uint32_t d) {  // host; 1 <= d <= 2^31
+  uint32_t l = 0;
+  while ((1ull << l) < d) ++l;
+  FastDiv f;
+  f.mul = static_cast<uint32_t>(((1ull << 32) * ((1ull << l) - d)) / d + 1);
+  f.sh1 = l < 1 ? l : 1;
+  f.sh2 = l ? l - 1 : 0;
+  return f;
+}
+__host__ __device__ __forceinline__ uint32_t fast_div(uint32_t n, const FastDiv& f) {
+#ifdef __CUDA_ARCH__
+  const uint32_t t = __umulhi(f.mul, n);
+#else
+  const uint32_t t = static_cast<uint32_t>((static_cast<unsigned long long>(f.mul) * n) >> 32);
+#endif
+  return (t + ((n - t) >> f.sh1)) >> f.sh2;
+}
+
 struct DenseParams {
   int M, N, K, batch;
   int tiles_m, tiles_n;  // tiles per matrix; a tile is (128*CG) x bn
   int num_tiles;         // batch * tiles_m * tiles_n
   int raster_group;      // tile rows swept together (column-wise inside the group)
+  // the scheduler's divisors: tiles per matrix, tiles per raster group, rows of a full group and of the last group, slots per matrix
+  FastDiv fd_matrix, fd_group, fd_rows, fd_last_rows, fd_list;
+  int kstep_shift;       // log2 of the K extent of a ring stage (kblk * atoms, a power of two)
   int bn;                // tile N (multiple of 64, <= 256)
   int stages;            // ring depth
   int num_kb;            // ring stages per tile = ceil(K / (64 * atoms))
@@ -146,7 +173,24 @@ struct TileCoord {
 // Linear tile id -> (batch, tile row, tile column).  Inside one matrix, tiles are visited in groups
 // of `raster_group` tile rows; inside a group the row index runs fastest, so the CTAs that are
 // resident together work on a compact block of the output and share A and B panels in L2.
-__device__ __forceinline__ TileCoord decode_tile(int t, int tiles_m, int tiles_n, int raster_group) {
+__device__ __forceinline__ TileCoord decode_tile(const DenseParams& p, int t) {
+  TileCoord c;
+  const int per_matrix = p.tiles_m * p.tiles_n;
+  c.batch = static_cast<int>(fast_div(static_cast<uint32_t>(t), p.fd_matrix));
+  const int r = t - c.batch * per_matrix;
+  const int group_sz = p.raster_group * p.tiles_n;
+  const int g = static_cast<int>(fast_div(static_cast<uint32_t>(r), p.fd_group));
+  const int first_m = g * p.raster_group;
+  const int gm = min(p.raster_group, p.tiles_m - first_m);
+  const int within = r - g * group_sz;
+  c.tn = static_cast<int>(fast_div(static_cast<uint32_t>(within), gm == p.raster_group ? p.fd_rows : p.fd_last_rows));
+  c.tm = first_m + (within - c.tn * gm);
+  return c;
+}
+
+// The same with plain divisions, for the wide pair kernel: its tiles last tens of thousands of cycles, and its register
+// allocation is at the limit where any change of this code has cost spills.
+__device__ __forceinline__ TileCoord decode_tile_div(int t, int tiles_m, int tiles_n, int raster_group) {
   TileCoord c;
   const int per_matrix = tiles_m * tiles_n;
   c.batch = t / per_matrix;
@@ -170,11 +214,11 @@ struct KRange {
 };
 __device__ __forceinline__ KRange k_range(const DenseParams& p, int row0, int rows, int col0, int cols) {
   KRange r{0, p.num_kb};
-  const int kstep = p.kblk * p.atoms;
-  if (p.a_tri == 1) r.hi = min(r.hi, (min(row0 + rows, p.M) - 1) / kstep + 1);       // k <= last row
-  else if (p.a_tri == 2) r.lo = max(r.lo, row0 / kstep);                              // k >= first row
-  if (p.b_tri == 1) r.lo = max(r.lo, col0 / kstep);                                   // k >= first column
-  else if (p.b_tri == 2) r.hi = min(r.hi, (min(col0 + cols, p.N) - 1) / kstep + 1);   // k <= last column
+  const int ks = p.kstep_shift;
+  if (p.a_tri == 1) r.hi = min(r.hi, ((min(row0 + rows, p.M) - 1) >> ks) + 1);       // k <= last row
+  else if (p.a_tri == 2) r.lo = max(r.lo, row0 >> ks);                                // k >= first row
+  if (p.b_tri == 1) r.lo = max(r.lo, col0 >> ks);                                     // k >= first column
+  else if (p.b_tri == 2) r.hi = min(r.hi, ((min(col0 + cols, p.N) - 1) >> ks) + 1);   // k <= last column
   if (r.lo >= r.hi) {
     r.lo = min(r.lo, p.num_kb - 1);
     r.hi = r.lo + 1;
@@ -190,7 +234,7 @@ struct WorkItem {
 template <bool kSplit>
 __device__ __forceinline__ int item_tile(const DenseParams& p, int item) {
   if (p.tile_list != nullptr) {  // (never together with a tail split); < 0: an empty slot
-    const int b = item / p.list_len;
+    const int b = static_cast<int>(fast_div(static_cast<uint32_t>(item), p.fd_list));
     const int t = __ldg(p.tile_list + (item - b * p.list_len));
     return t < 0 ? -1 : b * (p.tiles_m * p.tiles_n) + t;
   }
@@ -393,7 +437,10 @@ __device__ __forceinline__ void epilogue_math(float (&v)[32], const uint32_t (&a
 // Both single-issuer roles are run by a whole warp in uniform control flow; only the instructions that
 // must be issued once (TMA, tcgen05.mma, commits, barrier arrivals) sit under elect_one().  That keeps
 // addresses, descriptors and coordinates in uniform registers, which is what those instructions read.
-template <int CG, bool kSplit = false>
+// kJoinSetup (pairs): the warp enters before the CTA-wide end of set-up and joins it itself -- the block barrier and
+// the cluster barrier the other warps execute in the kernel body -- once it has worked out its first tile, so that
+// work overlaps the tensor-memory allocation and the wait for the peer CTA instead of following them.
+template <int CG, bool kSplit = false, bool kJoinSetup = false>
 __device__ __forceinline__ void producer_role(const DenseParams& p, const CUtensorMap* tmA, const CUtensorMap* tmB,
                                               uint32_t tiles_base, uint32_t full0, uint32_t empty0, uint32_t cta_rank,
                                               int cluster_id, int num_clusters, const WaitCtx& w) {
@@ -407,6 +454,7 @@ __device__ __forceinline__ void producer_role(const DenseParams& p, const CUtens
   const uint64_t pol_b = p.l2_hint_b == 2 ? l2_policy_evict_last() : (p.l2_hint_b == 1 ? l2_policy_evict_first() : l2_policy_evict_normal());
   const int kstep = p.kblk * p.atoms;
   uint32_t it = 0;
+  bool waited = false;
   const int n_items = kSplit ? p.num_items : p.num_tiles;
   for (int item = cluster_id; item < n_items; item += num_clusters, ++it) {
     const int tile = item_tile<kSplit>(p, item);
@@ -414,13 +462,26 @@ __device__ __forceinline__ void producer_role(const DenseParams& p, const CUtens
       --it;          // (the loop header adds the one back: buffer and phase bookkeeping follow the tiles actually computed)
       continue;
     }
-    const TileCoord tc = decode_tile(tile, p.tiles_m, p.tiles_n, p.raster_group);
+    const TileCoord tc = decode_tile(p, tile);
     const int m0 = tc.tm * (kCtaM * CG) + static_cast<int>(cta_rank) * kCtaM;
     const int n0 = tc.tn * p.bn + (CG == 2 ? static_cast<int>(cta_rank) * p.b_rows : 0);
     // Serpentine K: all CTAs advance through K roughly in step, so the K range a wave touched last is what L2
     // still holds when the next wave starts; walking it backwards re-uses those lines of the shared A band.
     const bool rev = p.k_serpentine && (it & 1u);
     const KRange kr = work_item<kSplit>(p, item, tile, tc.tm * (kCtaM * CG), kCtaM * CG, tc.tn * p.bn).kr;
+    // Everything above needs only the kernel's parameters (and the plan's own tile schedule), so it runs while the
+    // previous kernel of the stream is still finishing; its memory is touched from here on.
+    if (!waited) {
+      if constexpr (kJoinSetup) {
+        tc_fence_before();
+        __syncthreads();
+        cluster_arrive();  // the peer's barriers must exist before anything signals them
+        cluster_wait();
+        tc_fence_after();
+      }
+      griddep_wait();
+      waited = true;
+    }
     int k0 = rev ? (kr.hi - 1) * kstep : kr.lo * kstep;
     const int dk = rev ? -kstep : kstep;
     for (int kb = kr.lo; kb < kr.hi; ++kb, k0 += dk) {
@@ -462,6 +523,13 @@ __device__ __forceinline__ void producer_role(const DenseParams& p, const CUtens
       }
     }
   }
+  if (kJoinSetup && !waited) {  // no tile at all: the others still wait for this warp at the end of set-up
+    tc_fence_before();
+    __syncthreads();
+    cluster_arrive();
+    cluster_wait();
+    tc_fence_after();
+  }
 }
 
 template <int CG, bool kSplit = false>
@@ -495,7 +563,7 @@ __device__ __forceinline__ void mma_role(const DenseParams& p, uint32_t tiles_ba
     const bool rev = p.k_serpentine && (it & 1u);
     KRange kr{0, num_kb};
     if ((p.a_tri | p.b_tri) != 0 || (kSplit && item >= p.split_first_tile)) {
-      const TileCoord tc = decode_tile(tile, p.tiles_m, p.tiles_n, p.raster_group);
+      const TileCoord tc = decode_tile(p, tile);
       kr = work_item<kSplit>(p, item, tile, tc.tm * (kCtaM * CG), kCtaM * CG, tc.tn * p.bn).kr;
     }
     const int n_kb = kr.hi - kr.lo;
@@ -588,7 +656,7 @@ __device__ __forceinline__ void epilogue_role(const DenseParams& p, const CUtens
       --it;          // (the loop header adds the one back: buffer and phase bookkeeping follow the tiles actually computed)
       continue;
     }
-    const TileCoord tc = decode_tile(tile, p.tiles_m, p.tiles_n, p.raster_group);
+    const TileCoord tc = decode_tile(p, tile);
     const uint32_t buf = it & 1u;
     const uint32_t ph = (it >> 1) & 1u;
     if (!mbar_wait_warp(tfull0 + 8u * buf, ph, w, (3u << 8) | buf, 64u)) return;  // whole warp leaves the wait together
@@ -777,8 +845,10 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     // the other warps and starts the loads while those are still waiting for the tensor-memory allocation.
     __syncwarp();
     named_barrier_arrive(3, blockDim.x);
-    griddep_wait();  // from here on global memory is read
     producer_role<CG, kSplit>(p, &tmA, &tmB, base, full0, empty0, cta_rank, cluster_id, num_clusters, w);
+  } else if (CG == 2 && warp == 0) {
+    __syncwarp();  // (lane 0 set the barriers up)
+    producer_role<CG, kSplit, true>(p, &tmA, &tmB, base, full0, empty0, cta_rank, cluster_id, num_clusters, w);
   } else {
     tc_fence_before();
     if constexpr (CG == 1) {
@@ -790,11 +860,13 @@ dense_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     }
     tc_fence_after();
     tmem_base = *tmem_slot;
-    griddep_wait();  // barriers and tensor memory are set up; from here on global memory is read and written
+    // barriers and tensor memory are set up; from here on global memory is read and written (the producer warp makes
+    // this wait itself, once it has worked out its first tile)
+    if (warp != 0) griddep_wait();
   }
 
   if (warp == 0) {
-    if constexpr (CG == 2) producer_role<CG, kSplit>(p, &tmA, &tmB, base, full0, empty0, cta_rank, cluster_id, num_clusters, w);
+    // (ran above)
   } else if (warp == 1) {
     if (cta_rank == 0) mma_role<CG, kSplit>(p, base, full0, empty0, tfull0, tempty0, tmem_base, cluster_id, num_clusters, w);
   } else {

@@ -261,6 +261,33 @@ TileSchedule deal_tiles(const gemm_desc_t& d, int tile_m, int bn, int raster, in
   return sch;
 }
 
+// The tile scheduler's plan-time divisors (see FastDiv).  False if a division came out wrong (it cannot; checked on
+// the values the scheduler will actually meet at the ends of each range, so that a mistake here fails at plan time).
+bool set_scheduler_divisors(DenseParams& p) {
+  const uint32_t per_matrix = static_cast<uint32_t>(p.tiles_m) * p.tiles_n;
+  const uint32_t group = static_cast<uint32_t>(p.raster_group) * p.tiles_n;
+  const uint32_t last_rows = p.tiles_m % p.raster_group ? p.tiles_m % p.raster_group : p.raster_group;
+  const uint32_t list = p.list_len > 0 ? p.list_len : 1;
+  p.fd_matrix = make_fastdiv(per_matrix);
+  p.fd_group = make_fastdiv(group);
+  p.fd_rows = make_fastdiv(p.raster_group);
+  p.fd_last_rows = make_fastdiv(last_rows);
+  p.fd_list = make_fastdiv(list);
+  const int kstep = p.kblk * p.atoms;
+  p.kstep_shift = 0;
+  while ((1 << p.kstep_shift) < kstep) ++p.kstep_shift;
+  if ((1 << p.kstep_shift) != kstep) return false;
+  const struct {
+    const FastDiv* f;
+    uint32_t d;
+  } all[] = {{&p.fd_matrix, per_matrix}, {&p.fd_group, group}, {&p.fd_rows, static_cast<uint32_t>(p.raster_group)},
+             {&p.fd_last_rows, last_rows}, {&p.fd_list, list}};
+  for (const auto& e : all)
+    for (uint32_t n : {0u, 1u, e.d - 1, e.d, e.d + 1, 2 * e.d - 1, 2 * e.d, 1000003u, 0x7FFFFFFEu, 0x7FFFFFFFu, 0xFFFFFFFFu})
+      if (fast_div(n, *e.f) != n / e.d) return false;
+  return true;
+}
+
 // Tail split of the double-buffered dense kernels (on request, GEMM_FLAG_TAIL_SPLIT): when the tiles left over after the
 // full waves occupy at most half of the CTAs (pairs), each of them is cut into this many K slices, one per CTA (pair); the slice that
 // starts at K = 0 adds the others' raw accumulators from the workspace and finishes the tile.  1 = no split.
@@ -305,8 +332,8 @@ double estimate_dense_cycles(const gemm_desc_t& d, int sm_count, int variant, in
     if (split > 1) waves += 1.0 / split - 1.0 + 0.08;  // + hand-over of the partial accumulators
   }
   // tensor pipe: one 128 x bn x 16 MMA per CTA takes bn / 2 cycles; four per k-block and 128-row half
-  static const double eff1[3] = {0.45, 0.68, 0.82}, eff2[3] = {0.55, 0.80, 0.938};  // bn = 64, 128, 256 (measured: 8192^3, and K = 512 ... 4096)
-  const int bi = bn <= 64 ? 0 : (bn <= 128 ? 1 : 2);
+  static const double eff1[4] = {0.45, 0.68, 0.76, 0.82}, eff2[4] = {0.55, 0.80, 0.88, 0.938};  // bn = 64, 128, 192, 256 (measured: 8192^3, and K = 512 ... 4096; 192 in between)
+  const int bi = bn <= 64 ? 0 : (bn <= 128 ? 1 : (bn <= 192 ? 2 : 3));
   const double eff = wide ? 1.0 : (cg == 1 ? eff1[bi] : eff2[bi]);
   const double mma = kblocks * 4.0 * (bn / 2.0) * (rows_cta / 128.0) / eff;
   // operand feed: bytes this SM receives per k-block at ~90 B/clk
@@ -452,6 +479,7 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
     p.num_tiles = p.list_len * d.batch_count;  // slots, the empty ones included
     dealt_units = sch.units;
   }
+  if (!set_scheduler_divisors(p)) return GEMM_ERR_UNSUPPORTED;
   p.ldc = d.ldc;
   p.stride_c = d.batch_count > 1 ? d.stride_c : 0;
   p.debug_flags = 0u;  // set per run
@@ -549,6 +577,7 @@ gemm_status_t plan_wide(gemm_plan_s* pl, int forced_raster, int forced_stages) {
   p.b_desc_hi = b_kmajor ? make_smem_desc_hi(16, 1024) : make_smem_desc_hi(8192, 1024);
   p.a_kstep = a_kmajor ? kUmmaK * 2 : kUmmaK * 128;
   p.b_kstep = b_kmajor ? kUmmaK * 2 : kUmmaK * 128;
+  if (!set_scheduler_divisors(p)) return GEMM_ERR_UNSUPPORTED;
   p.out_dtype = d.c_dtype;
   p.epilogue = d.epilogue;
   p.bias_per_row = (d.flags & GEMM_FLAG_BIAS_PER_ROW) ? 1 : 0;
@@ -701,7 +730,7 @@ gemm_status_t plan_impl(const gemm_desc_t* desc, gemm_plan_t* out_plan, bool use
       const bool b_kmajor = d.transb == GEMM_OP_T;
       DenseCandidate best{GEMM_VARIANT_DENSE_1CTA, 64, 1e300};
       for (int v : {GEMM_VARIANT_DENSE_1CTA, GEMM_VARIANT_DENSE_2CTA, GEMM_VARIANT_DENSE_2CTA_WIDE}) {
-        for (int bn : {256, 128, 64}) {
+        for (int bn : {256, 192, 128, 64}) {
           if (v == GEMM_VARIANT_DENSE_2CTA_WIDE && bn != kWideTileN) continue;
           if (v == GEMM_VARIANT_DENSE_2CTA_WIDE &&
               (d.epilogue > GEMM_EPI_BIAS_GELU_ERF || d_tri_of(d) || d.structure ||

@@ -54,7 +54,7 @@ std::vector<uint32_t> first_round(const gemm_desc_t& d, const gemm_info_t& autom
     for (int bn : {64, 128, 256}) c.push_back(pack(GEMM_VARIANT_DENSE_1CTA, bn, 0, 0, 0));
   } else {
     for (int bn : {256, 128}) c.push_back(pack(GEMM_VARIANT_DENSE_1CTA, bn, 0, 0, 0));
-    for (int bn : {256, 128}) c.push_back(pack(GEMM_VARIANT_DENSE_2CTA, bn, 0, 0, 0));
+    for (int bn : {256, 192, 128}) c.push_back(pack(GEMM_VARIANT_DENSE_2CTA, bn, 0, 0, 0));  // (192: refused, hence skipped, when B is stored K x N)
     c.push_back(pack(GEMM_VARIANT_DENSE_2CTA_WIDE, 0, 0, 0, 0));
   }
   return c;

@@ -53,7 +53,7 @@ __device__ __forceinline__ void wide_producer_role(const DenseParams& p, const C
   bool stall_pending = (p.debug_flags & 1u) != 0u;
   const uint64_t pol = l2_policy_evict_normal();
   for (int tile = cluster_id; tile < p.num_tiles; tile += num_clusters, ++it) {
-    const TileCoord tc = decode_tile(tile, p.tiles_m, p.tiles_n, p.raster_group);
+    const TileCoord tc = decode_tile_div(tile, p.tiles_m, p.tiles_n, p.raster_group);
     const int m0 = tc.tm * (2 * kWideCtaM) + static_cast<int>(cta_rank) * kWideCtaM;
     const int n0 = tc.tn * kWideTileN + static_cast<int>(cta_rank) * p.b_rows;
     const bool rev = p.k_serpentine && (it & 1u);  // see dense_kernel.cuh: re-use what L2 touched last
@@ -216,7 +216,7 @@ __device__ __forceinline__ void wide_epilogue_role(const DenseParams& p, const C
   const uint32_t sw = lane & 7u;
   uint32_t it = 0, nstore = 0;
   for (int tile = cluster_id; tile < p.num_tiles; tile += num_clusters, ++it) {
-    const TileCoord tc = decode_tile(tile, p.tiles_m, p.tiles_n, p.raster_group);
+    const TileCoord tc = decode_tile_div(tile, p.tiles_m, p.tiles_n, p.raster_group);
     const int row_cta = tc.tm * (2 * kWideCtaM) + static_cast<int>(cta_rank) * kWideCtaM + static_cast<int>(q) * 32;
     const int colbase = tc.tn * kWideTileN + static_cast<int>(ch) * 128;
 #pragma unroll 1
