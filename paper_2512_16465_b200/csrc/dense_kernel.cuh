@@ -289,13 +289,14 @@ __device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
   return d;
 }
 // GELU with the exact error function, t * Phi(t) = 0.5 t (1 + erf(x)), x = t / sqrt(2), evaluated without branches:
-// g = erfc(|x|) = 2^p(z) with one degree-9 polynomial in z = |x| / 2 - 1 on |x| <= 4 (clamped beyond: erfc(4) = 1.5e-8),
+// g = erfc(|x|) = 2^p(z) with one degree-9 polynomial in z = |x| / 2 - 1 on |x| <= 4 (zero beyond: erfc(4) = 1.5e-8),
 // then 1 + erf(x) = g for x < 0 (no cancellation in the negative tail) and 2 - g otherwise.  Coefficients, their
 // derivation and the fp32 error report (max |error| 2.1e-7, relative error of erfc 3e-6) come from fit_gelu_poly.py
 // beside this file.  About half the instructions of erff(), which matters because the epilogue shares the power budget
 // with the tensor pipe.
 __device__ __forceinline__ float gelu_erf(float t) {
-  const float ax = fminf(fabsf(t) * 0.70710678118654752f, 4.0f);
+  const float ar = fabsf(t) * 0.70710678118654752f;
+  const float ax = fminf(ar, 4.0f);
   const float z = fmaf(ax, 0.5f, -1.0f);
   float p = 0.0007019337f;
   p = fmaf(p, z, -0.00019923763f);
@@ -309,6 +310,7 @@ __device__ __forceinline__ float gelu_erf(float t) {
   p = fmaf(p, z, -7.739975f);
   float g;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(g) : "f"(p));
+  g = ar > 4.0f ? 0.0f : g;  // beyond the fitted range erfc is 1.5e-8 and less: the tail goes to -0 (and to t), not to t * 7.7e-9
   return 0.5f * t * (t < 0.0f ? g : 2.0f - g);
 }
 

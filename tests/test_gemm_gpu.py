@@ -199,6 +199,78 @@ def test_exact_integer_inputs(case):
     H.check_workload(w, bg.make_flags(**fl), exact=True, repeats=2)
 
 
+def _random_case(seed):
+    """A seeded random problem: variant, dtypes, storage orders, ragged extents with padded leading dimensions, batch,
+    epilogue, scalars, structure flags and tuning fields all drawn independently (within what the ABI documents as
+    supported together)."""
+    rng = np.random.default_rng(1000 + seed)
+    pick = lambda xs: xs[int(rng.integers(len(xs)))]
+    variant = pick([0, 0, V1, V1, V2, V2, VW, VS])
+    ab = pick([wl.BF16, wl.BF16, wl.F16, wl.FP8_E4M3, wl.FP8_E5M2])
+    cd = pick([wl.F32, wl.BF16, wl.F16])
+    fp8 = ab in (wl.FP8_E4M3, wl.FP8_E5M2)
+    ta, tb = (0, 1) if (fp8 or variant == VS) else (int(rng.integers(2)), int(rng.integers(2)))
+    if variant == VS:
+        short, long_ = int(rng.integers(1, 65)), int(rng.integers(64, 1500))
+        M, N = (short, long_) if rng.integers(2) else (long_, short)
+        batch = 1
+    else:
+        M, N = int(rng.integers(1, 700)), int(rng.integers(1, 700))
+        if variant == VW:
+            M = max(M, 130)
+        batch = pick([1, 1, 2, 3])
+    K = int(rng.integers(1, 1100))
+    while M * N * K * batch > 2.5e8:
+        K = max(1, K // 2)
+    ea = 16 if fp8 else 8                     # elements per 16 bytes
+    ec = 4 if cd == wl.F32 else 8
+    up = lambda x, m: -(-x // m) * m
+    lda = up(M if ta else K, ea) + ea * int(rng.integers(0, 3))
+    ldb = up(K if tb else N, ea) + ea * int(rng.integers(0, 3))
+    ldc = up(N, ec) + ec * int(rng.integers(0, 3))
+    kw = dict(ta=ta, tb=tb, ab=ab, cd=cd, batch=batch, lda=lda, ldb=ldb, ldc=ldc,
+              alpha=pick([1.0, 1.0, 0.5, 2.0, -1.0]), beta=pick([0.0, 0.0, 1.0, -1.0, 0.5]))
+    if batch > 1:   # strides: tight or padded by a multiple of 16 bytes
+        kw["stride_a"] = (K if ta else M) * lda + ea * int(rng.integers(0, 5))
+        kw["stride_b"] = (N if tb else K) * ldb + ea * int(rng.integers(0, 5))
+        kw["stride_c"] = M * ldc + ec * int(rng.integers(0, 5))
+    epi = int(rng.integers(0, 6 if variant == VW else 10))
+    kw["epi"] = epi
+    if variant != VW and (epi & 1) and rng.integers(3) == 0:
+        kw["bias_per_row"] = True
+    fl = dict(variant=variant)
+    if variant in (0, V1, V2) and rng.integers(3) == 0:
+        kw["a_tri"] = int(rng.integers(3))
+        kw["b_tri"] = int(rng.integers(3))
+        kw["d_tri"] = int(rng.integers(3))
+    if variant in (V1, V2):
+        fl["tile_n"] = pick([0, 64, 128, 192, 256] if not (variant == V2 and tb == 0) else [0, 128, 256])
+        fl["kslices"] = pick([0, 1, 2])
+        fl["tail_split"] = bool(rng.integers(2))
+    if variant in (V1, V2, VW):
+        fl["raster"] = pick([0, 0, 1, 3])
+        fl["stages"] = pick([0, 0, 2, 3])
+        fl["no_k_serpentine"] = bool(rng.integers(4) == 0)
+    if variant == VS:
+        fl["kslices"] = pick([0, 1, 2, 3])
+    fl["no_early_launch"] = bool(rng.integers(4) == 0)
+    return M, N, K, kw, fl
+
+
+@pytest.mark.parametrize("seed", range(64))
+def test_random_problems(seed):
+    """Integer-valued inputs: bit-exact wherever the epilogue keeps integers (none, bias, ReLU; alpha and beta are powers
+    of two), the stated tolerance for the transcendental activations.  A combination the library documents as
+    unsupported must be refused with that code, never run wrong."""
+    M, N, K, kw, fl = _random_case(seed)
+    w = int_workload(f"random_{seed}", M, N, K, **kw)
+    try:
+        H.check_workload(w, bg.make_flags(**fl), exact=kw["epi"] <= 3, repeats=2)
+    except bg.GemmError as e:
+        assert e.status == bg.ERR_UNSUPPORTED, (M, N, K, kw, fl)
+        pytest.skip(f"refused as unsupported: {M}x{N}x{K} {kw} {fl}")
+
+
 def test_padded_leading_dimensions_and_strides():
     w = int_workload("padded", 200, 328, 136, batch=3, cd=wl.BF16, beta=1.0,
                      lda=136 + 8, ldb=136 + 24, ldc=328 + 16,
