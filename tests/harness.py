@@ -20,6 +20,12 @@ fraction f of such one-ulp flips the Frobenius distance is about u_out * sqrt(f)
 accumulation over K = 8192 terms with heavy cancellation (config c2) flips about 0.5 % of the
 elements, so the bar is set at f = 1 %, i.e. 0.1 * u_out.  The accumulator itself is held to 1e-4
 against y by re-running the same plan with fp32 output.
+A transcendental activation (GELU, SiLU) is evaluated in fp32 with the hardware's approximate exp2 and
+reciprocal, or erff() with the cancellation of 1 + erf(x) in its negative half: a relative error d_act of
+up to about 1e-5 in the value that is then rounded.  A rounding boundary of the output format lies within
+that distance of a fraction 2 * d_act / u_out of the values (4 % for fp16, 0.5 % for bf16), so for those
+epilogues the share of bit-identical elements is required to be 99 % minus that fraction; the one-ulp,
+per-element and Frobenius bars are unchanged.
 """
 from __future__ import annotations
 
@@ -31,6 +37,7 @@ import paper_2512_16465_b200 as bg
 import workloads as wl
 
 REL_TOL, ABS_TOL, FROB_TOL = 2e-3, 1e-5, 1e-4
+D_ACT = 1e-5   # relative fp32 error allowed to a transcendental activation before the output rounding (see above)
 U_OUT = {wl.BF16: 2.0 ** -8, wl.F16: 2.0 ** -11, wl.F32: 0.0}
 
 
@@ -154,6 +161,7 @@ def check_blocks(w: wl.Workload, inputs: dict, cbits: np.ndarray, blocks, c_dtyp
         got_bits = gather(cbits, w, batches, rows, cols)
         if not w.d_tri:
             reports.append(compare_block(got_bits, y, bound, cd))
+            reports[-1]["transcendental"] = w.epilogue >= 4
             continue
         # one triangle of D wanted: its elements are held to the usual bars; every other element must either be
         # untouched (still the NaN poison, or C_in when beta != 0) or hold its value of the plain product
@@ -167,6 +175,7 @@ def check_blocks(w: wl.Workload, inputs: dict, cbits: np.ndarray, blocks, c_dtyp
         rep["outside_ok"] = bool(np.all(untouched | plain))
         rep["outside_untouched"] = int(np.sum(untouched))
         rep["outside_n"] = int(untouched.size)
+        rep["transcendental"] = w.epilogue >= 4
         reports.append(rep)
     return reports
 
@@ -199,7 +208,8 @@ def assert_reports(reports, what=""):
         assert r["frob"] <= frob_tol_for(r["c_dtype"]), f"{what}: Frobenius error {r}"
         if r["c_dtype"] != wl.F32:
             assert r["max_ulp"] <= 1, f"{what}: more than one ulp from the rounded oracle {r}"
-            assert r["bit_identical"] >= 0.99, f"{what}: too many one-ulp flips {r}"
+            floor = 0.99 - (2.0 * D_ACT / U_OUT[r["c_dtype"]] if r.get("transcendental") else 0.0)
+            assert r["bit_identical"] >= floor, f"{what}: too many one-ulp flips {r}"
 
 
 def check_workload(w: wl.Workload, flags: int = 0, exact: bool = False, c_dtype=None, repeats: int = 1, inputs=None):

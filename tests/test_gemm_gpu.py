@@ -1,5 +1,6 @@
 """GPU parity tests: the CUDA path, called through the C-ABI binding, against the CPU oracle
 on the same seeded inputs.  Run with ``-m gpu`` on a B200."""
+import os
 from dataclasses import replace
 
 import numpy as np
@@ -257,7 +258,7 @@ def _random_case(seed):
     return M, N, K, kw, fl
 
 
-@pytest.mark.parametrize("seed", range(64))
+@pytest.mark.parametrize("seed", range(int(os.environ.get("B200GEMM_RANDOM_CASES", "64"))))   # (a longer sweep on request)
 def test_random_problems(seed):
     """Integer-valued inputs: bit-exact wherever the epilogue keeps integers (none, bias, ReLU; alpha and beta are powers
     of two), the stated tolerance for the transcendental activations.  A combination the library documents as
