@@ -876,6 +876,50 @@ def test_host_resident_gemm_exact(case):
         bg.gemm_host_destroy(handle)
 
 
+@pytest.mark.parametrize("seed", range(24))
+def test_host_resident_random_problems(seed):
+    """Seeded random problems through gemm_host_run: dtypes, storage order of B, ragged extents, padded pitches,
+    epilogue, scalars and the number of row panels drawn independently; integer inputs, so bit-exact wherever the
+    epilogue keeps integers."""
+    rng = np.random.default_rng(5000 + seed)
+    pick = lambda xs: xs[int(rng.integers(len(xs)))]
+    ab = pick([wl.BF16, wl.BF16, wl.F16, wl.FP8_E4M3])
+    cd = pick([wl.F32, wl.BF16, wl.F16])
+    fp8 = ab == wl.FP8_E4M3
+    tb = 1 if fp8 else int(rng.integers(2))
+    M, N, K = int(rng.integers(1, 1800)), int(rng.integers(1, 500)), int(rng.integers(1, 700))
+    ea, ec = (16 if fp8 else 8), (4 if cd == wl.F32 else 8)
+    up = lambda x, m: -(-x // m) * m
+    epi = int(rng.integers(0, 10))
+    kw = dict(ta=0, tb=tb, ab=ab, cd=cd, lda=up(K, ea) + ea * int(rng.integers(0, 3)), ldb=up(K if tb else N, ea) + ea * int(rng.integers(0, 3)),
+              ldc=up(N, ec) + ec * int(rng.integers(0, 3)), alpha=pick([1.0, 0.5, 2.0, -1.0]), beta=pick([0.0, 1.0, -1.0]), epi=epi)
+    if (epi & 1) and rng.integers(2):
+        kw["bias_per_row"] = True
+    w = int_workload(f"host_random_{seed}", M, N, K, **kw)
+    inputs = wl.make_inputs(w)
+    pin = lambda a: None if a is None else torch.from_numpy(a).pin_memory()
+    hA, hB, hbias = pin(inputs["A"]), pin(inputs["B"]), pin(inputs["bias"])
+    c_np = np.float32 if w.c_dtype == wl.F32 else np.uint16
+    sentinel = np.full(w.elems_c(), 0x4321 if c_np == np.uint16 else 1234.5, c_np)
+    handle = bg.gemm_host_create(H.desc_of(w), int(rng.integers(0, 7)))
+    try:
+        assert 1 <= bg.gemm_host_panels(handle) <= max(1, -(-M // 256))
+        hC = pin(inputs["C"].copy() if inputs["C"] is not None else sentinel.copy())
+        bg.gemm_host_run(handle, hA.data_ptr(), hB.data_ptr(), hC.data_ptr(), 0 if hbias is None else hbias.data_ptr(),
+                         float(w.alpha), float(w.beta))
+        got = hC.numpy()
+        reports = H.check_blocks(w, inputs, got, H.default_blocks(w))
+        H.assert_reports(reports, what=w.name)
+        if epi <= 3:
+            assert all(r["bit_identical"] == 1.0 for r in reports), (M, N, K, kw)
+        before = inputs["C"] if inputs["C"] is not None else sentinel
+        mask = np.ones(w.elems_c(), bool)
+        mask[(np.arange(w.M)[:, None] * w.ldc + np.arange(w.N)[None, :]).ravel()] = False
+        assert np.array_equal(got[mask], before[mask])
+    finally:
+        bg.gemm_host_destroy(handle)
+
+
 def test_host_resident_gemm_refusals():
     for kw in (dict(transa=bg.OP_T), dict(batch=2), dict(flags=bg.make_flags(a_lower=True))):
         with pytest.raises(bg.GemmError) as e:
