@@ -272,6 +272,35 @@ def test_random_problems(seed):
         pytest.skip(f"refused as unsupported: {M}x{N}x{K} {kw} {fl}")
 
 
+@pytest.mark.parametrize("seed", range(int(os.environ.get("B200GEMM_RANDOM_LARGE_CASES", "32"))))
+def test_random_large_problems(seed):
+    """The same draw at sizes where every CTA computes many tiles (several waves, ring and accumulator buffers wrapping
+    many times, multi-round dealt schedules): extents up to about 4000, checked on 48 seeded rows and columns plus the
+    tile-boundary indices."""
+    rng = np.random.default_rng(9000 + seed)
+    M, N, K, kw, fl = _random_case(10000 + seed)
+    if fl["variant"] == VS:
+        long_ = int(rng.integers(3000, 30000))
+        M, N = (M, long_) if M <= 64 else (long_, N)
+        K = int(rng.integers(256, 3000))
+    else:
+        M, N, K = int(rng.integers(600, 4200)), int(rng.integers(600, 4200)), int(rng.integers(64, 1600))
+    fp8 = kw["ab"] in (wl.FP8_E4M3, wl.FP8_E5M2)
+    ea, ec = (16 if fp8 else 8), (4 if kw["cd"] == wl.F32 else 8)
+    up = lambda x, m: -(-x // m) * m
+    kw.update(lda=up(M if kw["ta"] else K, ea) + ea, ldb=up(K if kw["tb"] else N, ea), ldc=up(N, ec) + ec)
+    for k in ("stride_a", "stride_b", "stride_c"):
+        kw.pop(k, None)
+    if kw["batch"] > 1 and M * N > 4e6:
+        kw["batch"] = 1
+    w = int_workload(f"random_large_{seed}", M, N, K, sample_rows=48, sample_cols=48, **kw)
+    try:
+        H.check_workload(w, bg.make_flags(**fl), exact=kw["epi"] <= 3)
+    except bg.GemmError as e:
+        assert e.status == bg.ERR_UNSUPPORTED, (M, N, K, kw, fl)
+        pytest.skip(f"refused as unsupported: {M}x{N}x{K} {kw} {fl}")
+
+
 def test_padded_leading_dimensions_and_strides():
     w = int_workload("padded", 200, 328, 136, batch=3, cd=wl.BF16, beta=1.0,
                      lda=136 + 8, ldb=136 + 24, ldc=328 + 16,
