@@ -161,7 +161,7 @@ class DeviceCase:
                          w.stride_a, w.stride_b, w.stride_c, w.epilogue,
                          flags | bg.make_flags(bias_per_row=w.bias_per_row, a_lower=w.a_tri == 1, a_upper=w.a_tri == 2,
                                                d_lower=w.d_tri == 1, d_upper=w.d_tri == 2),
-                        structure=w.b_tri)
+                        structure=w.b_tri | (4 if w.d_mirror else 0))
         self.plan = bg.Plan(d)
         self.plan.workspace(device)
         self.i = 0
@@ -404,7 +404,7 @@ def run_ours(args):
 
 def parse_shape(spec: str) -> wl.Workload:
     """'MxNxK' followed by optional ':key=value' fields: batch, ta, tb (1 = stored transposed), ab (bf16|f16|e4m3|e5m2), cd (bf16|f16|f32),
-    epi (none|bias|relu|bias_relu|gelu|bias_gelu|gelu_tanh|bias_gelu_tanh|silu|bias_silu), rowbias (0|1), tri (lower|upper: op(A) triangular), btri (the same for op(B)), dtri (lower|upper: only that triangle of D wanted), alpha, beta,
+    epi (none|bias|relu|bias_relu|gelu|bias_gelu|gelu_tanh|bias_gelu_tanh|silu|bias_silu), rowbias (0|1), tri (lower|upper: op(A) triangular), btri (the same for op(B)), dtri (lower|upper: only that triangle of D wanted), mirror (0|1: copy it into the other triangle), alpha, beta,
     lda, ldb, ldc.  Example: 28672x8x8192:beta=1:cd=f32."""
     head, *fields = spec.split(":")
     M, N, K = (int(x) for x in head.lower().split("x"))
@@ -429,6 +429,8 @@ def parse_shape(spec: str) -> wl.Workload:
             kw["a_tri"] = {"lower": 1, "upper": 2}[v]
         elif k == "btri":
             kw["b_tri"] = {"lower": 1, "upper": 2}[v]
+        elif k == "mirror":
+            kw["d_mirror"] = bool(int(v))
         elif k == "dtri":
             kw["d_tri"] = {"lower": 1, "upper": 2}[v]
         elif k == "rowbias":

@@ -84,7 +84,8 @@ typedef enum {
   GEMM_VARIANT_DENSE_1CTA = 1,      /* 128 x N tile per CTA, accumulator double buffered */
   GEMM_VARIANT_DENSE_2CTA = 2,      /* CTA pair, 256 x N pair tile, accumulator double buffered */
   GEMM_VARIANT_SKINNY_STREAMK = 3,  /* M <= 64 or N <= 64 (transa = N, transb = T, no batch): stream-K over the long operand */
-  GEMM_VARIANT_DENSE_2CTA_WIDE = 4  /* CTA pair, 512 x 256 pair tile: least operand traffic per FLOP */
+  GEMM_VARIANT_DENSE_2CTA_WIDE = 4  /* CTA pair, 512 x 256 pair tile: least operand traffic per FLOP (N * output element size a
+                                       multiple of 16 bytes; bias per column, ReLU and erf GELU only; no structure flags) */
 } gemm_variant_t;
 
 /* gemm_desc_t.flags: 0 = the plain problem, every choice left to the plan.  The first group are tuning fields (they
@@ -131,6 +132,10 @@ typedef enum {
  * most one of the two. */
 #define GEMM_STRUCT_B_LOWER 0x1u
 #define GEMM_STRUCT_B_UPPER 0x2u
+/* With GEMM_FLAG_D_LOWER or D_UPPER and M == N: after the product, the wanted triangle is copied into the other one, so
+ * that D comes out symmetric (every element beyond the diagonal holds the bits of its mirror image; the diagonal and
+ * the wanted triangle are those of the product).  A second, bandwidth-bound kernel on the same stream, per batch. */
+#define GEMM_STRUCT_D_MIRROR 0x4u
 #define GEMM_FLAG_BIAS_PER_ROW 0x1u         /* the bias is fp32[M], one value per output row (default: fp32[N], one per
                                               column); not a tuning knob: it changes what is computed */
 #define GEMM_FLAG_NO_EARLY_LAUNCH 0x4u       /* launch without programmatic dependent launch (default: the kernel may be
@@ -200,7 +205,8 @@ size_t gemm_workspace_bytes(gemm_plan_t plan);
  * (asynchronous; the hot path of Section 5.4).  A, B, C: device pointers, 16-byte
  * aligned, laid out as `desc` said.  bias: device fp32[N] (fp32[M] with
  * GEMM_FLAG_BIAS_PER_ROW), shared by all batches, required iff the epilogue
- * has a bias.  C is read only when beta != 0.  workspace: device
+ * has a bias.  C is read only when beta != 0, and only the M x N elements of D (per batch) are written: row padding
+ * (ldc > N) and gaps between batches keep their contents, so D may be a column block of a wider matrix.  workspace: device
  * memory of at least gemm_workspace_bytes(plan) bytes, 16-byte aligned (may be NULL when
  * that is 0).  Runs of one dense plan may overlap on the GPU; runs of one
  * stream-K plan must not (they share the plan's arrival counters, which every

@@ -21,7 +21,7 @@ BF16, F16, F32, FP8_E4M3, FP8_E5M2 = 0, 1, 2, 3, 4
 OP_N, OP_T = 0, 1
 (EPI_NONE, EPI_BIAS, EPI_RELU, EPI_BIAS_RELU, EPI_GELU_ERF, EPI_BIAS_GELU_ERF, EPI_GELU_TANH, EPI_BIAS_GELU_TANH,
  EPI_SILU, EPI_BIAS_SILU) = range(10)
-STRUCT_B_LOWER, STRUCT_B_UPPER = 0x1, 0x2     # gemm_desc_t.structure
+STRUCT_B_LOWER, STRUCT_B_UPPER, STRUCT_D_MIRROR = 0x1, 0x2, 0x4     # gemm_desc_t.structure
 VARIANT_AUTO, VARIANT_DENSE_1CTA, VARIANT_DENSE_2CTA, VARIANT_SKINNY_STREAMK, VARIANT_DENSE_2CTA_WIDE = 0, 1, 2, 3, 4
 REGIME_NAMES = {0: "memory-bound", 1: "middle-zone", 2: "compute-bound"}
 FLAG_DEBUG_STALL = 0x80000000

@@ -57,6 +57,10 @@ __host__ __device__ __forceinline__ uint32_t fast_div(uint32_t n, const FastDiv&
 
 struct DenseParams {
   int M, N, K, batch;
+  // Columns [0, n_full) of a row are whole 16-byte units and leave through the TMA store; a bulk tensor store writes
+  // whole 16-byte units, so when N * (output element size) is not a multiple of 16 the last columns [n_full, N) are
+  // written element by element from the registers instead, and the bytes behind column N - 1 stay untouched.
+  int n_full;
   int tiles_m, tiles_n;  // tiles per matrix; a tile is (128*CG) x bn
   int num_tiles;         // batch * tiles_m * tiles_n
   int raster_group;      // tile rows swept together (column-wise inside the group)
@@ -436,6 +440,22 @@ __device__ __forceinline__ void epilogue_math(float (&v)[32], const uint32_t (&a
   }
 }
 
+// The last columns of a row when they do not fill a 16-byte unit (see DenseParams::n_full): v holds the finished values
+// of columns col0 .. col0 + 31 of row `row`; rounding as in the packed path.
+__device__ __forceinline__ void store_ragged_columns(const DenseParams& p, const float (&v)[32], long long row, int col0, int batch) {
+  if (p.n_full == p.N || col0 + 32 <= p.n_full || col0 >= p.N || row >= p.M) return;
+  const long long off = static_cast<long long>(batch) * p.stride_c + row * p.ldc;
+  void* d = const_cast<void*>(p.c_in);  // (C and D share the buffer)
+#pragma unroll
+  for (int j = 0; j < 32; ++j) {
+    const int c = col0 + j;
+    if (c >= p.n_full && c < p.N) {
+      if (p.out_dtype == 2) static_cast<float*>(d)[off + c] = v[j];
+      else static_cast<uint16_t*>(d)[off + c] = static_cast<uint16_t>(p.out_dtype == 0 ? pack_bf16x2(v[j], 0.0f) : pack_f16x2(v[j], 0.0f));
+    }
+  }
+}
+
 // Both single-issuer roles are run by a whole warp in uniform control flow; only the instructions that
 // must be issued once (TMA, tcgen05.mma, commits, barrier arrivals) sit under elect_one().  That keeps
 // addresses, descriptors and coordinates in uniform registers, which is what those instructions read.
@@ -729,6 +749,7 @@ __device__ __forceinline__ void epilogue_role(const DenseParams& p, const CUtens
           tmem_ld_wait();
         }
         epilogue_math(v, acc, p, row, col0, tc.batch);
+        store_ragged_columns(p, v, row, col0, tc.batch);
 #pragma unroll
         for (int j = 0; j < 8; ++j)
           st_shared_v4(srow + ((static_cast<uint32_t>(j) ^ sw) << 4), __float_as_uint(v[4 * j]), __float_as_uint(v[4 * j + 1]),
@@ -757,6 +778,7 @@ __device__ __forceinline__ void epilogue_role(const DenseParams& p, const CUtens
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
           epilogue_math(v, h == 0 ? acc : acc1, p, row, col0 + h * 32, tc.batch);
+          store_ragged_columns(p, v, row, col0 + h * 32, tc.batch);
           uint32_t pk[16];
           if (p.out_dtype == 0) {
 #pragma unroll
@@ -774,7 +796,7 @@ __device__ __forceinline__ void epilogue_role(const DenseParams& p, const CUtens
       fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) {
-        if (row0 < p.M && col0 < p.N) {
+        if (row0 < p.M && col0 < p.n_full) {
           if (p.l2_hint_d) tma_store_3d_hint(tmD, sbuf, col0, row0, tc.batch, l2_policy_evict_first());
           else tma_store_3d(tmD, sbuf, col0, row0, tc.batch);
         }

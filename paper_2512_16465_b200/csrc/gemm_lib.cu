@@ -19,6 +19,7 @@
 #include <vector>
 
 #include "dense_kernel.cuh"
+#include "mirror_kernel.cuh"
 #include "skinny_kernel.cuh"
 #include "tune_cache.h"
 #include "wide_kernel.cuh"
@@ -144,7 +145,9 @@ gemm_status_t validate(const gemm_desc_t* d) {
   if (d->epilogue < GEMM_EPI_NONE || d->epilogue > GEMM_EPI_BIAS_SILU) return GEMM_ERR_INVALID_ARG;
   if ((d->flags & GEMM_FLAG_A_LOWER) && (d->flags & GEMM_FLAG_A_UPPER)) return GEMM_ERR_INVALID_ARG;
   if ((d->flags & GEMM_FLAG_D_LOWER) && (d->flags & GEMM_FLAG_D_UPPER)) return GEMM_ERR_INVALID_ARG;
-  if ((d->structure & ~(GEMM_STRUCT_B_LOWER | GEMM_STRUCT_B_UPPER)) || d->reserved != 0) return GEMM_ERR_INVALID_ARG;
+  if ((d->structure & ~(GEMM_STRUCT_B_LOWER | GEMM_STRUCT_B_UPPER | GEMM_STRUCT_D_MIRROR)) || d->reserved != 0) return GEMM_ERR_INVALID_ARG;
+  if ((d->structure & GEMM_STRUCT_D_MIRROR) && (!(d->flags & (GEMM_FLAG_D_LOWER | GEMM_FLAG_D_UPPER)) || d->M != d->N || d->batch_count > 65535))
+    return GEMM_ERR_INVALID_ARG;  // a triangle to copy from, and a square D
   if ((d->structure & GEMM_STRUCT_B_LOWER) && (d->structure & GEMM_STRUCT_B_UPPER)) return GEMM_ERR_INVALID_ARG;
   if (d->ab_dtype == GEMM_F32) return GEMM_ERR_UNSUPPORTED;
   // 8-bit operands: K-contiguous storage only (A stored M x K, B stored N x K)
@@ -426,6 +429,7 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   memset(&p, 0, sizeof p);
   p.M = static_cast<int>(d.M);
   p.N = static_cast<int>(d.N);
+  p.n_full = static_cast<int>(d.N - d.N % (16 / elem_bytes(d.c_dtype)));
   p.K = static_cast<int>(d.K);
   p.batch = d.batch_count;
   p.tiles_m = tiles_m;
@@ -531,6 +535,7 @@ gemm_status_t plan_wide(gemm_plan_s* pl, int forced_raster, int forced_stages) {
   // its epilogue covers the bias per column, ReLU and erf GELU only; its MMA schedule has no K-range skipping
   if (d.epilogue > GEMM_EPI_BIAS_GELU_ERF || (d.flags & (GEMM_FLAG_BIAS_PER_ROW | GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER))) return GEMM_ERR_UNSUPPORTED;
   if (d_tri_of(d) || d.structure) return GEMM_ERR_UNSUPPORTED;  // its scheduler has no tile list, its MMA schedule no K ranges
+  if ((d.N * elem_bytes(d.c_dtype)) % 16) return GEMM_ERR_UNSUPPORTED;  // its epilogue has no element-wise path for a partly filled last 16-byte unit of a row
   const int a_kmajor = d.transa == GEMM_OP_N;
   const int b_kmajor = d.transb == GEMM_OP_T;
   const int tile_m = 2 * kWideCtaM, bn = kWideTileN;
@@ -552,6 +557,7 @@ gemm_status_t plan_wide(gemm_plan_s* pl, int forced_raster, int forced_stages) {
   memset(&p, 0, sizeof p);
   p.M = static_cast<int>(d.M);
   p.N = static_cast<int>(d.N);
+  p.n_full = static_cast<int>(d.N - d.N % (16 / elem_bytes(d.c_dtype)));
   p.K = static_cast<int>(d.K);
   p.batch = d.batch_count;
   p.tiles_m = tiles_m;
@@ -733,7 +739,7 @@ gemm_status_t plan_impl(const gemm_desc_t* desc, gemm_plan_t* out_plan, bool use
         for (int bn : {256, 192, 128, 64}) {
           if (v == GEMM_VARIANT_DENSE_2CTA_WIDE && bn != kWideTileN) continue;
           if (v == GEMM_VARIANT_DENSE_2CTA_WIDE &&
-              (d.epilogue > GEMM_EPI_BIAS_GELU_ERF || d_tri_of(d) || d.structure ||
+              (d.epilogue > GEMM_EPI_BIAS_GELU_ERF || d_tri_of(d) || d.structure || (d.N * elem_bytes(d.c_dtype)) % 16 ||
                (d.flags & (GEMM_FLAG_BIAS_PER_ROW | GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER))))
             continue;
           if (v == GEMM_VARIANT_DENSE_2CTA && !b_kmajor && bn % 128) continue;  // 64-column boxes per CTA
@@ -955,7 +961,9 @@ gemm_status_t run_dense(gemm_plan_s* pl, const void* A, const void* B, void* C, 
   ok = ok && (p.b_kmajor ? encode_map(&tB, d.ab_dtype, B, d.K, d.N, batch, d.ldb, d.stride_b, p.kblk, p.b_rows)
                          : encode_map(&tB, d.ab_dtype, B, d.N, d.K, batch, d.ldb, d.stride_b, 64, kBlockK));
   const uint32_t slab_cols = d.c_dtype == GEMM_F32 ? 32 : 64;
-  ok = ok && encode_map(&tD, d.c_dtype, C, d.N, d.M, batch, d.ldc, d.stride_c, slab_cols, 32);
+  // (whole 16-byte units of a row only: the store engine writes whole units, see DenseParams::n_full)
+  const uint64_t d_cols = std::max<uint64_t>(p.n_full, 16 / elem_bytes(d.c_dtype));
+  ok = ok && encode_map(&tD, d.c_dtype, C, d_cols, d.M, batch, d.ldc, d.stride_c, slab_cols, 32);
   if (!ok) return GEMM_ERR_CUDA;
   p.alpha = alpha;
   p.beta = beta;
@@ -965,14 +973,32 @@ gemm_status_t run_dense(gemm_plan_s* pl, const void* A, const void* B, void* C, 
   p.status = pl->d_status;
   p.timeout_ns = static_cast<unsigned long long>(pl->timeout_ms) * 1000000ull;
   if (pl->variant == GEMM_VARIANT_DENSE_2CTA_WIDE) return launch_wide(pl, tA, tB, tD, p, stream);
+  gemm_status_t st;
   if (pl->split > 1) {
     p.partials = static_cast<float*>(workspace);
     p.split_flags = reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(pl->d_status) + 256);
-    if (pl->cg == 1) return pl->epi_wg == 2 ? launch_dense<1, 2, true>(pl, tA, tB, tD, p, stream) : launch_dense<1, 1, true>(pl, tA, tB, tD, p, stream);
-    return pl->epi_wg == 2 ? launch_dense<2, 2, true>(pl, tA, tB, tD, p, stream) : launch_dense<2, 1, true>(pl, tA, tB, tD, p, stream);
+    if (pl->cg == 1) st = pl->epi_wg == 2 ? launch_dense<1, 2, true>(pl, tA, tB, tD, p, stream) : launch_dense<1, 1, true>(pl, tA, tB, tD, p, stream);
+    else st = pl->epi_wg == 2 ? launch_dense<2, 2, true>(pl, tA, tB, tD, p, stream) : launch_dense<2, 1, true>(pl, tA, tB, tD, p, stream);
+  } else if (pl->cg == 1) {
+    st = pl->epi_wg == 2 ? launch_dense<1, 2, false>(pl, tA, tB, tD, p, stream) : launch_dense<1, 1, false>(pl, tA, tB, tD, p, stream);
+  } else {
+    st = pl->epi_wg == 2 ? launch_dense<2, 2, false>(pl, tA, tB, tD, p, stream) : launch_dense<2, 1, false>(pl, tA, tB, tD, p, stream);
   }
-  if (pl->cg == 1) return pl->epi_wg == 2 ? launch_dense<1, 2, false>(pl, tA, tB, tD, p, stream) : launch_dense<1, 1, false>(pl, tA, tB, tD, p, stream);
-  return pl->epi_wg == 2 ? launch_dense<2, 2, false>(pl, tA, tB, tD, p, stream) : launch_dense<2, 1, false>(pl, tA, tB, tD, p, stream);
+  if (st == GEMM_OK && (d.structure & GEMM_STRUCT_D_MIRROR)) {  // symmetric result: copy the computed triangle into the other one
+    MirrorParams mp;
+    mp.d = C;
+    mp.ldc = d.ldc;
+    mp.stride = d.batch_count > 1 ? d.stride_c : 0;
+    mp.n = static_cast<int>(d.M);
+    mp.blocks = ceil_div(d.M, 32);
+    mp.upper_source = (d.flags & GEMM_FLAG_D_UPPER) ? 1 : 0;
+    const cudaError_t e = mirror_launch(mp, elem_bytes(d.c_dtype), d.batch_count, stream);
+    if (e != cudaSuccess) {
+      note_cuda_error("mirror kernel launch", cudaGetErrorName(e));
+      return GEMM_ERR_CUDA;
+    }
+  }
+  return st;
 }
 
 gemm_status_t run_skinny(gemm_plan_s* pl, const void* A, const void* B, void* C, const float* bias, float alpha, float beta,
@@ -1102,7 +1128,8 @@ extern "C" gemm_status_t gemm_skinny_run_noalloc(const gemm_desc_t* desc, const 
   gemm_status_t st = validate(desc);
   if (st != GEMM_OK) return st;
   if (has_bias(desc->epilogue) && !bias) return GEMM_ERR_NULL;
-  if (desc->transa != GEMM_OP_N || desc->transb != GEMM_OP_T || desc->batch_count != 1 || desc->M > kSkinnyMaxM || is_fp8(desc->ab_dtype))
+  if (desc->transa != GEMM_OP_N || desc->transb != GEMM_OP_T || desc->batch_count != 1 || desc->M > kSkinnyMaxM || is_fp8(desc->ab_dtype) ||
+      (desc->structure & GEMM_STRUCT_D_MIRROR))  // (the mirror step belongs to the dense plans)
     return GEMM_ERR_UNSUPPORTED;
   auto misaligned = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; };
   if (misaligned(A) || misaligned(B) || misaligned(C) || (bias && misaligned(bias))) return GEMM_ERR_ALIGNMENT;

@@ -71,7 +71,7 @@ def desc_of(w: wl.Workload, flags: int = 0, c_dtype=None) -> bg.Desc:
     return bg.make_desc(w.M, w.N, w.K, w.transa, w.transb, w.ab_dtype, cd, w.lda, w.ldb, w.ldc, w.batch,
                         w.stride_a, w.stride_b, w.stride_c, w.epilogue, flags | bg.make_flags(bias_per_row=w.bias_per_row, a_lower=w.a_tri == 1, a_upper=w.a_tri == 2,
                                                                                            d_lower=w.d_tri == 1, d_upper=w.d_tri == 2),
-                        structure=w.b_tri)
+                        structure=w.b_tri | (4 if w.d_mirror else 0))
 
 
 def problem_of(w: wl.Workload, c_dtype=None) -> oracle.Problem:
@@ -172,6 +172,12 @@ def check_blocks(w: wl.Workload, inputs: dict, cbits: np.ndarray, blocks, c_dtyp
         untouched = np.isnan(out_val) if cin is None else out_bits == gather(cin, w, batches, rows, cols)[~keep]
         with np.errstate(invalid="ignore"):
             plain = np.abs(out_val - out_y) <= REL_TOL * out_bound + ABS_TOL + U_OUT[cd] * np.abs(out_y)
+        if w.d_mirror:   # symmetric result: every other element holds the bits of its mirror image
+            image = np.swapaxes(gather(cbits, w, batches, cols, rows), 1, 2)
+            rep["outside_ok"] = bool(np.array_equal(out_bits, image[~keep]))
+            rep["outside_untouched"], rep["outside_n"], rep["transcendental"] = 0, int(out_bits.size), w.epilogue >= 4
+            reports.append(rep)
+            continue
         rep["outside_ok"] = bool(np.all(untouched | plain))
         rep["outside_untouched"] = int(np.sum(untouched))
         rep["outside_n"] = int(untouched.size)
@@ -212,6 +218,24 @@ def assert_reports(reports, what=""):
             assert r["bit_identical"] >= floor, f"{what}: too many one-ulp flips {r}"
 
 
+def assert_padding_untouched(w: wl.Workload, inputs: dict, cbits: np.ndarray, c_dtype=None):
+    """Everything in the C buffer that is not an element of D -- the row padding behind column N - 1 when ldc > N, the
+    gaps between batches -- must still hold what it held before the run (C_in, or the NaN poison).  A matrix that is a
+    column block of a larger one has its neighbours' data there."""
+    cd = w.c_dtype if c_dtype is None else c_dtype
+    if w.elems_c() == w.batch * w.M * w.N:
+        return
+    mask = np.ones(w.elems_c(), bool)
+    for b in range(w.batch):
+        idx = b * w.stride_c + np.arange(w.M, dtype=np.int64)[:, None] * w.ldc + np.arange(w.N, dtype=np.int64)[None, :]
+        mask[idx.ravel()] = False
+    cin = c_in_as(inputs, w, cd)
+    if cin is not None:
+        assert np.array_equal(cbits[mask], cin[mask]), f"{w.name}: bytes outside D were overwritten"
+    else:
+        assert np.all(np.isnan(oracle.decode(cbits[mask].copy(), cd))), f"{w.name}: bytes outside D were overwritten"
+
+
 def check_workload(w: wl.Workload, flags: int = 0, exact: bool = False, c_dtype=None, repeats: int = 1, inputs=None):
     """Run + compare.  exact=True additionally requires bit equality with the rounded oracle
     (for integer-valued inputs whose every partial sum is exactly representable)."""
@@ -219,6 +243,7 @@ def check_workload(w: wl.Workload, flags: int = 0, exact: bool = False, c_dtype=
     cbits, info = run_gpu(w, inputs, flags, c_dtype, repeats=repeats)
     reports = check_blocks(w, inputs, cbits, default_blocks(w), c_dtype)
     assert_reports(reports, what=w.name)
+    assert_padding_untouched(w, inputs, cbits, c_dtype)
     if exact:
         for r in reports:
             assert r["bit_identical"] == 1.0, f"{w.name}: not bit-exact {r} {info}"

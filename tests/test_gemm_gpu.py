@@ -177,6 +177,13 @@ EXACT_CASES = [
     ("lower_a_upper_b", 712, 712, 712, dict(a_tri=1, b_tri=2, epi=bg.EPI_BIAS, beta=1.0), dict(variant=V1, tile_n=128)),
     ("upper_times_upper_batched_fp8", 384, 384, 384, dict(a_tri=2, b_tri=2, d_tri=2, batch=3, ab=wl.FP8_E4M3), dict(variant=V1, tile_n=64)),
     ("upper_times_upper_auto", 2048, 2048, 2048, dict(a_tri=2, b_tri=2, d_tri=2, cd=wl.BF16), dict()),
+    # symmetric result: the computed triangle copied into the other one (every element beyond the diagonal equals its mirror image)
+    ("mirror_lower_1cta", 700, 700, 200, dict(d_tri=1, d_mirror=True), dict(variant=V1, tile_n=128)),
+    ("mirror_upper_pair_bf16", 1104, 1104, 264, dict(d_tri=2, d_mirror=True, cd=wl.BF16), dict(variant=V2, tile_n=256)),
+    ("mirror_lower_ragged_blocks_f16", 1000, 1000, 136, dict(d_tri=1, d_mirror=True, ab=wl.F16, cd=wl.F16, beta=1.0, epi=bg.EPI_BIAS), dict(variant=V2, tile_n=192)),
+    ("mirror_upper_batched_padded", 200, 200, 72, dict(d_tri=2, d_mirror=True, batch=3, ldc=216, stride_c=200 * 216 + 64), dict(variant=V1, tile_n=64)),
+    ("mirror_lower_tiny", 5, 5, 8, dict(d_tri=1, d_mirror=True, ldc=8), dict(variant=V1)),
+    ("mirror_lower_auto_with_triangular_factors", 1536, 1536, 1536, dict(d_tri=1, a_tri=1, b_tri=1, d_mirror=True, cd=wl.BF16, sample_rows=96, sample_cols=96), dict()),
     # dealt schedules with empty slots in the middle of a CTA's sequence: more tiles than CTAs, not a multiple, batched
     ("d_lower_batched_two_rounds", 2304, 2304, 136, dict(d_tri=1, batch=2, cd=wl.BF16, sample_rows=96, sample_cols=96), dict(variant=V1, tile_n=128)),
     ("tri_upper_batched_two_rounds", 2304, 1152, 1160, dict(a_tri=2, batch=3, sample_rows=96, sample_cols=96), dict(variant=V1, tile_n=128)),
@@ -610,6 +617,42 @@ def test_tail_split_plans():
     assert i["split"] == 7 and i["grid"] == 56 and i["workspace_bytes"] == 4 * 2 * 6 * 128 * 256 * 4
 
 
+@pytest.mark.parametrize("cd,N", [(wl.BF16, 900), (wl.F16, 899), (wl.F32, 901), (wl.F32, 5), (wl.BF16, 3)])
+def test_output_is_a_column_block_of_a_larger_matrix(cd, N):
+    """D is columns [c0, c0 + N) of a wider row-major matrix whose other columns hold live data; N times the element
+    size is not a multiple of 16 bytes, so the last 16-byte unit of every row of D is shared with the neighbour.
+    Every dense family (the wide pair kernel where it accepts the shape) must leave the neighbours bit for bit."""
+    M, K, wide_cols = 300, 264, 1024
+    c0 = 96
+    w = int_workload("column_block", M, N, K, cd=cd, ldc=wide_cols, beta=1.0, epi=bg.EPI_BIAS_RELU)
+    inputs = wl.make_inputs(w)
+    A, B, bias = H.to_device(inputs["A"], w.ab_dtype), H.to_device(inputs["B"], w.ab_dtype), H.to_device(inputs["bias"], wl.F32)
+    esz = 4 if cd == wl.F32 else 2
+    for fl in (dict(variant=V1), dict(variant=V2, tile_n=128), dict(variant=VS) if N <= 64 else dict(variant=V1, tile_n=256, tail_split=True), dict()):
+        rng = np.random.default_rng(3)
+        full = rng.integers(1, 60000, size=(M, wide_cols)).astype(inputs["C"].dtype)   # a matrix of other data (bit patterns) ...
+        cin_rows = np.stack([inputs["C"][i * wide_cols: i * wide_cols + N] for i in range(M)])
+        full[:, c0:c0 + N] = cin_rows                                                   # ... with C_in as its column block
+        big = H.to_device(full.ravel(), cd)
+        plan = bg.Plan(H.desc_of(w, bg.make_flags(**fl)))
+        try:
+            ws = plan.workspace(big.device)
+            bg.gemm_run(plan.handle, A.data_ptr(), B.data_ptr(), big.data_ptr() + c0 * esz, bias.data_ptr(), float(w.alpha), float(w.beta),
+                        0 if ws is None else ws.data_ptr(), 0 if ws is None else ws.numel(), torch.cuda.current_stream().cuda_stream)
+            torch.cuda.synchronize()
+            assert plan.status() == bg.OK
+        finally:
+            plan.close()
+        got = H.to_host_bits(big, cd).reshape(M, wide_cols)
+        assert np.array_equal(got[:, :c0], full[:, :c0]) and np.array_equal(got[:, c0 + N:], full[:, c0 + N:]), fl
+        # D itself: lay the block out as the workload describes it (row pitch wide_cols, starting at column c0)
+        cbits = np.zeros(w.elems_c(), got.dtype)
+        flat = got.ravel()[c0:]
+        cbits[:flat.size] = flat
+        reports = H.check_blocks(w, inputs, cbits, H.default_blocks(w))
+        assert all(r["bit_identical"] == 1.0 for r in reports), fl
+
+
 def test_triangular_a_really_skips():
     """Lower-triangular A, 512 x 512: every kernel variant works on tile rows of at most 256 and ring stages of at most
     128 columns, so element (i, k) with k >= 256 (i // 256 + 1) lies in a stage no tile may visit.  NaN there must
@@ -686,6 +729,32 @@ def test_triangular_d_leaves_the_other_tiles_alone(d_tri):
     with pytest.raises(bg.GemmError) as e:
         bg.gemm_plan(H.desc_of(int_workload("d_tri_both", 256, 256, 64), bg.make_flags(d_lower=True, d_upper=True)))
     assert e.value.status == bg.ERR_INVALID_ARG
+
+
+def test_symmetric_result_is_symmetric_everywhere():
+    """D = A A^T, lower triangle computed and mirrored: the whole matrix against the oracle, equal to its transpose bit
+    for bit, padding untouched; and the option is refused where it has no meaning."""
+    w = wl.Workload("syrk_mirror", 900, 900, 520, transa=0, transb=1, c_dtype=wl.BF16, d_tri=1, d_mirror=True, ldc=912, seed=6)
+    inputs = wl.make_inputs(w)
+    inputs["B"] = inputs["A"].copy()
+    cbits, _ = H.run_gpu(w, inputs, 0)
+    H.assert_reports(H.check_blocks(w, inputs, cbits, H.default_blocks(w)), what="mirrored")
+    full = cbits.reshape(900, 912)
+    assert np.array_equal(full[:, :900], full[:, :900].T)
+    assert np.all(full[:, 900:] == 0x7FC0) or np.all(np.isnan(oracle.decode(full[:, 900:].copy(), wl.BF16)))   # NaN poison of the padding
+    # the symmetric product as a whole is the plain product: compare the mirrored half with the oracle as well
+    plain = replace(w, d_tri=0, d_mirror=False)
+    H.assert_reports(H.check_blocks(plain, inputs, cbits, H.default_blocks(plain)), what="against the plain product")
+    for kw, st in ((dict(structure=bg.STRUCT_D_MIRROR), bg.ERR_INVALID_ARG),                                        # no triangle named
+                   (dict(structure=bg.STRUCT_D_MIRROR, flags=bg.make_flags(d_lower=True), N=520), bg.ERR_INVALID_ARG)):  # not square
+        d = dict(M=512, N=512, K=64)
+        d.update(kw)
+        with pytest.raises(bg.GemmError) as e:
+            bg.gemm_plan(bg.make_desc(d.pop("M"), d.pop("N"), d.pop("K"), **d))
+        assert e.value.status == st
+    with pytest.raises(bg.GemmError) as e:
+        bg.gemm_plan(bg.make_desc(4096, 4096, 4096, flags=bg.make_flags(variant=VW, d_lower=True), structure=bg.STRUCT_D_MIRROR))
+    assert e.value.status == bg.ERR_UNSUPPORTED
 
 
 def test_triangular_d_general_values_symmetric_product():

@@ -114,6 +114,7 @@ class Workload:
     a_tri: int = 0               # structure of op(A): 0 dense, 1 lower triangular (zero for k > i), 2 upper (zero for k < i)
     b_tri: int = 0               # structure of op(B): 0 dense, 1 lower triangular (zero for k < j), 2 upper (zero for k > j)
     d_tri: int = 0               # part of D that is wanted: 0 all, 1 lower triangle (row >= column), 2 upper (row <= column)
+    d_mirror: bool = False       # with d_tri and M == N: the wanted triangle is copied into the other one (symmetric D)
     alpha: float = 1.0
     beta: float = 0.0
     dist_a: Dist = field(default_factory=lambda: Dist("normal", 0.0, 1.0))
