@@ -208,10 +208,10 @@ size_t gemm_workspace_bytes(gemm_plan_t plan);
  * has a bias.  C is read only when beta != 0, and only the M x N elements of D (per batch) are written: row padding
  * (ldc > N) and gaps between batches keep their contents, so D may be a column block of a wider matrix.  workspace: device
  * memory of at least gemm_workspace_bytes(plan) bytes, 16-byte aligned (may be NULL when
- * that is 0).  Runs of one dense plan may overlap on the GPU; runs of one
- * stream-K plan must not (they share the plan's arrival counters, which every
- * run leaves at zero): order them on one stream or with events, or make one
- * plan per stream.  alpha and beta are host scalars.  The call only encodes tensor maps on the
+ * that is 0).  Runs of one plan that needs no workspace may overlap on the GPU; runs of a plan that
+ * needs one (stream-K, or a dense plan with a tail split: gemm_workspace_bytes > 0) must not -- they
+ * share the plan's arrival counters or flags, which every run leaves at zero: order them on one
+ * stream or with events, or make one plan per stream.  alpha and beta are host scalars.  The call only encodes tensor maps on the
  * host and launches: once a plan has run once (which sets kernel attributes), further runs may be recorded by stream
  * capture into a CUDA graph (tested).  Errors are returned before anything is launched:
  * GEMM_ERR_NULL, GEMM_ERR_ALIGNMENT, GEMM_ERR_WORKSPACE, GEMM_ERR_ARCH,
