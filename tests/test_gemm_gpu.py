@@ -505,11 +505,13 @@ def test_runs_on_a_side_stream():
 
 def test_runs_are_capturable_in_a_cuda_graph():
     """gemm_run only encodes tensor maps on the host and launches: after one ordinary run (which sets the kernel
-    attributes) a chain of a dense and a stream-K GEMM is captured into a CUDA graph and replayed with new inputs."""
+    attributes) a chain of a dense, a stream-K and a mirrored symmetric GEMM is captured into a CUDA graph and replayed
+    with new inputs."""
     w1 = int_workload("graph_dense", 512, 384, 256, cd=wl.BF16)
     w2 = int_workload("graph_stream_k", 8, 512, 4096, beta=0.0)
+    w3 = int_workload("graph_symmetric", 520, 520, 264, cd=wl.BF16, d_tri=1, d_mirror=True)   # a dealt schedule and two kernels per run
     cases = []
-    for w in (w1, w2):
+    for w in (w1, w2, w3):
         inputs = wl.make_inputs(w)
         plan = bg.Plan(H.desc_of(w))
         A, B = H.to_device(inputs["A"], w.ab_dtype), H.to_device(inputs["B"], w.ab_dtype)
@@ -918,6 +920,32 @@ def test_tuning_results_survive_in_a_file(tmp_path):
     p = bg.Plan(bg.make_desc(1024, 1024, 512, c_dtype=bg.BF16, epilogue=bg.EPI_SILU))
     assert p.info["variant"] != VW
     p.close()
+    bg.gemm_tune_cache_clear()
+
+
+def test_tune_keeps_structure_flags():
+    """Measured plan selection on a structured problem (upper x upper -> upper, mirrored): the candidates keep the
+    caller's structure words, the kernels that cannot honour them are skipped, and the tuned plan is exact."""
+    bg.gemm_tune_cache_clear()
+    w = int_workload("tune_structured", 1104, 1104, 1104, cd=wl.BF16, a_tri=2, b_tri=2, d_tri=2, d_mirror=True)
+    inputs, A, B, C, desc, plan, rep = _tune_case(w)
+    assert rep["candidates_skipped"] >= 1 and rep["best_flags"] & 0x8000 and rep["best_flags"] & 0x800000     # D_UPPER, A_UPPER survive
+    C.fill_(float("nan"))
+    plan.run(A, B, C)
+    torch.cuda.synchronize()
+    assert plan.status() == bg.OK
+    got = H.to_host_bits(C, w.c_dtype)
+    reports = H.check_blocks(w, inputs, got, H.default_blocks(w))
+    H.assert_reports(reports, what="tuned structured plan")
+    assert all(r["bit_identical"] == 1.0 for r in reports)
+    full = got.reshape(1104, 1104)
+    assert np.array_equal(full, full.T)
+    again = bg.Plan(desc)                       # the remembered choice is keyed by the structure word too
+    assert again.info["variant"] == plan.info["variant"] and again.info["tile_n"] == plan.info["tile_n"]
+    plain = bg.Plan(bg.make_desc(1104, 1104, 1104, c_dtype=bg.BF16))
+    assert plain.info["flops"] > 1.9 * again.info["flops"]        # (the plain problem was not touched by the remembered choice)
+    for p in (plan, again, plain):
+        p.close()
     bg.gemm_tune_cache_clear()
 
 
