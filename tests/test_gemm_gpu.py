@@ -655,6 +655,32 @@ def test_output_is_a_column_block_of_a_larger_matrix(cd, N):
         assert all(r["bit_identical"] == 1.0 for r in reports), fl
 
 
+@pytest.mark.parametrize("fl,M,N", [(dict(variant=V1), 300, 264), (dict(variant=V2, tile_n=128), 300, 264), (dict(variant=VW), 600, 264),
+                                    (dict(variant=VS), 8, 520), (dict(variant=VS), 520, 8)])
+def test_non_finite_inputs_propagate_like_the_definition(fl, M, N):
+    """A NaN and infinities in A: exactly the output elements the definition makes NaN or infinite are (with the sign the
+    definition gives), every other element is untouched by them and within the usual tolerance."""
+    K = 520
+    w = wl.Workload("non_finite", M, N, K, transb=1, c_dtype=wl.F32, dist_a=wl.Dist("normal", 0, 1), dist_b=wl.Dist("normal", 0, 1), seed=21)
+    inputs = wl.make_inputs(w)
+    a = inputs["A"].reshape(M, K)
+    b = inputs["B"].reshape(N, K)
+    a[1, 7] = 0x7FC0                      # NaN: row 1 of D is NaN
+    a[3, 100] = 0x7F80                    # +Inf: row 3 is +-Inf by the sign of B[:, 100] ...
+    b[5, 100] = 0x0000                    # ... and NaN where that element of B is zero (Inf * 0)
+    a[M - 1, 0] = 0x7F80
+    a[M - 1, K - 1] = 0xFF80              # +Inf and -Inf in one row: NaN wherever the two products have opposite signs
+    cbits, _ = H.run_gpu(w, inputs, bg.make_flags(**fl))
+    got = cbits.reshape(M, N).astype(np.float64)
+    y, bound = oracle.gemm(H.problem_of(w), inputs["A"], inputs["B"])
+    y, bound = y[0], bound[0]
+    assert np.array_equal(np.isnan(got), np.isnan(y))
+    assert np.array_equal(np.isinf(got), np.isinf(y)) and np.array_equal(np.sign(got[np.isinf(y)]), np.sign(y[np.isinf(y)]))
+    assert np.isnan(y[1]).all() and np.isinf(y[3, 0]) and np.isnan(y[3, 5]) and np.isnan(y[M - 1]).any()      # the cases are really there
+    fin = np.isfinite(y)
+    assert np.all(np.abs(got[fin] - y[fin]) <= H.REL_TOL * bound[fin] + H.ABS_TOL)
+
+
 def test_triangular_a_really_skips():
     """Lower-triangular A, 512 x 512: every kernel variant works on tile rows of at most 256 and ring stages of at most
     128 columns, so element (i, k) with k >= 256 (i // 256 + 1) lies in a stage no tile may visit.  NaN there must
