@@ -681,6 +681,23 @@ def test_non_finite_inputs_propagate_like_the_definition(fl, M, N):
     assert np.all(np.abs(got[fin] - y[fin]) <= H.REL_TOL * bound[fin] + H.ABS_TOL)
 
 
+@pytest.mark.parametrize("ab", [wl.BF16, wl.F16])
+def test_subnormal_inputs_are_not_flushed(ab):
+    """A holds subnormal numbers of the input format, B large ones, so that every product is an ordinary number
+    (2^-10): a tensor pipe that flushed subnormal operands to zero would return zeros.  Exact in fp32 (powers of two)."""
+    small, large = (0x0001, 0x7D00) if ab == wl.BF16 else (0x0010, 0x6400)   # bf16: 2^-133 and 2^123; fp16: 2^-20 and 2^10
+    for fl, M, N in ((dict(variant=V1), 200, 264), (dict(variant=V2, tile_n=128), 300, 264), (dict(variant=VW), 600, 264), (dict(variant=VS), 8, 520)):
+        K = 64
+        w = wl.Workload("subnormal", M, N, K, transb=1, ab_dtype=ab, c_dtype=wl.F32, seed=3)
+        inputs = wl.make_inputs(w)
+        inputs["A"][:] = small
+        inputs["B"][:] = large
+        cbits, _ = H.run_gpu(w, inputs, bg.make_flags(**fl))
+        y, _ = oracle.gemm(H.problem_of(w), inputs["A"], inputs["B"])
+        assert y[0, 0, 0] == K * 2.0 ** -10
+        assert np.array_equal(cbits.reshape(M, N).astype(np.float64), y[0]), fl
+
+
 def test_triangular_a_really_skips():
     """Lower-triangular A, 512 x 512: every kernel variant works on tile rows of at most 256 and ring stages of at most
     128 columns, so element (i, k) with k >= 256 (i // 256 + 1) lies in a stage no tile may visit.  NaN there must
