@@ -631,7 +631,7 @@ gemm_status_t plan_skinny(gemm_plan_s* pl, int forced_stages, int forced_atoms) 
   const int small_extent = static_cast<int>(pl->skinny_tall ? d.N : d.M), big_extent = static_cast<int>(pl->skinny_tall ? d.M : d.N);
   if (forced_atoms > 3) return GEMM_ERR_UNSUPPORTED;
   if (!skinny_make_plan(&s, small_extent, big_extent, static_cast<int>(d.K), pl->sm_count, forced_stages, kMaxSmemOptin, forced_atoms,
-                        kblk_of(d.ab_dtype)))
+                        kblk_of(d.ab_dtype), /*align=*/true))
     return GEMM_ERR_UNSUPPORTED;
   pl->variant = GEMM_VARIANT_SKINNY_STREAMK;
   pl->cg = 1;
