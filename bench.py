@@ -40,7 +40,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the full-size ncu captures
 # summarised under profiles/ (dense_*_cN_*.txt, skinny_streamk_c5_*.txt; last line of each file).
-NCU_TRAFFIC_BYTES = {"c1": 1119488, "c2": 806943488, "c3": 1538906584, "c4": 545963520, "c5": 476679424}
+NCU_TRAFFIC_BYTES = {"c1": 1121536, "c2": 806143488, "c3": 1499963344, "c4": 545859840, "c5": 477242880}
 
 
 def load_peaks():

@@ -127,6 +127,17 @@ def test_stream_k_plan_geometry():
     assert i5["workspace_bytes"] == 148 * 2 * 128 * 16 * 4
     tiny = info_for(wl.Workload("t", 4, 100, 64), bg.make_flags(bg.VARIANT_SKINNY_STREAMK))
     assert tiny["grid"] == 1 and tiny["num_tiles"] == 1
+    # grids that line up with the tiles on mid-sized problems
+    sk = bg.make_flags(bg.VARIANT_SKINNY_STREAMK)
+    grid = lambda M, N, K: bg.Plan(bg.make_desc(M, N, K, flags=sk)).info["grid"]
+    assert grid(64, 4096, 4096) == 128        # 32 tiles x 64 units: four CTAs per tile
+    assert grid(16, 4096, 4096) == 128        # 32 tiles x 32 double units: four CTAs per tile
+    assert grid(64, 12288, 4096) == 96        # one whole tile per CTA (mid-sized: 100 MB streamed)
+    assert grid(64, 14336, 16384) == 112      # one whole tile per CTA: more than two thirds of the SMs, any size
+    assert grid(16, 11008, 16384) == 148      # 86 whole tiles would starve the memory system on 360 MB: unchanged
+    assert grid(64, 5120, 5120) == 80         # two CTAs per tile, smallest problems only
+    assert grid(64, 8192, 8192) == 148        # two CTAs per tile would cost what they save here
+    assert grid(8192, 64, 4096 * 2) == grid(64, 8192, 4096 * 2)   # the tall form shares the rule
 
 
 def test_forced_variants_and_tiles():
