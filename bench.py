@@ -10,9 +10,13 @@ metric is quoted on; ``--all`` (default on) adds one entry per benchmark configu
 ``configs_measured``.  Prints ONE JSON line on rank 0.
 
 Timing: CUDA events on the launching stream around K back-to-back steps, after W >= 3 warm-up
-steps; inputs rotate through enough seeded buffer sets to exceed twice the L2 capacity, so no
-step finds its operands in cache.  ``e2e`` repeats the measurement with host-resident pinned
+steps; every configuration rotates through at least two (HBM-bound ones: three) seeded sets of
+inputs AND outputs, and through as many as it takes to exceed twice the L2 capacity, so no step
+finds its operands, or a dirty copy of its output, in cache (the paper's Section 5.1 protocol:
+different random inputs per run).  ``e2e`` repeats the measurement with host-resident pinned
 inputs and output: every step copies A and B to the device, runs the GEMM and copies D back.
+``library_reference`` times the vendor GEMM (torch) on the same buffers in the same loop and
+``sustained`` repeats the headline for at least four seconds: both are context, outside the product.
 
 ``--impl reference`` times the CPU oracle (the fp64 triple loop) on a bounded sample of the same
 workload; it is a deliberately slow program and only a reported baseline.
@@ -38,9 +42,25 @@ L2_BYTES = 126 * 1024 * 1024
 NOMINAL = {"tensor_tflops": 2250.0, "hbm_gbs": 8000.0}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the full-size ncu captures
-# summarised under profiles/ (dense_*_cN_*.txt, skinny_streamk_c5_*.txt; last line of each file).
-NCU_TRAFFIC_BYTES = {"c1": 1121536, "c2": 806143488, "c3": 1499963344, "c4": 545859840, "c5": 477242880}
+# The ncu summary of each configuration's kernel (profiles/): its line "dram traffic per launch (read + write): N bytes"
+# is dram__bytes_read.sum + dram__bytes_write.sum of one captured launch and becomes roofline.traffic.
+PROFILE_OF = {"c1": "dense_1cta_c1_512_nn.txt", "c2": "wide_2cta_c2_square_8192.txt", "c3": "dense_2cta_c3_proj_bias_gelu.txt",
+              "c4": "wide_2cta_c4_batched_fp16.txt", "c5": "skinny_streamk_c5_8x28672x8192.txt"}
+
+
+def ncu_traffic_bytes(key: str):
+    """DRAM bytes per launch from the committed ncu summary of this configuration's kernel, or None."""
+    name = PROFILE_OF.get(key)
+    if not name:
+        return None
+    try:
+        with open(os.path.join(ROOT, "profiles", name)) as f:
+            for line in f:
+                if line.startswith("dram traffic per launch (read + write):"):
+                    return int(line.split(":")[1].split()[0])
+    except (OSError, ValueError):
+        pass
+    return None
 
 
 def load_peaks():
@@ -116,7 +136,7 @@ def roofline_for(w: wl.Workload, key: str, seconds: float, peaks: dict, peak_kin
     else:
         achieved, peak, unit, bound = w.min_bytes / seconds / 1e9, peaks["hbm_gbs"], "GB/s", "hbm"
     return {"bound": bound, "achieved": round(achieved, 2), "peak": peak, "unit": unit, "frac": round(achieved / peak, 4),
-            "traffic": NCU_TRAFFIC_BYTES.get(key), "peak_source": f"of {peak_kind}" + (" bf16 x 2 (nominal fp8 ratio)" if fp8 and bound == "tensor" else ""),
+            "traffic": ncu_traffic_bytes(key), "peak_source": f"of {peak_kind}" + (" bf16 x 2 (nominal fp8 ratio)" if fp8 and bound == "tensor" else ""),
             "frac_of_nominal": round(achieved / (NOMINAL["tensor_tflops"] * (2.0 if fp8 else 1.0) if bound == "tensor" else NOMINAL["hbm_gbs"]), 4),
             "algorithmic_flops": w.flops, "algorithmic_bytes": w.min_bytes}
 
@@ -140,10 +160,15 @@ def _to_torch(torch, arr, code, device=None, pin=False):
 class DeviceCase:
     """One benchmark configuration resident in HBM: R rotating input sets and a plan."""
 
-    def __init__(self, torch, bg, key: str, w: wl.Workload, flags: int, device):
+    def __init__(self, torch, bg, key: str, w: wl.Workload, flags: int, device, nsets_cap: int = 160):
         self.torch, self.bg, self.key, self.w, self.device = torch, bg, key, w, device
         footprint = w.min_bytes
-        self.nsets = int(max(1, min(160, -(-2 * L2_BYTES // int(footprint))))) if footprint < 2 * L2_BYTES else 1
+        # Rotating sets (inputs and output buffers, different seeds): as many as make the combined footprint exceed twice
+        # the L2, and never fewer than two -- three for an HBM-bound problem, whose time is all memory traffic -- so that
+        # a step finds neither its operands nor a dirty copy of its output in cache.  Capped at 12 GB of device memory.
+        hbm_bound = w.min_bytes / 6.5e12 > w.flops / 1.6e15
+        want = max(3 if hbm_bound else 2, -(-2 * L2_BYTES // int(footprint)))
+        self.nsets = int(max(1 if nsets_cap == 1 else 2, min(want, 160, nsets_cap, int(12e9 // footprint))))
         self.sets = []
         for r in range(self.nsets):
             inp = wl.make_inputs(w, seed_offset=1000 * r)
@@ -162,27 +187,46 @@ class DeviceCase:
                          flags | bg.make_flags(bias_per_row=w.bias_per_row, a_lower=w.a_tri == 1, a_upper=w.a_tri == 2,
                                                d_lower=w.d_tri == 1, d_upper=w.d_tri == 2),
                         structure=w.b_tri | (4 if w.d_mirror else 0))
+        self.desc = d
         self.plan = bg.Plan(d)
         self.plan.workspace(device)
         self.i = 0
-        self._args = None
+        self._calls = None
+        self.warm_launches = 0
+
+    def _bind(self, plan):
+        """One pre-marshalled gemm_run call per input set (C ABI, raw device addresses, current stream)."""
+        ws = plan.workspace(self.device)
+        wsp, wsb = (0, 0) if ws is None else (ws.data_ptr(), ws.numel())
+        stream = self.torch.cuda.current_stream(self.device).cuda_stream
+        return [self.bg.bind_run(plan.handle, A.data_ptr(), B.data_ptr(), C.data_ptr(), 0 if bias is None else bias.data_ptr(),
+                                 float(self.w.alpha), float(self.w.beta), wsp, wsb, stream) for A, B, C, bias in self.sets]
 
     def step(self):
-        """One pass of the hot path through the C ABI (gemm_run on raw device addresses, current stream)."""
-        if self._args is None:
-            ws = self.plan.workspace(self.device)
-            wsp, wsb = (0, 0) if ws is None else (ws.data_ptr(), ws.numel())
-            stream = self.torch.cuda.current_stream(self.device).cuda_stream
-            self._args = [(self.plan.handle, A.data_ptr(), B.data_ptr(), C.data_ptr(), 0 if bias is None else bias.data_ptr(),
-                           float(self.w.alpha), float(self.w.beta), wsp, wsb, stream) for A, B, C, bias in self.sets]
-        self.bg.gemm_run(*self._args[self.i % self.nsets])
+        """One pass of the hot path through the C ABI: gemm_run on the next input set."""
+        if self._calls is None:
+            self._calls = self._bind(self.plan)
+        self._calls[self.i % self.nsets]()
         self.i += 1
 
-    def time_steps(self, steps: int, warmup: int) -> float:
-        """Seconds per step over `steps` back-to-back steps (CUDA events on the launching stream)."""
+    def use_plan(self, flags: int):
+        """Replace the plan by one made with extra descriptor flags (same problem, same buffers)."""
+        d = self.bg.Desc.from_buffer_copy(self.desc)
+        d.flags |= flags
+        self.plan.close()
+        self.plan = self.bg.Plan(d)
+        self.plan.workspace(self.device)
+        self._calls = None
+
+    def time_steps(self, steps: int, warmup: int, step=None) -> float:
+        """Seconds per step over `steps` back-to-back steps (CUDA events on the launching stream).  `step` replaces the
+        library call by another function of no arguments (the vendor-library reference point runs in this same loop).
+        self.warm_launches counts the untimed launches that preceded the timed region."""
         torch = self.torch
+        step = step or self.step
+        self.warm_launches = warmup + 8
         for _ in range(warmup):
-            self.step()
+            step()
         torch.cuda.synchronize()
         # A configuration whose whole timed region lasts well under a millisecond would otherwise be measured while the
         # clocks are still ramping up from idle (the pause between configurations lets them drop): such a one keeps
@@ -190,23 +234,108 @@ class DeviceCase:
         # estimated from a second small batch.)
         t_warm = time.perf_counter()
         for _ in range(8):
-            self.step()
+            step()
         torch.cuda.synchronize()
         short_region = (time.perf_counter() - t_warm) / 8 * steps < 0.03
         while short_region and time.perf_counter() - t_warm < 0.03:
             for _ in range(16):
-                self.step()
+                step()
+            self.warm_launches += 16
             torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for _ in range(steps):
-            self.step()
+            step()
         e1.record()
         torch.cuda.synchronize()
         st = self.plan.status()
         if st != self.bg.OK:
             raise RuntimeError(f"device status {self.bg.status_string(st)} after timing {self.key}")
         return e0.elapsed_time(e1) * 1e-3 / steps
+
+    def library_step(self):
+        """The vendor library (torch -> cuBLAS) on this configuration's own buffers, as a function of no arguments for
+        time_steps, and a description of what it runs.  Reference point only: nothing in the product calls it."""
+        torch, w = self.torch, self.w
+        if w.ab_dtype not in (wl.BF16, wl.F16) or w.a_tri or w.b_tri or w.d_tri:
+            return None, "no plain library counterpart"
+        F = torch.nn.functional
+        views = []
+        for A, B, C, bias in self.sets:
+            a3 = torch.as_strided(A, (w.batch, w.K if w.transa else w.M, w.M if w.transa else w.K), (w.stride_a, w.lda, 1))
+            b3 = torch.as_strided(B, (w.batch, w.N if w.transb else w.K, w.K if w.transb else w.N), (w.stride_b, w.ldb, 1))
+            opa = a3.transpose(1, 2) if w.transa else a3
+            opb = b3.transpose(1, 2) if w.transb else b3
+            c3 = torch.as_strided(C, (w.batch, w.M, w.N), (w.stride_c, w.ldc, 1))
+            views.append((opa, opb, c3, bias))
+        same_out = w.c_dtype == w.ab_dtype
+        out_note = "" if same_out else " (output in the operand type: the library call has no fp32 output for 16-bit operands" + \
+            ("; beta * C is not applied)" if w.beta != 0.0 else ")")
+        fused_bias = w.batch == 1 and w.has_bias and not w.bias_per_row and (w.beta == 0.0 or not same_out)
+        bias16 = [None if b is None else b.to(_torch_dt(torch, w.ab_dtype)) for _, _, _, b in self.sets]
+        scratch = [torch.empty((w.batch, w.M, w.N), dtype=_torch_dt(torch, w.ab_dtype), device=self.device) for _ in self.sets] \
+            if not same_out else None
+        act = w.epilogue >> 1
+        i = [0]
+
+        def step():
+            opa, opb, c3, bias = views[i[0] % self.nsets]
+            out = c3 if same_out else scratch[i[0] % self.nsets]
+            k = i[0] % self.nsets
+            i[0] += 1
+            if fused_bias:   # one library call with the bias in its epilogue
+                torch.addmm(bias16[k], opa[0], opb[0], alpha=w.alpha, out=out[0])
+            elif w.alpha != 1.0 or (w.beta != 0.0 and same_out):
+                torch.baddbmm(c3 if same_out else out, opa, opb, beta=w.beta if same_out else 0.0, alpha=w.alpha, out=out)
+            else:
+                torch.bmm(opa, opb, out=out)
+            if w.has_bias and not fused_bias:
+                out.add_(bias16[k] if not w.bias_per_row else bias16[k][:, None])
+            if act == 1:
+                out.relu_()
+            elif act == 2:
+                out.copy_(F.gelu(out))
+            elif act == 3:
+                out.copy_(F.gelu(out, approximate="tanh"))
+            elif act == 4:
+                out.copy_(F.silu(out))
+        what = ("torch.addmm (bias in the library epilogue)" if fused_bias else "torch.bmm / baddbmm" + (", then bias add" if w.has_bias else "")) + \
+            " on the same buffers" + ({0: "", 1: ", then relu", 2: ", then gelu", 3: ", then gelu(tanh)", 4: ", then silu"}[act]) + \
+            (" as a separate kernel" if act else "") + out_note
+        return step, what
+
+    def time_sustained(self, seconds: float, step=None, sampler_index: int = 0):
+        """Back-to-back steps for at least `seconds` (after one second of the same load), timed with CUDA events on the
+        launching stream while the SM clock is sampled: what the configuration sustains under the power cap."""
+        torch = self.torch
+        step = step or self.step
+
+        def spin(duration, chunk=20):
+            n, t0 = 0, time.perf_counter()
+            while time.perf_counter() - t0 < duration:
+                for _ in range(chunk):
+                    step()
+                n += chunk
+                if n % (8 * chunk) == 0:
+                    torch.cuda.synchronize()   # keeps the launch queue short so that the loop ends on time
+            return n
+
+        spin(1.0)
+        torch.cuda.synchronize()
+        with ClockSampler(sampler_index) as clocks:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            n = spin(seconds)
+            e1.record()
+            torch.cuda.synchronize()
+        sec = e0.elapsed_time(e1) * 1e-3
+        c = clocks.summary()
+        per_step = sec / n
+        return {"value": round(metric_value(self.w, per_step), 2), "unit": "TFLOP/s", "seconds": round(sec, 2), "launches": n,
+                "ms_per_step": round(per_step * 1e3, 5), "sm_mhz_median": c["sm_mhz"], "reasons": c["reasons"],
+                # time x clock: SM cycles per step in millions; constant if the kernel is clock-bound, so run-to-run
+                # differences in the power-capped clock can be told from differences in the kernel
+                "mcycles_per_step": None if not c["sm_mhz"] else round(per_step * c["sm_mhz"], 3)}
 
     def time_e2e(self, steps: int, warmup: int):
         """Same metric with host-resident inputs and output, through gemm_host_run: every step copies A, B (and C_in,
@@ -325,6 +454,25 @@ def run_ours(args):
         sec = case.time_steps(steps, warmup)
         barrier()
     sec = max_over(sec)
+    warm_launches = case.warm_launches
+    # context: the vendor library on the same buffers in the same loop, and the headline held for seconds
+    library = sustained = None
+    if args.all and world == 1:
+        lib_step, lib_what = case.library_step()
+        if lib_step is not None:
+            time.sleep(1.0)
+            lib_sec = case.time_steps(steps, warmup, step=lib_step)
+            library = {"value": round(metric_value(w, lib_sec), 2), "unit": "TFLOP/s", "ms_per_step": round(lib_sec * 1e3, 5),
+                       "what": lib_what + "; same rotating buffers, same event-timed loop; context only, no part of the product"}
+        if args.sustained_seconds > 0:
+            time.sleep(1.0)
+            sustained = case.time_sustained(args.sustained_seconds, sampler_index=local_rank)
+            sustained["frac_of_sustained_peak"] = round(sustained["value"] / peaks["bf16_tflops_sustained"], 4)
+            if lib_step is not None:
+                time.sleep(1.0)
+                ls = case.time_sustained(args.sustained_seconds, step=lib_step, sampler_index=local_rank)
+                library["sustained"] = {k: ls[k] for k in ("value", "seconds", "launches", "sm_mhz_median", "mcycles_per_step")}
+            time.sleep(1.0)
     e2e_steps = max(2, min(steps, args.e2e_steps))
     barrier()
     if args.e2e_steps > 0:
@@ -337,11 +485,13 @@ def run_ours(args):
     out = {
         "metric": "GEMM TFLOP/s at 1 B200 and % of dense bf16 roofline (HBM GB/s for skinny)",
         "value": round(whole_job_value(w, sec, world), 2), "unit": "TFLOP/s", "n_gpus": world, "steps": steps, "warmup": warmup,
+        "warmup_launches_actual": warm_launches,
         "ms_per_step": round(sec * 1e3, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16 x bf16 -> fp32 accumulate", "data": "synthetic",
         "config": {"workload": w.name, "M": w.M, "N": w.N, "K": w.K, "batch": w.batch,
                    "layout": "A row-major, B stored N x K", "out_dtype": ["bf16", "f16", "f32"][w.c_dtype],
-                   "l2": f"inputs larger than L2: {case.nsets} rotating seeded input set(s), {w.min_bytes / 1e6:.0f} MB each",
+                   "l2": f"inputs larger than L2: {case.nsets} rotating seeded sets of inputs and output, {w.min_bytes / 1e6:.0f} MB each",
+                   "input_sets": case.nsets,
                    "multi_gpu": "replicas only (independent GEMMs, no collective)", "plan": case.plan.info},
         "e2e": None if args.e2e_steps <= 0 else {"value": round(metric_value(w, e2e_sec) * world, 3), "unit": "TFLOP/s", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": round(e2e_sec * 1e3, 3), "steps": e2e_steps,
@@ -351,6 +501,10 @@ def run_ours(args):
         "roofline": roofline_for(w, key, sec, peaks, peak_kind),
     }
     out["roofline"]["frac_of_sustained_peak"] = round(metric_value(w, sec) / peaks["bf16_tflops_sustained"], 4)
+    if library is not None:
+        out["library_reference"] = library
+    if sustained is not None:
+        out["sustained"] = sustained
     host_inputs = case.host_inputs
     case.close()
 
@@ -359,15 +513,30 @@ def run_ours(args):
         for k2, w2 in cfgs.items():
             if k2 == key:
                 measured.append({"config": k2, "workload": w2.name, "ms_per_step": out["ms_per_step"], "tflops": out["value"] / world,
-                                 "roofline": out["roofline"]})
+                                 "input_sets": out["config"]["input_sets"], "warmup_launches_actual": warm_launches,
+                                 "roofline": out["roofline"],
+                                 "library_reference_ms_per_step": None if library is None else library["ms_per_step"]})
                 continue
             c2 = DeviceCase(torch, bg, k2, w2, 0, device)
             torch.cuda.synchronize()
             time.sleep(1.5)  # let clocks and the power governor recover from the previous configuration's load
             s2 = max_over(c2.time_steps(steps, warmup))
-            measured.append({"config": k2, "workload": w2.name, "ms_per_step": round(s2 * 1e3, 5),
-                             "tflops": round(metric_value(w2, s2), 2), "gbs": round(w2.min_bytes / s2 / 1e9, 1),
-                             "input_sets": c2.nsets, "plan": c2.plan.info, "roofline": roofline_for(w2, k2, s2, peaks, peak_kind)})
+            row = {"config": k2, "workload": w2.name, "ms_per_step": round(s2 * 1e3, 5),
+                   "tflops": round(metric_value(w2, s2), 2), "gbs": round(w2.min_bytes / s2 / 1e9, 1),
+                   "input_sets": c2.nsets, "warmup_launches_actual": c2.warm_launches, "plan": c2.plan.info,
+                   "roofline": roofline_for(w2, k2, s2, peaks, peak_kind)}
+            if world == 1:
+                lib_step, lib_what = c2.library_step()
+                if lib_step is not None:     # the vendor library on the same buffers, same loop (context)
+                    time.sleep(0.5)
+                    row["library_reference_ms_per_step"] = round(c2.time_steps(steps, warmup, step=lib_step) * 1e3, 5)
+                    row["library_reference_what"] = lib_what
+                # the same plan launched without programmatic dependent launch: what the overlap of one kernel's set-up
+                # with its predecessor's tail is worth in this back-to-back loop
+                time.sleep(0.5)
+                c2.use_plan(bg.make_flags(no_early_launch=True))
+                row["ms_per_step_no_early_launch"] = round(c2.time_steps(steps, warmup) * 1e3, 5)
+            measured.append(row)
             c2.close()
         out["configs_measured"] = measured
 
@@ -468,24 +637,12 @@ def run_shapes(args):
                    "gbs": round(w.min_bytes / sec / 1e9, 1), "input_sets": case.nsets,
                    "plan": {k: case.plan.info[k] for k in ("variant", "tile_m", "tile_n", "stages", "cluster_size", "grid", "split")},
                    "roofline": roofline_for(w, spec, sec, peaks, peak_kind)}
-            if args.library_reference and w.batch == 1 and w.epilogue == wl.EPI_NONE and w.beta == 0.0 and w.alpha == 1.0 and \
-                    w.ab_dtype in (wl.BF16, wl.F16):
-                # context only: the vendor library on the same operands (no part of the product)
-                A, B, _, _ = case.sets[0]
-                a2 = A[: (w.K if w.transa else w.M) * w.lda].view(-1, w.lda)
-                b2 = B[: (w.N if w.transb else w.K) * w.ldb].view(-1, w.ldb)
-                opa = a2[:, : w.M].t() if w.transa else a2[:, : w.K]
-                opb = b2[:, : w.K].t() if w.transb else b2[:, : w.N]
-                for _ in range(warmup):
-                    torch.matmul(opa, opb)
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                torch.cuda.synchronize()
-                e0.record()
-                for _ in range(steps):
-                    torch.matmul(opa, opb)
-                e1.record()
-                torch.cuda.synchronize()
-                row["library_reference_ms"] = round(e0.elapsed_time(e1) / steps, 5)
+            if args.library_reference:
+                # context only: the vendor library on the same rotating buffers in the same loop (no part of the product)
+                lib_step, lib_what = case.library_step()
+                if lib_step is not None:
+                    row["library_reference_ms"] = round(case.time_steps(steps, warmup, step=lib_step) * 1e3, 5)
+                    row["library_reference_what"] = lib_what
             if args.tune:
                 # measured plan selection on the first input set (its C is scratch from here on), then the same timing
                 # loop again: the new plan picks the remembered choice up by itself
@@ -570,6 +727,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--sustained-seconds", type=float, default=4.0, help="length of the sustained leg of the headline config (0 = skip)")
     ap.add_argument("--ref-step-seconds", type=float, default=10.0, help="--impl reference: CPU time budget of one step")
     ap.add_argument("--shapes", default="", help="';'-separated MxNxK[:key=value...] problems to time instead of the five configurations")
     ap.add_argument("--tune-file", default="", help="--shapes --tune: write the measured choices to this file (gemm_tune_cache_save)")

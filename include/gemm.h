@@ -28,8 +28,9 @@
  * the caller owns every buffer (A, B, C, bias, workspace) and keeps it alive
  * until the stream work has completed.  The library owns the plan object and a
  * small device status word per plan.  No call synchronises the device except
- * gemm_plan_status().  Nothing throws; every failure is a gemm_status_t, and an
- * argument error launches nothing.
+ * gemm_plan_status() (gemm_plan_status_stream() waits for one stream only,
+ * gemm_plan_status_async() for nothing).  Nothing throws; every failure is a
+ * gemm_status_t, and an argument error launches nothing.
  */
 #ifndef B200_GEMM_H_
 #define B200_GEMM_H_
@@ -97,7 +98,7 @@ typedef enum {
 #define GEMM_FLAG_TILE_N_MASK 0x1F00u
 #define GEMM_FLAG_TAIL_SPLIT 0x2000u       /* when the last wave of a 1-CTA or pair plan would fill at most half of the SMs, cut
                                               its tiles into K slices, one per CTA or pair (the plan then wants a workspace for
-                                              the raw accumulators of the further slices).  Without the flag this happens only
+                                              the flag words and raw accumulators of the further slices).  Without the flag this happens only
                                               for a handful of tiles with a very long K (three or more slices each); otherwise
                                               it is left to the caller and to gemm_tune: under the power cap idle SMs lend
                                               their budget to the busy ones, so it pays only on small problems (measured:
@@ -185,8 +186,7 @@ typedef struct {
  * roofline (Section 4.3), choose the kernel variant, tile shape, pipeline depth,
  * cluster size, raster order and stream-K split, and return a plan (host
  * memory).  If a CUDA device is current, also allocates the plan's 16-byte
- * device status word (and, for the stream-K variant, its arrival counters, one
- * word per output tile) and reads the SM count; without a device the plan is still
+ * device status word and reads the SM count; without a device the plan is still
  * created (148 SMs assumed) so that planning can be inspected, and gemm_run
  * reports GEMM_ERR_ARCH.  Errors: NULL -> GEMM_ERR_NULL; extents < 1, leading
  * dimension smaller than the row length, unknown enum, wrong struct_size ->
@@ -196,8 +196,9 @@ typedef struct {
  */
 gemm_status_t gemm_plan(const gemm_desc_t* desc, gemm_plan_t* out_plan);
 
-/* Bytes of device workspace gemm_run needs for this plan (0 for the dense variants;
- * stream-K partial tiles for the skinny variant).  0 on a NULL plan. */
+/* Bytes of device workspace gemm_run needs for this plan: 0 for the plain dense variants; for stream-K the arrival
+ * words of the output tiles followed by the partial tiles, for a dense plan with a tail split the flag words followed
+ * by the partial accumulators.  The workspace needs no initialisation and may hold anything.  0 on a NULL plan. */
 size_t gemm_workspace_bytes(gemm_plan_t plan);
 
 /*
@@ -208,12 +209,16 @@ size_t gemm_workspace_bytes(gemm_plan_t plan);
  * has a bias.  C is read only when beta != 0, and only the M x N elements of D (per batch) are written: row padding
  * (ldc > N) and gaps between batches keep their contents, so D may be a column block of a wider matrix.  workspace: device
  * memory of at least gemm_workspace_bytes(plan) bytes, 16-byte aligned (may be NULL when
- * that is 0).  Runs of one plan that needs no workspace may overlap on the GPU; runs of a plan that
- * needs one (stream-K, or a dense plan with a tail split: gemm_workspace_bytes > 0) must not -- they
- * share the plan's arrival counters or flags, which every run leaves at zero: order them on one
- * stream or with events, or make one plan per stream.  alpha and beta are host scalars.  The call only encodes tensor maps on the
- * host and launches: once a plan has run once (which sets kernel attributes), further runs may be recorded by stream
- * capture into a CUDA graph (tested).  Errors are returned before anything is launched:
+ * that is 0), with any contents: the hand-shake words at its head carry a tag that is new with every run, so whatever
+ * the memory held before reads as "nothing yet".  Runs of one plan may overlap on the GPU (several streams, several host
+ * threads) as long as runs that overlap use DIFFERENT workspaces; they share only the status word, which then reports
+ * a timeout of any of them.  Runs that share a workspace must be ordered (one stream, or events).  alpha and beta are
+ * host scalars.  The call only fetches or encodes tensor maps on the host (a plan remembers the maps of the operand
+ * addresses it has seen, so a repeated address costs no encoding) and launches: once a plan has run once (which sets
+ * kernel attributes), further runs may be recorded by stream capture into a CUDA graph (tested).  A captured run replays
+ * with the tag it was captured with, which is safe because every run leaves its hand-shake words at zero; only after a
+ * GEMM_ERR_TIMEOUT must a captured graph of a plan with a workspace be captured again (or the first
+ * gemm_workspace_bytes bytes of that workspace be zeroed) before it is replayed.  Errors are returned before anything is launched:
  * GEMM_ERR_NULL, GEMM_ERR_ALIGNMENT, GEMM_ERR_WORKSPACE, GEMM_ERR_ARCH,
  * GEMM_ERR_INVALID_ARG (the current CUDA device is not the one the plan was
  * made on), GEMM_ERR_CUDA (tensor-map encoding or launch failure).
@@ -222,13 +227,26 @@ gemm_status_t gemm_run(gemm_plan_t plan, const void* A, const void* B, void* C, 
                        float beta, void* workspace, size_t workspace_bytes, gemm_stream_t stream);
 
 /*
- * gemm_plan_status -- synchronise the device and read the plan's status word:
- * GEMM_OK, or GEMM_ERR_TIMEOUT if a bounded device-side wait of an earlier run
- * expired (the kernel then returned early and its output is undefined; until
- * the word has been read, later runs of the plan may give up early as well,
- * and a stream-K plan does not finish split tiles).  The read clears the word
- * and puts the plan back in order.
+ * The plan's status word: GEMM_OK, or GEMM_ERR_TIMEOUT if a bounded device-side wait of an earlier run expired (the
+ * kernel then returned early and its output is undefined; until the word has been taken, later runs of the plan may
+ * give up early as well, and a stream-K plan does not finish split tiles).  Taking the word clears it and puts the
+ * plan back in order.  (The bounded waits are this library's; the paper's kernels have no counterpart.)  Three forms:
+ *
+ * gemm_plan_status_async -- enqueue on `stream` a one-thread kernel that takes the word into page-locked host
+ *   memory owned by the plan; returns at once and synchronises nothing (the first call on a plan allocates that
+ *   host word: make it outside stream capture).  gemm_plan_status_result then reports the word that was taken
+ *   last; the caller must first have waited, by any means (event, stream synchronise, graph completion), for the
+ *   stream to get past the enqueued kernel.  Without an earlier _async call it returns GEMM_OK.
+ * gemm_plan_status_stream -- the two together around cudaStreamSynchronize(stream): waits for that one stream only.
+ *   This is the form to use after runs on `stream`.
+ * gemm_plan_status -- the same after cudaDeviceSynchronize(): for callers that do not know which streams ran the
+ *   plan.  It stalls every stream of the device and must not be used while a stream capture is under way.
+ * Errors: GEMM_ERR_NULL; GEMM_ERR_ARCH (plan made without a device); GEMM_ERR_INVALID_ARG (the current device is not
+ * the plan's); GEMM_ERR_CUDA.
  */
+gemm_status_t gemm_plan_status_async(gemm_plan_t plan, gemm_stream_t stream);
+gemm_status_t gemm_plan_status_result(gemm_plan_t plan);
+gemm_status_t gemm_plan_status_stream(gemm_plan_t plan, gemm_stream_t stream);
 gemm_status_t gemm_plan_status(gemm_plan_t plan);
 
 /* Override the device-side wait limit of this plan (default 2000 ms; minimum 1 ms). */
@@ -236,6 +254,30 @@ gemm_status_t gemm_plan_set_timeout_ms(gemm_plan_t plan, uint32_t ms);
 
 /* Copy the plan's decisions into *out (out->struct_size must be sizeof(gemm_info_t)). */
 gemm_status_t gemm_plan_info(gemm_plan_t plan, gemm_info_t* out);
+
+/*
+ * gemm_plan_schedule -- list the work items of a plan in the order its CTAs execute them: which CTA (for the pair
+ * variants: which CTA pair) computes which output tile over which part of K.  This is the persistent tile scheduler
+ * with its swizzled (grouped) raster order -- the "thread-block swizzle" strategy of the paper's Table 1 -- the
+ * schedule dealt ahead of time for structured problems, the tail split and the stream-K decomposition, walked on the
+ * host by the same functions the kernels run; it needs no device.  Meant for inspection and for tests (every wanted
+ * tile exactly once, every K stage of a split tile exactly once).
+ *   items: host array of `capacity` entries (may be NULL when capacity is 0); *count receives the number of items
+ *   the plan has, which may exceed capacity (only the first `capacity` are written).
+ * Errors: GEMM_ERR_NULL.
+ */
+typedef struct {
+  int32_t cta;       /* CTA (pair variants: cluster) that executes the item; items of one CTA appear in execution order */
+  int32_t batch;     /* matrix of the batch */
+  int32_t tile_row;  /* output tile, in units of gemm_info_t.tile_m rows ... */
+  int32_t tile_col;  /* ... and tile_n columns (stream-K: the 128-wide tile along the long extent, the other index 0) */
+  int32_t k_begin;   /* ring stages [k_begin, k_end) of gemm_info_t.tile_k elements of K each */
+  int32_t k_end;
+  int32_t slice;     /* -1: the item computes its tile alone; >= 0: one of several K slices of the tile (0 finishes it
+                        in a tail split; stream-K: position among the tile's contributors, the last arrival finishes) */
+  int32_t reserved;
+} gemm_work_item_t;
+gemm_status_t gemm_plan_schedule(gemm_plan_t plan, gemm_work_item_t* items, size_t capacity, size_t* count);
 
 /* Free the plan and its status word.  NULL is accepted. */
 gemm_status_t gemm_destroy(gemm_plan_t plan);
@@ -249,13 +291,18 @@ gemm_status_t gemm_destroy(gemm_plan_t plan);
  * rule.  The call makes no cudaMalloc / cudaFree and uses no allocating library routine; the plan is built
  * on the stack and the kernel's scratch (status word, arrival counters, partial tiles) is a fixed 4 MiB
  * array inside the library, present on every GPU that loads the library until the process exits.
- *   desc, A, B, C, bias, alpha, beta, stream: as for gemm_plan / gemm_run (desc->flags is ignored).
+ *   desc, A, B, C, bias, alpha, beta, stream: as for gemm_plan / gemm_run.  The tuning fields of desc->flags are
+ *   ignored; a flag or structure bit that changes what is computed (GEMM_FLAG_A_*, GEMM_FLAG_D_*,
+ *   GEMM_FLAG_BIAS_PER_ROW, any GEMM_STRUCT_*) is refused with GEMM_ERR_UNSUPPORTED, as the stream-K plans refuse it.
  *   sync_and_check: 0 = asynchronous, only launch-time errors are reported; non-zero = wait for `stream`
  *   and return GEMM_ERR_TIMEOUT if a bounded device-side wait expired.
  * Limits and rules: problems whose scratch need exceeds the array (with 148 SMs: M > 16) are rejected
  * with GEMM_ERR_WORKSPACE and nothing is launched (gemm_last_cuda_error() gives the sizes).  The first
- * call on each device resolves the array's device address and sets a kernel attribute; make that first
- * call before any stream capture begins.  All calls on a device share the one array: it keeps the
+ * call on each device resolves the array's device address and sets a kernel attribute; under CUDA's lazy
+ * module loading it is also the moment the driver loads the library's module (the kernel image and the
+ * 4 MiB array), which takes device memory once and can fail on a GPU that has none left.  So make that
+ * first call during initialisation -- before the GPU's memory is handed to the caller's own pool and before
+ * any stream capture begins; every later call on the device allocates nothing.  All calls on a device share the one array: it keeps the
  * previous call's contents (the call clears what must start at zero), and two calls whose kernels overlap
  * on the GPU (different streams, or several host threads) race on it -- serialise them.
  */

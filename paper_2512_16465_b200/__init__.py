@@ -59,6 +59,10 @@ class Info(ctypes.Structure):
         return {k: getattr(self, k) for k, _ in self._fields_ if k != "struct_size"}
 
 
+class WorkItem(ctypes.Structure):
+    _fields_ = [(k, ctypes.c_int32) for k in ("cta", "batch", "tile_row", "tile_col", "k_begin", "k_end", "slice", "reserved")]
+
+
 TUNE_MAX_CANDIDATES = 32
 
 
@@ -74,7 +78,8 @@ class TuneReport(ctypes.Structure):
                 "tried": [(self.tried_flags[i], self.tried_ms[i]) for i in range(n)]}
 
 
-EXPORTS = ("gemm_plan", "gemm_workspace_bytes", "gemm_run", "gemm_plan_status", "gemm_plan_set_timeout_ms",
+EXPORTS = ("gemm_plan", "gemm_workspace_bytes", "gemm_run", "gemm_plan_status", "gemm_plan_status_async",
+           "gemm_plan_status_result", "gemm_plan_status_stream", "gemm_plan_schedule", "gemm_plan_set_timeout_ms",
            "gemm_plan_info", "gemm_destroy", "gemm_status_string", "gemm_last_cuda_error", "gemm_skinny_run_noalloc",
            "gemm_tune", "gemm_tune_workspace_bytes", "gemm_tune_cache_clear", "gemm_tune_cache_save", "gemm_tune_cache_load",
            "gemm_host_create", "gemm_host_run", "gemm_host_panels", "gemm_host_destroy")
@@ -94,6 +99,13 @@ def _load() -> ctypes.CDLL:
     L.gemm_run.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, ctypes.c_float, vp, ctypes.c_size_t, vp]
     L.gemm_plan_status.restype = ctypes.c_int
     L.gemm_plan_status.argtypes = [vp]
+    L.gemm_plan_status_result.restype = ctypes.c_int
+    L.gemm_plan_status_result.argtypes = [vp]
+    for fn in (L.gemm_plan_status_async, L.gemm_plan_status_stream):
+        fn.restype = ctypes.c_int
+        fn.argtypes = [vp, vp]
+    L.gemm_plan_schedule.restype = ctypes.c_int
+    L.gemm_plan_schedule.argtypes = [vp, ctypes.POINTER(WorkItem), ctypes.c_size_t, ctypes.POINTER(ctypes.c_size_t)]
     L.gemm_plan_set_timeout_ms.restype = ctypes.c_int
     L.gemm_plan_set_timeout_ms.argtypes = [vp, ctypes.c_uint32]
     L.gemm_plan_info.restype = ctypes.c_int
@@ -259,7 +271,57 @@ def gemm_host_destroy(handle: int) -> None:
 
 
 def gemm_plan_status(plan: int) -> int:
+    """``gemm_plan_status``: waits for the whole device, then takes the plan's status word."""
     return int(_lib.gemm_plan_status(plan))
+
+
+def gemm_plan_status_stream(plan: int, stream: int) -> int:
+    """``gemm_plan_status_stream``: waits for ``stream`` (a raw ``cudaStream_t`` value) only."""
+    return int(_lib.gemm_plan_status_stream(plan, stream or None))
+
+
+def gemm_plan_status_async(plan: int, stream: int) -> None:
+    """``gemm_plan_status_async``: enqueue the read of the status word on ``stream``; nothing is waited for."""
+    st = _lib.gemm_plan_status_async(plan, stream or None)
+    if st != OK:
+        raise GemmError(st, "gemm_plan_status_async")
+
+
+def gemm_plan_status_result(plan: int) -> int:
+    """``gemm_plan_status_result``: the word the last ``gemm_plan_status_async`` took (the caller waited for the stream)."""
+    return int(_lib.gemm_plan_status_result(plan))
+
+
+def bind_run(plan: int, A: int, B: int, C: int, bias: int, alpha: float, beta: float, workspace: int, workspace_bytes: int,
+             stream: int):
+    """The arguments of one ``gemm_run`` call converted to their C types once: returns a function of no arguments
+    that makes the call (and raises :class:`GemmError` on failure).  For loops that launch the same GEMM on the same
+    buffers again and again, where converting ten Python values per call costs more than the launch."""
+    vp = ctypes.c_void_p
+    args = (vp(plan), vp(A), vp(B), vp(C), vp(bias or None), ctypes.c_float(alpha), ctypes.c_float(beta), vp(workspace or None),
+            ctypes.c_size_t(workspace_bytes), vp(stream or None))
+    fn = _lib.gemm_run
+
+    def call():
+        st = fn(*args)
+        if st != OK:
+            raise GemmError(st, "gemm_run")
+    return call
+
+
+def gemm_plan_schedule(plan: int):
+    """``gemm_plan_schedule``: the plan's work items as a numpy array of shape (items, 7) with the columns
+    cta, batch, tile_row, tile_col, k_begin, k_end, slice, in the order the CTAs execute them (needs no device)."""
+    import numpy as np
+    n = ctypes.c_size_t(0)
+    st = _lib.gemm_plan_schedule(plan, None, 0, ctypes.byref(n))
+    if st != OK:
+        raise GemmError(st, "gemm_plan_schedule")
+    buf = (WorkItem * max(1, n.value))()
+    st = _lib.gemm_plan_schedule(plan, buf, n.value, ctypes.byref(n))
+    if st != OK:
+        raise GemmError(st, "gemm_plan_schedule")
+    return np.frombuffer(buf, dtype=np.int32).reshape(-1, 8)[: n.value, :7].copy()
 
 
 def gemm_plan_info(plan: int) -> dict:
@@ -335,8 +397,11 @@ class Plan:
                  float(alpha), float(beta), 0 if ws is None else ws.data_ptr(), 0 if ws is None else ws.numel(), s)
         return C
 
-    def status(self) -> int:
-        return gemm_plan_status(self.handle)
+    def status(self, stream: Optional[int] = None) -> int:
+        """The plan's status after its runs on ``stream`` (default: the current torch stream); waits for that stream only."""
+        import torch
+        s = torch.cuda.current_stream().cuda_stream if stream is None else stream
+        return gemm_plan_status_stream(self.handle, s)
 
     def set_timeout_ms(self, ms: int) -> None:
         _lib.gemm_plan_set_timeout_ms(self.handle, ms)

@@ -95,7 +95,11 @@ struct DenseParams {
   // the last wave, are cut into `split` slices of K each, one work item per slice; num_items counts whole tiles + slices.
   int split, split_first_tile, num_items;
   float* partials;                        // workspace: raw fp32 accumulators of slices 1..split-1, [tile][rank][slice-1][128][bn]
-  uint32_t* split_flags;                  // one word per such partial: 1 = written (reset to 0 by the reducing CTA)
+  // One word per such partial at the head of the workspace: it holds this run's tag once the partial is written (any
+  // other value -- zeros, another run's tag, whatever the memory held before -- means "not yet"), and the reducing CTA
+  // puts it back to zero so that a replay of the same launch starts clean.  No initialisation is needed.
+  unsigned long long* split_flags;
+  unsigned long long split_tag;           // this run's tag (48 bits, never 0)
   float alpha, beta;
   const float* bias;
   const void* c_in;                       // = D buffer; read when beta != 0
@@ -177,7 +181,9 @@ struct TileCoord {
 // Linear tile id -> (batch, tile row, tile column).  Inside one matrix, tiles are visited in groups
 // of `raster_group` tile rows; inside a group the row index runs fastest, so the CTAs that are
 // resident together work on a compact block of the output and share A and B panels in L2.
-__device__ __forceinline__ TileCoord decode_tile(const DenseParams& p, int t) {
+// (The scheduling functions from here to work_item also compile for the host: gemm_plan_schedule walks a plan's
+// schedule with the very code the kernels run.)
+__host__ __device__ __forceinline__ TileCoord decode_tile(const DenseParams& p, int t) {
   TileCoord c;
   const int per_matrix = p.tiles_m * p.tiles_n;
   c.batch = static_cast<int>(fast_div(static_cast<uint32_t>(t), p.fd_matrix));
@@ -194,7 +200,7 @@ __device__ __forceinline__ TileCoord decode_tile(const DenseParams& p, int t) {
 
 // The same with plain divisions, for the wide pair kernel: its tiles last tens of thousands of cycles, and its register
 // allocation is at the limit where any change of this code has cost spills.
-__device__ __forceinline__ TileCoord decode_tile_div(int t, int tiles_m, int tiles_n, int raster_group) {
+__host__ __device__ __forceinline__ TileCoord decode_tile_div(int t, int tiles_m, int tiles_n, int raster_group) {
   TileCoord c;
   const int per_matrix = tiles_m * tiles_n;
   c.batch = t / per_matrix;
@@ -216,7 +222,7 @@ __device__ __forceinline__ TileCoord decode_tile_div(int t, int tiles_m, int til
 struct KRange {
   int lo, hi;
 };
-__device__ __forceinline__ KRange k_range(const DenseParams& p, int row0, int rows, int col0, int cols) {
+__host__ __device__ __forceinline__ KRange k_range(const DenseParams& p, int row0, int rows, int col0, int cols) {
   KRange r{0, p.num_kb};
   const int ks = p.kstep_shift;
   if (p.a_tri == 1) r.hi = min(r.hi, ((min(row0 + rows, p.M) - 1) >> ks) + 1);       // k <= last row
@@ -236,17 +242,21 @@ struct WorkItem {
   KRange kr;
 };
 template <bool kSplit>
-__device__ __forceinline__ int item_tile(const DenseParams& p, int item) {
+__host__ __device__ __forceinline__ int item_tile(const DenseParams& p, int item) {
   if (p.tile_list != nullptr) {  // (never together with a tail split); < 0: an empty slot
     const int b = static_cast<int>(fast_div(static_cast<uint32_t>(item), p.fd_list));
+#ifdef __CUDA_ARCH__
     const int t = __ldg(p.tile_list + (item - b * p.list_len));
+#else
+    const int t = p.tile_list[item - b * p.list_len];  // (the host walks the plan's host copy of the list)
+#endif
     return t < 0 ? -1 : b * (p.tiles_m * p.tiles_n) + t;
   }
   if (!kSplit || item < p.split_first_tile) return item;
   return p.split_first_tile + (item - p.split_first_tile) / p.split;
 }
 template <bool kSplit>
-__device__ __forceinline__ WorkItem work_item(const DenseParams& p, int item, int tile, int row0, int rows, int col0) {
+__host__ __device__ __forceinline__ WorkItem work_item(const DenseParams& p, int item, int tile, int row0, int rows, int col0) {
   WorkItem wi{tile, -1, k_range(p, row0, rows, col0, p.bn)};
   if (kSplit && item >= p.split_first_tile) {
     wi.slice = (item - p.split_first_tile) - (tile - p.split_first_tile) * p.split;
@@ -257,13 +267,16 @@ __device__ __forceinline__ WorkItem work_item(const DenseParams& p, int item, in
 }
 // Bounded wait for a flag word another CTA of this launch sets (all CTAs of these persistent kernels are resident,
 // and the CTA that sets the flag never waits for anybody).  Warp-uniform; false = gave up (timeout or abort elsewhere).
-__device__ __noinline__ bool flag_wait_warp(const uint32_t* flag, const WaitCtx& w, uint32_t code) {
+__device__ __noinline__ bool flag_wait_warp(const unsigned long long* flag, unsigned long long tag, const WaitCtx& w, uint32_t code) {
   const uint64_t t0 = globaltimer_ns();
   uint32_t it = 0;
   while (true) {
-    uint32_t v = 0;
-    if (lane_id() == 0) v = ld_acquire_gpu(flag);
-    if (__shfl_sync(0xffffffffu, v, 0) != 0u) return true;
+    uint32_t hit = 0;
+    if (lane_id() == 0) hit = ld_acquire_gpu_u64(flag) == tag ? 1u : 0u;
+    if (__shfl_sync(0xffffffffu, hit, 0) != 0u) {
+      __syncwarp();  // orders the other lanes' later loads after lane 0's acquire (a shuffle alone orders no memory)
+      return true;
+    }
     __nanosleep(64);
     if ((++it & 31u) == 0u) {
       bool give_up = false;
@@ -686,7 +699,7 @@ __device__ __forceinline__ void epilogue_role(const DenseParams& p, const CUtens
     // split tile: slice `slice` of `p.split`; the partials of slices 1.. live at part0, flags at flag0
     int slice = -1;
     float* part0 = nullptr;
-    uint32_t* flag0 = nullptr;
+    unsigned long long* flag0 = nullptr;
     if (kSplit && item >= p.split_first_tile) {
       slice = (item - p.split_first_tile) - (tile - p.split_first_tile) * p.split;
       const size_t first = (static_cast<size_t>(tile - p.split_first_tile) * CG + cta_rank) * (p.split - 1);
@@ -713,14 +726,14 @@ __device__ __forceinline__ void epilogue_role(const DenseParams& p, const CUtens
         if constexpr (CG == 1) mbar_arrive(tempty0 + 8u * buf);
         else mbar_arrive_cluster(mapa(tempty0 + 8u * buf, 0));
       }
-      // the barrier orders every epilogue warp's stores before the one releasing increment of the flag
+      // the barrier orders every epilogue warp's stores before the one releasing store of the flag
       named_barrier_sync(2, 128 * EPI_WG);
-      if (ew == 0 && lane == 0) (void)atom_add_acq_rel_gpu(flag0 + (slice - 1), 1u);
+      if (ew == 0 && lane == 0) st_release_gpu_u64(flag0 + (slice - 1), p.split_tag);
       continue;
     }
     if (kSplit && slice == 0) {  // reducer: the other slices of this tile run in the same wave; wait for their partials
       for (int sidx = 0; sidx < p.split - 1; ++sidx)
-        if (!flag_wait_warp(flag0 + sidx, w, (3u << 8) | 0x40u | static_cast<uint32_t>(sidx))) return;
+        if (!flag_wait_warp(flag0 + sidx, p.split_tag, w, (3u << 8) | 0x40u | static_cast<uint32_t>(sidx))) return;
     }
     const int row0 = tc.tm * (kCtaM * CG) + static_cast<int>(cta_rank) * kCtaM + static_cast<int>(q) * 32;
     const long long row = row0 + static_cast<int>(lane);
@@ -813,7 +826,7 @@ __device__ __forceinline__ void epilogue_role(const DenseParams& p, const CUtens
     if (kSplit && slice == 0) {  // every epilogue warp has read the partials: lower the flags for the next launch
       named_barrier_sync(2, 128 * EPI_WG);
       if (ew == 0 && lane == 0)
-        for (int sidx = 0; sidx < p.split - 1; ++sidx) flag0[sidx] = 0u;
+        for (int sidx = 0; sidx < p.split - 1; ++sidx) flag0[sidx] = 0ull;
     }
   }
   if (lane == 0) bulk_wait_group_read<0>();  // staging may be released; the writes themselves complete with the grid

@@ -8,6 +8,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
@@ -100,6 +101,69 @@ int ceil_div(long long a, long long b) { return static_cast<int>((a + b - 1) / b
 
 }  // namespace
 
+namespace {
+
+// Tensor maps a plan has already encoded, by operand address.  Everything else a map depends on (extents, pitches,
+// box, element type) is fixed by the plan, so the base address alone identifies it.  One table per operand (A, B, D): a
+// caller that keeps its weights and changes its activations still finds two of the three.  128 entries each, four
+// probes from a hash of the address, the oldest of the four replaced on a miss.  Several host threads may run one
+// plan, hence the lock (held for a 128-byte copy).
+struct MapCache {
+  static constexpr int kEntries = 128, kProbes = 4;
+  struct alignas(64) Entry {
+    CUtensorMap map;
+    const void* key;
+    uint64_t stamp;  // 0 = empty
+  };
+  Entry table[3][kEntries];
+  uint64_t clock = 0;
+  std::atomic_flag lock = ATOMIC_FLAG_INIT;
+  MapCache() { memset(table, 0, sizeof table); }
+  static int slot_of(const void* key) {
+    uint64_t h = reinterpret_cast<uintptr_t>(key) >> 4;  // (operands are 16-byte aligned)
+    h *= 0x9E3779B97F4A7C15ull;
+    return static_cast<int>(h >> 57);  // 7 bits
+  }
+  // True and *out filled when `key` is known for operand `which`.
+  bool find(int which, const void* key, CUtensorMap* out) {
+    const int s0 = slot_of(key);
+    bool hit = false;
+    while (lock.test_and_set(std::memory_order_acquire)) {
+    }
+    for (int i = 0; i < kProbes; ++i) {
+      Entry& e = table[which][(s0 + i) & (kEntries - 1)];
+      if (e.stamp != 0 && e.key == key) {
+        *out = e.map;
+        e.stamp = ++clock;
+        hit = true;
+        break;
+      }
+    }
+    lock.clear(std::memory_order_release);
+    return hit;
+  }
+  void insert(int which, const void* key, const CUtensorMap& m) {
+    const int s0 = slot_of(key);
+    while (lock.test_and_set(std::memory_order_acquire)) {
+    }
+    Entry* victim = &table[which][s0];
+    for (int i = 0; i < kProbes; ++i) {
+      Entry& e = table[which][(s0 + i) & (kEntries - 1)];
+      if (e.stamp != 0 && e.key == key) {  // (another thread got there first)
+        victim = &e;
+        break;
+      }
+      if (e.stamp < victim->stamp) victim = &e;
+    }
+    victim->map = m;
+    victim->key = key;
+    victim->stamp = ++clock;
+    lock.clear(std::memory_order_release);
+  }
+};
+
+}  // namespace
+
 struct gemm_plan_s {
   gemm_desc_t d;
   gemm_info_t info;
@@ -115,14 +179,19 @@ struct gemm_plan_s {
   int device;            // CUDA device the plan was made on (-1: none); runs must use the same one
   bool has_device;
   bool arch_ok;
-  uint32_t* d_status;       // device: 16-byte status word, followed (256 bytes on) by the stream-K arrival counters
-  size_t d_counters_bytes = 0;  // plan-owned words after the status word: stream-K arrival counters or tail-split flags
+  uint32_t* d_status;       // device: 16-byte status word
+  uint32_t* h_status = nullptr;  // page-locked host copy written by gemm_plan_status_async (made on first use)
+  uint64_t tag_base = 0;        // plan identity, bits 24-47 of every run's tag (see run_tag)
+  MapCache* maps = nullptr;     // tensor maps already encoded for this plan, by operand address (made on first run)
   int split = 1;                // tail split factor of a dense plan
   int d_tri = 0;                // one triangle of D wanted: 1 lower, 2 upper (dense variants)
   int* d_tile_list = nullptr;   // device: the dealt tile schedule of one matrix (structured problems)
-  int* h_tile_list = nullptr;   // host copy, kept from planning until it has been uploaded
-  ~gemm_plan_s() { free(h_tile_list); }
-  size_t split_flag_bytes = 0;
+  int* h_tile_list = nullptr;   // host copy (uploaded at plan time; gemm_plan_schedule walks it)
+  ~gemm_plan_s() {
+    free(h_tile_list);
+    delete maps;
+  }
+  size_t split_flag_bytes = 0;  // head of a tail-split plan's workspace: one 64-bit flag word per partial tile
   unsigned long long runs = 0;  // launches so far (the timeout test hook acts on the first one only)
   uint32_t timeout_ms;
   DenseParams dense;     // filled at plan time except pointers / scalars
@@ -519,13 +588,13 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   p.split_first_tile = static_cast<int>(split > 1 ? num_tiles - rem : num_tiles);
   p.num_items = static_cast<int>(split > 1 ? num_tiles - rem + rem * split : num_tiles);
   pl->split = split;
-  pl->split_flag_bytes = split > 1 ? (static_cast<size_t>(rem) * cg * (split - 1) * 4 + 255) / 256 * 256 : 0;
+  pl->split_flag_bytes = split > 1 ? (static_cast<size_t>(rem) * cg * (split - 1) * 8 + 255) / 256 * 256 : 0;
   if (split > 1) pl->grid = static_cast<int>(std::min<long long>(p.num_items, units_i)) * cg;
   info.grid = pl->grid;
   info.split = split;
   info.smem_bytes = smem;
   info.num_tiles = num_tiles;
-  info.workspace_bytes = split > 1 ? static_cast<size_t>(rem) * cg * (split - 1) * kCtaM * bn * 4 : 0;
+  info.workspace_bytes = split > 1 ? pl->split_flag_bytes + static_cast<size_t>(rem) * cg * (split - 1) * kCtaM * bn * 4 : 0;
   return GEMM_OK;
 }
 
@@ -651,13 +720,25 @@ gemm_status_t plan_skinny(gemm_plan_s* pl, int forced_stages, int forced_atoms) 
   info.split = s.max_contributors;
   info.smem_bytes = s.smem_bytes;
   info.num_tiles = s.total_units;
-  info.workspace_bytes = s.workspace_bytes;
+  info.workspace_bytes = s.counters_bytes + s.workspace_bytes;  // arrival words, then the partial tiles
   return GEMM_OK;
 }
 
 }  // namespace
 
 namespace {
+
+// Identity of a plan (or of one allocation-free call), 24 bits, never 0: together with the run number it forms the tag
+// that marks a run's hand-shake words in a workspace, so that words left by anything else read as "nothing yet".
+uint64_t next_plan_identity() {
+  static std::atomic<uint64_t> counter{0};
+  uint64_t id;
+  do id = (counter.fetch_add(1, std::memory_order_relaxed) + 1) & 0xFFFFFFull;
+  while (id == 0);
+  return id;
+}
+// Tag of run number `run` of a plan: 48 bits, never 0 because the identity is not.
+uint64_t run_tag(uint64_t tag_base, unsigned long long run) { return tag_base | (run & 0xFFFFFFull); }
 
 // gemm_plan proper.  use_cache: take the tuning fields gemm_tune remembered for this shape (when the caller set none);
 // *cache_used tells whether that happened.
@@ -762,12 +843,12 @@ gemm_status_t plan_impl(const gemm_desc_t* desc, gemm_plan_t* out_plan, bool use
     delete pl;
     return st;
   }
+  pl->tag_base = next_plan_identity() << 24;
   if (pl->has_device && pl->arch_ok) {
-    // the counters start at zero here and every run leaves them at zero again (gemm_plan_status cleans up after a timeout)
-    pl->d_counters_bytes = pl->variant == GEMM_VARIANT_SKINNY_STREAMK ? pl->skinny.counters_bytes : pl->split_flag_bytes;
-    const size_t dev_bytes = pl->d_counters_bytes ? 256 + pl->d_counters_bytes : 16;
-    if (cudaMalloc(&pl->d_status, dev_bytes) != cudaSuccess || cudaMemset(pl->d_status, 0, dev_bytes) != cudaSuccess) {
+    pl->maps = new (std::nothrow) MapCache();
+    if (!pl->maps || cudaMalloc(&pl->d_status, 16) != cudaSuccess || cudaMemset(pl->d_status, 0, 16) != cudaSuccess) {
       note_cuda_error("cudaMalloc(status word)", cudaGetErrorName(cudaGetLastError()));
+      if (pl->d_status) cudaFree(pl->d_status);
       delete pl;
       return GEMM_ERR_CUDA;
     }
@@ -782,9 +863,7 @@ gemm_status_t plan_impl(const gemm_desc_t* desc, gemm_plan_t* out_plan, bool use
       delete pl;
       return GEMM_ERR_CUDA;
     }
-    pl->dense.tile_list = pl->d_tile_list;
-    free(pl->h_tile_list);
-    pl->h_tile_list = nullptr;
+    pl->dense.tile_list = pl->d_tile_list;  // (the host copy stays with the plan for gemm_plan_schedule)
   }
   if (getenv("B200GEMM_LOG")) {
     fprintf(stderr,
@@ -798,6 +877,16 @@ gemm_status_t plan_impl(const gemm_desc_t* desc, gemm_plan_t* out_plan, bool use
   return GEMM_OK;
 }
 
+}  // namespace
+
+namespace {
+// Take the status word: what a timed-out run left there goes to the plan's page-locked host word (read by
+// gemm_plan_status_result once the stream has got this far) and the device word is cleared in the same atomic step,
+// so a run on another stream that gives up at this very moment is not lost.
+__global__ void status_take_kernel(uint32_t* status, uint32_t* host_word) {
+  const uint32_t v = atomicExch(status, 0u);
+  if (v != 0u) *reinterpret_cast<volatile uint32_t*>(host_word) = v;
+}
 }  // namespace
 
 extern "C" {
@@ -825,24 +914,121 @@ gemm_status_t gemm_plan_set_timeout_ms(gemm_plan_t plan, uint32_t ms) {
   return GEMM_OK;
 }
 
+gemm_status_t gemm_plan_status_async(gemm_plan_t plan, gemm_stream_t stream) {
+  if (!plan) return GEMM_ERR_NULL;
+  if (!plan->d_status) return GEMM_ERR_ARCH;
+  int cur = -1;
+  if (cudaGetDevice(&cur) != cudaSuccess || cur != plan->device) return GEMM_ERR_INVALID_ARG;
+  cudaError_t e = cudaSuccess;
+  {
+    static std::mutex mu;  // first use only: the page-locked word the device writes the status into
+    std::lock_guard<std::mutex> lock(mu);
+    if (!plan->h_status) {
+      void* h = nullptr;
+      e = cudaHostAlloc(&h, 16, cudaHostAllocMapped | cudaHostAllocPortable);
+      if (e == cudaSuccess) {
+        memset(h, 0, 16);
+        plan->h_status = static_cast<uint32_t*>(h);
+      }
+    }
+  }
+  uint32_t* dev_view = nullptr;
+  if (e == cudaSuccess) e = cudaHostGetDevicePointer(reinterpret_cast<void**>(&dev_view), plan->h_status, 0);
+  if (e == cudaSuccess) {
+    status_take_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(plan->d_status, dev_view);
+    e = cudaGetLastError();
+  }
+  if (e != cudaSuccess) {
+    note_cuda_error("gemm_plan_status_async", cudaGetErrorName(e));
+    (void)cudaGetLastError();
+    return GEMM_ERR_CUDA;
+  }
+  return GEMM_OK;
+}
+
+gemm_status_t gemm_plan_status_result(gemm_plan_t plan) {
+  if (!plan) return GEMM_ERR_NULL;
+  if (!plan->h_status) return GEMM_OK;  // nothing was ever fetched
+  const uint32_t word = __atomic_exchange_n(plan->h_status, 0u, __ATOMIC_ACQUIRE);
+  if (word & kStatusTimeout) {
+    snprintf(g_last_cuda_error, sizeof g_last_cuda_error, "device wait expired: role %u detail 0x%02x", (word >> 8) & 0xFF,
+             word & 0xFF);
+    return GEMM_ERR_TIMEOUT;
+  }
+  return GEMM_OK;
+}
+
+gemm_status_t gemm_plan_status_stream(gemm_plan_t plan, gemm_stream_t stream) {
+  gemm_status_t st = gemm_plan_status_async(plan, stream);
+  if (st != GEMM_OK) return st;
+  const cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) {
+    note_cuda_error("gemm_plan_status_stream", cudaGetErrorName(e));
+    (void)cudaGetLastError();
+    return GEMM_ERR_CUDA;
+  }
+  return gemm_plan_status_result(plan);
+}
+
 gemm_status_t gemm_plan_status(gemm_plan_t plan) {
   if (!plan) return GEMM_ERR_NULL;
   if (!plan->d_status) return GEMM_ERR_ARCH;
-  uint32_t h[4] = {0, 0, 0, 0};
-  cudaError_t e = cudaDeviceSynchronize();
-  if (e == cudaSuccess) e = cudaMemcpy(h, plan->d_status, 16, cudaMemcpyDeviceToHost);
-  if (e == cudaSuccess) e = cudaMemset(plan->d_status, 0, 16);
-  if (e == cudaSuccess && h[0] != 0 && plan->d_counters_bytes)  // a run that gave up may have left arrivals half counted
-    e = cudaMemset(reinterpret_cast<char*>(plan->d_status) + 256, 0, plan->d_counters_bytes);
+  const cudaError_t e = cudaDeviceSynchronize();  // the plan does not know which streams ran it: wait for all of them
   if (e != cudaSuccess) {
     note_cuda_error("gemm_plan_status", cudaGetErrorName(e));
+    (void)cudaGetLastError();
     return GEMM_ERR_CUDA;
   }
-  if (h[0] & kStatusTimeout) {
-    snprintf(g_last_cuda_error, sizeof g_last_cuda_error, "device wait expired: role %u detail 0x%02x", (h[0] >> 8) & 0xFF,
-             h[0] & 0xFF);
-    return GEMM_ERR_TIMEOUT;
+  return gemm_plan_status_stream(plan, nullptr);
+}
+
+gemm_status_t gemm_plan_schedule(gemm_plan_t plan, gemm_work_item_t* items, size_t capacity, size_t* count) {
+  if (!plan || !count || (capacity > 0 && !items)) return GEMM_ERR_NULL;
+  size_t n = 0;
+  auto emit = [&](int cta, int batch, int row, int col, int k0, int k1, int slice) {
+    if (n < capacity) items[n] = gemm_work_item_t{cta, batch, row, col, k0, k1, slice, 0};
+    ++n;
+  };
+  if (plan->variant == GEMM_VARIANT_SKINNY_STREAMK) {
+    const SkinnyPlan& s = plan->skinny;
+    for (int c = 0; c < s.grid; ++c) {
+      const int u_end = sk_begin(c + 1, s.units_q, s.units_r);
+      for (int u = sk_begin(c, s.units_q, s.units_r); u < u_end;) {  // one item per tile this CTA's range touches
+        const int tile = u / s.kbs, tile_u0 = tile * s.kbs;
+        const int seg_end = std::min(u_end, tile_u0 + s.kbs);
+        const bool whole = u == tile_u0 && seg_end == tile_u0 + s.kbs;
+        const int slice = whole ? -1 : c - sk_owner(tile_u0, s.units_q, s.units_r);  // position among the tile's contributors
+        emit(c, 0, plan->skinny_tall ? tile : 0, plan->skinny_tall ? 0 : tile, u - tile_u0, seg_end - tile_u0, slice);
+        u = seg_end;
+      }
+    }
+  } else {
+    DenseParams p = plan->dense;
+    p.tile_list = plan->h_tile_list;  // (nullptr for an unstructured problem)
+    const int cg = plan->cg, clusters = plan->grid / cg;
+    const bool wide = plan->variant == GEMM_VARIANT_DENSE_2CTA_WIDE;
+    const int tile_rows = (wide ? kWideCtaM : kCtaM) * cg;
+    for (int c = 0; c < clusters; ++c) {
+      if (wide) {
+        for (int tile = c; tile < p.num_tiles; tile += clusters) {
+          const TileCoord tc = decode_tile_div(tile, p.tiles_m, p.tiles_n, p.raster_group);
+          emit(c, tc.batch, tc.tm, tc.tn, 0, p.num_kb, -1);
+        }
+        continue;
+      }
+      const bool split = plan->split > 1;
+      const int n_items = split ? p.num_items : p.num_tiles;
+      for (int item = c; item < n_items; item += clusters) {
+        const int tile = split ? item_tile<true>(p, item) : item_tile<false>(p, item);
+        if (tile < 0) continue;
+        const TileCoord tc = decode_tile(p, tile);
+        const WorkItem wi = split ? work_item<true>(p, item, tile, tc.tm * tile_rows, tile_rows, tc.tn * p.bn)
+                                  : work_item<false>(p, item, tile, tc.tm * tile_rows, tile_rows, tc.tn * p.bn);
+        emit(c, tc.batch, tc.tm, tc.tn, wi.kr.lo, wi.kr.hi, wi.slice);
+      }
+    }
   }
+  *count = n;
   return GEMM_OK;
 }
 
@@ -855,6 +1041,10 @@ gemm_status_t gemm_destroy(gemm_plan_t plan) {
   }
   if (plan->d_status && cudaFree(plan->d_status) != cudaSuccess) {
     note_cuda_error("cudaFree", cudaGetErrorName(cudaGetLastError()));
+    st = GEMM_ERR_CUDA;
+  }
+  if (plan->h_status && cudaFreeHost(plan->h_status) != cudaSuccess) {
+    note_cuda_error("cudaFreeHost", cudaGetErrorName(cudaGetLastError()));
     st = GEMM_ERR_CUDA;
   }
   delete plan;
@@ -949,21 +1139,33 @@ gemm_status_t launch_wide(const gemm_plan_s* pl, const CUtensorMap& tA, const CU
 }
 
 gemm_status_t run_dense(gemm_plan_s* pl, const void* A, const void* B, void* C, const float* bias, float alpha, float beta,
-                        void* workspace, cudaStream_t stream, bool stall) {
+                        void* workspace, cudaStream_t stream, bool stall, unsigned long long run_index) {
   const gemm_desc_t& d = pl->d;
   DenseParams p = pl->dense;
   CUtensorMap tA, tB, tD;
   const uint64_t batch = d.batch_count;
+  // Each map is encoded the first time its operand address is seen and fetched from the plan's table afterwards
+  // (an encoding costs the host about a microsecond, three of them more than the launch itself).
   // A: K-major -> rows are M, inner K, box 64 x 128; M-major (stored K x M) -> rows are K, inner M, box 64 x 64
   const uint32_t a_box_rows = pl->variant == GEMM_VARIANT_DENSE_2CTA_WIDE ? kWideCtaM : kCtaM;
-  bool ok = p.a_kmajor ? encode_map(&tA, d.ab_dtype, A, d.K, d.M, batch, d.lda, d.stride_a, p.kblk, a_box_rows)
-                       : encode_map(&tA, d.ab_dtype, A, d.M, d.K, batch, d.lda, d.stride_a, 64, kBlockK);
-  ok = ok && (p.b_kmajor ? encode_map(&tB, d.ab_dtype, B, d.K, d.N, batch, d.ldb, d.stride_b, p.kblk, p.b_rows)
-                         : encode_map(&tB, d.ab_dtype, B, d.N, d.K, batch, d.ldb, d.stride_b, 64, kBlockK));
-  const uint32_t slab_cols = d.c_dtype == GEMM_F32 ? 32 : 64;
-  // (whole 16-byte units of a row only: the store engine writes whole units, see DenseParams::n_full)
-  const uint64_t d_cols = std::max<uint64_t>(p.n_full, 16 / elem_bytes(d.c_dtype));
-  ok = ok && encode_map(&tD, d.c_dtype, C, d_cols, d.M, batch, d.ldc, d.stride_c, slab_cols, 32);
+  bool ok = true;
+  if (!pl->maps->find(0, A, &tA)) {
+    ok = p.a_kmajor ? encode_map(&tA, d.ab_dtype, A, d.K, d.M, batch, d.lda, d.stride_a, p.kblk, a_box_rows)
+                    : encode_map(&tA, d.ab_dtype, A, d.M, d.K, batch, d.lda, d.stride_a, 64, kBlockK);
+    if (ok) pl->maps->insert(0, A, tA);
+  }
+  if (ok && !pl->maps->find(1, B, &tB)) {
+    ok = p.b_kmajor ? encode_map(&tB, d.ab_dtype, B, d.K, d.N, batch, d.ldb, d.stride_b, p.kblk, p.b_rows)
+                    : encode_map(&tB, d.ab_dtype, B, d.N, d.K, batch, d.ldb, d.stride_b, 64, kBlockK);
+    if (ok) pl->maps->insert(1, B, tB);
+  }
+  if (ok && !pl->maps->find(2, C, &tD)) {
+    const uint32_t slab_cols = d.c_dtype == GEMM_F32 ? 32 : 64;
+    // (whole 16-byte units of a row only: the store engine writes whole units, see DenseParams::n_full)
+    const uint64_t d_cols = std::max<uint64_t>(p.n_full, 16 / elem_bytes(d.c_dtype));
+    ok = encode_map(&tD, d.c_dtype, C, d_cols, d.M, batch, d.ldc, d.stride_c, slab_cols, 32);
+    if (ok) pl->maps->insert(2, C, tD);
+  }
   if (!ok) return GEMM_ERR_CUDA;
   p.alpha = alpha;
   p.beta = beta;
@@ -975,8 +1177,10 @@ gemm_status_t run_dense(gemm_plan_s* pl, const void* A, const void* B, void* C, 
   if (pl->variant == GEMM_VARIANT_DENSE_2CTA_WIDE) return launch_wide(pl, tA, tB, tD, p, stream);
   gemm_status_t st;
   if (pl->split > 1) {
-    p.partials = static_cast<float*>(workspace);
-    p.split_flags = reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(pl->d_status) + 256);
+    // head of the workspace: the flag words (tagged per run, no initialisation needed); behind them the partial tiles
+    p.split_flags = static_cast<unsigned long long*>(workspace);
+    p.partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + pl->split_flag_bytes);
+    p.split_tag = run_tag(pl->tag_base, run_index);
     if (pl->cg == 1) st = pl->epi_wg == 2 ? launch_dense<1, 2, true>(pl, tA, tB, tD, p, stream) : launch_dense<1, 1, true>(pl, tA, tB, tD, p, stream);
     else st = pl->epi_wg == 2 ? launch_dense<2, 2, true>(pl, tA, tB, tD, p, stream) : launch_dense<2, 1, true>(pl, tA, tB, tD, p, stream);
   } else if (pl->cg == 1) {
@@ -1002,19 +1206,24 @@ gemm_status_t run_dense(gemm_plan_s* pl, const void* A, const void* B, void* C, 
 }
 
 gemm_status_t run_skinny(gemm_plan_s* pl, const void* A, const void* B, void* C, const float* bias, float alpha, float beta,
-                         void* workspace, cudaStream_t stream, bool stall) {
+                         void* workspace, cudaStream_t stream, bool stall, unsigned long long run_index) {
   const gemm_desc_t& d = pl->d;
   const SkinnyPlan& s = pl->skinny;
   CUtensorMap tW, tX;
   // weights W = B stored N x K (K contiguous): box 64 x 128; activations X = A stored M x K: box 64 x m_pad;
-  // a tall problem streams A in W's place and keeps B as the slab
-  bool ok;
-  if (pl->skinny_tall) {
-    ok = encode_map(&tW, d.ab_dtype, A, d.K, d.M, 1, d.lda, 0, s.kblk, kSkinnyTileN);
-    ok = ok && encode_map(&tX, d.ab_dtype, B, d.K, d.N, 1, d.ldb, 0, s.kblk, s.m_pad);
-  } else {
-    ok = encode_map(&tW, d.ab_dtype, B, d.K, d.N, 1, d.ldb, 0, s.kblk, kSkinnyTileN);
-    ok = ok && encode_map(&tX, d.ab_dtype, A, d.K, d.M, 1, d.lda, 0, s.kblk, s.m_pad);
+  // a tall problem streams A in W's place and keeps B as the slab.  Maps are remembered by operand address.
+  const void* w_ptr = pl->skinny_tall ? A : B;
+  const void* x_ptr = pl->skinny_tall ? B : A;
+  const int64_t w_rows = pl->skinny_tall ? d.M : d.N, w_ld = pl->skinny_tall ? d.lda : d.ldb;
+  const int64_t x_rows = pl->skinny_tall ? d.N : d.M, x_ld = pl->skinny_tall ? d.ldb : d.lda;
+  bool ok = true;
+  if (!pl->maps->find(0, w_ptr, &tW)) {
+    ok = encode_map(&tW, d.ab_dtype, w_ptr, d.K, w_rows, 1, w_ld, 0, s.kblk, kSkinnyTileN);
+    if (ok) pl->maps->insert(0, w_ptr, tW);
+  }
+  if (ok && !pl->maps->find(1, x_ptr, &tX)) {
+    ok = encode_map(&tX, d.ab_dtype, x_ptr, d.K, x_rows, 1, x_ld, 0, s.kblk, s.m_pad);
+    if (ok) pl->maps->insert(1, x_ptr, tX);
   }
   if (!ok) return GEMM_ERR_CUDA;
   SkinnyParams p;
@@ -1033,13 +1242,15 @@ gemm_status_t run_skinny(gemm_plan_s* pl, const void* A, const void* B, void* C,
   p.bias = bias;
   p.c = C;
   p.ldc = d.ldc;
-  p.partials = static_cast<float*>(workspace);
-  p.counters = reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(pl->d_status) + 256);
+  // head of the workspace: the arrival words (tagged per run, no initialisation needed); behind them the partial tiles
+  p.counters = static_cast<unsigned long long*>(workspace);
+  p.partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + s.counters_bytes);
+  p.tag = run_tag(pl->tag_base, run_index);
   p.debug_flags = stall ? 1u : 0u;
   p.status = pl->d_status;
   p.timeout_ns = static_cast<unsigned long long>(pl->timeout_ms) * 1000000ull;
   return static_cast<gemm_status_t>(
-      skinny_launch(p, tW, tX, pl->device, stream, g_last_cuda_error, sizeof g_last_cuda_error, pl->skinny_tall, /*zero_counters=*/false,
+      skinny_launch(p, tW, tX, pl->device, stream, g_last_cuda_error, sizeof g_last_cuda_error, pl->skinny_tall,
                     /*early_launch=*/!(d.flags & GEMM_FLAG_NO_EARLY_LAUNCH)));
 }
 
@@ -1060,11 +1271,11 @@ extern "C" gemm_status_t gemm_run(gemm_plan_t plan, const void* A, const void* B
   int cur = -1;
   if (cudaGetDevice(&cur) != cudaSuccess || cur != plan->device) return GEMM_ERR_INVALID_ARG;  // plan belongs to another device
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  // (atomic: a dense plan may be run from several host threads at once)
+  // (atomic: a plan may be run from several host threads at once)
   const unsigned long long run_index = __atomic_fetch_add(&plan->runs, 1ull, __ATOMIC_RELAXED);
   const bool stall = (plan->d.flags & GEMM_FLAG_DEBUG_STALL) && run_index == 0;  // test hook: the plan's first run only
-  if (plan->variant == GEMM_VARIANT_SKINNY_STREAMK) return run_skinny(plan, A, B, C, bias, alpha, beta, workspace, s, stall);
-  return run_dense(plan, A, B, C, bias, alpha, beta, workspace, s, stall);
+  if (plan->variant == GEMM_VARIANT_SKINNY_STREAMK) return run_skinny(plan, A, B, C, bias, alpha, beta, workspace, s, stall, run_index);
+  return run_dense(plan, A, B, C, bias, alpha, beta, workspace, s, stall, run_index);
 }
 
 // ---------------------------------------------------------------------------------------------------------
@@ -1128,8 +1339,11 @@ extern "C" gemm_status_t gemm_skinny_run_noalloc(const gemm_desc_t* desc, const 
   gemm_status_t st = validate(desc);
   if (st != GEMM_OK) return st;
   if (has_bias(desc->epilogue) && !bias) return GEMM_ERR_NULL;
+  // what the stream-K plans refuse is refused here too: every structure promise (this kernel skips nothing, so it would
+  // multiply a triangle the caller declared as not stored) and the per-row bias this entry point has no field for
   if (desc->transa != GEMM_OP_N || desc->transb != GEMM_OP_T || desc->batch_count != 1 || desc->M > kSkinnyMaxM || is_fp8(desc->ab_dtype) ||
-      (desc->structure & GEMM_STRUCT_D_MIRROR))  // (the mirror step belongs to the dense plans)
+      desc->structure != 0 ||
+      (desc->flags & (GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER | GEMM_FLAG_D_LOWER | GEMM_FLAG_D_UPPER | GEMM_FLAG_BIAS_PER_ROW)))
     return GEMM_ERR_UNSUPPORTED;
   auto misaligned = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; };
   if (misaligned(A) || misaligned(B) || misaligned(C) || (bias && misaligned(bias))) return GEMM_ERR_ALIGNMENT;
@@ -1158,8 +1372,9 @@ extern "C" gemm_status_t gemm_skinny_run_noalloc(const gemm_desc_t* desc, const 
       !encode_map(&tX, desc->ab_dtype, A, desc->K, desc->M, 1, desc->lda, 0, kBlockK, sp.m_pad))
     return GEMM_ERR_CUDA;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  // The array keeps whatever the previous call left: the status word must start at zero (the launch helper
-  // clears the arrival counters itself; the partial tiles are fully written before they are read).
+  // The array keeps whatever the previous call left: the status word must start at zero (the arrival words carry a
+  // tag that is new with every call, so the previous call's read as empty; the partial tiles are fully written
+  // before they are read).
   cudaError_t e = cudaMemsetAsync(nd.scratch, 0, kNoAllocHeaderBytes, s);
   if (e != cudaSuccess) {
     note_cuda_error("cudaMemsetAsync(status)", cudaGetErrorName(e));
@@ -1175,19 +1390,19 @@ extern "C" gemm_status_t gemm_skinny_run_noalloc(const gemm_desc_t* desc, const 
   p.idesc = make_idesc(desc->ab_dtype == GEMM_BF16, 0, 0, kSkinnyTileN, sp.m_pad);
   p.out_dtype = desc->c_dtype;
   p.epilogue = desc->epilogue;
-  p.bias_per_row = 0;  // desc->flags is ignored by this entry point
+  p.bias_per_row = 0;  // (refused above; the tuning fields of desc->flags are ignored)
   p.alpha = alpha;
   p.beta = beta;
   p.bias = bias;
   p.c = C;
   p.ldc = desc->ldc;
   p.status = reinterpret_cast<uint32_t*>(nd.scratch);
-  p.counters = reinterpret_cast<uint32_t*>(nd.scratch + kNoAllocHeaderBytes);
+  p.counters = reinterpret_cast<unsigned long long*>(nd.scratch + kNoAllocHeaderBytes);
   p.partials = reinterpret_cast<float*>(nd.scratch + kNoAllocHeaderBytes + sp.counters_bytes);
+  p.tag = run_tag(next_plan_identity() << 24, 0);
   p.timeout_ns = 2000ull * 1000000ull;
   st = static_cast<gemm_status_t>(
-      skinny_launch(p, tW, tX, dev, s, g_last_cuda_error, sizeof g_last_cuda_error, /*tall=*/false, /*zero_counters=*/true,
-                    /*early_launch=*/false));
+      skinny_launch(p, tW, tX, dev, s, g_last_cuda_error, sizeof g_last_cuda_error, /*tall=*/false, /*early_launch=*/false));
   if (st != GEMM_OK || !sync_and_check) return st;
   uint32_t word = 0;
   e = cudaStreamSynchronize(s);

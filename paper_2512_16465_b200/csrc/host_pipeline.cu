@@ -128,8 +128,9 @@ extern "C" gemm_status_t gemm_host_run(gemm_host_t h, const void* hA, const void
   if (bias_epilogue(d.epilogue) && !hbias) return GEMM_ERR_NULL;
   int cur = -1;
   if (cudaGetDevice(&cur) != cudaSuccess || cur != h->device) return GEMM_ERR_INVALID_ARG;
-  const size_t b_rows = d.transb == GEMM_OP_T ? d.N : d.K;
-  bool ok = cudaMemcpyAsync(h->dB, hB, b_rows * d.ldb * h->a_elem, cudaMemcpyHostToDevice, h->s_in) == cudaSuccess;
+  // B is copied up to the last element of its last row: the caller's buffer need not hold the padding behind it
+  const size_t b_rows = d.transb == GEMM_OP_T ? d.N : d.K, b_row_len = d.transb == GEMM_OP_T ? d.K : d.N;
+  bool ok = cudaMemcpyAsync(h->dB, hB, ((b_rows - 1) * d.ldb + b_row_len) * h->a_elem, cudaMemcpyHostToDevice, h->s_in) == cudaSuccess;
   if (ok && h->dbias) {
     const size_t n = (d.flags & GEMM_FLAG_BIAS_PER_ROW) ? d.M : d.N;
     ok = cudaMemcpyAsync(h->dbias, hbias, n * sizeof(float), cudaMemcpyHostToDevice, h->s_in) == cudaSuccess;
@@ -176,8 +177,8 @@ extern "C" gemm_status_t gemm_host_run(gemm_host_t h, const void* hA, const void
     (void)cudaGetLastError();
     return GEMM_ERR_CUDA;
   }
-  st = gemm_plan_status(h->plan_full);
-  if (st == GEMM_OK && h->plan_last != h->plan_full) st = gemm_plan_status(h->plan_last);
+  st = gemm_plan_status_stream(h->plan_full, h->s_mm);
+  if (st == GEMM_OK && h->plan_last != h->plan_full) st = gemm_plan_status_stream(h->plan_last, h->s_mm);
   return st;
 }
 

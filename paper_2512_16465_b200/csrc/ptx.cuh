@@ -100,6 +100,27 @@ __device__ __forceinline__ uint32_t ld_acquire_gpu(const uint32_t* addr) {
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(addr) : "memory");
   return v;
 }
+// 64-bit forms for the hand-shake words that live in a caller's workspace (a run tag in the upper bits, see
+// skinny_kernel.cuh): compare-and-swap with the same release / acquire meaning as the add above, and plain loads / stores.
+__device__ __forceinline__ unsigned long long atom_cas_acq_rel_gpu_u64(unsigned long long* addr, unsigned long long expect,
+                                                                       unsigned long long value) {
+  unsigned long long old;
+  asm volatile("atom.acq_rel.gpu.global.cas.b64 %0, [%1], %2, %3;" : "=l"(old) : "l"(addr), "l"(expect), "l"(value) : "memory");
+  return old;
+}
+__device__ __forceinline__ unsigned long long ld_acquire_gpu_u64(const unsigned long long* addr) {
+  unsigned long long v;
+  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ unsigned long long ld_relaxed_gpu_u64(const unsigned long long* addr) {
+  unsigned long long v;
+  asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release_gpu_u64(unsigned long long* addr, unsigned long long v) {
+  asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(addr), "l"(v) : "memory");
+}
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // L2 eviction-priority policies for bulk copies (whole address range, fraction 1.0)

@@ -10,8 +10,12 @@
 //   * a CTA whose range covers only part of a tile's K writes its fp32 partial to the workspace and
 //     bumps the tile's arrival counter; the CTA that arrives last adds the partials in contributor
 //     order (deterministic, no floating-point atomics), applies the epilogue, writes D and puts the
-//     counter back to zero, so the counters are clean again when the kernel ends.
-//     Nobody ever waits for another CTA.
+//     counter back to zero.  Nobody ever waits for another CTA.
+//   * the counters live at the head of the caller's workspace and need no initialisation: a counter word is
+//     (run tag << 16 | arrivals), the tag being unique to the run (plan identity and run number, never 0), and a
+//     word that carries any other tag -- zeros, a timed-out run's leftovers, whatever the memory held before --
+//     reads as "no arrivals yet".  Runs of one plan on different workspaces therefore share nothing but the
+//     status word and may overlap.
 //
 // The same kernel serves the mirrored case, a tall output with a handful of columns (N <= 64 < M, kTall): the long
 // operand A[M x K] then takes W's place and B[N x K] takes X's; only the addressing of C, D and the bias differs.
@@ -47,8 +51,8 @@ struct SkinnyPlan {
   int stage_bytes;       // atoms x (16 KB of W + m_pad * 128 bytes of X)
   int smem_bytes;
   int max_contributors;  // upper bound on CTAs touching one tile
-  size_t counters_bytes; // arrival counters: n_tiles x u32, padded to 256 bytes
-  size_t workspace_bytes;  // partial tiles: grid * 2 slots of [m_pad][128] floats
+  size_t counters_bytes; // arrival counters at the head of the workspace: n_tiles x u64, padded to 256 bytes
+  size_t workspace_bytes;  // partial tiles behind them: grid * 2 slots of [m_pad][128] floats
 };
 
 // First work unit of CTA c, and the CTA that owns unit u (32-bit arithmetic: these run on the device's critical path).
@@ -115,7 +119,7 @@ inline bool skinny_make_plan(SkinnyPlan* s, int M, int N, int K, int sm_count, i
   if (s->smem_bytes > max_smem) return false;
   const int per_cta = s->units_q;  // >= 1
   s->max_contributors = (s->kbs + per_cta - 1) / per_cta + 1;
-  s->counters_bytes = (static_cast<size_t>(s->n_tiles) * 4 + 255) / 256 * 256;
+  s->counters_bytes = (static_cast<size_t>(s->n_tiles) * 8 + 255) / 256 * 256;
   s->workspace_bytes = static_cast<size_t>(s->grid) * 2 * kSkinnyTileN * s->m_pad * 4;
   return true;
 }
@@ -132,12 +136,29 @@ struct SkinnyParams {
   void* c;                // D buffer (also C_in when beta != 0), row-major M x N
   long long ldc;
   float* partials;        // workspace: slot-major, each slot [m_pad][128] floats
-  uint32_t* counters;     // one arrival counter per n-tile, zero at launch and zero again at the end
+  unsigned long long* counters;  // one arrival word per n-tile: run tag << 16 | arrivals (any other tag reads as zero arrivals)
+  unsigned long long tag;        // this run's tag (48 bits, never 0)
   uint32_t* status;
   unsigned long long timeout_ns;
   uint32_t debug_flags;   // bit 0: withhold one producer arrival (timeout test hook)
   int ab_fp8;             // operands are 8-bit floats (tcgen05 kind::f8f6f4)
 };
+
+// Count this CTA in on a tile's arrival word and return how many had arrived before it.  A word whose tag is not this
+// run's counts as zero arrivals and is replaced.  Lock-free: an attempt fails only because another contributor's
+// succeeded, so the loop ends after at most as many rounds as the tile has contributors; the limit is a backstop
+// (0xffffffff = gave up, which the caller treats as "not the last").
+__device__ __forceinline__ uint32_t sk_arrive(unsigned long long* word, unsigned long long tag) {
+  unsigned long long cur = ld_relaxed_gpu_u64(word);
+  for (int attempt = 0; attempt < 4096; ++attempt) {
+    const bool mine = (cur >> 16) == tag;
+    const unsigned long long want = mine ? cur + 1ull : ((tag << 16) | 1ull);
+    const unsigned long long prev = atom_cas_acq_rel_gpu_u64(word, cur, want);
+    if (prev == cur) return mine ? static_cast<uint32_t>(cur & 0xffffull) : 0u;
+    cur = prev;
+  }
+  return 0xffffffffu;
+}
 
 // `big` is this thread's index along the long output extent, s0 the first of its 16 indices along the short one.
 // D is row-major M x N: the short extent is M (rows) unless kTall.
@@ -291,9 +312,9 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
     tmem_base = *tmem_slot;
   }
   griddep_wait();  // from here on global memory is read and written
-  // An earlier run of this plan that timed out may have left arrival counters half counted; the status word stays
-  // set until the host has read it (and cleaned the counters), and until then no run trusts them.  The load is
-  // issued here and consumed only by the fix-up, long after it has landed.
+  // While the status word is set (an earlier run of this plan timed out and the host has not read the word yet) no
+  // run finishes split tiles: a replay of a captured launch carries the tag of the run that may have left arrivals
+  // half counted.  The load is issued here and consumed only by the fix-up, long after it has landed.
   const uint32_t stale_status = *reinterpret_cast<volatile const uint32_t*>(p.status);
 
   // The producer and MMA roles run warp-uniform (one elected lane issues), with the (tile, k-block) position and
@@ -415,7 +436,9 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
       const bool by_chunk = sp.m_pad > 16;  // parked value 16 b + j = chunk b of the other contributor (else: chunk 0 of contributor b)
       const uint32_t park = base + bars_off + 16u * kMaxStages + 64u + (threadIdx.x - 64u) * 4u;  // value v lives at park + 512 v
       if (!whole && (by_chunk ? c_last - c_first == 1 : c_last - c_first <= 3)) {
-        if (leader) s_early[seg == 0 ? 0 : 1] = (stale_status == 0u && ld_acquire_gpu(p.counters + tile) == static_cast<uint32_t>(c_last - c_first)) ? 1u : 0u;
+        if (leader)
+          s_early[seg == 0 ? 0 : 1] =
+              (stale_status == 0u && ld_acquire_gpu_u64(p.counters + tile) == ((p.tag << 16) | static_cast<unsigned long long>(c_last - c_first))) ? 1u : 0u;
         named_barrier_sync(1, 128);
         early = s_early[seg == 0 ? 0 : 1] != 0u;
         if (early) {
@@ -488,14 +511,14 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty0 + 8u * buf);
       if (early) {
-        if (leader) p.counters[tile] = 0u;  // the others counted themselves in; leave the counter clean for the next launch
+        if (leader) p.counters[tile] = 0ull;  // the others counted themselves in; a replay of this launch (same tag) must find no arrivals
       } else if (!whole) {
         // Publish the partial and count the arrival; the last contributor reduces.  The barrier orders the four
         // warps' partial stores before the leader's atomic, whose release makes them visible to whoever reads the
         // count later and whose acquire, passed on by the second barrier, lets this CTA read the earlier partials.
         named_barrier_sync(1, 128);
         if (leader) {
-          const uint32_t old = stale_status == 0u ? atom_add_acq_rel_gpu(p.counters + tile, 1u) : 0xffffffffu;
+          const uint32_t old = stale_status == 0u ? sk_arrive(p.counters + tile, p.tag) : 0xffffffffu;
           *s_last = (old == static_cast<uint32_t>(c_last - c_first)) ? 1u : 0u;
         }
         named_barrier_sync(1, 128);
@@ -526,7 +549,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
             }
             if (n < big_extent) sk_finish16<kTall>(p, m0, n, sum, cin);
           }
-          if (leader) p.counters[tile] = 0u;  // leave the counter clean for the next launch
+          if (leader) p.counters[tile] = 0ull;  // a replay of this launch (same tag) must find no arrivals
         }
         named_barrier_sync(1, 128);  // s_last is reused by the next segment
       }
@@ -543,15 +566,12 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
   }
 }
 
-// Launch, after zeroing the arrival counters when the caller cannot vouch for them (`zero_counters`; a plan's own
-// counters are zero from their allocation on, since every run puts them back).  Returns a gemm_status_t value
-// (0 = ok, 7 = CUDA failure).
+// Launch.  Returns a gemm_status_t value (0 = ok, 7 = CUDA failure).
 // `tall` selects the mirrored addressing (tW then maps A, tX maps B).
 inline int skinny_launch(const SkinnyParams& p, const CUtensorMap& tW, const CUtensorMap& tX, int device, cudaStream_t stream,
-                         char* err, size_t err_len, bool tall, bool zero_counters, bool early_launch) {
+                         char* err, size_t err_len, bool tall, bool early_launch) {
   cudaError_t e = tall ? ensure_dynamic_smem(reinterpret_cast<const void*>(skinny_gemm_kernel<true>), kSlotSkinnyTall, device, p.plan.smem_bytes)
                        : ensure_dynamic_smem(reinterpret_cast<const void*>(skinny_gemm_kernel<false>), kSlotSkinny, device, p.plan.smem_bytes);
-  if (e == cudaSuccess && zero_counters) e = cudaMemsetAsync(p.counters, 0, p.plan.counters_bytes, stream);
   if (e == cudaSuccess) {
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);

@@ -119,7 +119,7 @@ gemm_status_t time_candidate(const gemm_desc_t& d, const Args& a, Timer& t, floa
   if (st == GEMM_OK && (cudaEventRecord(t.e1, a.stream) != cudaSuccess || cudaEventSynchronize(t.e1) != cudaSuccess)) st = GEMM_ERR_CUDA;
   float total = 0.0f;
   if (st == GEMM_OK && cudaEventElapsedTime(&total, t.e0, t.e1) != cudaSuccess) st = GEMM_ERR_CUDA;
-  if (st == GEMM_OK) st = gemm_plan_status(plan);  // a candidate whose device-side wait expired is an error, not a slow plan
+  if (st == GEMM_OK) st = gemm_plan_status_stream(plan, a.stream);  // a candidate whose device-side wait expired is an error, not a slow plan
   gemm_destroy(plan);
   if (st == GEMM_OK) *ms = total / static_cast<float>(a.iterations);
   (void)cudaGetLastError();

@@ -89,13 +89,33 @@ def c_in_as(inputs: dict, w: wl.Workload, c_dtype: int):
     return oracle.round_to(vals, c_dtype)
 
 
+_NAN_BITS = {wl.BF16: 0x7FC0, wl.F16: 0x7E00, wl.FP8_E4M3: 0x7F, wl.FP8_E5M2: 0x7F}
+
+
+def poison_operand_padding(arr: np.ndarray, dtype: int, rows: int, row_len: int, ld: int, batch: int, stride: int) -> np.ndarray:
+    """A copy of a stored operand (``batch`` matrices of ``rows`` x ``row_len`` elements, pitch ``ld``, ``stride`` apart)
+    in which every element that is not part of a matrix -- the padding behind each row and the gaps between batches --
+    holds a NaN.  A kernel that reads any of them (a tensor map with the pitch as its extent, a box that runs past
+    the row's end) turns its result into NaN."""
+    if ld == row_len and (batch == 1 or stride == rows * ld) and arr.size == batch * rows * ld:
+        return arr                                   # tightly packed: there is no padding
+    out = np.full_like(arr, _NAN_BITS[dtype])
+    idx = (np.arange(batch, dtype=np.int64)[:, None, None] * stride + np.arange(rows, dtype=np.int64)[None, :, None] * ld +
+           np.arange(row_len, dtype=np.int64)[None, None, :]).ravel()
+    out[idx] = arr[idx]
+    return out
+
+
 def run_gpu(w: wl.Workload, inputs: dict, flags: int = 0, c_dtype=None, poison: bool = True, repeats: int = 1):
-    """Run the workload through the binding; returns (host bit array of the whole C buffer, plan info)."""
+    """Run the workload through the binding; returns (host bit array of the whole C buffer, plan info).  The device
+    copies of A and B carry NaN in every padding element (the oracle sees the plain inputs)."""
     cd = w.c_dtype if c_dtype is None else c_dtype
     plan = bg.Plan(desc_of(w, flags, cd))
     try:
-        A = to_device(inputs["A"], w.ab_dtype)
-        B = to_device(inputs["B"], w.ab_dtype)
+        a_rows, a_len = (w.K, w.M) if w.transa else (w.M, w.K)
+        b_rows, b_len = (w.N, w.K) if w.transb else (w.K, w.N)
+        A = to_device(poison_operand_padding(inputs["A"], w.ab_dtype, a_rows, a_len, w.lda, w.batch, w.stride_a), w.ab_dtype)
+        B = to_device(poison_operand_padding(inputs["B"], w.ab_dtype, b_rows, b_len, w.ldb, w.batch, w.stride_b), w.ab_dtype)
         bias = None if inputs["bias"] is None else to_device(inputs["bias"], wl.F32)
         cin = c_in_as(inputs, w, cd)
         outs = []

@@ -270,13 +270,15 @@ def test_random_problems(seed):
     """Integer-valued inputs: bit-exact wherever the epilogue keeps integers (none, bias, ReLU; alpha and beta are powers
     of two), the stated tolerance for the transcendental activations.  A combination the library documents as
     unsupported must be refused with that code, never run wrong."""
-    M, N, K, kw, fl = _random_case(seed)
-    w = int_workload(f"random_{seed}", M, N, K, **kw)
-    try:
-        H.check_workload(w, bg.make_flags(**fl), exact=kw["epi"] <= 3, repeats=2)
-    except bg.GemmError as e:
-        assert e.status == bg.ERR_UNSUPPORTED, (M, N, K, kw, fl)
-        pytest.skip(f"refused as unsupported: {M}x{N}x{K} {kw} {fl}")
+    for attempt in range(20):     # a refused draw is replaced by the next one, so that every seed runs a problem
+        M, N, K, kw, fl = _random_case(seed + 100000 * attempt)
+        w = int_workload(f"random_{seed}_{attempt}", M, N, K, **kw)
+        try:
+            H.check_workload(w, bg.make_flags(**fl), exact=kw["epi"] <= 3, repeats=2)
+            return
+        except bg.GemmError as e:
+            assert e.status == bg.ERR_UNSUPPORTED, (M, N, K, kw, fl)
+    pytest.fail("twenty draws in a row refused as unsupported")
 
 
 @pytest.mark.parametrize("seed", range(int(os.environ.get("B200GEMM_RANDOM_LARGE_CASES", "32"))))
@@ -284,28 +286,30 @@ def test_random_large_problems(seed):
     """The same draw at sizes where every CTA computes many tiles (several waves, ring and accumulator buffers wrapping
     many times, multi-round dealt schedules): extents up to about 4000, checked on 48 seeded rows and columns plus the
     tile-boundary indices."""
-    rng = np.random.default_rng(9000 + seed)
-    M, N, K, kw, fl = _random_case(10000 + seed)
-    if fl["variant"] == VS:
-        long_ = int(rng.integers(3000, 30000))
-        M, N = (M, long_) if M <= 64 else (long_, N)
-        K = int(rng.integers(256, 3000))
-    else:
-        M, N, K = int(rng.integers(600, 4200)), int(rng.integers(600, 4200)), int(rng.integers(64, 1600))
-    fp8 = kw["ab"] in (wl.FP8_E4M3, wl.FP8_E5M2)
-    ea, ec = (16 if fp8 else 8), (4 if kw["cd"] == wl.F32 else 8)
-    up = lambda x, m: -(-x // m) * m
-    kw.update(lda=up(M if kw["ta"] else K, ea) + ea, ldb=up(K if kw["tb"] else N, ea), ldc=up(N, ec) + ec)
-    for k in ("stride_a", "stride_b", "stride_c"):
-        kw.pop(k, None)
-    if kw["batch"] > 1 and M * N > 4e6:
-        kw["batch"] = 1
-    w = int_workload(f"random_large_{seed}", M, N, K, sample_rows=48, sample_cols=48, **kw)
-    try:
-        H.check_workload(w, bg.make_flags(**fl), exact=kw["epi"] <= 3)
-    except bg.GemmError as e:
-        assert e.status == bg.ERR_UNSUPPORTED, (M, N, K, kw, fl)
-        pytest.skip(f"refused as unsupported: {M}x{N}x{K} {kw} {fl}")
+    for attempt in range(20):     # a refused draw is replaced by the next one, so that every seed runs a problem
+        rng = np.random.default_rng(9000 + seed + 100000 * attempt)
+        M, N, K, kw, fl = _random_case(10000 + seed + 100000 * attempt)
+        if fl["variant"] == VS:
+            long_ = int(rng.integers(3000, 30000))
+            M, N = (M, long_) if M <= 64 else (long_, N)
+            K = int(rng.integers(256, 3000))
+        else:
+            M, N, K = int(rng.integers(600, 4200)), int(rng.integers(600, 4200)), int(rng.integers(64, 1600))
+        fp8 = kw["ab"] in (wl.FP8_E4M3, wl.FP8_E5M2)
+        ea, ec = (16 if fp8 else 8), (4 if kw["cd"] == wl.F32 else 8)
+        up = lambda x, m: -(-x // m) * m
+        kw.update(lda=up(M if kw["ta"] else K, ea) + ea, ldb=up(K if kw["tb"] else N, ea), ldc=up(N, ec) + ec)
+        for k in ("stride_a", "stride_b", "stride_c"):
+            kw.pop(k, None)
+        if kw["batch"] > 1 and M * N > 4e6:
+            kw["batch"] = 1
+        w = int_workload(f"random_large_{seed}_{attempt}", M, N, K, sample_rows=48, sample_cols=48, **kw)
+        try:
+            H.check_workload(w, bg.make_flags(**fl), exact=kw["epi"] <= 3)
+            return
+        except bg.GemmError as e:
+            assert e.status == bg.ERR_UNSUPPORTED, (M, N, K, kw, fl)
+    pytest.fail("twenty draws in a row refused as unsupported")
 
 
 def test_padded_leading_dimensions_and_strides():
@@ -541,32 +545,148 @@ def test_runs_are_capturable_in_a_cuda_graph():
         plan.close()
 
 
-def test_one_dense_plan_on_two_streams_and_stream_k_plans_per_stream():
-    """Runs of one dense plan may overlap on the GPU (they share nothing but the status word); stream-K plans share
-    their arrival counters between runs, so concurrent streams get one plan each."""
+def test_one_plan_on_two_streams_with_a_workspace_per_stream():
+    """Runs of one plan may overlap on the GPU when the runs that overlap use different workspaces: the hand-shake words
+    (stream-K arrival words, tail-split flags) live in the workspace, and the runs share nothing but the status word.
+    A dense plan without a workspace, a stream-K plan and a dense plan with a tail split, each launched alternately on
+    two streams."""
     wd = int_workload("two_streams_dense", 1024, 1024, 512, cd=wl.BF16)
     ws = int_workload("two_streams_stream_k", 8, 4096, 4096, beta=0.0)
+    wt = int_workload("two_streams_tail_split", 1024, 1024, 2048, cd=wl.BF16)
     streams = [torch.cuda.Stream() for _ in range(2)]
-    for w, plans in ((wd, None), (ws, "per stream")):
+    for w, flags in ((wd, 0), (ws, 0), (wt, bg.make_flags(V2, 256, tail_split=True))):
         inputs = wl.make_inputs(w)
         A, B = H.to_device(inputs["A"], w.ab_dtype), H.to_device(inputs["B"], w.ab_dtype)
         outs = [torch.empty(w.elems_c(), dtype=H._TORCH_DT[w.c_dtype], device="cuda") for _ in streams]
-        shared = bg.Plan(H.desc_of(w))
-        per = [shared, shared] if plans is None else [shared, bg.Plan(H.desc_of(w))]
-        wss = [pl.workspace_bytes and torch.empty(pl.workspace_bytes, dtype=torch.uint8, device="cuda") for pl in per]
+        plan = bg.Plan(H.desc_of(w, flags))
+        assert (plan.workspace_bytes > 0) == (w is not wd)
+        wss = [torch.empty(max(plan.workspace_bytes, 16), dtype=torch.uint8, device="cuda") for _ in streams]
         torch.cuda.synchronize()
         for rep in range(4):                       # interleaved launches: the kernels of the two streams overlap
-            for st, pl, out, wsb in zip(streams, per, outs, wss):
+            for st, out, wsb in zip(streams, outs, wss):
                 with torch.cuda.stream(st):
-                    pl.run(A, B, out, workspace=wsb if pl.workspace_bytes else None)
-        torch.cuda.synchronize()
-        for pl in set(per):
-            assert pl.status() == bg.OK
+                    plan.run(A, B, out, workspace=wsb if plan.workspace_bytes else None)
+        for st in streams:
+            assert plan.status(st.cuda_stream) == bg.OK     # waits for that stream only
         for out in outs:
             reports = H.check_blocks(w, inputs, H.to_host_bits(out, w.c_dtype), H.default_blocks(w))
             assert all(r["bit_identical"] == 1.0 for r in reports)
-        for pl in set(per):
-            pl.close()
+        plan.close()
+
+
+@pytest.mark.parametrize("fill", ["ones", "random", "zeros", "previous_plan"])
+def test_workspace_needs_no_initialisation(fill):
+    """The hand-shake words at the head of a workspace carry a per-run tag, so whatever the memory held before -- all
+    bits set, random bytes, zeros, or the words another plan of the same shape left there -- reads as "nothing yet"."""
+    cases = [(int_workload("ws_stream_k", 8, 4096, 4096, beta=1.0), 0),
+             (int_workload("ws_stream_k_m40", 40, 1000, 8200, cd=wl.BF16), 0),
+             (int_workload("ws_tail_split", 1024, 1024, 2048, cd=wl.BF16), bg.make_flags(V2, 256, tail_split=True)),
+             (int_workload("ws_long_k_auto_split", 256, 256, 16384), 0)]
+    for w, flags in cases:
+        inputs = wl.make_inputs(w)
+        A, B = H.to_device(inputs["A"], w.ab_dtype), H.to_device(inputs["B"], w.ab_dtype)
+        plan = bg.Plan(H.desc_of(w, flags))
+        assert plan.workspace_bytes > 0
+        ws = torch.empty(plan.workspace_bytes, dtype=torch.uint8, device="cuda")
+        for rep in range(2):
+            if fill == "ones":
+                ws.fill_(0xFF)
+            elif fill == "random":
+                ws.copy_(torch.randint(0, 256, (ws.numel(),), dtype=torch.uint8, generator=torch.Generator().manual_seed(rep)).cuda())
+            elif fill == "zeros":
+                ws.zero_()
+            elif fill == "previous_plan" and rep == 1:   # a second plan of the same shape inherits the first one's workspace
+                plan.close()
+                plan = bg.Plan(H.desc_of(w, flags))
+            C = H.to_device(inputs["C"], w.c_dtype) if inputs["C"] is not None else \
+                torch.full((w.elems_c(),), float("nan"), dtype=H._TORCH_DT[w.c_dtype], device="cuda")
+            plan.run(A, B, C, alpha=w.alpha, beta=w.beta, workspace=ws)
+            assert plan.status() == bg.OK
+            reports = H.check_blocks(w, inputs, H.to_host_bits(C, w.c_dtype), H.default_blocks(w))
+            assert all(r["bit_identical"] == 1.0 for r in reports), (w.name, fill, rep)
+        plan.close()
+
+
+def test_status_word_forms():
+    """gemm_plan_status_async enqueues the read and waits for nothing; gemm_plan_status_result reports it once the
+    caller has waited for the stream; gemm_plan_status_stream waits for one stream; gemm_plan_status for the device.
+    A withheld producer arrival (test flag) makes the first run time out, and each form sees and clears the word."""
+    w = int_workload("status_forms", 512, 512, 256)
+    inputs = wl.make_inputs(w)
+    A, B = H.to_device(inputs["A"], w.ab_dtype), H.to_device(inputs["B"], w.ab_dtype)
+    C = torch.zeros(w.elems_c(), dtype=torch.float32, device="cuda")
+    side = torch.cuda.Stream()
+    for form in ("async", "stream", "device"):
+        plan = bg.Plan(H.desc_of(w, bg.make_flags(V1, 128, debug_stall=True)))
+        plan.set_timeout_ms(20)
+        assert bg.gemm_plan_status_result(plan.handle) == bg.OK      # nothing fetched yet
+        with torch.cuda.stream(side):
+            plan.run(A, B, C)
+            if form == "async":
+                bg.gemm_plan_status_async(plan.handle, side.cuda_stream)
+                done = torch.cuda.Event()
+                done.record(side)
+                done.synchronize()
+                got = bg.gemm_plan_status_result(plan.handle)
+            elif form == "stream":
+                got = bg.gemm_plan_status_stream(plan.handle, side.cuda_stream)
+            else:
+                got = bg.gemm_plan_status(plan.handle)
+        assert got == bg.ERR_TIMEOUT, form
+        assert bg.gemm_plan_status_result(plan.handle) == bg.OK      # the result was taken
+        assert bg.gemm_plan_status_stream(plan.handle, side.cuda_stream) == bg.OK   # and the device word cleared
+        with torch.cuda.stream(side):
+            plan.run(A, B, C)
+            assert plan.status(side.cuda_stream) == bg.OK
+        reports = H.check_blocks(w, inputs, H.to_host_bits(C, w.c_dtype), H.default_blocks(w))
+        assert all(r["bit_identical"] == 1.0 for r in reports)
+        plan.close()
+
+
+def test_tensor_maps_are_remembered_by_operand_address():
+    """A plan keeps the tensor maps of the operand addresses it has seen.  Alternating between buffers, moving to new
+    ones and cycling through more addresses than the table holds must each give the result of the buffers passed."""
+    w = int_workload("map_cache", 264, 328, 200, cd=wl.BF16)
+    ws_ = int_workload("map_cache_stream_k", 8, 520, 1032)
+    for wk in (w, ws_):
+        plan = bg.Plan(H.desc_of(wk))
+        sets = []
+        for i in range(3):
+            inp = wl.make_inputs(wk, seed_offset=10 * i)
+            sets.append((inp, H.to_device(inp["A"], wk.ab_dtype), H.to_device(inp["B"], wk.ab_dtype)))
+        C0 = torch.zeros(wk.elems_c(), dtype=H._TORCH_DT[wk.c_dtype], device="cuda")
+        C1 = torch.zeros_like(C0)
+        def check(inp, C):
+            assert plan.status() == bg.OK
+            reports = H.check_blocks(wk, inp, H.to_host_bits(C, wk.c_dtype), H.default_blocks(wk))
+            assert all(r["bit_identical"] == 1.0 for r in reports)
+        for rep in range(3):                      # same addresses again and again, in turn
+            for (inp, A, B), C in zip(sets, (C0, C1, C0)):
+                C.fill_(float("nan"))
+                plan.run(A, B, C)
+                check(inp, C)
+        inp0, A0, B0 = sets[0]                    # A of one set with B of another: maps are kept per operand
+        inp1, A1, B1 = sets[1]
+        mixed = dict(inp0, B=inp1["B"])
+        plan.run(A0, B1, C1)
+        check(mixed, C1)
+        # more distinct addresses than the table has entries (offsets into one large buffer), twice round
+        n = 300
+        stride = -(-wk.elems_c() // 64) * 64
+        big = torch.zeros(n * stride, dtype=C0.dtype, device="cuda")
+        for rnd in range(2):
+            big.fill_(float("nan"))
+            for i in range(n):
+                plan.run(A0, B0, big[i * stride: i * stride + wk.elems_c()])
+            assert plan.status() == bg.OK
+            want = None
+            for i in (0, 1, 127, 128, 129, 255, 256, n - 1):
+                got = H.to_host_bits(big[i * stride: i * stride + wk.elems_c()], wk.c_dtype)
+                if want is None:
+                    check(inp0, big[:wk.elems_c()])
+                    want = got
+                assert np.array_equal(got, want), i
+        plan.close()
 
 
 @pytest.mark.parametrize("variant", [V1, V2, VW, VS])
@@ -586,8 +706,8 @@ def test_bounded_wait_reports_timeout_and_context_survives(variant):
     torch.cuda.synchronize()
     assert plan.status() == bg.ERR_TIMEOUT
     assert plan.status() == bg.OK          # reading clears the word
-    # the hook acts on the first run only: the same plan must now give the exact result (for stream-K this needs the
-    # arrival counters of the abandoned runs to have been put back to zero)
+    # the hook acts on the first run only: the same plan must now give the exact result (for stream-K the arrival words
+    # the abandoned runs left in the workspace carry those runs' tags and read as empty)
     for _ in range(2):
         C.fill_(float("nan"))
         plan.run(A, B, C)
@@ -607,16 +727,17 @@ def test_tail_split_plans():
         bg.gemm_destroy(h)
         return i
     i = info(1024, 1024, 2048, variant=V2, tile_n=256, tail_split=True)     # 16 pair tiles on 74 pairs: two slices each
-    assert i["split"] == 2 and i["grid"] == 64 and i["workspace_bytes"] == 16 * 2 * 1 * 128 * 256 * 4
+    # (one 64-bit flag word per partial tile at the head of the workspace, padded to 256 bytes, then the partial tiles)
+    assert i["split"] == 2 and i["grid"] == 64 and i["workspace_bytes"] == 256 + 16 * 2 * 1 * 128 * 256 * 4
     i = info(1024, 1024, 2048, variant=V2, tile_n=256)                      # not asked for: whole tiles, no workspace
     assert i["split"] == 1 and i["workspace_bytes"] == 0
     assert info(1024, 1024, 256, variant=V2, tile_n=256, tail_split=True)["split"] == 1      # too little K to slice
     assert info(3072, 3072, 3072, variant=V2, tile_n=256, tail_split=True)["split"] == 1     # 144 tiles: the last wave is 70 of 74
     i = info(2560, 2560, 2560, variant=V2, tile_n=256, tail_split=True)                      # 100 tiles: 74 + 26, the 26 in two slices
-    assert i["split"] == 2 and i["workspace_bytes"] == 26 * 2 * 1 * 128 * 256 * 4
+    assert i["split"] == 2 and i["workspace_bytes"] == 512 + 26 * 2 * 1 * 128 * 256 * 4
     assert info(16384, 14336, 4096, variant=V2, tile_n=256, tail_split=True)["split"] == 1   # 48 full waves: not worth it
     i = info(512, 512, 16384, variant=V2, tile_n=256)                                      # 4 tiles, 256 ring stages each: by itself
-    assert i["split"] == 7 and i["grid"] == 56 and i["workspace_bytes"] == 4 * 2 * 6 * 128 * 256 * 4
+    assert i["split"] == 7 and i["grid"] == 56 and i["workspace_bytes"] == 512 + 4 * 2 * 6 * 128 * 256 * 4
 
 
 @pytest.mark.parametrize("cd,N", [(wl.BF16, 900), (wl.F16, 899), (wl.F32, 901), (wl.F32, 5), (wl.BF16, 3)])
@@ -1015,15 +1136,20 @@ def test_tune_argument_errors():
     ("host_row_bias_nn", 1000, 136, 200, dict(epi=bg.EPI_BIAS, bias_per_row=True, tb=0), 4),
     ("host_skinny_panel", 40, 520, 1032, dict(beta=1.0), 1),
     ("host_fp8", 600, 264, 272, dict(ab=wl.FP8_E4M3, cd=wl.F16), 2),
+    ("host_padded_b_nt", 300, 264, 136, dict(ldb=136 + 8, lda=136 + 16), 2),
+    ("host_padded_b_nn", 300, 264, 136, dict(tb=0, ldb=264 + 24), 2),
 ], ids=lambda c: c[0])
 def test_host_resident_gemm_exact(case):
     """gemm_host_run on pinned host buffers: bit-exact against the oracle, padding of the host C buffer untouched,
-    and the same again on a second run of the same handle."""
+    and the same again on a second run of the same handle.  The pinned A and B buffers end with the last element of
+    their last row (no padding behind it), so a copy that reads whole pitches past that point fails."""
     name, M, N, K, kw, panels = case
     w = int_workload(name, M, N, K, **kw)
     inputs = wl.make_inputs(w)
     pin = lambda a: None if a is None else torch.from_numpy(a).pin_memory()
-    hA, hB, hbias = pin(inputs["A"]), pin(inputs["B"]), pin(inputs["bias"])
+    tight_a = (w.M - 1) * w.lda + w.K                                   # (host path: A is stored M x K)
+    tight_b = (w.N - 1) * w.ldb + w.K if w.transb else (w.K - 1) * w.ldb + w.N
+    hA, hB, hbias = pin(inputs["A"][:tight_a].copy()), pin(inputs["B"][:tight_b].copy()), pin(inputs["bias"])
     c_np = np.float32 if w.c_dtype == wl.F32 else np.uint16
     sentinel = np.full(w.elems_c(), 0x4321 if c_np == np.uint16 else 1234.5, c_np)
     handle = bg.gemm_host_create(H.desc_of(w), panels)

@@ -123,8 +123,8 @@ def test_stream_k_plan_geometry():
     assert i5["num_tiles"] == 224 * 64               # (n-tile, 128-wide k-block) work units
     assert i5["grid"] == 148 and i5["tile_m"] == 128 and i5["tile_n"] == 16 and i5["tile_k"] == 128
     assert i5["split"] >= 2 and i5["stages"] == 4    # 4 stages of two 64-wide K slices: 144 KB in flight per SM
-    # 2 partial slots of 128 x 16 fp32 per CTA (the arrival counters belong to the plan, not to the workspace)
-    assert i5["workspace_bytes"] == 148 * 2 * 128 * 16 * 4
+    # one 64-bit arrival word per output tile (padded to 256 bytes), then 2 partial slots of 128 x 16 fp32 per CTA
+    assert i5["workspace_bytes"] == 224 * 8 + 148 * 2 * 128 * 16 * 4
     tiny = info_for(wl.Workload("t", 4, 100, 64), bg.make_flags(bg.VARIANT_SKINNY_STREAMK))
     assert tiny["grid"] == 1 and tiny["num_tiles"] == 1
     # grids that line up with the tiles on mid-sized problems
@@ -246,7 +246,8 @@ def test_tuning_entry_points_on_the_host():
     assert bg.gemm_tune_workspace_bytes(bg.make_desc(1024, 1024, 4096)) > 0           # a tail-split candidate wants room
     need = bg.gemm_tune_workspace_bytes(bg.make_desc(8, 4096, 2048))
     assert need >= 148 * 2 * 128 * 16 * 4
-    assert bg.gemm_tune_workspace_bytes(bg.make_desc(4096, 8, 2048)) == need      # mirrored
+    # mirrored: the same partial tiles (the flag words at the head of a tail-split candidate's workspace differ a little)
+    assert abs(bg.gemm_tune_workspace_bytes(bg.make_desc(4096, 8, 2048)) - need) <= 1024
     bg.gemm_tune_cache_clear()                                                    # harmless when empty
     import torch
     if not torch.cuda.is_available():

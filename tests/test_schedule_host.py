@@ -1,0 +1,170 @@
+"""Host-only checks of the device-side schedules: gemm_plan_schedule walks a plan with the functions the kernels run
+(tile decoding with the plan-time divisors, the grouped raster, dealt schedules of structured problems, tail split,
+stream-K ranges).  What must hold for any plan: every wanted output tile is computed exactly once, the K stages of a
+split tile are covered exactly once, and K stages left out under a triangular operand can only hold zeros."""
+import itertools
+
+import numpy as np
+import pytest
+
+import paper_2512_16465_b200 as bg
+
+V1, V2, VS, VW = bg.VARIANT_DENSE_1CTA, bg.VARIANT_DENSE_2CTA, bg.VARIANT_SKINNY_STREAMK, bg.VARIANT_DENSE_2CTA_WIDE
+CTA, BATCH, ROW, COL, K0, K1, SLICE = range(7)
+
+
+def plan_and_schedule(M, N, K, flags=0, **kw):
+    up = lambda x: -(-x // 8) * 8            # leading dimensions must span multiples of 16 bytes
+    batch = kw.get("batch", 1)
+    kw.update(lda=up(K), ldb=up(K), ldc=up(N), stride_a=M * up(K), stride_b=N * up(K), stride_c=M * up(N))
+    if batch == 1:
+        kw.update(stride_a=0, stride_b=0, stride_c=0)
+    h = bg.gemm_plan(bg.make_desc(M, N, K, flags=flags, **kw))
+    try:
+        return bg.gemm_plan_info(h), bg.gemm_plan_schedule(h)
+    finally:
+        bg.gemm_destroy(h)
+
+
+def wanted_tiles(info, M, N, batch, d_tri):
+    """(batch, tile row, tile column) of every tile that holds at least one wanted element of D."""
+    tm, tn = info["tile_m"], info["tile_n"]
+    out = set()
+    for i in range(-(-M // tm)):
+        for j in range(-(-N // tn)):
+            r0, r1 = i * tm, min((i + 1) * tm, M) - 1
+            c0, c1 = j * tn, min((j + 1) * tn, N) - 1
+            if d_tri == 1 and r1 < c0:      # lower triangle wanted (row >= column): the tile lies wholly above the diagonal
+                continue
+            if d_tri == 2 and r0 > c1:
+                continue
+            out.update((b, i, j) for b in range(batch))
+    return out
+
+
+def check_dense(info, sched, M, N, K, batch=1, d_tri=0, a_tri=0, b_tri=0):
+    clusters = info["grid"] // info["cluster_size"]
+    assert sched[:, CTA].min() >= 0 and sched[:, CTA].max() < clusters
+    stages = -(-K // info["tile_k"])
+    by_tile = {}
+    for it in sched:
+        by_tile.setdefault((it[BATCH], it[ROW], it[COL]), []).append(it)
+    assert set(by_tile) == wanted_tiles(info, M, N, batch, d_tri)          # every wanted tile, and no other
+    tm, tn, tk = info["tile_m"], info["tile_n"], info["tile_k"]
+    for (b, i, j), items in by_tile.items():
+        if len(items) == 1:
+            it = items[0]
+            assert it[SLICE] == -1
+            lo, hi = it[K0], it[K1]
+        else:                                                              # K slices: 0 .. n-1, contiguous, disjoint
+            items.sort(key=lambda it: it[SLICE])
+            assert [it[SLICE] for it in items] == list(range(len(items))) == list(range(info["split"]))
+            assert all(x[K1] == y[K0] for x, y in zip(items, items[1:]))
+            assert len({it[CTA] for it in items}) == len(items)            # side by side, one CTA (pair) each
+            lo, hi = items[0][K0], items[-1][K1]
+        assert 0 <= lo < hi <= stages
+        # a stage that was left out must lie wholly in the zero part of a triangular operand
+        r0, r1 = i * tm, min((i + 1) * tm, M) - 1
+        c0, c1 = j * tn, min((j + 1) * tn, N) - 1
+        for s in itertools.chain(range(0, lo), range(hi, stages)):
+            k0, k1 = s * tk, min((s + 1) * tk, K) - 1
+            zero_a = (a_tri == 1 and k0 > r1) or (a_tri == 2 and k1 < r0)   # lower: zero for k > i; upper: zero for k < i
+            zero_b = (b_tri == 1 and k1 < c0) or (b_tri == 2 and k0 > c1)   # lower: zero for k < j; upper: zero for k > j
+            assert zero_a or zero_b, ((b, i, j), s, (lo, hi))
+        if not (a_tri or b_tri):
+            assert (lo, hi) == (0, stages)
+    # execution order inside a CTA: the static round-robin visits its items in increasing order of the linear work id,
+    # which the list reports per CTA; the per-CTA loads differ by at most one item on an unstructured problem
+    if not (d_tri or a_tri or b_tri):
+        per = np.bincount(sched[:, CTA], minlength=clusters)
+        assert per.max() - per.min() <= 1
+
+
+DENSE_SHAPES = [(512, 512, 512), (1, 1, 1), (129, 257, 65), (1000, 1000, 1000), (2560, 2560, 2560), (4100, 4104, 4104),
+                (8192, 8192, 8192), (300, 70000, 64), (16384, 14336, 4096), (130, 258, 66000), (12345, 4328, 2056)]
+
+
+@pytest.mark.parametrize("shape", DENSE_SHAPES, ids=lambda s: "x".join(map(str, s)))
+@pytest.mark.parametrize("variant,tile_n", [(0, 0), (V1, 64), (V1, 128), (V1, 192), (V1, 256), (V2, 128), (V2, 256), (VW, 0)])
+def test_every_tile_once_dense(shape, variant, tile_n):
+    M, N, K = shape
+    if variant == VW and M <= 128:
+        pytest.skip("a pair needs two tile rows")
+    for raster in (0, 1, 3, 7, 100):
+        for batch in (1, 3):
+            if batch > 1 and M * N > 3e7:
+                continue
+            try:
+                info, sched = plan_and_schedule(M, N, K, bg.make_flags(variant, tile_n, raster=raster), batch=batch, c_dtype=bg.BF16)
+            except bg.GemmError as e:
+                assert e.status == bg.ERR_UNSUPPORTED
+                continue
+            check_dense(info, sched, M, N, K, batch)
+
+
+@pytest.mark.parametrize("shape", [(1024, 1024, 2048), (2560, 2560, 2560), (512, 512, 16384), (1536, 1536, 4096), (130, 258, 66000),
+                                   (1000, 1000, 1096), (1280, 4096, 512)], ids=lambda s: "x".join(map(str, s)))
+@pytest.mark.parametrize("variant,tile_n", [(V1, 128), (V1, 256), (V2, 128), (V2, 256)])
+def test_tail_split_covers_k_once(shape, variant, tile_n):
+    M, N, K = shape
+    info, sched = plan_and_schedule(M, N, K, bg.make_flags(variant, tile_n, tail_split=True), c_dtype=bg.BF16)
+    check_dense(info, sched, M, N, K)
+    if info["split"] > 1:
+        assert (sched[:, SLICE] >= 0).any() and info["workspace_bytes"] > 0
+        # the slices of a tile run in the same round of their CTAs: nobody waits for a CTA that is still busy elsewhere
+        pos = {}
+        for c in np.unique(sched[:, CTA]):
+            for k, row in enumerate(np.flatnonzero(sched[:, CTA] == c)):
+                pos[row] = k
+        for key in {tuple(it[[BATCH, ROW, COL]]) for it in sched if it[SLICE] >= 0}:
+            rows = [r for r in range(len(sched)) if tuple(sched[r, [BATCH, ROW, COL]]) == key]
+            assert len({pos[r] for r in rows}) == 1
+
+
+@pytest.mark.parametrize("a_tri,b_tri,d_tri", [(1, 0, 0), (2, 0, 0), (0, 1, 0), (0, 2, 0), (0, 0, 1), (0, 0, 2), (1, 1, 1), (2, 2, 2),
+                                               (1, 0, 2), (2, 1, 0)])
+@pytest.mark.parametrize("shape", [(512, 264, 512), (1000, 136, 200), (300, 264, 1000), (2048, 2048, 2048), (4100, 4104, 4104),
+                                   (600, 2000, 520)], ids=lambda s: "x".join(map(str, s)))
+def test_structured_problems(shape, a_tri, b_tri, d_tri):
+    M, N, K = shape
+    for variant, tile_n, batch in ((0, 0, 1), (V1, 128, 2), (V2, 128, 1), (V2, 256, 3), (V1, 64, 1)):
+        fl = bg.make_flags(variant, tile_n, a_lower=a_tri == 1, a_upper=a_tri == 2, d_lower=d_tri == 1, d_upper=d_tri == 2)
+        info, sched = plan_and_schedule(M, N, K, fl, structure=b_tri, batch=batch)
+        check_dense(info, sched, M, N, K, batch, d_tri, a_tri, b_tri)
+        # dealt ahead of time by work: no CTA carries more than the mean plus one tile's worth of K stages
+        # (one matrix: the deal is made per matrix and repeated for every matrix of a batch)
+        if batch == 1:
+            work = np.zeros(info["grid"] // info["cluster_size"])
+            np.add.at(work, sched[:, CTA], sched[:, K1] - sched[:, K0] + 1)
+            assert work.max() <= work.mean() + (sched[:, K1] - sched[:, K0]).max() + 1
+
+
+@pytest.mark.parametrize("short", [1, 8, 16, 33, 48, 64])
+@pytest.mark.parametrize("long_,K", [(128, 64), (256, 4096), (1864, 2136), (4096, 4096), (28672, 8192), (28672, 1024), (50264, 4096),
+                                     (4096, 14336), (12288, 4096), (1000, 520), (520, 66000)])
+def test_stream_k_units_once(short, long_, K):
+    for tall in (False, True):
+        M, N = (long_, short) if tall else (short, long_)
+        for kslices in (0, 1, 2, 3):
+            try:
+                info, sched = plan_and_schedule(M, N, K, bg.make_flags(VS, kslices=kslices))
+            except bg.GemmError as e:
+                assert e.status == bg.ERR_UNSUPPORTED
+                continue
+            tiles = -(-long_ // 128)
+            stages = -(-K // info["tile_k"])
+            assert info["num_tiles"] == tiles * stages and info["grid"] <= 148
+            tile_ix = sched[:, ROW] if tall else sched[:, COL]
+            assert (sched[:, COL if tall else ROW] == 0).all()
+            # CTAs in order walk the units in order: concatenating the items gives every (tile, stage) exactly once
+            units = np.concatenate([t * stages + np.arange(a, b) for t, a, b in zip(tile_ix, sched[:, K0], sched[:, K1])])
+            assert np.array_equal(units, np.arange(tiles * stages))
+            assert (np.diff(sched[:, CTA]) >= 0).all() and len(np.unique(sched[:, CTA])) == info["grid"]
+            per = np.zeros(info["grid"], int)
+            np.add.at(per, sched[:, CTA], sched[:, K1] - sched[:, K0])
+            assert per.max() - per.min() <= 1                                   # equal streaming work per SM
+            # contributors of a split tile are numbered 0, 1, 2 ... in CTA order; a whole tile has one item marked -1
+            for t in range(tiles):
+                sl = sched[tile_ix == t, SLICE]
+                assert (len(sl) == 1 and sl[0] == -1) or list(sl) == list(range(len(sl)))
+                assert len(sl) <= info["split"]

@@ -83,5 +83,12 @@ def test_noalloc_rejects_what_does_not_fit():
     with pytest.raises(bg.GemmError) as e:
         bg.gemm_skinny_run_noalloc(dense, buf.data_ptr(), buf.data_ptr(), out.data_ptr(), 0, 1.0, 0.0, 0)
     assert e.value.status == bg.ERR_UNSUPPORTED
+    # structure promises and the per-row bias are refused, as the stream-K plans refuse them (never silently ignored)
+    for kw in (dict(structure=bg.STRUCT_B_UPPER), dict(structure=bg.STRUCT_B_LOWER), dict(flags=bg.make_flags(a_lower=True)),
+               dict(flags=bg.make_flags(d_upper=True)), dict(flags=bg.make_flags(bias_per_row=True), epilogue=bg.EPI_BIAS)):
+        with pytest.raises(bg.GemmError) as e:
+            bg.gemm_skinny_run_noalloc(bg.make_desc(8, 256, 256, **kw), buf.data_ptr(), buf.data_ptr(), out.data_ptr(), out.data_ptr(),
+                                       1.0, 0.0, 0)
+        assert e.value.status == bg.ERR_UNSUPPORTED, kw
     torch.cuda.synchronize()
     assert float(out.abs().sum()) == 0.0                     # nothing was launched
