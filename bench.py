@@ -304,6 +304,26 @@ class DeviceCase:
             (" as a separate kernel" if act else "") + out_note
         return step, what
 
+    def time_isolated(self, n: int = 10):
+        """Single launches, each on an idle GPU with a flushed L2 and bracketed by its own pair of events: (median, best) in
+        seconds.  This is the situation of a launch under the profiler (nothing overlaps its set-up, caches are cold, one
+        launch never meets the power cap), so it is the event-timed counterpart of the ncu durations in profiles/; the
+        best one is also how the dense peak this pool's roofline uses was measured (best of 10 single launches)."""
+        torch = self.torch
+        flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=self.device)
+        times = []
+        for _ in range(n):
+            flush.zero_()
+            torch.cuda.synchronize()
+            time.sleep(0.002)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            self.step()
+            e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1) * 1e-3)
+        return statistics.median(times), min(times)
+
     def time_sustained(self, seconds: float, step=None, sampler_index: int = 0):
         """Back-to-back steps for at least `seconds` (after one second of the same load), timed with CUDA events on the
         launching stream while the SM clock is sampled: what the configuration sustains under the power cap."""
@@ -457,6 +477,7 @@ def run_ours(args):
     warm_launches = case.warm_launches
     # context: the vendor library on the same buffers in the same loop, and the headline held for seconds
     library = sustained = None
+    iso_med, iso_best = case.time_isolated() if args.all else (None, None)
     if args.all and world == 1:
         lib_step, lib_what = case.library_step()
         if lib_step is not None:
@@ -501,6 +522,12 @@ def run_ours(args):
         "roofline": roofline_for(w, key, sec, peaks, peak_kind),
     }
     out["roofline"]["frac_of_sustained_peak"] = round(metric_value(w, sec) / peaks["bf16_tflops_sustained"], 4)
+    if iso_med is not None:
+        # single isolated launches: the median is what a launch under the profiler corresponds to; the best of ten is the
+        # protocol the measured dense peak was taken with, so `frac_of_peak` compares like with like
+        out["isolated_launch"] = {"ms_median": round(iso_med * 1e3, 5), "ms_best_of_10": round(iso_best * 1e3, 5),
+                                  "best_value": round(metric_value(w, iso_best), 2), "unit": "TFLOP/s",
+                                  "best_frac_of_peak": round(roofline_for(w, key, iso_best, peaks, peak_kind)["frac"], 4)}
     if library is not None:
         out["library_reference"] = library
     if sustained is not None:
@@ -514,6 +541,7 @@ def run_ours(args):
             if k2 == key:
                 measured.append({"config": k2, "workload": w2.name, "ms_per_step": out["ms_per_step"], "tflops": out["value"] / world,
                                  "input_sets": out["config"]["input_sets"], "warmup_launches_actual": warm_launches,
+                                 "ms_isolated_launch": None if iso_med is None else round(iso_med * 1e3, 5),
                                  "roofline": out["roofline"],
                                  "library_reference_ms_per_step": None if library is None else library["ms_per_step"]})
                 continue
@@ -525,6 +553,7 @@ def run_ours(args):
                    "tflops": round(metric_value(w2, s2), 2), "gbs": round(w2.min_bytes / s2 / 1e9, 1),
                    "input_sets": c2.nsets, "warmup_launches_actual": c2.warm_launches, "plan": c2.plan.info,
                    "roofline": roofline_for(w2, k2, s2, peaks, peak_kind)}
+            row["ms_isolated_launch"] = round(c2.time_isolated()[0] * 1e3, 5)
             if world == 1:
                 lib_step, lib_what = c2.library_step()
                 if lib_step is not None:     # the vendor library on the same buffers, same loop (context)
