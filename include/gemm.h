@@ -137,6 +137,12 @@ typedef enum {
  * that D comes out symmetric (every element beyond the diagonal holds the bits of its mirror image; the diagonal and
  * the wanted triangle are those of the product).  A second, bandwidth-bound kernel on the same stream, per batch. */
 #define GEMM_STRUCT_D_MIRROR 0x4u
+/* gemm_desc_t.options.  GEMM_OPT_STREAMK_WORKSPACE: a stream-K plan hands its partial tiles over through the workspace
+ * even where the CTAs of each output tile could be launched as a thread-block cluster and add them up in shared memory
+ * (the default wherever all clusters fit on the device at once; it needs no workspace and is several microseconds
+ * faster on mid-sized problems).  Results are bit-identical either way.  For callers that want no cluster launches,
+ * and for tests. */
+#define GEMM_OPT_STREAMK_WORKSPACE 0x1u
 #define GEMM_FLAG_BIAS_PER_ROW 0x1u         /* the bias is fp32[M], one value per output row (default: fp32[N], one per
                                               column); not a tuning knob: it changes what is computed */
 #define GEMM_FLAG_NO_EARLY_LAUNCH 0x4u       /* launch without programmatic dependent launch (default: the kernel may be
@@ -160,7 +166,7 @@ typedef struct {
   int32_t epilogue;           /* gemm_epilogue_t */
   int64_t stride_a, stride_b, stride_c; /* elements between consecutive matrices; ignored when batch_count == 1 */
   uint32_t structure;         /* GEMM_STRUCT_*: further structure promises (flags has no bit left); 0 = none */
-  uint32_t reserved;          /* must be 0 */
+  uint32_t options;           /* GEMM_OPT_*: 0 = none; unknown bits are an error */
 } gemm_desc_t;
 
 typedef struct {

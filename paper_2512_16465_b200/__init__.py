@@ -22,6 +22,7 @@ OP_N, OP_T = 0, 1
 (EPI_NONE, EPI_BIAS, EPI_RELU, EPI_BIAS_RELU, EPI_GELU_ERF, EPI_BIAS_GELU_ERF, EPI_GELU_TANH, EPI_BIAS_GELU_TANH,
  EPI_SILU, EPI_BIAS_SILU) = range(10)
 STRUCT_B_LOWER, STRUCT_B_UPPER, STRUCT_D_MIRROR = 0x1, 0x2, 0x4     # gemm_desc_t.structure
+OPT_STREAMK_WORKSPACE = 0x1                                          # gemm_desc_t.options
 VARIANT_AUTO, VARIANT_DENSE_1CTA, VARIANT_DENSE_2CTA, VARIANT_SKINNY_STREAMK, VARIANT_DENSE_2CTA_WIDE = 0, 1, 2, 3, 4
 REGIME_NAMES = {0: "memory-bound", 1: "middle-zone", 2: "compute-bound"}
 FLAG_DEBUG_STALL = 0x80000000
@@ -44,7 +45,7 @@ class Desc(ctypes.Structure):
                 ("lda", ctypes.c_int64), ("ldb", ctypes.c_int64), ("ldc", ctypes.c_int64),
                 ("batch_count", ctypes.c_int32), ("epilogue", ctypes.c_int32),
                 ("stride_a", ctypes.c_int64), ("stride_b", ctypes.c_int64), ("stride_c", ctypes.c_int64),
-                ("structure", ctypes.c_uint32), ("reserved", ctypes.c_uint32)]
+                ("structure", ctypes.c_uint32), ("options", ctypes.c_uint32)]
 
 
 class Info(ctypes.Structure):
@@ -156,8 +157,9 @@ def make_flags(variant: int = 0, tile_n: int = 0, raster: int = 0, stages: int =
 
 
 def make_desc(M, N, K, transa=OP_N, transb=OP_T, ab_dtype=BF16, c_dtype=F32, lda=0, ldb=0, ldc=0, batch=1,
-              stride_a=0, stride_b=0, stride_c=0, epilogue=EPI_NONE, flags=0, structure=0) -> Desc:
-    """Build a ``gemm_desc_t``; zero leading dimensions / strides mean "tight"; ``structure`` takes ``STRUCT_*`` bits."""
+              stride_a=0, stride_b=0, stride_c=0, epilogue=EPI_NONE, flags=0, structure=0, options=0) -> Desc:
+    """Build a ``gemm_desc_t``; zero leading dimensions / strides mean "tight"; ``structure`` takes ``STRUCT_*`` bits,
+    ``options`` ``OPT_*`` bits."""
     lda = lda or (M if transa else K)
     ldb = ldb or (K if transb else N)
     ldc = ldc or N
@@ -165,7 +167,7 @@ def make_desc(M, N, K, transa=OP_N, transb=OP_T, ab_dtype=BF16, c_dtype=F32, lda
     stride_b = stride_b or (N if transb else K) * ldb
     stride_c = stride_c or M * ldc
     return Desc(ctypes.sizeof(Desc), flags, M, N, K, transa, transb, ab_dtype, c_dtype, lda, ldb, ldc, batch, epilogue,
-                stride_a, stride_b, stride_c, structure, 0)
+                stride_a, stride_b, stride_c, structure, options)
 
 
 # ----------------------------------------------------------------------- C-named calls

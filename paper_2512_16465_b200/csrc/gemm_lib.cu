@@ -86,8 +86,12 @@ bool encode_map(CUtensorMap* m, int dtype, const void* base, uint64_t inner, uin
   cuuint64_t strides[2] = {ld * eb, (batch > 1 ? batch_stride : rows * ld) * eb};
   cuuint32_t box[3] = {box_inner, box_rows, 1};
   cuuint32_t estr[3] = {1, 1, 1};
+  // L2 fetches in 256-byte units only when the rows start on 128-byte lines: with any other pitch seven of eight box
+  // rows straddle two lines, and promoting each straddled piece to 256 bytes over-fetches (measured on
+  // 4100 x 4104 x 4104: 164 -> 144 us without promotion; no difference on aligned pitches)
+  const CUtensorMapL2promotion promotion = (ld * eb) % 128 == 0 ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_NONE;
   CUresult r = fn(m, tm_dtype(dtype), 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                  CU_TENSOR_MAP_SWIZZLE_128B, promotion, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
     char buf[64];
     snprintf(buf, sizeof buf, "CUresult %d", static_cast<int>(r));
@@ -214,7 +218,7 @@ gemm_status_t validate(const gemm_desc_t* d) {
   if (d->epilogue < GEMM_EPI_NONE || d->epilogue > GEMM_EPI_BIAS_SILU) return GEMM_ERR_INVALID_ARG;
   if ((d->flags & GEMM_FLAG_A_LOWER) && (d->flags & GEMM_FLAG_A_UPPER)) return GEMM_ERR_INVALID_ARG;
   if ((d->flags & GEMM_FLAG_D_LOWER) && (d->flags & GEMM_FLAG_D_UPPER)) return GEMM_ERR_INVALID_ARG;
-  if ((d->structure & ~(GEMM_STRUCT_B_LOWER | GEMM_STRUCT_B_UPPER | GEMM_STRUCT_D_MIRROR)) || d->reserved != 0) return GEMM_ERR_INVALID_ARG;
+  if ((d->structure & ~(GEMM_STRUCT_B_LOWER | GEMM_STRUCT_B_UPPER | GEMM_STRUCT_D_MIRROR)) || (d->options & ~GEMM_OPT_STREAMK_WORKSPACE)) return GEMM_ERR_INVALID_ARG;
   if ((d->structure & GEMM_STRUCT_D_MIRROR) && (!(d->flags & (GEMM_FLAG_D_LOWER | GEMM_FLAG_D_UPPER)) || d->M != d->N || d->batch_count > 65535))
     return GEMM_ERR_INVALID_ARG;  // a triangle to copy from, and a square D
   if ((d->structure & GEMM_STRUCT_B_LOWER) && (d->structure & GEMM_STRUCT_B_UPPER)) return GEMM_ERR_INVALID_ARG;
@@ -689,6 +693,49 @@ gemm_status_t plan_wide(gemm_plan_s* pl, int forced_raster, int forced_stages) {
   return GEMM_OK;
 }
 
+// How many clusters of c = 2 ... 8 CTAs of the stream-K kernel (one CTA per SM: it takes nearly all shared memory) the
+// device holds at once, asked of the occupancy calculator once per device.  A cluster must fit inside one GPC, so for
+// some sizes this is fewer than SM count / c, and a plan whose clusters do not all fit would run in two waves.
+const int* skinny_cluster_room(int device) {
+  static int room[kMaxDevices][9];
+  static bool known[kMaxDevices];
+  static std::mutex mu;
+  if (device < 0 || device >= kMaxDevices) return nullptr;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!known[device]) {
+    const void* kern = reinterpret_cast<const void*>(skinny_gemm_kernel<false, true>);
+    if (ensure_dynamic_smem(kern, kSlotSkinnyCluster, device, kMaxSmemOptin) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return nullptr;
+    }
+    for (int c = 2; c <= 8; ++c) {
+      cudaLaunchConfig_t cfg;
+      memset(&cfg, 0, sizeof cfg);
+      cfg.gridDim = dim3(c * 16, 1, 1);
+      cfg.blockDim = dim3(kSkinnyThreads, 1, 1);
+      cfg.dynamicSmemBytes = kMaxSmemOptin;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = c;
+      attr[0].val.clusterDim.y = 1;
+      attr[0].val.clusterDim.z = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = 1;
+      int n = 0;
+      if (cudaOccupancyMaxActiveClusters(&n, skinny_gemm_kernel<false, true>, &cfg) != cudaSuccess) {
+        (void)cudaGetLastError();
+        n = 0;  // unknown: no clusters of this size
+      }
+      room[device][c] = n;
+    }
+    known[device] = true;
+    if (getenv("B200GEMM_LOG"))
+      fprintf(stderr, "[b200gemm] stream-K clusters that fit at once, sizes 2..8: %d %d %d %d %d %d %d\n", room[device][2], room[device][3],
+              room[device][4], room[device][5], room[device][6], room[device][7], room[device][8]);
+  }
+  return room[device];
+}
+
 gemm_status_t plan_skinny(gemm_plan_s* pl, int forced_stages, int forced_atoms) {
   const gemm_desc_t& d = pl->d;
   if (d.transa != GEMM_OP_N || d.transb != GEMM_OP_T) return GEMM_ERR_UNSUPPORTED;  // both operands K-contiguous
@@ -700,7 +747,8 @@ gemm_status_t plan_skinny(gemm_plan_s* pl, int forced_stages, int forced_atoms) 
   const int small_extent = static_cast<int>(pl->skinny_tall ? d.N : d.M), big_extent = static_cast<int>(pl->skinny_tall ? d.M : d.N);
   if (forced_atoms > 3) return GEMM_ERR_UNSUPPORTED;
   if (!skinny_make_plan(&s, small_extent, big_extent, static_cast<int>(d.K), pl->sm_count, forced_stages, kMaxSmemOptin, forced_atoms,
-                        kblk_of(d.ab_dtype), /*align=*/true))
+                        kblk_of(d.ab_dtype), /*align=*/true, (pl->has_device && pl->arch_ok) ? skinny_cluster_room(pl->device) : nullptr,
+                        /*clusters=*/!(d.options & GEMM_OPT_STREAMK_WORKSPACE)))
     return GEMM_ERR_UNSUPPORTED;
   pl->variant = GEMM_VARIANT_SKINNY_STREAMK;
   pl->cg = 1;
@@ -714,7 +762,7 @@ gemm_status_t plan_skinny(gemm_plan_s* pl, int forced_stages, int forced_atoms) 
   info.tile_n = s.m_pad;
   info.tile_k = s.kblk * s.atoms;
   info.stages = s.stages;
-  info.cluster_size = 1;
+  info.cluster_size = s.cluster;  // > 1: the CTAs of one output tile form a cluster and hand over through shared memory
   info.grid = s.grid;
   info.raster_group = 1;
   info.split = s.max_contributors;
@@ -992,12 +1040,13 @@ gemm_status_t gemm_plan_schedule(gemm_plan_t plan, gemm_work_item_t* items, size
   if (plan->variant == GEMM_VARIANT_SKINNY_STREAMK) {
     const SkinnyPlan& s = plan->skinny;
     for (int c = 0; c < s.grid; ++c) {
-      const int u_end = sk_begin(c + 1, s.units_q, s.units_r);
-      for (int u = sk_begin(c, s.units_q, s.units_r); u < u_end;) {  // one item per tile this CTA's range touches
+      const int u_end = sk_cta_begin(s, c + 1);
+      for (int u = sk_cta_begin(s, c); u < u_end;) {  // one item per tile this CTA's range touches
         const int tile = u / s.kbs, tile_u0 = tile * s.kbs;
         const int seg_end = std::min(u_end, tile_u0 + s.kbs);
         const bool whole = u == tile_u0 && seg_end == tile_u0 + s.kbs;
-        const int slice = whole ? -1 : c - sk_owner(tile_u0, s.units_q, s.units_r);  // position among the tile's contributors
+        // position among the tile's contributors (cluster mode: the rank in the cluster)
+        const int slice = whole ? -1 : (s.cluster > 1 ? c % s.cluster : c - sk_owner(tile_u0, s.units_q, s.units_r));
         emit(c, 0, plan->skinny_tall ? tile : 0, plan->skinny_tall ? 0 : tile, u - tile_u0, seg_end - tile_u0, slice);
         u = seg_end;
       }

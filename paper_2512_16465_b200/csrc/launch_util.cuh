@@ -7,7 +7,7 @@
 namespace b200 {
 
 constexpr int kMaxDevices = 64;
-enum KernelSlot { kSlotDense11 = 0, kSlotDense12, kSlotDense21, kSlotDense22, kSlotDenseSplit11, kSlotDenseSplit12, kSlotDenseSplit21, kSlotDenseSplit22, kSlotWide, kSlotWideFp8, kSlotSkinny, kSlotSkinnyTall, kNumKernelSlots };
+enum KernelSlot { kSlotDense11 = 0, kSlotDense12, kSlotDense21, kSlotDense22, kSlotDenseSplit11, kSlotDenseSplit12, kSlotDenseSplit21, kSlotDenseSplit22, kSlotWide, kSlotWideFp8, kSlotSkinny, kSlotSkinnyTall, kSlotSkinnyCluster, kSlotSkinnyTallCluster, kNumKernelSlots };
 
 // Opt a kernel in to `bytes` of dynamic shared memory on the current device.  The attribute is per kernel and per
 // device, and only ever needs to grow, so the largest value set so far is remembered per (kernel, device).

@@ -17,6 +17,13 @@
 //     reads as "no arrivals yet".  Runs of one plan on different workspaces therefore share nothing but the
 //     status word and may overlap.
 //
+//   * cluster mode (kCluster): when the plan gives every output tile to exactly c CTAs (c <= 8 dividing the tile's work
+//     units), those c CTAs are launched as one thread-block cluster and the hand-over goes through shared memory instead:
+//     each CTA parks its partial tile in its own (by then idle) ring memory, the cluster meets at a hardware barrier, and
+//     every CTA finishes the 16-row chunks of the short extent that fall to its rank, adding the c partials in rank order
+//     with loads from the peers' shared memory.  No workspace, no arrival word, no trip through L2; the order of the
+//     additions is fixed, so results are bit-identical to the workspace path's.
+//
 // The same kernel serves the mirrored case, a tall output with a handful of columns (N <= 64 < M, kTall): the long
 // operand A[M x K] then takes W's place and B[N x K] takes X's; only the addressing of C, D and the bias differs.
 // Below, "big" is the long output extent (128 per tile, on the TMEM lanes) and "small" the short one.
@@ -50,6 +57,7 @@ struct SkinnyPlan {
   int stages;
   int stage_bytes;       // atoms x (16 KB of W + m_pad * 128 bytes of X)
   int smem_bytes;
+  int cluster;           // > 1: CTAs per output tile, launched as one thread-block cluster (hand-over through shared memory)
   int max_contributors;  // upper bound on CTAs touching one tile
   size_t counters_bytes; // arrival counters at the head of the workspace: n_tiles x u64, padded to 256 bytes
   size_t workspace_bytes;  // partial tiles behind them: grid * 2 slots of [m_pad][128] floats
@@ -62,9 +70,11 @@ __host__ __device__ inline int sk_owner(int u, int q, int r) {
   return u < head ? u / (q + 1) : r + (u - head) / q;
 }
 
+// max_clusters (may be null): max_clusters[c] = clusters of c CTAs of this kernel that the device holds at once, c = 2 ... 8
+// (without it: SM count / c, which real GPUs undercut for some sizes because a cluster must sit inside one GPC).
 // M is the small output extent and N the big one (for a tall problem the caller passes them swapped).
 inline bool skinny_make_plan(SkinnyPlan* s, int M, int N, int K, int sm_count, int forced_stages, int max_smem, int forced_atoms = 0,
-                             int kblk = kBlockK, bool align = false) {
+                             int kblk = kBlockK, bool align = false, const int* max_clusters = nullptr, bool clusters = true) {
   if (M < 1 || M > kSkinnyMaxM) return false;
   s->m_pad = ((M + 15) / 16) * 16;
   s->n_tiles = (N + kSkinnyTileN - 1) / kSkinnyTileN;
@@ -80,31 +90,49 @@ inline bool skinny_make_plan(SkinnyPlan* s, int M, int N, int K, int sm_count, i
   s->total_units = static_cast<long long>(s->n_tiles) * s->kbs;
   if (s->total_units > 0x7fffffffll) return false;
   s->grid = static_cast<int>(s->total_units < sm_count ? s->total_units : sm_count);
-  // CTA ranges that line up with the tiles save most of the hand-over of partial tiles, which on mid-sized problems
-  // costs as much as the streaming itself.  Best of all is one whole tile per CTA (no partial tile at all) when that
-  // keeps at least two thirds of the SMs busy, or half of them on a mid-sized problem; next, c >= 3 CTAs per tile with c dividing the tile's units, so that no CTA
-  // contributes to two tiles, when that keeps four fifths busy (with two CTAs per tile the smaller grid costs what
-  // the alignment saves); last, several whole tiles per CTA on problems of a few dozen units per CTA.  Measured on
-  // sixty shapes with short extents 8 ... 64: 5 to 23 % faster wherever a rule applies (64 x 4096 x 4096: 22.3 ->
-  // 17.7 us on 128 CTAs, 64 x 11008 x 4096: 30.9 -> 24.5 us on 86), unchanged elsewhere.
-  if (align && s->total_units >= sm_count) {
+  // Grids that line up with the tiles.  The hand-over of partial tiles through the workspace costs a mid-sized problem as
+  // much as the streaming itself (for a short extent of 64, 12 us of tail behind 7 us of streaming), so:
+  //  (1) one whole tile per CTA, no hand-over at all, when that keeps two thirds of the SMs busy;
+  //  (2) else c <= 8 CTAs per tile launched as one cluster each, the tile's units dealt to them as evenly as they go and
+  //      the partial tiles added up through shared memory (about 2 us), when all clusters fit on the device at once and
+  //      fill six tenths of it (any small problem: there the alternative is one CTA per unit);
+  //  (3) else c > 8 CTAs per tile with c dividing the tile's units (workspace path, but no CTA contributes to two tiles),
+  //      whole tiles on half of the SMs for a mid-sized problem, or several whole tiles per CTA;
+  //  (4) else equal contiguous ranges over all SMs, straddling the tiles (the large problems, whose tail does not matter).
+  // Measured against the plain rule (4) on shapes with short extents 8 ... 64: 64 x 4096 x 4096 22.3 -> 12.0 us,
+  // 64 x 8192 x 8192 36.0 -> 27.7, 64 x 4096 x 14336 34.4 -> 24.3, 8 x 4096 x 4096 13.3 -> 10.7; the large ones unchanged.
+  s->cluster = 1;
+  if (align) {
     int best = 0;
-    // (about a hundred SMs saturate the memory system, so a grid of that size streams as fast as a full one; a smaller
-    // one pays in streaming time what it saves in hand-overs once the streamed operand exceeds some 160 MB)
+    const bool small_problem = s->total_units < 2ll * sm_count;
     const double streamed_mb = static_cast<double>(s->total_units) * s->atoms * (kSkinnyTileN * 128) / 1.0e6;
-    if (s->n_tiles <= sm_count && (s->n_tiles * 100 >= sm_count * 68 || (2 * s->n_tiles >= sm_count && streamed_mb <= 160.0))) best = s->n_tiles;
-    if (!best)
-      for (int c = 3; c <= s->kbs; ++c)
+    if (s->total_units >= sm_count && s->n_tiles <= sm_count && s->n_tiles * 100 >= sm_count * 68) best = s->n_tiles;
+    if (!best && clusters)
+      for (int c = 2; c <= 8 && 2 * c <= s->kbs; ++c) {
+        const int room = max_clusters ? max_clusters[c] : sm_count / c;
+        if (s->n_tiles > room) continue;
+        if (!small_problem && s->n_tiles * c * 10 < sm_count * 6) continue;
+        if (s->n_tiles * c > best) {
+          best = s->n_tiles * c;
+          s->cluster = c;
+        }
+      }
+    if (!best && s->total_units >= sm_count) {
+      for (int c = clusters ? 9 : 3; c <= s->kbs; ++c)
         if (s->kbs % c == 0 && static_cast<long long>(s->n_tiles) * c <= sm_count && s->n_tiles * c * 5 >= sm_count * 4)
           best = best > s->n_tiles * c ? best : s->n_tiles * c;
-    if (!best && s->kbs % 2 == 0 && s->total_units / s->grid < 24 && 2 * s->n_tiles <= sm_count && 4 * s->n_tiles >= sm_count)
-      best = 2 * s->n_tiles;  // two CTAs per tile: only on the smallest problems (5120 x 5120: -6 to -13 %)
-    if (!best && s->total_units / s->grid < 64)
-      for (int t = 2; t <= s->n_tiles; ++t)
-        if (s->n_tiles % t == 0 && s->n_tiles / t <= sm_count && (s->n_tiles / t) * 5 >= sm_count * 4) {
-          best = s->n_tiles / t;
-          break;
-        }
+      // (about a hundred SMs saturate the memory system; fewer pay in streaming time what they save in hand-overs once the
+      // streamed operand exceeds some 160 MB)
+      // (the wider the short extent, the dearer the hand-over through the workspace: 12 us at 64 against 5 at 16)
+      const double whole_tiles_up_to_mb = 160.0 + (s->m_pad > 32 ? (s->m_pad - 32) * 6.0 : 0.0);
+      if (!best && s->n_tiles <= sm_count && 2 * s->n_tiles >= sm_count && streamed_mb <= whole_tiles_up_to_mb) best = s->n_tiles;
+      if (!best && s->total_units / s->grid < 64)
+        for (int t = 2; t <= s->n_tiles; ++t)
+          if (s->n_tiles % t == 0 && s->n_tiles / t <= sm_count && (s->n_tiles / t) * 5 >= sm_count * 4) {
+            best = s->n_tiles / t;
+            break;
+          }
+    }
     if (best) s->grid = best;
   }
   s->units_q = static_cast<int>(s->total_units / s->grid);
@@ -121,7 +149,18 @@ inline bool skinny_make_plan(SkinnyPlan* s, int M, int N, int K, int sm_count, i
   s->max_contributors = (s->kbs + per_cta - 1) / per_cta + 1;
   s->counters_bytes = (static_cast<size_t>(s->n_tiles) * 8 + 255) / 256 * 256;
   s->workspace_bytes = static_cast<size_t>(s->grid) * 2 * kSkinnyTileN * s->m_pad * 4;
+  if (s->cluster > 1) s->counters_bytes = s->workspace_bytes = 0;  // nothing leaves the cluster
   return true;
+}
+
+// First work unit of CTA `cta` (cta = grid gives the total).  Cluster mode: the c CTAs of a cluster share out the units of
+// their tile; otherwise all units are cut into `grid` equal contiguous ranges.
+__host__ __device__ inline int sk_cta_begin(const SkinnyPlan& s, int cta) {
+  if (s.cluster > 1) {
+    const int tile = cta / s.cluster, rank = cta - tile * s.cluster;
+    return tile * s.kbs + sk_begin(rank, s.kbs / s.cluster, s.kbs % s.cluster);
+  }
+  return sk_begin(cta, s.units_q, s.units_r);
 }
 
 struct SkinnyParams {
@@ -248,7 +287,7 @@ __device__ __forceinline__ void sk_finish16(const SkinnyParams& p, int s0, int b
   }
 }
 
-template <bool kTall>
+template <bool kTall, bool kCluster = false>
 __global__ void __launch_bounds__(kSkinnyThreads, 1)
 skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, const SkinnyParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -274,8 +313,8 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
   const WaitCtx w{s_abort, p.status, p.timeout_ns};
   // This CTA's contiguous range of work units (computed while the barriers and tensor memory are being set up).
   const int uq = sp.units_q, ur = sp.units_r;
-  const int u_begin = sk_begin(static_cast<int>(blockIdx.x), uq, ur);
-  const int u_end = sk_begin(static_cast<int>(blockIdx.x) + 1, uq, ur);
+  const int u_begin = sk_cta_begin(sp, static_cast<int>(blockIdx.x));
+  const int u_end = sk_cta_begin(sp, static_cast<int>(blockIdx.x) + 1);
   const int tile0 = u_begin / sp.kbs;
   const int kb0 = u_begin - tile0 * sp.kbs;
   const int n_units = u_end - u_begin;
@@ -315,7 +354,9 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
   // While the status word is set (an earlier run of this plan timed out and the host has not read the word yet) no
   // run finishes split tiles: a replay of a captured launch carries the tag of the run that may have left arrivals
   // half counted.  The load is issued here and consumed only by the fix-up, long after it has landed.
-  const uint32_t stale_status = *reinterpret_cast<volatile const uint32_t*>(p.status);
+  // (Only the warps that finish tiles ask: the producer's first load must not queue behind it.)
+  uint32_t stale_status = 0u;
+  if (warp >= 2) stale_status = *reinterpret_cast<volatile const uint32_t*>(p.status);
 
   // The producer and MMA roles run warp-uniform (one elected lane issues), with the (tile, k-block) position and
   // the ring slot advanced incrementally: the single issuing thread must sustain one 18 KB stage every few hundred
@@ -401,6 +442,23 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
       done += seg_units;
       kb = 0;
       ++seg;
+    }
+  } else if constexpr (kCluster) {
+    // This CTA's one segment: the raw accumulators go to its own ring memory (every MMA that read the ring has
+    // completed once the accumulator is), laid out [short index][128 long indices] like a workspace partial.
+    const uint32_t q = warp & 3u;
+    const uint32_t n_local = q * 32u + lane;
+    if (mbar_wait_warp(tfull0, 0u, w, (3u << 8), 64u)) {
+      tc_fence_after();
+      const uint32_t t_row = tmem_base + ((q * 32u) << 16);
+      for (int c0 = 0; c0 < sp.m_pad; c0 += 16) {
+        uint32_t acc[16];
+        tmem_ld_32x16(t_row + static_cast<uint32_t>(c0), acc);
+        tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < 16; ++j) st_shared_b32(base + static_cast<uint32_t>(c0 + j) * (kSkinnyTileN * 4u) + n_local * 4u, acc[j]);
+      }
+      tc_fence_before();
     }
   } else {
     const uint32_t q = warp & 3u;
@@ -558,6 +616,40 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
     }
   }
 
+  if constexpr (kCluster) {
+    // Every thread of the cluster meets here (also after a timeout: the roles above fall through to this point), so
+    // the partial tiles of all ranks are visible cluster-wide behind the barrier.  Rank r then finishes the 16-row
+    // chunks r, r + c, ... of the short extent: the c partials are added in rank order (the order of the K ranges),
+    // read from the peers' shared memory.  C_in is requested before the wait so that its latency hides behind it.
+    const uint32_t crank = cluster_ctarank();
+    const uint32_t csize = static_cast<uint32_t>(sp.cluster);
+    const uint32_t n_local = (warp & 3u) * 32u + lane;
+    const int n = tile0 * kSkinnyTileN + static_cast<int>(n_local);
+    const bool finisher = warp >= 2 && n < big_extent;
+    float cin[16];
+    cluster_arrive();
+    if (finisher && static_cast<int>(crank) * 16 < small_extent) sk_load_cin16<kTall>(p, static_cast<int>(crank) * 16, n, cin);
+    cluster_wait();
+    if (finisher && *s_abort == 0u && stale_status == 0u) {
+      for (int m0 = static_cast<int>(crank) * 16; m0 < small_extent; m0 += static_cast<int>(csize) * 16) {
+        if (m0 != static_cast<int>(crank) * 16) sk_load_cin16<kTall>(p, m0, n, cin);
+        float sum[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) sum[j] = 0.0f;
+        for (uint32_t r = 0; r < csize; ++r) {
+          const uint32_t peer = mapa(base + static_cast<uint32_t>(m0) * (kSkinnyTileN * 4u) + n_local * 4u, r);
+          float v[16];
+#pragma unroll
+          for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(ld_shared_cluster_b32(peer + static_cast<uint32_t>(j) * (kSkinnyTileN * 4u)));
+#pragma unroll
+          for (int j = 0; j < 16; ++j) sum[j] += v[j];
+        }
+        sk_finish16<kTall>(p, m0, n, sum, cin);
+      }
+    }
+    cluster_arrive();  // nobody's shared memory may go away while a peer still reads it
+    cluster_wait();
+  }
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
@@ -570,8 +662,11 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
 // `tall` selects the mirrored addressing (tW then maps A, tX maps B).
 inline int skinny_launch(const SkinnyParams& p, const CUtensorMap& tW, const CUtensorMap& tX, int device, cudaStream_t stream,
                          char* err, size_t err_len, bool tall, bool early_launch) {
-  cudaError_t e = tall ? ensure_dynamic_smem(reinterpret_cast<const void*>(skinny_gemm_kernel<true>), kSlotSkinnyTall, device, p.plan.smem_bytes)
-                       : ensure_dynamic_smem(reinterpret_cast<const void*>(skinny_gemm_kernel<false>), kSlotSkinny, device, p.plan.smem_bytes);
+  const bool cluster = p.plan.cluster > 1;
+  const void* kern = tall ? (cluster ? reinterpret_cast<const void*>(skinny_gemm_kernel<true, true>) : reinterpret_cast<const void*>(skinny_gemm_kernel<true, false>))
+                          : (cluster ? reinterpret_cast<const void*>(skinny_gemm_kernel<false, true>) : reinterpret_cast<const void*>(skinny_gemm_kernel<false, false>));
+  const KernelSlot slot = tall ? (cluster ? kSlotSkinnyTallCluster : kSlotSkinnyTall) : (cluster ? kSlotSkinnyCluster : kSlotSkinny);
+  cudaError_t e = ensure_dynamic_smem(kern, slot, device, p.plan.smem_bytes);
   if (e == cudaSuccess) {
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);
@@ -579,12 +674,24 @@ inline int skinny_launch(const SkinnyParams& p, const CUtensorMap& tW, const CUt
     cfg.blockDim = dim3(kSkinnyThreads, 1, 1);
     cfg.dynamicSmemBytes = p.plan.smem_bytes;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // set-up may overlap the previous kernel's tail
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute attr[2];
+    int na = 0;
+    if (early_launch) {
+      attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // set-up may overlap the previous kernel's tail
+      attr[na].val.programmaticStreamSerializationAllowed = 1;
+      ++na;
+    }
+    if (cluster) {
+      attr[na].id = cudaLaunchAttributeClusterDimension;
+      attr[na].val.clusterDim.x = p.plan.cluster;
+      attr[na].val.clusterDim.y = 1;
+      attr[na].val.clusterDim.z = 1;
+      ++na;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = early_launch ? 1 : 0;
-    e = tall ? cudaLaunchKernelEx(&cfg, skinny_gemm_kernel<true>, tW, tX, p) : cudaLaunchKernelEx(&cfg, skinny_gemm_kernel<false>, tW, tX, p);
+    cfg.numAttrs = na;
+    if (tall) e = cluster ? cudaLaunchKernelEx(&cfg, skinny_gemm_kernel<true, true>, tW, tX, p) : cudaLaunchKernelEx(&cfg, skinny_gemm_kernel<true, false>, tW, tX, p);
+    else e = cluster ? cudaLaunchKernelEx(&cfg, skinny_gemm_kernel<false, true>, tW, tX, p) : cudaLaunchKernelEx(&cfg, skinny_gemm_kernel<false, false>, tW, tX, p);
   }
   if (e != cudaSuccess) {
     snprintf(err, err_len, "skinny launch: %s", cudaGetErrorName(e));

@@ -66,12 +66,12 @@ def to_host_bits(t: torch.Tensor, dtype: int) -> np.ndarray:
     return t.view(torch.int16).cpu().numpy().view(np.uint16)
 
 
-def desc_of(w: wl.Workload, flags: int = 0, c_dtype=None) -> bg.Desc:
+def desc_of(w: wl.Workload, flags: int = 0, c_dtype=None, options: int = 0) -> bg.Desc:
     cd = w.c_dtype if c_dtype is None else c_dtype
     return bg.make_desc(w.M, w.N, w.K, w.transa, w.transb, w.ab_dtype, cd, w.lda, w.ldb, w.ldc, w.batch,
                         w.stride_a, w.stride_b, w.stride_c, w.epilogue, flags | bg.make_flags(bias_per_row=w.bias_per_row, a_lower=w.a_tri == 1, a_upper=w.a_tri == 2,
                                                                                            d_lower=w.d_tri == 1, d_upper=w.d_tri == 2),
-                        structure=w.b_tri | (4 if w.d_mirror else 0))
+                        structure=w.b_tri | (4 if w.d_mirror else 0), options=options)
 
 
 def problem_of(w: wl.Workload, c_dtype=None) -> oracle.Problem:
@@ -106,11 +106,11 @@ def poison_operand_padding(arr: np.ndarray, dtype: int, rows: int, row_len: int,
     return out
 
 
-def run_gpu(w: wl.Workload, inputs: dict, flags: int = 0, c_dtype=None, poison: bool = True, repeats: int = 1):
+def run_gpu(w: wl.Workload, inputs: dict, flags: int = 0, c_dtype=None, poison: bool = True, repeats: int = 1, options: int = 0):
     """Run the workload through the binding; returns (host bit array of the whole C buffer, plan info).  The device
     copies of A and B carry NaN in every padding element (the oracle sees the plain inputs)."""
     cd = w.c_dtype if c_dtype is None else c_dtype
-    plan = bg.Plan(desc_of(w, flags, cd))
+    plan = bg.Plan(desc_of(w, flags, cd, options))
     try:
         a_rows, a_len = (w.K, w.M) if w.transa else (w.M, w.K)
         b_rows, b_len = (w.N, w.K) if w.transb else (w.K, w.N)
@@ -256,11 +256,11 @@ def assert_padding_untouched(w: wl.Workload, inputs: dict, cbits: np.ndarray, c_
         assert np.all(np.isnan(oracle.decode(cbits[mask].copy(), cd))), f"{w.name}: bytes outside D were overwritten"
 
 
-def check_workload(w: wl.Workload, flags: int = 0, exact: bool = False, c_dtype=None, repeats: int = 1, inputs=None):
+def check_workload(w: wl.Workload, flags: int = 0, exact: bool = False, c_dtype=None, repeats: int = 1, inputs=None, options: int = 0):
     """Run + compare.  exact=True additionally requires bit equality with the rounded oracle
     (for integer-valued inputs whose every partial sum is exactly representable)."""
     inputs = wl.make_inputs(w) if inputs is None else inputs
-    cbits, info = run_gpu(w, inputs, flags, c_dtype, repeats=repeats)
+    cbits, info = run_gpu(w, inputs, flags, c_dtype, repeats=repeats, options=options)
     reports = check_blocks(w, inputs, cbits, default_blocks(w), c_dtype)
     assert_reports(reports, what=w.name)
     assert_padding_untouched(w, inputs, cbits, c_dtype)

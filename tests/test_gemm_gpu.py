@@ -98,6 +98,16 @@ EXACT_CASES = [
     ("skinny_one_slice_stages", 8, 256, 4096, {}, dict(variant=VS, kslices=1)),
     ("skinny_three_slice_stages", 8, 384, 1100 - 4, {}, dict(variant=VS, kslices=3)),
     ("skinny_k_slice_past_the_end", 8, 256, 1080, {}, dict(variant=VS)),
+    # stream-K with exactly c CTAs per output tile: the c CTAs form a cluster and hand over through shared memory
+    ("cluster_4_m8", 8, 4096, 4096, {}, dict(variant=VS)),
+    ("cluster_4_m64_f16_beta", 64, 4096, 4096, dict(ab=wl.F16, cd=wl.F16, alpha=0.5, beta=1.0), dict(variant=VS)),
+    ("cluster_8_m16_bias_bf16", 16, 2048, 8192, dict(cd=wl.BF16, epi=bg.EPI_BIAS), dict(variant=VS)),
+    ("cluster_4_ragged_m33", 33, 4000, 4608, dict(beta=1.0, epi=bg.EPI_BIAS_RELU), dict(variant=VS)),
+    ("cluster_4_tall_n8", 4096, 8, 4096, dict(beta=1.0), dict(variant=VS)),
+    ("cluster_4_tall_n48_padded", 4000, 48, 4608, dict(cd=wl.BF16, ldc=56, epi=bg.EPI_BIAS, bias_per_row=True), dict(variant=VS)),
+    ("cluster_4_fp8", 8, 4096, 8192, dict(ab=wl.FP8_E4M3), dict(variant=VS)),
+    ("cluster_auto_plan", 64, 4096, 4096, dict(cd=wl.BF16), dict()),
+    ("cluster_no_early_launch", 8, 4096, 4096, dict(beta=1.0), dict(variant=VS, no_early_launch=True)),
     ("no_early_launch_1cta", 264, 328, 200, {}, dict(variant=V1, tile_n=128, no_early_launch=True)),
     ("no_early_launch_skinny", 8, 256, 4096, dict(beta=1.0), dict(variant=VS, no_early_launch=True)),
     # triangular op(A): K ranges that can only contribute zeros are skipped
@@ -204,7 +214,11 @@ EXACT_CASES = [
 def test_exact_integer_inputs(case):
     name, M, N, K, kw, fl = case
     w = int_workload(name, M, N, K, **kw)
-    H.check_workload(w, bg.make_flags(**fl), exact=True, repeats=2)
+    _, info = H.check_workload(w, bg.make_flags(**fl), exact=True, repeats=2)
+    if info["variant"] == VS and info["cluster_size"] > 1:
+        # the plan handed the partial tiles over inside clusters: the same problem through the workspace as well
+        _, info = H.check_workload(w, bg.make_flags(**fl), exact=True, repeats=2, options=bg.OPT_STREAMK_WORKSPACE)
+        assert info["cluster_size"] == 1
 
 
 def _random_case(seed):
@@ -274,7 +288,8 @@ def test_random_problems(seed):
         M, N, K, kw, fl = _random_case(seed + 100000 * attempt)
         w = int_workload(f"random_{seed}_{attempt}", M, N, K, **kw)
         try:
-            H.check_workload(w, bg.make_flags(**fl), exact=kw["epi"] <= 3, repeats=2)
+            # (stream-K draws alternate between the hand-over inside clusters, where the plan would use it, and the workspace)
+            H.check_workload(w, bg.make_flags(**fl), exact=kw["epi"] <= 3, repeats=2, options=bg.OPT_STREAMK_WORKSPACE if seed % 2 else 0)
             return
         except bg.GemmError as e:
             assert e.status == bg.ERR_UNSUPPORTED, (M, N, K, kw, fl)
@@ -305,7 +320,7 @@ def test_random_large_problems(seed):
             kw["batch"] = 1
         w = int_workload(f"random_large_{seed}_{attempt}", M, N, K, sample_rows=48, sample_cols=48, **kw)
         try:
-            H.check_workload(w, bg.make_flags(**fl), exact=kw["epi"] <= 3)
+            H.check_workload(w, bg.make_flags(**fl), exact=kw["epi"] <= 3, options=bg.OPT_STREAMK_WORKSPACE if seed % 2 else 0)
             return
         except bg.GemmError as e:
             assert e.status == bg.ERR_UNSUPPORTED, (M, N, K, kw, fl)
@@ -474,7 +489,7 @@ def test_run_argument_errors_launch_nothing():
         bg.gemm_run(plan.handle, 0, B.data_ptr(), C.data_ptr(), bias.data_ptr(), 1.0, 0.0, 0, 0, s)
     assert e.value.status == bg.ERR_NULL
     plan.close()
-    sk = bg.Plan(bg.make_desc(8, 1024, 1024, flags=bg.make_flags(VS)))
+    sk = bg.Plan(bg.make_desc(8, 1024, 1024, flags=bg.make_flags(VS), options=bg.OPT_STREAMK_WORKSPACE))
     assert sk.workspace_bytes > 0
     X = torch.zeros(8 * 1024, dtype=torch.bfloat16, device="cuda")
     Wt = torch.zeros(1024 * 1024, dtype=torch.bfloat16, device="cuda")
@@ -551,7 +566,7 @@ def test_one_plan_on_two_streams_with_a_workspace_per_stream():
     A dense plan without a workspace, a stream-K plan and a dense plan with a tail split, each launched alternately on
     two streams."""
     wd = int_workload("two_streams_dense", 1024, 1024, 512, cd=wl.BF16)
-    ws = int_workload("two_streams_stream_k", 8, 4096, 4096, beta=0.0)
+    ws = int_workload("two_streams_stream_k", 8, 11000, 8200, beta=0.0)   # (CTA ranges that straddle tiles: the workspace path)
     wt = int_workload("two_streams_tail_split", 1024, 1024, 2048, cd=wl.BF16)
     streams = [torch.cuda.Stream() for _ in range(2)]
     for w, flags in ((wd, 0), (ws, 0), (wt, bg.make_flags(V2, 256, tail_split=True))):
@@ -578,8 +593,8 @@ def test_one_plan_on_two_streams_with_a_workspace_per_stream():
 def test_workspace_needs_no_initialisation(fill):
     """The hand-shake words at the head of a workspace carry a per-run tag, so whatever the memory held before -- all
     bits set, random bytes, zeros, or the words another plan of the same shape left there -- reads as "nothing yet"."""
-    cases = [(int_workload("ws_stream_k", 8, 4096, 4096, beta=1.0), 0),
-             (int_workload("ws_stream_k_m40", 40, 1000, 8200, cd=wl.BF16), 0),
+    cases = [(int_workload("ws_stream_k", 8, 11000, 8200, beta=1.0), 0),
+             (int_workload("ws_stream_k_m40", 40, 10240, 8200, cd=wl.BF16), 0),
              (int_workload("ws_tail_split", 1024, 1024, 2048, cd=wl.BF16), bg.make_flags(V2, 256, tail_split=True)),
              (int_workload("ws_long_k_auto_split", 256, 256, 16384), 0)]
     for w, flags in cases:
@@ -689,11 +704,15 @@ def test_tensor_maps_are_remembered_by_operand_address():
         plan.close()
 
 
-@pytest.mark.parametrize("variant", [V1, V2, VW, VS])
+@pytest.mark.parametrize("variant", [V1, V2, VW, VS, "stream-K through the workspace"])
 def test_bounded_wait_reports_timeout_and_context_survives(variant):
     """A producer arrival is withheld by a test flag, so a device-side wait runs into its limit; the
     kernel must return on its own, the plan must report GEMM_ERR_TIMEOUT and later work must run."""
-    w = int_workload("stall", 8 if variant == VS else 512, 512, 256 if variant != VS else 8192)  # stream-K: split tiles
+    # stream-K: split tiles, once handed over inside clusters and once through the workspace
+    w = int_workload("stall", 8, 11000, 8200) if variant == "stream-K through the workspace" else \
+        int_workload("stall", 8 if variant == VS else 512, 512, 256 if variant != VS else 8192)
+    if variant == "stream-K through the workspace":
+        variant = VS
     inputs = wl.make_inputs(w)
     tile_n = 0 if variant in (VW, VS) else 128
     plan = bg.Plan(H.desc_of(w, bg.make_flags(variant, tile_n, debug_stall=True)))
@@ -1124,8 +1143,8 @@ def test_tune_argument_errors():
         bg.gemm_tune(bg.make_desc(256, 256, 64, epilogue=bg.EPI_BIAS), A.data_ptr(), A.data_ptr(), C.data_ptr(), 0, 1.0, 0.0, 0, 0, 0)
     assert e.value.status == bg.ERR_NULL
     with pytest.raises(bg.GemmError) as e:                                          # short-extent shape whose automatic plan needs a workspace
-        bg.gemm_tune(bg.make_desc(8, 256, 4096), A.data_ptr(), A.data_ptr(), C.data_ptr(), 0, 1.0, 0.0, 0, 0, 0)
-    assert e.value.status == bg.ERR_WORKSPACE
+        bg.gemm_tune(bg.make_desc(8, 256, 4096, options=bg.OPT_STREAMK_WORKSPACE), A.data_ptr(), A.data_ptr(), C.data_ptr(), 0, 1.0, 0.0, 0, 0, 0)
+    assert e.value.status == bg.ERR_WORKSPACE                                       # (refused before anything runs)
 
 
 # ----------------------------------------------------------------------------- host-resident operands

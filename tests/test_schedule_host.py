@@ -168,3 +168,24 @@ def test_stream_k_units_once(short, long_, K):
                 sl = sched[tile_ix == t, SLICE]
                 assert (len(sl) == 1 and sl[0] == -1) or list(sl) == list(range(len(sl)))
                 assert len(sl) <= info["split"]
+
+
+def test_cluster_mode_of_stream_k():
+    """Exactly c <= 8 CTAs per output tile: the plan launches them as clusters and asks for no workspace; otherwise the
+    partial tiles go through a workspace."""
+    def info(M, N, K, **kw):
+        return plan_and_schedule(M, N, K, bg.make_flags(VS), **kw)[0]
+    import torch
+    for (M, N, K), c in (((8, 4096, 4096), 4), ((64, 4096, 4096), 4), ((16, 2048, 8192), 8), ((33, 4000, 4608), 4),
+                         ((4096, 8, 4096), 4), ((4000, 48, 4608), 4), ((64, 6144, 6144), 3), ((48, 4096, 11008), 4)):
+        i = info(M, N, K)
+        if torch.cuda.is_available():    # how many clusters of a size fit at once is the device's to say
+            assert 2 <= i["cluster_size"] <= c
+        else:
+            assert i["cluster_size"] == c
+        assert i["workspace_bytes"] == 0 and i["grid"] == -(-max(M, N) // 128) * i["cluster_size"], (M, N, K, i)
+    i = info(8, 4096, 8192, ab_dtype=bg.FP8_E4M3)
+    assert i["cluster_size"] >= 2 and i["workspace_bytes"] == 0
+    for M, N, K in ((8, 28672, 8192), (8, 10000, 2136), (40, 10240, 8200), (8, 11000, 8200), (33, 10880, 6144)):
+        i = info(M, N, K)
+        assert i["cluster_size"] == 1 and i["workspace_bytes"] > 0, (M, N, K, i)

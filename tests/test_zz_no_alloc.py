@@ -23,7 +23,7 @@ pytestmark = pytest.mark.gpu
 
 def run_regular(w, inputs):
     """Existing path: gemm_plan + gemm_run with a caller workspace (stream-K variant)."""
-    cbits, info = H.run_gpu(w, inputs, bg.make_flags(bg.VARIANT_SKINNY_STREAMK), poison=False)
+    cbits, info = H.run_gpu(w, inputs, bg.make_flags(bg.VARIANT_SKINNY_STREAMK), poison=False, options=bg.OPT_STREAMK_WORKSPACE)
     assert info["variant"] == bg.VARIANT_SKINNY_STREAMK and info["workspace_bytes"] > 0
     return cbits
 
