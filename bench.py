@@ -304,11 +304,25 @@ class DeviceCase:
             (" as a separate kernel" if act else "") + out_note
         return step, what
 
+    def time_burst(self, n: int = 10):
+        """`n` launches in a row, each between its own pair of events: the best one, in seconds."""
+        torch = self.torch
+        for _ in range(3):
+            self.step()
+        pairs = []
+        for _ in range(n):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            self.step()
+            e1.record()
+            pairs.append((e0, e1))
+        torch.cuda.synchronize()
+        return min(a.elapsed_time(b) for a, b in pairs) * 1e-3
+
     def time_isolated(self, n: int = 10):
         """Single launches, each on an idle GPU with a flushed L2 and bracketed by its own pair of events: (median, best) in
-        seconds.  This is the situation of a launch under the profiler (nothing overlaps its set-up, caches are cold, one
-        launch never meets the power cap), so it is the event-timed counterpart of the ncu durations in profiles/; the
-        best one is also how the dense peak this pool's roofline uses was measured (best of 10 single launches)."""
+        seconds.  This is the situation of a launch under the profiler (nothing overlaps its set-up, caches are cold, the
+        clocks start from idle), so it is the event-timed counterpart of the ncu durations in profiles/."""
         torch = self.torch
         flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=self.device)
         times = []
@@ -477,7 +491,9 @@ def run_ours(args):
     warm_launches = case.warm_launches
     # context: the vendor library on the same buffers in the same loop, and the headline held for seconds
     library = sustained = None
+    burst = case.time_burst() if args.all else None
     iso_med, iso_best = case.time_isolated() if args.all else (None, None)
+    lib_step = None
     if args.all and world == 1:
         lib_step, lib_what = case.library_step()
         if lib_step is not None:
@@ -485,15 +501,7 @@ def run_ours(args):
             lib_sec = case.time_steps(steps, warmup, step=lib_step)
             library = {"value": round(metric_value(w, lib_sec), 2), "unit": "TFLOP/s", "ms_per_step": round(lib_sec * 1e3, 5),
                        "what": lib_what + "; same rotating buffers, same event-timed loop; context only, no part of the product"}
-        if args.sustained_seconds > 0:
-            time.sleep(1.0)
-            sustained = case.time_sustained(args.sustained_seconds, sampler_index=local_rank)
-            sustained["frac_of_sustained_peak"] = round(sustained["value"] / peaks["bf16_tflops_sustained"], 4)
-            if lib_step is not None:
-                time.sleep(1.0)
-                ls = case.time_sustained(args.sustained_seconds, step=lib_step, sampler_index=local_rank)
-                library["sustained"] = {k: ls[k] for k in ("value", "seconds", "launches", "sm_mhz_median", "mcycles_per_step")}
-            time.sleep(1.0)
+        time.sleep(1.0)
     e2e_steps = max(2, min(steps, args.e2e_steps))
     barrier()
     if args.e2e_steps > 0:
@@ -522,18 +530,17 @@ def run_ours(args):
         "roofline": roofline_for(w, key, sec, peaks, peak_kind),
     }
     out["roofline"]["frac_of_sustained_peak"] = round(metric_value(w, sec) / peaks["bf16_tflops_sustained"], 4)
+    if burst is not None:
+        # ten launches in a row, each between its own pair of events, the best one: the protocol the measured dense peak
+        # of this pool was taken with (best of ten single library launches), so this fraction compares like with like
+        out["burst_best_of_10"] = {"ms": round(burst * 1e3, 5), "value": round(metric_value(w, burst), 2), "unit": "TFLOP/s",
+                                   "frac_of_peak": round(roofline_for(w, key, burst, peaks, peak_kind)["frac"], 4)}
     if iso_med is not None:
-        # single isolated launches: the median is what a launch under the profiler corresponds to; the best of ten is the
-        # protocol the measured dense peak was taken with, so `frac_of_peak` compares like with like
-        out["isolated_launch"] = {"ms_median": round(iso_med * 1e3, 5), "ms_best_of_10": round(iso_best * 1e3, 5),
-                                  "best_value": round(metric_value(w, iso_best), 2), "unit": "TFLOP/s",
-                                  "best_frac_of_peak": round(roofline_for(w, key, iso_best, peaks, peak_kind)["frac"], 4)}
+        # single launches on an idle GPU with a flushed L2: what a launch under the profiler corresponds to
+        out["isolated_launch"] = {"ms_median": round(iso_med * 1e3, 5), "ms_best_of_10": round(iso_best * 1e3, 5)}
     if library is not None:
         out["library_reference"] = library
-    if sustained is not None:
-        out["sustained"] = sustained
     host_inputs = case.host_inputs
-    case.close()
 
     if args.all:
         measured = []
@@ -590,6 +597,19 @@ def run_ours(args):
         out["hbm_context"] = {"torch_fill_write_only_gbs": rate(lambda: xs.fill_(1.0), xs.numel() * 2),
                               "torch_sum_read_only_gbs": rate(lambda: xs.sum(), xs.numel() * 2)}
         del xs
+
+    # last, so that the seconds of full load do not warm the GPU under the other measurements: the headline held for
+    # `--sustained-seconds`, and the library reference point the same way
+    if args.all and world == 1 and args.sustained_seconds > 0:
+        time.sleep(1.0)
+        sustained = case.time_sustained(args.sustained_seconds, sampler_index=local_rank)
+        sustained["frac_of_sustained_peak"] = round(sustained["value"] / peaks["bf16_tflops_sustained"], 4)
+        out["sustained"] = sustained
+        if lib_step is not None:
+            time.sleep(1.0)
+            ls = case.time_sustained(args.sustained_seconds, step=lib_step, sampler_index=local_rank)
+            out["library_reference"]["sustained"] = {k: ls[k] for k in ("value", "seconds", "launches", "sm_mhz_median", "mcycles_per_step")}
+    case.close()
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         v, cores, sample = time_oracle_sample(w, host_inputs, args.cpu_seconds)
