@@ -482,8 +482,8 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         return p.partials + (static_cast<size_t>(c) * 2 + (c == c_first ? first_slot : 0)) * (kSkinnyTileN * sp.m_pad);
       };
       // While the main loop of this segment runs, these warps have nothing to do.  The usual case for the CTA that
-      // computes the head of a split tile is that all other contributors finished long ago; if the count says so,
-      // their partials (and C_in) are fetched now, this CTA never publishes its own partial and the tail of the kernel
+      // computes the head of a split tile is that all other contributors finish before it does; as soon as the count says so,
+      // their partials (and C_in) are fetched, this CTA never publishes its own partial and the tail of the kernel
       // is one tensor-memory read, a few adds and the stores.  The fetched values are parked in shared memory: the
       // store cannot issue before its load has landed, which pins the loads to this side of the wait (left in
       // registers, the loads were scheduled after the wait, next to their use, and the tail paid their latency).
@@ -494,11 +494,29 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
       const bool by_chunk = sp.m_pad > 16;  // parked value 16 b + j = chunk b of the other contributor (else: chunk 0 of contributor b)
       const uint32_t park = base + bars_off + 16u * kMaxStages + 64u + (threadIdx.x - 64u) * 4u;  // value v lives at park + 512 v
       if (!whole && (by_chunk ? c_last - c_first == 1 : c_last - c_first <= 3)) {
-        if (leader)
-          s_early[seg == 0 ? 0 : 1] =
-              (stale_status == 0u && ld_acquire_gpu_u64(p.counters + tile) == ((p.tag << 16) | static_cast<unsigned long long>(c_last - c_first))) ? 1u : 0u;
-        named_barrier_sync(1, 128);
-        early = s_early[seg == 0 ? 0 : 1] != 0u;
+        // The leader looks at the arrival word again and again (about once a microsecond) until either all other
+        // contributors have arrived -- for the CTA that holds the head of a tile they are always done before its own
+        // range is, since their share of the tile is shorter than its whole range -- or its own accumulator is complete,
+        // in which case the partial is published as usual.  (Also bounded by the plan's wait limit.)
+        const unsigned long long all_others = (p.tag << 16) | static_cast<unsigned long long>(c_last - c_first);
+        volatile uint32_t* verdict_slot = s_early + (seg == 0 ? 0 : 1);
+        const uint64_t poll_t0 = globaltimer_ns();
+        uint32_t verdict = 0u;  // 1: the others are all in; 2: stop looking
+        while (true) {
+          if (leader) {
+            uint32_t v = 0u;
+            if (stale_status != 0u || *s_abort != 0u) v = 2u;
+            else if (ld_acquire_gpu_u64(p.counters + tile) == all_others) v = 1u;
+            else if (mbar_try_wait(tfull0 + 8u * buf, (seg >> 1) & 1u) || globaltimer_ns() - poll_t0 > p.timeout_ns) v = 2u;
+            *verdict_slot = v;
+          }
+          named_barrier_sync(1, 128);
+          verdict = *verdict_slot;
+          named_barrier_sync(1, 128);  // everybody has read the verdict before the leader writes the next one
+          if (verdict != 0u) break;
+          __nanosleep(400);
+        }
+        early = verdict == 1u;
         if (early) {
           const int other = c_first == static_cast<int>(blockIdx.x) ? c_last : c_first;
           float pre[4][16], cin0[16];
@@ -581,7 +599,40 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         }
         named_barrier_sync(1, 128);
         const bool last = *s_last != 0u;
-        if (last) {
+        if (last && c_last - c_first == 1 && small_extent > 16) {
+          // Two contributors and several 16-row chunks (the usual case of a wide short extent on a large problem, where a
+          // CTA's range is longer than a tile): the chunks are double buffered by hand -- the partials and C_in of chunk
+          // i + 1 are requested before chunk i is added up and stored -- because the compiler may not move those loads
+          // above the stores to D, and a chunk at a time costs one round trip to L2 plus one to HBM each (8 us for four
+          // chunks, measured).  Same additions in the same order as the loop below.
+          const float* q0 = partial_of(c_first) + n_local;
+          const float* q1 = partial_of(c_last) + n_local;
+          auto request = [&](int m0, float (&v)[2][16], float (&ci)[16]) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {  // m0 + j < m_pad
+              v[0][j] = __ldcg(q0 + (m0 + j) * kSkinnyTileN);
+              v[1][j] = __ldcg(q1 + (m0 + j) * kSkinnyTileN);
+            }
+            if (n < big_extent) sk_load_cin16<kTall>(p, m0, n, ci);
+          };
+          auto finish = [&](int m0, const float (&v)[2][16], const float (&ci)[16]) {
+            float sum[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) sum[j] = (0.0f + v[0][j]) + v[1][j];
+            if (n < big_extent) sk_finish16<kTall>(p, m0, n, sum, ci);
+          };
+          float va[2][16], vb[2][16], ca[16], cb[16];
+          request(0, va, ca);
+          for (int m0 = 0; m0 < small_extent; m0 += 32) {
+            const bool second = m0 + 16 < small_extent;
+            if (second) request(m0 + 16, vb, cb);
+            finish(m0, va, ca);
+            if (!second) break;
+            if (m0 + 32 < small_extent) request(m0 + 32, va, ca);
+            finish(m0 + 16, vb, cb);
+          }
+          if (leader) p.counters[tile] = 0ull;  // a replay of this launch (same tag) must find no arrivals
+        } else if (last) {
           for (int m0 = 0; m0 < small_extent; m0 += 16) {
             float sum[16], cin[16];
 #pragma unroll

@@ -107,6 +107,10 @@ EXACT_CASES = [
     ("cluster_4_tall_n48_padded", 4000, 48, 4608, dict(cd=wl.BF16, ldc=56, epi=bg.EPI_BIAS, bias_per_row=True), dict(variant=VS)),
     ("cluster_4_fp8", 8, 4096, 8192, dict(ab=wl.FP8_E4M3), dict(variant=VS)),
     ("cluster_auto_plan", 64, 4096, 4096, dict(cd=wl.BF16), dict()),
+    # CTA ranges longer than a tile: every split tile has two contributors, several 16-row chunks each (double-buffered fix-up)
+    ("skinny_m64_two_contributors", 64, 20480, 2048, dict(beta=1.0, epi=bg.EPI_BIAS), dict(variant=VS)),
+    ("tall_n48_two_contributors", 20480, 48, 2048, dict(cd=wl.BF16, beta=1.0, ldc=56), dict(variant=VS)),
+    ("skinny_m33_two_contributors_fp8", 33, 20000, 4096, dict(ab=wl.FP8_E4M3, cd=wl.F16), dict(variant=VS)),
     ("cluster_no_early_launch", 8, 4096, 4096, dict(beta=1.0), dict(variant=VS, no_early_launch=True)),
     ("no_early_launch_1cta", 264, 328, 200, {}, dict(variant=V1, tile_n=128, no_early_launch=True)),
     ("no_early_launch_skinny", 8, 256, 4096, dict(beta=1.0), dict(variant=VS, no_early_launch=True)),
