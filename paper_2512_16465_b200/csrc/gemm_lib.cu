@@ -109,11 +109,12 @@ namespace {
 
 // Tensor maps a plan has already encoded, by operand address.  Everything else a map depends on (extents, pitches,
 // box, element type) is fixed by the plan, so the base address alone identifies it.  One table per operand (A, B, D): a
-// caller that keeps its weights and changes its activations still finds two of the three.  128 entries each, four
-// probes from a hash of the address, the oldest of the four replaced on a miss.  Several host threads may run one
-// plan, hence the lock (held for a 128-byte copy).
+// caller that keeps its weights and changes its activations still finds two of the three.  256 entries each, eight
+// probes from a hash of the address, the oldest of the eight replaced on a miss (a loop over 126 buffer sets, the
+// benchmark's small configuration, then never misses; with 128 entries and four probes it re-encoded about every third
+// map).  Several host threads may run one plan, hence the lock (held for a 128-byte copy).
 struct MapCache {
-  static constexpr int kEntries = 128, kProbes = 4;
+  static constexpr int kEntries = 256, kProbes = 8;
   struct alignas(64) Entry {
     CUtensorMap map;
     const void* key;
@@ -126,7 +127,7 @@ struct MapCache {
   static int slot_of(const void* key) {
     uint64_t h = reinterpret_cast<uintptr_t>(key) >> 4;  // (operands are 16-byte aligned)
     h *= 0x9E3779B97F4A7C15ull;
-    return static_cast<int>(h >> 57);  // 7 bits
+    return static_cast<int>(h >> 56);  // 8 bits
   }
   // True and *out filled when `key` is known for operand `which`.
   bool find(int which, const void* key, CUtensorMap* out) {
