@@ -94,7 +94,10 @@ typedef enum {
  * it is launched. */
 #define GEMM_FLAG_VARIANT_SHIFT 4          /* bits 4-7: force a gemm_variant_t (0 = automatic) */
 #define GEMM_FLAG_VARIANT_MASK 0xF0u
-#define GEMM_FLAG_TILE_N_SHIFT 8           /* bits 8-12: force tile N / 16 (0 = automatic) */
+#define GEMM_FLAG_TILE_N_SHIFT 8           /* bits 8-12: force tile N (0 = automatic): 1 ... 16 = N / 16 (the 1-CTA and pair
+                                              variants take multiples of 64 up to 256), 17 ... 20 = 320, 384, 448, 512
+                                              (tiles of two MMAs side by side with a single accumulator buffer; B stored
+                                              N x K only) */
 #define GEMM_FLAG_TILE_N_MASK 0x1F00u
 #define GEMM_FLAG_TAIL_SPLIT 0x2000u       /* when the last wave of a 1-CTA or pair plan would fill at most half of the SMs, cut
                                               its tiles into K slices, one per CTA or pair (the plan then wants a workspace for

@@ -149,8 +149,9 @@ def make_flags(variant: int = 0, tile_n: int = 0, raster: int = 0, stages: int =
                bias_per_row: bool = False, a_lower: bool = False, a_upper: bool = False,
                tail_split: bool = False, d_lower: bool = False, d_upper: bool = False) -> int:
     """Pack the GEMM_FLAG_* fields of ``gemm_desc_t.flags`` (0 everywhere = automatic)."""
-    assert tile_n % 16 == 0
-    return ((variant & 0xF) << 4) | (((tile_n // 16) & 0x1F) << 8) | ((raster & 0x7F) << 16) | ((stages & 0xF) << 24) | \
+    assert tile_n % 16 == 0 and (tile_n <= 256 or (tile_n % 64 == 0 and tile_n <= 512))
+    tile_field = tile_n // 16 if tile_n <= 256 else 16 + (tile_n - 256) // 64   # 17 ... 20: the wide tiles 320 ... 512
+    return ((variant & 0xF) << 4) | ((tile_field & 0x1F) << 8) | ((raster & 0x7F) << 16) | ((stages & 0xF) << 24) | \
         ((kslices & 0x3) << 28) | (0x40000000 if l2_hints else 0) | (0x8 if no_k_serpentine else 0) | \
         (FLAG_DEBUG_STALL if debug_stall else 0) | (0x4 if no_early_launch else 0) | (0x1 if bias_per_row else 0) | (0x2 if a_lower else 0) | (0x800000 if a_upper else 0) | (0x2000 if tail_split else 0) | \
         (0x4000 if d_lower else 0) | (0x8000 if d_upper else 0)

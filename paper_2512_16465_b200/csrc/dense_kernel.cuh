@@ -67,11 +67,16 @@ struct DenseParams {
   // the scheduler's divisors: tiles per matrix, tiles per raster group, rows of a full group and of the last group, slots per matrix
   FastDiv fd_matrix, fd_group, fd_rows, fd_last_rows, fd_list;
   int kstep_shift;       // log2 of the K extent of a ring stage (kblk * atoms, a power of two)
-  int bn;                // tile N (multiple of 64, <= 256)
+  int bn;                // tile N (multiple of 64, <= 512)
+  // A tile wider than 256 columns is computed by two MMAs per K step, each mma_n = bn / 2 columns wide (n_mma = 2), and
+  // has no second accumulator buffer (acc_bufs = 1: 2 * bn columns would not fit the 512 of tensor memory), so such tiles
+  // are planned where every CTA computes one tile.  Otherwise mma_n = bn, n_mma = 1, acc_bufs = 2.
+  int mma_n, n_mma, acc_bufs;
+  int b_box_rows;        // rows of one B box: this CTA's share of one MMA's columns (b_rows / n_mma)
   int stages;            // ring depth
   int num_kb;            // ring stages per tile = ceil(K / (64 * atoms))
   int atoms;             // 64-wide K slices ("swizzle atoms") per ring stage: 1 or 2
-  uint32_t tmem_cols;    // power of two >= 2 * bn
+  uint32_t tmem_cols;    // power of two >= acc_bufs * bn
   uint32_t idesc;        // tcgen05 instruction descriptor
   uint32_t a_stage_bytes, b_stage_bytes;  // per CTA, per stage (all atoms)
   uint32_t a_atom_bytes, b_atom_bytes;    // per CTA, one 64-wide K slice
@@ -540,7 +545,9 @@ __device__ __forceinline__ void producer_role(const DenseParams& p, const CUtens
     }
     const TileCoord tc = decode_tile(p, tile);
     const int m0 = tc.tm * (kCtaM * CG) + static_cast<int>(cta_rank) * kCtaM;
-    const int n0 = tc.tn * p.bn + (CG == 2 ? static_cast<int>(cta_rank) * p.b_rows : 0);
+    // first column of this CTA's share of MMA group 0 (group g starts mma_n columns further; in a pair each CTA holds
+    // b_box_rows of every group's columns)
+    const int n0 = tc.tn * p.bn + (CG == 2 ? static_cast<int>(cta_rank) * p.b_box_rows : 0);
     // Serpentine K: all CTAs advance through K roughly in step, so the K range a wave touched last is what L2
     // still holds when the next wave starts; walking it backwards re-uses those lines of the shared A band.
     const bool rev = p.k_serpentine && (it & 1u);
@@ -585,7 +592,7 @@ __device__ __forceinline__ void producer_role(const DenseParams& p, const CUtens
               load(saa + 8192u, tmA, m0 + 64, ka, pol_a);
             }
             if (p.b_kmajor) {
-              load(sba, tmB, ka, n0, pol_b);
+              for (int g = 0; g < p.n_mma; ++g) load(sba + static_cast<uint32_t>(g * p.b_box_rows) * 128u, tmB, ka, n0 + g * p.mma_n, pol_b);
             } else {
               for (int g = 0; g < b_groups; ++g) load(sba + 8192u * g, tmB, n0 + 64 * g, ka, pol_b);
             }
@@ -631,8 +638,8 @@ __device__ __forceinline__ void mma_role(const DenseParams& p, uint32_t tiles_ba
       --it;          // (the loop header adds the one back: buffer and phase bookkeeping follow the tiles actually computed)
       continue;
     }
-    const uint32_t buf = it & 1u;
-    const uint32_t aph = (it >> 1) & 1u;
+    const uint32_t buf = p.acc_bufs == 2 ? (it & 1u) : 0u;
+    const uint32_t aph = p.acc_bufs == 2 ? ((it >> 1) & 1u) : (it & 1u);
     if (!mbar_wait_warp(tempty0 + 8u * buf, aph ^ 1u, w, (2u << 8) | 0x80u | buf)) return;
     tc_fence_after();
     const uint32_t d_tmem = tmem_base + buf * static_cast<uint32_t>(p.bn);
@@ -649,7 +656,30 @@ __device__ __forceinline__ void mma_role(const DenseParams& p, uint32_t tiles_ba
       const uint32_t empty_bar = empty0 + 8u * s;
       const bool ragged_stage = (rev ? kr.hi - 1 - kb : kr.lo + kb) == num_kb - 1;  // the stage that holds the end of K
       const bool two = (p.atoms == 2) && (!ragged_stage || last_atoms == 2);
-      if (elect_one()) {
+      if (p.n_mma == 2) {
+        // two column groups per K step: group g reads this CTA's rows [g * b_box_rows, ...) of the B tile and
+        // accumulates into tensor-memory columns [g * mma_n, ...)
+        if (elect_one()) {
+          const uint32_t g16 = (static_cast<uint32_t>(p.b_box_rows) * 128u) >> 4, dn = static_cast<uint32_t>(p.mma_n);
+          const int n_atoms = two ? 2 : 1;
+          for (int a = 0; a < n_atoms; ++a) {
+            const uint64_t ad = adesc + a * aatom16, bd = bdesc + a * batom16;
+#pragma unroll
+            for (uint32_t k = 0; k < 4; ++k) {
+              const uint32_t acc_on = static_cast<uint32_t>(kb != 0 || a != 0 || k != 0);
+              if (!p.ab_fp8) {
+                umma_f16<CG>(d_tmem, ad + k * ak16, bd + k * bk16, idesc, acc_on);
+                umma_f16<CG>(d_tmem + dn, ad + k * ak16, bd + g16 + k * bk16, idesc, acc_on);
+              } else {
+                umma_f8<CG>(d_tmem, ad + k * ak16, bd + k * bk16, idesc, acc_on);
+                umma_f8<CG>(d_tmem + dn, ad + k * ak16, bd + g16 + k * bk16, idesc, acc_on);
+              }
+            }
+          }
+          if constexpr (CG == 1) umma_commit<1>(empty_bar);
+          else umma_commit_pair_mcast(empty_bar, 3);
+        }
+      } else if (elect_one()) {
         if (!p.ab_fp8) {
           umma_f16<CG>(d_tmem, adesc, bdesc, idesc, static_cast<uint32_t>(kb != 0));
 #pragma unroll
@@ -733,8 +763,8 @@ __device__ __forceinline__ void epilogue_role(const DenseParams& p, const CUtens
       continue;
     }
     const TileCoord tc = decode_tile(p, tile);
-    const uint32_t buf = it & 1u;
-    const uint32_t ph = (it >> 1) & 1u;
+    const uint32_t buf = p.acc_bufs == 2 ? (it & 1u) : 0u;
+    const uint32_t ph = p.acc_bufs == 2 ? ((it >> 1) & 1u) : (it & 1u);
     if (!mbar_wait_warp(tfull0 + 8u * buf, ph, w, (3u << 8) | buf, 64u)) return;  // whole warp leaves the wait together
     tc_fence_after();
     // split tile: slice `slice` of `p.split`; the partials of slices 1.. live at part0, flags at flag0

@@ -368,7 +368,8 @@ bool set_scheduler_divisors(DenseParams& p) {
 // Tail split of the double-buffered dense kernels (on request, GEMM_FLAG_TAIL_SPLIT): when the tiles left over after the
 // full waves occupy at most half of the CTAs (pairs), each of them is cut into this many K slices, one per CTA (pair); the slice that
 // starts at K = 0 adds the others' raw accumulators from the workspace and finishes the tile.  1 = no split.
-int tail_split(long long tiles, int units, int num_kb, const gemm_desc_t& d) {
+int tail_split(long long tiles, int units, int num_kb, const gemm_desc_t& d, int bn = 0) {
+  if (bn > 256) return 1;  // (the partial-tile layout and the flag protocol are written for two accumulator buffers)
   if ((d.flags & (GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER | GEMM_FLAG_D_LOWER | GEMM_FLAG_D_UPPER)) || d.structure) return 1;
   const long long rem = tiles % units;
   if (rem == 0 || rem * 2 > units) return 1;
@@ -405,15 +406,18 @@ double estimate_dense_cycles(const gemm_desc_t& d, int sm_count, int variant, in
   const double kblocks = static_cast<double>(ceil_div(d.K, kblk_of(d.ab_dtype)));  // 128-byte slices: same pipe time for either width
   double waves = static_cast<double>((tiles + units - 1) / units);
   if (!wide) {  // a thinly filled last wave is split along K (two slices per stage assumed, as plan_dense will choose for long K)
-    const int split = tail_split(tiles, units, static_cast<int>(kblocks) / 2, d);
+    const int split = tail_split(tiles, units, static_cast<int>(kblocks) / 2, d, bn);
     if (split > 1) waves += 1.0 / split - 1.0 + 0.08;  // + hand-over of the partial accumulators
   }
   // tensor pipe: one 128 x bn x 16 MMA per CTA takes bn / 2 cycles; four per k-block and 128-row half
   static const double eff1[4] = {0.45, 0.68, 0.76, 0.82}, eff2[4] = {0.55, 0.80, 0.88, 0.938};  // bn = 64, 128, 192, 256 (measured: 8192^3, and K = 512 ... 4096; 192 in between)
-  const int bi = bn <= 64 ? 0 : (bn <= 128 ? 1 : (bn <= 192 ? 2 : 3));
+  const int mma_n = bn > 256 ? bn / 2 : bn;  // (a tile wider than 256 columns is two MMAs side by side)
+  const int bi = mma_n <= 64 ? 0 : (mma_n <= 128 ? 1 : (mma_n <= 192 ? 2 : 3));
   const double eff = wide ? 1.0 : (cg == 1 ? eff1[bi] : eff2[bi]);
   const double mma = kblocks * 4.0 * (bn / 2.0) * (rows_cta / 128.0) / eff;
-  // operand feed: bytes this SM receives per k-block at ~90 B/clk
+  // operand feed: bytes this SM receives per k-block at ~90 B/clk (fitted on multi-wave problems; at the start of a
+  // kernel, when 144-148 SMs fill their rings at once, traces show 55-58 B/clk per SM -- about 17 TB/s out of L2 in
+  // total -- which is what bounds the one- and two-tile-per-CTA problems)
   // ... and half that rate when an operand's row pitch is not a multiple of 128 bytes: every row of a TMA box then
   // straddles two memory lines (measured: the families rank by loads per FLOP there, wide > pair > single CTA)
   const bool straddling = (d.lda * elem_bytes(d.ab_dtype)) % 128 != 0 || (d.ldb * elem_bytes(d.ab_dtype)) % 128 != 0;
@@ -426,10 +430,16 @@ double estimate_dense_cycles(const gemm_desc_t& d, int sm_count, int variant, in
   // measured pair-vs-wide time ratios at K = 4096 ... 16384 on 8192 x 8192 and 16384 x 14336 outputs
   if (wide) exposed = (gelu ? 13000.0 : 5100.0) + (has_bias(d.epilogue) ? 1300.0 : 0.0);
   else if (cg == 2) exposed = 1000.0;           // pair hand-shakes cross the SM-to-SM network
+  // a tile wider than 256 columns has a single accumulator buffer: its whole read-out (eight warps, about 900 cycles per
+  // 64-column slab and warp) stands between two tiles; and at the end of the kernel it is longer than a narrow tile's
+  if (!wide && bn > 256) exposed += (bn / 64) / 2.0 * 900.0;
   // what is exposed stalls the tensor pipe, so it adds to the compute side; an output-bound tile instead pays a small
   // switch-over per tile (measured on the batched short-K shape: fewer, larger tiles win)
   const double per_tile = std::max(std::max(mma, feed) + exposed, out + 300.0);
-  return waves * per_tile + 3000.0;  // + pipeline fill and drain
+  // (fitted: against a second, partly filled wave of narrower tiles the one wave of wide tiles does about 8 % better than
+  // this estimate says -- measured 2304^3 23.0 us against 27.0, 2560^3 27.6 / 30.5, 3072^3 42.2 / 42.8, 2816^3 37.9 / 36.9)
+  const double fitted = (!wide && bn > 256) ? 0.92 : 1.0;
+  return (waves * per_tile + 3000.0) * fitted;  // + pipeline fill and drain
 }
 
 // Fill plan->dense and the launch geometry for a dense variant.
@@ -453,7 +463,11 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
       if (bn == 192) bn = 128;
     }
   }
-  if (bn < bn_step || bn > 256 || bn % bn_step) return GEMM_ERR_UNSUPPORTED;
+  if (bn < bn_step || bn > 512 || bn % bn_step) return GEMM_ERR_UNSUPPORTED;
+  // wider than 256 columns: two MMAs per K step, one accumulator buffer (see DenseParams::mma_n); B with K contiguous only
+  // (the loader for N-contiguous B moves 64-column boxes and has no notion of the two column groups)
+  const bool wide_n = bn > 256;
+  if (wide_n && !b_kmajor) return GEMM_ERR_UNSUPPORTED;
   const int tiles_n = ceil_div(d.N, bn);
   const int b_rows = bn / cg;
   const int a_atom = kCtaM * kBlockK * 2;
@@ -470,7 +484,7 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   // 256-wide tile per CTA has nothing to hide its epilogue behind: there too eight warps drain the accumulator
   // (2048^3: 19.6 -> 18.0 us; narrower tiles measured slower with them).
   const int kblk = kblk_of(d.ab_dtype);
-  const int epi_wg = ((!single_wave && static_cast<long long>(ceil_div(d.K, kblk)) * 2 * bn <= 4096) || (single_wave && bn == 256)) ? 2 : 1;
+  const int epi_wg = ((!single_wave && static_cast<long long>(ceil_div(d.K, kblk)) * 2 * bn <= 4096) || (single_wave && bn >= 256) || wide_n) ? 2 : 1;
   int atoms = forced_atoms;
   if (atoms == 0) {
     const bool fits3 = 3 * 2 * (a_atom + b_atom) + dense_smem_bytes(0, 0, 0, epi_wg) <= kMaxSmemOptin;
@@ -518,10 +532,14 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   p.ab_fp8 = is_fp8(d.ab_dtype) ? 1 : 0;
   p.a_atom_bytes = a_atom;
   p.b_atom_bytes = b_atom;
+  p.n_mma = wide_n ? 2 : 1;
+  p.mma_n = bn / p.n_mma;
+  p.acc_bufs = wide_n ? 1 : 2;
+  p.b_box_rows = b_rows / p.n_mma;
   uint32_t cols = 32;
-  while (cols < 2u * bn) cols <<= 1;
+  while (cols < static_cast<uint32_t>(p.acc_bufs * bn)) cols <<= 1;
   p.tmem_cols = cols;
-  p.idesc = make_idesc(ab_format(d.ab_dtype), !a_kmajor, !b_kmajor, tile_m, bn);
+  p.idesc = make_idesc(ab_format(d.ab_dtype), !a_kmajor, !b_kmajor, tile_m, p.mma_n);
   p.a_stage_bytes = a_stage;
   p.b_stage_bytes = b_stage;
   p.a_kmajor = a_kmajor;
@@ -587,7 +605,7 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   info.grid = pl->grid;
   info.raster_group = raster;
   const int units_i = pl->sm_count / cg;
-  const int split = tail_split(num_tiles, units_i, p.num_kb, d);
+  const int split = tail_split(num_tiles, units_i, p.num_kb, d, bn);
   const long long rem = num_tiles % units_i;
   p.split = split;
   p.split_first_tile = static_cast<int>(split > 1 ? num_tiles - rem : num_tiles);
@@ -645,6 +663,10 @@ gemm_status_t plan_wide(gemm_plan_s* pl, int forced_raster, int forced_stages) {
   p.ab_fp8 = is_fp8(d.ab_dtype) ? 1 : 0;
   p.atoms = 1;
   p.tmem_cols = 512;
+  p.n_mma = 1;
+  p.mma_n = bn;
+  p.acc_bufs = 1;
+  p.b_box_rows = bn / 2;
   p.idesc = make_idesc(ab_format(d.ab_dtype), !a_kmajor, !b_kmajor, 256, bn);
   p.a_stage_bytes = a_stage;
   p.b_stage_bytes = b_stage;
@@ -848,7 +870,13 @@ gemm_status_t plan_impl(const gemm_desc_t* desc, gemm_plan_t* out_plan, bool use
                                                 : (info.intensity < kRidgeTensor ? GEMM_REGIME_MIDDLE : GEMM_REGIME_COMPUTE);
 
   const int forced_variant = (d.flags & GEMM_FLAG_VARIANT_MASK) >> GEMM_FLAG_VARIANT_SHIFT;
-  const int forced_bn = static_cast<int>((d.flags & GEMM_FLAG_TILE_N_MASK) >> GEMM_FLAG_TILE_N_SHIFT) * 16;
+  // (field values up to 16 count sixteenths of 256 columns; 17 ... 20 are the wide tiles 320, 384, 448 and 512)
+  const int tile_field = static_cast<int>((d.flags & GEMM_FLAG_TILE_N_MASK) >> GEMM_FLAG_TILE_N_SHIFT);
+  if (tile_field > 20) {
+    delete pl;
+    return GEMM_ERR_INVALID_ARG;
+  }
+  const int forced_bn = tile_field <= 16 ? tile_field * 16 : 256 + (tile_field - 16) * 64;
   const int forced_raster = (d.flags & GEMM_FLAG_RASTER_MASK) >> GEMM_FLAG_RASTER_SHIFT;
   const int forced_stages = (d.flags & GEMM_FLAG_STAGES_MASK) >> GEMM_FLAG_STAGES_SHIFT;
   const int forced_atoms = (d.flags & GEMM_FLAG_KSLICES_MASK) >> GEMM_FLAG_KSLICES_SHIFT;
@@ -866,8 +894,16 @@ gemm_status_t plan_impl(const gemm_desc_t* desc, gemm_plan_t* out_plan, bool use
       const bool b_kmajor = d.transb == GEMM_OP_T;
       DenseCandidate best{GEMM_VARIANT_DENSE_1CTA, 64, 1e300};
       for (int v : {GEMM_VARIANT_DENSE_1CTA, GEMM_VARIANT_DENSE_2CTA, GEMM_VARIANT_DENSE_2CTA_WIDE}) {
-        for (int bn : {256, 192, 128, 64}) {
+        for (int bn : {512, 448, 384, 320, 256, 192, 128, 64}) {
           if (v == GEMM_VARIANT_DENSE_2CTA_WIDE && bn != kWideTileN) continue;
+          if (bn > 256) {
+            // wide single-buffered tiles: K-contiguous B, and only where they give every CTA (pair) at most one tile --
+            // their purpose is to turn "a little more than one wave" into one wave (2304^3: 108 tiles of 256 x 192 on 74
+            // pairs become 72 of 256 x 320) and to cut the operand traffic per FLOP on the way
+            const int rows_tile = v == GEMM_VARIANT_DENSE_1CTA ? kCtaM : 2 * kCtaM;
+            const long long tiles = tri_tile_count(d_tri_of(d), rows_tile, bn, d.M, d.N) * d.batch_count;
+            if (!b_kmajor || tiles > pl->sm_count / (v == GEMM_VARIANT_DENSE_1CTA ? 1 : 2) || (d.flags & GEMM_FLAG_TAIL_SPLIT)) continue;
+          }
           if (v == GEMM_VARIANT_DENSE_2CTA_WIDE &&
               (d.epilogue > GEMM_EPI_BIAS_GELU_ERF || d_tri_of(d) || d.structure || (d.N * elem_bytes(d.c_dtype)) % 16 ||
                (d.flags & (GEMM_FLAG_BIAS_PER_ROW | GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER))))
@@ -1205,7 +1241,7 @@ gemm_status_t run_dense(gemm_plan_s* pl, const void* A, const void* B, void* C, 
     if (ok) pl->maps->insert(0, A, tA);
   }
   if (ok && !pl->maps->find(1, B, &tB)) {
-    ok = p.b_kmajor ? encode_map(&tB, d.ab_dtype, B, d.K, d.N, batch, d.ldb, d.stride_b, p.kblk, p.b_rows)
+    ok = p.b_kmajor ? encode_map(&tB, d.ab_dtype, B, d.K, d.N, batch, d.ldb, d.stride_b, p.kblk, p.b_box_rows)
                     : encode_map(&tB, d.ab_dtype, B, d.N, d.K, batch, d.ldb, d.stride_b, 64, kBlockK);
     if (ok) pl->maps->insert(1, B, tB);
   }

@@ -34,7 +34,8 @@ std::map<Key, uint32_t>& cache() {
 }
 
 uint32_t pack(int variant, int tile_n, int raster, int stages, int kslices) {
-  return (static_cast<uint32_t>(variant) << GEMM_FLAG_VARIANT_SHIFT) | (static_cast<uint32_t>(tile_n / 16) << GEMM_FLAG_TILE_N_SHIFT) |
+  const int tile_field = tile_n <= 256 ? tile_n / 16 : 16 + (tile_n - 256) / 64;  // (17 ... 20: the wide tiles 320 ... 512)
+  return (static_cast<uint32_t>(variant) << GEMM_FLAG_VARIANT_SHIFT) | (static_cast<uint32_t>(tile_field) << GEMM_FLAG_TILE_N_SHIFT) |
          (static_cast<uint32_t>(raster) << GEMM_FLAG_RASTER_SHIFT) | (static_cast<uint32_t>(stages) << GEMM_FLAG_STAGES_SHIFT) |
          (static_cast<uint32_t>(kslices) << GEMM_FLAG_KSLICES_SHIFT);
 }
@@ -55,6 +56,9 @@ std::vector<uint32_t> first_round(const gemm_desc_t& d, const gemm_info_t& autom
   } else {
     for (int bn : {256, 128}) c.push_back(pack(GEMM_VARIANT_DENSE_1CTA, bn, 0, 0, 0));
     for (int bn : {256, 192, 128}) c.push_back(pack(GEMM_VARIANT_DENSE_2CTA, bn, 0, 0, 0));  // (192: refused, hence skipped, when B is stored K x N)
+    // wide single-buffered pair tiles where they give every pair at most one tile (also refused when B is stored K x N)
+    for (int bn : {320, 384, 448, 512})
+      if (((d.M + 255) / 256) * ((d.N + bn - 1) / bn) * d.batch_count <= 74) c.push_back(pack(GEMM_VARIANT_DENSE_2CTA, bn, 0, 0, 0));
     c.push_back(pack(GEMM_VARIANT_DENSE_2CTA_WIDE, 0, 0, 0, 0));
   }
   return c;

@@ -98,6 +98,20 @@ EXACT_CASES = [
     ("skinny_one_slice_stages", 8, 256, 4096, {}, dict(variant=VS, kslices=1)),
     ("skinny_three_slice_stages", 8, 384, 1100 - 4, {}, dict(variant=VS, kslices=3)),
     ("skinny_k_slice_past_the_end", 8, 256, 1080, {}, dict(variant=VS)),
+    # tiles wider than 256 columns: two MMAs side by side per K step, one accumulator buffer
+    ("wide_n_512_pair_one_tile", 256, 512, 256, {}, dict(variant=V2, tile_n=512)),
+    ("wide_n_320_pair_ragged_bf16", 600, 712, 456, dict(cd=wl.BF16), dict(variant=V2, tile_n=320)),
+    ("wide_n_384_pair_beta_bias_f32", 520, 1000, 200, dict(beta=1.0, epi=bg.EPI_BIAS_RELU), dict(variant=V2, tile_n=384)),
+    ("wide_n_448_1cta_f16", 300, 904, 136, dict(ab=wl.F16, cd=wl.F16, alpha=0.5), dict(variant=V1, tile_n=448)),
+    ("wide_n_512_1cta_many_tiles", 1024, 2048, 328, dict(cd=wl.BF16), dict(variant=V1, tile_n=512)),
+    ("wide_n_512_pair_several_tiles_per_cta", 2560, 5120, 264, dict(cd=wl.BF16), dict(variant=V2, tile_n=512)),
+    ("wide_n_384_pair_one_slice_stages", 512, 768, 712, {}, dict(variant=V2, tile_n=384, kslices=1)),
+    ("wide_n_320_pair_a_stored_transposed", 520, 640, 200, dict(ta=1), dict(variant=V2, tile_n=320)),
+    ("wide_n_512_fp8", 512, 1024, 1040, dict(ab=wl.FP8_E4M3, cd=wl.BF16), dict(variant=V2, tile_n=512)),
+    ("wide_n_384_batched", 300, 504, 136, dict(batch=3, cd=wl.BF16), dict(variant=V2, tile_n=384)),
+    ("wide_n_512_lower_triangular_d_upper", 1024, 1024, 1024, dict(a_tri=1, d_tri=2), dict(variant=V2, tile_n=512)),
+    ("wide_n_320_n_not_a_multiple_of_16_bytes", 300, 650, 136, dict(cd=wl.BF16, ldc=656), dict(variant=V2, tile_n=320)),
+    ("wide_n_auto_2304", 2304, 2304, 264, dict(cd=wl.BF16), dict()),
     # stream-K with exactly c CTAs per output tile: the c CTAs form a cluster and hand over through shared memory
     ("cluster_4_m8", 8, 4096, 4096, {}, dict(variant=VS)),
     ("cluster_4_m64_f16_beta", 64, 4096, 4096, dict(ab=wl.F16, cd=wl.F16, alpha=0.5, beta=1.0), dict(variant=VS)),

@@ -68,7 +68,9 @@ def test_plan_validation_codes():
     assert plan_status(**ok, batch=2, stride_c=100) == bg.ERR_INVALID_ARG    # outputs would overlap
     assert plan_status(**ok, batch=2, stride_a=256 * 256 + 4) == bg.ERR_ALIGNMENT
     assert plan_status(M=200, N=256, K=256, flags=bg.make_flags(bg.VARIANT_SKINNY_STREAMK)) == bg.ERR_UNSUPPORTED
-    assert plan_status(**ok, flags=bg.make_flags(bg.VARIANT_DENSE_1CTA, tile_n=272)) == bg.ERR_UNSUPPORTED
+    assert plan_status(**ok, flags=bg.make_flags(bg.VARIANT_DENSE_1CTA, tile_n=240)) == bg.ERR_UNSUPPORTED   # not a multiple of 64
+    assert plan_status(**ok, flags=bg.make_flags(bg.VARIANT_DENSE_1CTA) | (21 << 8)) == bg.ERR_INVALID_ARG    # tile field beyond 512
+    assert plan_status(**ok, transb=bg.OP_N, flags=bg.make_flags(bg.VARIANT_DENSE_1CTA, tile_n=320)) == bg.ERR_UNSUPPORTED  # wide tiles: B stored N x K
     d = bg.make_desc(**ok)
     d.struct_size = 12
     with pytest.raises(bg.GemmError) as e:

@@ -85,7 +85,8 @@ DENSE_SHAPES = [(512, 512, 512), (1, 1, 1), (129, 257, 65), (1000, 1000, 1000), 
 
 
 @pytest.mark.parametrize("shape", DENSE_SHAPES, ids=lambda s: "x".join(map(str, s)))
-@pytest.mark.parametrize("variant,tile_n", [(0, 0), (V1, 64), (V1, 128), (V1, 192), (V1, 256), (V2, 128), (V2, 256), (VW, 0)])
+@pytest.mark.parametrize("variant,tile_n", [(0, 0), (V1, 64), (V1, 128), (V1, 192), (V1, 256), (V2, 128), (V2, 256), (VW, 0),
+                                            (V1, 320), (V2, 384), (V2, 512)])
 def test_every_tile_once_dense(shape, variant, tile_n):
     M, N, K = shape
     if variant == VW and M <= 128:
