@@ -307,6 +307,8 @@ class DeviceCase:
     def time_burst(self, n: int = 10):
         """`n` launches in a row, each between its own pair of events: the best one, in seconds."""
         torch = self.torch
+        torch.cuda.synchronize()
+        time.sleep(1.5)   # from a rested GPU, as a peak measurement would be taken
         for _ in range(3):
             self.step()
         pairs = []
@@ -562,11 +564,11 @@ def run_ours(args):
                    "roofline": roofline_for(w2, k2, s2, peaks, peak_kind)}
             row["ms_isolated_launch"] = round(c2.time_isolated()[0] * 1e3, 5)
             if world == 1:
-                lib_step, lib_what = c2.library_step()
-                if lib_step is not None:     # the vendor library on the same buffers, same loop (context)
+                lib2, lib2_what = c2.library_step()
+                if lib2 is not None:     # the vendor library on the same buffers, same loop (context)
                     time.sleep(0.5)
-                    row["library_reference_ms_per_step"] = round(c2.time_steps(steps, warmup, step=lib_step) * 1e3, 5)
-                    row["library_reference_what"] = lib_what
+                    row["library_reference_ms_per_step"] = round(c2.time_steps(steps, warmup, step=lib2) * 1e3, 5)
+                    row["library_reference_what"] = lib2_what
                 # the same plan launched without programmatic dependent launch: what the overlap of one kernel's set-up
                 # with its predecessor's tail is worth in this back-to-back loop
                 time.sleep(0.5)
