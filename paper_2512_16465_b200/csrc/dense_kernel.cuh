@@ -270,22 +270,24 @@ __host__ __device__ __forceinline__ WorkItem work_item(const DenseParams& p, int
   }
   return wi;
 }
-// Bounded wait for a flag word another CTA of this launch sets (all CTAs of these persistent kernels are resident,
-// and the CTA that sets the flag never waits for anybody).  Warp-uniform; false = gave up (timeout or abort elsewhere).
-__device__ __noinline__ bool flag_wait_warp(const unsigned long long* flag, unsigned long long tag, const WaitCtx& w, uint32_t code) {
+// Bounded wait for up to 32 consecutive flag words that other CTAs of this launch set to `tag` (all CTAs of these
+// persistent kernels are resident, and a CTA that sets a flag never waits for anybody).  Lane l looks at word l, so the
+// wait costs one round trip to memory however many words there are (one wait after the other cost a round trip each:
+// 4 us for the seven slices of 256 x 256 x 32768).  Warp-uniform; false = gave up (timeout or abort elsewhere).
+__device__ __noinline__ bool flags_wait_warp(const unsigned long long* flags, int n, unsigned long long tag, const WaitCtx& w, uint32_t code) {
   const uint64_t t0 = globaltimer_ns();
+  const int l = static_cast<int>(lane_id());
   uint32_t it = 0;
   while (true) {
-    uint32_t hit = 0;
-    if (lane_id() == 0) hit = ld_acquire_gpu_u64(flag) == tag ? 1u : 0u;
-    if (__shfl_sync(0xffffffffu, hit, 0) != 0u) {
-      __syncwarp();  // orders the other lanes' later loads after lane 0's acquire (a shuffle alone orders no memory)
+    const bool hit = l >= n || ld_acquire_gpu_u64(flags + l) == tag;
+    if (__all_sync(0xffffffffu, hit)) {
+      __syncwarp();  // (orders every lane's later loads after the acquiring loads of the others)
       return true;
     }
     __nanosleep(64);
     if ((++it & 31u) == 0u) {
       bool give_up = false;
-      if (lane_id() == 0) {
+      if (l == 0) {
         if (*w.s_abort || *reinterpret_cast<volatile uint32_t*>(w.g_status) != 0u) {
           *w.s_abort = 1u;
           give_up = true;
@@ -803,8 +805,7 @@ __device__ __forceinline__ void epilogue_role(const DenseParams& p, const CUtens
       continue;
     }
     if (kSplit && slice == 0) {  // reducer: the other slices of this tile run in the same wave; wait for their partials
-      for (int sidx = 0; sidx < p.split - 1; ++sidx)
-        if (!flag_wait_warp(flag0 + sidx, p.split_tag, w, (3u << 8) | 0x40u | static_cast<uint32_t>(sidx))) return;
+      if (!flags_wait_warp(flag0, p.split - 1, p.split_tag, w, (3u << 8) | 0x40u)) return;  // (at most 16 slices)
     }
     const int row0 = tc.tm * (kCtaM * CG) + static_cast<int>(cta_rank) * kCtaM + static_cast<int>(q) * 32;
     const long long row = row0 + static_cast<int>(lane);
