@@ -499,24 +499,24 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
         // range is, since their share of the tile is shorter than its whole range -- or its own accumulator is complete,
         // in which case the partial is published as usual.  (Also bounded by the plan's wait limit.)
         const unsigned long long all_others = (p.tag << 16) | static_cast<unsigned long long>(c_last - c_first);
-        volatile uint32_t* verdict_slot = s_early + (seg == 0 ? 0 : 1);
+        volatile uint32_t* answer_slot = s_early + (seg == 0 ? 0 : 1);
         const uint64_t poll_t0 = globaltimer_ns();
-        uint32_t verdict = 0u;  // 1: the others are all in; 2: stop looking
+        uint32_t answer = 0u;  // 1: the others are all in; 2: stop looking
         while (true) {
           if (leader) {
             uint32_t v = 0u;
             if (stale_status != 0u || *s_abort != 0u) v = 2u;
             else if (ld_acquire_gpu_u64(p.counters + tile) == all_others) v = 1u;
             else if (mbar_try_wait(tfull0 + 8u * buf, (seg >> 1) & 1u) || globaltimer_ns() - poll_t0 > p.timeout_ns) v = 2u;
-            *verdict_slot = v;
+            *answer_slot = v;
           }
           named_barrier_sync(1, 128);
-          verdict = *verdict_slot;
-          named_barrier_sync(1, 128);  // everybody has read the verdict before the leader writes the next one
-          if (verdict != 0u) break;
+          answer = *answer_slot;
+          named_barrier_sync(1, 128);  // everybody has read the answer before the leader writes the next one
+          if (answer != 0u) break;
           __nanosleep(400);
         }
-        early = verdict == 1u;
+        early = answer == 1u;
         if (early) {
           const int other = c_first == static_cast<int>(blockIdx.x) ? c_last : c_first;
           float pre[4][16], cin0[16];
