@@ -73,9 +73,10 @@ CUtensorMapDataType tm_dtype(int dtype) {
 }
 
 // 3-D tiled map over a row-major matrix batch: dim0 = contiguous extent, dim1 = rows, dim2 = batch.
-// 128-byte swizzle, out-of-bounds elements read as zero / are not written.
+// 128-byte swizzle (or, for a store from a plain row-major staging buffer, none), out-of-bounds elements read as zero /
+// are not written.
 bool encode_map(CUtensorMap* m, int dtype, const void* base, uint64_t inner, uint64_t rows, uint64_t batch, uint64_t ld,
-                uint64_t batch_stride, uint32_t box_inner, uint32_t box_rows) {
+                uint64_t batch_stride, uint32_t box_inner, uint32_t box_rows, bool swizzle = true) {
   EncodeFn fn = get_encode_fn();
   if (!fn) {
     note_cuda_error("cuTensorMapEncodeTiled", "driver entry point not found");
@@ -91,7 +92,7 @@ bool encode_map(CUtensorMap* m, int dtype, const void* base, uint64_t inner, uin
   // 4100 x 4104 x 4104: 164 -> 144 us without promotion; no difference on aligned pitches)
   const CUtensorMapL2promotion promotion = (ld * eb) % 128 == 0 ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_NONE;
   CUresult r = fn(m, tm_dtype(dtype), 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                  CU_TENSOR_MAP_SWIZZLE_128B, promotion, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                  swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, promotion, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
     char buf[64];
     snprintf(buf, sizeof buf, "CUresult %d", static_cast<int>(r));
@@ -1295,9 +1296,10 @@ gemm_status_t run_skinny(gemm_plan_s* pl, const void* A, const void* B, void* C,
                          void* workspace, cudaStream_t stream, bool stall, unsigned long long run_index) {
   const gemm_desc_t& d = pl->d;
   const SkinnyPlan& s = pl->skinny;
-  CUtensorMap tW, tX;
+  CUtensorMap tW, tX, tD;
   // weights W = B stored N x K (K contiguous): box 64 x 128; activations X = A stored M x K: box 64 x m_pad;
   // a tall problem streams A in W's place and keeps B as the slab.  Maps are remembered by operand address.
+  // D (unless tall): plain row-major boxes of 16 rows x 32 columns over the whole 16-byte units of each row.
   const void* w_ptr = pl->skinny_tall ? A : B;
   const void* x_ptr = pl->skinny_tall ? B : A;
   const int64_t w_rows = pl->skinny_tall ? d.M : d.N, w_ld = pl->skinny_tall ? d.lda : d.ldb;
@@ -1311,10 +1313,19 @@ gemm_status_t run_skinny(gemm_plan_s* pl, const void* A, const void* B, void* C,
     ok = encode_map(&tX, d.ab_dtype, x_ptr, d.K, x_rows, 1, x_ld, 0, s.kblk, s.m_pad);
     if (ok) pl->maps->insert(1, x_ptr, tX);
   }
+  const int64_t per16 = 16 / elem_bytes(d.c_dtype);
+  const int n_full = pl->skinny_tall ? 0 : static_cast<int>(d.N / per16 * per16);
+  if (n_full == 0) {
+    tD = tW;  // never used
+  } else if (ok && !pl->maps->find(2, C, &tD)) {
+    ok = encode_map(&tD, d.c_dtype, C, n_full, d.M, 1, d.ldc, 0, 32, 16, /*swizzle=*/false);
+    if (ok) pl->maps->insert(2, C, tD);
+  }
   if (!ok) return GEMM_ERR_CUDA;
   SkinnyParams p;
   memset(&p, 0, sizeof p);
   p.plan = s;
+  p.n_full = n_full;
   p.M = static_cast<int>(d.M);
   p.N = static_cast<int>(d.N);
   p.K = static_cast<int>(d.K);
@@ -1336,7 +1347,7 @@ gemm_status_t run_skinny(gemm_plan_s* pl, const void* A, const void* B, void* C,
   p.status = pl->d_status;
   p.timeout_ns = static_cast<unsigned long long>(pl->timeout_ms) * 1000000ull;
   return static_cast<gemm_status_t>(
-      skinny_launch(p, tW, tX, pl->device, stream, g_last_cuda_error, sizeof g_last_cuda_error, pl->skinny_tall,
+      skinny_launch(p, tW, tX, tD, pl->device, stream, g_last_cuda_error, sizeof g_last_cuda_error, pl->skinny_tall,
                     /*early_launch=*/!(d.flags & GEMM_FLAG_NO_EARLY_LAUNCH)));
 }
 
@@ -1453,9 +1464,14 @@ extern "C" gemm_status_t gemm_skinny_run_noalloc(const gemm_desc_t* desc, const 
              kNoAllocScratchBytes);
     return GEMM_ERR_WORKSPACE;
   }
-  CUtensorMap tW, tX;
+  CUtensorMap tW, tX, tD;
   if (!encode_map(&tW, desc->ab_dtype, B, desc->K, desc->N, 1, desc->ldb, 0, kBlockK, kSkinnyTileN) ||
       !encode_map(&tX, desc->ab_dtype, A, desc->K, desc->M, 1, desc->lda, 0, kBlockK, sp.m_pad))
+    return GEMM_ERR_CUDA;
+  const int64_t per16 = 16 / elem_bytes(desc->c_dtype);
+  const int n_full = static_cast<int>(desc->N / per16 * per16);  // D leaves through the copy engine in whole 16-byte units
+  if (n_full == 0) tD = tW;                                      // (never used)
+  else if (!encode_map(&tD, desc->c_dtype, C, n_full, desc->M, 1, desc->ldc, 0, 32, 16, /*swizzle=*/false))
     return GEMM_ERR_CUDA;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   // The array keeps whatever the previous call left: the status word must start at zero (the arrival words carry a
@@ -1475,6 +1491,7 @@ extern "C" gemm_status_t gemm_skinny_run_noalloc(const gemm_desc_t* desc, const 
   p.K = static_cast<int>(desc->K);
   p.idesc = make_idesc(desc->ab_dtype == GEMM_BF16, 0, 0, kSkinnyTileN, sp.m_pad);
   p.out_dtype = desc->c_dtype;
+  p.n_full = n_full;
   p.epilogue = desc->epilogue;
   p.bias_per_row = 0;  // (refused above; the tuning fields of desc->flags are ignored)
   p.alpha = alpha;
@@ -1488,7 +1505,7 @@ extern "C" gemm_status_t gemm_skinny_run_noalloc(const gemm_desc_t* desc, const 
   p.tag = run_tag(next_plan_identity() << 24, 0);
   p.timeout_ns = 2000ull * 1000000ull;
   st = static_cast<gemm_status_t>(
-      skinny_launch(p, tW, tX, dev, s, g_last_cuda_error, sizeof g_last_cuda_error, /*tall=*/false, /*early_launch=*/false));
+      skinny_launch(p, tW, tX, tD, dev, s, g_last_cuda_error, sizeof g_last_cuda_error, /*tall=*/false, /*early_launch=*/false));
   if (st != GEMM_OK || !sync_and_check) return st;
   uint32_t word = 0;
   e = cudaStreamSynchronize(s);

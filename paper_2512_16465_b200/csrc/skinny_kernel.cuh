@@ -181,6 +181,7 @@ struct SkinnyParams {
   unsigned long long timeout_ns;
   uint32_t debug_flags;   // bit 0: withhold one producer arrival (timeout test hook)
   int ab_fp8;             // operands are 8-bit floats (tcgen05 kind::f8f6f4)
+  int n_full;             // columns of D covered by whole 16-byte units of a row (those leave through the copy engine; unused when tall)
 };
 
 // Count this CTA in on a tile's arrival word and return how many had arrived before it.  A word whose tag is not this
@@ -205,18 +206,18 @@ template <bool kTall>
 __device__ __forceinline__ long long sk_index(const SkinnyParams& p, int small, int big) {
   return kTall ? static_cast<long long>(big) * p.ldc + small : static_cast<long long>(small) * p.ldc + big;
 }
-// Fetch the 16 C_in values (zeros when beta == 0).  Kept apart from sk_finish16 so that the loads can be issued
+// Fetch the 16 C_in values (zeros when beta == 0).  Kept apart from sk_values16 so that the loads can be issued
 // before other long-latency loads, and before any store to the same buffer (C_in and D are one buffer: a load
 // placed after a store could not be moved ahead of it and the rows would cost one round trip each).
 template <bool kTall>
-__device__ __forceinline__ void sk_load_cin16(const SkinnyParams& p, int s0, int big, float (&cin)[16]) {
+__device__ __forceinline__ void sk_load_cin16(const SkinnyParams& p, int s0, int big, bool big_ok, float (&cin)[16]) {
   const int small_extent = kTall ? p.N : p.M;
 #pragma unroll
   for (int j = 0; j < 16; ++j) cin[j] = 0.0f;
-  if (p.beta == 0.0f) return;
+  if (p.beta == 0.0f || !big_ok) return;
   const long long i0 = sk_index<kTall>(p, s0, big);
   const long long step = kTall ? 1 : p.ldc;
-  if (p.out_dtype == 2) {  // (the type switch stays outside the loop, see sk_finish16)
+  if (p.out_dtype == 2) {  // (the type switch stays outside the loop, see sk_values16)
     const float* c = static_cast<const float*>(p.c) + i0;
 #pragma unroll
     for (int j = 0; j < 16; ++j)
@@ -236,18 +237,20 @@ __device__ __forceinline__ void sk_load_cin16(const SkinnyParams& p, int s0, int
 // The switches on activation and output type sit outside the loops over the 16 values: this code runs once per
 // kernel, from a cold instruction cache, and a branch per value (each jumping over the inlined bodies of the other
 // cases) cost hundreds of cycles per value in instruction fetches.
+// sk_values16: bias, alpha / beta and the activation for 16 values along the short extent (`big_ok`: this thread's
+// index along the long extent exists; otherwise nothing is read and the values are never written).
 template <bool kTall>
-__device__ __forceinline__ void sk_finish16(const SkinnyParams& p, int s0, int big, const float (&acc)[16], const float (&cin)[16]) {
+__device__ __forceinline__ void sk_values16(const SkinnyParams& p, int s0, int big, bool big_ok, const float (&acc)[16],
+                                            const float (&cin)[16], float (&v)[16]) {
   const int small_extent = kTall ? p.N : p.M;
   const bool has_bias = (p.epilogue & 1) != 0;
   // the bias runs along N (the long extent unless kTall) or, per row, along M
   const bool bias_along_big = kTall ? p.bias_per_row != 0 : p.bias_per_row == 0;
-  float v[16];
   if (has_bias && !bias_along_big) {
 #pragma unroll
     for (int j = 0; j < 16; ++j) v[j] = (s0 + j < small_extent) ? __ldg(p.bias + s0 + j) : 0.0f;
   } else {
-    const float bias_big = has_bias ? __ldg(p.bias + big) : 0.0f;
+    const float bias_big = (has_bias && big_ok) ? __ldg(p.bias + big) : 0.0f;
 #pragma unroll
     for (int j = 0; j < 16; ++j) v[j] = bias_big;
   }
@@ -267,29 +270,91 @@ __device__ __forceinline__ void sk_finish16(const SkinnyParams& p, int s0, int b
 #pragma unroll
     for (int j = 0; j < 16; ++j) v[j] = silu(v[j]);
   }
+}
+// Plain stores of 16 finished values.  Tall: the 16 values are adjacent in a row of D (64 bytes as fp32), written as
+// 16-byte pieces when all 16 exist (rows start on 16-byte boundaries, s0 is a multiple of 16).  Otherwise: one
+// value per row of D.
+template <bool kTall>
+__device__ __forceinline__ void sk_store16(const SkinnyParams& p, int s0, int big, const float (&v)[16]) {
+  const int small_extent = kTall ? p.N : p.M;
   const long long i0 = sk_index<kTall>(p, s0, big);
   const long long step = kTall ? 1 : p.ldc;  // from one of the 16 values to the next
   if (p.out_dtype == 2) {
     float* d = static_cast<float*>(p.c) + i0;
+    if (kTall && s0 + 16 <= small_extent) {
+#pragma unroll
+      for (int j = 0; j < 16; j += 4) *reinterpret_cast<float4*>(d + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+      return;
+    }
 #pragma unroll
     for (int j = 0; j < 16; ++j)
       if (s0 + j < small_extent) d[j * step] = v[j];
   } else if (p.out_dtype == 0) {
     __nv_bfloat16* d = static_cast<__nv_bfloat16*>(p.c) + i0;
+    if (kTall && s0 + 16 <= small_extent) {
+      uint32_t w[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        w[j] = static_cast<uint32_t>(__bfloat16_as_ushort(__float2bfloat16_rn(v[2 * j]))) |
+               (static_cast<uint32_t>(__bfloat16_as_ushort(__float2bfloat16_rn(v[2 * j + 1]))) << 16);
+      *reinterpret_cast<uint4*>(d) = make_uint4(w[0], w[1], w[2], w[3]);
+      *reinterpret_cast<uint4*>(d + 8) = make_uint4(w[4], w[5], w[6], w[7]);
+      return;
+    }
 #pragma unroll
     for (int j = 0; j < 16; ++j)
       if (s0 + j < small_extent) d[j * step] = __float2bfloat16_rn(v[j]);
   } else {
     __half* d = static_cast<__half*>(p.c) + i0;
+    if (kTall && s0 + 16 <= small_extent) {
+      uint32_t w[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        w[j] = static_cast<uint32_t>(__half_as_ushort(__float2half_rn(v[2 * j]))) |
+               (static_cast<uint32_t>(__half_as_ushort(__float2half_rn(v[2 * j + 1]))) << 16);
+      *reinterpret_cast<uint4*>(d) = make_uint4(w[0], w[1], w[2], w[3]);
+      *reinterpret_cast<uint4*>(d + 8) = make_uint4(w[4], w[5], w[6], w[7]);
+      return;
+    }
 #pragma unroll
     for (int j = 0; j < 16; ++j)
       if (s0 + j < small_extent) d[j * step] = __float2half_rn(v[j]);
   }
 }
+// Not tall: a warp holds 16 rows x 32 adjacent columns of D, one column per lane.  Stored from registers that is 16
+// store instructions of 128 bytes each per warp, and issuing them took half a microsecond per 16 rows (measured: the
+// four chunks of a 64-row tile 3.6 us with the stores, 1.6 us without).  Instead the warp writes the slab row-major
+// into shared memory (`slab`, 16 x 32 elements) and one lane hands it to the copy engine as one tile store, which
+// clips at the matrix bounds; the warp goes on at once.  The copy engine writes whole 16-byte units only, so the
+// map ends at the last whole unit of a row (n_full) and the few columns behind it are stored from registers.
+// Called by all 32 lanes together.  The slab may lie over this chunk's parked values, which every lane has read by
+// the time of the first __syncwarp.
+__device__ __forceinline__ void sk_stage16(const SkinnyParams& p, const CUtensorMap* tmD, uint32_t slab, uint32_t lane, int s0, int n,
+                                           int col0, const float (&v)[16]) {
+  __syncwarp();
+  if (p.out_dtype == 2) {
+#pragma unroll
+    for (int j = 0; j < 16; ++j) st_shared_b32(slab + static_cast<uint32_t>(j) * 128u + lane * 4u, __float_as_uint(v[j]));
+  } else if (p.out_dtype == 0) {
+#pragma unroll
+    for (int j = 0; j < 16; ++j) st_shared_b16(slab + static_cast<uint32_t>(j) * 64u + lane * 2u, __bfloat16_as_ushort(__float2bfloat16_rn(v[j])));
+  } else {
+#pragma unroll
+    for (int j = 0; j < 16; ++j) st_shared_b16(slab + static_cast<uint32_t>(j) * 64u + lane * 2u, __half_as_ushort(__float2half_rn(v[j])));
+  }
+  fence_proxy_async_smem();
+  __syncwarp();
+  if (lane == 0 && col0 < p.n_full) {
+    tma_store_3d(tmD, slab, col0, s0, 0);
+    bulk_commit_group();
+  }
+  if (n >= p.n_full && n < p.N) sk_store16<false>(p, s0, n, v);
+}
 
 template <bool kTall, bool kCluster = false>
 __global__ void __launch_bounds__(kSkinnyThreads, 1)
-skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, const SkinnyParams p) {
+skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmD,
+                   const SkinnyParams p) {
   extern __shared__ uint8_t smem_raw[];
   griddep_launch_dependents();  // the next kernel's set-up may overlap this one; it waits below before touching global memory
   const uint32_t raw = smem_addr(smem_raw);
@@ -333,6 +398,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
     fence_mbar_init();
     prefetch_tensormap(&tmW);
     prefetch_tensormap(&tmX);
+    if (!kTall) prefetch_tensormap(&tmD);
   }
   if (warp == 1) {
     tmem_alloc<1>(smem_addr(const_cast<uint32_t*>(tmem_slot)), tmem_cols);
@@ -357,6 +423,22 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
   // (Only the warps that finish tiles ask: the producer's first load must not queue behind it.)
   uint32_t stale_status = 0u;
   if (warp >= 2) stale_status = *reinterpret_cast<volatile const uint32_t*>(p.status);
+  // Shared memory of the warps that finish tiles, 80 rows of 32 floats per warp (row v, lane l at + 128 v + 4 l): values
+  // fetched ahead of their use are parked here, and finished 16 x 32 slabs of D are staged here for the copy engine
+  // (chunk c0 in rows c0 ... c0 + 15, over the parked values of that chunk once they have been used).
+  const uint32_t fin_warp = base + bars_off + 16u * kMaxStages + 64u + (warp & 3u) * (80u * 128u);
+  // Finish 16 values per thread (rows m0 ... m0 + 15 of the short extent at this thread's index n along the long one)
+  // and write them: through the staged tile store, or directly when tall.  Called by whole warps.
+  auto emit16 = [&](int m0, int n, int col0, const float (&acc)[16], const float (&cin)[16]) {
+    const bool n_ok = n < big_extent;
+    float v[16];
+    sk_values16<kTall>(p, m0, n, n_ok, acc, cin, v);
+    if constexpr (kTall) {
+      if (n_ok) sk_store16<true>(p, m0, n, v);
+    } else {
+      sk_stage16(p, &tmD, fin_warp + static_cast<uint32_t>(m0) * 128u, lane, m0, n, col0, v);
+    }
+  };
 
   // The producer and MMA roles run warp-uniform (one elected lane issues), with the (tile, k-block) position and
   // the ring slot advanced incrementally: the single issuing thread must sustain one 18 KB stage every few hundred
@@ -472,6 +554,12 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
       const int seg_end = min(u_end, tile_u0 + sp.kbs);
       const uint32_t buf = seg & 1u;
       const int n = tile * kSkinnyTileN + n_local;
+      const int col0 = tile * kSkinnyTileN + static_cast<int>(q * 32u);
+      const bool n_ok = n < big_extent;
+      if (seg != 0u) {  // the copy engine has read the slabs staged for the previous tile before anything else is put there
+        if (lane == 0) bulk_wait_group_read<0>();
+        __syncwarp();
+      }
       const bool whole = (u == tile_u0) && (seg_end == tile_u0 + sp.kbs);  // this CTA owns the tile's whole K
       // contributors of a split tile: c_first reaches it at the end of its range (second slot) unless its range starts
       // exactly here; every later contributor starts inside the tile (first slot)
@@ -492,7 +580,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
       // same values in the same order, so the result does not depend on which one ran.
       bool early = false;
       const bool by_chunk = sp.m_pad > 16;  // parked value 16 b + j = chunk b of the other contributor (else: chunk 0 of contributor b)
-      const uint32_t park = base + bars_off + 16u * kMaxStages + 64u + (threadIdx.x - 64u) * 4u;  // value v lives at park + 512 v
+      const uint32_t park = fin_warp + lane * 4u;  // value v lives at park + 128 v
       if (!whole && (by_chunk ? c_last - c_first == 1 : c_last - c_first <= 3)) {
         // The leader looks at the arrival word again and again (about once a microsecond) until either all other
         // contributors have arrived -- for the CTA that holds the head of a tile they are always done before its own
@@ -528,16 +616,14 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
 #pragma unroll
             for (int j = 0; j < 16; ++j) pre[b][j] = __ldcg(part + j * kSkinnyTileN + n_local);
           }
-#pragma unroll
-          for (int j = 0; j < 16; ++j) cin0[j] = 0.0f;
-          if (n < big_extent) sk_load_cin16<kTall>(p, 0, n, cin0);
+          sk_load_cin16<kTall>(p, 0, n, n_ok, cin0);
 #pragma unroll
           for (int b = 0; b < 4; ++b) {
 #pragma unroll
-            for (int j = 0; j < 16; ++j) st_shared_b32(park + 512u * (16 * b + j), __float_as_uint(pre[b][j]));
+            for (int j = 0; j < 16; ++j) st_shared_b32(park + 128u * (16 * b + j), __float_as_uint(pre[b][j]));
           }
 #pragma unroll
-          for (int j = 0; j < 16; ++j) st_shared_b32(park + 512u * (64 + j), __float_as_uint(cin0[j]));
+          for (int j = 0; j < 16; ++j) st_shared_b32(park + 128u * (64 + j), __float_as_uint(cin0[j]));
         }
       }
       if (!mbar_wait_warp(tfull0 + 8u * buf, (seg >> 1) & 1u, w, (3u << 8) | buf, 64u)) break;
@@ -552,17 +638,15 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
           float accf[16], cin[16];
 #pragma unroll
           for (int j = 0; j < 16; ++j) accf[j] = __uint_as_float(acc[j]);
-          if (n < big_extent) {
-            sk_load_cin16<kTall>(p, c0, n, cin);
-            sk_finish16<kTall>(p, c0, n, accf, cin);
-          }
+          sk_load_cin16<kTall>(p, c0, n, n_ok, cin);
+          emit16(c0, n, col0, accf, cin);
         } else if (early) {
           float sum[16], cin[16];
 #pragma unroll
           for (int j = 0; j < 16; ++j) sum[j] = 0.0f;
 #pragma unroll
-          for (int j = 0; j < 16; ++j) cin[j] = __uint_as_float(ld_shared_b32(park + 512u * (64 + j)));
-          if (c0 != 0 && n < big_extent) sk_load_cin16<kTall>(p, c0, n, cin);
+          for (int j = 0; j < 16; ++j) cin[j] = __uint_as_float(ld_shared_b32(park + 128u * (64 + j)));
+          if (c0 != 0) sk_load_cin16<kTall>(p, c0, n, n_ok, cin);
 #pragma unroll
           for (int b = 0; b < 4; ++b) {
             // by contributor: b-th contributor; by chunk: the two contributors in order, the other one's chunk c0 / 16
@@ -571,12 +655,12 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
               const bool own = cc == static_cast<int>(blockIdx.x);
 #pragma unroll
               for (int j = 0; j < 16; ++j) {
-                const float other_v = __uint_as_float(ld_shared_b32(park + 512u * ((by_chunk ? c0 : 16 * b) + j)));
+                const float other_v = __uint_as_float(ld_shared_b32(park + 128u * ((by_chunk ? c0 : 16 * b) + j)));
                 sum[j] += own ? __uint_as_float(acc[j]) : other_v;
               }
             }
           }
-          if (n < big_extent) sk_finish16<kTall>(p, c0, n, sum, cin);
+          emit16(c0, n, col0, sum, cin);
         } else {
 #pragma unroll
           for (int j = 0; j < 16; ++j)
@@ -613,13 +697,13 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
               v[0][j] = __ldcg(q0 + (m0 + j) * kSkinnyTileN);
               v[1][j] = __ldcg(q1 + (m0 + j) * kSkinnyTileN);
             }
-            if (n < big_extent) sk_load_cin16<kTall>(p, m0, n, ci);
+            sk_load_cin16<kTall>(p, m0, n, n_ok, ci);
           };
           auto finish = [&](int m0, const float (&v)[2][16], const float (&ci)[16]) {
             float sum[16];
 #pragma unroll
             for (int j = 0; j < 16; ++j) sum[j] = (0.0f + v[0][j]) + v[1][j];
-            if (n < big_extent) sk_finish16<kTall>(p, m0, n, sum, ci);
+            emit16(m0, n, col0, sum, ci);
           };
           float va[2][16], vb[2][16], ca[16], cb[16];
           request(0, va, ca);
@@ -637,7 +721,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
             float sum[16], cin[16];
 #pragma unroll
             for (int j = 0; j < 16; ++j) sum[j] = 0.0f;
-            if (n < big_extent) sk_load_cin16<kTall>(p, m0, n, cin);  // in flight together with the partials
+            sk_load_cin16<kTall>(p, m0, n, n_ok, cin);  // in flight together with the partials
             // Contributor order, so that the result does not depend on arrival order; four contributors' loads are in
             // flight at a time.  The loads are unconditional (past the last contributor they repeat it) because loads
             // under a condition were scheduled one contributor, and one round trip to memory, after the other.
@@ -656,7 +740,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
                   for (int j = 0; j < 16; ++j) sum[j] += v[b][j];
                 }
             }
-            if (n < big_extent) sk_finish16<kTall>(p, m0, n, sum, cin);
+            emit16(m0, n, col0, sum, cin);
           }
           if (leader) p.counters[tile] = 0ull;  // a replay of this launch (same tag) must find no arrivals
         }
@@ -676,14 +760,16 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
     const uint32_t csize = static_cast<uint32_t>(sp.cluster);
     const uint32_t n_local = (warp & 3u) * 32u + lane;
     const int n = tile0 * kSkinnyTileN + static_cast<int>(n_local);
-    const bool finisher = warp >= 2 && n < big_extent;
+    const int col0 = tile0 * kSkinnyTileN + static_cast<int>((warp & 3u) * 32u);
+    const bool finisher = warp >= 2;
+    const bool n_ok = n < big_extent;
     float cin[16];
     cluster_arrive();
-    if (finisher && static_cast<int>(crank) * 16 < small_extent) sk_load_cin16<kTall>(p, static_cast<int>(crank) * 16, n, cin);
+    if (finisher && static_cast<int>(crank) * 16 < small_extent) sk_load_cin16<kTall>(p, static_cast<int>(crank) * 16, n, n_ok, cin);
     cluster_wait();
     if (finisher && *s_abort == 0u && stale_status == 0u) {
       for (int m0 = static_cast<int>(crank) * 16; m0 < small_extent; m0 += static_cast<int>(csize) * 16) {
-        if (m0 != static_cast<int>(crank) * 16) sk_load_cin16<kTall>(p, m0, n, cin);
+        if (m0 != static_cast<int>(crank) * 16) sk_load_cin16<kTall>(p, m0, n, n_ok, cin);
         float sum[16];
 #pragma unroll
         for (int j = 0; j < 16; ++j) sum[j] = 0.0f;
@@ -695,12 +781,13 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
 #pragma unroll
           for (int j = 0; j < 16; ++j) sum[j] += v[j];
         }
-        sk_finish16<kTall>(p, m0, n, sum, cin);
+        emit16(m0, n, col0, sum, cin);
       }
     }
     cluster_arrive();  // nobody's shared memory may go away while a peer still reads it
     cluster_wait();
   }
+  if (!kTall && warp >= 2 && lane == 0) bulk_wait_group_read<0>();  // staged slabs are read; the writes complete with the grid
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
@@ -710,8 +797,8 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
 }
 
 // Launch.  Returns a gemm_status_t value (0 = ok, 7 = CUDA failure).
-// `tall` selects the mirrored addressing (tW then maps A, tX maps B).
-inline int skinny_launch(const SkinnyParams& p, const CUtensorMap& tW, const CUtensorMap& tX, int device, cudaStream_t stream,
+// `tall` selects the mirrored addressing (tW then maps A, tX maps B; tD, the store map of D, is then unused).
+inline int skinny_launch(const SkinnyParams& p, const CUtensorMap& tW, const CUtensorMap& tX, const CUtensorMap& tD, int device, cudaStream_t stream,
                          char* err, size_t err_len, bool tall, bool early_launch) {
   const bool cluster = p.plan.cluster > 1;
   const void* kern = tall ? (cluster ? reinterpret_cast<const void*>(skinny_gemm_kernel<true, true>) : reinterpret_cast<const void*>(skinny_gemm_kernel<true, false>))
@@ -741,8 +828,8 @@ inline int skinny_launch(const SkinnyParams& p, const CUtensorMap& tW, const CUt
     }
     cfg.attrs = attr;
     cfg.numAttrs = na;
-    if (tall) e = cluster ? cudaLaunchKernelEx(&cfg, skinny_gemm_kernel<true, true>, tW, tX, p) : cudaLaunchKernelEx(&cfg, skinny_gemm_kernel<true, false>, tW, tX, p);
-    else e = cluster ? cudaLaunchKernelEx(&cfg, skinny_gemm_kernel<false, true>, tW, tX, p) : cudaLaunchKernelEx(&cfg, skinny_gemm_kernel<false, false>, tW, tX, p);
+    if (tall) e = cluster ? cudaLaunchKernelEx(&cfg, skinny_gemm_kernel<true, true>, tW, tX, tD, p) : cudaLaunchKernelEx(&cfg, skinny_gemm_kernel<true, false>, tW, tX, tD, p);
+    else e = cluster ? cudaLaunchKernelEx(&cfg, skinny_gemm_kernel<false, true>, tW, tX, tD, p) : cudaLaunchKernelEx(&cfg, skinny_gemm_kernel<false, false>, tW, tX, tD, p);
   }
   if (e != cudaSuccess) {
     snprintf(err, err_len, "skinny launch: %s", cudaGetErrorName(e));
