@@ -1084,7 +1084,7 @@ gemm_status_t gemm_plan_schedule(gemm_plan_t plan, gemm_work_item_t* items, size
         const int seg_end = std::min(u_end, tile_u0 + s.kbs);
         const bool whole = u == tile_u0 && seg_end == tile_u0 + s.kbs;
         // position among the tile's contributors (cluster mode: the rank in the cluster)
-        const int slice = whole ? -1 : (s.cluster > 1 ? c % s.cluster : c - sk_owner(tile_u0, s.units_q, s.units_r));
+        const int slice = whole ? -1 : (s.cluster > 1 ? c % s.cluster : c - sk_unit_owner(s, tile_u0));
         emit(c, 0, plan->skinny_tall ? tile : 0, plan->skinny_tall ? 0 : tile, u - tile_u0, seg_end - tile_u0, slice);
         u = seg_end;
       }

@@ -58,6 +58,8 @@ struct SkinnyPlan {
   int stage_bytes;       // atoms x (16 KB of W + m_pad * 128 bytes of X)
   int smem_bytes;
   int cluster;           // > 1: CTAs per output tile, launched as one thread-block cluster (hand-over through shared memory)
+  int group_tiles;       // t > 0: every t consecutive tiles are shared by t + 1 CTAs (see sk_group_begin); units_q / units_r unused
+  int group_lead;        // work units by which a tile's tail is done before the CTA holding its head is
   int max_contributors;  // upper bound on CTAs touching one tile
   size_t counters_bytes; // arrival counters at the head of the workspace: n_tiles x u64, padded to 256 bytes
   size_t workspace_bytes;  // partial tiles behind them: grid * 2 slots of [m_pad][128] floats
@@ -68,6 +70,22 @@ __host__ __device__ inline int sk_begin(int c, int q, int r) { return c * q + (c
 __host__ __device__ inline int sk_owner(int u, int q, int r) {
   const int head = r * (q + 1);
   return u < head ? u / (q + 1) : r + (u - head) / q;
+}
+
+// Grouped ranges.  t tiles (t * kbs units) are shared by t + 1 CTAs in unit order: CTA 0 computes the head of tile 0,
+// CTA i the tail of tile i - 1 and then the head of tile i, CTA t the tail of tile t - 1.  Every tile has two
+// contributors, and the one holding the head finishes it from the other's partial tile, which it fetches ahead of
+// time as soon as the arrival word says the partial is there (the cheap hand-over of the stream-K kernel).  That
+// needs the tail to be done, published and fetched before the head is: with equal ranges it holds for every
+// tile but the last, whose tail is CTA t's whole range and ends with everybody else's.  So CTA t takes
+// t * (kbs - lead) / (t + 1) units, `lead` units short of an equal share plus its own head start, and the other t
+// CTAs share the rest equally.  Returns the first unit, relative to the group, of CTA i (i = t + 1: the total).
+__host__ __device__ inline int sk_group_begin(int kbs, int t, int lead, int i) {
+  const int total = t * kbs;
+  if (i > t) return total;
+  const int rest = total - t * (kbs - lead) / (t + 1);
+  const int q = rest / t, r = rest - q * t;
+  return i * q + (i < r ? i : r);
 }
 
 // max_clusters (may be null): max_clusters[c] = clusters of c CTAs of this kernel that the device holds at once, c = 2 ... 8
@@ -97,11 +115,14 @@ inline bool skinny_make_plan(SkinnyPlan* s, int M, int N, int K, int sm_count, i
   //      the partial tiles added up through shared memory (about 2 us), when all clusters fit on the device at once and
   //      fill six tenths of it (any small problem: there the alternative is one CTA per unit);
   //  (3) else c > 8 CTAs per tile with c dividing the tile's units (workspace path, but no CTA contributes to two tiles),
-  //      whole tiles on half of the SMs for a mid-sized problem, or several whole tiles per CTA;
+  //      three tiles per four CTAs (grouped ranges, see sk_group_begin) when the tiles alone would keep between half
+  //      and two thirds of the SMs busy, or several whole tiles per CTA;
   //  (4) else equal contiguous ranges over all SMs, straddling the tiles (the large problems, whose tail does not matter).
   // Measured against the plain rule (4) on shapes with short extents 8 ... 64: 64 x 4096 x 4096 22.3 -> 12.0 us,
   // 64 x 8192 x 8192 36.0 -> 27.7, 64 x 4096 x 14336 34.4 -> 24.3, 8 x 4096 x 4096 13.3 -> 10.7; the large ones unchanged.
   s->cluster = 1;
+  s->group_tiles = 0;
+  s->group_lead = 0;
   if (align) {
     int best = 0;
     const bool small_problem = s->total_units < 2ll * sm_count;
@@ -121,9 +142,27 @@ inline bool skinny_make_plan(SkinnyPlan* s, int M, int N, int K, int sm_count, i
       for (int c = clusters ? 9 : 3; c <= s->kbs; ++c)
         if (s->kbs % c == 0 && static_cast<long long>(s->n_tiles) * c <= sm_count && s->n_tiles * c * 5 >= sm_count * 4)
           best = best > s->n_tiles * c ? best : s->n_tiles * c;
-      // (about a hundred SMs saturate the memory system; fewer pay in streaming time what they save in hand-overs once the
-      // streamed operand exceeds some 160 MB)
-      // (the wider the short extent, the dearer the hand-over through the workspace: 12 us at 64 against 5 at 16)
+      // About a hundred SMs saturate the memory system; 74 ... 100 tiles with one CTA each leave a quarter of the streaming
+      // rate unused, and equal ranges over all SMs put three contributors on most tiles, all finishing at the same time
+      // (the dear hand-over: publish, count, the last one fetches and adds, 8 ... 13 us at a short extent of 64).  Grouped
+      // ranges use a third more CTAs than tiles and keep the cheap hand-over on every tile.  The lead (in work units) is
+      // what a tail holder needs to publish its partial tile plus what the head holder needs to notice and fetch it
+      // (measured 4 ... 6.5 us from 16 to 64 rows), at the rate a CTA streams: its share of some 6.5 TB/s, or what one
+      // SM takes in alone (87 GB/s measured on 80 CTAs).
+      if (!best && 2 * s->n_tiles >= sm_count && s->n_tiles + (s->n_tiles + 2) / 3 <= sm_count && s->kbs >= 32) {
+        const int t = 3, left = s->n_tiles % t;
+        const int grid = (s->n_tiles / t) * (t + 1) + (left ? left + 1 : 0);
+        const double unit_w = s->atoms * (kSkinnyTileN * 128.0), unit_all = unit_w + s->atoms * (s->m_pad * 128.0);
+        const double hbm = 6.5e6 / (grid * unit_w), one_sm = 87.0e3 / unit_all;  // work units per microsecond
+        const double lead_us = 3.5 + 0.75 * (s->m_pad / 16);
+        int lead = static_cast<int>(lead_us * (hbm < one_sm ? hbm : one_sm) + 0.999);
+        lead = lead < 2 ? 2 : (lead > s->kbs / 4 ? s->kbs / 4 : lead);
+        s->group_tiles = t;
+        s->group_lead = lead;
+        best = grid;
+      }
+      // (short K: whole tiles on half of the SMs, as long as the streamed operand is small; the wider the short extent, the
+      // dearer the alternative)
       const double whole_tiles_up_to_mb = 160.0 + (s->m_pad > 32 ? (s->m_pad - 32) * 6.0 : 0.0);
       if (!best && s->n_tiles <= sm_count && 2 * s->n_tiles >= sm_count && streamed_mb <= whole_tiles_up_to_mb) best = s->n_tiles;
       if (!best && s->total_units / s->grid < 64)
@@ -146,10 +185,18 @@ inline bool skinny_make_plan(SkinnyPlan* s, int M, int N, int K, int sm_count, i
   s->smem_bytes = fixed + stages * s->stage_bytes;
   if (s->smem_bytes > max_smem) return false;
   const int per_cta = s->units_q;  // >= 1
-  s->max_contributors = (s->kbs + per_cta - 1) / per_cta + 1;
+  s->max_contributors = s->group_tiles ? 2 : (s->kbs + per_cta - 1) / per_cta + 1;
   s->counters_bytes = (static_cast<size_t>(s->n_tiles) * 8 + 255) / 256 * 256;
   s->workspace_bytes = static_cast<size_t>(s->grid) * 2 * kSkinnyTileN * s->m_pad * 4;
   if (s->cluster > 1) s->counters_bytes = s->workspace_bytes = 0;  // nothing leaves the cluster
+  // A short extent of 64 takes single slices above because four double stages do not fit.  That choice was measured with
+  // every SM streaming; a grid that leaves SMs idle has fewer requests in flight and gains more from two adjacent
+  // pieces per weight row than it loses with a ring of three (64 x 10240 x 8192 on 80 CTAs 41.7 -> 39.3 us,
+  // 64 x 6144 x 6144 on 96 20.4 -> 19.9, 64 x 4096 x 4096 on 128 11.9 -> 11.6; on all 148 it costs 1 %).
+  if (!forced_atoms && !forced_stages && s->atoms == 1 && s->grid < sm_count && K >= 16 * kblk && (max_smem - fixed) / (2 * slice_bytes) >= 3) {
+    SkinnyPlan two;
+    if (skinny_make_plan(&two, M, N, K, sm_count, 0, max_smem, 2, kblk, align, max_clusters, clusters) && two.grid < sm_count) *s = two;
+  }
   return true;
 }
 
@@ -160,7 +207,30 @@ __host__ __device__ inline int sk_cta_begin(const SkinnyPlan& s, int cta) {
     const int tile = cta / s.cluster, rank = cta - tile * s.cluster;
     return tile * s.kbs + sk_begin(rank, s.kbs / s.cluster, s.kbs % s.cluster);
   }
+  if (s.group_tiles > 0) {
+    if (cta >= s.grid) return static_cast<int>(s.total_units);
+    const int t = s.group_tiles, full = s.n_tiles / t;  // `full` whole groups, then one group of the n_tiles % t tiles left
+    const int g = cta / (t + 1);
+    if (g < full) return g * t * s.kbs + sk_group_begin(s.kbs, t, s.group_lead, cta - g * (t + 1));
+    return full * t * s.kbs + sk_group_begin(s.kbs, s.n_tiles - full * t, s.group_lead, cta - full * (t + 1));
+  }
   return sk_begin(cta, s.units_q, s.units_r);
+}
+// The CTA whose range holds work unit u (equal ranges or grouped ranges; not used in cluster mode).
+__host__ __device__ inline int sk_unit_owner(const SkinnyPlan& s, int u) {
+  if (s.group_tiles > 0) {
+    const int t = s.group_tiles, full = s.n_tiles / t;
+    int g = u / (t * s.kbs), tg = t;
+    if (g >= full) {
+      g = full;
+      tg = s.n_tiles - full * t;
+    }
+    const int rel = u - g * t * s.kbs;
+    int i = 0;
+    while (i < tg && sk_group_begin(s.kbs, tg, s.group_lead, i + 1) <= rel) ++i;
+    return g * (t + 1) + i;
+  }
+  return sk_owner(u, s.units_q, s.units_r);
 }
 
 struct SkinnyParams {
@@ -377,7 +447,6 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
   volatile uint32_t* s_early = tmem_slot + 3;  // two words: a CTA has at most two partial segments (its first and its last)
   const WaitCtx w{s_abort, p.status, p.timeout_ns};
   // This CTA's contiguous range of work units (computed while the barriers and tensor memory are being set up).
-  const int uq = sp.units_q, ur = sp.units_r;
   const int u_begin = sk_cta_begin(sp, static_cast<int>(blockIdx.x));
   const int u_end = sk_cta_begin(sp, static_cast<int>(blockIdx.x) + 1);
   const int tile0 = u_begin / sp.kbs;
@@ -563,9 +632,9 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
       const bool whole = (u == tile_u0) && (seg_end == tile_u0 + sp.kbs);  // this CTA owns the tile's whole K
       // contributors of a split tile: c_first reaches it at the end of its range (second slot) unless its range starts
       // exactly here; every later contributor starts inside the tile (first slot)
-      const int c_first = whole ? 0 : sk_owner(tile_u0, uq, ur);
-      const int c_last = whole ? 0 : sk_owner(tile_u0 + sp.kbs - 1, uq, ur);
-      const int first_slot = (whole || sk_begin(c_first, uq, ur) == tile_u0) ? 0 : 1;
+      const int c_first = whole ? 0 : sk_unit_owner(sp, tile_u0);
+      const int c_last = whole ? 0 : sk_unit_owner(sp, tile_u0 + sp.kbs - 1);
+      const int first_slot = (whole || sk_cta_begin(sp, c_first) == tile_u0) ? 0 : 1;
       auto partial_of = [&](int c) {
         return p.partials + (static_cast<size_t>(c) * 2 + (c == c_first ? first_slot : 0)) * (kSkinnyTileN * sp.m_pad);
       };

@@ -125,6 +125,15 @@ EXACT_CASES = [
     ("skinny_m64_two_contributors", 64, 20480, 2048, dict(beta=1.0, epi=bg.EPI_BIAS), dict(variant=VS)),
     ("tall_n48_two_contributors", 20480, 48, 2048, dict(cd=wl.BF16, beta=1.0, ldc=56), dict(variant=VS)),
     ("skinny_m33_two_contributors_fp8", 33, 20000, 4096, dict(ab=wl.FP8_E4M3, cd=wl.F16), dict(variant=VS)),
+    # 74 ... 100 tiles: three tiles per four CTAs, the tail of every tile handed to the CTA that holds its head
+    ("grouped_m64_beta_bias", 64, 10240, 4096, dict(beta=1.0, epi=bg.EPI_BIAS), dict(variant=VS)),
+    ("grouped_m8_bf16_ragged_columns", 8, 11003, 4104, dict(cd=wl.BF16, ldc=11008), dict(variant=VS)),
+    ("grouped_tall_n40_f16", 12288, 40, 4096, dict(ab=wl.F16, cd=wl.F16, beta=1.0), dict(variant=VS)),
+    ("grouped_fp8_m16", 16, 9600, 8192, dict(ab=wl.FP8_E4M3), dict(variant=VS)),
+    # results leave through staged tile stores in whole 16-byte units; the columns behind the last whole unit from registers
+    ("skinny_columns_not_a_multiple_of_16_bytes_bf16", 24, 1003, 520, dict(cd=wl.BF16, ldc=1008, epi=bg.EPI_BIAS), dict(variant=VS)),
+    ("skinny_columns_not_a_multiple_of_16_bytes_f32", 64, 1001, 1032, dict(beta=1.0, ldc=1004), dict(variant=VS)),
+    ("skinny_three_columns", 8, 3, 520, dict(ldc=4), dict(variant=VS)),
     ("cluster_no_early_launch", 8, 4096, 4096, dict(beta=1.0), dict(variant=VS, no_early_launch=True)),
     ("no_early_launch_1cta", 264, 328, 200, {}, dict(variant=V1, tile_n=128, no_early_launch=True)),
     ("no_early_launch_skinny", 8, 256, 4096, dict(beta=1.0), dict(variant=VS, no_early_launch=True)),

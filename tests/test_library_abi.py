@@ -137,8 +137,9 @@ def test_stream_k_plan_geometry():
     assert grid(64, 4096, 4096) in (96, 128)  # 32 tiles: four CTAs per tile, as clusters that hand over through shared memory
     assert grid(16, 4096, 4096) in (96, 128)
     assert grid(64, 14336, 16384) == 112      # one whole tile per CTA: more than two thirds of the SMs, any size
-    assert grid(16, 11008, 16384) == 148      # 86 whole tiles would starve the memory system on 360 MB: equal ranges on all SMs
-    assert grid(64, 12288, 4096) == 96        # 96 tiles: whole tiles on two thirds of the SMs (100 MB streamed)
+    assert grid(16, 11008, 16384) == 115      # 86 tiles: three tiles per four CTAs (28 such groups, two tiles left to three CTAs)
+    assert grid(64, 12288, 4096) == 128       # 96 tiles: 32 groups of four CTAs
+    assert grid(64, 12288, 1024) == 96        # short K: whole tiles
     assert grid(64, 5120, 5120) in (80, 120)  # 40 tiles: clusters of three (or two)
     assert grid(64, 8192, 8192) == 128        # 64 tiles: clusters of two
     assert grid(64, 9472, 4096) in (74, 148)  # 74 tiles: clusters of two on all SMs when they all fit

@@ -163,7 +163,10 @@ def test_stream_k_units_once(short, long_, K):
             assert (np.diff(sched[:, CTA]) >= 0).all() and len(np.unique(sched[:, CTA])) == info["grid"]
             per = np.zeros(info["grid"], int)
             np.add.at(per, sched[:, CTA], sched[:, K1] - sched[:, K0])
-            assert per.max() - per.min() <= 1                                   # equal streaming work per SM
+            if per.max() - per.min() > 1:
+                # grouped ranges (three tiles per four CTAs): two contributors on every tile, the last CTA of a group shorter
+                assert info["grid"] == 4 * (tiles // 3) + (tiles % 3 + 1 if tiles % 3 else 0) and info["split"] == 2
+                assert all((tile_ix == t).sum() == 2 for t in range(tiles)) and per.max() <= 1.2 * per.mean()
             # contributors of a split tile are numbered 0, 1, 2 ... in CTA order; a whole tile has one item marked -1
             for t in range(tiles):
                 sl = sched[tile_ix == t, SLICE]
@@ -190,3 +193,33 @@ def test_cluster_mode_of_stream_k():
     for M, N, K in ((8, 28672, 8192), (8, 10000, 2136), (40, 10240, 8200), (8, 11000, 8200), (33, 10880, 6144)):
         i = info(M, N, K)
         assert i["cluster_size"] == 1 and i["workspace_bytes"] > 0, (M, N, K, i)
+
+
+@pytest.mark.parametrize("short", [8, 16, 40, 64])
+@pytest.mark.parametrize("long_,K", [(10240, 8192), (11008, 4096), (12288, 4096), (9600, 16384), (12800, 4096), (11000, 8200)])
+def test_grouped_ranges_of_stream_k(short, long_, K):
+    """74 ... 100 tiles: every three tiles are shared by four CTAs (the tiles left over by one more CTA than tiles), each
+    tile by two, and the CTA that holds a tile's tail is through with it before the CTA that holds its head has
+    finished its own range -- by a margin, so that the head holder can fetch the partial tile ahead of its own end."""
+    for tall in (False, True):
+        M, N = (long_, short) if tall else (short, long_)
+        info, sched = plan_and_schedule(M, N, K, bg.make_flags(VS), options=bg.OPT_STREAMK_WORKSPACE)
+        tiles = -(-long_ // 128)
+        stages = -(-K // info["tile_k"])
+        assert 74 <= tiles <= 100
+        assert info["grid"] == 4 * (tiles // 3) + (tiles % 3 + 1 if tiles % 3 else 0), info
+        assert info["split"] == 2 and info["cluster_size"] == 1 and info["workspace_bytes"] > 0
+        tile_ix = sched[:, ROW] if tall else sched[:, COL]
+        per = np.zeros(info["grid"], int)
+        np.add.at(per, sched[:, CTA], sched[:, K1] - sched[:, K0])
+        first = np.concatenate([[0], np.cumsum(per)])        # first unit of every CTA
+        margins = []
+        for t in range(tiles):
+            rows = sched[tile_ix == t]
+            assert len(rows) == 2 and list(rows[:, SLICE]) == [0, 1]
+            head, tail = rows[0], rows[1]
+            assert head[K0] == 0 and head[K1] == tail[K0] and tail[K1] == stages and head[CTA] + 1 == tail[CTA]
+            # the head is the end of its CTA's range, the tail the start of the next CTA's
+            assert t * stages + head[K1] == first[head[CTA] + 1]
+            margins.append(per[head[CTA]] - (tail[K1] - tail[K0]))
+        assert min(margins) >= 2 and per.max() <= 1.2 * per.mean(), (min(margins), per.max(), per.mean())
