@@ -218,8 +218,10 @@ size_t gemm_workspace_bytes(gemm_plan_t plan);
  * has a bias.  C is read only when beta != 0, and only the M x N elements of D (per batch) are written: row padding
  * (ldc > N) and gaps between batches keep their contents, so D may be a column block of a wider matrix.  workspace: device
  * memory of at least gemm_workspace_bytes(plan) bytes, 16-byte aligned (may be NULL when
- * that is 0), with any contents: the hand-shake words at its head carry a tag that is new with every run, so whatever
- * the memory held before reads as "nothing yet".  Runs of one plan may overlap on the GPU (several streams, several host
+ * that is 0), with any contents: the hand-shake words at its head carry a 48-bit tag that is new with every run and
+ * spread pseudo-randomly over its bits, so whatever the memory held before reads as "nothing yet" (a stale 64-bit word
+ * passes for this run's only if 48 of its bits equal that one value; a caller who wants certainty zeroes the workspace
+ * once after allocating it).  Runs of one plan may overlap on the GPU (several streams, several host
  * threads) as long as runs that overlap use DIFFERENT workspaces; they share only the status word, which then reports
  * a timeout of any of them.  Runs that share a workspace must be ordered (one stream, or events).  alpha and beta are
  * host scalars.  The call only fetches or encodes tensor maps on the host (a plan remembers the maps of the operand

@@ -9,6 +9,7 @@
 
 #include <algorithm>
 #include <atomic>
+#include <chrono>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
@@ -16,6 +17,7 @@
 #include <mutex>
 #include <new>
 #include <queue>
+#include <random>
 #include <utility>
 #include <vector>
 
@@ -809,8 +811,39 @@ uint64_t next_plan_identity() {
   while (id == 0);
   return id;
 }
-// Tag of run number `run` of a plan: 48 bits, never 0 because the identity is not.
-uint64_t run_tag(uint64_t tag_base, unsigned long long run) { return tag_base | (run & 0xFFFFFFull); }
+// Tag of run number `run` of a plan: 48 bits, never 0.  The pair (identity, run number) is unique, but as a bit pattern
+// it is a small number next to zeros, and so is much of what a recycled workspace holds: 16-bit floats of small integer
+// value between zeros read, as a 64-bit word, exactly like "identity 0x5b, run 0, count x" (found by a randomised
+// sweep: one tile of one problem in 240 was never finished because a stale word passed for this run's arrival
+// word).  So the pair goes through a bijection of the 48-bit numbers that spreads it over all bits -- distinct pairs
+// still give distinct tags -- after an exclusive-or with a per-process random number, so that words left by another
+// process that used this library do not repeat this process's tags either.  What remains is the chance that arbitrary
+// stale data equals one given 48-bit value.
+uint64_t tag_salt() {
+  static const uint64_t salt = [] {
+    uint64_t s = 0x9E3779B97F4A7C15ull ^ static_cast<uint64_t>(std::chrono::steady_clock::now().time_since_epoch().count());
+    s ^= static_cast<uint64_t>(std::chrono::system_clock::now().time_since_epoch().count()) << 17;
+    s ^= reinterpret_cast<uintptr_t>(&s) << 7;
+    try {
+      std::random_device rd;
+      s ^= (static_cast<uint64_t>(rd()) << 32) ^ rd();
+    } catch (...) {
+    }
+    return s & 0xFFFFFFFFFFFFull;
+  }();
+  return salt;
+}
+uint64_t run_tag(uint64_t tag_base, unsigned long long run) {
+  const uint64_t mask = 0xFFFFFFFFFFFFull;
+  uint64_t x = ((tag_base | (run & 0xFFFFFFull)) ^ tag_salt()) & mask;
+  // every step is a bijection of the 48-bit numbers (exclusive-or with a right shift; multiplication by an odd number)
+  x ^= x >> 23;
+  x = (x * 0x2127599BF4325ull) & mask;
+  x ^= x >> 19;
+  x = (x * 0x880355F21E6D1ull) & mask;
+  x ^= x >> 25;
+  return x ? x : 0x5DEECE66Dull;  // (the one pair that maps to 0 shares this tag with one other pair)
+}
 
 // gemm_plan proper.  use_cache: take the tuning fields gemm_tune remembered for this shape (when the caller set none);
 // *cache_used tells whether that happened.

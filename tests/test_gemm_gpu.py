@@ -649,6 +649,41 @@ def test_workspace_needs_no_initialisation(fill):
         plan.close()
 
 
+def test_stale_words_that_look_like_small_counters_are_not_this_runs():
+    """What a recycled workspace typically holds are small numbers next to zeros (16-bit floats of small integer value, old
+    counters).  A run's tag must not be such a pattern: with tags built as `plan number << 24 | run number`, a stale word
+    like 0x00005b00'00000007 passed for "plan 0x5b, run 0, seven arrivals" and one tile of a run was never finished.  Every
+    word of the workspace is filled with k << 40 | count for k = 1 ... 400 in turn (the plans of a process are numbered from
+    one), with a count that would make the first arrival look like the last or like one of many; each run must give the
+    result of the run on a zeroed workspace."""
+    cases = [(int_workload("stale_stream_k", 8, 11000, 4200, beta=1.0), 0, 3),   # grouped ranges: two contributors per tile
+             (int_workload("stale_tail_split", 256, 256, 16384), 0, 0)]          # split-tile flags of the dense kernels
+    for w, flags, count in cases:
+        inputs = wl.make_inputs(w)
+        A, B = H.to_device(inputs["A"], w.ab_dtype), H.to_device(inputs["B"], w.ab_dtype)
+        plan = bg.Plan(H.desc_of(w, flags))
+        assert plan.workspace_bytes > 0
+        ws = torch.zeros(plan.workspace_bytes // 8, dtype=torch.int64, device="cuda")
+        c0 = H.to_device(inputs["C"], w.c_dtype) if inputs["C"] is not None else torch.zeros(w.elems_c(), dtype=H._TORCH_DT[w.c_dtype], device="cuda")
+        want = None
+        runs = 0                                        # (the run number was the low half of such a tag)
+        for k in range(0, 401):
+            for shift in ((40, 24) if k else (0,)):     # the stream-K word (tag << 16 | count) and the flag word (the tag itself) of that scheme
+                ws.fill_((k << shift) | (runs << (shift - 24)) | (count if shift == 40 else 0) if k else 0)
+                C = c0.clone()
+                plan.run(A, B, C, alpha=w.alpha, beta=w.beta, workspace=ws.view(torch.uint8))
+                runs += 1
+                if want is None:
+                    assert plan.status() == bg.OK
+                    want = C.clone()
+                    reports = H.check_blocks(w, inputs, H.to_host_bits(C, w.c_dtype), H.default_blocks(w))
+                    assert all(r["bit_identical"] == 1.0 for r in reports), w.name
+                else:
+                    assert torch.equal(C.view(torch.int16 if C.element_size() == 2 else torch.int32), want.view(torch.int16 if C.element_size() == 2 else torch.int32)), (w.name, k, shift)
+        assert plan.status() == bg.OK
+        plan.close()
+
+
 def test_status_word_forms():
     """gemm_plan_status_async enqueues the read and waits for nothing; gemm_plan_status_result reports it once the
     caller has waited for the stream; gemm_plan_status_stream waits for one stream; gemm_plan_status for the device.
