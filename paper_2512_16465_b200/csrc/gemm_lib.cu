@@ -371,16 +371,23 @@ bool set_scheduler_divisors(DenseParams& p) {
 // Tail split of the double-buffered dense kernels (on request, GEMM_FLAG_TAIL_SPLIT): when the tiles left over after the
 // full waves occupy at most half of the CTAs (pairs), each of them is cut into this many K slices, one per CTA (pair); the slice that
 // starts at K = 0 adds the others' raw accumulators from the workspace and finishes the tile.  1 = no split.
-int tail_split(long long tiles, int units, int num_kb, const gemm_desc_t& d, int bn = 0) {
+int tail_split(long long tiles, int units, int num_kb, const gemm_desc_t& d, int bn, int cg, int atoms) {
   if (bn > 256) return 1;  // (the partial-tile layout and the flag protocol are written for two accumulator buffers)
   if ((d.flags & (GEMM_FLAG_A_LOWER | GEMM_FLAG_A_UPPER | GEMM_FLAG_D_LOWER | GEMM_FLAG_D_UPPER)) || d.structure) return 1;
   const long long rem = tiles % units;
   if (rem == 0 || rem * 2 > units) return 1;
   if (tiles / units >= 8) return 1;  // many full waves: the last one is a few per cent at most; keep the plain kernel
-  // The reducing CTA reads one partial tile per further slice (about 5000 cycles each), a ring stage takes about 1000:
-  // beyond sqrt(stages / 5) slices the reading costs more than the shorter main loop saves.
-  int by_length = 2;
-  while ((by_length + 1) * (by_length + 1) * 5 <= num_kb && by_length < 16) ++by_length;
+  // s slices shorten a tile's main loop to 1 / s of its T cycles and make the reducing CTA read s - 1 partial tiles of
+  // R cycles each (128 x bn floats at the 58 B/clk one SM takes from L2; the flags of all slices are polled together):
+  // T / s + (s - 1) R is least at s = sqrt(T / R).  T per 128-byte K slice: the operand feed at the same rate or the
+  // tensor pipe, whichever is slower.  (Measured, us at the old rule's count -> at this one's: 384 x 384 x 8192 18.0 at 3
+  // -> 14.8 at 6, 256 x 512 x 8192 18.1 at 3 -> 14.5 at 9, 256 x 256 x 32768 27.0 at 7 -> 21.7 at 16; the old rule
+  // charged 5000 cycles per partial tile, from before the flags were polled together.)
+  const double width = bn > 0 ? bn : 128;
+  const double per_slice = std::max((128.0 + width / cg) * 128.0 / 58.0, 4.0 * (width / 2.0) / 0.8);
+  const double read_partial = 128.0 * width * 4.0 / 58.0;
+  int by_length = static_cast<int>(std::lround(std::sqrt(static_cast<double>(num_kb) * atoms * per_slice / read_partial)));
+  by_length = std::max(2, std::min(by_length, 16));
   int split = static_cast<int>(std::min<long long>(units / rem, by_length));
   split = std::min(split, num_kb / 4);  // a slice of fewer than four ring stages is all pipeline fill
   split = std::max(split, 1);
@@ -408,9 +415,13 @@ double estimate_dense_cycles(const gemm_desc_t& d, int sm_count, int variant, in
   const long long tiles = tri_tile_count(d_tri_of(d), rows_tile, bn, d.M, d.N) * d.batch_count;
   const double kblocks = static_cast<double>(ceil_div(d.K, kblk_of(d.ab_dtype)));  // 128-byte slices: same pipe time for either width
   double waves = static_cast<double>((tiles + units - 1) / units);
+  double handover = 0.0;
   if (!wide) {  // a thinly filled last wave is split along K (two slices per stage assumed, as plan_dense will choose for long K)
-    const int split = tail_split(tiles, units, static_cast<int>(kblocks) / 2, d, bn);
-    if (split > 1) waves += 1.0 / split - 1.0 + 0.08;  // + hand-over of the partial accumulators
+    const int split = tail_split(tiles, units, static_cast<int>(kblocks) / 2, d, bn, cg, 2);
+    if (split > 1) {
+      waves += 1.0 / split - 1.0;
+      handover = (split - 1) * (128.0 * bn * 4.0 / 58.0) + 2500.0;  // the reducing CTA reads the other slices' accumulators
+    }
   }
   // tensor pipe: one 128 x bn x 16 MMA per CTA takes bn / 2 cycles; four per k-block and 128-row half
   static const double eff1[4] = {0.45, 0.68, 0.76, 0.82}, eff2[4] = {0.55, 0.80, 0.88, 0.938};  // bn = 64, 128, 192, 256 (measured: 8192^3, and K = 512 ... 4096; 192 in between)
@@ -442,7 +453,7 @@ double estimate_dense_cycles(const gemm_desc_t& d, int sm_count, int variant, in
   // (fitted: against a second, partly filled wave of narrower tiles the one wave of wide tiles does about 8 % better than
   // this estimate says -- measured 2304^3 23.0 us against 27.0, 2560^3 27.6 / 30.5, 3072^3 42.2 / 42.8, 2816^3 37.9 / 36.9)
   const double fitted = (!wide && bn > 256) ? 0.92 : 1.0;
-  return (waves * per_tile + 3000.0) * fitted;  // + pipeline fill and drain
+  return (waves * per_tile + 3000.0 + handover) * fitted;  // + pipeline fill and drain
 }
 
 // Fill plan->dense and the launch geometry for a dense variant.
@@ -608,7 +619,7 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   info.grid = pl->grid;
   info.raster_group = raster;
   const int units_i = pl->sm_count / cg;
-  const int split = tail_split(num_tiles, units_i, p.num_kb, d, bn);
+  const int split = tail_split(num_tiles, units_i, p.num_kb, d, bn, cg, atoms);
   const long long rem = num_tiles % units_i;
   p.split = split;
   p.split_first_tile = static_cast<int>(split > 1 ? num_tiles - rem : num_tiles);

@@ -807,18 +807,19 @@ def test_tail_split_plans():
         i = bg.gemm_plan_info(h)
         bg.gemm_destroy(h)
         return i
-    i = info(1024, 1024, 2048, variant=V2, tile_n=256, tail_split=True)     # 16 pair tiles on 74 pairs: two slices each
+    i = info(1024, 1024, 2048, variant=V2, tile_n=256, tail_split=True)     # 16 pair tiles on 74 pairs: three slices each
     # (one 64-bit flag word per partial tile at the head of the workspace, padded to 256 bytes, then the partial tiles)
-    assert i["split"] == 2 and i["grid"] == 64 and i["workspace_bytes"] == 256 + 16 * 2 * 1 * 128 * 256 * 4
-    i = info(1024, 1024, 2048, variant=V2, tile_n=256)                      # not asked for: whole tiles, no workspace
+    assert i["split"] == 3 and i["grid"] == 96 and i["workspace_bytes"] == 512 + 16 * 2 * 2 * 128 * 256 * 4
+    i = info(1024, 1024, 1024, variant=V2, tile_n=256)                      # not asked for, and two slices at most: whole tiles, no workspace
     assert i["split"] == 1 and i["workspace_bytes"] == 0
+    assert info(1024, 1024, 1024, variant=V2, tile_n=256, tail_split=True)["split"] == 2
     assert info(1024, 1024, 256, variant=V2, tile_n=256, tail_split=True)["split"] == 1      # too little K to slice
     assert info(3072, 3072, 3072, variant=V2, tile_n=256, tail_split=True)["split"] == 1     # 144 tiles: the last wave is 70 of 74
     i = info(2560, 2560, 2560, variant=V2, tile_n=256, tail_split=True)                      # 100 tiles: 74 + 26, the 26 in two slices
     assert i["split"] == 2 and i["workspace_bytes"] == 512 + 26 * 2 * 1 * 128 * 256 * 4
     assert info(16384, 14336, 4096, variant=V2, tile_n=256, tail_split=True)["split"] == 1   # 48 full waves: not worth it
     i = info(512, 512, 16384, variant=V2, tile_n=256)                                      # 4 tiles, 256 ring stages each: by itself
-    assert i["split"] == 7 and i["grid"] == 56 and i["workspace_bytes"] == 512 + 4 * 2 * 6 * 128 * 256 * 4
+    assert i["split"] == 9 and i["grid"] == 72 and i["workspace_bytes"] == 512 + 4 * 2 * 8 * 128 * 256 * 4
 
 
 @pytest.mark.parametrize("cd,N", [(wl.BF16, 900), (wl.F16, 899), (wl.F32, 901), (wl.F32, 5), (wl.BF16, 3)])
