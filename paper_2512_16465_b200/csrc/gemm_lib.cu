@@ -392,8 +392,10 @@ int tail_split(long long tiles, int units, int num_kb, const gemm_desc_t& d, int
   split = std::min(split, num_kb / 4);  // a slice of fewer than four ring stages is all pipeline fill
   split = std::max(split, 1);
   // Without the flag only the extreme case splits by itself: a handful of tiles (no full wave) whose K is long enough for
-  // three or more slices each, where whole tiles would leave most of the GPU idle for the whole run.
-  if (!(d.flags & GEMM_FLAG_TAIL_SPLIT) && !(tiles < units && split >= 3)) return 1;
+  // three or more slices each, where whole tiles would leave most of the GPU idle for the whole run -- or for two slices
+  // when K has 48 or more 128-byte slices (measured with two slices allowed: 1024 x 1024 x 4096 20.6 -> 17.8 us,
+  // 2048 x 512 x 4096 20.8 -> 17.9, 1024 x 1024 x 8192 27.2 -> 25.5, but 1280 x 1280 x 2560 15.8 -> 18.5).
+  if (!(d.flags & GEMM_FLAG_TAIL_SPLIT) && !(tiles < units && (split >= 3 || (split == 2 && num_kb * atoms >= 48)))) return 1;
   return split;
 }
 
