@@ -223,7 +223,11 @@ size_t gemm_workspace_bytes(gemm_plan_t plan);
  * passes for this run's only if 48 of its bits equal that one value; a caller who wants certainty zeroes the workspace
  * once after allocating it).  Runs of one plan may overlap on the GPU (several streams, several host
  * threads) as long as runs that overlap use DIFFERENT workspaces; they share only the status word, which then reports
- * a timeout of any of them.  Runs that share a workspace must be ordered (one stream, or events).  alpha and beta are
+ * a timeout of any of them.  Runs that share a workspace must be ordered (one stream, or events).  One kind of plan
+ * wants the SMs it was planned for: a dense plan that cuts tiles along K (a dense variant with gemm_workspace_bytes > 0)
+ * has one CTA per tile wait, within the plan's time limit, for the other slices of that tile, which are CTAs of the same
+ * launch; if other work on the device keeps those from becoming resident the wait can run out (GEMM_ERR_TIMEOUT, never a
+ * hang).  Stream-K plans never wait for another CTA, inside clusters only at the hardware's cluster barrier.  alpha and beta are
  * host scalars.  The call only fetches or encodes tensor maps on the host (a plan remembers the maps of the operand
  * addresses it has seen, so a repeated address costs no encoding) and launches: once a plan has run once (which sets
  * kernel attributes), further runs may be recorded by stream capture into a CUDA graph (tested).  A captured run replays
