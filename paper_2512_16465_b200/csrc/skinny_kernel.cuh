@@ -711,21 +711,34 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constan
           emit16(c0, n, col0, accf, cin);
         } else if (early) {
           float sum[16], cin[16];
+          if (c0 == 0) {
 #pragma unroll
-          for (int j = 0; j < 16; ++j) sum[j] = 0.0f;
+            for (int j = 0; j < 16; ++j) cin[j] = __uint_as_float(ld_shared_b32(park + 128u * (64 + j)));
+          } else {
+            sk_load_cin16<kTall>(p, c0, n, n_ok, cin);
+          }
+          if (by_chunk) {
+            // two contributors, added in their order: ((0 + first) + second), as every other path adds them
+            const bool own_first = c_first == static_cast<int>(blockIdx.x);
 #pragma unroll
-          for (int j = 0; j < 16; ++j) cin[j] = __uint_as_float(ld_shared_b32(park + 128u * (64 + j)));
-          if (c0 != 0) sk_load_cin16<kTall>(p, c0, n, n_ok, cin);
+            for (int j = 0; j < 16; ++j) {
+              const float other_v = __uint_as_float(ld_shared_b32(park + 128u * (c0 + j)));
+              const float mine = __uint_as_float(acc[j]);
+              sum[j] = (0.0f + (own_first ? mine : other_v)) + (own_first ? other_v : mine);
+            }
+          } else {
 #pragma unroll
-          for (int b = 0; b < 4; ++b) {
-            // by contributor: b-th contributor; by chunk: the two contributors in order, the other one's chunk c0 / 16
-            const int cc = c_first + b;
-            if (cc <= c_last) {
-              const bool own = cc == static_cast<int>(blockIdx.x);
+            for (int j = 0; j < 16; ++j) sum[j] = 0.0f;
 #pragma unroll
-              for (int j = 0; j < 16; ++j) {
-                const float other_v = __uint_as_float(ld_shared_b32(park + 128u * ((by_chunk ? c0 : 16 * b) + j)));
-                sum[j] += own ? __uint_as_float(acc[j]) : other_v;
+            for (int b = 0; b < 4; ++b) {  // the b-th contributor's chunk 0
+              const int cc = c_first + b;
+              if (cc <= c_last) {
+                const bool own = cc == static_cast<int>(blockIdx.x);
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                  const float other_v = __uint_as_float(ld_shared_b32(park + 128u * (16 * b + j)));
+                  sum[j] += own ? __uint_as_float(acc[j]) : other_v;
+                }
               }
             }
           }
