@@ -821,14 +821,34 @@ __device__ __forceinline__ void epilogue_role(const DenseParams& p, const CUtens
       float v[32];
       if (p.out_dtype == 2) {
         tmem_ld_32x32(t_row + static_cast<uint32_t>(sl * 32), acc);
-        if (kSplit && slice == 0) {  // the partials are requested while the tensor-memory read is in flight
-          float4 pv[8];
-          load_partial(pv, reinterpret_cast<const float4*>(part0), q, sl, p.bn / 32, lane);
-          tmem_ld_wait();
-          add_partial(acc, pv);
-          for (int sidx = 1; sidx < p.split - 1; ++sidx) {  // further slices, in slice order
-            load_partial(pv, reinterpret_cast<const float4*>(part0 + sidx * partial_elems), q, sl, p.bn / 32, lane);
-            add_partial(acc, pv);
+        if (kSplit && slice == 0) {
+          // The partials are requested while the tensor-memory read is in flight, and two slices' loads are kept in
+          // flight: one after the other, every slice cost a round trip to L2 (about 0.5 us each on 256 x 256 x 32768
+          // with 16 slices).  Added in slice order all the same.
+          // (with two epilogue warpgroups the register limit is 168 and there is nothing to spare: one slice at a time)
+          const int n = p.split - 1;
+          const int groups = p.bn / 32;
+          float4 pa[8];
+          load_partial(pa, reinterpret_cast<const float4*>(part0), q, sl, groups, lane);
+          if constexpr (EPI_WG == 1) {
+            float4 pb[8];
+            if (n > 1) load_partial(pb, reinterpret_cast<const float4*>(part0 + partial_elems), q, sl, groups, lane);
+            tmem_ld_wait();
+            for (int sidx = 0; sidx < n; sidx += 2) {
+              add_partial(acc, pa);
+              if (sidx + 2 < n) load_partial(pa, reinterpret_cast<const float4*>(part0 + (sidx + 2) * partial_elems), q, sl, groups, lane);
+              if (sidx + 1 < n) {
+                add_partial(acc, pb);
+                if (sidx + 3 < n) load_partial(pb, reinterpret_cast<const float4*>(part0 + (sidx + 3) * partial_elems), q, sl, groups, lane);
+              }
+            }
+          } else {
+            tmem_ld_wait();
+            add_partial(acc, pa);
+            for (int sidx = 1; sidx < n; ++sidx) {  // further slices, in slice order
+              load_partial(pa, reinterpret_cast<const float4*>(part0 + sidx * partial_elems), q, sl, groups, lane);
+              add_partial(acc, pa);
+            }
           }
         } else {
           tmem_ld_wait();
@@ -845,17 +865,46 @@ __device__ __forceinline__ void epilogue_role(const DenseParams& p, const CUtens
         tmem_ld_32x32(t_row + static_cast<uint32_t>(sl * 64), acc);
         tmem_ld_32x32(t_row + static_cast<uint32_t>(sl * 64 + 32), acc1);
         if (kSplit && slice == 0) {
-          float4 pv[8], pv1[8];
-          load_partial(pv, reinterpret_cast<const float4*>(part0), q, 2 * sl, p.bn / 32, lane);
-          load_partial(pv1, reinterpret_cast<const float4*>(part0), q, 2 * sl + 1, p.bn / 32, lane);
-          tmem_ld_wait();
-          add_partial(acc, pv);
-          add_partial(acc1, pv1);
-          for (int sidx = 1; sidx < p.split - 1; ++sidx) {
-            load_partial(pv, reinterpret_cast<const float4*>(part0 + sidx * partial_elems), q, 2 * sl, p.bn / 32, lane);
-            load_partial(pv1, reinterpret_cast<const float4*>(part0 + sidx * partial_elems), q, 2 * sl + 1, p.bn / 32, lane);
+          const int n = p.split - 1;
+          const int groups = p.bn / 32;
+          if constexpr (EPI_WG == 1) {  // (registers to spare: two slices' loads in flight, as above)
+            float4 pa[8], pa1[8], pb[8], pb1[8];
+            load_partial(pa, reinterpret_cast<const float4*>(part0), q, 2 * sl, groups, lane);
+            load_partial(pa1, reinterpret_cast<const float4*>(part0), q, 2 * sl + 1, groups, lane);
+            if (n > 1) {
+              load_partial(pb, reinterpret_cast<const float4*>(part0 + partial_elems), q, 2 * sl, groups, lane);
+              load_partial(pb1, reinterpret_cast<const float4*>(part0 + partial_elems), q, 2 * sl + 1, groups, lane);
+            }
+            tmem_ld_wait();
+            for (int sidx = 0; sidx < n; sidx += 2) {
+              add_partial(acc, pa);
+              add_partial(acc1, pa1);
+              if (sidx + 2 < n) {
+                load_partial(pa, reinterpret_cast<const float4*>(part0 + (sidx + 2) * partial_elems), q, 2 * sl, groups, lane);
+                load_partial(pa1, reinterpret_cast<const float4*>(part0 + (sidx + 2) * partial_elems), q, 2 * sl + 1, groups, lane);
+              }
+              if (sidx + 1 < n) {
+                add_partial(acc, pb);
+                add_partial(acc1, pb1);
+                if (sidx + 3 < n) {
+                  load_partial(pb, reinterpret_cast<const float4*>(part0 + (sidx + 3) * partial_elems), q, 2 * sl, groups, lane);
+                  load_partial(pb1, reinterpret_cast<const float4*>(part0 + (sidx + 3) * partial_elems), q, 2 * sl + 1, groups, lane);
+                }
+              }
+            }
+          } else {
+            float4 pv[8], pv1[8];
+            load_partial(pv, reinterpret_cast<const float4*>(part0), q, 2 * sl, groups, lane);
+            load_partial(pv1, reinterpret_cast<const float4*>(part0), q, 2 * sl + 1, groups, lane);
+            tmem_ld_wait();
             add_partial(acc, pv);
             add_partial(acc1, pv1);
+            for (int sidx = 1; sidx < n; ++sidx) {
+              load_partial(pv, reinterpret_cast<const float4*>(part0 + sidx * partial_elems), q, 2 * sl, groups, lane);
+              load_partial(pv1, reinterpret_cast<const float4*>(part0 + sidx * partial_elems), q, 2 * sl + 1, groups, lane);
+              add_partial(acc, pv);
+              add_partial(acc1, pv1);
+            }
           }
         } else {
           tmem_ld_wait();
