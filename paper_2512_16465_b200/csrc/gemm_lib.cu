@@ -290,7 +290,8 @@ struct TileSchedule {
   int units = 0;        // CTAs (pairs) dealt to
   long long tiles = 0;  // real tiles
 };
-TileSchedule deal_tiles(const gemm_desc_t& d, int tile_m, int bn, int raster, int kstep, int num_kb, int max_units) {
+// `batches` > 1: the tiles of all matrices are dealt together (the list then holds tile ids of the whole batch).
+TileSchedule deal_tiles(const gemm_desc_t& d, int tile_m, int bn, int raster, int kstep, int num_kb, int max_units, int batches = 1) {
   const int d_tri = d_tri_of(d);
   const int a_tri = (d.flags & GEMM_FLAG_A_LOWER) ? 1 : ((d.flags & GEMM_FLAG_A_UPPER) ? 2 : 0);
   const int b_tri = (d.structure & GEMM_STRUCT_B_LOWER) ? 1 : ((d.structure & GEMM_STRUCT_B_UPPER) ? 2 : 0);
@@ -300,7 +301,8 @@ TileSchedule deal_tiles(const gemm_desc_t& d, int tile_m, int bn, int raster, in
     long long work;
   };
   std::vector<Item> order;
-  int t = 0;
+  for (int b = 0; b < batches; ++b) {
+  int t = b * tiles_m * tiles_n;
   for (int first = 0; first < tiles_m; first += raster) {
     const int gm = std::min(raster, tiles_m - first);
     for (int tn = 0; tn < tiles_n; ++tn)
@@ -319,6 +321,7 @@ TileSchedule deal_tiles(const gemm_desc_t& d, int tile_m, int bn, int raster, in
         const long long stages = std::max<long long>(1, hi - lo);
         order.push_back(Item{t, stages * (kstep / 64) * 2 * bn + 1000});
       }
+  }
   }
   TileSchedule sch;
   sch.tiles = static_cast<long long>(order.size());
@@ -581,14 +584,17 @@ gemm_status_t plan_dense(gemm_plan_s* pl, int cg, int forced_bn, int forced_rast
   pl->d_tri = d_tri;
   int dealt_units = 0;
   if (d_tri || p.a_tri || p.b_tri) {  // structured problem: tiles left out and / or unequal K ranges -> dealt ahead of time
-    const TileSchedule sch = deal_tiles(d, tile_m, bn, raster, kblk * atoms, p.num_kb, units);
-    if (static_cast<long long>(sch.slots.size()) * d.batch_count > 0x7FFFFFFFll) return GEMM_ERR_UNSUPPORTED;
+    // A batch is dealt as a whole (one list over all its matrices) unless that list would be very long; then the deal of
+    // one matrix is repeated for every matrix, which loads the CTAs less evenly: who gets the heavy tiles gets them every time.
+    const bool whole_batch = d.batch_count > 1 && static_cast<long long>(tiles_m) * tiles_n * d.batch_count <= (1ll << 22);
+    const TileSchedule sch = deal_tiles(d, tile_m, bn, raster, kblk * atoms, p.num_kb, units, whole_batch ? static_cast<int>(d.batch_count) : 1);
+    if (static_cast<long long>(sch.slots.size()) * (whole_batch ? 1 : d.batch_count) > 0x7FFFFFFFll) return GEMM_ERR_UNSUPPORTED;
     free(pl->h_tile_list);
     pl->h_tile_list = static_cast<int*>(malloc(sch.slots.size() * sizeof(int)));
     if (!pl->h_tile_list) return GEMM_ERR_CUDA;
     memcpy(pl->h_tile_list, sch.slots.data(), sch.slots.size() * sizeof(int));
     p.list_len = static_cast<int>(sch.slots.size());
-    p.num_tiles = p.list_len * d.batch_count;  // slots, the empty ones included
+    p.num_tiles = whole_batch ? p.list_len : p.list_len * static_cast<int>(d.batch_count);  // slots, the empty ones included
     dealt_units = sch.units;
   }
   if (!set_scheduler_divisors(p)) return GEMM_ERR_UNSUPPORTED;
