@@ -236,7 +236,10 @@ class DeviceCase:
         for _ in range(8):
             step()
         torch.cuda.synchronize()
-        short_region = (time.perf_counter() - t_warm) / 8 * steps < 0.03
+        step_sec = (time.perf_counter() - t_warm) / 8
+        # (short steps only: a step of several hundred microseconds has ramped the clocks up within the requested warm-up,
+        # and tens of further launches would only move it from the rested towards the power-capped state)
+        short_region = step_sec * steps < 0.03 and step_sec < 2.0e-4
         while short_region and time.perf_counter() - t_warm < 0.03:
             for _ in range(16):
                 step()
