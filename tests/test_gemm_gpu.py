@@ -323,6 +323,65 @@ def test_random_problems(seed):
     pytest.fail("twenty draws in a row refused as unsupported")
 
 
+@pytest.mark.parametrize("seed", range(int(os.environ.get("B200GEMM_RANDOM_STREAM_K_CASES", "24"))))
+def test_random_stream_k_problems_with_long_k(seed):
+    """Seeded stream-K problems with K long enough for every plan form -- equal ranges over all SMs, whole tiles, clusters,
+    three tiles per four CTAs (odd seeds draw 74 ... 100 tiles) -- skinny and tall, all element types, ragged extents,
+    run twice on a workspace that holds whatever earlier tests left in the allocator's memory.  (A sweep of this kind,
+    240 draws, found the one stale workspace word in 10^8 that passed for a run's own; B200GEMM_RANDOM_STREAM_K_CASES
+    makes it longer.)"""
+    rng = np.random.default_rng(77000 + seed)
+    pick = lambda xs: xs[int(rng.integers(len(xs)))]
+    ab = pick([wl.BF16, wl.BF16, wl.F16, wl.FP8_E4M3])
+    cd = pick([wl.F32, wl.BF16, wl.F16])
+    short = int(rng.integers(1, 65))
+    long_ = int(rng.integers(9400, 12900)) if seed % 2 else int(rng.integers(2000, 30000))
+    M, N = (long_, short) if rng.integers(3) == 0 else (short, long_)
+    ea, ec = (16 if ab == wl.FP8_E4M3 else 8), (4 if cd == wl.F32 else 8)
+    up = lambda x, m: -(-x // m) * m
+    K = up(int(rng.integers(512, 1200)) * 8, ea)
+    kw = dict(ta=0, tb=1, ab=ab, cd=cd, lda=K + ea * int(rng.integers(0, 2)), ldb=K, ldc=up(N, ec) + ec * int(rng.integers(0, 3)),
+              alpha=pick([1.0, 0.5, -1.0]), beta=pick([0.0, 1.0, -1.0]), epi=int(rng.integers(0, 4)))
+    if (kw["epi"] & 1) and rng.integers(3) == 0:
+        kw["bias_per_row"] = True
+    w = int_workload(f"random_stream_k_{seed}", M, N, K, sample_rows=48, sample_cols=48, **kw)
+    H.check_workload(w, bg.make_flags(VS, no_early_launch=bool(rng.integers(4) == 0)), exact=True, repeats=2,
+                     options=bg.OPT_STREAMK_WORKSPACE if seed % 3 == 0 else 0)
+
+
+@pytest.mark.parametrize("seed", range(int(os.environ.get("B200GEMM_RANDOM_SPLIT_CASES", "24"))))
+def test_random_dense_problems_with_few_tiles(seed):
+    """Seeded dense problems of the kinds whose plans cut tiles along K or use the widest tiles: a few tiles with a long K,
+    a little more than one wave, cubes of 2-3 K; automatic and forced variants, every storage order, run twice."""
+    rng = np.random.default_rng(88000 + seed)
+    pick = lambda xs: xs[int(rng.integers(len(xs)))]
+    variant = pick([0, 0, V1, V2, V2])
+    ab = pick([wl.BF16, wl.BF16, wl.F16, wl.FP8_E4M3])
+    cd = pick([wl.F32, wl.BF16, wl.F16])
+    fp8 = ab == wl.FP8_E4M3
+    if seed % 3 == 0:
+        M, N, K = int(rng.integers(65, 1100)), int(rng.integers(65, 1100)), int(rng.integers(2048, 40000))
+    elif seed % 3 == 1:
+        M, N, K = int(rng.integers(1500, 4300)), int(rng.integers(1500, 4300)), int(rng.integers(256, 3000))
+    else:
+        M = N = int(rng.integers(2000, 3300))
+        K = int(rng.integers(512, 3000))
+    ta, tb = (0, 1) if fp8 else (int(rng.integers(2)), int(rng.integers(2)))
+    ea, ec = (16 if fp8 else 8), (4 if cd == wl.F32 else 8)
+    up = lambda x, m: -(-x // m) * m
+    kw = dict(ta=ta, tb=tb, ab=ab, cd=cd, lda=up(M if ta else K, ea), ldb=up(K if tb else N, ea) + ea * int(rng.integers(0, 2)),
+              ldc=up(N, ec) + ec * int(rng.integers(0, 3)), alpha=pick([1.0, 0.5, -1.0]), beta=pick([0.0, 1.0, -1.0]), epi=int(rng.integers(0, 4)))
+    fl = dict(variant=variant, no_early_launch=bool(rng.integers(4) == 0))
+    if variant in (V1, V2):
+        fl["tail_split"] = bool(rng.integers(2))
+        fl["tile_n"] = pick([0, 0, 64, 128, 256] if not (variant == V2 and tb == 0) else [0, 128, 256])
+    w = int_workload(f"random_few_tiles_{seed}", M, N, K, sample_rows=48, sample_cols=48, **kw)
+    try:
+        H.check_workload(w, bg.make_flags(**fl), exact=True, repeats=2)
+    except bg.GemmError as e:
+        assert e.status == bg.ERR_UNSUPPORTED, (M, N, K, kw, fl)
+
+
 @pytest.mark.parametrize("seed", range(int(os.environ.get("B200GEMM_RANDOM_LARGE_CASES", "32"))))
 def test_random_large_problems(seed):
     """The same draw at sizes where every CTA computes many tiles (several waves, ring and accumulator buffers wrapping
